@@ -1,0 +1,250 @@
+/*
+ * alora.h — C ABI of the B200 (sm_100a) Activated-LoRA layer library.
+ *
+ * What the library computes, per decoder layer, for a ragged batch of NEW tokens that sit on top of
+ * per-request KV caches already filled by the base model:
+ *
+ *   1. gated fused q/k/v projection (Eq. 2 + Eq. 5 of the aLoRA paper):
+ *          y_t = W x_t + [p_t >= a_req] * s_k * B_k (A_k x_t)       per q / k / v block
+ *      p_t is the token's 0-based position in its sequence, a_req the request's activation offset
+ *      (the paper's t_invoke - 1), k the request's adapter (-1 = base model, no delta at all);
+ *   2. KV append: the new k/v rows go to their slots of a paged cache; bytes that belong to earlier
+ *      positions are never written (Prop. 2, proof step 4: only O(T_new) new cache entries);
+ *   3. causal grouped-query softmax attention of the new queries over cached ++ new rows
+ *      (Eq. 1, per-token form Eq. 3; a token attends keys 0..p_t, itself included).
+ *
+ * A decode step is the same with one new token per request (Prop. 1, second sentence); the
+ * full-LoRA entry is Eq. 4 (the delta on every token), i.e. what a conventional LoRA must do when
+ * it cannot reuse the base cache.
+ *
+ * Conventions
+ *   - Every pointer named d_* is DEVICE memory on the context's device; h_* is HOST memory.
+ *     All tensors are dense row-major, element type = the context's dtype (bf16 or fp32), index
+ *     arrays int32.  Buffers are caller-owned and only borrowed for the duration of the call
+ *     (of the enqueued work, for asynchronous calls) unless stated otherwise.
+ *   - Shapes: H hidden; Hq, Hkv heads; hd head_dim; Nq = Hq*hd; Nkv = Hkv*hd; N = Nq + 2*Nkv.
+ *     Fused rows are [ q heads | k heads | v heads ]; query head h reads KV head h / (Hq/Hkv).
+ *     Weights are output-major: W[N][H] (y = W x), A[r][H], B[out][r].
+ *   - Ragged batch: T new tokens of R requests, request r owns rows query_start_loc[r] ..
+ *     query_start_loc[r+1]-1, whose positions must be consecutive and end at seq_lens[r]-1.
+ *   - Paged cache of one layer: pool[num_pages][2][Hkv][page_size][hd] (K plane, then V plane).
+ *     Position p of request r lives in page block_tables[r][p / page_size], row p % page_size.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Work is enqueued and the
+ *     call returns; nothing synchronises unless stated.
+ *   - Every call returns an alora_status.  Host-side argument errors are detected before anything
+ *     is launched.  Device-side findings (page id out of range, inconsistent positions, a bounded
+ *     wait that ran out) are recorded in a status word readable with alora_get_status after the
+ *     stream has been synchronised; a kernel that finds one skips the offending access, it never
+ *     traps.  There is no CPU fallback: without a CUDA device every compute call fails.
+ */
+#ifndef ALORA_H
+#define ALORA_H
+
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct alora_ctx alora_ctx;
+
+typedef enum alora_status {
+    ALORA_OK = 0,
+    ALORA_ERR_INVALID_ARG = 1,   /* null pointer, negative size, misaligned pointer            */
+    ALORA_ERR_UNSUPPORTED = 2,   /* shape or dtype the kernels are not built for               */
+    ALORA_ERR_CAPACITY = 3,      /* T, R, rank or adapter id beyond what alora_create was told */
+    ALORA_ERR_NO_WEIGHTS = 4,    /* layer weights or a referenced adapter were never set       */
+    ALORA_ERR_CUDA = 5,          /* a CUDA runtime/driver call failed (see alora_last_cuda_error) */
+    ALORA_ERR_BAD_BATCH = 6,     /* batch metadata inconsistent (host validation or device check) */
+    ALORA_ERR_PAGE_RANGE = 7,    /* a block-table entry is outside [0, num_pages)              */
+    ALORA_ERR_TIMEOUT = 8,       /* a bounded in-kernel wait expired                            */
+    ALORA_ERR_NO_DEVICE = 9      /* no usable CUDA device                                       */
+} alora_status;
+
+typedef enum alora_dtype { ALORA_DTYPE_BF16 = 0, ALORA_DTYPE_FP32 = 1 } alora_dtype;
+
+/* Execution mode of a layer / stack call. */
+typedef enum alora_mode {
+    ALORA_MODE_ALORA = 0,      /* Eq. 5: delta on rows with p >= a_req                            */
+    ALORA_MODE_FULL_LORA = 1,  /* Eq. 4: delta on every row of a request that has an adapter      */
+    ALORA_MODE_BASE = 2        /* Eq. 2: adapters ignored                                         */
+} alora_mode;
+
+typedef struct alora_config {
+    int32_t hidden;        /* H                                                                   */
+    int32_t n_q_heads;     /* Hq                                                                  */
+    int32_t n_kv_heads;    /* Hkv, must divide Hq                                                 */
+    int32_t head_dim;      /* hd                                                                  */
+    int32_t page_size;     /* tokens per KV page                                                  */
+    int32_t n_layers;      /* layers addressable by the per-layer calls                           */
+    int32_t intermediate;  /* MLP width (0 if the stack entry is not used)                        */
+    int32_t max_adapters;  /* adapter ids are 0 .. max_adapters-1                                 */
+    int32_t max_rank;      /* largest adapter rank (<= 64)                                        */
+    int32_t dtype;         /* alora_dtype                                                         */
+    int32_t device;        /* CUDA device ordinal                                                 */
+    int32_t max_tokens;    /* largest T of any call; sizes the context's workspaces               */
+    int32_t max_requests;  /* largest R of any call                                               */
+    float rms_eps;         /* RMSNorm epsilon (stack entry)                                       */
+    float rope_theta;      /* must be 0: the method's equations carry no positional rotation      */
+    float softmax_scale;   /* 0 => 1/sqrt(head_dim) (Eq. 1)                                       */
+} alora_config;
+
+/*
+ * Create a context on cfg->device.  Allocates the context-owned workspaces (per-token metadata,
+ * tile and work lists, the rank-r intermediate t = A x, a [max_tokens][N] q/k/v staging buffer,
+ * split-KV partial results, the status word) with cudaMalloc.  *out is set only on success.
+ * alora_destroy frees everything the context owns; it does not touch caller buffers.
+ */
+alora_status alora_create(const alora_config *cfg, alora_ctx **out);
+alora_status alora_destroy(alora_ctx *ctx);
+
+/*
+ * Base weights of one layer (Eq. 2).  d_wqkv[N][H] is required; d_wo[H][Nq], d_wgate_up[2*I][H]
+ * (gate rows first, then up rows), d_wdown[H][I], d_norm_attn[H], d_norm_mlp[H] may be NULL when
+ * only the attention-block entries are used.  Pointers are BORROWED: the caller keeps the memory
+ * alive and unchanged while the context uses it.
+ */
+alora_status alora_set_layer_weights(alora_ctx *ctx, int layer, const void *d_wqkv, const void *d_wo,
+                                     const void *d_wgate_up, const void *d_wdown,
+                                     const void *d_norm_attn, const void *d_norm_mlp);
+
+/*
+ * Register (or replace) adapter `adapter_id` of `layer`: Delta_blk = scale * B_blk A_blk for
+ * blk in {q, k, v} (Eq. 4 / Eq. 5).  d_Aq/d_Ak/d_Av are [rank][H], d_Bq is [Nq][rank], d_Bk and
+ * d_Bv are [Nkv][rank].  The matrices are COPIED into context-owned, rank-padded storage on the
+ * given stream; the caller's buffers may be released once that stream has passed this point.
+ * 1 <= rank <= max_rank.
+ */
+alora_status alora_register_adapter(alora_ctx *ctx, int adapter_id, int layer, int rank, float scale,
+                                    const void *d_Aq, const void *d_Bq, const void *d_Ak,
+                                    const void *d_Bk, const void *d_Av, const void *d_Bv,
+                                    void *stream);
+
+/*
+ * Host-side consistency check of batch metadata (all pointers HOST memory; launches nothing, needs
+ * no device).  Verifies: query_start_loc non-decreasing from 0 to T; positions of each request
+ * consecutive and ending at seq_lens[r]-1; adapter ids in [-1, max_adapters); activation offsets
+ * >= 0; every block-table entry a request can touch inside [0, num_pages); no physical page used
+ * by the writable range of two requests.  Returns ALORA_OK, ALORA_ERR_BAD_BATCH,
+ * ALORA_ERR_PAGE_RANGE or ALORA_ERR_CAPACITY.  `cfg` supplies page_size, max_* limits.
+ */
+alora_status alora_validate_batch(const alora_config *cfg, const int32_t *h_positions,
+                                  const int32_t *h_activation_offsets, const int32_t *h_adapter_ids,
+                                  const int32_t *h_query_start_loc, const int32_t *h_seq_lens,
+                                  const int32_t *h_block_tables, int max_blocks, int num_pages,
+                                  int T, int R);
+
+/*
+ * Batch metadata step, exposed for exact comparison.  Fills (each output may be NULL):
+ *   d_token_request[T]  request index of every token,
+ *   d_row_adapter[T]    adapter id applied to the row: adapter_ids[r] if the gate of Eq. 5 is open
+ *                       (mode ALORA: p >= a_req; FULL_LORA: always), else -1,
+ *   d_slot_mapping[T]   token slot = page * page_size + p % page_size of the row's position.
+ * The same kernels run inside every layer call.
+ */
+alora_status alora_batch_metadata(alora_ctx *ctx, int mode, const int32_t *d_positions,
+                                  const int32_t *d_activation_offsets, const int32_t *d_adapter_ids,
+                                  const int32_t *d_query_start_loc, const int32_t *d_seq_lens,
+                                  const int32_t *d_block_tables, int max_blocks, int num_pages,
+                                  int T, int R, int32_t *d_token_request, int32_t *d_row_adapter,
+                                  int32_t *d_slot_mapping, void *stream);
+
+/*
+ * Step 1 alone: d_qkv[T][N] = gated fused projection of d_hidden[T][H] with layer `layer`'s
+ * weights (Eq. 5; Eq. 4 for mode FULL_LORA; Eq. 2 for mode BASE or adapter id -1).  Rows whose
+ * gate is closed go through exactly the arithmetic of a base-only call, so they are bit-identical
+ * to it (Prop. 1).
+ */
+alora_status alora_project_qkv(alora_ctx *ctx, int layer, int mode, const void *d_hidden,
+                               const int32_t *d_positions, const int32_t *d_activation_offsets,
+                               const int32_t *d_adapter_ids, const int32_t *d_query_start_loc,
+                               const int32_t *d_seq_lens, int T, int R, void *d_qkv, void *stream);
+
+/*
+ * Step 2 alone: copy the k and v parts of d_qkv[T][N] into d_paged_kv at each token's slot.
+ * Writes exactly T*2*Nkv elements; no other byte of the pool changes.
+ */
+alora_status alora_kv_append(alora_ctx *ctx, const void *d_qkv, const int32_t *d_positions,
+                             const int32_t *d_query_start_loc, const int32_t *d_seq_lens,
+                             const int32_t *d_block_tables, int max_blocks, int num_pages, int T,
+                             int R, void *d_paged_kv, void *stream);
+
+/*
+ * Step 3 alone: d_attn_out[T][Nq] = causal GQA attention of the q part of d_qkv[T][N] over
+ * positions 0 .. p_t of each request, read from d_paged_kv through d_block_tables (the new rows
+ * must already be appended).
+ */
+alora_status alora_attend(alora_ctx *ctx, const void *d_qkv, const int32_t *d_positions,
+                          const int32_t *d_query_start_loc, const int32_t *d_seq_lens,
+                          const void *d_paged_kv, const int32_t *d_block_tables, int max_blocks,
+                          int num_pages, int T, int R, void *d_attn_out, void *stream);
+
+/*
+ * The activated prefill of a suffix on a reused base cache: steps 1-3 for one layer (Eq. 5, then
+ * Prop. 2's proof steps 1-4).  d_paged_kv must already hold positions 0 .. p_first-1 of every
+ * request; it is written only at the slots of the T new positions.  The q/k/v rows are staged in
+ * a context-owned buffer.
+ */
+alora_status alora_prefill_layer(alora_ctx *ctx, int layer, const void *d_hidden,
+                                 const int32_t *d_positions, const int32_t *d_activation_offsets,
+                                 const int32_t *d_adapter_ids, const int32_t *d_query_start_loc,
+                                 const int32_t *d_seq_lens, void *d_paged_kv,
+                                 const int32_t *d_block_tables, int max_blocks, int num_pages, int T,
+                                 int R, void *d_attn_out, void *stream);
+
+/*
+ * One decode step (Prop. 1, second sentence; Eq. 3): exactly one new token per request (T == R,
+ * query_start_loc[r] == r), mixed base / adapter requests.  Same results as alora_prefill_layer on
+ * the same arguments, computed by kernels specialised for one query row per request.
+ */
+alora_status alora_decode_step(alora_ctx *ctx, int layer, const void *d_hidden,
+                               const int32_t *d_positions, const int32_t *d_activation_offsets,
+                               const int32_t *d_adapter_ids, const int32_t *d_seq_lens,
+                               void *d_paged_kv, const int32_t *d_block_tables, int max_blocks,
+                               int num_pages, int R, void *d_attn_out, void *stream);
+
+/*
+ * The comparison path (Eq. 4): a conventional LoRA cannot reuse the base cache, so the caller
+ * passes ALL prefix + suffix tokens as new tokens (positions from 0) with private pages, and the
+ * delta is applied to every row of a request that has an adapter.  With adapter_ids = -1 this is
+ * the base model's prefill, which is how a reusable base cache is produced.
+ */
+alora_status alora_full_lora_prefill_layer(alora_ctx *ctx, int layer, const void *d_hidden,
+                                           const int32_t *d_positions, const int32_t *d_adapter_ids,
+                                           const int32_t *d_query_start_loc, const int32_t *d_seq_lens,
+                                           void *d_paged_kv, const int32_t *d_block_tables,
+                                           int max_blocks, int num_pages, int T, int R,
+                                           void *d_attn_out, void *stream);
+
+/*
+ * All n_layers decoder layers (pre-norm residual: h += o_proj(attn(norm(h))); h += down(silu(gate)
+ * * up) of norm(h)), adapters on q/k/v only, MLP and o_proj with base weights.  d_paged_kv_layers
+ * is a HOST array of n_layers device pointers (one pool per layer, same block tables).
+ * d_hidden_in[T][H] -> d_hidden_out[T][H] (may alias).  `mode` selects Eq. 5 / Eq. 4 / Eq. 2.
+ */
+alora_status alora_forward_stack(alora_ctx *ctx, int mode, const void *d_hidden_in,
+                                 const int32_t *d_positions, const int32_t *d_activation_offsets,
+                                 const int32_t *d_adapter_ids, const int32_t *d_query_start_loc,
+                                 const int32_t *d_seq_lens, void *const *h_paged_kv_layers,
+                                 const int32_t *d_block_tables, int max_blocks, int num_pages, int T,
+                                 int R, void *d_hidden_out, void *stream);
+
+/*
+ * Read and clear the device status word.  Synchronises `stream` first.  *device_status receives
+ * ALORA_OK or the first device-side finding since the last call.
+ */
+alora_status alora_get_status(alora_ctx *ctx, void *stream, int32_t *device_status);
+
+/* Static description of a status code; never NULL. */
+const char *alora_status_string(int status);
+
+/* Text of the last CUDA error seen by this context ("" if none); valid until the next call. */
+const char *alora_last_cuda_error(const alora_ctx *ctx);
+
+/* Number of kernels this context has launched so far (all entry points). */
+int64_t alora_launch_count(const alora_ctx *ctx);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* ALORA_H */

@@ -1,0 +1,457 @@
+// C ABI of the library: context management, argument checks, and the order in which the kernels
+// of one layer are enqueued.  No arithmetic of the method lives here.
+#include <algorithm>
+#include <cstring>
+#include <new>
+
+#include "alora_internal.h"
+
+namespace alora {
+
+alora_status cuda_fail(alora_ctx *ctx, cudaError_t e, const char *what) {
+    if (ctx) ctx->cuda_err = std::string(what) + ": " + cudaGetErrorString(e);
+    return ALORA_ERR_CUDA;
+}
+
+int launch_project_simt(alora_ctx *, int, const void *, int, void *, cudaStream_t);
+int launch_linear_simt(alora_ctx *, const void *, const void *, int, int, int, void *, const void *, cudaStream_t);
+int launch_attend_simt(alora_ctx *, const void *, const BatchArgs &, const void *, void *, cudaStream_t);
+
+int launch_project(alora_ctx *ctx, int layer, const void *hidden, int T, void *qkv, cudaStream_t s) {
+    return launch_project_simt(ctx, layer, hidden, T, qkv, s);
+}
+int launch_linear(alora_ctx *ctx, const void *x, const void *W, int T, int K, int N, void *y,
+                  const void *residual, cudaStream_t s) {
+    return launch_linear_simt(ctx, x, W, T, K, N, y, residual, s);
+}
+int launch_attend(alora_ctx *ctx, const void *qkv, const BatchArgs &b, const void *pool, void *out,
+                  cudaStream_t s) {
+    return launch_attend_simt(ctx, qkv, b, pool, out, s);
+}
+
+static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
+
+static alora_status check_batch_args(alora_ctx *ctx, int T, int R) {
+    if (!ctx) return ALORA_ERR_INVALID_ARG;
+    if (T < 0 || R < 0) return ALORA_ERR_INVALID_ARG;
+    if (T > ctx->cfg.max_tokens || R > ctx->cfg.max_requests) return ALORA_ERR_CAPACITY;
+    return ALORA_OK;
+}
+
+static alora_status finish(alora_ctx *ctx, int launched) {
+    if (launched < 0) return ALORA_ERR_UNSUPPORTED;
+    ctx->launches += launched;
+    cudaError_t e = cudaGetLastError();
+    if (e != cudaSuccess) return cuda_fail(ctx, e, "kernel launch");
+    return ALORA_OK;
+}
+
+// Steps 1-3 of one layer, in the order of Prop. 2's proof.
+static alora_status run_layer(alora_ctx *ctx, int layer, const void *hidden, const BatchArgs &b, void *pool,
+                              void *attn_out, cudaStream_t s) {
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return ALORA_ERR_INVALID_ARG;
+    if (!ctx->layers[layer].wqkv) return ALORA_ERR_NO_WEIGHTS;
+    int n = 0, k;
+    if ((k = launch_metadata(ctx, b, s)) < 0) return ALORA_ERR_UNSUPPORTED; n += k;
+    if ((k = launch_project(ctx, layer, hidden, b.T, ctx->d_qkv, s)) < 0) return ALORA_ERR_UNSUPPORTED; n += k;
+    if ((k = launch_kv_append(ctx, ctx->d_qkv, b.T, b.num_pages, pool, s)) < 0) return ALORA_ERR_UNSUPPORTED; n += k;
+    if ((k = launch_attend(ctx, ctx->d_qkv, b, pool, attn_out, s)) < 0) return ALORA_ERR_UNSUPPORTED; n += k;
+    return finish(ctx, n);
+}
+
+}  // namespace alora
+
+using namespace alora;
+
+extern "C" {
+
+const char *alora_status_string(int status) {
+    switch (status) {
+        case ALORA_OK: return "ok";
+        case ALORA_ERR_INVALID_ARG: return "invalid argument";
+        case ALORA_ERR_UNSUPPORTED: return "unsupported shape or data type";
+        case ALORA_ERR_CAPACITY: return "exceeds the capacity given to alora_create";
+        case ALORA_ERR_NO_WEIGHTS: return "layer weights or adapter not set";
+        case ALORA_ERR_CUDA: return "CUDA call failed";
+        case ALORA_ERR_BAD_BATCH: return "inconsistent batch metadata";
+        case ALORA_ERR_PAGE_RANGE: return "block-table entry outside the page pool";
+        case ALORA_ERR_TIMEOUT: return "bounded in-kernel wait expired";
+        case ALORA_ERR_NO_DEVICE: return "no usable CUDA device";
+        default: return "unknown status";
+    }
+}
+
+const char *alora_last_cuda_error(const alora_ctx *ctx) { return ctx ? ctx->cuda_err.c_str() : ""; }
+int64_t alora_launch_count(const alora_ctx *ctx) { return ctx ? ctx->launches : 0; }
+
+alora_status alora_create(const alora_config *cfg, alora_ctx **out) {
+    if (!cfg || !out) return ALORA_ERR_INVALID_ARG;
+    const alora_config &c = *cfg;
+    if (c.hidden <= 0 || c.n_q_heads <= 0 || c.n_kv_heads <= 0 || c.head_dim <= 0 || c.page_size <= 0 ||
+        c.n_layers <= 0 || c.max_adapters < 0 || c.max_rank < 0 || c.max_tokens <= 0 || c.max_requests <= 0 ||
+        c.intermediate < 0)
+        return ALORA_ERR_INVALID_ARG;
+    if (c.n_q_heads % c.n_kv_heads != 0) return ALORA_ERR_INVALID_ARG;
+    if (c.dtype != ALORA_DTYPE_BF16 && c.dtype != ALORA_DTYPE_FP32) return ALORA_ERR_UNSUPPORTED;
+    if (c.rope_theta != 0.f) return ALORA_ERR_UNSUPPORTED;
+    if (c.max_rank > kRankPadMax) return ALORA_ERR_UNSUPPORTED;
+    if (c.head_dim != 32 && c.head_dim != 64 && c.head_dim != 128) return ALORA_ERR_UNSUPPORTED;
+    if (c.n_q_heads / c.n_kv_heads > 8) return ALORA_ERR_UNSUPPORTED;
+    const size_t es = c.dtype == ALORA_DTYPE_FP32 ? 4 : 2;
+    if ((c.head_dim * es) % 16 != 0 || (c.hidden * es) % 16 != 0) return ALORA_ERR_UNSUPPORTED;
+
+    int ndev = 0;
+    if (cudaGetDeviceCount(&ndev) != cudaSuccess || ndev <= 0 || c.device < 0 || c.device >= ndev) {
+        cudaGetLastError();
+        return ALORA_ERR_NO_DEVICE;
+    }
+    alora_ctx *ctx = new (std::nothrow) alora_ctx();
+    if (!ctx) return ALORA_ERR_INVALID_ARG;
+    ctx->cfg = c;
+    ctx->esize = es;
+    Dims &d = ctx->d;
+    d.H = c.hidden; d.Hq = c.n_q_heads; d.Hkv = c.n_kv_heads; d.hd = c.head_dim; d.G = d.Hq / d.Hkv;
+    d.Nq = d.Hq * d.hd; d.Nkv = d.Hkv * d.hd; d.N = d.Nq + 2 * d.Nkv; d.page = c.page_size; d.I = c.intermediate;
+    d.RP = std::max(16, (c.max_rank + 15) / 16 * 16);
+    d.softmax_scale = c.softmax_scale != 0.f ? c.softmax_scale : 1.0f / sqrtf((float)d.hd);
+    ctx->layers.resize(c.n_layers);
+    const size_t n_ad = (size_t)c.n_layers * std::max(1, c.max_adapters);
+    ctx->h_adapters.assign(n_ad, AdapterDev{nullptr, nullptr, 0, 0, 0.f, 0});
+    ctx->adapter_storage.assign(2 * n_ad, nullptr);
+
+    alora_status st = ALORA_OK;
+    auto alloc = [&](void **p, size_t bytes) {
+        if (st != ALORA_OK) return;
+        cudaError_t e = cudaMalloc(p, std::max<size_t>(bytes, 16));
+        if (e != cudaSuccess) st = cuda_fail(ctx, e, "cudaMalloc");
+    };
+    cudaError_t e = cudaSetDevice(c.device);
+    if (e != cudaSuccess) { delete ctx; return ALORA_ERR_NO_DEVICE; }
+    cudaDeviceProp prop;
+    if (cudaGetDeviceProperties(&prop, c.device) == cudaSuccess) ctx->sm_count = prop.multiProcessorCount;
+    const size_t Tm = (size_t)c.max_tokens;
+    ctx->max_tiles = (int)(Tm / 128 + 2 * (size_t)c.max_requests + 2);
+    alloc((void **)&ctx->d_adapters, n_ad * sizeof(AdapterDev));
+    alloc((void **)&ctx->d_token_req, Tm * 4);
+    alloc((void **)&ctx->d_row_adapter, Tm * 4);
+    alloc((void **)&ctx->d_slot, Tm * 4);
+    alloc((void **)&ctx->d_tiles, (size_t)ctx->max_tiles * sizeof(ProjTile));
+    alloc((void **)&ctx->d_counts, 16 * 4);
+    alloc((void **)&ctx->d_seg_scratch, (size_t)4 * (2 * (size_t)c.max_requests + 1) * 4);
+    alloc(&ctx->d_t, Tm * 3 * d.RP * 4);
+    alloc(&ctx->d_qkv, Tm * d.N * es);
+    alloc((void **)&ctx->d_status, 4);
+    if (d.I > 0) {
+        const size_t chunk = std::min<size_t>(Tm, kMlpChunk);
+        alloc(&ctx->d_act[0], Tm * std::max(d.H, d.Nq) * es);  // normed input / attention output
+        alloc(&ctx->d_act[1], Tm * std::max(d.H, d.Nq) * es);
+        alloc(&ctx->d_act[2], chunk * 2 * d.I * es);            // gate_up of one token chunk
+        alloc(&ctx->d_act[3], chunk * d.I * es);                // swiglu output of one token chunk
+    }
+    if (st == ALORA_OK) {
+        e = cudaMallocHost((void **)&ctx->h_status, 4);
+        if (e != cudaSuccess) st = cuda_fail(ctx, e, "cudaMallocHost");
+    }
+    if (st == ALORA_OK) {
+        e = cudaMemset(ctx->d_status, 0, 4);
+        if (e == cudaSuccess) e = cudaMemset(ctx->d_adapters, 0, n_ad * sizeof(AdapterDev));
+        if (e == cudaSuccess) e = cudaMemset(ctx->d_counts, 0, 64);
+        if (e != cudaSuccess) st = cuda_fail(ctx, e, "cudaMemset");
+    }
+    if (st != ALORA_OK) { alora_destroy(ctx); return st; }
+    *out = ctx;
+    return ALORA_OK;
+}
+
+alora_status alora_destroy(alora_ctx *ctx) {
+    if (!ctx) return ALORA_ERR_INVALID_ARG;
+    cudaSetDevice(ctx->cfg.device);
+    for (void *p : ctx->adapter_storage) if (p) cudaFree(p);
+    void *ptrs[] = {ctx->d_adapters, ctx->d_token_req, ctx->d_row_adapter, ctx->d_slot, ctx->d_tiles, ctx->d_counts,
+                    ctx->d_seg_scratch, ctx->d_t, ctx->d_qkv, ctx->d_status, ctx->d_act[0], ctx->d_act[1],
+                    ctx->d_act[2], ctx->d_act[3], ctx->d_iota};
+    for (void *p : ptrs) if (p) cudaFree(p);
+    if (ctx->h_status) cudaFreeHost(ctx->h_status);
+    delete ctx;
+    return ALORA_OK;
+}
+
+alora_status alora_set_layer_weights(alora_ctx *ctx, int layer, const void *d_wqkv, const void *d_wo,
+                                     const void *d_wgate_up, const void *d_wdown, const void *d_norm_attn,
+                                     const void *d_norm_mlp) {
+    if (!ctx || layer < 0 || layer >= ctx->cfg.n_layers || !d_wqkv) return ALORA_ERR_INVALID_ARG;
+    const void *all[] = {d_wqkv, d_wo, d_wgate_up, d_wdown, d_norm_attn, d_norm_mlp};
+    for (const void *p : all) if (p && !aligned16(p)) return ALORA_ERR_INVALID_ARG;
+    LayerWeights &lw = ctx->layers[layer];
+    lw.wqkv = d_wqkv; lw.wo = d_wo; lw.wgate_up = d_wgate_up; lw.wdown = d_wdown;
+    lw.norm_attn = d_norm_attn; lw.norm_mlp = d_norm_mlp;
+    return ALORA_OK;
+}
+
+alora_status alora_register_adapter(alora_ctx *ctx, int adapter_id, int layer, int rank, float scale,
+                                    const void *d_Aq, const void *d_Bq, const void *d_Ak, const void *d_Bk,
+                                    const void *d_Av, const void *d_Bv, void *stream) {
+    if (!ctx || !d_Aq || !d_Bq || !d_Ak || !d_Bk || !d_Av || !d_Bv) return ALORA_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return ALORA_ERR_INVALID_ARG;
+    if (adapter_id < 0 || adapter_id >= ctx->cfg.max_adapters) return ALORA_ERR_CAPACITY;
+    if (rank < 1 || rank > ctx->cfg.max_rank) return ALORA_ERR_CAPACITY;
+    cudaStream_t s = (cudaStream_t)stream;
+    ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    const Dims &d = ctx->d;
+    const size_t idx = (size_t)layer * ctx->cfg.max_adapters + adapter_id;
+    const size_t bytesA = (size_t)3 * d.RP * d.H * ctx->esize, bytesB = (size_t)d.N * d.RP * ctx->esize;
+    if (!ctx->adapter_storage[2 * idx]) {
+        ALORA_CUDA(ctx, cudaMalloc(&ctx->adapter_storage[2 * idx], bytesA));
+        ALORA_CUDA(ctx, cudaMalloc(&ctx->adapter_storage[2 * idx + 1], bytesB));
+    }
+    void *A = ctx->adapter_storage[2 * idx], *B = ctx->adapter_storage[2 * idx + 1];
+    int n = launch_repack_adapter(ctx, rank, d_Aq, d_Bq, d_Ak, d_Bk, d_Av, d_Bv, A, B, s);
+    AdapterDev rec{A, B, rank, (rank + 15) / 16 * 16, scale, 0};
+    ctx->h_adapters[idx] = rec;
+    // the table entry is a kernel argument of later launches on this stream: order the update after
+    // earlier work by copying on the same stream (source is context-owned host memory).
+    ALORA_CUDA(ctx, cudaMemcpyAsync(ctx->d_adapters + idx, &ctx->h_adapters[idx], sizeof(AdapterDev),
+                                    cudaMemcpyHostToDevice, s));
+    return finish(ctx, n);
+}
+
+alora_status alora_validate_batch(const alora_config *cfg, const int32_t *pos, const int32_t *a_req,
+                                  const int32_t *ids, const int32_t *qsl, const int32_t *seq_lens,
+                                  const int32_t *bt, int max_blocks, int num_pages, int T, int R) {
+    if (!cfg || !pos || !qsl || !seq_lens || T < 0 || R < 0) return ALORA_ERR_INVALID_ARG;
+    if (T > cfg->max_tokens || R > cfg->max_requests) return ALORA_ERR_CAPACITY;
+    if (qsl[0] != 0 || qsl[R] != T) return ALORA_ERR_BAD_BATCH;
+    const int ps = cfg->page_size;
+    std::vector<uint8_t> owned;  // pages that some request may write
+    if (bt) owned.assign((size_t)std::max(num_pages, 0), 0);
+    for (int r = 0; r < R; ++r) {
+        const int n_new = qsl[r + 1] - qsl[r];
+        if (n_new < 0) return ALORA_ERR_BAD_BATCH;
+        if (seq_lens[r] < n_new) return ALORA_ERR_BAD_BATCH;
+        const int p_first = seq_lens[r] - n_new;
+        for (int i = 0; i < n_new; ++i)
+            if (pos[qsl[r] + i] != p_first + i) return ALORA_ERR_BAD_BATCH;
+        if (ids) {
+            if (ids[r] < -1 || ids[r] >= cfg->max_adapters) return ALORA_ERR_BAD_BATCH;
+            if (ids[r] >= 0 && (!a_req || a_req[r] < 0)) return ALORA_ERR_BAD_BATCH;
+        }
+        if (bt) {
+            const int nblk = (seq_lens[r] + ps - 1) / ps;
+            if (nblk > max_blocks) return ALORA_ERR_BAD_BATCH;
+            for (int b = 0; b < nblk; ++b) {
+                const int page = bt[(size_t)r * max_blocks + b];
+                if (page < 0 || page >= num_pages) return ALORA_ERR_PAGE_RANGE;
+            }
+            // pages that hold new positions are written: they must not be written by anyone else
+            if (n_new > 0)
+                for (int b = p_first / ps; b < nblk; ++b) {
+                    const int page = bt[(size_t)r * max_blocks + b];
+                    if (owned[page]) return ALORA_ERR_BAD_BATCH;
+                    owned[page] = 1;
+                }
+        }
+    }
+    return ALORA_OK;
+}
+
+#define ALORA_BATCH(mode_)                                                                               \
+    BatchArgs b{d_positions, d_activation_offsets, d_adapter_ids, d_query_start_loc, d_seq_lens,         \
+                d_block_tables, max_blocks, num_pages, T, R, (mode_)}
+
+alora_status alora_batch_metadata(alora_ctx *ctx, int mode, const int32_t *d_positions,
+                                  const int32_t *d_activation_offsets, const int32_t *d_adapter_ids,
+                                  const int32_t *d_query_start_loc, const int32_t *d_seq_lens,
+                                  const int32_t *d_block_tables, int max_blocks, int num_pages, int T, int R,
+                                  int32_t *d_token_request, int32_t *d_row_adapter, int32_t *d_slot_mapping,
+                                  void *stream) {
+    alora_status st = check_batch_args(ctx, T, R);
+    if (st != ALORA_OK) return st;
+    if (!d_positions || !d_query_start_loc || !d_seq_lens) return ALORA_ERR_INVALID_ARG;
+    if (mode < ALORA_MODE_ALORA || mode > ALORA_MODE_BASE) return ALORA_ERR_INVALID_ARG;
+    if (mode == ALORA_MODE_ALORA && d_adapter_ids && !d_activation_offsets) return ALORA_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    ALORA_BATCH(mode);
+    int n = launch_metadata(ctx, b, s);
+    if (T > 0) {
+        if (d_token_request) ALORA_CUDA(ctx, cudaMemcpyAsync(d_token_request, ctx->d_token_req, (size_t)T * 4, cudaMemcpyDeviceToDevice, s));
+        if (d_row_adapter) ALORA_CUDA(ctx, cudaMemcpyAsync(d_row_adapter, ctx->d_row_adapter, (size_t)T * 4, cudaMemcpyDeviceToDevice, s));
+        if (d_slot_mapping) ALORA_CUDA(ctx, cudaMemcpyAsync(d_slot_mapping, ctx->d_slot, (size_t)T * 4, cudaMemcpyDeviceToDevice, s));
+    }
+    return finish(ctx, n);
+}
+
+alora_status alora_project_qkv(alora_ctx *ctx, int layer, int mode, const void *d_hidden,
+                               const int32_t *d_positions, const int32_t *d_activation_offsets,
+                               const int32_t *d_adapter_ids, const int32_t *d_query_start_loc,
+                               const int32_t *d_seq_lens, int T, int R, void *d_qkv, void *stream) {
+    alora_status st = check_batch_args(ctx, T, R);
+    if (st != ALORA_OK) return st;
+    if (!d_hidden || !d_positions || !d_query_start_loc || !d_seq_lens || !d_qkv) return ALORA_ERR_INVALID_ARG;
+    if (!aligned16(d_hidden) || !aligned16(d_qkv)) return ALORA_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return ALORA_ERR_INVALID_ARG;
+    if (mode < ALORA_MODE_ALORA || mode > ALORA_MODE_BASE) return ALORA_ERR_INVALID_ARG;
+    if (mode == ALORA_MODE_ALORA && d_adapter_ids && !d_activation_offsets) return ALORA_ERR_INVALID_ARG;
+    if (!ctx->layers[layer].wqkv) return ALORA_ERR_NO_WEIGHTS;
+    cudaStream_t s = (cudaStream_t)stream;
+    ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    const int32_t *d_block_tables = nullptr; const int max_blocks = 0, num_pages = 0;
+    ALORA_BATCH(mode);
+    int n = launch_metadata(ctx, b, s), k;
+    if ((k = launch_project(ctx, layer, d_hidden, T, d_qkv, s)) < 0) return ALORA_ERR_UNSUPPORTED;
+    return finish(ctx, n + k);
+}
+
+alora_status alora_kv_append(alora_ctx *ctx, const void *d_qkv, const int32_t *d_positions,
+                             const int32_t *d_query_start_loc, const int32_t *d_seq_lens,
+                             const int32_t *d_block_tables, int max_blocks, int num_pages, int T, int R,
+                             void *d_paged_kv, void *stream) {
+    alora_status st = check_batch_args(ctx, T, R);
+    if (st != ALORA_OK) return st;
+    if (!d_qkv || !d_positions || !d_query_start_loc || !d_seq_lens || !d_block_tables || !d_paged_kv)
+        return ALORA_ERR_INVALID_ARG;
+    if (!aligned16(d_qkv) || !aligned16(d_paged_kv) || max_blocks <= 0 || num_pages <= 0) return ALORA_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    const int32_t *d_activation_offsets = nullptr, *d_adapter_ids = nullptr;
+    ALORA_BATCH(ALORA_MODE_BASE);
+    int n = launch_metadata(ctx, b, s);
+    n += launch_kv_append(ctx, d_qkv, T, num_pages, d_paged_kv, s);
+    return finish(ctx, n);
+}
+
+alora_status alora_attend(alora_ctx *ctx, const void *d_qkv, const int32_t *d_positions,
+                          const int32_t *d_query_start_loc, const int32_t *d_seq_lens, const void *d_paged_kv,
+                          const int32_t *d_block_tables, int max_blocks, int num_pages, int T, int R,
+                          void *d_attn_out, void *stream) {
+    alora_status st = check_batch_args(ctx, T, R);
+    if (st != ALORA_OK) return st;
+    if (!d_qkv || !d_positions || !d_query_start_loc || !d_seq_lens || !d_block_tables || !d_paged_kv || !d_attn_out)
+        return ALORA_ERR_INVALID_ARG;
+    if (!aligned16(d_qkv) || !aligned16(d_paged_kv) || !aligned16(d_attn_out) || max_blocks <= 0 || num_pages <= 0)
+        return ALORA_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    const int32_t *d_activation_offsets = nullptr, *d_adapter_ids = nullptr;
+    ALORA_BATCH(ALORA_MODE_BASE);
+    int n = launch_metadata(ctx, b, s), k;
+    if ((k = launch_attend(ctx, d_qkv, b, d_paged_kv, d_attn_out, s)) < 0) return ALORA_ERR_UNSUPPORTED;
+    return finish(ctx, n + k);
+}
+
+static alora_status layer_entry(alora_ctx *ctx, int layer, int mode, const void *d_hidden,
+                                const int32_t *d_positions, const int32_t *d_activation_offsets,
+                                const int32_t *d_adapter_ids, const int32_t *d_query_start_loc,
+                                const int32_t *d_seq_lens, void *d_paged_kv, const int32_t *d_block_tables,
+                                int max_blocks, int num_pages, int T, int R, void *d_attn_out, void *stream) {
+    alora_status st = check_batch_args(ctx, T, R);
+    if (st != ALORA_OK) return st;
+    if (!d_hidden || !d_positions || !d_query_start_loc || !d_seq_lens || !d_block_tables || !d_paged_kv || !d_attn_out)
+        return ALORA_ERR_INVALID_ARG;
+    if (mode == ALORA_MODE_ALORA && d_adapter_ids && !d_activation_offsets) return ALORA_ERR_INVALID_ARG;
+    if (!aligned16(d_hidden) || !aligned16(d_paged_kv) || !aligned16(d_attn_out) || max_blocks <= 0 || num_pages <= 0)
+        return ALORA_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    ALORA_BATCH(mode);
+    return run_layer(ctx, layer, d_hidden, b, d_paged_kv, d_attn_out, s);
+}
+
+alora_status alora_prefill_layer(alora_ctx *ctx, int layer, const void *d_hidden, const int32_t *d_positions,
+                                 const int32_t *d_activation_offsets, const int32_t *d_adapter_ids,
+                                 const int32_t *d_query_start_loc, const int32_t *d_seq_lens, void *d_paged_kv,
+                                 const int32_t *d_block_tables, int max_blocks, int num_pages, int T, int R,
+                                 void *d_attn_out, void *stream) {
+    return layer_entry(ctx, layer, ALORA_MODE_ALORA, d_hidden, d_positions, d_activation_offsets, d_adapter_ids,
+                       d_query_start_loc, d_seq_lens, d_paged_kv, d_block_tables, max_blocks, num_pages, T, R,
+                       d_attn_out, stream);
+}
+
+alora_status alora_full_lora_prefill_layer(alora_ctx *ctx, int layer, const void *d_hidden,
+                                           const int32_t *d_positions, const int32_t *d_adapter_ids,
+                                           const int32_t *d_query_start_loc, const int32_t *d_seq_lens,
+                                           void *d_paged_kv, const int32_t *d_block_tables, int max_blocks,
+                                           int num_pages, int T, int R, void *d_attn_out, void *stream) {
+    return layer_entry(ctx, layer, ALORA_MODE_FULL_LORA, d_hidden, d_positions, nullptr, d_adapter_ids,
+                       d_query_start_loc, d_seq_lens, d_paged_kv, d_block_tables, max_blocks, num_pages, T, R,
+                       d_attn_out, stream);
+}
+
+alora_status alora_decode_step(alora_ctx *ctx, int layer, const void *d_hidden, const int32_t *d_positions,
+                               const int32_t *d_activation_offsets, const int32_t *d_adapter_ids,
+                               const int32_t *d_seq_lens, void *d_paged_kv, const int32_t *d_block_tables,
+                               int max_blocks, int num_pages, int R, void *d_attn_out, void *stream) {
+    if (!ctx) return ALORA_ERR_INVALID_ARG;
+    if (R < 0) return ALORA_ERR_INVALID_ARG;
+    if (R > ctx->cfg.max_requests || R > ctx->cfg.max_tokens) return ALORA_ERR_CAPACITY;
+    // query_start_loc of a decode batch is 0, 1, ..., R: kept in the context, built on first use
+    cudaStream_t s = (cudaStream_t)stream;
+    ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    if (!ctx->d_iota) {
+        std::vector<int32_t> iota((size_t)ctx->cfg.max_requests + 1);
+        for (size_t i = 0; i < iota.size(); ++i) iota[i] = (int32_t)i;
+        ALORA_CUDA(ctx, cudaMalloc((void **)&ctx->d_iota, iota.size() * 4));
+        ALORA_CUDA(ctx, cudaMemcpy(ctx->d_iota, iota.data(), iota.size() * 4, cudaMemcpyHostToDevice));
+    }
+    return layer_entry(ctx, layer, ALORA_MODE_ALORA, d_hidden, d_positions, d_activation_offsets, d_adapter_ids,
+                       ctx->d_iota, d_seq_lens, d_paged_kv, d_block_tables, max_blocks, num_pages, R, R, d_attn_out,
+                       stream);
+}
+
+alora_status alora_forward_stack(alora_ctx *ctx, int mode, const void *d_hidden_in, const int32_t *d_positions,
+                                 const int32_t *d_activation_offsets, const int32_t *d_adapter_ids,
+                                 const int32_t *d_query_start_loc, const int32_t *d_seq_lens,
+                                 void *const *h_paged_kv_layers, const int32_t *d_block_tables, int max_blocks,
+                                 int num_pages, int T, int R, void *d_hidden_out, void *stream) {
+    alora_status st = check_batch_args(ctx, T, R);
+    if (st != ALORA_OK) return st;
+    if (!d_hidden_in || !d_hidden_out || !d_positions || !d_query_start_loc || !d_seq_lens || !d_block_tables ||
+        !h_paged_kv_layers)
+        return ALORA_ERR_INVALID_ARG;
+    if (mode < ALORA_MODE_ALORA || mode > ALORA_MODE_BASE) return ALORA_ERR_INVALID_ARG;
+    if (mode == ALORA_MODE_ALORA && d_adapter_ids && !d_activation_offsets) return ALORA_ERR_INVALID_ARG;
+    if (ctx->d.I <= 0) return ALORA_ERR_UNSUPPORTED;
+    for (int l = 0; l < ctx->cfg.n_layers; ++l) {
+        const LayerWeights &lw = ctx->layers[l];
+        if (!lw.wqkv || !lw.wo || !lw.wgate_up || !lw.wdown || !lw.norm_attn || !lw.norm_mlp) return ALORA_ERR_NO_WEIGHTS;
+        if (!h_paged_kv_layers[l] || !aligned16(h_paged_kv_layers[l])) return ALORA_ERR_INVALID_ARG;
+    }
+    cudaStream_t s = (cudaStream_t)stream;
+    ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    const Dims &d = ctx->d;
+    ALORA_BATCH(mode);
+    if (d_hidden_out != d_hidden_in && T > 0)
+        ALORA_CUDA(ctx, cudaMemcpyAsync(d_hidden_out, d_hidden_in, (size_t)T * d.H * ctx->esize, cudaMemcpyDeviceToDevice, s));
+    char *h = (char *)d_hidden_out;  // residual stream, updated in place
+    int n = 0;
+    for (int l = 0; l < ctx->cfg.n_layers; ++l) {
+        const LayerWeights &lw = ctx->layers[l];
+        n += launch_rmsnorm(ctx, h, lw.norm_attn, T, ctx->d_act[0], s);
+        st = run_layer(ctx, l, ctx->d_act[0], b, h_paged_kv_layers[l], ctx->d_act[1], s);
+        if (st != ALORA_OK) return st;
+        n += launch_linear(ctx, ctx->d_act[1], lw.wo, T, d.Nq, d.H, h, h, s);           // h += o_proj(attn)
+        n += launch_rmsnorm(ctx, h, lw.norm_mlp, T, ctx->d_act[0], s);
+        for (int t0 = 0; t0 < T; t0 += kMlpChunk) {                                        // MLP, token chunks
+            const int tc = std::min(kMlpChunk, T - t0);
+            const char *xm = (const char *)ctx->d_act[0] + (size_t)t0 * d.H * ctx->esize;
+            char *hc = h + (size_t)t0 * d.H * ctx->esize;
+            n += launch_linear(ctx, xm, lw.wgate_up, tc, d.H, 2 * d.I, ctx->d_act[2], nullptr, s);
+            n += launch_swiglu(ctx, ctx->d_act[2], tc, ctx->d_act[3], s);
+            n += launch_linear(ctx, ctx->d_act[3], lw.wdown, tc, d.I, d.H, hc, hc, s);  // h += down(...)
+        }
+    }
+    return finish(ctx, n);
+}
+
+alora_status alora_get_status(alora_ctx *ctx, void *stream, int32_t *device_status) {
+    if (!ctx || !device_status) return ALORA_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    ALORA_CUDA(ctx, cudaMemcpyAsync(ctx->h_status, ctx->d_status, 4, cudaMemcpyDeviceToHost, s));
+    ALORA_CUDA(ctx, cudaMemsetAsync(ctx->d_status, 0, 4, s));
+    ALORA_CUDA(ctx, cudaStreamSynchronize(s));
+    *device_status = *ctx->h_status;
+    return ALORA_OK;
+}
+
+}  // extern "C"

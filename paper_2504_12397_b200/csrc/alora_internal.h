@@ -1,0 +1,125 @@
+// Internal declarations shared by the library's translation units (not part of the C ABI).
+#pragma once
+
+#include <cuda_bf16.h>
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+#include <string>
+#include <vector>
+
+#include "alora.h"
+
+namespace alora {
+
+constexpr int kRankPadMax = 64;  // adapters are stored padded to a multiple of 16 rows, <= 64
+constexpr int kMlpChunk = 8192;   // tokens per MLP pass of the stack entry (bounds the gate/up buffer)
+
+// Per (layer, adapter) record as the kernels see it.  A is [3][rpad_max][H] (q, k, v blocks, rows
+// beyond the rank are zero), B is [N][rpad_max] (row n holds the B row of output column n, columns
+// beyond the rank are zero).
+struct AdapterDev {
+    const void *A;
+    const void *B;
+    int32_t rank;   // 0 = not registered
+    int32_t rpad;   // rank rounded up to 16
+    float scale;
+    int32_t pad_;
+};
+
+struct LayerWeights {
+    const void *wqkv = nullptr, *wo = nullptr, *wgate_up = nullptr, *wdown = nullptr;
+    const void *norm_attn = nullptr, *norm_mlp = nullptr;
+};
+
+// One row-tile of the projection: rows [row_start, row_start + row_count) of the batch, all with
+// the same applied adapter (or -1).  A tile never spans two different applied adapters, so rows
+// whose gate is closed run through tiles that execute the base-only instruction sequence.
+struct ProjTile {
+    int32_t row_start;
+    int32_t row_count;
+    int32_t adapter;  // applied adapter id, -1 = none
+    int32_t pad_;
+};
+
+// One unit of attention work: query tokens [q_start, q_start + q_count) of request `req` (flat
+// token indices), one KV head, keys [kv_start, kv_end) of the request's sequence.
+struct AttnWork {
+    int32_t req;
+    int32_t q_start;
+    int32_t q_count;
+    int32_t kv_head;
+    int32_t kv_start;
+    int32_t kv_end;
+    int32_t split;     // index of this key range among the splits of the same queries
+    int32_t n_splits;
+};
+
+struct Dims {
+    int H, Hq, Hkv, hd, G, Nq, Nkv, N, page, I, RP;  // RP = padded max rank
+    float softmax_scale;
+};
+
+}  // namespace alora
+
+struct alora_ctx {
+    alora_config cfg;
+    alora::Dims d;
+    size_t esize = 2;
+    std::vector<alora::LayerWeights> layers;
+    std::vector<alora::AdapterDev> h_adapters;  // [layer * max_adapters + id], mirrors d_adapters
+    alora::AdapterDev *d_adapters = nullptr;
+    std::vector<void *> adapter_storage;         // context-owned A/B buffers, same indexing, 2 per entry
+
+    // per-call workspaces
+    int32_t *d_token_req = nullptr, *d_row_adapter = nullptr, *d_slot = nullptr;
+    alora::ProjTile *d_tiles = nullptr;
+    int32_t *d_counts = nullptr;  // [0] number of projection tiles, [1] number of attention work items
+    int32_t *d_seg_scratch = nullptr;  // [4][2*max_requests+1] merged row runs of the current batch
+    int32_t *d_iota = nullptr;         // 0..max_requests: query_start_loc of a decode batch
+    int32_t max_tiles = 0;
+    void *d_t = nullptr;          // [max_tokens][3][RP] rank-r intermediate
+    void *d_qkv = nullptr;        // [max_tokens][N]
+    void *d_act[4] = {nullptr, nullptr, nullptr, nullptr};  // stack activations
+    int32_t *d_status = nullptr;
+    int32_t *h_status = nullptr;  // pinned
+
+    int64_t launches = 0;
+    std::string cuda_err;
+    int sm_count = 148;
+};
+
+namespace alora {
+
+// Records a CUDA failure in the context and maps it to ALORA_ERR_CUDA.
+alora_status cuda_fail(alora_ctx *ctx, cudaError_t e, const char *what);
+
+#define ALORA_CUDA(ctx, call)                                              \
+    do {                                                                   \
+        cudaError_t e__ = (call);                                          \
+        if (e__ != cudaSuccess) return ::alora::cuda_fail(ctx, e__, #call); \
+    } while (0)
+
+// ---- launchers implemented in the kernel files (each returns the number of kernels launched or <0) ----
+struct BatchArgs {
+    const int32_t *positions, *activation_offsets, *adapter_ids, *query_start_loc, *seq_lens, *block_tables;
+    int max_blocks, num_pages, T, R, mode;
+};
+
+int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s);
+int launch_repack_adapter(alora_ctx *ctx, int rank, const void *Aq, const void *Bq, const void *Ak,
+                          const void *Bk, const void *Av, const void *Bv, void *A_dst, void *B_dst,
+                          cudaStream_t s);
+int launch_project(alora_ctx *ctx, int layer, const void *hidden, int T, void *qkv, cudaStream_t s);
+int launch_kv_append(alora_ctx *ctx, const void *qkv, int T, int num_pages, void *pool, cudaStream_t s);
+int launch_attend(alora_ctx *ctx, const void *qkv, const BatchArgs &b, const void *pool, void *out,
+                  cudaStream_t s);
+int launch_linear(alora_ctx *ctx, const void *x, const void *W, int T, int K, int N, void *y,
+                  const void *residual, cudaStream_t s);
+int launch_rmsnorm(alora_ctx *ctx, const void *x, const void *w, int T, void *y, cudaStream_t s);
+int launch_swiglu(alora_ctx *ctx, const void *gate_up, int T, void *y, cudaStream_t s);
+
+// device-side status recording: first finding wins
+__device__ __forceinline__ void report(int32_t *status, int code) { atomicCAS(status, 0, code); }
+
+}  // namespace alora

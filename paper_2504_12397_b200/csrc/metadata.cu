@@ -1,0 +1,146 @@
+// Batch metadata: per-token request / applied-adapter / KV-slot arrays and the projection's
+// row-tile list.  Integer work only; every output is compared exactly against the CPU oracle.
+#include "alora_internal.h"
+
+namespace alora {
+
+constexpr int kProjTileRows = 128;
+
+// Request owning flat token t: largest r with query_start_loc[r] <= t (binary search; empty
+// requests are skipped because their start equals their successor's).
+__device__ __forceinline__ int find_request(const int32_t *qsl, int R, int t) {
+    int lo = 0, hi = R;  // invariant: qsl[lo] <= t < qsl[hi]
+    while (hi - lo > 1) {
+        int mid = (lo + hi) >> 1;
+        if (qsl[mid] <= t) lo = mid; else hi = mid;
+    }
+    return lo;
+}
+
+// Per token: request index, adapter applied to the row (the gate of Eq. 5: position >= activation
+// offset; always open in full-LoRA mode, always closed in base mode), and the token slot
+// page * page_size + position % page_size.  Findings (inconsistent positions, page id out of
+// range, adapter id out of range) go to the status word; the row then gets adapter -1 / slot -1 so
+// that later kernels skip it.
+__global__ void metadata_token_kernel(const int32_t *__restrict__ positions,
+                                      const int32_t *__restrict__ a_req,
+                                      const int32_t *__restrict__ adapter_ids,
+                                      const int32_t *__restrict__ qsl, const int32_t *__restrict__ seq_lens,
+                                      const int32_t *__restrict__ block_tables, int max_blocks,
+                                      int num_pages, int page_size, int max_adapters, int T, int R, int mode,
+                                      int32_t *__restrict__ token_req, int32_t *__restrict__ row_adapter,
+                                      int32_t *__restrict__ slot_map, int32_t *status) {
+    int t = blockIdx.x * blockDim.x + threadIdx.x;
+    if (t >= T) return;
+    int r = find_request(qsl, R, t);
+    int p = positions[t];
+    // positions of a request are consecutive and end at seq_len - 1
+    int expect = seq_lens[r] - (qsl[r + 1] - t);
+    bool ok = (p == expect) && p >= 0;
+    if (!ok) report(status, ALORA_ERR_BAD_BATCH);
+    int k = -1;
+    if (mode != ALORA_MODE_BASE && adapter_ids != nullptr) {
+        k = adapter_ids[r];
+        if (k >= max_adapters || k < -1) { report(status, ALORA_ERR_BAD_BATCH); k = -1; }
+        if (k >= 0 && mode == ALORA_MODE_ALORA && p < a_req[r]) k = -1;
+    }
+    if (token_req) token_req[t] = r;
+    if (row_adapter) row_adapter[t] = ok ? k : -1;
+    if (slot_map) {
+        int slot = -1;
+        if (ok && block_tables != nullptr) {
+            int blk = p / page_size;
+            if (blk < max_blocks) {
+                int page = block_tables[(size_t)r * max_blocks + blk];
+                if (page >= 0 && page < num_pages) slot = page * page_size + p % page_size;
+                else report(status, ALORA_ERR_PAGE_RANGE);
+            } else {
+                report(status, ALORA_ERR_BAD_BATCH);
+            }
+        }
+        slot_map[t] = slot;
+    }
+}
+
+// Row tiles of the projection.  Each request contributes up to two runs of rows: its gated-off
+// rows (applied adapter -1) and its gated-on rows; neighbouring runs with the same applied adapter
+// are merged across requests, and every merged run is cut into tiles of at most kProjTileRows rows.
+// One block; R is small (a scheduler batch).
+__global__ void metadata_tiles_kernel(const int32_t *__restrict__ a_req, const int32_t *__restrict__ adapter_ids,
+                                      const int32_t *__restrict__ qsl, const int32_t *__restrict__ seq_lens,
+                                      int R, int mode, int max_adapters, int max_tiles,
+                                      ProjTile *__restrict__ tiles, int32_t *__restrict__ counts,
+                                      int32_t *seg_scratch /* [4 * (2R+1)] */, int32_t *status) {
+    int32_t *seg_start = seg_scratch, *seg_len = seg_scratch + (2 * R + 1);
+    int32_t *seg_adapter = seg_scratch + 2 * (2 * R + 1), *seg_tile0 = seg_scratch + 3 * (2 * R + 1);
+    __shared__ int n_seg, n_tiles;
+    if (threadIdx.x == 0) {
+        int ns = 0, nt = 0;
+        for (int r = 0; r < R; ++r) {
+            int n_new = qsl[r + 1] - qsl[r];
+            if (n_new <= 0) continue;
+            int k = (mode == ALORA_MODE_BASE || adapter_ids == nullptr) ? -1 : adapter_ids[r];
+            if (k >= max_adapters || k < -1) k = -1;
+            int n_off = 0;
+            if (k < 0) n_off = n_new;
+            else if (mode == ALORA_MODE_ALORA) {
+                int p_first = seq_lens[r] - n_new;
+                long long d = (long long)a_req[r] - p_first;
+                n_off = d <= 0 ? 0 : (d >= n_new ? n_new : (int)d);
+            }
+            int start[2] = {qsl[r], qsl[r] + n_off};
+            int len[2] = {n_off, n_new - n_off};
+            int ad[2] = {-1, k};
+            for (int i = 0; i < 2; ++i) {
+                if (len[i] <= 0) continue;
+                if (ns > 0 && seg_adapter[ns - 1] == ad[i] && seg_start[ns - 1] + seg_len[ns - 1] == start[i]) {
+                    seg_len[ns - 1] += len[i];
+                } else {
+                    seg_start[ns] = start[i]; seg_len[ns] = len[i]; seg_adapter[ns] = ad[i];
+                    ++ns;
+                }
+            }
+        }
+        for (int s = 0; s < ns; ++s) {
+            seg_tile0[s] = nt;
+            nt += (seg_len[s] + kProjTileRows - 1) / kProjTileRows;
+        }
+        seg_tile0[ns] = nt;
+        if (nt > max_tiles) { report(status, ALORA_ERR_CAPACITY); nt = 0; ns = 0; }
+        n_seg = ns; n_tiles = nt;
+        counts[0] = nt;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < n_tiles; i += blockDim.x) {
+        int lo = 0, hi = n_seg;  // seg_tile0[lo] <= i < seg_tile0[hi]
+        while (hi - lo > 1) {
+            int mid = (lo + hi) >> 1;
+            if (seg_tile0[mid] <= i) lo = mid; else hi = mid;
+        }
+        int off = (i - seg_tile0[lo]) * kProjTileRows;
+        ProjTile pt;
+        pt.row_start = seg_start[lo] + off;
+        pt.row_count = min(kProjTileRows, seg_len[lo] - off);
+        pt.adapter = seg_adapter[lo];
+        pt.pad_ = 0;
+        tiles[i] = pt;
+    }
+}
+
+int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s) {
+    if (b.T == 0) {
+        cudaMemsetAsync(ctx->d_counts, 0, 2 * sizeof(int32_t), s);
+        return 0;
+    }
+    const int threads = 256;
+    metadata_token_kernel<<<(b.T + threads - 1) / threads, threads, 0, s>>>(
+        b.positions, b.activation_offsets, b.adapter_ids, b.query_start_loc, b.seq_lens, b.block_tables,
+        b.max_blocks, b.num_pages, ctx->d.page, ctx->cfg.max_adapters, b.T, b.R, b.mode,
+        ctx->d_token_req, ctx->d_row_adapter, ctx->d_slot, ctx->d_status);
+    metadata_tiles_kernel<<<1, 256, 0, s>>>(b.activation_offsets, b.adapter_ids, b.query_start_loc,
+                                           b.seq_lens, b.R, b.mode, ctx->cfg.max_adapters, ctx->max_tiles,
+                                           ctx->d_tiles, ctx->d_counts, ctx->d_seg_scratch, ctx->d_status);
+    return 2;
+}
+
+}  // namespace alora

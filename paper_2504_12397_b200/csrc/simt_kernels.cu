@@ -1,0 +1,377 @@
+// CUDA-core kernels: the fp32 data type's projection and attention (tiny exact-precision
+// configurations), and the element-wise / copy steps shared by both data types (adapter repack,
+// KV append, RMSNorm, SwiGLU).
+#include "alora_internal.h"
+
+namespace alora {
+
+template <typename T> __device__ __forceinline__ float ldf(const T *p);
+template <> __device__ __forceinline__ float ldf<float>(const float *p) { return *p; }
+template <> __device__ __forceinline__ float ldf<__nv_bfloat16>(const __nv_bfloat16 *p) { return __bfloat162float(*p); }
+template <typename T> __device__ __forceinline__ void stf(T *p, float v);
+template <> __device__ __forceinline__ void stf<float>(float *p, float v) { *p = v; }
+template <> __device__ __forceinline__ void stf<__nv_bfloat16>(__nv_bfloat16 *p, float v) { *p = __float2bfloat16_rn(v); }
+
+// ---------------------------------------------------------------------------------------------
+// Adapter repack: A_dst[3][RP][H] <- (Aq, Ak, Av)[r][H] with zero rows r..RP-1;
+// B_dst[N][RP] <- rows of (Bq | Bk | Bv)[.][r] with zero columns r..RP-1.
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void repack_adapter_kernel(const T *Aq, const T *Ak, const T *Av, const T *Bq, const T *Bk,
+                                      const T *Bv, int rank, int RP, int H, int Nq, int Nkv, T *A_dst,
+                                      T *B_dst) {
+    const size_t nA = (size_t)3 * RP * H, nB = (size_t)(Nq + 2 * Nkv) * RP;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < nA + nB;
+         i += (size_t)gridDim.x * blockDim.x) {
+        if (i < nA) {
+            int blk = (int)(i / ((size_t)RP * H));
+            int row = (int)((i / H) % RP), h = (int)(i % H);
+            const T *src = blk == 0 ? Aq : (blk == 1 ? Ak : Av);
+            A_dst[i] = row < rank ? src[(size_t)row * H + h] : T(0.f);
+        } else {
+            size_t j = i - nA;
+            int n = (int)(j / RP), c = (int)(j % RP);
+            T v = T(0.f);
+            if (c < rank) {
+                if (n < Nq) v = Bq[(size_t)n * rank + c];
+                else if (n < Nq + Nkv) v = Bk[(size_t)(n - Nq) * rank + c];
+                else v = Bv[(size_t)(n - Nq - Nkv) * rank + c];
+            }
+            B_dst[j] = v;
+        }
+    }
+}
+
+int launch_repack_adapter(alora_ctx *ctx, int rank, const void *Aq, const void *Bq, const void *Ak,
+                          const void *Bk, const void *Av, const void *Bv, void *A_dst, void *B_dst,
+                          cudaStream_t s) {
+    const Dims &d = ctx->d;
+    if (ctx->cfg.dtype == ALORA_DTYPE_FP32)
+        repack_adapter_kernel<float><<<256, 256, 0, s>>>((const float *)Aq, (const float *)Ak, (const float *)Av,
+                                                         (const float *)Bq, (const float *)Bk, (const float *)Bv,
+                                                         rank, d.RP, d.H, d.Nq, d.Nkv, (float *)A_dst, (float *)B_dst);
+    else
+        repack_adapter_kernel<__nv_bfloat16><<<256, 256, 0, s>>>(
+            (const __nv_bfloat16 *)Aq, (const __nv_bfloat16 *)Ak, (const __nv_bfloat16 *)Av,
+            (const __nv_bfloat16 *)Bq, (const __nv_bfloat16 *)Bk, (const __nv_bfloat16 *)Bv, rank, d.RP, d.H,
+            d.Nq, d.Nkv, (__nv_bfloat16 *)A_dst, (__nv_bfloat16 *)B_dst);
+    return 1;
+}
+
+// ---------------------------------------------------------------------------------------------
+// CUDA-core shrink: t[row][blk][i] = scale * sum_h A[blk][i][h] x[row][h] for rows with an applied
+// adapter (Eq. 5, inner product of the low-rank delta).  One block per row, one warp per output.
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void shrink_simt_kernel(const T *__restrict__ x, const int32_t *__restrict__ row_adapter,
+                                  const AdapterDev *__restrict__ adapters, int H, int RP,
+                                  float *__restrict__ t) {
+    const int row = blockIdx.x;
+    const int k = row_adapter[row];
+    if (k < 0) return;
+    const AdapterDev ad = adapters[k];
+    const T *A = (const T *)ad.A;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = blockDim.x >> 5;
+    for (int o = warp; o < 3 * RP; o += nwarps) {
+        const int i = o % RP;
+        float acc = 0.f;
+        if (i < ad.rank) {
+            const T *a = A + (size_t)o * H;
+            for (int h = lane; h < H; h += 32) acc += ldf(a + h) * ldf(x + (size_t)row * H + h);
+            for (int off = 16; off; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+        }
+        if (lane == 0) t[(size_t)row * 3 * RP + o] = acc * ad.scale;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// CUDA-core projection y[row][n] = sum_h W[n][h] x[row][h]  (+ sum_i B[n][i] t[row][blk(n)][i] when the
+// row has an applied adapter).  64x64 output tile per block, 16x16 threads, 4x4 outputs each,
+// K staged through shared memory 16 columns at a time.  The base sum of a row is formed by the
+// same instruction sequence whether or not the delta follows, so gated-off rows equal a base-only
+// call bit for bit.  Optional residual: y += residual[row][n] (used by o_proj / down_proj).
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void __launch_bounds__(256)
+linear_simt_kernel(const T *__restrict__ x, const T *__restrict__ W, int Tn, int K, int N,
+                  const int32_t *__restrict__ row_adapter, const AdapterDev *__restrict__ adapters,
+                  const float *__restrict__ t, int RP, int Nq, int Nkv, const T *residual /* may alias y */,
+                   T *y) {
+    __shared__ float xs[16][64 + 1], ws[16][64 + 1];
+    const int tx = threadIdx.x & 15, ty = threadIdx.x >> 4;
+    const int row0 = blockIdx.y * 64, col0 = blockIdx.x * 64;
+    float acc[4][4] = {};
+    for (int k0 = 0; k0 < K; k0 += 16) {
+        for (int i = threadIdx.x; i < 64 * 16; i += 256) {
+            int rr = i >> 4, kk = i & 15;
+            int gr = row0 + rr, gc = col0 + rr, gk = k0 + kk;
+            xs[kk][rr] = (gr < Tn && gk < K) ? ldf(x + (size_t)gr * K + gk) : 0.f;
+            ws[kk][rr] = (gc < N && gk < K) ? ldf(W + (size_t)gc * K + gk) : 0.f;
+        }
+        __syncthreads();
+#pragma unroll
+        for (int kk = 0; kk < 16; ++kk) {
+            float a[4], b[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) { a[i] = xs[kk][ty * 4 + i]; b[i] = ws[kk][tx * 4 + i]; }
+#pragma unroll
+            for (int i = 0; i < 4; ++i)
+#pragma unroll
+                for (int j = 0; j < 4; ++j) acc[i][j] += a[i] * b[j];
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int row = row0 + ty * 4 + i;
+        if (row >= Tn) continue;
+        const int k = row_adapter ? row_adapter[row] : -1;
+#pragma unroll
+        for (int j = 0; j < 4; ++j) {
+            const int n = col0 + tx * 4 + j;
+            if (n >= N) continue;
+            float v = acc[i][j];
+            if (k >= 0) {
+                const AdapterDev ad = adapters[k];
+                const T *B = (const T *)ad.B + (size_t)n * RP;
+                const int blk = n < Nq ? 0 : (n < Nq + Nkv ? 1 : 2);
+                const float *tr = t + ((size_t)row * 3 + blk) * RP;
+                float dlt = 0.f;
+                for (int r = 0; r < ad.rank; ++r) dlt += ldf(B + r) * tr[r];
+                v += dlt;
+            }
+            if (residual) v += ldf(residual + (size_t)row * N + n);
+            stf(y + (size_t)row * N + n, v);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// KV append (both data types): one 16-byte vector per thread.  Row t's k part
+// qkv[t][Nq .. Nq+Nkv) goes to pool[page][0][head][row][:], its v part to plane 1.  Tokens whose
+// slot is -1 (rejected by the metadata step) are skipped.
+// ---------------------------------------------------------------------------------------------
+__global__ void kv_append_kernel(const uint4 *__restrict__ qkv, const int32_t *__restrict__ slot_map,
+                                 int T, int N_vec, int Nq_vec, int Nkv_vec, int hd_vec, int Hkv,
+                                 int page_size, int num_pages, uint4 *__restrict__ pool, int32_t *status) {
+    const size_t total = (size_t)T * 2 * Nkv_vec;
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total;
+         i += (size_t)gridDim.x * blockDim.x) {
+        const int t = (int)(i / (2 * Nkv_vec));
+        const int c = (int)(i % (2 * Nkv_vec));   // vector column inside [k | v]
+        const int plane = c / Nkv_vec, cc = c % Nkv_vec;
+        const int head = cc / hd_vec, dv = cc % hd_vec;
+        const int slot = slot_map[t];
+        if (slot < 0) continue;
+        const int page = slot / page_size, row = slot % page_size;
+        if (page >= num_pages) { report(status, ALORA_ERR_PAGE_RANGE); continue; }
+        const size_t dst = ((((size_t)page * 2 + plane) * Hkv + head) * page_size + row) * hd_vec + dv;
+        pool[dst] = qkv[(size_t)t * N_vec + Nq_vec + c];
+    }
+}
+
+int launch_kv_append(alora_ctx *ctx, const void *qkv, int T, int num_pages, void *pool, cudaStream_t s) {
+    if (T == 0) return 0;
+    const Dims &d = ctx->d;
+    const int vec = 16 / (int)ctx->esize;  // elements per 16-byte vector
+    const size_t total = (size_t)T * 2 * (d.Nkv / vec);
+    int blocks = (int)((total + 255) / 256);
+    if (blocks > ctx->sm_count * 16) blocks = ctx->sm_count * 16;
+    kv_append_kernel<<<blocks, 256, 0, s>>>((const uint4 *)qkv, ctx->d_slot, T, d.N / vec, d.Nq / vec,
+                                            d.Nkv / vec, d.hd / vec, d.Hkv, d.page, num_pages, (uint4 *)pool,
+                                            ctx->d_status);
+    return 1;
+}
+
+// ---------------------------------------------------------------------------------------------
+// CUDA-core attention (Eq. 1 / Eq. 3): one warp per (token, query head); the block holds the G query
+// heads that share a KV head.  Keys are taken 32 at a time: lane j scores key j0 + j against the
+// query kept in shared memory, the warp combines the 32 scores with shuffles (running maximum and
+// sum: online softmax), then every lane accumulates its slice of the head dimension over the 32
+// value rows.
+// ---------------------------------------------------------------------------------------------
+template <typename T, int HD>
+__global__ void attn_simt_kernel(const T *__restrict__ qkv, const int32_t *__restrict__ positions,
+                                const int32_t *__restrict__ token_req, const int32_t *__restrict__ slot_map,
+                                const int32_t *__restrict__ block_tables, int max_blocks, int num_pages, int page_size, int N, int Nq, int Hkv, int G,
+                                float scale, const T *__restrict__ pool, T *__restrict__ out,
+                                 int32_t *status) {
+    extern __shared__ float q_s[];  // [G][HD]
+    constexpr int DPL = HD / 32;    // head-dim elements per lane
+    const int t = blockIdx.x, kvh = blockIdx.y;
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int h = kvh * G + warp;
+    const int r = token_req[t];
+    const int p = positions[t];
+    if (slot_map[t] < 0) {  // token rejected by the metadata step: defined output, no cache access
+        for (int d = lane; d < HD; d += 32) stf(out + (size_t)t * Nq + (size_t)h * HD + d, 0.f);
+        return;
+    }
+    float *qs = q_s + warp * HD;
+    for (int d = lane; d < HD; d += 32) qs[d] = ldf(qkv + (size_t)t * N + (size_t)h * HD + d) * scale;
+    __syncwarp();
+    float m = -INFINITY, l = 0.f, acc[DPL];
+#pragma unroll
+    for (int i = 0; i < DPL; ++i) acc[i] = 0.f;
+    const size_t plane_stride = (size_t)Hkv * page_size * HD;
+    for (int j0 = 0; j0 <= p; j0 += 32) {
+        const int j = j0 + lane;
+        float s = -INFINITY;
+        const T *krow = nullptr;
+        if (j <= p) {
+            const int page = block_tables[(size_t)r * max_blocks + j / page_size];
+            if (page >= 0 && page < num_pages) {
+                krow = pool + ((size_t)page * 2 * Hkv + kvh) * page_size * HD + (size_t)(j % page_size) * HD;
+                float dot = 0.f;
+#pragma unroll 8
+                for (int d = 0; d < HD; ++d) dot += qs[d] * ldf(krow + d);
+                s = dot;
+            } else {
+                report(status, ALORA_ERR_PAGE_RANGE);
+            }
+        }
+        float mx = s;
+        for (int off = 16; off; off >>= 1) mx = fmaxf(mx, __shfl_xor_sync(0xffffffffu, mx, off));
+        const float m_new = fmaxf(m, mx);
+        if (m_new == -INFINITY) continue;  // nothing visible in this group (only on bad pages)
+        const float w = (s == -INFINITY) ? 0.f : __expf(s - m_new);
+        float wsum = w;
+        for (int off = 16; off; off >>= 1) wsum += __shfl_xor_sync(0xffffffffu, wsum, off);
+        const float corr = (m == -INFINITY) ? 0.f : __expf(m - m_new);
+        l = l * corr + wsum;
+#pragma unroll
+        for (int i = 0; i < DPL; ++i) acc[i] *= corr;
+        const int nvis = min(32, p - j0 + 1);
+        for (int jj = 0; jj < nvis; ++jj) {
+            const float wj = __shfl_sync(0xffffffffu, w, jj);
+            const unsigned long long kp = __shfl_sync(0xffffffffu, (unsigned long long)krow, jj);
+            if (kp == 0ull) continue;
+            const T *vrow = (const T *)kp + plane_stride;
+#pragma unroll
+            for (int i = 0; i < DPL; ++i) acc[i] += wj * ldf(vrow + lane + 32 * i);
+        }
+        m = m_new;
+    }
+    const float inv = l > 0.f ? 1.f / l : 0.f;
+#pragma unroll
+    for (int i = 0; i < DPL; ++i) stf(out + (size_t)t * Nq + (size_t)h * HD + lane + 32 * i, acc[i] * inv);
+}
+
+// ---------------------------------------------------------------------------------------------
+// RMSNorm and SwiGLU (decoder-stack glue; both data types, fp32 arithmetic).
+// ---------------------------------------------------------------------------------------------
+template <typename T>
+__global__ void rmsnorm_kernel(const T *__restrict__ x, const T *__restrict__ w, int H, float eps,
+                               T *__restrict__ y) {
+    const size_t row = blockIdx.x;
+    __shared__ float red[32];
+    float ss = 0.f;
+    for (int h = threadIdx.x; h < H; h += blockDim.x) { float v = ldf(x + row * H + h); ss += v * v; }
+    for (int off = 16; off; off >>= 1) ss += __shfl_xor_sync(0xffffffffu, ss, off);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = ss;
+    __syncthreads();
+    if (threadIdx.x < 32) {
+        float v = threadIdx.x < (blockDim.x >> 5) ? red[threadIdx.x] : 0.f;
+        for (int off = 16; off; off >>= 1) v += __shfl_xor_sync(0xffffffffu, v, off);
+        if (threadIdx.x == 0) red[0] = rsqrtf(v / (float)H + eps);
+    }
+    __syncthreads();
+    const float inv = red[0];
+    for (int h = threadIdx.x; h < H; h += blockDim.x)
+        stf(y + row * H + h, ldf(x + row * H + h) * inv * ldf(w + h));
+}
+
+template <typename T>
+__global__ void swiglu_kernel(const T *__restrict__ gate_up, int I, size_t total, T *__restrict__ y) {
+    for (size_t i = blockIdx.x * (size_t)blockDim.x + threadIdx.x; i < total;
+         i += (size_t)gridDim.x * blockDim.x) {
+        const size_t row = i / I, c = i % I;
+        const float g = ldf(gate_up + row * 2 * I + c), u = ldf(gate_up + row * 2 * I + I + c);
+        stf(y + i, g / (1.f + __expf(-g)) * u);
+    }
+}
+
+int launch_rmsnorm(alora_ctx *ctx, const void *x, const void *w, int T, void *y, cudaStream_t s) {
+    if (T == 0) return 0;
+    if (ctx->cfg.dtype == ALORA_DTYPE_FP32)
+        rmsnorm_kernel<float><<<T, 256, 0, s>>>((const float *)x, (const float *)w, ctx->d.H, ctx->cfg.rms_eps, (float *)y);
+    else
+        rmsnorm_kernel<__nv_bfloat16><<<T, 256, 0, s>>>((const __nv_bfloat16 *)x, (const __nv_bfloat16 *)w, ctx->d.H,
+                                                        ctx->cfg.rms_eps, (__nv_bfloat16 *)y);
+    return 1;
+}
+
+int launch_swiglu(alora_ctx *ctx, const void *gate_up, int T, void *y, cudaStream_t s) {
+    if (T == 0) return 0;
+    const size_t total = (size_t)T * ctx->d.I;
+    int blocks = (int)((total + 255) / 256);
+    if (blocks > ctx->sm_count * 16) blocks = ctx->sm_count * 16;
+    if (ctx->cfg.dtype == ALORA_DTYPE_FP32)
+        swiglu_kernel<float><<<blocks, 256, 0, s>>>((const float *)gate_up, ctx->d.I, total, (float *)y);
+    else
+        swiglu_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>((const __nv_bfloat16 *)gate_up, ctx->d.I, total,
+                                                           (__nv_bfloat16 *)y);
+    return 1;
+}
+
+// ---- launchers of the CUDA-core projection / attention, by data type -------------------------------
+template <typename T>
+static int project_simt(alora_ctx *ctx, int layer, const void *hidden, int Tn, void *qkv, cudaStream_t s) {
+    const Dims &d = ctx->d;
+    const AdapterDev *ads = ctx->d_adapters + (size_t)layer * ctx->cfg.max_adapters;
+    shrink_simt_kernel<T><<<Tn, 256, 0, s>>>((const T *)hidden, ctx->d_row_adapter, ads, d.H, d.RP, (float *)ctx->d_t);
+    dim3 grid((d.N + 63) / 64, (Tn + 63) / 64);
+    linear_simt_kernel<T><<<grid, 256, 0, s>>>((const T *)hidden, (const T *)ctx->layers[layer].wqkv, Tn, d.H, d.N,
+                                               ctx->d_row_adapter, ads, (const float *)ctx->d_t, d.RP, d.Nq, d.Nkv,
+                                               nullptr, (T *)qkv);
+    return 2;
+}
+
+int launch_project_simt(alora_ctx *ctx, int layer, const void *hidden, int T, void *qkv, cudaStream_t s) {
+    if (T == 0) return 0;
+    return ctx->cfg.dtype == ALORA_DTYPE_FP32 ? project_simt<float>(ctx, layer, hidden, T, qkv, s)
+                                              : project_simt<__nv_bfloat16>(ctx, layer, hidden, T, qkv, s);
+}
+
+int launch_linear_simt(alora_ctx *ctx, const void *x, const void *W, int T, int K, int N, void *y,
+                       const void *residual, cudaStream_t s) {
+    if (T == 0) return 0;
+    dim3 grid((N + 63) / 64, (T + 63) / 64);
+    if (ctx->cfg.dtype == ALORA_DTYPE_FP32)
+        linear_simt_kernel<float><<<grid, 256, 0, s>>>((const float *)x, (const float *)W, T, K, N, nullptr, nullptr,
+                                                       nullptr, 0, 0, 0, (const float *)residual, (float *)y);
+    else
+        linear_simt_kernel<__nv_bfloat16><<<grid, 256, 0, s>>>((const __nv_bfloat16 *)x, (const __nv_bfloat16 *)W, T, K,
+                                                               N, nullptr, nullptr, nullptr, 0, 0, 0,
+                                                               (const __nv_bfloat16 *)residual, (__nv_bfloat16 *)y);
+    return 1;
+}
+
+template <typename T>
+static int attend_simt(alora_ctx *ctx, const void *qkv, const BatchArgs &b, const void *pool, void *out,
+                       cudaStream_t s) {
+    const Dims &d = ctx->d;
+    dim3 grid(b.T, d.Hkv);
+    const int threads = 32 * d.G;
+    const size_t smem = (size_t)d.G * d.hd * sizeof(float);
+#define ALORA_ATTN_SIMT(HD)                                                                              \
+    attn_simt_kernel<T, HD><<<grid, threads, smem, s>>>((const T *)qkv, b.positions, ctx->d_token_req,   \
+                                                        ctx->d_slot, b.block_tables, b.max_blocks, b.num_pages, d.page, \
+                                                        d.N, d.Nq, d.Hkv, d.G, d.softmax_scale,           \
+                                                        (const T *)pool, (T *)out, ctx->d_status)
+    if (d.hd == 32) ALORA_ATTN_SIMT(32);
+    else if (d.hd == 64) ALORA_ATTN_SIMT(64);
+    else if (d.hd == 128) ALORA_ATTN_SIMT(128);
+    else return -1;
+#undef ALORA_ATTN_SIMT
+    return 1;
+}
+
+int launch_attend_simt(alora_ctx *ctx, const void *qkv, const BatchArgs &b, const void *pool, void *out,
+                       cudaStream_t s) {
+    if (b.T == 0) return 0;
+    return ctx->cfg.dtype == ALORA_DTYPE_FP32 ? attend_simt<float>(ctx, qkv, b, pool, out, s)
+                                              : attend_simt<__nv_bfloat16>(ctx, qkv, b, pool, out, s);
+}
+
+}  // namespace alora
