@@ -244,6 +244,19 @@ const char *alora_last_cuda_error(const alora_ctx *ctx);
 /* Number of kernels this context has launched so far (all entry points). */
 int64_t alora_launch_count(const alora_ctx *ctx);
 
+/*
+ * Optional per-kernel timing (a measurement aid; the paper has no counterpart).  While enabled,
+ * every kernel family launched by this context is bracketed by CUDA events on the launching stream.
+ * alora_profile_enable(ctx, 1) clears what was accumulated and starts, (ctx, 0) stops.
+ * alora_profile_read synchronises the device and adds up, per family, the elapsed milliseconds and
+ * the number of bracketed launch groups; both arrays have ALORA_PROFILE_KINDS entries.
+ * Families: 0 batch metadata, 1 rank-r shrink (t = A x), 2 q/k/v projection, 3 KV append,
+ * 4 attention, 5 split-KV merge, 6 other dense projections (o_proj, MLP), 7 norm / activation glue.
+ */
+#define ALORA_PROFILE_KINDS 8
+alora_status alora_profile_enable(alora_ctx *ctx, int on);
+alora_status alora_profile_read(alora_ctx *ctx, double *ms_by_kind, int64_t *groups_by_kind);
+
 #ifdef __cplusplus
 }
 #endif

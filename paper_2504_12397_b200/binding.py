@@ -60,7 +60,9 @@ def _signatures(lib):
     lib.alora_last_cuda_error.restype = C.c_char_p
     lib.alora_launch_count.argtypes = [_VP]
     lib.alora_launch_count.restype = C.c_int64
-    for name in ("alora_create", "alora_destroy", "alora_set_layer_weights", "alora_register_adapter",
+    lib.alora_profile_enable.argtypes = [_VP, _I]
+    lib.alora_profile_read.argtypes = [_VP, C.POINTER(C.c_double), C.POINTER(C.c_int64)]
+    for name in ("alora_profile_enable", "alora_profile_read", "alora_create", "alora_destroy", "alora_set_layer_weights", "alora_register_adapter",
                  "alora_validate_batch", "alora_batch_metadata", "alora_project_qkv", "alora_kv_append",
                  "alora_attend", "alora_prefill_layer", "alora_decode_step",
                  "alora_full_lora_prefill_layer", "alora_forward_stack", "alora_get_status"):
@@ -240,3 +242,18 @@ def alora_get_status(ctx, stream=None) -> int:
 
 def alora_launch_count(ctx) -> int:
     return int(load_library().alora_launch_count(ctx))
+
+
+PROFILE_KINDS = ("metadata", "shrink", "project_qkv", "kv_append", "attention", "attn_merge", "linear", "glue")
+
+
+def alora_profile_enable(ctx, on: bool) -> None:
+    _check(ctx, load_library().alora_profile_enable(ctx, int(bool(on))), "alora_profile_enable")
+
+
+def alora_profile_read(ctx) -> dict:
+    """{family: (milliseconds, launch groups)} accumulated since profiling was enabled."""
+    ms = (C.c_double * len(PROFILE_KINDS))()
+    n = (C.c_int64 * len(PROFILE_KINDS))()
+    _check(ctx, load_library().alora_profile_read(ctx, ms, n), "alora_profile_read")
+    return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(PROFILE_KINDS)}

@@ -172,6 +172,7 @@ alora_status alora_destroy(alora_ctx *ctx) {
                     ctx->d_act[2], ctx->d_act[3], ctx->d_iota};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (ctx->h_status) cudaFreeHost(ctx->h_status);
+    for (ProfEvent &e : ctx->prof_events) { if (e.begin) cudaEventDestroy(e.begin); if (e.end) cudaEventDestroy(e.end); }
     delete ctx;
     return ALORA_OK;
 }
@@ -441,6 +442,29 @@ alora_status alora_forward_stack(alora_ctx *ctx, int mode, const void *d_hidden_
         }
     }
     return finish(ctx, n);
+}
+
+alora_status alora_profile_enable(alora_ctx *ctx, int on) {
+    if (!ctx) return ALORA_ERR_INVALID_ARG;
+    ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    ALORA_CUDA(ctx, cudaDeviceSynchronize());
+    ctx->profiling = on != 0;
+    if (on) ctx->prof_used = 0;
+    return ALORA_OK;
+}
+
+alora_status alora_profile_read(alora_ctx *ctx, double *ms_by_kind, int64_t *groups_by_kind) {
+    if (!ctx || !ms_by_kind || !groups_by_kind) return ALORA_ERR_INVALID_ARG;
+    ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    ALORA_CUDA(ctx, cudaDeviceSynchronize());
+    for (int k = 0; k < ALORA_PROFILE_KINDS; ++k) { ms_by_kind[k] = 0.0; groups_by_kind[k] = 0; }
+    for (size_t i = 0; i < ctx->prof_used; ++i) {
+        const ProfEvent &e = ctx->prof_events[i];
+        float ms = 0.f;
+        ALORA_CUDA(ctx, cudaEventElapsedTime(&ms, e.begin, e.end));
+        if (e.kind >= 0 && e.kind < ALORA_PROFILE_KINDS) { ms_by_kind[e.kind] += ms; groups_by_kind[e.kind] += 1; }
+    }
+    return ALORA_OK;
 }
 
 alora_status alora_get_status(alora_ctx *ctx, void *stream, int32_t *device_status) {

@@ -55,6 +55,15 @@ struct AttnWork {
     int32_t n_splits;
 };
 
+// Kernel families, for the optional per-kernel timing (alora_profile_*).
+enum KernelKind { KK_METADATA = 0, KK_SHRINK, KK_PROJECT, KK_KV_APPEND, KK_ATTENTION, KK_ATTN_MERGE, KK_LINEAR,
+                  KK_GLUE, KK_COUNT };
+
+struct ProfEvent {
+    cudaEvent_t begin, end;
+    int kind;
+};
+
 struct Dims {
     int H, Hq, Hkv, hd, G, Nq, Nkv, N, page, I, RP;  // RP = padded max rank
     float softmax_scale;
@@ -84,6 +93,9 @@ struct alora_ctx {
     int32_t *d_status = nullptr;
     int32_t *h_status = nullptr;  // pinned
 
+    bool profiling = false;
+    std::vector<alora::ProfEvent> prof_events;  // event pairs recorded since profiling was enabled
+    size_t prof_used = 0;
     int64_t launches = 0;
     std::string cuda_err;
     int sm_count = 148;
@@ -99,6 +111,26 @@ alora_status cuda_fail(alora_ctx *ctx, cudaError_t e, const char *what);
         cudaError_t e__ = (call);                                          \
         if (e__ != cudaSuccess) return ::alora::cuda_fail(ctx, e__, #call); \
     } while (0)
+
+// Brackets the launches of one kernel family with CUDA events while profiling is on.
+struct ProfScope {
+    alora_ctx *ctx;
+    cudaStream_t s;
+    cudaEvent_t end = nullptr;
+    ProfScope(alora_ctx *c, int kind, cudaStream_t st) : ctx(c), s(st) {
+        if (!c->profiling) return;
+        if (c->prof_used == c->prof_events.size()) {
+            ProfEvent e{nullptr, nullptr, kind};
+            if (cudaEventCreate(&e.begin) != cudaSuccess || cudaEventCreate(&e.end) != cudaSuccess) return;
+            c->prof_events.push_back(e);
+        }
+        ProfEvent &e = c->prof_events[c->prof_used++];
+        e.kind = kind;
+        cudaEventRecord(e.begin, st);
+        end = e.end;
+    }
+    ~ProfScope() { if (end) cudaEventRecord(end, s); }
+};
 
 // ---- launchers implemented in the kernel files (each returns the number of kernels launched or <0) ----
 struct BatchArgs {

@@ -132,6 +132,7 @@ int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s) {
         cudaMemsetAsync(ctx->d_counts, 0, 2 * sizeof(int32_t), s);
         return 0;
     }
+    ProfScope prof(ctx, KK_METADATA, s);
     const int threads = 256;
     metadata_token_kernel<<<(b.T + threads - 1) / threads, threads, 0, s>>>(
         b.positions, b.activation_offsets, b.adapter_ids, b.query_start_loc, b.seq_lens, b.block_tables,

@@ -173,6 +173,7 @@ __global__ void kv_append_kernel(const uint4 *__restrict__ qkv, const int32_t *_
 int launch_kv_append(alora_ctx *ctx, const void *qkv, int T, int num_pages, void *pool, cudaStream_t s) {
     if (T == 0) return 0;
     const Dims &d = ctx->d;
+    ProfScope prof(ctx, KK_KV_APPEND, s);
     const int vec = 16 / (int)ctx->esize;  // elements per 16-byte vector
     const size_t total = (size_t)T * 2 * (d.Nkv / vec);
     int blocks = (int)((total + 255) / 256);
@@ -293,6 +294,7 @@ __global__ void swiglu_kernel(const T *__restrict__ gate_up, int I, size_t total
 
 int launch_rmsnorm(alora_ctx *ctx, const void *x, const void *w, int T, void *y, cudaStream_t s) {
     if (T == 0) return 0;
+    ProfScope prof(ctx, KK_GLUE, s);
     if (ctx->cfg.dtype == ALORA_DTYPE_FP32)
         rmsnorm_kernel<float><<<T, 256, 0, s>>>((const float *)x, (const float *)w, ctx->d.H, ctx->cfg.rms_eps, (float *)y);
     else
@@ -303,6 +305,7 @@ int launch_rmsnorm(alora_ctx *ctx, const void *x, const void *w, int T, void *y,
 
 int launch_swiglu(alora_ctx *ctx, const void *gate_up, int T, void *y, cudaStream_t s) {
     if (T == 0) return 0;
+    ProfScope prof(ctx, KK_GLUE, s);
     const size_t total = (size_t)T * ctx->d.I;
     int blocks = (int)((total + 255) / 256);
     if (blocks > ctx->sm_count * 16) blocks = ctx->sm_count * 16;
@@ -319,7 +322,11 @@ template <typename T>
 static int project_simt(alora_ctx *ctx, int layer, const void *hidden, int Tn, void *qkv, cudaStream_t s) {
     const Dims &d = ctx->d;
     const AdapterDev *ads = ctx->d_adapters + (size_t)layer * ctx->cfg.max_adapters;
-    shrink_simt_kernel<T><<<Tn, 256, 0, s>>>((const T *)hidden, ctx->d_row_adapter, ads, d.H, d.RP, (float *)ctx->d_t);
+    {
+        ProfScope prof(ctx, KK_SHRINK, s);
+        shrink_simt_kernel<T><<<Tn, 256, 0, s>>>((const T *)hidden, ctx->d_row_adapter, ads, d.H, d.RP, (float *)ctx->d_t);
+    }
+    ProfScope prof(ctx, KK_PROJECT, s);
     dim3 grid((d.N + 63) / 64, (Tn + 63) / 64);
     linear_simt_kernel<T><<<grid, 256, 0, s>>>((const T *)hidden, (const T *)ctx->layers[layer].wqkv, Tn, d.H, d.N,
                                                ctx->d_row_adapter, ads, (const float *)ctx->d_t, d.RP, d.Nq, d.Nkv,
@@ -336,6 +343,7 @@ int launch_project_simt(alora_ctx *ctx, int layer, const void *hidden, int T, vo
 int launch_linear_simt(alora_ctx *ctx, const void *x, const void *W, int T, int K, int N, void *y,
                        const void *residual, cudaStream_t s) {
     if (T == 0) return 0;
+    ProfScope prof(ctx, KK_LINEAR, s);
     dim3 grid((N + 63) / 64, (T + 63) / 64);
     if (ctx->cfg.dtype == ALORA_DTYPE_FP32)
         linear_simt_kernel<float><<<grid, 256, 0, s>>>((const float *)x, (const float *)W, T, K, N, nullptr, nullptr,
@@ -351,6 +359,7 @@ template <typename T>
 static int attend_simt(alora_ctx *ctx, const void *qkv, const BatchArgs &b, const void *pool, void *out,
                        cudaStream_t s) {
     const Dims &d = ctx->d;
+    ProfScope prof(ctx, KK_ATTENTION, s);
     dim3 grid(b.T, d.Hkv);
     const int threads = 32 * d.G;
     const size_t smem = (size_t)d.G * d.hd * sizeof(float);
