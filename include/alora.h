@@ -253,6 +253,40 @@ int64_t alora_launch_count(const alora_ctx *ctx);
  * Families: 0 batch metadata, 1 rank-r shrink (t = A x), 2 q/k/v projection, 3 KV append,
  * 4 attention, 5 split-KV merge, 6 other dense projections (o_proj, MLP), 7 norm / activation glue.
  */
+/*
+ * Gated q/k/v projection (same result as alora_project_qkv in mode ALORA with one adapter) for
+ * callers that cannot allocate device memory.  (The paper has no counterpart: this is an
+ * integration aid.)  Typical callers: a plug-in running inside a serving engine that already owns
+ * all device memory through its own pool, or a latency-critical loop that must avoid the implicit
+ * synchronisation of cudaMalloc/cudaFree.  They cannot use alora_create, which allocates the
+ * context's workspaces, so this call needs no context and takes everything as arguments:
+ *   dtype, hidden (H), n_q (Nq), n_kv (Nkv)         layer shape, N = n_q + 2*n_kv
+ *   d_hidden[T][H], d_wqkv[N][H]                    inputs, device memory, element type = dtype
+ *   d_positions[T], d_query_start_loc[R+1], d_activation_offsets[R]   as for alora_project_qkv
+ *   d_adapter_on[R]                                 non-zero = request uses the adapter; NULL = all do
+ *   rank, scale, d_Aq/d_Ak/d_Av[rank][H], d_Bq[n_q][rank], d_Bk/d_Bv[n_kv][rank]   the adapter,
+ *                                                   read in place (nothing is copied or repacked)
+ *   d_qkv[T][N]                                     output
+ * It calls no cudaMalloc, cudaFree or allocating library routine.  Its scratch (one int32 gate per
+ * row and the fp32 intermediate s*A x) lives in a fixed array inside the library image of
+ * ALORA_STATIC_MAX_TOKENS * (4 + 12 * ALORA_STATIC_MAX_RANK) bytes (about 3 MiB), which every GPU
+ * that loads the library holds until the process exits.  T > ALORA_STATIC_MAX_TOKENS or
+ * rank > ALORA_STATIC_MAX_RANK returns ALORA_ERR_CAPACITY and launches nothing.
+ * The device that is current when the call is made is used.  The first call on a device looks up
+ * the array's device address (a set-up step); make that first call before any stream capture.
+ * All calls on a device share the array and it keeps the previous call's contents; each call
+ * rewrites whatever it reads, so no clearing is needed, but calls that overlap on the same GPU
+ * (different streams or host threads) race on it: serialise them.
+ */
+#define ALORA_STATIC_MAX_TOKENS 4096
+#define ALORA_STATIC_MAX_RANK 64
+alora_status alora_project_qkv_static(int dtype, int hidden, int n_q, int n_kv, const void *d_hidden,
+                                      const void *d_wqkv, const int32_t *d_positions,
+                                      const int32_t *d_query_start_loc, const int32_t *d_activation_offsets,
+                                      const int32_t *d_adapter_on, int rank, float scale, const void *d_Aq,
+                                      const void *d_Bq, const void *d_Ak, const void *d_Bk, const void *d_Av,
+                                      const void *d_Bv, int T, int R, void *d_qkv, void *stream);
+
 #define ALORA_PROFILE_KINDS 8
 alora_status alora_profile_enable(alora_ctx *ctx, int on);
 alora_status alora_profile_read(alora_ctx *ctx, double *ms_by_kind, int64_t *groups_by_kind);

@@ -257,3 +257,21 @@ def alora_profile_read(ctx) -> dict:
     n = (C.c_int64 * len(PROFILE_KINDS))()
     _check(ctx, load_library().alora_profile_read(ctx, ms, n), "alora_profile_read")
     return {k: (float(ms[i]), int(n[i])) for i, k in enumerate(PROFILE_KINDS)}
+
+
+STATIC_MAX_TOKENS, STATIC_MAX_RANK = 4096, 64
+
+
+def alora_project_qkv_static(dtype, hidden, n_q, n_kv, d_hidden, d_wqkv, positions, query_start_loc,
+                             activation_offsets, adapter_on, rank, scale, Aq, Bq, Ak, Bk, Av, Bv, T, R, qkv,
+                             stream=None) -> int:
+    """Context-free gated projection that allocates nothing (scratch is a fixed array in the library).
+    For callers that may not call cudaMalloc.  Returns the status code instead of raising, so that the
+    capacity errors can be inspected."""
+    lib = load_library()
+    f = lib.alora_project_qkv_static
+    f.argtypes = [_I] * 4 + [_VP] * 6 + [_I, C.c_float] + [_VP] * 6 + [_I, _I, _VP, _VP]
+    f.restype = C.c_int
+    return f(dtype, hidden, n_q, n_kv, _ptr(d_hidden), _ptr(d_wqkv), _ptr(positions), _ptr(query_start_loc),
+             _ptr(activation_offsets), _ptr(adapter_on), rank, scale, _ptr(Aq), _ptr(Bq), _ptr(Ak), _ptr(Bk),
+             _ptr(Av), _ptr(Bv), T, R, _ptr(qkv), _stream(stream))
