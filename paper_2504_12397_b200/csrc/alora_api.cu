@@ -17,11 +17,18 @@ int launch_project_simt(alora_ctx *, int, const void *, int, void *, cudaStream_
 int launch_linear_simt(alora_ctx *, const void *, const void *, int, int, int, void *, const void *, cudaStream_t);
 int launch_attend_simt(alora_ctx *, const void *, const BatchArgs &, const void *, void *, cudaStream_t);
 
+int launch_project_tc(alora_ctx *, int, const void *, int, void *, cudaStream_t);
+int launch_linear_tc(alora_ctx *, const void *, const void *, int, int, int, void *, const void *, cudaStream_t);
+bool build_layer_maps(alora_ctx *ctx, int layer);
+
+// bf16 runs on the tensor cores; the fp32 data type (tiny exact-precision configurations) on CUDA cores.
 int launch_project(alora_ctx *ctx, int layer, const void *hidden, int T, void *qkv, cudaStream_t s) {
+    if (ctx->cfg.dtype == ALORA_DTYPE_BF16) return launch_project_tc(ctx, layer, hidden, T, qkv, s);
     return launch_project_simt(ctx, layer, hidden, T, qkv, s);
 }
 int launch_linear(alora_ctx *ctx, const void *x, const void *W, int T, int K, int N, void *y,
                   const void *residual, cudaStream_t s) {
+    if (ctx->cfg.dtype == ALORA_DTYPE_BF16) return launch_linear_tc(ctx, x, W, T, K, N, y, residual, s);
     return launch_linear_simt(ctx, x, W, T, K, N, y, residual, s);
 }
 int launch_attend(alora_ctx *ctx, const void *qkv, const BatchArgs &b, const void *pool, void *out,
@@ -112,7 +119,9 @@ alora_status alora_create(const alora_config *cfg, alora_ctx **out) {
     Dims &d = ctx->d;
     d.H = c.hidden; d.Hq = c.n_q_heads; d.Hkv = c.n_kv_heads; d.hd = c.head_dim; d.G = d.Hq / d.Hkv;
     d.Nq = d.Hq * d.hd; d.Nkv = d.Hkv * d.hd; d.N = d.Nq + 2 * d.Nkv; d.page = c.page_size; d.I = c.intermediate;
-    d.RP = std::max(16, (c.max_rank + 15) / 16 * 16);
+    // adapters are stored rank-padded: to 64 columns on the tensor-core path (one 128-byte swizzle row),
+    // to the next multiple of 16 on the fp32 path
+    d.RP = c.dtype == ALORA_DTYPE_BF16 ? 64 : std::max(16, (c.max_rank + 15) / 16 * 16);
     d.softmax_scale = c.softmax_scale != 0.f ? c.softmax_scale : 1.0f / sqrtf((float)d.hd);
     ctx->layers.resize(c.n_layers);
     const size_t n_ad = (size_t)c.n_layers * std::max(1, c.max_adapters);
@@ -141,6 +150,24 @@ alora_status alora_create(const alora_config *cfg, alora_ctx **out) {
     alloc(&ctx->d_t, Tm * 3 * d.RP * 4);
     alloc(&ctx->d_qkv, Tm * d.N * es);
     alloc((void **)&ctx->d_status, 4);
+    ctx->layer_has_adapter.assign(c.n_layers, 0);
+    if (c.dtype == ALORA_DTYPE_BF16) {
+        const size_t na = (size_t)std::max(1, c.max_adapters);
+        ctx->tc_a_all.assign(c.n_layers, nullptr);
+        ctx->tc_b_all.assign(c.n_layers, nullptr);
+        ctx->tc_maps.resize(c.n_layers);
+        for (int l = 0; l < c.n_layers && st == ALORA_OK; ++l) {
+            const size_t bytesA = na * 3 * d.RP * d.H * es, bytesB = na * (size_t)d.N * d.RP * es;
+            alloc(&ctx->tc_a_all[l], bytesA);
+            alloc(&ctx->tc_b_all[l], bytesB);
+            if (st == ALORA_OK) {
+                cudaError_t e2 = cudaMemset(ctx->tc_a_all[l], 0, bytesA);
+                if (e2 == cudaSuccess) e2 = cudaMemset(ctx->tc_b_all[l], 0, bytesB);
+                if (e2 != cudaSuccess) st = cuda_fail(ctx, e2, "cudaMemset");
+                else if (!build_layer_maps(ctx, l)) st = ALORA_ERR_UNSUPPORTED;
+            }
+        }
+    }
     if (d.I > 0) {
         const size_t chunk = std::min<size_t>(Tm, kMlpChunk);
         alloc(&ctx->d_act[0], Tm * std::max(d.H, d.Nq) * es);  // normed input / attention output
@@ -167,6 +194,8 @@ alora_status alora_destroy(alora_ctx *ctx) {
     if (!ctx) return ALORA_ERR_INVALID_ARG;
     cudaSetDevice(ctx->cfg.device);
     for (void *p : ctx->adapter_storage) if (p) cudaFree(p);
+    for (void *p : ctx->tc_a_all) if (p) cudaFree(p);
+    for (void *p : ctx->tc_b_all) if (p) cudaFree(p);
     void *ptrs[] = {ctx->d_adapters, ctx->d_token_req, ctx->d_row_adapter, ctx->d_slot, ctx->d_tiles, ctx->d_counts,
                     ctx->d_seg_scratch, ctx->d_t, ctx->d_qkv, ctx->d_status, ctx->d_act[0], ctx->d_act[1],
                     ctx->d_act[2], ctx->d_act[3], ctx->d_iota};
@@ -186,6 +215,10 @@ alora_status alora_set_layer_weights(alora_ctx *ctx, int layer, const void *d_wq
     LayerWeights &lw = ctx->layers[layer];
     lw.wqkv = d_wqkv; lw.wo = d_wo; lw.wgate_up = d_wgate_up; lw.wdown = d_wdown;
     lw.norm_attn = d_norm_attn; lw.norm_mlp = d_norm_mlp;
+    if (ctx->cfg.dtype == ALORA_DTYPE_BF16) {
+        ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+        if (!build_layer_maps(ctx, layer)) return ALORA_ERR_UNSUPPORTED;
+    }
     return ALORA_OK;
 }
 
@@ -201,11 +234,19 @@ alora_status alora_register_adapter(alora_ctx *ctx, int adapter_id, int layer, i
     const Dims &d = ctx->d;
     const size_t idx = (size_t)layer * ctx->cfg.max_adapters + adapter_id;
     const size_t bytesA = (size_t)3 * d.RP * d.H * ctx->esize, bytesB = (size_t)d.N * d.RP * ctx->esize;
-    if (!ctx->adapter_storage[2 * idx]) {
-        ALORA_CUDA(ctx, cudaMalloc(&ctx->adapter_storage[2 * idx], bytesA));
-        ALORA_CUDA(ctx, cudaMalloc(&ctx->adapter_storage[2 * idx + 1], bytesB));
+    void *A, *B;
+    if (ctx->cfg.dtype == ALORA_DTYPE_BF16) {
+        // one slab per layer holds every adapter's rows, so that one tensor map addresses them all
+        A = (char *)ctx->tc_a_all[layer] + (size_t)adapter_id * bytesA;
+        B = (char *)ctx->tc_b_all[layer] + (size_t)adapter_id * bytesB;
+    } else {
+        if (!ctx->adapter_storage[2 * idx]) {
+            ALORA_CUDA(ctx, cudaMalloc(&ctx->adapter_storage[2 * idx], bytesA));
+            ALORA_CUDA(ctx, cudaMalloc(&ctx->adapter_storage[2 * idx + 1], bytesB));
+        }
+        A = ctx->adapter_storage[2 * idx]; B = ctx->adapter_storage[2 * idx + 1];
     }
-    void *A = ctx->adapter_storage[2 * idx], *B = ctx->adapter_storage[2 * idx + 1];
+    ctx->layer_has_adapter[layer] = 1;
     int n = launch_repack_adapter(ctx, rank, d_Aq, d_Bq, d_Ak, d_Bk, d_Av, d_Bv, A, B, s);
     AdapterDev rec{A, B, rank, (rank + 15) / 16 * 16, scale, 0};
     ctx->h_adapters[idx] = rec;

@@ -1,6 +1,7 @@
 // Internal declarations shared by the library's translation units (not part of the C ABI).
 #pragma once
 
+#include <cuda.h>
 #include <cuda_bf16.h>
 #include <cuda_runtime.h>
 #include <stdint.h>
@@ -64,6 +65,14 @@ struct ProfEvent {
     int kind;
 };
 
+// Tensor maps of one layer that depend only on registered weights (bf16 tensor-core path).
+struct TcLayerMaps {
+    CUtensorMap wqkv[2];      // W_qkv [N][H], boxes of 128 / 256 rows
+    CUtensorMap a_all;        // all adapters' A rows [max_adapters*192][H], box 192 rows
+    CUtensorMap b_all;        // unused placeholder with the same geometry as b_all_bn (shrink launches)
+    CUtensorMap b_all_bn[2];  // all adapters' B rows [max_adapters*N][64], boxes of 128 / 256 rows
+};
+
 struct Dims {
     int H, Hq, Hkv, hd, G, Nq, Nkv, N, page, I, RP;  // RP = padded max rank
     float softmax_scale;
@@ -79,6 +88,11 @@ struct alora_ctx {
     std::vector<alora::AdapterDev> h_adapters;  // [layer * max_adapters + id], mirrors d_adapters
     alora::AdapterDev *d_adapters = nullptr;
     std::vector<void *> adapter_storage;         // context-owned A/B buffers, same indexing, 2 per entry
+
+    // bf16 tensor-core path: per-layer adapter storage shared by all adapters of the layer
+    std::vector<void *> tc_a_all, tc_b_all;          // [layer] -> [max_adapters][3*64][H], [max_adapters][N][64]
+    std::vector<alora::TcLayerMaps> tc_maps;         // [layer]
+    std::vector<char> layer_has_adapter;             // [layer] any adapter registered
 
     // per-call workspaces
     int32_t *d_token_req = nullptr, *d_row_adapter = nullptr, *d_slot = nullptr;

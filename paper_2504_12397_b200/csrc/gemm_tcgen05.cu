@@ -1,0 +1,384 @@
+// bf16 dense contraction on the 5th-generation tensor cores: out[rows][N] = act[rows][K] . W[N][K]^T
+// with the aLoRA delta fused in.
+//
+// One persistent block per SM, three roles:
+//   warp 0 (one lane)  TMA producer: streams 128 x 64 activation tiles and BN x 64 weight tiles
+//                      (128-byte swizzle) through a 4-deep shared-memory ring;
+//   warp 1 (one lane)  MMA issuer: tcgen05.mma 128 x BN x 16 steps into one of two fp32 accumulators in
+//                      tensor memory, releasing ring slots and publishing accumulators via
+//                      tcgen05.commit;
+//   warps 2-5          epilogue: tcgen05.ld the accumulator (one row per thread), optional residual
+//                      add / scale, round to bf16, 16-byte row-predicated stores.  The second
+//                      accumulator lets the next tile's main loop overlap this epilogue.
+//
+// Row tiles come from the batch-metadata step: all rows of a tile have the same applied adapter.
+// For a tile with an adapter the main K loop (the base term W x of Eq. 5) is followed by one more
+// K block whose operands are t = s A x (rows of the tile) and the adapter's B rows of this column
+// tile, i.e. the delta s B (A x) is accumulated by the same tensor-core instruction stream.  Tiles
+// without an adapter execute exactly the base-only sequence: that is what makes gated-off rows
+// bit-identical to a base-only call (Prop. 1).  The same kernel in "shrink" mode computes
+// t = s A x for the adapter tiles.  No split-K, no atomics: results are run-to-run deterministic.
+//
+// Every wait is bounded (tc::mbar_wait); on expiry the block records ALORA_ERR_TIMEOUT, drains its
+// outstanding copies and tensor-core work with bounded waits, frees its tensor memory and returns.
+#include "alora_internal.h"
+#include "tc_common.cuh"
+
+namespace alora {
+
+constexpr int kBM = 128;      // rows per tile (UMMA M)
+constexpr int kBK = 64;       // K elements per ring slot (one 128-byte swizzle row)
+constexpr int kStages = 4;
+constexpr int kGemmThreads = 192;
+constexpr int kTensorRP = 64; // the tensor path stores adapters padded to 64 rank columns
+
+struct GemmArgs {
+    const ProjTile *tiles;        // nullptr: dense row tiles 0..ceil(M/128)-1, no adapters
+    const int32_t *n_row_tiles;   // device count of `tiles` entries (when tiles != nullptr)
+    int M, N, K;
+    __nv_bfloat16 *out;
+    int ldo;
+    const __nv_bfloat16 *residual;  // optional, same layout as out, may alias it
+    const AdapterDev *adapters;     // this layer's adapter table (expand / shrink), or nullptr
+    int shrink;                     // 1: out = t, B operand = the tile adapter's A rows, scaled by s
+    int Nq, Nkv;                    // block boundaries of the fused output row (expand)
+    int total_adapter_rows;         // rows per adapter in the B_all map (= N of the layer)
+    int32_t *status;
+};
+
+template <int BN>
+struct GemmSmem {
+    static constexpr int kABytes = kBM * kBK * 2;
+    static constexpr int kBBytes = BN * kBK * 2;
+    static constexpr int kStageBytes = kABytes + kBBytes;
+    static constexpr int kBarOffset = kStages * kStageBytes;
+    static constexpr int kTotal = kBarOffset + 256 + 1024;  // barriers + slack for 1024-byte alignment
+};
+
+__device__ __forceinline__ ProjTile load_tile(const GemmArgs &a, int m) {
+    if (a.tiles) return a.tiles[m];
+    ProjTile t;
+    t.row_start = m * kBM;
+    t.row_count = min(kBM, a.M - m * kBM);
+    t.adapter = -1;
+    t.pad_ = 0;
+    return t;
+}
+
+template <int BN>
+__global__ void __launch_bounds__(kGemmThreads, 1)
+gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
+                    const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUtensorMap tmL,
+                    const GemmArgs a) {
+    using S = GemmSmem<BN>;
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t smem_base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t *smem_al = smem_raw + (smem_base - tc::smem_u32(smem_raw));
+    uint64_t *bars = reinterpret_cast<uint64_t *>(smem_al + S::kBarOffset);
+    // barrier words: full[kStages], empty[kStages], acc_full[2], acc_empty[2], drain
+    const uint32_t bar0 = smem_base + S::kBarOffset;
+    auto full_bar = [&](int s) { return bar0 + 8u * s; };
+    auto empty_bar = [&](int s) { return bar0 + 8u * (kStages + s); };
+    auto accf_bar = [&](int i) { return bar0 + 8u * (2 * kStages + i); };
+    auto acce_bar = [&](int i) { return bar0 + 8u * (2 * kStages + 2 + i); };
+    const uint32_t drain_bar = bar0 + 8u * (2 * kStages + 4);
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(bars + 2 * kStages + 5);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 2 * kStages + 6);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    constexpr uint32_t kTmemCols = (2 * BN <= 256) ? 256 : 512;
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < kStages; ++s) { tc::mbar_init(full_bar(s), 1); tc::mbar_init(empty_bar(s), 1); }
+        for (int i = 0; i < 2; ++i) { tc::mbar_init(accf_bar(i), 1); tc::mbar_init(acce_bar(i), 4); }
+        tc::mbar_init(drain_bar, 1);
+        *abort_flag = 0;
+        tc::fence_barrier_init();
+        tc::fence_proxy_async();
+    }
+    if (warp == 1) tc::tmem_alloc(tc::smem_u32((const void *)tmem_slot), kTmemCols);
+    tc::tc_fence_before();
+    __syncthreads();
+    tc::tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+
+    const int n_m = a.tiles ? *a.n_row_tiles : (a.M + kBM - 1) / kBM;
+    const int n_n = (a.N + BN - 1) / BN;
+    const int total = n_m * n_n;
+    const int kb_main = (a.K + kBK - 1) / kBK;
+
+    if (warp == 0) {
+        if (lane == 0) {
+            // ------------------------------ TMA producer ------------------------------
+            tc::tma_prefetch_desc(&tmA); tc::tma_prefetch_desc(&tmB);
+            uint32_t kc = 0;        // ring slots filled so far
+            bool ok = true;
+            for (int item = blockIdx.x; item < total && ok; item += gridDim.x) {
+                const int m = item / n_n, n0 = (item % n_n) * BN;
+                const ProjTile t = load_tile(a, m);
+                if (a.shrink && t.adapter < 0) continue;
+                const int extra = (!a.shrink && t.adapter >= 0) ? 1 : 0;
+                const int b_row0 = a.shrink ? t.adapter * BN : n0;
+                for (int kb = 0; kb < kb_main + extra; ++kb, ++kc) {
+                    const int s = kc % kStages;
+                    if (!tc::mbar_wait(empty_bar(s), ((kc / kStages) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                    const uint32_t sa = smem_base + s * S::kStageBytes, sb = sa + S::kABytes;
+                    tc::mbar_arrive_expect_tx(full_bar(s), S::kStageBytes);
+                    if (kb < kb_main) {
+                        tc::tma_load_2d(sa, &tmA, full_bar(s), kb * kBK, t.row_start);
+                        tc::tma_load_2d(sb, &tmB, full_bar(s), kb * kBK, b_row0);
+                    } else {
+                        const int blk = n0 < a.Nq ? 0 : (n0 < a.Nq + a.Nkv ? 1 : 2);
+                        tc::tma_load_2d(sa, &tmT, full_bar(s), blk * kTensorRP, t.row_start);
+                        tc::tma_load_2d(sb, &tmL, full_bar(s), 0, t.adapter * a.total_adapter_rows + n0);
+                    }
+                }
+            }
+            if (!ok) {
+                // give copies already in flight time to land before the block's shared memory is released
+                const uint32_t first = kc > (uint32_t)kStages ? kc - kStages : 0;
+                for (uint32_t i = first; i < kc; ++i) {
+                    const long long t0 = clock64();
+                    while (!tc::mbar_try_wait(full_bar(i % kStages), (i / kStages) & 1) &&
+                           clock64() - t0 < tc::kWaitCycleLimit) {}
+                }
+            }
+        }
+    } else if (warp == 1) {
+        if (lane == 0) {
+            // ------------------------------ MMA issuer ------------------------------
+            constexpr uint32_t idesc = tc::idesc_bf16_f32(kBM, BN);
+            uint32_t kc = 0, it = 0;
+            bool ok = true;
+            for (int item = blockIdx.x; item < total && ok; item += gridDim.x) {
+                const int m = item / n_n;
+                const ProjTile t = load_tile(a, m);
+                if (a.shrink && t.adapter < 0) continue;
+                const int extra = (!a.shrink && t.adapter >= 0) ? 1 : 0;
+                const int extra_steps = extra ? a.adapters[t.adapter].rpad / 16 : 0;
+                const uint32_t acc = it & 1;
+                if (!tc::mbar_wait(acce_bar(acc), ((it >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                tc::tc_fence_after();
+                const uint32_t d_tmem = tmem_base + acc * BN;
+                for (int kb = 0; kb < kb_main + extra; ++kb, ++kc) {
+                    const int s = kc % kStages;
+                    if (!tc::mbar_wait(full_bar(s), (kc / kStages) & 1, abort_flag)) { ok = false; break; }
+                    tc::tc_fence_after();
+                    const uint32_t sa = smem_base + s * S::kStageBytes, sb = sa + S::kABytes;
+                    const uint64_t da = tc::smem_desc_k_sw128(sa), db = tc::smem_desc_k_sw128(sb);
+                    const int steps = kb < kb_main ? kBK / 16 : extra_steps;
+                    for (int k = 0; k < steps; ++k)
+                        tc::mma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                    tc::mma_commit(empty_bar(s));  // slot reusable once these MMAs have read it
+                }
+                if (!ok) break;
+                tc::mma_commit(accf_bar(acc));      // accumulator complete
+                ++it;
+            }
+            if (!ok) {
+                tc::mma_commit(drain_bar);          // wait (bounded) for tensor-core work still in flight
+                const long long t0 = clock64();
+                while (!tc::mbar_try_wait(drain_bar, 0) && clock64() - t0 < tc::kWaitCycleLimit) {}
+            }
+        }
+    } else {
+        // ------------------------------ epilogue (warps 2..5) ------------------------------
+        const int q = warp & 3;  // tensor-memory lane quarter this warp may read
+        uint32_t it = 0;
+        bool ok = true;
+        for (int item = blockIdx.x; item < total && ok; item += gridDim.x) {
+            const int m = item / n_n, n0 = (item % n_n) * BN;
+            const ProjTile t = load_tile(a, m);
+            if (a.shrink && t.adapter < 0) continue;
+            const uint32_t acc = it & 1;
+            if (!tc::mbar_wait(accf_bar(acc), (it >> 1) & 1, abort_flag)) { ok = false; break; }
+            tc::tc_fence_after();
+            const int r = q * 32 + lane;
+            const bool row_ok = r < t.row_count;
+            const float scale = a.shrink ? a.adapters[t.adapter].scale : 1.f;
+            __nv_bfloat16 *orow = a.out + (size_t)(t.row_start + r) * a.ldo + n0;
+            const __nv_bfloat16 *rrow = a.residual ? a.residual + (size_t)(t.row_start + r) * a.ldo + n0 : nullptr;
+#pragma unroll 1
+            for (int c = 0; c < BN; c += 32) {
+                uint32_t v[32];
+                tc::tmem_ld_32x32(tmem_base + acc * BN + c + ((uint32_t)(q * 32) << 16), v);
+                tc::tmem_ld_wait();
+                if (row_ok) {
+#pragma unroll
+                    for (int j = 0; j < 4; ++j) {
+                        if (n0 + c + 8 * j >= a.N) break;
+                        float f[8];
+#pragma unroll
+                        for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[8 * j + e]) * scale;
+                        if (rrow) {
+                            const uint4 rv = *reinterpret_cast<const uint4 *>(rrow + c + 8 * j);
+                            const uint32_t rw[4] = {rv.x, rv.y, rv.z, rv.w};
+#pragma unroll
+                            for (int e = 0; e < 4; ++e) {
+                                const __nv_bfloat162 b2 = *reinterpret_cast<const __nv_bfloat162 *>(&rw[e]);
+                                f[2 * e] += __low2float(b2);
+                                f[2 * e + 1] += __high2float(b2);
+                            }
+                        }
+                        uint4 o;
+                        o.x = tc::pack_bf16(f[0], f[1]); o.y = tc::pack_bf16(f[2], f[3]);
+                        o.z = tc::pack_bf16(f[4], f[5]); o.w = tc::pack_bf16(f[6], f[7]);
+                        *reinterpret_cast<uint4 *>(orow + c + 8 * j) = o;
+                    }
+                }
+            }
+            tc::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(acce_bar(acc));  // accumulator may be overwritten
+            ++it;
+        }
+    }
+
+    tc::tc_fence_before();
+    __syncthreads();
+    if (threadIdx.x == 0 && *abort_flag) report(a.status, ALORA_ERR_TIMEOUT);
+    if (warp == 1) {
+        tc::tc_fence_after();
+        tc::tmem_dealloc(tmem_base, kTmemCols);
+    }
+}
+
+// ---- host side -------------------------------------------------------------------------------------
+
+typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
+                                  const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+static EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    if (!fn) {
+        void *p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = (EncodeTiledFn)p;
+    }
+    return fn;
+}
+
+// Row-major bf16 matrix [rows][cols] (row pitch ld elements) viewed in boxes of 64 columns x box_rows
+// rows, 128-byte swizzle, out-of-range elements read as zero.
+bool make_tensor_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint64_t ld,
+                          uint32_t box_rows) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn || !base || rows == 0 || cols == 0) return false;
+    if ((reinterpret_cast<uintptr_t>(base) & 15u) || (ld * 2) % 16 != 0 || box_rows == 0 || box_rows > 256) return false;
+    cuuint64_t dims[2] = {cols, rows};
+    cuuint64_t strides[1] = {ld * 2};
+    cuuint32_t box[2] = {(cuuint32_t)kBK, box_rows};
+    cuuint32_t estr[2] = {1, 1};
+    return fn(map, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(base), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+template <int BN>
+static bool launch_gemm_bn(alora_ctx *ctx, const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtensorMap &tmT,
+                           const CUtensorMap &tmL, const GemmArgs &args, int max_items, cudaStream_t s) {
+    static bool attr_set[64] = {};
+    const int dev = ctx->cfg.device;
+    if (dev >= 0 && dev < 64 && !attr_set[dev]) {
+        if (cudaFuncSetAttribute(gemm_tcgen05_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                 GemmSmem<BN>::kTotal) != cudaSuccess)
+            return false;
+        attr_set[dev] = true;
+    }
+    const int grid = std::max(1, std::min(ctx->sm_count, max_items));
+    gemm_tcgen05_kernel<BN><<<grid, kGemmThreads, GemmSmem<BN>::kTotal, s>>>(tmA, tmB, tmT, tmL, args);
+    return true;
+}
+
+// Picks the column-tile width: 256 when the q/k/v block boundaries allow it, else 128.
+static int pick_bn(int N, int Nq, int Nkv, bool lora) {
+    if (lora) {
+        if (Nq % 256 == 0 && Nkv % 256 == 0) return 256;
+        if (Nq % 128 == 0 && Nkv % 128 == 0) return 128;
+        return 0;
+    }
+    return (N % 256 == 0 || N > 1024) ? 256 : 128;
+}
+
+// q/k/v projection of one layer on the tensor cores: shrink (t = s A x on adapter tiles), then the
+// base GEMM with the expand step fused.  Returns kernels launched, or -1 when the shape is unsupported.
+int launch_project_tc(alora_ctx *ctx, int layer, const void *hidden, int T, void *qkv, cudaStream_t s) {
+    if (T == 0) return 0;
+    const Dims &d = ctx->d;
+    const bool have_adapters = ctx->layer_has_adapter[layer];
+    const int BN = pick_bn(d.N, d.Nq, d.Nkv, true);
+    if (BN == 0 || d.H % 8 != 0) return -1;
+    CUtensorMap tmX, tmTt;
+    if (!make_tensor_map_bf16(&tmX, hidden, T, d.H, d.H, kBM)) return -1;
+    if (!make_tensor_map_bf16(&tmTt, ctx->d_t, ctx->cfg.max_tokens, 3 * kTensorRP, 3 * kTensorRP, kBM)) return -1;
+    const TcLayerMaps &lm = ctx->tc_maps[layer];
+    const AdapterDev *ads = ctx->d_adapters + (size_t)layer * ctx->cfg.max_adapters;
+    const int max_row_tiles = ctx->max_tiles < (T / kBM + 2 * ctx->cfg.max_requests + 2)
+                                  ? ctx->max_tiles : (T / kBM + 2 * ctx->cfg.max_requests + 2);
+    int n = 0;
+    if (have_adapters) {
+        ProfScope prof(ctx, KK_SHRINK, s);
+        GemmArgs g{};
+        g.tiles = ctx->d_tiles; g.n_row_tiles = ctx->d_counts; g.M = T; g.N = 3 * kTensorRP; g.K = d.H;
+        g.out = (__nv_bfloat16 *)ctx->d_t; g.ldo = 3 * kTensorRP; g.residual = nullptr; g.adapters = ads;
+        g.shrink = 1; g.Nq = d.Nq; g.Nkv = d.Nkv; g.total_adapter_rows = d.N; g.status = ctx->d_status;
+        if (!launch_gemm_bn<3 * kTensorRP>(ctx, tmX, lm.a_all, tmTt, lm.b_all, g, max_row_tiles, s)) return -1;
+        ++n;
+    }
+    {
+        ProfScope prof(ctx, KK_PROJECT, s);
+        GemmArgs g{};
+        g.tiles = ctx->d_tiles; g.n_row_tiles = ctx->d_counts; g.M = T; g.N = d.N; g.K = d.H;
+        g.out = (__nv_bfloat16 *)qkv; g.ldo = d.N; g.residual = nullptr; g.adapters = ads; g.shrink = 0;
+        g.Nq = d.Nq; g.Nkv = d.Nkv; g.total_adapter_rows = d.N; g.status = ctx->d_status;
+        const int items = max_row_tiles * ((d.N + BN - 1) / BN);
+        const bool ok = BN == 256 ? launch_gemm_bn<256>(ctx, tmX, lm.wqkv[1], tmTt, lm.b_all_bn[1], g, items, s)
+                                  : launch_gemm_bn<128>(ctx, tmX, lm.wqkv[0], tmTt, lm.b_all_bn[0], g, items, s);
+        if (!ok) return -1;
+        ++n;
+    }
+    return n;
+}
+
+// Plain dense projection y = x W^T (+ residual) for o_proj and the MLP matrices.
+int launch_linear_tc(alora_ctx *ctx, const void *x, const void *W, int T, int K, int N, void *y,
+                     const void *residual, cudaStream_t s) {
+    if (T == 0) return 0;
+    if (K % 8 != 0 || N % 8 != 0) return -1;
+    ProfScope prof(ctx, KK_LINEAR, s);
+    const int BN = pick_bn(N, 0, 0, false);
+    CUtensorMap tmX, tmW;
+    if (!make_tensor_map_bf16(&tmX, x, T, K, K, kBM)) return -1;
+    if (!make_tensor_map_bf16(&tmW, W, N, K, K, BN)) return -1;
+    GemmArgs g{};
+    g.tiles = nullptr; g.n_row_tiles = nullptr; g.M = T; g.N = N; g.K = K; g.out = (__nv_bfloat16 *)y; g.ldo = N;
+    g.residual = (const __nv_bfloat16 *)residual; g.adapters = nullptr; g.shrink = 0; g.Nq = N; g.Nkv = 0;
+    g.total_adapter_rows = 0; g.status = ctx->d_status;
+    const int items = ((T + kBM - 1) / kBM) * ((N + BN - 1) / BN);
+    const bool ok = BN == 256 ? launch_gemm_bn<256>(ctx, tmX, tmW, tmX, tmW, g, items, s)
+                              : launch_gemm_bn<128>(ctx, tmX, tmW, tmX, tmW, g, items, s);
+    return ok ? 1 : -1;
+}
+
+// Tensor maps that depend only on registered weights; (re)built when weights or adapters are set.
+bool build_layer_maps(alora_ctx *ctx, int layer) {
+    const Dims &d = ctx->d;
+    TcLayerMaps &lm = ctx->tc_maps[layer];
+    const LayerWeights &lw = ctx->layers[layer];
+    bool ok = true;
+    if (lw.wqkv) {
+        ok &= make_tensor_map_bf16(&lm.wqkv[0], lw.wqkv, d.N, d.H, d.H, 128);
+        ok &= make_tensor_map_bf16(&lm.wqkv[1], lw.wqkv, d.N, d.H, d.H, 256);
+    }
+    const size_t na = (size_t)std::max(1, ctx->cfg.max_adapters);
+    ok &= make_tensor_map_bf16(&lm.a_all, ctx->tc_a_all[layer], na * 3 * kTensorRP, d.H, d.H, 3 * kTensorRP);
+    ok &= make_tensor_map_bf16(&lm.b_all, ctx->tc_b_all[layer], na * d.N, kTensorRP, kTensorRP, 3 * kTensorRP);
+    ok &= make_tensor_map_bf16(&lm.b_all_bn[0], ctx->tc_b_all[layer], na * d.N, kTensorRP, kTensorRP, 128);
+    ok &= make_tensor_map_bf16(&lm.b_all_bn[1], ctx->tc_b_all[layer], na * d.N, kTensorRP, kTensorRP, 256);
+    return ok;
+}
+
+}  // namespace alora
