@@ -20,6 +20,7 @@ int launch_attend_simt(alora_ctx *, const void *, const BatchArgs &, const void 
 int launch_project_tc(alora_ctx *, int, const void *, int, void *, cudaStream_t);
 int launch_linear_tc(alora_ctx *, const void *, const void *, int, int, int, void *, const void *, cudaStream_t);
 bool build_layer_maps(alora_ctx *ctx, int layer);
+int launch_attend_tc(alora_ctx *, const void *, const BatchArgs &, const void *, void *, cudaStream_t);
 
 // bf16 runs on the tensor cores; the fp32 data type (tiny exact-precision configurations) on CUDA cores.
 int launch_project(alora_ctx *ctx, int layer, const void *hidden, int T, void *qkv, cudaStream_t s) {
@@ -33,6 +34,7 @@ int launch_linear(alora_ctx *ctx, const void *x, const void *W, int T, int K, in
 }
 int launch_attend(alora_ctx *ctx, const void *qkv, const BatchArgs &b, const void *pool, void *out,
                   cudaStream_t s) {
+    if (ctx->cfg.dtype == ALORA_DTYPE_BF16) return launch_attend_tc(ctx, qkv, b, pool, out, s);
     return launch_attend_simt(ctx, qkv, b, pool, out, s);
 }
 
@@ -151,6 +153,13 @@ alora_status alora_create(const alora_config *cfg, alora_ctx **out) {
     alloc(&ctx->d_qkv, Tm * d.N * es);
     alloc((void **)&ctx->d_status, 4);
     ctx->layer_has_adapter.assign(c.n_layers, 0);
+    if (c.dtype == ALORA_DTYPE_BF16 && 128 % d.G == 0) {
+        // tensor-core attention: one work item per (request, KV head, block of 2 * 128/G tokens)
+        ctx->attn_q_block = 2 * (128 / d.G);
+        ctx->max_attn_items = (int)((Tm / ctx->attn_q_block + (size_t)c.max_requests) * d.Hkv);
+        alloc((void **)&ctx->d_attn_items, (size_t)ctx->max_attn_items * sizeof(AttnWork));
+        alloc((void **)&ctx->d_attn_off, ((size_t)c.max_requests + 1) * 4);
+    }
     if (c.dtype == ALORA_DTYPE_BF16) {
         const size_t na = (size_t)std::max(1, c.max_adapters);
         ctx->tc_a_all.assign(c.n_layers, nullptr);
@@ -198,7 +207,7 @@ alora_status alora_destroy(alora_ctx *ctx) {
     for (void *p : ctx->tc_b_all) if (p) cudaFree(p);
     void *ptrs[] = {ctx->d_adapters, ctx->d_token_req, ctx->d_row_adapter, ctx->d_slot, ctx->d_tiles, ctx->d_counts,
                     ctx->d_seg_scratch, ctx->d_t, ctx->d_qkv, ctx->d_status, ctx->d_act[0], ctx->d_act[1],
-                    ctx->d_act[2], ctx->d_act[3], ctx->d_iota};
+                    ctx->d_act[2], ctx->d_act[3], ctx->d_iota, ctx->d_attn_items, ctx->d_attn_off};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (ctx->h_status) cudaFreeHost(ctx->h_status);
     for (ProfEvent &e : ctx->prof_events) { if (e.begin) cudaEventDestroy(e.begin); if (e.end) cudaEventDestroy(e.end); }

@@ -101,6 +101,9 @@ struct alora_ctx {
     int32_t *d_seg_scratch = nullptr;  // [4][2*max_requests+1] merged row runs of the current batch
     int32_t *d_iota = nullptr;         // 0..max_requests: query_start_loc of a decode batch
     int32_t max_tiles = 0;
+    alora::AttnWork *d_attn_items = nullptr;  // tensor-core attention work list (bf16)
+    int32_t *d_attn_off = nullptr;            // [max_requests+1] block offsets per request
+    int32_t max_attn_items = 0, attn_q_block = 0;
     void *d_t = nullptr;          // [max_tokens][3][RP] rank-r intermediate
     void *d_qkv = nullptr;        // [max_tokens][N]
     void *d_act[4] = {nullptr, nullptr, nullptr, nullptr};  // stack activations

@@ -249,7 +249,7 @@ typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
                                   CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
 
-static EncodeTiledFn encode_fn() {
+EncodeTiledFn tensor_map_encoder() {
     static EncodeTiledFn fn = nullptr;
     if (!fn) {
         void *p = nullptr;
@@ -265,7 +265,7 @@ static EncodeTiledFn encode_fn() {
 // rows, 128-byte swizzle, out-of-range elements read as zero.
 bool make_tensor_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uint64_t cols, uint64_t ld,
                           uint32_t box_rows) {
-    EncodeTiledFn fn = encode_fn();
+    EncodeTiledFn fn = tensor_map_encoder();
     if (!fn || !base || rows == 0 || cols == 0) return false;
     if ((reinterpret_cast<uintptr_t>(base) & 15u) || (ld * 2) % 16 != 0 || box_rows == 0 || box_rows > 256) return false;
     cuuint64_t dims[2] = {cols, rows};

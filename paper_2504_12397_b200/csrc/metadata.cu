@@ -127,6 +127,53 @@ __global__ void metadata_tiles_kernel(const int32_t *__restrict__ a_req, const i
     }
 }
 
+// Attention work items of a prefill batch: each request's new tokens are cut into blocks of
+// `q_block` tokens; one item per (request, KV head, block), blocks of the same KV stream adjacent so
+// that blocks running at the same time share their K/V pages in L2.  Keys 0 .. position of the
+// block's last token are visible to the block (causal limit); per-row limits are applied in the kernel.
+__global__ void metadata_attn_items_kernel(const int32_t *__restrict__ qsl, const int32_t *__restrict__ seq_lens,
+                                           int R, int Hkv, int q_block, int max_items,
+                                           AttnWork *__restrict__ items, int32_t *__restrict__ counts,
+                                           int32_t *__restrict__ blk_off /* [R+1] */, int32_t *status) {
+    __shared__ int total;
+    if (threadIdx.x == 0) {
+        int acc = 0;
+        for (int r = 0; r < R; ++r) {
+            blk_off[r] = acc;
+            const int n_new = qsl[r + 1] - qsl[r];
+            acc += n_new > 0 ? (n_new + q_block - 1) / q_block : 0;
+        }
+        blk_off[R] = acc;
+        int n = acc * Hkv;
+        if (n > max_items) { report(status, ALORA_ERR_CAPACITY); n = 0; }
+        total = n;
+        counts[1] = n;
+    }
+    __syncthreads();
+    for (int i = threadIdx.x; i < total; i += blockDim.x) {
+        int lo = 0, hi = R;      // blk_off[lo] * Hkv <= i < blk_off[hi] * Hkv
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (blk_off[mid] * Hkv <= i) lo = mid; else hi = mid;
+        }
+        const int r = lo;
+        const int nblk = blk_off[r + 1] - blk_off[r];
+        const int rem = i - blk_off[r] * Hkv;
+        const int kvh = rem / nblk, blk = rem % nblk;
+        const int n_new = qsl[r + 1] - qsl[r];
+        AttnWork w;
+        w.req = r;
+        w.q_start = qsl[r] + blk * q_block;
+        w.q_count = min(q_block, n_new - blk * q_block);
+        w.kv_head = kvh;
+        w.kv_start = 0;
+        w.kv_end = seq_lens[r] - n_new + blk * q_block + w.q_count;  // last token's position + 1
+        w.split = 0;
+        w.n_splits = 1;
+        items[i] = w;
+    }
+}
+
 int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s) {
     if (b.T == 0) {
         cudaMemsetAsync(ctx->d_counts, 0, 2 * sizeof(int32_t), s);
@@ -141,7 +188,11 @@ int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s) {
     metadata_tiles_kernel<<<1, 256, 0, s>>>(b.activation_offsets, b.adapter_ids, b.query_start_loc,
                                            b.seq_lens, b.R, b.mode, ctx->cfg.max_adapters, ctx->max_tiles,
                                            ctx->d_tiles, ctx->d_counts, ctx->d_seg_scratch, ctx->d_status);
-    return 2;
+    if (ctx->d_attn_items == nullptr || b.block_tables == nullptr) return 2;
+    metadata_attn_items_kernel<<<1, 256, 0, s>>>(b.query_start_loc, b.seq_lens, b.R, ctx->d.Hkv, ctx->attn_q_block,
+                                                ctx->max_attn_items, ctx->d_attn_items, ctx->d_counts,
+                                                ctx->d_attn_off, ctx->d_status);
+    return 3;
 }
 
 }  // namespace alora
