@@ -11,8 +11,9 @@
 //            read from tensor memory (it overwrites S_w in bf16) and V consumed in place (MN-major);
 //   warps 0-3, 4-7   softmax groups w = 0, 1, one thread per score row: running maximum and sum
 //            (online softmax; a thread owns its whole row, so the row reductions need no
-//            cross-lane traffic), P_w written back to tensor memory, the PV_w products of the
-//            previous tile folded into fp32 output registers, final normalisation and store.
+//            cross-lane traffic), P_w written back to tensor memory; the output O_w accumulates in
+//            tensor memory across tiles and is rescaled only when a row's maximum has moved by more
+//            than 2^8 since the exponent reference was last set; final normalisation and store.
 // While one group does its exponentials the tensor pipe works for the other group.
 //
 // Masking: key j is visible to a row at position p iff j <= p; masked probabilities are set to
@@ -81,6 +82,17 @@ __device__ __forceinline__ void tmem_st_32x16(uint32_t taddr, const uint32_t (&r
           "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15])
         : "memory");
 }
+__device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&r)[32]) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], "
+        "{%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]),
+          "r"(r[8]), "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]),
+          "r"(r[16]), "r"(r[17]), "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]),
+          "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ void tma_load_3d(uint32_t smem_dst, const CUtensorMap *map, uint32_t bar, int c0, int c1,
@@ -139,7 +151,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    // tensor-memory columns: S_w / P_w at w*128, PV_w at 256 + w*128
+    // tensor-memory columns: S_w / P_w at w*128, O_w at 256 + w*128
     const int n_items = *a.n_items;
     const int tok_per_group = 128 / a.G;
     const int pages_per_tile = kKeysPerTile / a.page_size;
@@ -233,7 +245,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         const uint32_t va = smem_base + S::kVOff + st * S::kKvBytes;
                         for (int k = 0; k < kKeysPerTile / 16; ++k)  // 16 keys per step: 8 packed columns of P
                             mma_bf16_ts(tmem_base + 256 + g * 128, tmem_base + g * 128 + 8 * k,
-                                        smem_desc_mn_sw128(va + k * 2048, kHalfQ), idesc_pv, k != 0 ? 1u : 0u);
+                                        smem_desc_mn_sw128(va + k * 2048, kHalfQ), idesc_pv, (j | k) != 0 ? 1u : 0u);
                         tc::mma_commit(pv_done(g));
                         if (g == 1) tc::mma_commit(v_free(st));
                         if (more) {
@@ -261,8 +273,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const int row = q * 32 + lane;           // score row of this thread inside the group's tile
         const uint32_t lane_off = (uint32_t)(q * 32) << 16;
         const uint32_t s_addr = tmem_base + g * 128 + lane_off;
-        const uint32_t pv_addr = tmem_base + 256 + g * 128 + lane_off;
-        uint32_t n_s = 0, n_pv = 0, kt = 0;
+        const uint32_t o_addr = tmem_base + 256 + g * 128 + lane_off;
+        uint32_t n_s = 0, kt = 0;
         bool ok = true;
         for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
             const AttnWork w = a.items[it];
@@ -271,77 +283,69 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             const bool row_valid = tok_local < w.q_count;
             // position of this row's token; rows past the end of the block behave like its last token
             const int pos = w.kv_end - w.q_count + min(tok_local, w.q_count - 1);
-            float m_run = -INFINITY, l_run = 0.f, m_o = -INFINITY;
-            float o[HD];
-#pragma unroll
-            for (int d = 0; d < HD; ++d) o[d] = 0.f;
+            // exponent reference (a running maximum that is only moved when it has drifted by more than
+            // 2^8, so the accumulator in tensor memory rarely needs rescaling) and row sum
+            float m_ref = -INFINITY, l_run = 0.f;
             for (int j = 0; j < n_tiles && ok; ++j, ++kt) {
                 const int kbase = j * kKeysPerTile;
                 if (!tc::mbar_wait(s_full(g), n_s & 1, abort_flag)) { ok = false; break; }
                 ++n_s;
                 tc::tc_fence_after();
-                const bool need_mask = kbase + kKeysPerTile - 1 > pos;
-                // pass 1: row maximum of the visible scores of this tile
+                uint32_t sv[kKeysPerTile];
+#pragma unroll
+                for (int c = 0; c < kKeysPerTile; c += 32)
+                    tc::tmem_ld_32x32(s_addr + c, reinterpret_cast<uint32_t(&)[32]>(sv[c]));
+                tc::tmem_ld_wait();
                 float m_tile = -INFINITY;
+                if (kbase + kKeysPerTile - 1 > pos) {  // tile crosses this row's causal limit: mask
+#pragma unroll
+                    for (int e = 0; e < kKeysPerTile; ++e) {
+                        if (kbase + e > pos) sv[e] = 0xff800000u;  // -inf
+                        m_tile = fmaxf(m_tile, __uint_as_float(sv[e]));
+                    }
+                } else {
+#pragma unroll
+                    for (int e = 0; e < kKeysPerTile; ++e) m_tile = fmaxf(m_tile, __uint_as_float(sv[e]));
+                }
+                const bool bump = (m_tile - m_ref) * a.scale_log2 > 8.f;  // always true on an item's first tile
+                float alpha = 1.f;
+                if (bump) {
+                    alpha = fast_exp2((m_ref - m_tile) * a.scale_log2);
+                    m_ref = m_tile;
+                    l_run *= alpha;
+                }
+                if (j > 0 && __any_sync(0xffffffffu, bump)) {
+                    // O_w holds the earlier tiles' products relative to the old reference: once the last P V
+                    // has completed, scale the rows of this warp whose reference moved
+                    if (!tc::mbar_wait(pv_done(g), n_s & 1, abort_flag)) { ok = false; break; }
+                    tc::tc_fence_after();
 #pragma unroll 1
-                for (int c = 0; c < kKeysPerTile; c += 32) {
-                    uint32_t v[32];
-                    tc::tmem_ld_32x32(s_addr + c, v);
-                    tc::tmem_ld_wait();
-                    if (need_mask) {
+                    for (int c = 0; c < HD; c += 32) {
+                        uint32_t v[32];
+                        tc::tmem_ld_32x32(o_addr + c, v);
+                        tc::tmem_ld_wait();
 #pragma unroll
-                        for (int e = 0; e < 32; ++e)
-                            if (kbase + c + e <= pos) m_tile = fmaxf(m_tile, __uint_as_float(v[e]));
-                    } else {
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) m_tile = fmaxf(m_tile, __uint_as_float(v[e]));
+                        for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha);
+                        tmem_st_32x32(o_addr + c, v);
                     }
                 }
-                const float m_new = fmaxf(m_run, m_tile);
-                const float mb = m_new * a.scale_log2;
-                // pass 2: probabilities, row sum, bf16 P written over the S columns already consumed
-                float l_tile = 0.f;
-#pragma unroll 1
+                // probabilities (bf16) over the score columns, row sum in fp32
+                const float mb = m_ref * a.scale_log2;
+                float l0 = 0.f, l1 = 0.f;
+#pragma unroll
                 for (int c = 0; c < kKeysPerTile; c += 32) {
-                    uint32_t v[32];
-                    tc::tmem_ld_32x32(s_addr + c, v);
-                    tc::tmem_ld_wait();
                     uint32_t pk[16];
 #pragma unroll
                     for (int e = 0; e < 32; e += 2) {
-                        float p0 = fast_exp2(fmaf(__uint_as_float(v[e]), a.scale_log2, -mb));
-                        float p1 = fast_exp2(fmaf(__uint_as_float(v[e + 1]), a.scale_log2, -mb));
-                        if (need_mask) {
-                            if (kbase + c + e > pos) p0 = 0.f;
-                            if (kbase + c + e + 1 > pos) p1 = 0.f;
-                        }
-                        // the sum uses the rounded values that the tensor core will multiply with V
-                        const __nv_bfloat162 b2 = __floats2bfloat162_rn(p0, p1);
-                        l_tile += __low2float(b2) + __high2float(b2);
-                        pk[e >> 1] = *reinterpret_cast<const uint32_t *>(&b2);
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(sv[c + e]), a.scale_log2, -mb));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(sv[c + e + 1]), a.scale_log2, -mb));
+                        l0 += p0;
+                        l1 += p1;
+                        pk[e >> 1] = tc::pack_bf16(p0, p1);
                     }
                     tmem_st_32x16(s_addr + (c >> 1), pk);
                 }
-                l_run = l_run * fast_exp2((m_run - m_new) * a.scale_log2) + l_tile;
-                // fold the previous tile's P V (formed relative to m_run, the maximum after that tile) into
-                // the output registers (relative to m_o); both are brought to the new maximum
-                if (j > 0) {
-                    if (!tc::mbar_wait(pv_done(g), n_pv & 1, abort_flag)) { ok = false; break; }
-                    ++n_pv;
-                    tc::tc_fence_after();
-                    const float alpha = fast_exp2((m_o - m_new) * a.scale_log2);
-                    const float beta = fast_exp2((m_run - m_new) * a.scale_log2);
-#pragma unroll
-                    for (int c = 0; c < HD; c += 32) {
-                        uint32_t v[32];
-                        tc::tmem_ld_32x32(pv_addr + c, v);
-                        tc::tmem_ld_wait();
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) o[c + e] = fmaf(o[c + e], alpha, __uint_as_float(v[e]) * beta);
-                    }
-                    m_o = m_new;
-                }
-                m_run = m_new;
+                l_run += l0 + l1;
                 // V rows of keys at or beyond the item's causal limit are cleared before P V uses them
                 if (kbase + kKeysPerTile > w.kv_end) {
                     const int st = kt % kKvStages;
@@ -358,23 +362,22 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 tmem_st_wait();
                 tc::tc_fence_before();
                 __syncwarp();
-                if (lane == 0) tc::mbar_arrive(p_ready(g));  // P_w complete, PV_w buffer consumed
+                if (lane == 0) tc::mbar_arrive(p_ready(g));  // P_w (and O_w, if it was rescaled) ready for P V
             }
             if (!ok) break;
-            // last tile's P V, normalisation, store
-            if (!tc::mbar_wait(pv_done(g), n_pv & 1, abort_flag)) { ok = false; break; }
-            ++n_pv;
+            // the item's last P V, normalisation, store
+            if (!tc::mbar_wait(pv_done(g), (n_s - 1) & 1, abort_flag)) { ok = false; break; }
             tc::tc_fence_after();
+            float o[HD];
             {
-                const float alpha = fast_exp2((m_o - m_run) * a.scale_log2);
                 const float inv = 1.f / l_run;
 #pragma unroll
                 for (int c = 0; c < HD; c += 32) {
                     uint32_t v[32];
-                    tc::tmem_ld_32x32(pv_addr + c, v);
+                    tc::tmem_ld_32x32(o_addr + c, v);
                     tc::tmem_ld_wait();
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) o[c + e] = (fmaf(o[c + e], alpha, __uint_as_float(v[e]))) * inv;
+                    for (int e = 0; e < 32; ++e) o[c + e] = __uint_as_float(v[e]) * inv;
                 }
             }
             tc::tc_fence_before();
