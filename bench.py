@@ -46,75 +46,94 @@ def measured_peaks():
 
 
 class ClockSampler:
-    """Samples SM clock and throttle reasons with nvidia-smi while the timed region runs."""
-    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
-         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
-         "clocks_event_reasons.sw_power_cap")
+    """Samples SM clock and throttle reasons through NVML in a background thread while the timed work runs
+    (read-only queries; nothing is set)."""
+    REASONS = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40,
+               "hw_power_brake_slowdown": 0x80}
 
-    def __init__(self, gpu_index: int):
-        self.gpu = gpu_index
-        self.proc = None
-        self.lines = []
+    def __init__(self, gpu_index: int, period_s: float = 0.005):
+        self.gpu, self.period = gpu_index, period_s
+        self.sm, self.reasons, self.power = [], set(), []
+        self.stop_flag = threading.Event()
+        self.thread = None
+        self.err = None
+        self.max_mhz = None
+
+    def _physical_index(self) -> int:
+        vis = os.environ.get("CUDA_VISIBLE_DEVICES")
+        if vis:
+            ids = [v.strip() for v in vis.split(",") if v.strip()]
+            if self.gpu < len(ids) and ids[self.gpu].isdigit():
+                return int(ids[self.gpu])
+        return self.gpu
 
     def start(self):
         try:
-            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
-                                          "-lms", "100", "-i", str(self.gpu)], stdout=subprocess.PIPE,
-                                         stderr=subprocess.DEVNULL, text=True)
-            self.t = threading.Thread(target=self._read, daemon=True)
-            self.t.start()
-        except OSError:
-            self.proc = None
+            import pynvml
+            pynvml.nvmlInit()
+            self.nv = pynvml
+            vis = os.environ.get("CUDA_VISIBLE_DEVICES", "").split(",")
+            if self.gpu < len(vis) and vis[self.gpu].strip().startswith("GPU-"):
+                self.h = pynvml.nvmlDeviceGetHandleByUUID(vis[self.gpu].strip())
+            else:
+                self.h = pynvml.nvmlDeviceGetHandleByIndex(self._physical_index())
+            self.max_mhz = float(pynvml.nvmlDeviceGetMaxClockInfo(self.h, pynvml.NVML_CLOCK_SM))
+        except Exception as e:  # noqa: BLE001 - any NVML failure just disables the sampler
+            self.err = f"nvml unavailable: {e}"
+            return
+        self.thread = threading.Thread(target=self._run, daemon=True)
+        self.thread.start()
 
-    def _read(self):
-        for line in self.proc.stdout:
-            self.lines.append(line.strip())
+    def _run(self):
+        nv = self.nv
+        while not self.stop_flag.is_set():
+            try:
+                self.sm.append(float(nv.nvmlDeviceGetClockInfo(self.h, nv.NVML_CLOCK_SM)))
+                bits = int(nv.nvmlDeviceGetCurrentClocksEventReasons(self.h))
+                for name, bit in self.REASONS.items():
+                    if bits & bit:
+                        self.reasons.add(name)
+                self.power.append(nv.nvmlDeviceGetPowerUsage(self.h) / 1e3)
+            except Exception as e:  # noqa: BLE001
+                self.err = str(e)
+                return
+            time.sleep(self.period)
 
     def stop(self) -> dict:
-        if self.proc is None:
-            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
-        self.proc.terminate()
-        try:
-            self.proc.wait(timeout=5)
-        except subprocess.TimeoutExpired:
-            self.proc.kill()
-        sm, mx, reasons = [], [], set()
-        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
-        for ln in self.lines:
-            f = [x.strip() for x in ln.split(",")]
-            if len(f) < 9:
-                continue
-            try:
-                sm.append(float(f[1])); mx.append(float(f[2]))
-            except ValueError:
-                continue
-            for n, v in zip(names, f[5:9]):
-                if v.lower().startswith("active"):
-                    reasons.add(n)
-        return {"sm_mhz": float(np.median(sm)) if sm else None, "sm_max_mhz": max(mx) if mx else None,
-                "reasons": sorted(reasons), "samples": len(sm)}
+        if self.thread is None:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": [self.err or "not started"], "samples": 0}
+        self.stop_flag.set()
+        self.thread.join(timeout=2)
+        return {"sm_mhz": float(np.median(self.sm)) if self.sm else None, "sm_max_mhz": self.max_mhz,
+                "reasons": sorted(self.reasons), "samples": len(self.sm),
+                "power_w_max": max(self.power) if self.power else None}
 
 
-def oracle_sample_rate(w: wl.Workload, pool_np: np.ndarray, n_tokens: int, repeats: int = 1):
-    """Times the CPU oracle on the first n_tokens suffix tokens of request 0 (projection of those rows +
-    their attention over the request's cache).  Returns (tokens/s, threads, seconds per pass)."""
+def oracle_sample_rate(w: wl.Workload, pool_np: np.ndarray, n_tokens: int, requests=(0,), budget_s: float = 1e9):
+    """Times the CPU oracle on the first n_tokens suffix tokens of each listed request (projection of those
+    rows + their attention over the request's cache), stopping once budget_s has been spent.
+    Returns (tokens/s, threads, seconds, tokens done)."""
     from oracle import Oracle
     import helpers as hp
     orc = Oracle("f64")
     shape, b = w.shape, w.batch
-    P = int(b.prefix_lens[0])
-    K0, V0 = orc.paged_gather(pool_np, b.block_tables[0], P, shape.n_kv_heads, shape.page_size, shape.head_dim)
-    sub = wl.Batch(positions=b.positions[:n_tokens], query_start_loc=np.array([0, n_tokens], np.int32),
-                   seq_lens=np.array([P + n_tokens], np.int32), prefix_lens=b.prefix_lens[:1],
-                   activation_offsets=b.activation_offsets[:1], adapter_ids=b.adapter_ids[:1],
-                   block_tables=b.block_tables[:1], num_pages=b.num_pages, hidden=b.hidden[:n_tokens])
-    best = None
-    for _ in range(repeats):
+    total_s, done = 0.0, 0
+    for r in requests:
+        P = int(b.prefix_lens[r])
+        q0 = int(b.query_start_loc[r])
+        n = min(n_tokens, int(b.query_start_loc[r + 1]) - q0)
+        K0, V0 = orc.paged_gather(pool_np, b.block_tables[r], P, shape.n_kv_heads, shape.page_size, shape.head_dim)
+        sub = wl.Batch(positions=b.positions[q0:q0 + n], query_start_loc=np.array([0, n], np.int32),
+                       seq_lens=np.array([P + n], np.int32), prefix_lens=b.prefix_lens[r:r + 1],
+                       activation_offsets=b.activation_offsets[r:r + 1], adapter_ids=b.adapter_ids[r:r + 1],
+                       block_tables=b.block_tables[r:r + 1], num_pages=b.num_pages, hidden=b.hidden[q0:q0 + n])
         t0 = time.perf_counter()
         hp.oracle_block(orc, shape, w.wqkv, w.adapters, sub, [K0], [V0])
-        dt = time.perf_counter() - t0
-        best = dt if best is None else min(best, dt)
-    return n_tokens / best, orc.threads, best
+        total_s += time.perf_counter() - t0
+        done += n
+        if total_s > budget_s:
+            break
+    return done / total_s, orc.threads, total_s, done
 
 
 def run_reference(args):
@@ -129,7 +148,7 @@ def run_reference(args):
         oracle_sample_rate(w, pool_np, 2)
     times = []
     for _ in range(args.steps):
-        rate, threads, dt = oracle_sample_rate(w, pool_np, n_tok)
+        rate, threads, dt, _ = oracle_sample_rate(w, pool_np, n_tok)
         times.append(dt)
     ms = 1e3 * float(np.mean(times))
     value = n_tok / (ms / 1e3)
@@ -147,8 +166,8 @@ def run_reference(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
-    ap.add_argument("--warmup", type=int, default=5)
+    ap.add_argument("--steps", type=int, default=200)
+    ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours")
     ap.add_argument("--no-recompute", action="store_true", help="skip the full-LoRA recompute comparison")
     ap.add_argument("--no-cpu-baseline", action="store_true")
@@ -324,10 +343,10 @@ def main():
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        n_tok = 256
-        rate, threads, dt = oracle_sample_rate(w, pool_np, n_tok)
+        rate, threads, dt, done = oracle_sample_rate(w, pool_np, int(S_.max()), requests=range(R), budget_s=20.0)
         cpu = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle",
-               "sample": f"first {n_tok} suffix tokens of request 0 (projection + attention over {int(P_[0])}+ keys), {dt:.1f} s"}
+               "sample": f"{done} of the step's {T} suffix tokens, whole requests in order (projection + attention "
+                         f"over each request's cached keys), {dt:.1f} s of oracle time"}
 
     if rank == 0:
         print(json.dumps({

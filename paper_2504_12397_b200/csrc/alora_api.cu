@@ -148,7 +148,9 @@ alora_status alora_create(const alora_config *cfg, alora_ctx **out) {
     alloc((void **)&ctx->d_slot, Tm * 4);
     alloc((void **)&ctx->d_tiles, (size_t)ctx->max_tiles * sizeof(ProjTile));
     alloc((void **)&ctx->d_counts, 16 * 4);
-    alloc((void **)&ctx->d_seg_scratch, (size_t)4 * (2 * (size_t)c.max_requests + 1) * 4);
+    alloc((void **)&ctx->d_seg_scratch, (size_t)5 * (2 * (size_t)c.max_requests + 1) * 4);
+    alloc((void **)&ctx->d_shrink_tiles, (size_t)ctx->max_tiles * 4);
+    alloc((void **)&ctx->d_t_ready, (size_t)ctx->max_tiles * 4);
     alloc(&ctx->d_t, Tm * 3 * d.RP * 4);
     alloc(&ctx->d_qkv, Tm * d.N * es);
     alloc((void **)&ctx->d_status, 4);
@@ -206,7 +208,7 @@ alora_status alora_destroy(alora_ctx *ctx) {
     for (void *p : ctx->tc_a_all) if (p) cudaFree(p);
     for (void *p : ctx->tc_b_all) if (p) cudaFree(p);
     void *ptrs[] = {ctx->d_adapters, ctx->d_token_req, ctx->d_row_adapter, ctx->d_slot, ctx->d_tiles, ctx->d_counts,
-                    ctx->d_seg_scratch, ctx->d_t, ctx->d_qkv, ctx->d_status, ctx->d_act[0], ctx->d_act[1],
+                    ctx->d_seg_scratch, ctx->d_shrink_tiles, ctx->d_t_ready, ctx->d_t, ctx->d_qkv, ctx->d_status, ctx->d_act[0], ctx->d_act[1],
                     ctx->d_act[2], ctx->d_act[3], ctx->d_iota, ctx->d_attn_items, ctx->d_attn_off};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (ctx->h_status) cudaFreeHost(ctx->h_status);

@@ -69,7 +69,6 @@ struct ProfEvent {
 struct TcLayerMaps {
     CUtensorMap wqkv[2];      // W_qkv [N][H], boxes of 128 / 256 rows
     CUtensorMap a_all;        // all adapters' A rows [max_adapters*192][H], box 192 rows
-    CUtensorMap b_all;        // unused placeholder with the same geometry as b_all_bn (shrink launches)
     CUtensorMap b_all_bn[2];  // all adapters' B rows [max_adapters*N][64], boxes of 128 / 256 rows
 };
 
@@ -97,8 +96,10 @@ struct alora_ctx {
     // per-call workspaces
     int32_t *d_token_req = nullptr, *d_row_adapter = nullptr, *d_slot = nullptr;
     alora::ProjTile *d_tiles = nullptr;
-    int32_t *d_counts = nullptr;  // [0] number of projection tiles, [1] number of attention work items
-    int32_t *d_seg_scratch = nullptr;  // [4][2*max_requests+1] merged row runs of the current batch
+    int32_t *d_counts = nullptr;  // [0] projection row tiles, [1] attention work items, [2] row tiles with an adapter
+    int32_t *d_seg_scratch = nullptr;  // [5][2*max_requests+1] merged row runs of the current batch
+    int32_t *d_shrink_tiles = nullptr; // [max_tiles] indices of the row tiles with an adapter
+    int32_t *d_t_ready = nullptr;      // [max_tiles] per row tile: epilogue warps that have published t
     int32_t *d_iota = nullptr;         // 0..max_requests: query_start_loc of a decode batch
     int32_t max_tiles = 0;
     alora::AttnWork *d_attn_items = nullptr;  // tensor-core attention work list (bf16)

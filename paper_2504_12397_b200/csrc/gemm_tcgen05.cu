@@ -16,8 +16,16 @@
 // K block whose operands are t = s A x (rows of the tile) and the adapter's B rows of this column
 // tile, i.e. the delta s B (A x) is accumulated by the same tensor-core instruction stream.  Tiles
 // without an adapter execute exactly the base-only sequence: that is what makes gated-off rows
-// bit-identical to a base-only call (Prop. 1).  The same kernel in "shrink" mode computes
-// t = s A x for the adapter tiles.  No split-K, no atomics: results are run-to-run deterministic.
+// bit-identical to a base-only call (Prop. 1).
+//
+// Where t = s A x comes from.  With 256-wide column tiles the shrink is part of this kernel: the first
+// work items of the launch are one "shrink item" per adapter row tile, whose B operand is the adapter's
+// 192 A rows (q, k, v blocks, rank padded to 64) and whose epilogue writes t and then raises a per-tile
+// ready counter in global memory.  A projection item of an adapter tile waits (bounded) for that
+// counter before it loads t for its extra K block; since every block walks the item list in increasing
+// order and shrink items come first, the block that owns a shrink item never waits before finishing it.
+// With 128-wide column tiles the shrink runs as a separate cluster split-K kernel (shrink_tcgen05.cu).
+// No split-K, no atomics in the arithmetic: results are run-to-run deterministic.
 //
 // Every wait is bounded (tc::mbar_wait); on expiry the block records ALORA_ERR_TIMEOUT, drains its
 // outstanding copies and tensor-core work with bounded waits, frees its tensor memory and returns.
@@ -39,10 +47,13 @@ struct GemmArgs {
     __nv_bfloat16 *out;
     int ldo;
     const __nv_bfloat16 *residual;  // optional, same layout as out, may alias it
-    const AdapterDev *adapters;     // this layer's adapter table (expand / shrink), or nullptr
-    int shrink;                     // 1: out = t, B operand = the tile adapter's A rows, scaled by s
+    const AdapterDev *adapters;     // this layer's adapter table (expand), or nullptr
     int Nq, Nkv;                    // block boundaries of the fused output row (expand)
     int total_adapter_rows;         // rows per adapter in the B_all map (= N of the layer)
+    const int32_t *shrink_tiles;    // fused shrink: row-tile indices that have an adapter ...
+    const int32_t *n_shrink_tiles;  // ... and their count (nullptr: no shrink items in this launch)
+    int32_t *t_ready;               // [row tile] epilogue warps that have published their part of t
+    __nv_bfloat16 *t_out;           // [tokens][192]
     int32_t *status;
 };
 
@@ -65,11 +76,44 @@ __device__ __forceinline__ ProjTile load_tile(const GemmArgs &a, int m) {
     return t;
 }
 
+constexpr int kShrinkCols = 3 * kTensorRP;  // 192 columns of t: q, k, v blocks of 64 padded rank columns
+
+// Work item `item` of a launch: shrink items first (one per adapter row tile), then the projection's
+// (row tile, column tile) pairs.
+struct GemmItem {
+    ProjTile t;
+    int m;        // row-tile index
+    int n0;       // first output column (projection items)
+    bool shrink;
+};
+__device__ __forceinline__ GemmItem decode_item(const GemmArgs &a, int item, int n_shrink, int n_n, int BN) {
+    GemmItem g;
+    if (item < n_shrink) {
+        g.m = a.shrink_tiles[item];
+        g.n0 = 0;
+        g.shrink = true;
+    } else {
+        const int j = item - n_shrink;
+        g.m = j / n_n;
+        g.n0 = (j % n_n) * BN;
+        g.shrink = false;
+    }
+    g.t = load_tile(a, g.m);
+    return g;
+}
+
+__device__ __forceinline__ int ld_acquire(const int32_t *p) {
+    int v;
+    asm volatile("ld.acquire.gpu.global.s32 %0, [%1];" : "=r"(v) : "l"(p) : "memory");
+    return v;
+}
+__device__ __forceinline__ void fence_proxy_async_global() { asm volatile("fence.proxy.async.global;" ::: "memory"); }
+
 template <int BN>
 __global__ void __launch_bounds__(kGemmThreads, 1)
 gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_constant__ CUtensorMap tmB,
                     const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUtensorMap tmL,
-                    const GemmArgs a) {
+                    const __grid_constant__ CUtensorMap tmS, const GemmArgs a) {
     using S = GemmSmem<BN>;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
@@ -104,7 +148,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
 
     const int n_m = a.tiles ? *a.n_row_tiles : (a.M + kBM - 1) / kBM;
     const int n_n = (a.N + BN - 1) / BN;
-    const int total = n_m * n_n;
+    const int n_shrink = (BN >= kShrinkCols && a.n_shrink_tiles) ? *a.n_shrink_tiles : 0;
+    const int total = n_shrink + n_m * n_n;
     const int kb_main = (a.K + kBK - 1) / kBK;
 
     if (warp == 0) {
@@ -114,20 +159,34 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             uint32_t kc = 0;        // ring slots filled so far
             bool ok = true;
             for (int item = blockIdx.x; item < total && ok; item += gridDim.x) {
-                const int m = item / n_n, n0 = (item % n_n) * BN;
-                const ProjTile t = load_tile(a, m);
-                if (a.shrink && t.adapter < 0) continue;
-                const int extra = (!a.shrink && t.adapter >= 0) ? 1 : 0;
-                const int b_row0 = a.shrink ? t.adapter * BN : n0;
+                const GemmItem g = decode_item(a, item, n_shrink, n_n, BN);
+                const ProjTile t = g.t;
+                const int n0 = g.n0;
+                const int extra = (!g.shrink && t.adapter >= 0) ? 1 : 0;
                 for (int kb = 0; kb < kb_main + extra; ++kb, ++kc) {
                     const int s = kc % kStages;
                     if (!tc::mbar_wait(empty_bar(s), ((kc / kStages) & 1) ^ 1, abort_flag)) { ok = false; break; }
                     const uint32_t sa = smem_base + s * S::kStageBytes, sb = sa + S::kABytes;
-                    tc::mbar_arrive_expect_tx(full_bar(s), S::kStageBytes);
-                    if (kb < kb_main) {
+                    if (g.shrink) {
+                        tc::mbar_arrive_expect_tx(full_bar(s), S::kABytes + kShrinkCols * kBK * 2);
                         tc::tma_load_2d(sa, &tmA, full_bar(s), kb * kBK, t.row_start);
-                        tc::tma_load_2d(sb, &tmB, full_bar(s), kb * kBK, b_row0);
+                        tc::tma_load_2d(sb, &tmS, full_bar(s), kb * kBK, t.adapter * kShrinkCols);
+                    } else if (kb < kb_main) {
+                        tc::mbar_arrive_expect_tx(full_bar(s), S::kStageBytes);
+                        tc::tma_load_2d(sa, &tmA, full_bar(s), kb * kBK, t.row_start);
+                        tc::tma_load_2d(sb, &tmB, full_bar(s), kb * kBK, n0);
                     } else {
+                        if (n_shrink > 0) {
+                            // t of this row tile is written by another block's shrink item: wait until its four
+                            // epilogue warps have published, then order the TMA read after their writes
+                            const long long t0 = clock64();
+                            while (ld_acquire(a.t_ready + g.m) < 4) {
+                                if (*abort_flag || clock64() - t0 > tc::kWaitCycleLimit) { *abort_flag = 1; ok = false; break; }
+                            }
+                            if (!ok) break;
+                            fence_proxy_async_global();
+                        }
+                        tc::mbar_arrive_expect_tx(full_bar(s), S::kStageBytes);
                         const int blk = n0 < a.Nq ? 0 : (n0 < a.Nq + a.Nkv ? 1 : 2);
                         tc::tma_load_2d(sa, &tmT, full_bar(s), blk * kTensorRP, t.row_start);
                         tc::tma_load_2d(sb, &tmL, full_bar(s), 0, t.adapter * a.total_adapter_rows + n0);
@@ -147,15 +206,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     } else if (warp == 1) {
         if (lane == 0) {
             // ------------------------------ MMA issuer ------------------------------
-            constexpr uint32_t idesc = tc::idesc_bf16_f32(kBM, BN);
+            constexpr uint32_t idesc_main = tc::idesc_bf16_f32(kBM, BN);
+            constexpr uint32_t idesc_shrink = tc::idesc_bf16_f32(kBM, BN >= kShrinkCols ? kShrinkCols : BN);
             uint32_t kc = 0, it = 0;
             bool ok = true;
             for (int item = blockIdx.x; item < total && ok; item += gridDim.x) {
-                const int m = item / n_n;
-                const ProjTile t = load_tile(a, m);
-                if (a.shrink && t.adapter < 0) continue;
-                const int extra = (!a.shrink && t.adapter >= 0) ? 1 : 0;
+                const GemmItem g = decode_item(a, item, n_shrink, n_n, BN);
+                const ProjTile t = g.t;
+                const int extra = (!g.shrink && t.adapter >= 0) ? 1 : 0;
                 const int extra_steps = extra ? a.adapters[t.adapter].rpad / 16 : 0;
+                const uint32_t idesc = g.shrink ? idesc_shrink : idesc_main;
                 const uint32_t acc = it & 1;
                 if (!tc::mbar_wait(acce_bar(acc), ((it >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
                 tc::tc_fence_after();
@@ -187,15 +247,47 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         uint32_t it = 0;
         bool ok = true;
         for (int item = blockIdx.x; item < total && ok; item += gridDim.x) {
-            const int m = item / n_n, n0 = (item % n_n) * BN;
-            const ProjTile t = load_tile(a, m);
-            if (a.shrink && t.adapter < 0) continue;
+            const GemmItem g = decode_item(a, item, n_shrink, n_n, BN);
+            const ProjTile t = g.t;
+            const int n0 = g.n0;
             const uint32_t acc = it & 1;
             if (!tc::mbar_wait(accf_bar(acc), (it >> 1) & 1, abort_flag)) { ok = false; break; }
             tc::tc_fence_after();
             const int r = q * 32 + lane;
             const bool row_ok = r < t.row_count;
-            const float scale = a.shrink ? a.adapters[t.adapter].scale : 1.f;
+            if (g.shrink) {
+                // t = s A x of this row tile: 192 columns, scaled, rounded to bf16
+                const float scale = a.adapters[t.adapter].scale;
+                __nv_bfloat16 *trow = a.t_out + (size_t)(t.row_start + r) * kShrinkCols;
+#pragma unroll 1
+                for (int c = 0; c < kShrinkCols && c < BN; c += 32) {
+                    uint32_t v[32];
+                    tc::tmem_ld_32x32(tmem_base + acc * BN + c + ((uint32_t)(q * 32) << 16), v);
+                    tc::tmem_ld_wait();
+                    if (row_ok) {
+#pragma unroll
+                        for (int j = 0; j < 4; ++j) {
+                            uint4 o;
+                            o.x = tc::pack_bf16(__uint_as_float(v[8 * j]) * scale, __uint_as_float(v[8 * j + 1]) * scale);
+                            o.y = tc::pack_bf16(__uint_as_float(v[8 * j + 2]) * scale, __uint_as_float(v[8 * j + 3]) * scale);
+                            o.z = tc::pack_bf16(__uint_as_float(v[8 * j + 4]) * scale, __uint_as_float(v[8 * j + 5]) * scale);
+                            o.w = tc::pack_bf16(__uint_as_float(v[8 * j + 6]) * scale, __uint_as_float(v[8 * j + 7]) * scale);
+                            *reinterpret_cast<uint4 *>(trow + c + 8 * j) = o;
+                        }
+                    }
+                }
+                tc::tc_fence_before();
+                // publish: the rows are read by other blocks through TMA (async proxy)
+                fence_proxy_async_global();
+                __threadfence();
+                __syncwarp();
+                if (lane == 0) {
+                    atomicAdd(a.t_ready + g.m, 1);
+                    tc::mbar_arrive(acce_bar(acc));
+                }
+                ++it;
+                continue;
+            }
             __nv_bfloat16 *orow = a.out + (size_t)(t.row_start + r) * a.ldo + n0;
             const __nv_bfloat16 *rrow = a.residual ? a.residual + (size_t)(t.row_start + r) * a.ldo + n0 : nullptr;
 #pragma unroll 1
@@ -209,7 +301,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         if (n0 + c + 8 * j >= a.N) break;
                         float f[8];
 #pragma unroll
-                        for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[8 * j + e]) * scale;
+                        for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[8 * j + e]);
                         if (rrow) {
                             const uint4 rv = *reinterpret_cast<const uint4 *>(rrow + c + 8 * j);
                             const uint32_t rw[4] = {rv.x, rv.y, rv.z, rv.w};
@@ -279,7 +371,8 @@ bool make_tensor_map_bf16(CUtensorMap *map, const void *base, uint64_t rows, uin
 
 template <int BN>
 static bool launch_gemm_bn(alora_ctx *ctx, const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtensorMap &tmT,
-                           const CUtensorMap &tmL, const GemmArgs &args, int max_items, cudaStream_t s) {
+                           const CUtensorMap &tmL, const CUtensorMap &tmS, const GemmArgs &args, int max_items,
+                           cudaStream_t s) {
     static bool attr_set[64] = {};
     const int dev = ctx->cfg.device;
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
@@ -289,9 +382,12 @@ static bool launch_gemm_bn(alora_ctx *ctx, const CUtensorMap &tmA, const CUtenso
         attr_set[dev] = true;
     }
     const int grid = std::max(1, std::min(ctx->sm_count, max_items));
-    gemm_tcgen05_kernel<BN><<<grid, kGemmThreads, GemmSmem<BN>::kTotal, s>>>(tmA, tmB, tmT, tmL, args);
+    gemm_tcgen05_kernel<BN><<<grid, kGemmThreads, GemmSmem<BN>::kTotal, s>>>(tmA, tmB, tmT, tmL, tmS, args);
     return true;
 }
+
+bool launch_shrink_tc(alora_ctx *ctx, const CUtensorMap &tmX, const CUtensorMap &tmA, const AdapterDev *adapters,
+                      int K, int max_row_tiles, cudaStream_t s);  // shrink_tcgen05.cu
 
 // Picks the column-tile width: 256 when the q/k/v block boundaries allow it, else 128.
 static int pick_bn(int N, int Nq, int Nkv, bool lora) {
@@ -319,24 +415,26 @@ int launch_project_tc(alora_ctx *ctx, int layer, const void *hidden, int T, void
     const int max_row_tiles = ctx->max_tiles < (T / kBM + 2 * ctx->cfg.max_requests + 2)
                                   ? ctx->max_tiles : (T / kBM + 2 * ctx->cfg.max_requests + 2);
     int n = 0;
-    if (have_adapters) {
+    const bool fuse_shrink = have_adapters && BN == 256;
+    if (have_adapters && !fuse_shrink) {
         ProfScope prof(ctx, KK_SHRINK, s);
-        GemmArgs g{};
-        g.tiles = ctx->d_tiles; g.n_row_tiles = ctx->d_counts; g.M = T; g.N = 3 * kTensorRP; g.K = d.H;
-        g.out = (__nv_bfloat16 *)ctx->d_t; g.ldo = 3 * kTensorRP; g.residual = nullptr; g.adapters = ads;
-        g.shrink = 1; g.Nq = d.Nq; g.Nkv = d.Nkv; g.total_adapter_rows = d.N; g.status = ctx->d_status;
-        if (!launch_gemm_bn<3 * kTensorRP>(ctx, tmX, lm.a_all, tmTt, lm.b_all, g, max_row_tiles, s)) return -1;
+        if (!launch_shrink_tc(ctx, tmX, lm.a_all, ads, d.H, max_row_tiles, s)) return -1;
         ++n;
     }
     {
         ProfScope prof(ctx, KK_PROJECT, s);
         GemmArgs g{};
         g.tiles = ctx->d_tiles; g.n_row_tiles = ctx->d_counts; g.M = T; g.N = d.N; g.K = d.H;
-        g.out = (__nv_bfloat16 *)qkv; g.ldo = d.N; g.residual = nullptr; g.adapters = ads; g.shrink = 0;
+        g.out = (__nv_bfloat16 *)qkv; g.ldo = d.N; g.residual = nullptr; g.adapters = ads;
         g.Nq = d.Nq; g.Nkv = d.Nkv; g.total_adapter_rows = d.N; g.status = ctx->d_status;
-        const int items = max_row_tiles * ((d.N + BN - 1) / BN);
-        const bool ok = BN == 256 ? launch_gemm_bn<256>(ctx, tmX, lm.wqkv[1], tmTt, lm.b_all_bn[1], g, items, s)
-                                  : launch_gemm_bn<128>(ctx, tmX, lm.wqkv[0], tmTt, lm.b_all_bn[0], g, items, s);
+        if (fuse_shrink) {
+            g.shrink_tiles = ctx->d_shrink_tiles; g.n_shrink_tiles = ctx->d_counts + 2;
+            g.t_ready = ctx->d_t_ready; g.t_out = (__nv_bfloat16 *)ctx->d_t;
+        }
+        const int items = max_row_tiles * ((d.N + BN - 1) / BN + (fuse_shrink ? 1 : 0));
+        const bool ok = BN == 256
+                            ? launch_gemm_bn<256>(ctx, tmX, lm.wqkv[1], tmTt, lm.b_all_bn[1], lm.a_all, g, items, s)
+                            : launch_gemm_bn<128>(ctx, tmX, lm.wqkv[0], tmTt, lm.b_all_bn[0], lm.a_all, g, items, s);
         if (!ok) return -1;
         ++n;
     }
@@ -355,11 +453,11 @@ int launch_linear_tc(alora_ctx *ctx, const void *x, const void *W, int T, int K,
     if (!make_tensor_map_bf16(&tmW, W, N, K, K, BN)) return -1;
     GemmArgs g{};
     g.tiles = nullptr; g.n_row_tiles = nullptr; g.M = T; g.N = N; g.K = K; g.out = (__nv_bfloat16 *)y; g.ldo = N;
-    g.residual = (const __nv_bfloat16 *)residual; g.adapters = nullptr; g.shrink = 0; g.Nq = N; g.Nkv = 0;
+    g.residual = (const __nv_bfloat16 *)residual; g.adapters = nullptr; g.Nq = N; g.Nkv = 0;
     g.total_adapter_rows = 0; g.status = ctx->d_status;
     const int items = ((T + kBM - 1) / kBM) * ((N + BN - 1) / BN);
-    const bool ok = BN == 256 ? launch_gemm_bn<256>(ctx, tmX, tmW, tmX, tmW, g, items, s)
-                              : launch_gemm_bn<128>(ctx, tmX, tmW, tmX, tmW, g, items, s);
+    const bool ok = BN == 256 ? launch_gemm_bn<256>(ctx, tmX, tmW, tmX, tmW, tmW, g, items, s)
+                              : launch_gemm_bn<128>(ctx, tmX, tmW, tmX, tmW, tmW, g, items, s);
     return ok ? 1 : -1;
 }
 
@@ -375,7 +473,6 @@ bool build_layer_maps(alora_ctx *ctx, int layer) {
     }
     const size_t na = (size_t)std::max(1, ctx->cfg.max_adapters);
     ok &= make_tensor_map_bf16(&lm.a_all, ctx->tc_a_all[layer], na * 3 * kTensorRP, d.H, d.H, 3 * kTensorRP);
-    ok &= make_tensor_map_bf16(&lm.b_all, ctx->tc_b_all[layer], na * d.N, kTensorRP, kTensorRP, 3 * kTensorRP);
     ok &= make_tensor_map_bf16(&lm.b_all_bn[0], ctx->tc_b_all[layer], na * d.N, kTensorRP, kTensorRP, 128);
     ok &= make_tensor_map_bf16(&lm.b_all_bn[1], ctx->tc_b_all[layer], na * d.N, kTensorRP, kTensorRP, 256);
     return ok;

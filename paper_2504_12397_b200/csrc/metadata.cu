@@ -22,7 +22,7 @@ __device__ __forceinline__ int find_request(const int32_t *qsl, int R, int t) {
 // page * page_size + position % page_size.  Findings (inconsistent positions, page id out of
 // range, adapter id out of range) go to the status word; the row then gets adapter -1 / slot -1 so
 // that later kernels skip it.
-__global__ void metadata_token_kernel(const int32_t *__restrict__ positions,
+__device__ __forceinline__ void metadata_tokens(const int32_t *__restrict__ positions,
                                       const int32_t *__restrict__ a_req,
                                       const int32_t *__restrict__ adapter_ids,
                                       const int32_t *__restrict__ qsl, const int32_t *__restrict__ seq_lens,
@@ -66,13 +66,15 @@ __global__ void metadata_token_kernel(const int32_t *__restrict__ positions,
 // rows (applied adapter -1) and its gated-on rows; neighbouring runs with the same applied adapter
 // are merged across requests, and every merged run is cut into tiles of at most kProjTileRows rows.
 // One block; R is small (a scheduler batch).
-__global__ void metadata_tiles_kernel(const int32_t *__restrict__ a_req, const int32_t *__restrict__ adapter_ids,
+__device__ __forceinline__ void metadata_tiles(const int32_t *__restrict__ a_req, const int32_t *__restrict__ adapter_ids,
                                       const int32_t *__restrict__ qsl, const int32_t *__restrict__ seq_lens,
                                       int R, int mode, int max_adapters, int max_tiles,
                                       ProjTile *__restrict__ tiles, int32_t *__restrict__ counts,
-                                      int32_t *seg_scratch /* [4 * (2R+1)] */, int32_t *status) {
+                                      int32_t *seg_scratch /* [5 * (2R+1)] */, int32_t *__restrict__ shrink_tiles,
+                                      int32_t *__restrict__ t_ready, int32_t *status) {
     int32_t *seg_start = seg_scratch, *seg_len = seg_scratch + (2 * R + 1);
     int32_t *seg_adapter = seg_scratch + 2 * (2 * R + 1), *seg_tile0 = seg_scratch + 3 * (2 * R + 1);
+    int32_t *seg_shrink0 = seg_scratch + 4 * (2 * R + 1);  // adapter tiles before the segment
     __shared__ int n_seg, n_tiles;
     if (threadIdx.x == 0) {
         int ns = 0, nt = 0;
@@ -101,14 +103,19 @@ __global__ void metadata_tiles_kernel(const int32_t *__restrict__ a_req, const i
                 }
             }
         }
+        int n_ad = 0;
         for (int s = 0; s < ns; ++s) {
             seg_tile0[s] = nt;
-            nt += (seg_len[s] + kProjTileRows - 1) / kProjTileRows;
+            seg_shrink0[s] = n_ad;
+            const int n = (seg_len[s] + kProjTileRows - 1) / kProjTileRows;
+            nt += n;
+            if (seg_adapter[s] >= 0) n_ad += n;
         }
         seg_tile0[ns] = nt;
-        if (nt > max_tiles) { report(status, ALORA_ERR_CAPACITY); nt = 0; ns = 0; }
+        if (nt > max_tiles) { report(status, ALORA_ERR_CAPACITY); nt = 0; ns = 0; n_ad = 0; }
         n_seg = ns; n_tiles = nt;
         counts[0] = nt;
+        counts[2] = n_ad;
     }
     __syncthreads();
     for (int i = threadIdx.x; i < n_tiles; i += blockDim.x) {
@@ -124,6 +131,9 @@ __global__ void metadata_tiles_kernel(const int32_t *__restrict__ a_req, const i
         pt.adapter = seg_adapter[lo];
         pt.pad_ = 0;
         tiles[i] = pt;
+        // list of the tiles that need t = s A x, and their "t is ready" counters, cleared for this batch
+        if (pt.adapter >= 0) shrink_tiles[seg_shrink0[lo] + (i - seg_tile0[lo])] = i;
+        t_ready[i] = 0;
     }
 }
 
@@ -131,7 +141,7 @@ __global__ void metadata_tiles_kernel(const int32_t *__restrict__ a_req, const i
 // `q_block` tokens; one item per (request, KV head, block), blocks of the same KV stream adjacent so
 // that blocks running at the same time share their K/V pages in L2.  Keys 0 .. position of the
 // block's last token are visible to the block (causal limit); per-row limits are applied in the kernel.
-__global__ void metadata_attn_items_kernel(const int32_t *__restrict__ qsl, const int32_t *__restrict__ seq_lens,
+__device__ __forceinline__ void metadata_attn_items(const int32_t *__restrict__ qsl, const int32_t *__restrict__ seq_lens,
                                            int R, int Hkv, int q_block, int max_items,
                                            AttnWork *__restrict__ items, int32_t *__restrict__ counts,
                                            int32_t *__restrict__ blk_off /* [R+1] */, int32_t *status) {
@@ -174,25 +184,41 @@ __global__ void metadata_attn_items_kernel(const int32_t *__restrict__ qsl, cons
     }
 }
 
+// The whole metadata step as one launch: every block handles 256 tokens; block 0 then builds the two
+// work lists (their serial parts are O(R)).
+__global__ void __launch_bounds__(256)
+metadata_kernel(const int32_t *__restrict__ positions, const int32_t *__restrict__ a_req,
+                const int32_t *__restrict__ adapter_ids, const int32_t *__restrict__ qsl,
+                const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ block_tables, int max_blocks,
+                int num_pages, int page_size, int max_adapters, int T, int R, int mode,
+                int32_t *__restrict__ token_req, int32_t *__restrict__ row_adapter, int32_t *__restrict__ slot_map,
+                int max_tiles, ProjTile *__restrict__ tiles, int32_t *__restrict__ counts, int32_t *seg_scratch,
+                int32_t *__restrict__ shrink_tiles, int32_t *__restrict__ t_ready,
+                int Hkv, int q_block, int max_items, AttnWork *__restrict__ items, int32_t *__restrict__ blk_off,
+                int32_t *status) {
+    metadata_tokens(positions, a_req, adapter_ids, qsl, seq_lens, block_tables, max_blocks, num_pages, page_size,
+                    max_adapters, T, R, mode, token_req, row_adapter, slot_map, status);
+    if (blockIdx.x != 0) return;
+    metadata_tiles(a_req, adapter_ids, qsl, seq_lens, R, mode, max_adapters, max_tiles, tiles, counts, seg_scratch,
+                   shrink_tiles, t_ready, status);
+    if (items != nullptr && block_tables != nullptr)
+        metadata_attn_items(qsl, seq_lens, R, Hkv, q_block, max_items, items, counts, blk_off, status);
+}
+
 int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s) {
     if (b.T == 0) {
-        cudaMemsetAsync(ctx->d_counts, 0, 2 * sizeof(int32_t), s);
+        cudaMemsetAsync(ctx->d_counts, 0, 3 * sizeof(int32_t), s);
         return 0;
     }
     ProfScope prof(ctx, KK_METADATA, s);
     const int threads = 256;
-    metadata_token_kernel<<<(b.T + threads - 1) / threads, threads, 0, s>>>(
+    metadata_kernel<<<(b.T + threads - 1) / threads, threads, 0, s>>>(
         b.positions, b.activation_offsets, b.adapter_ids, b.query_start_loc, b.seq_lens, b.block_tables,
-        b.max_blocks, b.num_pages, ctx->d.page, ctx->cfg.max_adapters, b.T, b.R, b.mode,
-        ctx->d_token_req, ctx->d_row_adapter, ctx->d_slot, ctx->d_status);
-    metadata_tiles_kernel<<<1, 256, 0, s>>>(b.activation_offsets, b.adapter_ids, b.query_start_loc,
-                                           b.seq_lens, b.R, b.mode, ctx->cfg.max_adapters, ctx->max_tiles,
-                                           ctx->d_tiles, ctx->d_counts, ctx->d_seg_scratch, ctx->d_status);
-    if (ctx->d_attn_items == nullptr || b.block_tables == nullptr) return 2;
-    metadata_attn_items_kernel<<<1, 256, 0, s>>>(b.query_start_loc, b.seq_lens, b.R, ctx->d.Hkv, ctx->attn_q_block,
-                                                ctx->max_attn_items, ctx->d_attn_items, ctx->d_counts,
-                                                ctx->d_attn_off, ctx->d_status);
-    return 3;
+        b.max_blocks, b.num_pages, ctx->d.page, ctx->cfg.max_adapters, b.T, b.R, b.mode, ctx->d_token_req,
+        ctx->d_row_adapter, ctx->d_slot, ctx->max_tiles, ctx->d_tiles, ctx->d_counts, ctx->d_seg_scratch,
+        ctx->d_shrink_tiles, ctx->d_t_ready,
+        ctx->d.Hkv, ctx->attn_q_block, ctx->max_attn_items, ctx->d_attn_items, ctx->d_attn_off, ctx->d_status);
+    return 1;
 }
 
 }  // namespace alora
