@@ -161,6 +161,16 @@ alora_status alora_create(const alora_config *cfg, alora_ctx **out) {
         ctx->max_attn_items = (int)((Tm / ctx->attn_q_block + (size_t)c.max_requests) * d.Hkv);
         alloc((void **)&ctx->d_attn_items, (size_t)ctx->max_attn_items * sizeof(AttnWork));
         alloc((void **)&ctx->d_attn_off, ((size_t)c.max_requests + 1) * 4);
+        if (16 % d.G == 0 && (d.hd == 64 || d.hd == 128)) {
+            // few-row attention: at most 16 * n_sm key ranges plus one per (request, KV head, row block)
+            ctx->small_max_tokens = 16;
+            const int blocks_per_req = std::max(1, (16 * d.G + 63) / 64);
+            ctx->max_split_items = 16 * ctx->sm_count + c.max_requests * blocks_per_req * d.Hkv;
+            alloc((void **)&ctx->d_split_items, (size_t)ctx->max_split_items * sizeof(AttnSplitWork));
+            alloc((void **)&ctx->d_req_scratch, (size_t)2 * c.max_requests * 4);
+            alloc((void **)&ctx->d_part_o, (size_t)ctx->max_split_items * 64 * d.hd * 4);
+            alloc((void **)&ctx->d_part_ml, (size_t)ctx->max_split_items * 64 * 2 * 4);
+        }
     }
     if (c.dtype == ALORA_DTYPE_BF16) {
         const size_t na = (size_t)std::max(1, c.max_adapters);
@@ -209,7 +219,8 @@ alora_status alora_destroy(alora_ctx *ctx) {
     for (void *p : ctx->tc_b_all) if (p) cudaFree(p);
     void *ptrs[] = {ctx->d_adapters, ctx->d_token_req, ctx->d_row_adapter, ctx->d_slot, ctx->d_tiles, ctx->d_counts,
                     ctx->d_seg_scratch, ctx->d_shrink_tiles, ctx->d_t_ready, ctx->d_t, ctx->d_qkv, ctx->d_status, ctx->d_act[0], ctx->d_act[1],
-                    ctx->d_act[2], ctx->d_act[3], ctx->d_iota, ctx->d_attn_items, ctx->d_attn_off};
+                    ctx->d_act[2], ctx->d_act[3], ctx->d_iota, ctx->d_attn_items, ctx->d_attn_off, ctx->d_split_items,
+                    ctx->d_req_scratch, ctx->d_part_o, ctx->d_part_ml};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (ctx->h_status) cudaFreeHost(ctx->h_status);
     for (ProfEvent &e : ctx->prof_events) { if (e.begin) cudaEventDestroy(e.begin); if (e.end) cudaEventDestroy(e.end); }
@@ -309,7 +320,7 @@ alora_status alora_validate_batch(const alora_config *cfg, const int32_t *pos, c
 
 #define ALORA_BATCH(mode_)                                                                               \
     BatchArgs b{d_positions, d_activation_offsets, d_adapter_ids, d_query_start_loc, d_seq_lens,         \
-                d_block_tables, max_blocks, num_pages, T, R, (mode_)}
+                d_block_tables, max_blocks, num_pages, T, R, (mode_), 0}
 
 alora_status alora_batch_metadata(alora_ctx *ctx, int mode, const int32_t *d_positions,
                                   const int32_t *d_activation_offsets, const int32_t *d_adapter_ids,
@@ -396,7 +407,8 @@ static alora_status layer_entry(alora_ctx *ctx, int layer, int mode, const void 
                                 const int32_t *d_positions, const int32_t *d_activation_offsets,
                                 const int32_t *d_adapter_ids, const int32_t *d_query_start_loc,
                                 const int32_t *d_seq_lens, void *d_paged_kv, const int32_t *d_block_tables,
-                                int max_blocks, int num_pages, int T, int R, void *d_attn_out, void *stream) {
+                                int max_blocks, int num_pages, int T, int R, void *d_attn_out, void *stream,
+                                bool one_token_per_request = false) {
     alora_status st = check_batch_args(ctx, T, R);
     if (st != ALORA_OK) return st;
     if (!d_hidden || !d_positions || !d_query_start_loc || !d_seq_lens || !d_block_tables || !d_paged_kv || !d_attn_out)
@@ -407,6 +419,7 @@ static alora_status layer_entry(alora_ctx *ctx, int layer, int mode, const void 
     cudaStream_t s = (cudaStream_t)stream;
     ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
     ALORA_BATCH(mode);
+    b.all_small = one_token_per_request ? 1 : 0;
     return run_layer(ctx, layer, d_hidden, b, d_paged_kv, d_attn_out, s);
 }
 
@@ -438,7 +451,6 @@ alora_status alora_decode_step(alora_ctx *ctx, int layer, const void *d_hidden, 
     if (R < 0) return ALORA_ERR_INVALID_ARG;
     if (R > ctx->cfg.max_requests || R > ctx->cfg.max_tokens) return ALORA_ERR_CAPACITY;
     // query_start_loc of a decode batch is 0, 1, ..., R: kept in the context, built on first use
-    cudaStream_t s = (cudaStream_t)stream;
     ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
     if (!ctx->d_iota) {
         std::vector<int32_t> iota((size_t)ctx->cfg.max_requests + 1);
@@ -448,7 +460,7 @@ alora_status alora_decode_step(alora_ctx *ctx, int layer, const void *d_hidden, 
     }
     return layer_entry(ctx, layer, ALORA_MODE_ALORA, d_hidden, d_positions, d_activation_offsets, d_adapter_ids,
                        ctx->d_iota, d_seq_lens, d_paged_kv, d_block_tables, max_blocks, num_pages, R, R, d_attn_out,
-                       stream);
+                       stream, /*one_token_per_request=*/true);
 }
 
 alora_status alora_forward_stack(alora_ctx *ctx, int mode, const void *d_hidden_in, const int32_t *d_positions,

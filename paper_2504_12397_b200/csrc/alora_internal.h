@@ -56,6 +56,16 @@ struct AttnWork {
     int32_t n_splits;
 };
 
+// One unit of few-row (decode / short suffix) attention work: score rows of `q_count` tokens starting at
+// flat token q_start (rows are (token, query head of the group) pairs, `mt` tiles of 16 rows), one KV
+// head, keys [kv_start, kv_end) of the request.  The `n_splits` key ranges of the same rows are
+// consecutive items; their partial results are merged afterwards.
+struct AttnSplitWork {
+    int32_t req, q_start, q_count, kv_head;
+    int32_t kv_start, kv_end, pos0, mt;      // pos0 = position of the first token of the block
+    int32_t split, n_splits, pad0_, pad1_;
+};
+
 // Kernel families, for the optional per-kernel timing (alora_profile_*).
 enum KernelKind { KK_METADATA = 0, KK_SHRINK, KK_PROJECT, KK_KV_APPEND, KK_ATTENTION, KK_ATTN_MERGE, KK_LINEAR,
                   KK_GLUE, KK_COUNT };
@@ -105,6 +115,11 @@ struct alora_ctx {
     alora::AttnWork *d_attn_items = nullptr;  // tensor-core attention work list (bf16)
     int32_t *d_attn_off = nullptr;            // [max_requests+1] block offsets per request
     int32_t max_attn_items = 0, attn_q_block = 0;
+    // few-row attention (requests with at most small_max_tokens new tokens): split-KV work list and partials
+    alora::AttnSplitWork *d_split_items = nullptr;
+    int32_t *d_req_scratch = nullptr;   // [2][max_requests] items per request, item offset per request
+    float *d_part_o = nullptr, *d_part_ml = nullptr;
+    int32_t max_split_items = 0, small_max_tokens = 0;
     void *d_t = nullptr;          // [max_tokens][3][RP] rank-r intermediate
     void *d_qkv = nullptr;        // [max_tokens][N]
     void *d_act[4] = {nullptr, nullptr, nullptr, nullptr};  // stack activations
@@ -154,6 +169,7 @@ struct ProfScope {
 struct BatchArgs {
     const int32_t *positions, *activation_offsets, *adapter_ids, *query_start_loc, *seq_lens, *block_tables;
     int max_blocks, num_pages, T, R, mode;
+    int all_small;  // host-side knowledge that no request has more than small_max_tokens new tokens (decode)
 };
 
 int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s);

@@ -413,9 +413,19 @@ EncodeTiledFn tensor_map_encoder();  // gemm_tcgen05.cu
 
 // Prefill attention on the tensor cores.  Returns kernels launched, or -1 when the shape is unsupported
 // (head dim other than 64/128, group size not dividing 128, page size not a power of two in 8..128).
+int launch_attend_splitkv(alora_ctx *ctx, const void *qkv, const BatchArgs &b, const void *pool, void *out,
+                          cudaStream_t s);  // attn_splitkv.cu
+
 int launch_attend_tc(alora_ctx *ctx, const void *qkv, const BatchArgs &b, const void *pool, void *out,
                      cudaStream_t s) {
     if (b.T == 0) return 0;
+    // requests with few new tokens (decode, short suffixes) are on the few-row work list
+    int n_small = 0;
+    if (ctx->max_split_items > 0) {
+        n_small = launch_attend_splitkv(ctx, qkv, b, pool, out, s);
+        if (n_small < 0) return -1;
+        if (b.all_small) return n_small;
+    }
     const Dims &d = ctx->d;
     const bool page_ok = d.page >= 8 && d.page <= 128 && (d.page & (d.page - 1)) == 0;
     if ((d.hd != 64 && d.hd != 128) || 128 % d.G != 0 || !page_ok) return -1;
@@ -462,7 +472,7 @@ int launch_attend_tc(alora_ctx *ctx, const void *qkv, const BatchArgs &b, const 
     }
     if (hi) attn_tcgen05_kernel<128><<<grid, kAttnThreads, AttnSmem<128>::kTotal, s>>>(tmQ, tmKV, a);
     else attn_tcgen05_kernel<64><<<grid, kAttnThreads, AttnSmem<64>::kTotal, s>>>(tmQ, tmKV, a);
-    return 1;
+    return 1 + n_small;
 }
 
 }  // namespace alora

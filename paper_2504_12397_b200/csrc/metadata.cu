@@ -142,7 +142,7 @@ __device__ __forceinline__ void metadata_tiles(const int32_t *__restrict__ a_req
 // that blocks running at the same time share their K/V pages in L2.  Keys 0 .. position of the
 // block's last token are visible to the block (causal limit); per-row limits are applied in the kernel.
 __device__ __forceinline__ void metadata_attn_items(const int32_t *__restrict__ qsl, const int32_t *__restrict__ seq_lens,
-                                           int R, int Hkv, int q_block, int max_items,
+                                           int R, int Hkv, int q_block, int small_max, int max_items,
                                            AttnWork *__restrict__ items, int32_t *__restrict__ counts,
                                            int32_t *__restrict__ blk_off /* [R+1] */, int32_t *status) {
     __shared__ int total;
@@ -151,7 +151,7 @@ __device__ __forceinline__ void metadata_attn_items(const int32_t *__restrict__ 
         for (int r = 0; r < R; ++r) {
             blk_off[r] = acc;
             const int n_new = qsl[r + 1] - qsl[r];
-            acc += n_new > 0 ? (n_new + q_block - 1) / q_block : 0;
+            acc += n_new > small_max ? (n_new + q_block - 1) / q_block : 0;  // short requests: few-row list
         }
         blk_off[R] = acc;
         int n = acc * Hkv;
@@ -184,6 +184,94 @@ __device__ __forceinline__ void metadata_attn_items(const int32_t *__restrict__ 
     }
 }
 
+// Work list of the few-row attention kernel: requests with 1 .. small_max new tokens.  Their score rows
+// (token, query head of the group) are cut into blocks of 16 * mt rows (mt = 1, 2 or 4 tiles, the
+// smallest that holds all rows, else 4), and the keys 0 .. causal limit of each block into ranges of
+// `chunk` 64-key units, chosen so that about 16 ranges per SM exist in total (at least 256 keys each).
+// The ranges of one (block, KV head) are consecutive items.
+__device__ __forceinline__ void small_block_shape(int n_new, int G, int &mt, int &tok_per_blk, int &nblk) {
+    const int rows = n_new * G;
+    mt = rows <= 16 ? 1 : (rows <= 32 ? 2 : 4);
+    tok_per_blk = 16 * mt / G;
+    nblk = (n_new + tok_per_blk - 1) / tok_per_blk;
+}
+
+__device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__ qsl, const int32_t *__restrict__ seq_lens,
+                                                     int R, int Hkv, int G, int n_sm, int small_max, int max_items,
+                                                     AttnSplitWork *__restrict__ items, int32_t *__restrict__ counts,
+                                                     int32_t *__restrict__ req_scratch /* [2][R] */, int32_t *status) {
+    __shared__ unsigned long long tot_units;
+    __shared__ int chunk_units, total_items;
+    int32_t *req_cnt = req_scratch, *req_off = req_scratch + R;
+    if (threadIdx.x == 0) tot_units = 0ull;
+    __syncthreads();
+    for (int r = threadIdx.x; r < R; r += blockDim.x) {
+        const int n_new = qsl[r + 1] - qsl[r];
+        if (n_new <= 0 || n_new > small_max) continue;
+        int mt, tpb, nblk;
+        small_block_shape(n_new, G, mt, tpb, nblk);
+        unsigned long long units = 0;
+        for (int blk = 0; blk < nblk; ++blk) {
+            const int kv_end = seq_lens[r] - n_new + min(n_new, (blk + 1) * tpb);
+            units += (unsigned long long)((kv_end + 63) / 64);
+        }
+        atomicAdd(&tot_units, units * (unsigned long long)Hkv);
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const unsigned long long target = 16ull * (unsigned long long)max(n_sm, 1);
+        chunk_units = (int)max(4ull, (tot_units + target - 1) / target);
+    }
+    __syncthreads();
+    const int chunk = chunk_units;
+    for (int r = threadIdx.x; r < R; r += blockDim.x) {
+        const int n_new = qsl[r + 1] - qsl[r];
+        int cnt = 0;
+        if (n_new > 0 && n_new <= small_max) {
+            int mt, tpb, nblk;
+            small_block_shape(n_new, G, mt, tpb, nblk);
+            for (int blk = 0; blk < nblk; ++blk) {
+                const int kv_end = seq_lens[r] - n_new + min(n_new, (blk + 1) * tpb);
+                cnt += (((kv_end + 63) / 64) + chunk - 1) / chunk;
+            }
+            cnt *= Hkv;
+        }
+        req_cnt[r] = cnt;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int acc = 0;
+        for (int r = 0; r < R; ++r) { req_off[r] = acc; acc += req_cnt[r]; }
+        if (acc > max_items) { report(status, ALORA_ERR_CAPACITY); acc = 0; }
+        total_items = acc;
+        counts[3] = acc;
+    }
+    __syncthreads();
+    if (total_items == 0) return;
+    for (int r = threadIdx.x; r < R; r += blockDim.x) {
+        const int n_new = qsl[r + 1] - qsl[r];
+        if (n_new <= 0 || n_new > small_max) continue;
+        int mt, tpb, nblk;
+        small_block_shape(n_new, G, mt, tpb, nblk);
+        int idx = req_off[r];
+        for (int blk = 0; blk < nblk; ++blk) {
+            const int q_count = min(tpb, n_new - blk * tpb);
+            const int pos0 = seq_lens[r] - n_new + blk * tpb;
+            const int kv_end = pos0 + q_count;   // last token's position + 1
+            const int units = (kv_end + 63) / 64;
+            const int n_splits = (units + chunk - 1) / chunk;
+            for (int kvh = 0; kvh < Hkv; ++kvh)
+                for (int sp = 0; sp < n_splits; ++sp) {
+                    AttnSplitWork w;
+                    w.req = r; w.q_start = qsl[r] + blk * tpb; w.q_count = q_count; w.kv_head = kvh;
+                    w.kv_start = sp * chunk * 64; w.kv_end = min(kv_end, (sp + 1) * chunk * 64);
+                    w.pos0 = pos0; w.mt = mt; w.split = sp; w.n_splits = n_splits; w.pad0_ = 0; w.pad1_ = 0;
+                    items[idx++] = w;
+                }
+        }
+    }
+}
+
 // The whole metadata step as one launch: every block handles 256 tokens; block 0 then builds the two
 // work lists (their serial parts are O(R)).
 __global__ void __launch_bounds__(256)
@@ -195,19 +283,23 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *__restrict
                 int max_tiles, ProjTile *__restrict__ tiles, int32_t *__restrict__ counts, int32_t *seg_scratch,
                 int32_t *__restrict__ shrink_tiles, int32_t *__restrict__ t_ready,
                 int Hkv, int q_block, int max_items, AttnWork *__restrict__ items, int32_t *__restrict__ blk_off,
-                int32_t *status) {
+                int G, int n_sm, int small_max, int max_split_items, AttnSplitWork *__restrict__ split_items,
+                int32_t *__restrict__ req_scratch, int32_t *status) {
     metadata_tokens(positions, a_req, adapter_ids, qsl, seq_lens, block_tables, max_blocks, num_pages, page_size,
                     max_adapters, T, R, mode, token_req, row_adapter, slot_map, status);
     if (blockIdx.x != 0) return;
     metadata_tiles(a_req, adapter_ids, qsl, seq_lens, R, mode, max_adapters, max_tiles, tiles, counts, seg_scratch,
                    shrink_tiles, t_ready, status);
     if (items != nullptr && block_tables != nullptr)
-        metadata_attn_items(qsl, seq_lens, R, Hkv, q_block, max_items, items, counts, blk_off, status);
+        metadata_attn_items(qsl, seq_lens, R, Hkv, q_block, small_max, max_items, items, counts, blk_off, status);
+    if (split_items != nullptr && block_tables != nullptr)
+        metadata_split_items(qsl, seq_lens, R, Hkv, G, n_sm, small_max, max_split_items, split_items, counts,
+                             req_scratch, status);
 }
 
 int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s) {
     if (b.T == 0) {
-        cudaMemsetAsync(ctx->d_counts, 0, 3 * sizeof(int32_t), s);
+        cudaMemsetAsync(ctx->d_counts, 0, 4 * sizeof(int32_t), s);
         return 0;
     }
     ProfScope prof(ctx, KK_METADATA, s);
@@ -217,7 +309,9 @@ int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s) {
         b.max_blocks, b.num_pages, ctx->d.page, ctx->cfg.max_adapters, b.T, b.R, b.mode, ctx->d_token_req,
         ctx->d_row_adapter, ctx->d_slot, ctx->max_tiles, ctx->d_tiles, ctx->d_counts, ctx->d_seg_scratch,
         ctx->d_shrink_tiles, ctx->d_t_ready,
-        ctx->d.Hkv, ctx->attn_q_block, ctx->max_attn_items, ctx->d_attn_items, ctx->d_attn_off, ctx->d_status);
+        ctx->d.Hkv, ctx->attn_q_block, ctx->max_attn_items, ctx->d_attn_items, ctx->d_attn_off, ctx->d.G,
+        ctx->sm_count, ctx->small_max_tokens, ctx->max_split_items, ctx->d_split_items, ctx->d_req_scratch,
+        ctx->d_status);
     return 1;
 }
 

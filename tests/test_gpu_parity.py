@@ -192,6 +192,36 @@ def test_sub_steps_compose_to_the_layer_call(oracle64):
         g.close()
 
 
+def test_projection_with_128_wide_kv_blocks(oracle64):
+    """One KV head of 128 columns: the q/k/v block boundaries force 128-wide column tiles, and the rank-r
+    shrink then runs as the separate cluster split-K kernel."""
+    shape = wl.LayerShape(hidden=1536, n_q_heads=4, n_kv_heads=1, head_dim=128, page_size=16, dtype="bf16")
+    rng = np.random.default_rng(41)
+    w = wl.make_wqkv(shape, rng)
+    ads = [wl.make_adapter(shape, r, rng, scale=s) for r, s in ((64, 1.0), (8, 2.0))]
+    for a in ads:
+        for n in ("Bq", "Bk", "Bv"):
+            setattr(a, n, wl.bf16_round(getattr(a, n) * 8))
+    b = wl.make_batch(shape, [0, 50, 10], [300, 140, 77], [0, 1, 0], rng, activation_offsets=[100, 50, 0])
+    g = hp.GpuLayers(shape, [dict(wqkv=w)], [ads], b.T, b.R)
+    try:
+        d = hp.DevBatch(b, shape.dtype)
+        qkv, base = g.empty(b.T, shape.N), g.empty(b.T, shape.N)
+        for mode, dst in ((ab.MODE_ALORA, qkv), (ab.MODE_BASE, base)):
+            ab.alora_project_qkv(g.ctx, 0, mode, d.hidden, d.positions, d.a_req, d.ids, d.qsl, d.seq_lens, d.T, d.R, dst)
+        assert g.status() == 0
+        want, gate = oracle64.project_qkv(b.hidden, w, shape.Nq, shape.Nkv, b.positions, b.query_start_loc,
+                                          b.activation_offsets, b.adapter_ids, hp.oracle_adapters(ads))
+        qkv_h, base_h = hp.to_host(qkv), hp.to_host(base)
+        assert hp.rel_err(qkv_h, want) <= 2e-2
+        off = gate == 0
+        assert off.sum() == 100 and (~off).sum() > 300
+        assert np.array_equal(qkv_h[off].view(np.uint32), base_h[off].view(np.uint32))
+        assert hp.rel_err(base_h[~off], want[~off]) > 5e-2
+    finally:
+        g.close()
+
+
 def test_full_lora_recompute_matches_eq4(oracle64):
     w, ads, b = _mid_workload(seed=13)
     fb = hp.full_sequence_batch(MID, b)
