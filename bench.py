@@ -163,14 +163,168 @@ def run_reference(args):
     }))
 
 
+def _events(n):
+    import torch
+    return [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
+
+
+def timed(step, n, stream, flush):
+    """Mean CUDA-event duration (ms) of n calls of step() on `stream`, L2 flushed before each call."""
+    import torch
+    ev = _events(n)
+    for e0, e1 in ev:
+        if flush is not None:
+            flush.zero_()
+        e0.record(stream)
+        step()
+        e1.record(stream)
+    torch.cuda.synchronize()
+    return float(np.mean([e0.elapsed_time(e1) for e0, e1 in ev]))
+
+
+def profiled(ab, ctx, step, n, flush):
+    """Per kernel family: mean milliseconds per step over n steps (event pairs recorded by the library)."""
+    import torch
+    ab.alora_profile_enable(ctx, True)
+    for _ in range(n):
+        if flush is not None:
+            flush.zero_()
+        step()
+    torch.cuda.synchronize()
+    prof = ab.alora_profile_read(ctx)
+    ab.alora_profile_enable(ctx, False)
+    return {k: ms / n for k, (ms, cnt) in prof.items() if cnt > 0}
+
+
+class PrefillCase:
+    """Device buffers of one suffix-prefill batch at the 8B layer shape plus its full-LoRA recompute twin."""
+
+    def __init__(self, hp, shape, requests, prefix, suffix, seed, with_recompute):
+        import torch
+        self.w = wl.config2(seed=seed, requests=requests, prefix=prefix, suffix=suffix)
+        b = self.b = self.w.batch
+        self.T, self.R = b.T, b.R
+        self.full_T = int(b.seq_lens.sum())
+        self.d = hp.DevBatch(b, "bf16")
+        g = torch.Generator(device="cuda"); g.manual_seed(seed + 1000)
+        # stands in for the base model's prefix cache: N(0,1) values (the byte and flop counts do not depend on them)
+        self.pool = torch.randn((b.num_pages, 2, shape.n_kv_heads, shape.page_size, shape.head_dim), generator=g,
+                                device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        self.out = torch.empty((self.T, shape.Nq), dtype=torch.bfloat16, device="cuda")
+        if with_recompute:
+            self.fpos = torch.cat([torch.arange(int(n), dtype=torch.int32) for n in b.seq_lens]).cuda()
+            self.fqsl = torch.from_numpy(np.concatenate([[0], np.cumsum(b.seq_lens)]).astype(np.int32)).cuda()
+            self.fhid = torch.randn((self.full_T, shape.hidden), generator=g, device="cuda",
+                                    dtype=torch.float32).to(torch.bfloat16)
+            self.fpool = torch.zeros_like(self.pool)
+            self.fout = torch.empty((self.full_T, shape.Nq), dtype=torch.bfloat16, device="cuda")
+
+    def step(self, ab, ctx, stream):
+        d, b = self.d, self.b
+        ab.alora_prefill_layer(ctx, 0, d.hidden, d.positions, d.a_req, d.ids, d.qsl, d.seq_lens, self.pool, d.bt,
+                               d.max_blocks, b.num_pages, self.T, self.R, self.out, stream)
+
+    def recompute_step(self, ab, ctx, stream):
+        d, b = self.d, self.b
+        ab.alora_full_lora_prefill_layer(ctx, 0, self.fhid, self.fpos, d.ids, self.fqsl, d.seq_lens, self.fpool, d.bt,
+                                         d.max_blocks, b.num_pages, self.full_T, self.R, self.fout, stream)
+
+    def flops_bytes(self, shape, rank):
+        b = self.b
+        H, N, Nq, hd, Hq = shape.hidden, shape.N, shape.Nq, shape.head_dim, shape.n_q_heads
+        P_, S_ = b.prefix_lens.astype(np.int64), (b.seq_lens - b.prefix_lens).astype(np.int64)
+        proj = 2.0 * self.T * H * (N + 3 * rank) + 2.0 * self.T * rank * N
+        pairs = float((S_ * P_ + S_ * (S_ + 1) // 2).sum())
+        attn = 4.0 * hd * Hq * pairs
+        kv_bytes = float(b.seq_lens.sum()) * shape.n_kv_heads * hd * 2 * 2
+        return proj, attn, kv_bytes + 2.0 * self.T * Nq * 2
+
+
+def decode_leg(ab, hp, ctx, shape, stream, flush, peaks, steps=256, seed=5, ctx_max=32768):
+    """Config 5: 64 requests (base + 4 rank-32 adapters), contexts U[1024, 32768], one token per request per
+    step, `steps` steps with the cache growing by one position per step."""
+    import torch
+    rng = np.random.default_rng(seed)
+    R = 64
+    ctx_len = rng.integers(min(1024, ctx_max), ctx_max + 1, R)
+    ids = rng.integers(-1, 4, R).astype(np.int32)
+    a_req = np.maximum(ctx_len - 1 - rng.integers(0, 64, R), 0).astype(np.int32)
+    ps = shape.page_size
+    blocks = (ctx_len + steps + ps - 1) // ps
+    num_pages = int(blocks.sum()) + 3
+    order = rng.permutation(num_pages)
+    bt = np.zeros((R, int(blocks.max())), np.int32)
+    nxt = 0
+    for r in range(R):
+        bt[r, :blocks[r]] = order[nxt:nxt + blocks[r]]
+        nxt += int(blocks[r])
+    g = torch.Generator(device="cuda"); g.manual_seed(seed)
+    pool = torch.empty((num_pages, 2, shape.n_kv_heads, ps, shape.head_dim), device="cuda", dtype=torch.bfloat16)
+    for i in range(0, num_pages, 65536):  # filled in slices: no fp32 copy of the whole pool
+        n = min(65536, num_pages - i)
+        pool[i:i + n] = torch.randn((n,) + tuple(pool.shape[1:]), generator=g, device="cuda",
+                                    dtype=torch.float32).to(torch.bfloat16)
+    hidden = torch.randn((R, shape.hidden), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+    out = torch.empty((R, shape.Nq), dtype=torch.bfloat16, device="cuda")
+    # positions / sequence lengths of every step, resident on the device
+    pos_all = torch.from_numpy((ctx_len[None, :] - 1 + np.arange(steps)[:, None]).astype(np.int32)).cuda()
+    len_all = (pos_all + 1).contiguous()
+    d_bt, d_ids, d_areq = hp.idev(bt), hp.idev(ids), hp.idev(a_req)
+
+    def run(n):
+        for i in range(n):
+            ab.alora_decode_step(ctx, 0, hidden, pos_all[i], d_areq, d_ids, len_all[i], pool, d_bt, bt.shape[1],
+                                 num_pages, R, out, stream)
+    run(8)
+    torch.cuda.synchronize()
+    assert ab.alora_get_status(ctx) == 0, "device-side finding in the decode leg"
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record(stream); run(steps); e1.record(stream)
+    torch.cuda.synchronize()
+    ms = e0.elapsed_time(e1) / steps
+    kern = profiled(ab, ctx, lambda: run(1), 32, None)
+    attn_ms = kern.get("attention", 0.0) + kern.get("attn_merge", 0.0)
+    kv_bytes = float((ctx_len + steps / 2.0).sum()) * shape.n_kv_heads * shape.head_dim * 2 * 2
+    kv_bytes_prof = float(ctx_len.sum()) * shape.n_kv_heads * shape.head_dim * 2 * 2
+    gbs = kv_bytes_prof / (attn_ms / 1e3) / 1e9 if attn_ms else None
+    return {"workload": f"config5: {R} requests, contexts U[1024,{ctx_max}] (mean {ctx_len.mean():.0f}), base + 4 rank-32 "
+                        f"adapters, {steps} steps, shuffled 16-token pages; the {kv_bytes_prof / 1e9:.2f} GB cache read per "
+                        "step exceeds L2",
+            "ms_per_step": ms, "decode_tokens_per_s": R / (ms / 1e3),
+            "kv_bytes_per_step": kv_bytes, "per_kernel_ms": {k: round(v, 4) for k, v in kern.items()},
+            "attention_hbm_gbs": gbs, "attention_frac_of_hbm_peak": gbs / peaks["hbm_gbs"] if gbs else None,
+            "step_hbm_gbs": (kv_bytes + 2.0 * shape.N * shape.hidden) / (ms / 1e3) / 1e9,
+            "peak_source": peaks["source"]}
+
+
+def short_suffix_leg(ab, hp, ctx, shape, stream, flush, peaks, requests, prefix, suffix, seed=7):
+    """The paper-shaped short invocation: `suffix` new tokens per request on a reused cache (HBM-bound attention)."""
+    c = PrefillCase(hp, shape, requests, prefix, suffix, seed, with_recompute=False)
+    for _ in range(5):
+        c.step(ab, ctx, stream)
+    ms = timed(lambda: c.step(ab, ctx, stream), 50, stream, flush)
+    kern = profiled(ab, ctx, lambda: c.step(ab, ctx, stream), 50, flush)
+    attn_ms = kern.get("attention", 0.0) + kern.get("attn_merge", 0.0)
+    _, _, attn_bytes = c.flops_bytes(shape, 32)
+    gbs = attn_bytes / (attn_ms / 1e3) / 1e9 if attn_ms else None
+    return {"requests": requests, "prefix": prefix, "suffix": suffix, "ms_per_step": ms,
+            "tokens_per_s": c.T / (ms / 1e3), "per_kernel_ms": {k: round(v, 4) for k, v in kern.items()},
+            "attention_hbm_gbs": gbs, "attention_frac_of_hbm_peak": gbs / peaks["hbm_gbs"] if gbs else None}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
     ap.add_argument("--steps", type=int, default=200)
     ap.add_argument("--warmup", type=int, default=10)
     ap.add_argument("--impl", default="ours")
-    ap.add_argument("--no-recompute", action="store_true", help="skip the full-LoRA recompute comparison")
+    ap.add_argument("--no-recompute", action="store_true", help="skip the full-LoRA recompute comparisons")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-extra", action="store_true", help="skip the decode and short-suffix legs")
+    ap.add_argument("--legs", default="decode,short,recompute8k",
+                    help="extra legs to run after the main workload (comma list of decode, short, recompute8k)")
+    ap.add_argument("--decode-steps", type=int, default=256)
+    ap.add_argument("--decode-ctx-max", type=int, default=32768)
     ap.add_argument("--requests", type=int, default=8)
     ap.add_argument("--prefix", type=int, default=4096)
     ap.add_argument("--suffix", type=int, default=256)
@@ -197,31 +351,39 @@ def main():
             dist.barrier()
         torch.cuda.synchronize()
 
-    w = wl.config2(seed=SEED, requests=args.requests, prefix=args.prefix, suffix=args.suffix)
-    shape, b = w.shape, w.batch
-    rng = np.random.default_rng(SEED + 1000)
-    pool_np = wl.random_kv_pool(shape, b.num_pages, rng)   # stands in for the base model's prefix cache
-    T, R = b.T, b.R
-    full_T = int(b.seq_lens.sum())
+    def max_over_ranks(x):
+        if world > 1:
+            t = torch.tensor([x], device="cuda")
+            dist.all_reduce(t, op=dist.ReduceOp.MAX)
+            return float(t.item())
+        return x
+
+    shape = wl.SHAPE_8B
+    extra = not args.no_extra and world == 1
+    legs = set(x for x in args.legs.split(",") if x) if extra else set()
+    recomp = not args.no_recompute
+    main_case = PrefillCase(hp, shape, args.requests, args.prefix, args.suffix, SEED, with_recompute=recomp)
+    case_8k = PrefillCase(hp, shape, 8, 8192, 256, SEED + 1, with_recompute=True) if (recomp and "recompute8k" in legs) else None
+    T, R = main_case.T, main_case.R
+    max_tokens = max([T] + ([main_case.full_T] if recomp else []) + ([case_8k.full_T] if case_8k else []))
     cfg = ab.make_config(hidden=shape.hidden, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
-                         head_dim=shape.head_dim, page_size=shape.page_size, max_adapters=1, max_rank=32,
-                         dtype=ab.DTYPE_BF16, device=local, max_tokens=max(T, 0 if args.no_recompute else full_T),
-                         max_requests=R)
+                         head_dim=shape.head_dim, page_size=shape.page_size, max_adapters=4, max_rank=32,
+                         dtype=ab.DTYPE_BF16, device=local, max_tokens=max_tokens, max_requests=max(R, 64))
     ctx = ab.alora_create(cfg)
+    w = main_case.w
     wq = hp.to_dev(w.wqkv, "bf16")
     ab.alora_set_layer_weights(ctx, 0, wq)
-    a = w.adapters[0]
-    mats = [hp.to_dev(getattr(a, n), "bf16") for n in ("Aq", "Bq", "Ak", "Bk", "Av", "Bv")]
-    ab.alora_register_adapter(ctx, 0, 0, a.rank, a.scale, *mats)
-    d = hp.DevBatch(b, "bf16")
-    pool = hp.to_dev(pool_np, "bf16")
-    out = torch.empty((T, shape.Nq), dtype=torch.bfloat16, device="cuda")
+    rng_ad = np.random.default_rng(SEED + 17)
+    adapters = [w.adapters[0]] + [wl.make_adapter(shape, 32, rng_ad) for _ in range(3)]
+    keep = []
+    for i, a in enumerate(adapters):
+        mats = [hp.to_dev(getattr(a, n), "bf16") for n in ("Aq", "Bq", "Ak", "Bk", "Av", "Bv")]
+        keep.append(mats)
+        ab.alora_register_adapter(ctx, i, 0, a.rank, a.scale, *mats)
+    a = adapters[0]
     flush = torch.empty(256 * 1024 * 1024, dtype=torch.uint8, device="cuda")  # > L2 (126 MB)
     stream = torch.cuda.current_stream()
-
-    def step():
-        ab.alora_prefill_layer(ctx, 0, d.hidden, d.positions, d.a_req, d.ids, d.qsl, d.seq_lens, pool, d.bt,
-                               d.max_blocks, b.num_pages, T, R, out, stream)
+    step = lambda: main_case.step(ab, ctx, stream)  # noqa: E731
 
     for _ in range(args.warmup):
         step()
@@ -230,29 +392,17 @@ def main():
 
     # ---- timed region: K steps, each bracketed by CUDA events, L2 flushed between steps ----------
     sampler = ClockSampler(local)
-    ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    ab.alora_profile_enable(ctx, True)
     launches0 = ab.alora_launch_count(ctx)
     barrier()
     sampler.start()
-    for e0, e1 in ev:
-        flush.zero_()
-        e0.record(stream)
-        step()
-        e1.record(stream)
+    step_ms = timed(step, args.steps, stream, flush)
     barrier()
-    clocks = sampler.stop()
     launches = ab.alora_launch_count(ctx) - launches0
-    prof = ab.alora_profile_read(ctx)
-    ab.alora_profile_enable(ctx, False)
-    step_ms = float(np.mean([e0.elapsed_time(e1) for e0, e1 in ev]))
-    if world > 1:
-        tmax = torch.tensor([step_ms], device="cuda")
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        step_ms = float(tmax.item())
+    step_ms = max_over_ranks(step_ms)
     value = world * T / (step_ms / 1e3)
 
     # ---- end to end through the C ABI with host buffers: H2D of the step's inputs, D2H of the result ----
+    d = main_case.d
     h_hidden = d.hidden.cpu().pin_memory()
     ints = [d.positions, d.a_req, d.ids, d.qsl, d.seq_lens, d.bt]
     h_ints = [t.cpu().pin_memory() for t in ints]
@@ -264,38 +414,22 @@ def main():
         d_hidden2.copy_(h_hidden, non_blocking=True)
         for dst, src in zip(d_ints2, h_ints):
             dst.copy_(src, non_blocking=True)
-        ab.alora_prefill_layer(ctx, 0, d_hidden2, d_ints2[0], d_ints2[1], d_ints2[2], d_ints2[3], d_ints2[4], pool,
-                               d_ints2[5], d.max_blocks, b.num_pages, T, R, out, stream)
-        h_out.copy_(out, non_blocking=True)
+        ab.alora_prefill_layer(ctx, 0, d_hidden2, d_ints2[0], d_ints2[1], d_ints2[2], d_ints2[3], d_ints2[4],
+                               main_case.pool, d_ints2[5], d.max_blocks, main_case.b.num_pages, T, R, main_case.out,
+                               stream)
+        h_out.copy_(main_case.out, non_blocking=True)
 
     for _ in range(3):
         e2e_step()
     barrier()
-    e2e_ev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(args.steps)]
-    for e0, e1 in e2e_ev:
-        flush.zero_()
-        e0.record(stream)
-        e2e_step()
-        e1.record(stream)
-    barrier()
-    e2e_ms = float(np.mean([e0.elapsed_time(e1) for e0, e1 in e2e_ev]))
-    if world > 1:
-        tmax = torch.tensor([e2e_ms], device="cuda")
-        dist.all_reduce(tmax, op=dist.ReduceOp.MAX)
-        e2e_ms = float(tmax.item())
+    e2e_ms = max_over_ranks(timed(e2e_step, args.steps, stream, flush))
     h2d = h_hidden.numel() * 2 + sum(t.numel() * 4 for t in h_ints)
     d2h = h_out.numel() * 2
 
-    # ---- roofline of the dominant kernel (per-kernel event times gathered during the timed region) ----
+    # ---- roofline of the dominant kernel: per-kernel event times from a separate profiled pass -----
     peaks = measured_peaks()
-    H, N, Nq, hd, Hq = shape.hidden, shape.N, shape.Nq, shape.head_dim, shape.n_q_heads
-    r = a.rank
-    P_, S_ = b.prefix_lens.astype(np.int64), (b.seq_lens - b.prefix_lens).astype(np.int64)
-    proj_flops = 2.0 * T * H * (N + 3 * r) + 2.0 * T * r * N
-    pairs = float((S_ * P_ + S_ * (S_ + 1) // 2).sum())
-    attn_flops = 4.0 * hd * Hq * pairs
-    attn_bytes = float(b.seq_lens.sum()) * shape.n_kv_heads * hd * 2 * 2 + 2.0 * T * Nq * 2
-    kern = {k: (ms / max(n, 1)) for k, (ms, n) in prof.items() if n > 0}
+    kern = profiled(ab, ctx, step, min(args.steps, 50), flush)
+    proj_flops, attn_flops, attn_bytes = main_case.flops_bytes(shape, a.rank)
     proj_ms = kern.get("project_qkv", 0.0) + kern.get("shrink", 0.0)
     attn_ms = kern.get("attention", 0.0) + kern.get("attn_merge", 0.0)
     dominant = "attention" if attn_ms >= proj_ms else "project_qkv"
@@ -315,34 +449,38 @@ def main():
                               "frac_of_tensor_peak": attn_flops / (attn_ms / 1e3) / 1e12 / peak if attn_ms else None}}
 
     # ---- the comparison path: full-LoRA recompute of prefix + suffix on the same box -------------
-    recompute = None
-    if not args.no_recompute:
-        fpos = torch.cat([torch.arange(int(n), dtype=torch.int32) for n in b.seq_lens]).cuda()
-        fqsl = torch.from_numpy(np.concatenate([[0], np.cumsum(b.seq_lens)]).astype(np.int32)).cuda()
-        g = torch.Generator(device="cuda"); g.manual_seed(SEED)
-        fhid = torch.randn((full_T, H), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
-        fpool = torch.zeros_like(pool)
-        fout = torch.empty((full_T, Nq), dtype=torch.bfloat16, device="cuda")
+    def recompute_of(case, alora_ms):
+        rs = lambda: case.recompute_step(ab, ctx, stream)  # noqa: E731
+        rs(); rs()
+        rms = timed(rs, max(1, min(args.steps, 10)), stream, flush)
+        return {"prefix": int(case.b.prefix_lens[0]), "suffix": int(case.T // case.R), "requests": case.R,
+                "alora_ms_per_step": alora_ms, "full_lora_ms_per_step": rms, "tokens": case.full_T,
+                "speedup_alora_vs_full_lora": rms / alora_ms,
+                "prefix_plus_suffix_over_suffix": float(case.full_T) / case.T}
 
-        def rstep():
-            ab.alora_full_lora_prefill_layer(ctx, 0, fhid, fpos, d.ids, fqsl, d.seq_lens, fpool, d.bt, d.max_blocks,
-                                             b.num_pages, full_T, R, fout, stream)
-        rstep()
-        torch.cuda.synchronize()
-        n_rec = max(1, min(args.steps, 5))
-        rev = [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n_rec)]
-        for e0, e1 in rev:
-            flush.zero_()
-            e0.record(stream); rstep(); e1.record(stream)
-        torch.cuda.synchronize()
-        rms = float(np.mean([e0.elapsed_time(e1) for e0, e1 in rev]))
-        recompute = {"ms_per_step": rms, "tokens": full_T, "speedup_alora_vs_full_lora": rms / step_ms,
-                     "prefix_plus_suffix_over_suffix": float(full_T) / T}
+    recompute = recompute_of(main_case, step_ms) if recomp else None
+    recompute_8k = None
+    if case_8k is not None:
+        s8 = lambda: case_8k.step(ab, ctx, stream)  # noqa: E731
+        for _ in range(5):
+            s8()
+        recompute_8k = recompute_of(case_8k, timed(s8, 50, stream, flush))
+
+    decode = short = None
+    if "decode" in legs:
+        decode = decode_leg(ab, hp, ctx, shape, stream, flush, peaks, steps=args.decode_steps,
+                            ctx_max=args.decode_ctx_max)
+    if "short" in legs:
+        short = [short_suffix_leg(ab, hp, ctx, shape, stream, flush, peaks, r_, 4096, s_)
+                 for r_, s_ in ((8, 4), (8, 16), (64, 4), (64, 16))]
+    clocks = sampler.stop()
     status = ab.alora_get_status(ctx)
     ab.alora_destroy(ctx)
 
     cpu = None
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        pool_np = main_case.pool.to(torch.float32).cpu().numpy()
+        S_ = (main_case.b.seq_lens - main_case.b.prefix_lens)
         rate, threads, dt, done = oracle_sample_rate(w, pool_np, int(S_.max()), requests=range(R), budget_s=20.0)
         cpu = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle",
                "sample": f"{done} of the step's {T} suffix tokens, whole requests in order (projection + attention "
@@ -359,7 +497,8 @@ def main():
             "clocks": clocks, "e2e": {"value": world * T / (e2e_ms / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
                                       "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
             "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
-            "full_lora_recompute": recompute, "device_status": status,
+            "full_lora_recompute": recompute, "full_lora_recompute_8k_prefix": recompute_8k,
+            "decode": decode, "short_suffix": short, "device_status": status,
         }))
     if world > 1:
         dist.destroy_process_group()
