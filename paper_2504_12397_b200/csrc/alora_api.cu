@@ -162,14 +162,17 @@ alora_status alora_create(const alora_config *cfg, alora_ctx **out) {
         alloc((void **)&ctx->d_attn_items, (size_t)ctx->max_attn_items * sizeof(AttnWork));
         alloc((void **)&ctx->d_attn_off, ((size_t)c.max_requests + 1) * 4);
         if (16 % d.G == 0 && (d.hd == 64 || d.hd == 128)) {
-            // few-row attention: at most 16 * n_sm key ranges plus one per (request, KV head, row block)
+            // few-row attention: at most kSplitItemsPerSm * n_sm key ranges plus one per (request, KV head, row
+            // block); a range of mt row tiles owns 16 * mt rows of the partial-result arrays
             ctx->small_max_tokens = 16;
             const int blocks_per_req = std::max(1, (16 * d.G + 63) / 64);
-            ctx->max_split_items = 16 * ctx->sm_count + c.max_requests * blocks_per_req * d.Hkv;
+            const int groups = c.max_requests * blocks_per_req * d.Hkv;
+            ctx->max_split_items = kSplitItemsPerSm * ctx->sm_count + groups;
+            ctx->max_split_rows = 16 * (kSplitItemsPerSm * ctx->sm_count + 4 * groups);
             alloc((void **)&ctx->d_split_items, (size_t)ctx->max_split_items * sizeof(AttnSplitWork));
-            alloc((void **)&ctx->d_req_scratch, (size_t)2 * c.max_requests * 4);
-            alloc((void **)&ctx->d_part_o, (size_t)ctx->max_split_items * 64 * d.hd * 4);
-            alloc((void **)&ctx->d_part_ml, (size_t)ctx->max_split_items * 64 * 2 * 4);
+            alloc((void **)&ctx->d_req_scratch, (size_t)3 * c.max_requests * 4);
+            alloc((void **)&ctx->d_part_o, (size_t)ctx->max_split_rows * d.hd * 4);
+            alloc((void **)&ctx->d_part_ml, (size_t)ctx->max_split_rows * 2 * 4);
         }
     }
     if (c.dtype == ALORA_DTYPE_BF16) {

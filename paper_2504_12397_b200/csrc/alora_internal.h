@@ -63,8 +63,9 @@ struct AttnWork {
 struct AttnSplitWork {
     int32_t req, q_start, q_count, kv_head;
     int32_t kv_start, kv_end, pos0, mt;      // pos0 = position of the first token of the block
-    int32_t split, n_splits, pad0_, pad1_;
+    int32_t split, n_splits, part_row0, pad_;  // part_row0 = first row of this item in the partial-result arrays
 };
+constexpr int kSplitItemsPerSm = 48;   // target number of (row tile, key range) pairs per SM
 
 // Kernel families, for the optional per-kernel timing (alora_profile_*).
 enum KernelKind { KK_METADATA = 0, KK_SHRINK, KK_PROJECT, KK_KV_APPEND, KK_ATTENTION, KK_ATTN_MERGE, KK_LINEAR,
@@ -117,9 +118,9 @@ struct alora_ctx {
     int32_t max_attn_items = 0, attn_q_block = 0;
     // few-row attention (requests with at most small_max_tokens new tokens): split-KV work list and partials
     alora::AttnSplitWork *d_split_items = nullptr;
-    int32_t *d_req_scratch = nullptr;   // [2][max_requests] items per request, item offset per request
+    int32_t *d_req_scratch = nullptr;   // [3][max_requests] items per request, item offset, partial-row offset
     float *d_part_o = nullptr, *d_part_ml = nullptr;
-    int32_t max_split_items = 0, small_max_tokens = 0;
+    int32_t max_split_items = 0, max_split_rows = 0, small_max_tokens = 0;
     void *d_t = nullptr;          // [max_tokens][3][RP] rank-r intermediate
     void *d_qkv = nullptr;        // [max_tokens][N]
     void *d_act[4] = {nullptr, nullptr, nullptr, nullptr};  // stack activations

@@ -6,16 +6,17 @@
 // into key ranges (split-KV) so that a batch of a few requests still fills every SM; ranges of the
 // same rows are merged afterwards by their running maximum and sum (attn_merge_kernel).
 // One persistent block per SM:
-//   warp 4      producer: walks the item list, looks up the pages of the next 64 keys in the block
-//               table and fetches their K and V rows with TMA (one box per page and 64-wide half of
-//               the head dim, 128-byte swizzle) into a 4-deep shared-memory ring; it runs ahead across
+//   warp 8      producer: walks the item list, looks up the pages of the next 64 keys in the block
+//               table and fetches their K and V rows with TMA (one 4-D box per page: both planes and
+//               both 64-wide halves of the head dim, 128-byte swizzle) into a 6-deep shared-memory ring; it runs ahead across
 //               item boundaries, so the HBM stream never drains between items;
-//   warps 0-3   consumers: 16 score rows each (rows are (token, query head of the group) pairs).
+//   warps 0-7   consumers: 16 score rows each (rows are (token, query head of the group) pairs).
 //               Scores with mma.sync m16n8k16 (Q fragments in registers, K fragments by ldmatrix),
 //               online softmax in registers with quad shuffles for the row maximum and sum,
-//               P V with V fragments by ldmatrix.trans.  With 16 rows in the item the four warps take
-//               different 16-key sub-blocks of a stage and combine their partial results through
-//               shared memory at the end of the item; with 32 / 64 rows they take 2 / 1 sub-block sets.
+//               P V with V fragments by ldmatrix.trans.  The 16-key sub-blocks of the ring are dealt
+//               round-robin to the 8 / 4 / 2 warps that share a row tile (16 / 32 / 64 rows in the item);
+//               their partial results are combined through shared memory at the end of the item.
+//               Two warps per scheduler hide each other's dependent chains (score, softmax, P V).
 // Masking is by select (a masked score becomes -inf whatever bits the cache holds), and V rows of keys
 // at or beyond the end of the item's key range are cleared in shared memory before use.
 // All waits are bounded; on expiry ALORA_ERR_TIMEOUT is recorded and the block leaves normally.
@@ -26,9 +27,10 @@
 
 namespace alora {
 
-constexpr int kSkThreads = 160;
+constexpr int kSkConsumerWarps = 8;
+constexpr int kSkThreads = (kSkConsumerWarps + 1) * 32;
 constexpr int kSkStageKeys = 64;
-constexpr int kSkStages = 4;
+constexpr int kSkStages = 6;
 
 struct SplitArgs {
     const AttnSplitWork *items;
@@ -40,8 +42,8 @@ struct SplitArgs {
     float scale_log2;
     const __nv_bfloat16 *qkv;   // [T][N], query part first
     __nv_bfloat16 *out;         // [T][Nq]
-    float *part_o;              // [item][64 rows][HD], unnormalised, relative to the item's maximum
-    float *part_ml;             // [item][64 rows][2]: maximum (scaled, log2 units), sum
+    float *part_o;              // [partial row][HD], unnormalised, relative to the row's maximum in the item
+    float *part_ml;             // [partial row][2]: maximum (scaled, log2 units), sum
     int32_t *status;
 };
 
@@ -49,11 +51,8 @@ template <int HD>
 struct SkSmem {
     static constexpr int kPlaneBytes = kSkStageKeys * HD * 2;    // K or V of one stage
     static constexpr int kStageBytes = 2 * kPlaneBytes;
-    static constexpr int kQStride = HD * 2 + 16;                  // padded query row
-    static constexpr int kQOff = kSkStages * kStageBytes;
-    static constexpr int kQBytes = 4 * 16 * kQStride;             // one 16-row tile per consumer warp
     static constexpr int kOStride = HD + 4;                       // floats
-    static constexpr int kOOff = kQOff + kQBytes;
+    static constexpr int kOOff = kSkStages * kStageBytes;
     static constexpr int kOBytes = 4 * 16 * kOStride * 4;
     static constexpr int kMlOff = kOOff + kOBytes;
     static constexpr int kMlBytes = 4 * 16 * 2 * 4;
@@ -77,20 +76,27 @@ __device__ __forceinline__ void mma_16816(float (&d)[4], uint32_t a0, uint32_t a
                  : "+f"(d[0]), "+f"(d[1]), "+f"(d[2]), "+f"(d[3])
                  : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
 }
+__device__ __forceinline__ void tma_load_4d(uint32_t smem_dst, const CUtensorMap *map, uint32_t bar, int c0, int c1,
+                                            int c2, int c3) {
+    asm volatile(
+        "cp.async.bulk.tensor.4d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%3, %4, %5, %6}], [%2];"
+        ::"r"(smem_dst), "l"((uint64_t)map), "r"(bar), "r"(c0), "r"(c1), "r"(c2), "r"(c3)
+        : "memory");
+}
 __device__ __forceinline__ float ex2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
     return y;
 }
-__device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, 128;" ::: "memory"); }
-// Barrier over the 128 consumer threads that also returns the OR of `pred` over all of them, so that
+__device__ __forceinline__ void consumer_barrier() { asm volatile("bar.sync 1, 256;" ::: "memory"); }
+// Barrier over the 256 consumer threads that also returns the OR of `pred` over all of them, so that
 // every consumer takes the same decision.
 __device__ __forceinline__ bool consumer_barrier_or(bool pred) {
     uint32_t r;
     asm volatile(
         "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.u32 q, %1, 0;\n\t"
-        "bar.red.or.pred p, 1, 128, q;\n\t"
+        "bar.red.or.pred p, 1, 256, q;\n\t"
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(r) : "r"((uint32_t)pred) : "memory");
     return r != 0;
@@ -101,7 +107,12 @@ __global__ void __launch_bounds__(kSkThreads, 1)
 attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmKV, const SplitArgs a) {
     using S = SkSmem<HD>;
     constexpr int kHalves = HD / 64;
-    constexpr int kHalfBytes = kSkStageKeys * 128;   // one 64-wide half of a plane: 64 keys x 128 bytes
+    // A stage holds 64 keys as 64 / box_rows units; one unit is one TMA box:
+    // [plane K, V][64-wide half of the head dim][box_rows keys][128 bytes], 128-byte swizzle inside each half block.
+    const uint32_t half_bytes = (uint32_t)a.box_rows * 128u;
+    const uint32_t plane_bytes = half_bytes * kHalves;
+    const uint32_t unit_bytes = plane_bytes * 2u;
+    const int box_shift = 31 - __clz(a.box_rows);
     constexpr int kKSteps = HD / 16;                 // k-steps of Q K^T
     constexpr int kNTiles = HD / 8;                  // 8-wide output column tiles of P V
     extern __shared__ uint8_t smem_raw[];
@@ -114,7 +125,7 @@ attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmKV, const SplitArgs a)
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        for (int s = 0; s < kSkStages; ++s) { tc::mbar_init(full_bar(s), 1); tc::mbar_init(empty_bar(s), 4); }
+        for (int s = 0; s < kSkStages; ++s) { tc::mbar_init(full_bar(s), 1); tc::mbar_init(empty_bar(s), kSkConsumerWarps); }
         *abort_flag = 0;
         tc::fence_barrier_init();
         tc::fence_proxy_async();
@@ -122,11 +133,10 @@ attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmKV, const SplitArgs a)
     __syncthreads();
     const int n_items = *a.n_items;
 
-    if (warp == 4) {
+    if (warp == kSkConsumerWarps) {
         // ------------------------------ producer ------------------------------
         if (lane == 0) tc::tma_prefetch_desc(&tmKV);
         const int units_per_stage = kSkStageKeys / a.box_rows;
-        const uint32_t unit_bytes = (uint32_t)a.box_rows * 128u;
         uint32_t kt = 0;
         bool ok = true;
         for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
@@ -146,18 +156,12 @@ attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmKV, const SplitArgs a)
                 const unsigned valid = __ballot_sync(0xffffffffu, row >= 0);
                 if (lane == 0) {
                     ok = tc::mbar_wait(empty_bar(st), ((kt / kSkStages) & 1) ^ 1, abort_flag);
-                    if (ok) tc::mbar_arrive_expect_tx(full_bar(st), (uint32_t)__popc(valid) * unit_bytes * kHalves * 2);
+                    if (ok) tc::mbar_arrive_expect_tx(full_bar(st), (uint32_t)__popc(valid) * unit_bytes);
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
                 if (ok && row >= 0) {
-                    const uint32_t dst = smem_base + st * S::kStageBytes + lane * unit_bytes;
-                    const int plane_rows = a.Hkv * a.page_size;  // K plane -> V plane of the same page
-#pragma unroll
-                    for (int plane = 0; plane < 2; ++plane)
-#pragma unroll
-                        for (int h = 0; h < kHalves; ++h)
-                            tc::tma_load_2d(dst + plane * S::kPlaneBytes + h * kHalfBytes, &tmKV, full_bar(st), h * 64,
-                                            row + plane * plane_rows);
+                    // one box: both planes, both halves, box_rows keys of this page and KV head
+                    tma_load_4d(smem_base + st * S::kStageBytes + lane * unit_bytes, &tmKV, full_bar(st), 0, row, 0, 0);
                 }
             }
         }
@@ -171,10 +175,8 @@ attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmKV, const SplitArgs a)
             }
         }
     } else {
-        // ------------------------------ consumers (warps 0..3) ------------------------------
+        // ------------------------------ consumers (warps 0..7) ------------------------------
         const int qr = lane >> 2, qc = lane & 3;          // fragment row (and +8), column pair
-        uint8_t *q_tile = smem_al + S::kQOff + warp * 16 * S::kQStride;
-        const uint32_t q_tile_u32 = smem_base + S::kQOff + warp * 16 * S::kQStride;
         float *o_s = reinterpret_cast<float *>(smem_al + S::kOOff);
         float *ml_s = reinterpret_cast<float *>(smem_al + S::kMlOff);
         uint32_t kt = 0;
@@ -184,30 +186,26 @@ attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmKV, const SplitArgs a)
             const int mt_cnt = w.mt;                  // 1, 2 or 4 row tiles of 16
             const int my_mt = warp % mt_cnt;          // row tile of this warp
             const int kg = warp / mt_cnt;             // which share of the 16-key sub-blocks
-            const int n_kg = 4 / mt_cnt;
+            const int n_kg = kSkConsumerWarps / mt_cnt;   // 8, 4 or 2 key shares
             const int n_st = (w.kv_end - w.kv_start + kSkStageKeys - 1) / kSkStageKeys;
 
-            // ---- this warp's 16 query rows -> shared memory -> A fragments
-            {
-                constexpr int kChunks = HD / 8;  // 16-byte chunks per row
-                for (int i = lane; i < 16 * kChunks; i += 32) {
-                    const int r = i / kChunks, c = i % kChunks;
-                    const int rg = my_mt * 16 + r;
-                    const int tok = rg / a.G;
-                    uint4 v = make_uint4(0, 0, 0, 0);
-                    if (tok < w.q_count)
-                        v = *reinterpret_cast<const uint4 *>(a.qkv + (size_t)(w.q_start + tok) * a.N +
-                                                             (size_t)(w.kv_head * a.G + rg % a.G) * HD + c * 8);
-                    *reinterpret_cast<uint4 *>(q_tile + r * S::kQStride + c * 16) = v;
-                }
-                __syncwarp();
-            }
+            // ---- this warp's 16 query rows as A fragments, straight from global memory (4 KB per warp and item):
+            // registers 0 / 1 hold rows qr / qr + 8 at columns 16 ks + 2 qc, registers 2 / 3 the same rows 8 columns on
             uint32_t qa[kKSteps][4];
+            {
+                const int rg_lo = my_mt * 16 + qr, rg_hi = rg_lo + 8;
+                const bool v_lo = rg_lo / a.G < w.q_count, v_hi = rg_hi / a.G < w.q_count;
+                const uint32_t *q_lo = reinterpret_cast<const uint32_t *>(
+                    a.qkv + (size_t)(w.q_start + (v_lo ? rg_lo / a.G : 0)) * a.N + (size_t)(w.kv_head * a.G + rg_lo % a.G) * HD);
+                const uint32_t *q_hi = reinterpret_cast<const uint32_t *>(
+                    a.qkv + (size_t)(w.q_start + (v_hi ? rg_hi / a.G : 0)) * a.N + (size_t)(w.kv_head * a.G + rg_hi % a.G) * HD);
 #pragma unroll
-            for (int ks = 0; ks < kKSteps; ++ks) {
-                const int r = (lane & 7) + ((lane >> 3) & 1) * 8;
-                const int c = ks * 2 + (lane >> 4);
-                ldsm_x4(q_tile_u32 + r * S::kQStride + c * 16, qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3]);
+                for (int ks = 0; ks < kKSteps; ++ks) {
+                    qa[ks][0] = v_lo ? __ldg(q_lo + ks * 8 + qc) : 0u;
+                    qa[ks][1] = v_hi ? __ldg(q_hi + ks * 8 + qc) : 0u;
+                    qa[ks][2] = v_lo ? __ldg(q_lo + ks * 8 + 4 + qc) : 0u;
+                    qa[ks][3] = v_hi ? __ldg(q_hi + ks * 8 + 4 + qc) : 0u;
+                }
             }
             // causal limits of this thread's two rows (clamped to the item's key range)
             const int tok_lo = min((my_mt * 16 + qr) / a.G, w.q_count - 1);
@@ -224,20 +222,22 @@ attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmKV, const SplitArgs a)
                 const int st = kt % kSkStages;
                 if (!__all_sync(0xffffffffu, tc::mbar_wait(full_bar(st), (kt / kSkStages) & 1, abort_flag))) { ok = false; break; }
                 const uint32_t k_u32 = smem_base + st * S::kStageBytes;
-                const uint32_t v_u32 = k_u32 + S::kPlaneBytes;
                 const int kbase = w.kv_start + j * kSkStageKeys;
 #pragma unroll 1
-                for (int sb = kg; sb < 4; sb += n_kg) {
+                for (int sb = 0; sb < 4; ++sb) {
+                    // 16-key sub-blocks are dealt round-robin over the key shares, across stages
+                    if (((j * 4 + sb) & (n_kg - 1)) != kg) continue;
                     const int k0 = kbase + sb * 16;
                     if (k0 >= w.kv_end) break;
                     if (k0 + 16 > w.kv_end) {
                         // rows of keys beyond the range may hold anything: clear their V rows
-                        uint8_t *v_gen = smem_al + st * S::kStageBytes + S::kPlaneBytes;
+                        uint8_t *v_gen = smem_al + st * S::kStageBytes + plane_bytes;
                         for (int i = lane; i < 16 * 8 * kHalves; i += 32) {
                             const int r = i / (8 * kHalves), c = i % (8 * kHalves);
+                            const int key_l = sb * 16 + r;
                             if (k0 + r >= w.kv_end)
-                                *reinterpret_cast<uint4 *>(v_gen + (c / 8) * kHalfBytes + (sb * 16 + r) * 128 + (c % 8) * 16) =
-                                    make_uint4(0, 0, 0, 0);
+                                *reinterpret_cast<uint4 *>(v_gen + (key_l >> box_shift) * unit_bytes + (c / 8) * half_bytes +
+                                                           (key_l & (a.box_rows - 1)) * 128 + (c % 8) * 16) = make_uint4(0, 0, 0, 0);
                         }
                         tc::fence_proxy_async();
                         __syncwarp();
@@ -248,13 +248,13 @@ attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmKV, const SplitArgs a)
                     for (int n = 0; n < 2; ++n) { s[n][0] = 0.f; s[n][1] = 0.f; s[n][2] = 0.f; s[n][3] = 0.f; }
                     {
                         const int key_l = sb * 16 + (lane >> 4) * 8 + (lane & 7);
-                        const uint32_t krow = k_u32 + key_l * 128;
+                        const uint32_t krow = k_u32 + (key_l >> box_shift) * unit_bytes + (key_l & (a.box_rows - 1)) * 128;
                         const int sw = key_l & 7;
 #pragma unroll
                         for (int ks = 0; ks < kKSteps; ++ks) {
                             const int chunk = 2 * (ks & 3) + ((lane >> 3) & 1);
                             uint32_t b0, b1, b2, b3;
-                            ldsm_x4(krow + (ks >> 2) * kHalfBytes + ((chunk ^ sw) << 4), b0, b1, b2, b3);
+                            ldsm_x4(krow + (ks >> 2) * half_bytes + ((chunk ^ sw) << 4), b0, b1, b2, b3);
                             mma_16816(s[0], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b0, b1);
                             mma_16816(s[1], qa[ks][0], qa[ks][1], qa[ks][2], qa[ks][3], b2, b3);
                         }
@@ -298,13 +298,14 @@ attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmKV, const SplitArgs a)
                     const uint32_t pa2 = tc::pack_bf16(s[1][0], s[1][1]), pa3 = tc::pack_bf16(s[1][2], s[1][3]);
                     {
                         const int key_l = sb * 16 + ((lane >> 3) & 1) * 8 + (lane & 7);
-                        const uint32_t vrow = v_u32 + key_l * 128;
+                        const uint32_t vrow = k_u32 + plane_bytes + (key_l >> box_shift) * unit_bytes +
+                                              (key_l & (a.box_rows - 1)) * 128;
                         const int sw = key_l & 7;
 #pragma unroll
                         for (int cp = 0; cp < kNTiles / 2; ++cp) {
                             const int c16 = 2 * cp + (lane >> 4);
                             uint32_t b0, b1, b2, b3;
-                            ldsm_x4_trans(vrow + (c16 >> 3) * kHalfBytes + (((c16 & 7) ^ sw) << 4), b0, b1, b2, b3);
+                            ldsm_x4_trans(vrow + (c16 >> 3) * half_bytes + (((c16 & 7) ^ sw) << 4), b0, b1, b2, b3);
                             mma_16816(o[2 * cp], pa0, pa1, pa2, pa3, b0, b1);
                             mma_16816(o[2 * cp + 1], pa0, pa1, pa2, pa3, b2, b3);
                         }
@@ -316,31 +317,57 @@ attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmKV, const SplitArgs a)
             // ---- combine the warps that share a row tile, then store the item's result
             l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 1); l_lo += __shfl_xor_sync(0xffffffffu, l_lo, 2);
             l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 1); l_hi += __shfl_xor_sync(0xffffffffu, l_hi, 2);
-            {
-                float *ow = o_s + warp * 16 * S::kOStride;
+            // warps 4..7 hand their partial result to warps 0..3 (same row tile, same fragment layout) ...
+            if (warp >= 4) {
+                float *ow = o_s + (warp - 4) * 16 * S::kOStride;
 #pragma unroll
                 for (int n = 0; n < kNTiles; ++n) {
                     *reinterpret_cast<float2 *>(ow + qr * S::kOStride + n * 8 + 2 * qc) = make_float2(o[n][0], o[n][1]);
                     *reinterpret_cast<float2 *>(ow + (qr + 8) * S::kOStride + n * 8 + 2 * qc) = make_float2(o[n][2], o[n][3]);
                 }
                 if (qc == 0) {
-                    ml_s[(warp * 16 + qr) * 2] = m_lo; ml_s[(warp * 16 + qr) * 2 + 1] = l_lo;
-                    ml_s[(warp * 16 + qr + 8) * 2] = m_hi; ml_s[(warp * 16 + qr + 8) * 2 + 1] = l_hi;
+                    ml_s[((warp - 4) * 16 + qr) * 2] = m_lo; ml_s[((warp - 4) * 16 + qr) * 2 + 1] = l_lo;
+                    ml_s[((warp - 4) * 16 + qr + 8) * 2] = m_hi; ml_s[((warp - 4) * 16 + qr + 8) * 2 + 1] = l_hi;
+                }
+            }
+            consumer_barrier();
+            // ... which fold it into their own and publish the sum for the final combination
+            if (warp < 4) {
+                float *ow = o_s + warp * 16 * S::kOStride;
+                const float m2_lo = ml_s[(warp * 16 + qr) * 2], l2_lo = ml_s[(warp * 16 + qr) * 2 + 1];
+                const float m2_hi = ml_s[(warp * 16 + qr + 8) * 2], l2_hi = ml_s[(warp * 16 + qr + 8) * 2 + 1];
+                const float M_lo = fmaxf(m_lo, m2_lo), M_hi = fmaxf(m_hi, m2_hi);
+                const float mu_lo = M_lo == -INFINITY ? 0.f : M_lo, mu_hi = M_hi == -INFINITY ? 0.f : M_hi;
+                const float a1_lo = ex2(m_lo - mu_lo), a2_lo = ex2(m2_lo - mu_lo);
+                const float a1_hi = ex2(m_hi - mu_hi), a2_hi = ex2(m2_hi - mu_hi);
+                __syncwarp();  // all lanes have read the row statistics before lane qc == 0 rewrites them
+#pragma unroll
+                for (int n = 0; n < kNTiles; ++n) {
+                    float2 *p_lo = reinterpret_cast<float2 *>(ow + qr * S::kOStride + n * 8 + 2 * qc);
+                    float2 *p_hi = reinterpret_cast<float2 *>(ow + (qr + 8) * S::kOStride + n * 8 + 2 * qc);
+                    const float2 v_lo = *p_lo, v_hi = *p_hi;
+                    *p_lo = make_float2(o[n][0] * a1_lo + v_lo.x * a2_lo, o[n][1] * a1_lo + v_lo.y * a2_lo);
+                    *p_hi = make_float2(o[n][2] * a1_hi + v_hi.x * a2_hi, o[n][3] * a1_hi + v_hi.y * a2_hi);
+                }
+                if (qc == 0) {
+                    ml_s[(warp * 16 + qr) * 2] = M_lo; ml_s[(warp * 16 + qr) * 2 + 1] = l_lo * a1_lo + l2_lo * a2_lo;
+                    ml_s[(warp * 16 + qr + 8) * 2] = M_hi; ml_s[(warp * 16 + qr + 8) * 2 + 1] = l_hi * a1_hi + l2_hi * a2_hi;
                 }
             }
             if (consumer_barrier_or(!ok)) break;  // a wait expired somewhere: all consumers leave together
-            {
+            if (warp < 4) {
+                const int n_src = 4 / mt_cnt;             // warps 0..3 that hold the same row tile
                 constexpr int kCols = HD / 8;             // columns per thread: 8 threads cover a row
                 const int t = threadIdx.x;                // 0..127
                 const int r = t >> 3, c0 = (t & 7) * kCols;
                 for (int mt = 0; mt < mt_cnt; ++mt) {
                     float M = -INFINITY;
-                    for (int g = 0; g < n_kg; ++g) M = fmaxf(M, ml_s[((mt + mt_cnt * g) * 16 + r) * 2]);
+                    for (int g = 0; g < n_src; ++g) M = fmaxf(M, ml_s[((mt + mt_cnt * g) * 16 + r) * 2]);
                     const float Mu = M == -INFINITY ? 0.f : M;
                     float L = 0.f, acc[kCols];
 #pragma unroll
                     for (int c = 0; c < kCols; ++c) acc[c] = 0.f;
-                    for (int g = 0; g < n_kg; ++g) {
+                    for (int g = 0; g < n_src; ++g) {
                         const int src = mt + mt_cnt * g;
                         const float wgt = ex2(ml_s[(src * 16 + r) * 2] - Mu);
                         L += ml_s[(src * 16 + r) * 2 + 1] * wgt;
@@ -366,13 +393,13 @@ attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmKV, const SplitArgs a)
                             *reinterpret_cast<uint4 *>(dst + c) = u;
                         }
                     } else {
-                        float *dst = a.part_o + ((size_t)it * 64 + rg) * HD + c0;
+                        float *dst = a.part_o + ((size_t)w.part_row0 + rg) * HD + c0;
 #pragma unroll
                         for (int c = 0; c < kCols; c += 4)
                             *reinterpret_cast<float4 *>(dst + c) = make_float4(acc[c], acc[c + 1], acc[c + 2], acc[c + 3]);
                         if ((t & 7) == 0) {
-                            a.part_ml[((size_t)it * 64 + rg) * 2] = M;
-                            a.part_ml[((size_t)it * 64 + rg) * 2 + 1] = L;
+                            a.part_ml[((size_t)w.part_row0 + rg) * 2] = M;
+                            a.part_ml[((size_t)w.part_row0 + rg) * 2 + 1] = L;
                         }
                     }
                 }
@@ -397,20 +424,21 @@ attn_merge_kernel(const AttnSplitWork *__restrict__ items, const int32_t *__rest
     if (w.split != 0 || w.n_splits <= 1) return;
     constexpr int kCols = HD / 8;
     const int t = threadIdx.x, r = t >> 3, c0 = (t & 7) * kCols;
+    const int rows = 16 * w.mt;  // partial rows per key range of this group
     for (int mt = 0; mt < w.mt; ++mt) {
         const int rg = mt * 16 + r;
         const int tok = rg / G;
         if (tok >= w.q_count) continue;
         float M = -INFINITY;
-        for (int s = 0; s < w.n_splits; ++s) M = fmaxf(M, part_ml[((size_t)(it + s) * 64 + rg) * 2]);
+        for (int s = 0; s < w.n_splits; ++s) M = fmaxf(M, part_ml[((size_t)w.part_row0 + (size_t)s * rows + rg) * 2]);
         float L = 0.f, acc[kCols];
 #pragma unroll
         for (int c = 0; c < kCols; ++c) acc[c] = 0.f;
         for (int s = 0; s < w.n_splits; ++s) {
-            const float *ml = part_ml + ((size_t)(it + s) * 64 + rg) * 2;
+            const float *ml = part_ml + ((size_t)w.part_row0 + (size_t)s * rows + rg) * 2;
             const float wgt = ex2(ml[0] - M);
             L += ml[1] * wgt;
-            const float *src = part_o + ((size_t)(it + s) * 64 + rg) * HD + c0;
+            const float *src = part_o + ((size_t)w.part_row0 + (size_t)s * rows + rg) * HD + c0;
 #pragma unroll
             for (int c = 0; c < kCols; c += 4) {
                 const float4 v = *reinterpret_cast<const float4 *>(src + c);
@@ -443,11 +471,14 @@ int launch_attend_splitkv(alora_ctx *ctx, const void *qkv, const BatchArgs &b, c
     const int box_rows = std::min(d.page, kSkStageKeys);
     CUtensorMap tmKV;
     {
-        cuuint64_t dims[2] = {(cuuint64_t)d.hd, (cuuint64_t)b.num_pages * 2 * d.Hkv * d.page};
-        cuuint64_t strides[1] = {(cuuint64_t)d.hd * 2};
-        cuuint32_t box[2] = {64, (cuuint32_t)box_rows};
-        cuuint32_t es[2] = {1, 1};
-        if (enc(&tmKV, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(pool), dims, strides, box, es,
+        // the pool as (64 columns, cache rows, 64-wide halves of the head dim, K / V plane): one box fetches
+        // box_rows keys of one page and KV head, both halves, both planes
+        const cuuint64_t halves = (cuuint64_t)d.hd / 64;
+        cuuint64_t dims[4] = {64, (cuuint64_t)b.num_pages * 2 * d.Hkv * d.page, halves, 2};
+        cuuint64_t strides[3] = {(cuuint64_t)d.hd * 2, 128, (cuuint64_t)d.Hkv * d.page * d.hd * 2};
+        cuuint32_t box[4] = {64, (cuuint32_t)box_rows, (cuuint32_t)halves, 2};
+        cuuint32_t es[4] = {1, 1, 1, 1};
+        if (enc(&tmKV, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 4, const_cast<void *>(pool), dims, strides, box, es,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return -1;

@@ -187,7 +187,8 @@ __device__ __forceinline__ void metadata_attn_items(const int32_t *__restrict__ 
 // Work list of the few-row attention kernel: requests with 1 .. small_max new tokens.  Their score rows
 // (token, query head of the group) are cut into blocks of 16 * mt rows (mt = 1, 2 or 4 tiles, the
 // smallest that holds all rows, else 4), and the keys 0 .. causal limit of each block into ranges of
-// `chunk` 64-key units, chosen so that about 16 ranges per SM exist in total (at least 256 keys each).
+// `chunk` 64-key units, chosen so that about kSplitItemsPerSm row tiles x ranges per SM exist in total (at
+// least 256 keys each).
 // The ranges of one (block, KV head) are consecutive items.
 __device__ __forceinline__ void small_block_shape(int n_new, int G, int &mt, int &tok_per_blk, int &nblk) {
     const int rows = n_new * G;
@@ -197,14 +198,15 @@ __device__ __forceinline__ void small_block_shape(int n_new, int G, int &mt, int
 }
 
 __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__ qsl, const int32_t *__restrict__ seq_lens,
-                                                     int R, int Hkv, int G, int n_sm, int small_max, int max_items,
+                                                     int R, int Hkv, int G, int n_sm, int small_max, int max_items, int max_rows,
                                                      AttnSplitWork *__restrict__ items, int32_t *__restrict__ counts,
-                                                     int32_t *__restrict__ req_scratch /* [2][R] */, int32_t *status) {
+                                                     int32_t *__restrict__ req_scratch /* [3][R] */, int32_t *status) {
     __shared__ unsigned long long tot_units;
     __shared__ int chunk_units, total_items;
-    int32_t *req_cnt = req_scratch, *req_off = req_scratch + R;
+    int32_t *req_cnt = req_scratch, *req_off = req_scratch + R, *req_row = req_scratch + 2 * R;
     if (threadIdx.x == 0) tot_units = 0ull;
     __syncthreads();
+    // 64-key units of all blocks, weighted by the blocks' row tiles (an item of mt tiles needs mt * 16 partial rows)
     for (int r = threadIdx.x; r < R; r += blockDim.x) {
         const int n_new = qsl[r + 1] - qsl[r];
         if (n_new <= 0 || n_new > small_max) continue;
@@ -215,20 +217,20 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
             const int kv_end = seq_lens[r] - n_new + min(n_new, (blk + 1) * tpb);
             units += (unsigned long long)((kv_end + 63) / 64);
         }
-        atomicAdd(&tot_units, units * (unsigned long long)Hkv);
+        atomicAdd(&tot_units, units * (unsigned long long)(Hkv * mt));
     }
     __syncthreads();
     if (threadIdx.x == 0) {
-        const unsigned long long target = 16ull * (unsigned long long)max(n_sm, 1);
+        const unsigned long long target = (unsigned long long)kSplitItemsPerSm * (unsigned long long)max(n_sm, 1);
         chunk_units = (int)max(4ull, (tot_units + target - 1) / target);
     }
     __syncthreads();
     const int chunk = chunk_units;
     for (int r = threadIdx.x; r < R; r += blockDim.x) {
         const int n_new = qsl[r + 1] - qsl[r];
-        int cnt = 0;
+        int cnt = 0, mt = 1;
         if (n_new > 0 && n_new <= small_max) {
-            int mt, tpb, nblk;
+            int tpb, nblk;
             small_block_shape(n_new, G, mt, tpb, nblk);
             for (int blk = 0; blk < nblk; ++blk) {
                 const int kv_end = seq_lens[r] - n_new + min(n_new, (blk + 1) * tpb);
@@ -237,12 +239,20 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
             cnt *= Hkv;
         }
         req_cnt[r] = cnt;
+        req_row[r] = cnt * 16 * mt;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
-        int acc = 0;
-        for (int r = 0; r < R; ++r) { req_off[r] = acc; acc += req_cnt[r]; }
-        if (acc > max_items) { report(status, ALORA_ERR_CAPACITY); acc = 0; }
+        int acc = 0, rows = 0;
+        for (int r = 0; r < R; ++r) {
+            const int c = req_cnt[r], n = req_row[r];
+            req_off[r] = acc; req_row[r] = rows;
+            acc += c; rows += n;
+        }
+        if (acc > max_items || rows > max_rows) {
+            report(status, ALORA_ERR_CAPACITY);
+            acc = 0;
+        }
         total_items = acc;
         counts[3] = acc;
     }
@@ -253,7 +263,7 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
         if (n_new <= 0 || n_new > small_max) continue;
         int mt, tpb, nblk;
         small_block_shape(n_new, G, mt, tpb, nblk);
-        int idx = req_off[r];
+        int idx = req_off[r], row0 = req_row[r];
         for (int blk = 0; blk < nblk; ++blk) {
             const int q_count = min(tpb, n_new - blk * tpb);
             const int pos0 = seq_lens[r] - n_new + blk * tpb;
@@ -265,8 +275,9 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
                     AttnSplitWork w;
                     w.req = r; w.q_start = qsl[r] + blk * tpb; w.q_count = q_count; w.kv_head = kvh;
                     w.kv_start = sp * chunk * 64; w.kv_end = min(kv_end, (sp + 1) * chunk * 64);
-                    w.pos0 = pos0; w.mt = mt; w.split = sp; w.n_splits = n_splits; w.pad0_ = 0; w.pad1_ = 0;
+                    w.pos0 = pos0; w.mt = mt; w.split = sp; w.n_splits = n_splits; w.part_row0 = row0; w.pad_ = 0;
                     items[idx++] = w;
+                    row0 += 16 * mt;
                 }
         }
     }
@@ -283,7 +294,8 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *__restrict
                 int max_tiles, ProjTile *__restrict__ tiles, int32_t *__restrict__ counts, int32_t *seg_scratch,
                 int32_t *__restrict__ shrink_tiles, int32_t *__restrict__ t_ready,
                 int Hkv, int q_block, int max_items, AttnWork *__restrict__ items, int32_t *__restrict__ blk_off,
-                int G, int n_sm, int small_max, int max_split_items, AttnSplitWork *__restrict__ split_items,
+                int G, int n_sm, int small_max, int max_split_items, int max_split_rows,
+                AttnSplitWork *__restrict__ split_items,
                 int32_t *__restrict__ req_scratch, int32_t *status) {
     metadata_tokens(positions, a_req, adapter_ids, qsl, seq_lens, block_tables, max_blocks, num_pages, page_size,
                     max_adapters, T, R, mode, token_req, row_adapter, slot_map, status);
@@ -293,7 +305,7 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *__restrict
     if (items != nullptr && block_tables != nullptr)
         metadata_attn_items(qsl, seq_lens, R, Hkv, q_block, small_max, max_items, items, counts, blk_off, status);
     if (split_items != nullptr && block_tables != nullptr)
-        metadata_split_items(qsl, seq_lens, R, Hkv, G, n_sm, small_max, max_split_items, split_items, counts,
+        metadata_split_items(qsl, seq_lens, R, Hkv, G, n_sm, small_max, max_split_items, max_split_rows, split_items, counts,
                              req_scratch, status);
 }
 
@@ -310,7 +322,8 @@ int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s) {
         ctx->d_row_adapter, ctx->d_slot, ctx->max_tiles, ctx->d_tiles, ctx->d_counts, ctx->d_seg_scratch,
         ctx->d_shrink_tiles, ctx->d_t_ready,
         ctx->d.Hkv, ctx->attn_q_block, ctx->max_attn_items, ctx->d_attn_items, ctx->d_attn_off, ctx->d.G,
-        ctx->sm_count, ctx->small_max_tokens, ctx->max_split_items, ctx->d_split_items, ctx->d_req_scratch,
+        ctx->sm_count, ctx->small_max_tokens, ctx->max_split_items, ctx->max_split_rows, ctx->d_split_items,
+        ctx->d_req_scratch,
         ctx->d_status);
     return 1;
 }
