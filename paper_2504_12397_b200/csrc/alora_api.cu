@@ -173,6 +173,7 @@ alora_status alora_create(const alora_config *cfg, alora_ctx **out) {
             alloc((void **)&ctx->d_req_scratch, (size_t)3 * c.max_requests * 4);
             alloc((void **)&ctx->d_part_o, (size_t)ctx->max_split_rows * d.hd * 4);
             alloc((void **)&ctx->d_part_ml, (size_t)ctx->max_split_rows * 2 * 4);
+            alloc((void **)&ctx->d_group_done, (size_t)ctx->max_split_items * 4);
         }
     }
     if (c.dtype == ALORA_DTYPE_BF16) {
@@ -223,7 +224,7 @@ alora_status alora_destroy(alora_ctx *ctx) {
     void *ptrs[] = {ctx->d_adapters, ctx->d_token_req, ctx->d_row_adapter, ctx->d_slot, ctx->d_tiles, ctx->d_counts,
                     ctx->d_seg_scratch, ctx->d_shrink_tiles, ctx->d_t_ready, ctx->d_t, ctx->d_qkv, ctx->d_status, ctx->d_act[0], ctx->d_act[1],
                     ctx->d_act[2], ctx->d_act[3], ctx->d_iota, ctx->d_attn_items, ctx->d_attn_off, ctx->d_split_items,
-                    ctx->d_req_scratch, ctx->d_part_o, ctx->d_part_ml};
+                    ctx->d_req_scratch, ctx->d_part_o, ctx->d_part_ml, ctx->d_group_done};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (ctx->h_status) cudaFreeHost(ctx->h_status);
     for (ProfEvent &e : ctx->prof_events) { if (e.begin) cudaEventDestroy(e.begin); if (e.end) cudaEventDestroy(e.end); }

@@ -65,7 +65,7 @@ struct AttnSplitWork {
     int32_t kv_start, kv_end, pos0, mt;      // pos0 = position of the first token of the block
     int32_t split, n_splits, part_row0, pad_;  // part_row0 = first row of this item in the partial-result arrays
 };
-constexpr int kSplitItemsPerSm = 48;   // target number of (row tile, key range) pairs per SM
+constexpr int kSplitItemsPerSm = 16;   // target number of (row tile, key range) pairs per SM
 
 // Kernel families, for the optional per-kernel timing (alora_profile_*).
 enum KernelKind { KK_METADATA = 0, KK_SHRINK, KK_PROJECT, KK_KV_APPEND, KK_ATTENTION, KK_ATTN_MERGE, KK_LINEAR,
@@ -107,7 +107,8 @@ struct alora_ctx {
     // per-call workspaces
     int32_t *d_token_req = nullptr, *d_row_adapter = nullptr, *d_slot = nullptr;
     alora::ProjTile *d_tiles = nullptr;
-    int32_t *d_counts = nullptr;  // [0] projection row tiles, [1] attention work items, [2] row tiles with an adapter
+    int32_t *d_counts = nullptr;  // [0] projection row tiles, [1] attention work items, [2] row tiles with an adapter,
+                                  // [3] few-row attention items, [4] next unclaimed few-row item
     int32_t *d_seg_scratch = nullptr;  // [5][2*max_requests+1] merged row runs of the current batch
     int32_t *d_shrink_tiles = nullptr; // [max_tiles] indices of the row tiles with an adapter
     int32_t *d_t_ready = nullptr;      // [max_tiles] per row tile: epilogue warps that have published t
@@ -120,6 +121,7 @@ struct alora_ctx {
     alora::AttnSplitWork *d_split_items = nullptr;
     int32_t *d_req_scratch = nullptr;   // [3][max_requests] items per request, item offset, partial-row offset
     float *d_part_o = nullptr, *d_part_ml = nullptr;
+    int32_t *d_group_done = nullptr;    // [max_split_items] finished key ranges per group (first item's index)
     int32_t max_split_items = 0, max_split_rows = 0, small_max_tokens = 0;
     void *d_t = nullptr;          // [max_tokens][3][RP] rank-r intermediate
     void *d_qkv = nullptr;        // [max_tokens][N]

@@ -3,9 +3,10 @@
 // is bound by reading the cache from HBM, not by arithmetic.
 //
 // Work item = (request, KV head, block of up to 64 score rows, key range).  Long contexts are cut
-// into key ranges (split-KV) so that a batch of a few requests still fills every SM; ranges of the
-// same rows are merged afterwards by their running maximum and sum (attn_merge_kernel).
-// One persistent block per SM:
+// into key ranges (split-KV) so that a batch of a few requests still fills every SM; the block that
+// finishes the last range of a block of rows merges the ranges by their running maximum and sum.
+// One persistent block per SM; items are claimed from a global counter, so a block that drew short
+// items simply takes more of them:
 //   warp 8      producer: walks the item list, looks up the pages of the next 64 keys in the block
 //               table and fetches their K and V rows with TMA (one 4-D box per page: both planes and
 //               both 64-wide halves of the head dim, 128-byte swizzle) into a 6-deep shared-memory ring; it runs ahead across
@@ -31,6 +32,7 @@ constexpr int kSkConsumerWarps = 8;
 constexpr int kSkThreads = (kSkConsumerWarps + 1) * 32;
 constexpr int kSkStageKeys = 64;
 constexpr int kSkStages = 6;
+constexpr int kSkItemSlots = 4;
 
 struct SplitArgs {
     const AttnSplitWork *items;
@@ -44,6 +46,8 @@ struct SplitArgs {
     __nv_bfloat16 *out;         // [T][Nq]
     float *part_o;              // [partial row][HD], unnormalised, relative to the row's maximum in the item
     float *part_ml;             // [partial row][2]: maximum (scaled, log2 units), sum
+    int32_t *work_counter;      // next unclaimed item (cleared by the metadata step)
+    int32_t *group_done;        // [item] per group (indexed by its first item): key ranges finished so far
     int32_t *status;
 };
 
@@ -57,7 +61,7 @@ struct SkSmem {
     static constexpr int kMlOff = kOOff + kOBytes;
     static constexpr int kMlBytes = 4 * 16 * 2 * 4;
     static constexpr int kBarOff = kMlOff + kMlBytes;
-    static constexpr int kTotal = kBarOff + 128 + 1024;
+    static constexpr int kTotal = kBarOff + 256 + 1024;
 };
 
 __device__ __forceinline__ void ldsm_x4(uint32_t addr, uint32_t &r0, uint32_t &r1, uint32_t &r2, uint32_t &r3) {
@@ -102,6 +106,46 @@ __device__ __forceinline__ bool consumer_barrier_or(bool pred) {
     return r != 0;
 }
 
+// Merge of the key ranges of one block of rows: out = sum_s O_s 2^(m_s - M) / sum_s l_s 2^(m_s - M).
+// `w` is the group's first range; called by 128 threads (threadIdx.x 0..127).
+template <int HD>
+__device__ __forceinline__ void merge_group(const AttnSplitWork w, const float *part_o, const float *part_ml, int G,
+                                            int Nq, __nv_bfloat16 *out) {
+    constexpr int kCols = HD / 8;
+    const int t = threadIdx.x, r = t >> 3, c0 = (t & 7) * kCols;
+    const int rows = 16 * w.mt;  // partial rows per key range of this group
+    for (int mt = 0; mt < w.mt; ++mt) {
+        const int rg = mt * 16 + r;
+        const int tok = rg / G;
+        if (tok >= w.q_count) continue;
+        float M = -INFINITY;
+        for (int s = 0; s < w.n_splits; ++s) M = fmaxf(M, __ldcg(part_ml + ((size_t)w.part_row0 + (size_t)s * rows + rg) * 2));
+        float L = 0.f, acc[kCols];
+#pragma unroll
+        for (int c = 0; c < kCols; ++c) acc[c] = 0.f;
+        for (int s = 0; s < w.n_splits; ++s) {
+            const float *ml = part_ml + ((size_t)w.part_row0 + (size_t)s * rows + rg) * 2;
+            const float wgt = ex2(__ldcg(ml) - M);
+            L += __ldcg(ml + 1) * wgt;
+            const float *src = part_o + ((size_t)w.part_row0 + (size_t)s * rows + rg) * HD + c0;
+#pragma unroll
+            for (int c = 0; c < kCols; c += 4) {
+                const float4 v = __ldcg(reinterpret_cast<const float4 *>(src + c));
+                acc[c] += v.x * wgt; acc[c + 1] += v.y * wgt; acc[c + 2] += v.z * wgt; acc[c + 3] += v.w * wgt;
+            }
+        }
+        const float inv = 1.f / L;
+        __nv_bfloat16 *dst = out + (size_t)(w.q_start + tok) * Nq + (size_t)(w.kv_head * G + rg % G) * HD + c0;
+#pragma unroll
+        for (int c = 0; c < kCols; c += 8) {
+            uint4 u;
+            u.x = tc::pack_bf16(acc[c] * inv, acc[c + 1] * inv); u.y = tc::pack_bf16(acc[c + 2] * inv, acc[c + 3] * inv);
+            u.z = tc::pack_bf16(acc[c + 4] * inv, acc[c + 5] * inv); u.w = tc::pack_bf16(acc[c + 6] * inv, acc[c + 7] * inv);
+            *reinterpret_cast<uint4 *>(dst + c) = u;
+        }
+    }
+}
+
 template <int HD>
 __global__ void __launch_bounds__(kSkThreads, 1)
 attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmKV, const SplitArgs a) {
@@ -121,11 +165,17 @@ attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmKV, const SplitArgs a)
     const uint32_t bar0 = smem_base + S::kBarOff;
     auto full_bar = [&](int s) { return bar0 + 8u * s; };
     auto empty_bar = [&](int s) { return bar0 + 8u * (kSkStages + s); };
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_al + S::kBarOff + 8 * 2 * kSkStages);
+    // claimed item indices travel from the producer to the consumers through a small ring of their own
+    auto item_full = [&](int s) { return bar0 + 8u * (2 * kSkStages + s); };
+    auto item_empty = [&](int s) { return bar0 + 8u * (2 * kSkStages + kSkItemSlots + s); };
+    volatile int *item_ring = reinterpret_cast<volatile int *>(smem_al + S::kBarOff + 8 * (2 * kSkStages + 2 * kSkItemSlots));
+    volatile int *abort_flag = item_ring + kSkItemSlots;
+    volatile int *merge_flag = item_ring + kSkItemSlots + 1;
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
         for (int s = 0; s < kSkStages; ++s) { tc::mbar_init(full_bar(s), 1); tc::mbar_init(empty_bar(s), kSkConsumerWarps); }
+        for (int s = 0; s < kSkItemSlots; ++s) { tc::mbar_init(item_full(s), 1); tc::mbar_init(item_empty(s), kSkConsumerWarps); }
         *abort_flag = 0;
         tc::fence_barrier_init();
         tc::fence_proxy_async();
@@ -137,9 +187,28 @@ attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmKV, const SplitArgs a)
         // ------------------------------ producer ------------------------------
         if (lane == 0) tc::tma_prefetch_desc(&tmKV);
         const int units_per_stage = kSkStageKeys / a.box_rows;
-        uint32_t kt = 0;
+        uint32_t kt = 0, n_it = 0;
         bool ok = true;
-        for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
+        // items are handed out in list order to whichever block is free; the claim of the item after the current
+        // one is issued before the current item's loads, so its latency is hidden behind them
+        int it_next = 0;
+        if (lane == 0) it_next = atomicAdd(a.work_counter, 1);
+        while (ok) {
+            int it = -1;
+            if (lane == 0) {
+                it = it_next < n_items ? it_next : -1;
+                if (it >= 0) it_next = atomicAdd(a.work_counter, 1);
+                const int slot = n_it % kSkItemSlots;
+                ok = tc::mbar_wait(item_empty(slot), ((n_it / kSkItemSlots) & 1) ^ 1, abort_flag);
+                if (ok) {
+                    item_ring[slot] = it;
+                    tc::mbar_arrive(item_full(slot));
+                }
+            }
+            it = __shfl_sync(0xffffffffu, it, 0);
+            ok = __shfl_sync(0xffffffffu, ok, 0);
+            ++n_it;
+            if (!ok || it < 0) break;
             const AttnSplitWork w = a.items[it];
             const int n_st = (w.kv_end - w.kv_start + kSkStageKeys - 1) / kSkStageKeys;
             for (int j = 0; j < n_st && ok; ++j, ++kt) {
@@ -179,9 +248,17 @@ attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmKV, const SplitArgs a)
         const int qr = lane >> 2, qc = lane & 3;          // fragment row (and +8), column pair
         float *o_s = reinterpret_cast<float *>(smem_al + S::kOOff);
         float *ml_s = reinterpret_cast<float *>(smem_al + S::kMlOff);
-        uint32_t kt = 0;
+        uint32_t kt = 0, n_it = 0;
         bool ok = true;
-        for (int it = blockIdx.x; it < n_items; it += gridDim.x) {
+        while (true) {
+            const int slot = n_it % kSkItemSlots;
+            const bool got = __all_sync(0xffffffffu, tc::mbar_wait(item_full(slot), (n_it / kSkItemSlots) & 1, abort_flag));
+            const int it = got ? item_ring[slot] : -1;
+            __syncwarp();
+            if (lane == 0 && got) tc::mbar_arrive(item_empty(slot));
+            ++n_it;
+            if (consumer_barrier_or(!got)) break;     // a wait expired: all consumers leave together
+            if (it < 0) break;                        // the producer found the list exhausted (same value in every warp)
             const AttnSplitWork w = a.items[it];
             const int mt_cnt = w.mt;                  // 1, 2 or 4 row tiles of 16
             const int my_mt = warp % mt_cnt;          // row tile of this warp
@@ -404,57 +481,24 @@ attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmKV, const SplitArgs a)
                     }
                 }
             }
-            consumer_barrier();  // the exchange buffers are rewritten by the next item
+            if (w.n_splits > 1) {
+                // the block that completes the last key range of a group merges the group (ranges in index order,
+                // whichever block does it: the result does not depend on timing)
+                __threadfence();
+                consumer_barrier();
+                if (threadIdx.x == 0) *merge_flag = atomicAdd(a.group_done + (it - w.split), 1) == w.n_splits - 1;
+                consumer_barrier();
+                if (*merge_flag && warp < 4) {
+                    __threadfence();
+                    merge_group<HD>(a.items[it - w.split], a.part_o, a.part_ml, a.G, a.Nq, a.out);
+                }
+            } else {
+                consumer_barrier();  // the exchange buffers are rewritten by the next item
+            }
         }
     }
     __syncthreads();
     if (threadIdx.x == 0 && *abort_flag) report(a.status, ALORA_ERR_TIMEOUT);
-}
-
-// Merge of the key ranges of one block of rows: out = sum_s O_s 2^(m_s - M) / sum_s l_s 2^(m_s - M).
-// One thread block per item; only the block of a group's first range does the work.
-template <int HD>
-__global__ void __launch_bounds__(128)
-attn_merge_kernel(const AttnSplitWork *__restrict__ items, const int32_t *__restrict__ n_items,
-                  const float *__restrict__ part_o, const float *__restrict__ part_ml, int G, int Nq,
-                  __nv_bfloat16 *__restrict__ out) {
-    const int it = blockIdx.x;
-    if (it >= *n_items) return;
-    const AttnSplitWork w = items[it];
-    if (w.split != 0 || w.n_splits <= 1) return;
-    constexpr int kCols = HD / 8;
-    const int t = threadIdx.x, r = t >> 3, c0 = (t & 7) * kCols;
-    const int rows = 16 * w.mt;  // partial rows per key range of this group
-    for (int mt = 0; mt < w.mt; ++mt) {
-        const int rg = mt * 16 + r;
-        const int tok = rg / G;
-        if (tok >= w.q_count) continue;
-        float M = -INFINITY;
-        for (int s = 0; s < w.n_splits; ++s) M = fmaxf(M, part_ml[((size_t)w.part_row0 + (size_t)s * rows + rg) * 2]);
-        float L = 0.f, acc[kCols];
-#pragma unroll
-        for (int c = 0; c < kCols; ++c) acc[c] = 0.f;
-        for (int s = 0; s < w.n_splits; ++s) {
-            const float *ml = part_ml + ((size_t)w.part_row0 + (size_t)s * rows + rg) * 2;
-            const float wgt = ex2(ml[0] - M);
-            L += ml[1] * wgt;
-            const float *src = part_o + ((size_t)w.part_row0 + (size_t)s * rows + rg) * HD + c0;
-#pragma unroll
-            for (int c = 0; c < kCols; c += 4) {
-                const float4 v = *reinterpret_cast<const float4 *>(src + c);
-                acc[c] += v.x * wgt; acc[c + 1] += v.y * wgt; acc[c + 2] += v.z * wgt; acc[c + 3] += v.w * wgt;
-            }
-        }
-        const float inv = 1.f / L;
-        __nv_bfloat16 *dst = out + (size_t)(w.q_start + tok) * Nq + (size_t)(w.kv_head * G + rg % G) * HD + c0;
-#pragma unroll
-        for (int c = 0; c < kCols; c += 8) {
-            uint4 u;
-            u.x = tc::pack_bf16(acc[c] * inv, acc[c + 1] * inv); u.y = tc::pack_bf16(acc[c + 2] * inv, acc[c + 3] * inv);
-            u.z = tc::pack_bf16(acc[c + 4] * inv, acc[c + 5] * inv); u.w = tc::pack_bf16(acc[c + 6] * inv, acc[c + 7] * inv);
-            *reinterpret_cast<uint4 *>(dst + c) = u;
-        }
-    }
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -488,7 +532,8 @@ int launch_attend_splitkv(alora_ctx *ctx, const void *qkv, const BatchArgs &b, c
     a.max_blocks = b.max_blocks; a.num_pages = b.num_pages; a.Hkv = d.Hkv; a.G = d.G; a.page_size = d.page;
     a.box_rows = box_rows; a.N = d.N; a.Nq = d.Nq; a.scale_log2 = d.softmax_scale * 1.4426950408889634f;
     a.qkv = (const __nv_bfloat16 *)qkv; a.out = (__nv_bfloat16 *)out; a.part_o = ctx->d_part_o;
-    a.part_ml = ctx->d_part_ml; a.status = ctx->d_status;
+    a.part_ml = ctx->d_part_ml; a.work_counter = ctx->d_counts + 4; a.group_done = ctx->d_group_done;
+    a.status = ctx->d_status;
     static bool attr_set[2][64] = {};
     const int dev = ctx->cfg.device, hi = d.hd == 128;
     if (dev >= 0 && dev < 64 && !attr_set[hi][dev]) {
@@ -505,12 +550,7 @@ int launch_attend_splitkv(alora_ctx *ctx, const void *qkv, const BatchArgs &b, c
         if (hi) attn_splitkv_kernel<128><<<grid, kSkThreads, SkSmem<128>::kTotal, s>>>(tmKV, a);
         else attn_splitkv_kernel<64><<<grid, kSkThreads, SkSmem<64>::kTotal, s>>>(tmKV, a);
     }
-    {
-        ProfScope prof(ctx, KK_ATTN_MERGE, s);
-        if (hi) attn_merge_kernel<128><<<ctx->max_split_items, 128, 0, s>>>(a.items, a.n_items, a.part_o, a.part_ml, d.G, d.Nq, a.out);
-        else attn_merge_kernel<64><<<ctx->max_split_items, 128, 0, s>>>(a.items, a.n_items, a.part_o, a.part_ml, d.G, d.Nq, a.out);
-    }
-    return 2;
+    return 1;
 }
 
 }  // namespace alora

@@ -187,8 +187,7 @@ __device__ __forceinline__ void metadata_attn_items(const int32_t *__restrict__ 
 // Work list of the few-row attention kernel: requests with 1 .. small_max new tokens.  Their score rows
 // (token, query head of the group) are cut into blocks of 16 * mt rows (mt = 1, 2 or 4 tiles, the
 // smallest that holds all rows, else 4), and the keys 0 .. causal limit of each block into ranges of
-// `chunk` 64-key units, chosen so that about kSplitItemsPerSm row tiles x ranges per SM exist in total (at
-// least 256 keys each).
+// at most `chunk` 64-key units (see the choice of `chunk` below; at most kSplitItemsPerSm ranges per SM).
 // The ranges of one (block, KV head) are consecutive items.
 __device__ __forceinline__ void small_block_shape(int n_new, int G, int &mt, int &tok_per_blk, int &nblk) {
     const int rows = n_new * G;
@@ -200,7 +199,8 @@ __device__ __forceinline__ void small_block_shape(int n_new, int G, int &mt, int
 __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__ qsl, const int32_t *__restrict__ seq_lens,
                                                      int R, int Hkv, int G, int n_sm, int small_max, int max_items, int max_rows,
                                                      AttnSplitWork *__restrict__ items, int32_t *__restrict__ counts,
-                                                     int32_t *__restrict__ req_scratch /* [3][R] */, int32_t *status) {
+                                                     int32_t *__restrict__ req_scratch /* [3][R] */,
+                                                     int32_t *__restrict__ group_done, int32_t *status) {
     __shared__ unsigned long long tot_units;
     __shared__ int chunk_units, total_items;
     int32_t *req_cnt = req_scratch, *req_off = req_scratch + R, *req_row = req_scratch + 2 * R;
@@ -221,7 +221,14 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
     }
     __syncthreads();
     if (threadIdx.x == 0) {
-        const unsigned long long target = (unsigned long long)kSplitItemsPerSm * (unsigned long long)max(n_sm, 1);
+        // Range length: a range costs a fixed few microseconds beyond its streaming time (query fetch, combining
+        // the warps, publishing the partial result), and the last ranges of a launch leave SMs idle for up to one
+        // range.  With t = streaming time of all units on one SM (0.74 us per 64-key unit at an SM's share of
+        // the HBM bandwidth) the sum of both losses is smallest near sqrt(t / 3 us) ranges per SM, capped by the
+        // capacity of the work list.
+        const float t_us = (float)tot_units * 0.74f / (float)max(n_sm, 1);
+        const float per_sm = fminf(fmaxf(sqrtf(t_us / 3.f), 1.f), (float)kSplitItemsPerSm);
+        const unsigned long long target = (unsigned long long)ceilf(per_sm * (float)max(n_sm, 1));
         chunk_units = (int)max(4ull, (tot_units + target - 1) / target);
     }
     __syncthreads();
@@ -255,6 +262,7 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
         }
         total_items = acc;
         counts[3] = acc;
+        counts[4] = 0;   // work counter of the few-row kernel
     }
     __syncthreads();
     if (total_items == 0) return;
@@ -270,12 +278,14 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
             const int kv_end = pos0 + q_count;   // last token's position + 1
             const int units = (kv_end + 63) / 64;
             const int n_splits = (units + chunk - 1) / chunk;
+            const int per = (units + n_splits - 1) / n_splits;   // equal ranges rather than full ones and a stub
             for (int kvh = 0; kvh < Hkv; ++kvh)
                 for (int sp = 0; sp < n_splits; ++sp) {
                     AttnSplitWork w;
                     w.req = r; w.q_start = qsl[r] + blk * tpb; w.q_count = q_count; w.kv_head = kvh;
-                    w.kv_start = sp * chunk * 64; w.kv_end = min(kv_end, (sp + 1) * chunk * 64);
+                    w.kv_start = sp * per * 64; w.kv_end = min(kv_end, (sp + 1) * per * 64);
                     w.pos0 = pos0; w.mt = mt; w.split = sp; w.n_splits = n_splits; w.part_row0 = row0; w.pad_ = 0;
+                    group_done[idx] = 0;
                     items[idx++] = w;
                     row0 += 16 * mt;
                 }
@@ -296,7 +306,7 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *__restrict
                 int Hkv, int q_block, int max_items, AttnWork *__restrict__ items, int32_t *__restrict__ blk_off,
                 int G, int n_sm, int small_max, int max_split_items, int max_split_rows,
                 AttnSplitWork *__restrict__ split_items,
-                int32_t *__restrict__ req_scratch, int32_t *status) {
+                int32_t *__restrict__ req_scratch, int32_t *__restrict__ group_done, int32_t *status) {
     metadata_tokens(positions, a_req, adapter_ids, qsl, seq_lens, block_tables, max_blocks, num_pages, page_size,
                     max_adapters, T, R, mode, token_req, row_adapter, slot_map, status);
     if (blockIdx.x != 0) return;
@@ -306,12 +316,12 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *__restrict
         metadata_attn_items(qsl, seq_lens, R, Hkv, q_block, small_max, max_items, items, counts, blk_off, status);
     if (split_items != nullptr && block_tables != nullptr)
         metadata_split_items(qsl, seq_lens, R, Hkv, G, n_sm, small_max, max_split_items, max_split_rows, split_items, counts,
-                             req_scratch, status);
+                             req_scratch, group_done, status);
 }
 
 int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s) {
     if (b.T == 0) {
-        cudaMemsetAsync(ctx->d_counts, 0, 4 * sizeof(int32_t), s);
+        cudaMemsetAsync(ctx->d_counts, 0, 5 * sizeof(int32_t), s);
         return 0;
     }
     ProfScope prof(ctx, KK_METADATA, s);
@@ -323,7 +333,7 @@ int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s) {
         ctx->d_shrink_tiles, ctx->d_t_ready,
         ctx->d.Hkv, ctx->attn_q_block, ctx->max_attn_items, ctx->d_attn_items, ctx->d_attn_off, ctx->d.G,
         ctx->sm_count, ctx->small_max_tokens, ctx->max_split_items, ctx->max_split_rows, ctx->d_split_items,
-        ctx->d_req_scratch,
+        ctx->d_req_scratch, ctx->d_group_done,
         ctx->d_status);
     return 1;
 }
