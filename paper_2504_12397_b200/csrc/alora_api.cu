@@ -148,7 +148,7 @@ alora_status alora_create(const alora_config *cfg, alora_ctx **out) {
     alloc((void **)&ctx->d_slot, Tm * 4);
     alloc((void **)&ctx->d_tiles, (size_t)ctx->max_tiles * sizeof(ProjTile));
     alloc((void **)&ctx->d_counts, 16 * 4);
-    alloc((void **)&ctx->d_seg_scratch, (size_t)5 * (2 * (size_t)c.max_requests + 1) * 4);
+    alloc((void **)&ctx->d_seg_scratch, ((size_t)14 * c.max_requests + 5) * 4);
     alloc((void **)&ctx->d_shrink_tiles, (size_t)ctx->max_tiles * 4);
     alloc((void **)&ctx->d_t_ready, (size_t)ctx->max_tiles * 4);
     alloc(&ctx->d_t, Tm * 3 * d.RP * 4);
@@ -177,6 +177,7 @@ alora_status alora_create(const alora_config *cfg, alora_ctx **out) {
         }
     }
     if (c.dtype == ALORA_DTYPE_BF16) {
+        alloc((void **)&ctx->d_row_delta, std::min<size_t>(Tm, kRowwiseMaxTokens) * d.N * 4);
         const size_t na = (size_t)std::max(1, c.max_adapters);
         ctx->tc_a_all.assign(c.n_layers, nullptr);
         ctx->tc_b_all.assign(c.n_layers, nullptr);
@@ -224,7 +225,7 @@ alora_status alora_destroy(alora_ctx *ctx) {
     void *ptrs[] = {ctx->d_adapters, ctx->d_token_req, ctx->d_row_adapter, ctx->d_slot, ctx->d_tiles, ctx->d_counts,
                     ctx->d_seg_scratch, ctx->d_shrink_tiles, ctx->d_t_ready, ctx->d_t, ctx->d_qkv, ctx->d_status, ctx->d_act[0], ctx->d_act[1],
                     ctx->d_act[2], ctx->d_act[3], ctx->d_iota, ctx->d_attn_items, ctx->d_attn_off, ctx->d_split_items,
-                    ctx->d_req_scratch, ctx->d_part_o, ctx->d_part_ml, ctx->d_group_done};
+                    ctx->d_req_scratch, ctx->d_part_o, ctx->d_part_ml, ctx->d_group_done, ctx->d_row_delta};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (ctx->h_status) cudaFreeHost(ctx->h_status);
     for (ProfEvent &e : ctx->prof_events) { if (e.begin) cudaEventDestroy(e.begin); if (e.end) cudaEventDestroy(e.end); }

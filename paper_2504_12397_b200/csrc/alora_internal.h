@@ -14,6 +14,7 @@
 namespace alora {
 
 constexpr int kRankPadMax = 64;  // adapters are stored padded to a multiple of 16 rows, <= 64
+constexpr int kRowwiseMaxTokens = 1024;  // largest batch that may take the row-wise delta route of the projection
 constexpr int kMlpChunk = 8192;   // tokens per MLP pass of the stack entry (bounds the gate/up buffer)
 
 // Per (layer, adapter) record as the kernels see it.  A is [3][rpad_max][H] (q, k, v blocks, rows
@@ -108,8 +109,9 @@ struct alora_ctx {
     int32_t *d_token_req = nullptr, *d_row_adapter = nullptr, *d_slot = nullptr;
     alora::ProjTile *d_tiles = nullptr;
     int32_t *d_counts = nullptr;  // [0] projection row tiles, [1] attention work items, [2] row tiles with an adapter,
-                                  // [3] few-row attention items, [4] next unclaimed few-row item
-    int32_t *d_seg_scratch = nullptr;  // [5][2*max_requests+1] merged row runs of the current batch
+                                  // [3] few-row attention items, [4] next unclaimed few-row item,
+                                  // [5] 1 = the projection takes the row-wise route for this batch
+    int32_t *d_seg_scratch = nullptr;  // [14*max_requests+5] per-request values and merged row runs of the current batch
     int32_t *d_shrink_tiles = nullptr; // [max_tiles] indices of the row tiles with an adapter
     int32_t *d_t_ready = nullptr;      // [max_tiles] per row tile: epilogue warps that have published t
     int32_t *d_iota = nullptr;         // 0..max_requests: query_start_loc of a decode batch
@@ -124,6 +126,7 @@ struct alora_ctx {
     int32_t *d_group_done = nullptr;    // [max_split_items] finished key ranges per group (first item's index)
     int32_t max_split_items = 0, max_split_rows = 0, small_max_tokens = 0;
     void *d_t = nullptr;          // [max_tokens][3][RP] rank-r intermediate
+    float *d_row_delta = nullptr; // [min(max_tokens, kRowwiseMaxTokens)][N] fp32 delta rows (bf16 row-wise route)
     void *d_qkv = nullptr;        // [max_tokens][N]
     void *d_act[4] = {nullptr, nullptr, nullptr, nullptr};  // stack activations
     int32_t *d_status = nullptr;

@@ -54,6 +54,12 @@ struct GemmArgs {
     const int32_t *n_shrink_tiles;  // ... and their count (nullptr: no shrink items in this launch)
     int32_t *t_ready;               // [row tile] epilogue warps that have published their part of t
     __nv_bfloat16 *t_out;           // [tokens][192]
+    // Row-wise route (batches of few rows per tile): when *rowwise_flag is set by the metadata step the launch
+    // ignores the tile list, walks dense row tiles without any adapter, and its epilogue adds row_delta[row][n]
+    // (fp32, made by lora_delta_rows_kernel) to the rows whose row_adapter is >= 0.
+    const int32_t *rowwise_flag;
+    const float *row_delta;
+    const int32_t *row_adapter;
     int32_t *status;
 };
 
@@ -66,8 +72,8 @@ struct GemmSmem {
     static constexpr int kTotal = kBarOffset + 256 + 1024;  // barriers + slack for 1024-byte alignment
 };
 
-__device__ __forceinline__ ProjTile load_tile(const GemmArgs &a, int m) {
-    if (a.tiles) return a.tiles[m];
+__device__ __forceinline__ ProjTile load_tile(const GemmArgs &a, int m, bool dense) {
+    if (a.tiles && !dense) return a.tiles[m];
     ProjTile t;
     t.row_start = m * kBM;
     t.row_count = min(kBM, a.M - m * kBM);
@@ -86,7 +92,7 @@ struct GemmItem {
     int n0;       // first output column (projection items)
     bool shrink;
 };
-__device__ __forceinline__ GemmItem decode_item(const GemmArgs &a, int item, int n_shrink, int n_n, int BN) {
+__device__ __forceinline__ GemmItem decode_item(const GemmArgs &a, int item, int n_shrink, int n_n, int BN, bool dense) {
     GemmItem g;
     if (item < n_shrink) {
         g.m = a.shrink_tiles[item];
@@ -98,7 +104,7 @@ __device__ __forceinline__ GemmItem decode_item(const GemmArgs &a, int item, int
         g.n0 = (j % n_n) * BN;
         g.shrink = false;
     }
-    g.t = load_tile(a, g.m);
+    g.t = load_tile(a, g.m, dense);
     return g;
 }
 
@@ -146,9 +152,10 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     tc::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
 
-    const int n_m = a.tiles ? *a.n_row_tiles : (a.M + kBM - 1) / kBM;
+    const bool dense = a.rowwise_flag != nullptr && *a.rowwise_flag != 0;
+    const int n_m = (a.tiles && !dense) ? *a.n_row_tiles : (a.M + kBM - 1) / kBM;
     const int n_n = (a.N + BN - 1) / BN;
-    const int n_shrink = (BN >= kShrinkCols && a.n_shrink_tiles) ? *a.n_shrink_tiles : 0;
+    const int n_shrink = (BN >= kShrinkCols && a.n_shrink_tiles && !dense) ? *a.n_shrink_tiles : 0;
     const int total = n_shrink + n_m * n_n;
     const int kb_main = (a.K + kBK - 1) / kBK;
 
@@ -159,7 +166,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             uint32_t kc = 0;        // ring slots filled so far
             bool ok = true;
             for (int item = blockIdx.x; item < total && ok; item += gridDim.x) {
-                const GemmItem g = decode_item(a, item, n_shrink, n_n, BN);
+                const GemmItem g = decode_item(a, item, n_shrink, n_n, BN, dense);
                 const ProjTile t = g.t;
                 const int n0 = g.n0;
                 const int extra = (!g.shrink && t.adapter >= 0) ? 1 : 0;
@@ -211,7 +218,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             uint32_t kc = 0, it = 0;
             bool ok = true;
             for (int item = blockIdx.x; item < total && ok; item += gridDim.x) {
-                const GemmItem g = decode_item(a, item, n_shrink, n_n, BN);
+                const GemmItem g = decode_item(a, item, n_shrink, n_n, BN, dense);
                 const ProjTile t = g.t;
                 const int extra = (!g.shrink && t.adapter >= 0) ? 1 : 0;
                 const int extra_steps = extra ? a.adapters[t.adapter].rpad / 16 : 0;
@@ -247,7 +254,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         uint32_t it = 0;
         bool ok = true;
         for (int item = blockIdx.x; item < total && ok; item += gridDim.x) {
-            const GemmItem g = decode_item(a, item, n_shrink, n_n, BN);
+            const GemmItem g = decode_item(a, item, n_shrink, n_n, BN, dense);
             const ProjTile t = g.t;
             const int n0 = g.n0;
             const uint32_t acc = it & 1;
@@ -290,6 +297,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             }
             __nv_bfloat16 *orow = a.out + (size_t)(t.row_start + r) * a.ldo + n0;
             const __nv_bfloat16 *rrow = a.residual ? a.residual + (size_t)(t.row_start + r) * a.ldo + n0 : nullptr;
+            // row-wise delta: only rows with an applied adapter add anything (a gated-off row never sees "+ 0")
+            const float *drow = (dense && row_ok && a.row_adapter[t.row_start + r] >= 0)
+                                    ? a.row_delta + (size_t)(t.row_start + r) * a.N + n0 : nullptr;
 #pragma unroll 1
             for (int c = 0; c < BN; c += 32) {
                 uint32_t v[32];
@@ -302,6 +312,12 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         float f[8];
 #pragma unroll
                         for (int e = 0; e < 8; ++e) f[e] = __uint_as_float(v[8 * j + e]);
+                        if (drow) {
+                            const float4 d0 = *reinterpret_cast<const float4 *>(drow + c + 8 * j);
+                            const float4 d1 = *reinterpret_cast<const float4 *>(drow + c + 8 * j + 4);
+                            f[0] += d0.x; f[1] += d0.y; f[2] += d0.z; f[3] += d0.w;
+                            f[4] += d1.x; f[5] += d1.y; f[6] += d1.z; f[7] += d1.w;
+                        }
                         if (rrow) {
                             const uint4 rv = *reinterpret_cast<const uint4 *>(rrow + c + 8 * j);
                             const uint32_t rw[4] = {rv.x, rv.y, rv.z, rv.w};
@@ -386,6 +402,7 @@ static bool launch_gemm_bn(alora_ctx *ctx, const CUtensorMap &tmA, const CUtenso
     return true;
 }
 
+int launch_lora_delta_rows(alora_ctx *ctx, int layer, const void *hidden, int T, cudaStream_t s);  // simt_kernels.cu
 bool launch_shrink_tc(alora_ctx *ctx, const CUtensorMap &tmX, const CUtensorMap &tmA, const AdapterDev *adapters,
                       int K, int max_row_tiles, cudaStream_t s);  // shrink_tcgen05.cu
 
@@ -415,6 +432,13 @@ int launch_project_tc(alora_ctx *ctx, int layer, const void *hidden, int T, void
     const int max_row_tiles = ctx->max_tiles < (T / kBM + 2 * ctx->cfg.max_requests + 2)
                                   ? ctx->max_tiles : (T / kBM + 2 * ctx->cfg.max_requests + 2);
     int n = 0;
+    // Batches whose row tiles would hold only a few rows each may be switched to the row-wise route by the
+    // metadata step (a device-side decision): the delta rows are prepared here, and both kernels read the flag.
+    const bool may_rowwise = have_adapters && T <= kRowwiseMaxTokens && ctx->d_row_delta != nullptr;
+    if (may_rowwise) {
+        ProfScope prof(ctx, KK_SHRINK, s);
+        n += launch_lora_delta_rows(ctx, layer, hidden, T, s);
+    }
     const bool fuse_shrink = have_adapters && BN == 256;
     if (have_adapters && !fuse_shrink) {
         ProfScope prof(ctx, KK_SHRINK, s);
@@ -427,6 +451,9 @@ int launch_project_tc(alora_ctx *ctx, int layer, const void *hidden, int T, void
         g.tiles = ctx->d_tiles; g.n_row_tiles = ctx->d_counts; g.M = T; g.N = d.N; g.K = d.H;
         g.out = (__nv_bfloat16 *)qkv; g.ldo = d.N; g.residual = nullptr; g.adapters = ads;
         g.Nq = d.Nq; g.Nkv = d.Nkv; g.total_adapter_rows = d.N; g.status = ctx->d_status;
+        if (may_rowwise) {
+            g.rowwise_flag = ctx->d_counts + 5; g.row_delta = ctx->d_row_delta; g.row_adapter = ctx->d_row_adapter;
+        }
         if (fuse_shrink) {
             g.shrink_tiles = ctx->d_shrink_tiles; g.n_shrink_tiles = ctx->d_counts + 2;
             g.t_ready = ctx->d_t_ready; g.t_out = (__nv_bfloat16 *)ctx->d_t;

@@ -5,6 +5,7 @@
 namespace alora {
 
 constexpr int kProjTileRows = 128;
+constexpr int kMetaSmemInts = 8192;   // 32 KB: batches of up to 585 requests
 
 // Request owning flat token t: largest r with query_start_loc[r] <= t (binary search; empty
 // requests are skipped because their start equals their successor's).
@@ -70,29 +71,37 @@ __device__ __forceinline__ void metadata_tiles(const int32_t *__restrict__ a_req
                                       const int32_t *__restrict__ qsl, const int32_t *__restrict__ seq_lens,
                                       int R, int mode, int max_adapters, int max_tiles,
                                       ProjTile *__restrict__ tiles, int32_t *__restrict__ counts,
-                                      int32_t *seg_scratch /* [5 * (2R+1)] */, int32_t *__restrict__ shrink_tiles,
+                                      int32_t *seg_scratch /* [14R + 5] */, int T, int rowwise_cap, int32_t *__restrict__ shrink_tiles,
                                       int32_t *__restrict__ t_ready, int32_t *status) {
     int32_t *seg_start = seg_scratch, *seg_len = seg_scratch + (2 * R + 1);
     int32_t *seg_adapter = seg_scratch + 2 * (2 * R + 1), *seg_tile0 = seg_scratch + 3 * (2 * R + 1);
     int32_t *seg_shrink0 = seg_scratch + 4 * (2 * R + 1);  // adapter tiles before the segment
+    int32_t *rq_start = seg_scratch + 5 * (2 * R + 1), *rq_new = rq_start + R, *rq_off = rq_new + R, *rq_k = rq_off + R;
     __shared__ int n_seg, n_tiles;
+    // per request, in parallel: first row, new rows, gated-off rows, adapter
+    for (int r = threadIdx.x; r < R; r += blockDim.x) {
+        const int n_new = qsl[r + 1] - qsl[r];
+        int k = (mode == ALORA_MODE_BASE || adapter_ids == nullptr) ? -1 : adapter_ids[r];
+        if (k >= max_adapters || k < -1) k = -1;
+        int n_off = 0;
+        if (k < 0) n_off = max(n_new, 0);
+        else if (mode == ALORA_MODE_ALORA) {
+            const int p_first = seq_lens[r] - n_new;
+            const long long d = (long long)a_req[r] - p_first;
+            n_off = d <= 0 ? 0 : (d >= n_new ? n_new : (int)d);
+        }
+        rq_start[r] = qsl[r]; rq_new[r] = n_new; rq_off[r] = n_off; rq_k[r] = k;
+    }
+    __syncthreads();
     if (threadIdx.x == 0) {
         int ns = 0, nt = 0;
         for (int r = 0; r < R; ++r) {
-            int n_new = qsl[r + 1] - qsl[r];
+            const int n_new = rq_new[r];
             if (n_new <= 0) continue;
-            int k = (mode == ALORA_MODE_BASE || adapter_ids == nullptr) ? -1 : adapter_ids[r];
-            if (k >= max_adapters || k < -1) k = -1;
-            int n_off = 0;
-            if (k < 0) n_off = n_new;
-            else if (mode == ALORA_MODE_ALORA) {
-                int p_first = seq_lens[r] - n_new;
-                long long d = (long long)a_req[r] - p_first;
-                n_off = d <= 0 ? 0 : (d >= n_new ? n_new : (int)d);
-            }
-            int start[2] = {qsl[r], qsl[r] + n_off};
+            const int n_off = rq_off[r];
+            int start[2] = {rq_start[r], rq_start[r] + n_off};
             int len[2] = {n_off, n_new - n_off};
-            int ad[2] = {-1, k};
+            int ad[2] = {-1, rq_k[r]};
             for (int i = 0; i < 2; ++i) {
                 if (len[i] <= 0) continue;
                 if (ns > 0 && seg_adapter[ns - 1] == ad[i] && seg_start[ns - 1] + seg_len[ns - 1] == start[i]) {
@@ -116,6 +125,10 @@ __device__ __forceinline__ void metadata_tiles(const int32_t *__restrict__ a_req
         n_seg = ns; n_tiles = nt;
         counts[0] = nt;
         counts[2] = n_ad;
+        // Row tiles that hold only a few rows each (decode steps, short suffixes of many requests with different
+        // adapters) waste the tensor cores: when the tiles cover more than twice the batch's rows, the projection
+        // takes the row-wise route (dense row tiles + a per-row delta) instead.
+        counts[5] = (n_ad > 0 && T <= rowwise_cap && (long long)nt * kProjTileRows > 2ll * T + 2 * kProjTileRows) ? 1 : 0;
     }
     __syncthreads();
     for (int i = threadIdx.x; i < n_tiles; i += blockDim.x) {
@@ -144,14 +157,19 @@ __device__ __forceinline__ void metadata_tiles(const int32_t *__restrict__ a_req
 __device__ __forceinline__ void metadata_attn_items(const int32_t *__restrict__ qsl, const int32_t *__restrict__ seq_lens,
                                            int R, int Hkv, int q_block, int small_max, int max_items,
                                            AttnWork *__restrict__ items, int32_t *__restrict__ counts,
-                                           int32_t *__restrict__ blk_off /* [R+1] */, int32_t *status) {
+                                           int32_t *blk_off /* [R+1] */, int32_t *status) {
     __shared__ int total;
+    for (int r = threadIdx.x; r < R; r += blockDim.x) {
+        const int n_new = qsl[r + 1] - qsl[r];
+        blk_off[r] = n_new > small_max ? (n_new + q_block - 1) / q_block : 0;  // short requests: few-row list
+    }
+    __syncthreads();
     if (threadIdx.x == 0) {
         int acc = 0;
         for (int r = 0; r < R; ++r) {
+            const int n = blk_off[r];
             blk_off[r] = acc;
-            const int n_new = qsl[r + 1] - qsl[r];
-            acc += n_new > small_max ? (n_new + q_block - 1) / q_block : 0;  // short requests: few-row list
+            acc += n;
         }
         blk_off[R] = acc;
         int n = acc * Hkv;
@@ -199,7 +217,7 @@ __device__ __forceinline__ void small_block_shape(int n_new, int G, int &mt, int
 __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__ qsl, const int32_t *__restrict__ seq_lens,
                                                      int R, int Hkv, int G, int n_sm, int small_max, int max_items, int max_rows,
                                                      AttnSplitWork *__restrict__ items, int32_t *__restrict__ counts,
-                                                     int32_t *__restrict__ req_scratch /* [3][R] */,
+                                                     int32_t *req_scratch /* [3][R] */,
                                                      int32_t *__restrict__ group_done, int32_t *status) {
     __shared__ unsigned long long tot_units;
     __shared__ int chunk_units, total_items;
@@ -303,17 +321,24 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *__restrict
                 int32_t *__restrict__ token_req, int32_t *__restrict__ row_adapter, int32_t *__restrict__ slot_map,
                 int max_tiles, ProjTile *__restrict__ tiles, int32_t *__restrict__ counts, int32_t *seg_scratch,
                 int32_t *__restrict__ shrink_tiles, int32_t *__restrict__ t_ready,
-                int Hkv, int q_block, int max_items, AttnWork *__restrict__ items, int32_t *__restrict__ blk_off,
+                int Hkv, int q_block, int max_items, AttnWork *__restrict__ items, int32_t *blk_off,
                 int G, int n_sm, int small_max, int max_split_items, int max_split_rows,
                 AttnSplitWork *__restrict__ split_items,
-                int32_t *__restrict__ req_scratch, int32_t *__restrict__ group_done, int32_t *status) {
+                int32_t *req_scratch, int32_t *__restrict__ group_done, int rowwise_cap, int32_t *status) {
     metadata_tokens(positions, a_req, adapter_ids, qsl, seq_lens, block_tables, max_blocks, num_pages, page_size,
                     max_adapters, T, R, mode, token_req, row_adapter, slot_map, status);
     if (blockIdx.x != 0) return;
+    // the per-request scratch of the list builders (their serial parts walk it) lives in shared memory when the
+    // batch is small enough, else in the context's global scratch
+    __shared__ int32_t smem_scratch[kMetaSmemInts];
+    if (14 * R + 5 <= kMetaSmemInts) seg_scratch = blk_off = req_scratch = smem_scratch;
+    __syncthreads();
     metadata_tiles(a_req, adapter_ids, qsl, seq_lens, R, mode, max_adapters, max_tiles, tiles, counts, seg_scratch,
-                   shrink_tiles, t_ready, status);
+                   T, rowwise_cap, shrink_tiles, t_ready, status);
+    __syncthreads();  // the next builder reuses the scratch
     if (items != nullptr && block_tables != nullptr)
         metadata_attn_items(qsl, seq_lens, R, Hkv, q_block, small_max, max_items, items, counts, blk_off, status);
+    __syncthreads();
     if (split_items != nullptr && block_tables != nullptr)
         metadata_split_items(qsl, seq_lens, R, Hkv, G, n_sm, small_max, max_split_items, max_split_rows, split_items, counts,
                              req_scratch, group_done, status);
@@ -321,7 +346,7 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *__restrict
 
 int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s) {
     if (b.T == 0) {
-        cudaMemsetAsync(ctx->d_counts, 0, 5 * sizeof(int32_t), s);
+        cudaMemsetAsync(ctx->d_counts, 0, 6 * sizeof(int32_t), s);
         return 0;
     }
     ProfScope prof(ctx, KK_METADATA, s);
@@ -333,7 +358,7 @@ int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s) {
         ctx->d_shrink_tiles, ctx->d_t_ready,
         ctx->d.Hkv, ctx->attn_q_block, ctx->max_attn_items, ctx->d_attn_items, ctx->d_attn_off, ctx->d.G,
         ctx->sm_count, ctx->small_max_tokens, ctx->max_split_items, ctx->max_split_rows, ctx->d_split_items,
-        ctx->d_req_scratch, ctx->d_group_done,
+        ctx->d_req_scratch, ctx->d_group_done, ctx->d_row_delta ? kRowwiseMaxTokens : 0,
         ctx->d_status);
     return 1;
 }

@@ -65,7 +65,7 @@ shrink_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_cons
                       const ShrinkArgs a) {
     using S = ShrinkSmem;
     // the whole cluster takes the same decision: blockIdx.y selects the row tile
-    if ((int)blockIdx.y >= *a.n_row_tiles) return;
+    if ((int)blockIdx.y >= *a.n_row_tiles || a.n_row_tiles[5] != 0) return;  // [5]: batch takes the row-wise route
     const ProjTile tile = a.tiles[blockIdx.y];
     if (tile.adapter < 0) return;
 

@@ -85,6 +85,96 @@ __global__ void shrink_simt_kernel(const T *__restrict__ x, const int32_t *__res
 }
 
 // ---------------------------------------------------------------------------------------------
+// Row-wise low-rank delta for batches of few rows per adapter (bf16):
+//     delta[row][n] = s * sum_i B[n][i] (A x_row)[blk(n)][i]          (Eq. 5, the term behind the gate)
+// for every row with an applied adapter, in fp32.  One block per (row, q/k/v block): the row of x is staged in
+// shared memory, each warp forms up to 8 of the block's `rank` inner products with A at once (16-byte loads,
+// eight independent loads in flight per lane), then each thread forms outputs of the block's columns from its
+// B rows.  Adapter storage is the rank-padded tensor-core layout A[3][64][H], B[N][64].  The kernel does
+// nothing unless the metadata step chose the row-wise route for this batch (*rowwise_flag).
+// ---------------------------------------------------------------------------------------------
+__global__ void __launch_bounds__(256)
+lora_delta_rows_kernel(const __nv_bfloat16 *__restrict__ x, const int32_t *__restrict__ row_adapter,
+                       const AdapterDev *__restrict__ adapters, const int32_t *__restrict__ rowwise_flag, int H,
+                       int Nq, int Nkv, int N, float *__restrict__ delta) {
+    extern __shared__ uint4 x_s4[];  // H bf16
+    __shared__ float t_s[kRankPadMax];
+    if (*rowwise_flag == 0) return;
+    const int row = blockIdx.x, blk = blockIdx.y;
+    const int k = row_adapter[row];
+    if (k < 0) return;
+    const AdapterDev ad = adapters[k];
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int hv = H / 8;  // 16-byte vectors per row
+    const uint4 *xg = reinterpret_cast<const uint4 *>(x + (size_t)row * H);
+    for (int i = threadIdx.x; i < hv; i += blockDim.x) x_s4[i] = xg[i];
+    __syncthreads();
+    {
+        // outputs warp, warp + 8, ..., below rank (rank <= 64: at most 8 per warp)
+        const uint4 *A4 = reinterpret_cast<const uint4 *>(ad.A) + (size_t)blk * kRankPadMax * hv;
+        float acc[8];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) acc[j] = 0.f;
+        for (int v = lane; v < hv; v += 32) {
+            const uint4 xv = x_s4[v];
+            const __nv_bfloat162 *x2 = reinterpret_cast<const __nv_bfloat162 *>(&xv);
+            float xf[8];
+#pragma unroll
+            for (int e = 0; e < 4; ++e) { const float2 f = __bfloat1622float2(x2[e]); xf[2 * e] = f.x; xf[2 * e + 1] = f.y; }
+            uint4 av[8];
+#pragma unroll
+            for (int j = 0; j < 8; ++j)
+                av[j] = (warp + 8 * j < ad.rank) ? A4[(size_t)(warp + 8 * j) * hv + v] : make_uint4(0, 0, 0, 0);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const __nv_bfloat162 *a2 = reinterpret_cast<const __nv_bfloat162 *>(&av[j]);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 af = __bfloat1622float2(a2[e]);
+                    acc[j] = fmaf(af.x, xf[2 * e], acc[j]);
+                    acc[j] = fmaf(af.y, xf[2 * e + 1], acc[j]);
+                }
+            }
+        }
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            float a = acc[j];
+            for (int off = 16; off; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
+            if (lane == 0 && warp + 8 * j < kRankPadMax) t_s[warp + 8 * j] = (warp + 8 * j < ad.rank) ? a * ad.scale : 0.f;
+        }
+    }
+    __syncthreads();
+    const int n_begin = blk == 0 ? 0 : (blk == 1 ? Nq : Nq + Nkv);
+    const int n_end = blk == 0 ? Nq : (blk == 1 ? Nq + Nkv : N);
+    const uint4 *B4 = reinterpret_cast<const uint4 *>(ad.B);
+    const int rv = (ad.rank + 7) / 8;  // 16-byte vectors of a B row that hold non-zero columns (padding is zero)
+    for (int n = n_begin + threadIdx.x; n < n_end; n += blockDim.x) {
+        const uint4 *brow = B4 + (size_t)n * (kRankPadMax / 8);
+        float acc = 0.f;
+        for (int v = 0; v < rv; ++v) {
+            const uint4 bv = brow[v];
+            const __nv_bfloat162 *b2 = reinterpret_cast<const __nv_bfloat162 *>(&bv);
+#pragma unroll
+            for (int e = 0; e < 4; ++e) {
+                const float2 bf = __bfloat1622float2(b2[e]);
+                acc = fmaf(bf.x, t_s[v * 8 + 2 * e], acc);       // t_s is zero beyond the rank
+                acc = fmaf(bf.y, t_s[v * 8 + 2 * e + 1], acc);
+            }
+        }
+        delta[(size_t)row * N + n] = acc;
+    }
+}
+
+int launch_lora_delta_rows(alora_ctx *ctx, int layer, const void *hidden, int T, cudaStream_t s) {
+    const Dims &d = ctx->d;
+    const AdapterDev *ads = ctx->d_adapters + (size_t)layer * ctx->cfg.max_adapters;
+    lora_delta_rows_kernel<<<dim3(T, 3), 256, (size_t)d.H * 2, s>>>((const __nv_bfloat16 *)hidden, ctx->d_row_adapter, ads,
+                                                                   ctx->d_counts + 5, d.H, d.Nq, d.Nkv, d.N,
+                                                                   ctx->d_row_delta);
+    return 1;
+}
+
+// ---------------------------------------------------------------------------------------------
 // CUDA-core projection y[row][n] = sum_h W[n][h] x[row][h]  (+ sum_i B[n][i] t[row][blk(n)][i] when the
 // row has an applied adapter).  64x64 output tile per block, 16x16 threads, 4x4 outputs each,
 // K staged through shared memory 16 columns at a time.  The base sum of a row is formed by the

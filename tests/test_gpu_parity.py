@@ -192,22 +192,20 @@ def test_sub_steps_compose_to_the_layer_call(oracle64):
         g.close()
 
 
-def test_projection_with_128_wide_kv_blocks(oracle64):
-    """One KV head of 128 columns: the q/k/v block boundaries force 128-wide column tiles, and the rank-r
-    shrink then runs as the separate cluster split-K kernel."""
-    shape = wl.LayerShape(hidden=1536, n_q_heads=4, n_kv_heads=1, head_dim=128, page_size=16, dtype="bf16")
-    rng = np.random.default_rng(41)
-    w = wl.make_wqkv(shape, rng)
-    ads = [wl.make_adapter(shape, r, rng, scale=s) for r, s in ((64, 1.0), (8, 2.0))]
-    for a in ads:
+def _boosted_adapters(shape, rng, spec):
+    ads = [wl.make_adapter(shape, r, rng, scale=s) for r, s in spec]
+    for a in ads:  # lift the delta well above bf16 rounding noise so a wrong or missing delta is visible
         for n in ("Bq", "Bk", "Bv"):
             setattr(a, n, wl.bf16_round(getattr(a, n) * 8))
-    b = wl.make_batch(shape, [0, 50, 10], [300, 140, 77], [0, 1, 0], rng, activation_offsets=[100, 50, 0])
+    return ads
+
+
+def _check_projection(oracle64, shape, w, ads, b, n_off_expected=None):
     g = hp.GpuLayers(shape, [dict(wqkv=w)], [ads], b.T, b.R)
     try:
         d = hp.DevBatch(b, shape.dtype)
-        qkv, base = g.empty(b.T, shape.N), g.empty(b.T, shape.N)
-        for mode, dst in ((ab.MODE_ALORA, qkv), (ab.MODE_BASE, base)):
+        qkv, base, again = g.empty(b.T, shape.N), g.empty(b.T, shape.N), g.empty(b.T, shape.N)
+        for mode, dst in ((ab.MODE_ALORA, qkv), (ab.MODE_BASE, base), (ab.MODE_ALORA, again)):
             ab.alora_project_qkv(g.ctx, 0, mode, d.hidden, d.positions, d.a_req, d.ids, d.qsl, d.seq_lens, d.T, d.R, dst)
         assert g.status() == 0
         want, gate = oracle64.project_qkv(b.hidden, w, shape.Nq, shape.Nkv, b.positions, b.query_start_loc,
@@ -215,11 +213,53 @@ def test_projection_with_128_wide_kv_blocks(oracle64):
         qkv_h, base_h = hp.to_host(qkv), hp.to_host(base)
         assert hp.rel_err(qkv_h, want) <= 2e-2
         off = gate == 0
-        assert off.sum() == 100 and (~off).sum() > 300
+        if n_off_expected is not None:
+            assert off.sum() == n_off_expected
+        assert off.sum() > 0 and (~off).sum() > 0
+        # rows whose gate is closed: bit-identical to the GPU base-only projection (Prop. 1)
         assert np.array_equal(qkv_h[off].view(np.uint32), base_h[off].view(np.uint32))
+        # rows whose gate is open really carry the delta
         assert hp.rel_err(base_h[~off], want[~off]) > 5e-2
+        # run-to-run determinism
+        assert np.array_equal(hp.to_host(again).view(np.uint32), qkv_h.view(np.uint32))
     finally:
         g.close()
+
+
+def test_projection_row_tile_route_with_fused_shrink(oracle64):
+    """Long requests at 256-wide column tiles: row tiles segmented by (adapter, gate), the rank-r shrink
+    running as leading work items of the projection kernel."""
+    rng = np.random.default_rng(43)
+    w = wl.make_wqkv(MID, rng)
+    ads = _boosted_adapters(MID, rng, ((8, 1.0), (64, 0.5), (32, 2.0)))
+    b = wl.make_batch(MID, [0, 300, 20, 5], [500, 390, 130, 260], [1, 0, -1, 2], rng, activation_offsets=[130, 300, 0, 200])
+    _check_projection(oracle64, MID, w, ads, b, n_off_expected=130 + 130 + 195)
+
+
+def test_projection_row_wise_route_many_short_requests(oracle64):
+    """Many requests of 1..9 new tokens over different adapters and the base model, some gated off: the row
+    tiles would hold a few rows each, so the batch takes the row-wise delta route."""
+    rng = np.random.default_rng(44)
+    w = wl.make_wqkv(MID, rng)
+    ads = _boosted_adapters(MID, rng, ((8, 1.0), (64, 0.5), (32, 2.0), (16, 1.0)))
+    R = 40
+    S = [1 + (i * 7) % 9 for i in range(R)]
+    P = [(i * 37) % 200 for i in range(R)]
+    ids = [(i % 5) - 1 for i in range(R)]
+    a_req = [P[i] + (3 if i % 4 == 0 else 0) for i in range(R)]   # every fourth request opens its gate 3 tokens late
+    b = wl.make_batch(MID, P, S, ids, rng, activation_offsets=a_req)
+    _check_projection(oracle64, MID, w, ads, b)
+
+
+def test_projection_with_128_wide_kv_blocks(oracle64):
+    """One KV head of 128 columns: the q/k/v block boundaries force 128-wide column tiles, and the rank-r
+    shrink then runs as the separate cluster split-K kernel."""
+    shape = wl.LayerShape(hidden=1536, n_q_heads=4, n_kv_heads=1, head_dim=128, page_size=16, dtype="bf16")
+    rng = np.random.default_rng(41)
+    w = wl.make_wqkv(shape, rng)
+    ads = _boosted_adapters(shape, rng, ((64, 1.0), (8, 2.0)))
+    b = wl.make_batch(shape, [0, 50, 10], [600, 440, 277], [0, 1, 0], rng, activation_offsets=[100, 50, 0])
+    _check_projection(oracle64, shape, w, ads, b, n_off_expected=100)
 
 
 def test_full_lora_recompute_matches_eq4(oracle64):
