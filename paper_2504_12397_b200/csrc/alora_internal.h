@@ -79,9 +79,9 @@ struct ProfEvent {
 
 // Tensor maps of one layer that depend only on registered weights (bf16 tensor-core path).
 struct TcLayerMaps {
-    CUtensorMap wqkv[2];      // W_qkv [N][H], boxes of 128 / 256 rows
+    CUtensorMap wqkv[3];      // W_qkv [N][H], boxes of 128 / 256 / 64 rows
     CUtensorMap a_all;        // all adapters' A rows [max_adapters*192][H], box 192 rows
-    CUtensorMap b_all_bn[2];  // all adapters' B rows [max_adapters*N][64], boxes of 128 / 256 rows
+    CUtensorMap b_all_bn[3];  // all adapters' B rows [max_adapters*N][64], boxes of 128 / 256 / 64 rows
 };
 
 struct Dims {

@@ -36,7 +36,6 @@ namespace alora {
 
 constexpr int kBM = 128;      // rows per tile (UMMA M)
 constexpr int kBK = 64;       // K elements per ring slot (one 128-byte swizzle row)
-constexpr int kStages = 4;
 constexpr int kGemmThreads = 192;
 constexpr int kTensorRP = 64; // the tensor path stores adapters padded to 64 rank columns
 
@@ -65,6 +64,9 @@ struct GemmArgs {
 
 template <int BN>
 struct GemmSmem {
+    // ring depth: 4 slots of 32 .. 48 KB for the wide tiles; the 64-wide tile of the skinny (few rows, weight
+    // streaming) case gets 8 slots of 24 KB so that enough bytes are in flight per SM
+    static constexpr int kStages = BN <= 64 ? 8 : 4;
     static constexpr int kABytes = kBM * kBK * 2;
     static constexpr int kBBytes = BN * kBK * 2;
     static constexpr int kStageBytes = kABytes + kBBytes;
@@ -121,6 +123,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     const __grid_constant__ CUtensorMap tmT, const __grid_constant__ CUtensorMap tmL,
                     const __grid_constant__ CUtensorMap tmS, const GemmArgs a) {
     using S = GemmSmem<BN>;
+    constexpr int kStages = S::kStages;
     extern __shared__ uint8_t smem_raw[];
     const uint32_t smem_base = (tc::smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t *smem_al = smem_raw + (smem_base - tc::smem_u32(smem_raw));
@@ -389,7 +392,7 @@ template <int BN>
 static bool launch_gemm_bn(alora_ctx *ctx, const CUtensorMap &tmA, const CUtensorMap &tmB, const CUtensorMap &tmT,
                            const CUtensorMap &tmL, const CUtensorMap &tmS, const GemmArgs &args, int max_items,
                            cudaStream_t s) {
-    static bool attr_set[64] = {};
+    static bool attr_set[64] = {};  // one per instantiation
     const int dev = ctx->cfg.device;
     if (dev >= 0 && dev < 64 && !attr_set[dev]) {
         if (cudaFuncSetAttribute(gemm_tcgen05_kernel<BN>, cudaFuncAttributeMaxDynamicSharedMemorySize,
@@ -406,8 +409,10 @@ int launch_lora_delta_rows(alora_ctx *ctx, int layer, const void *hidden, int T,
 bool launch_shrink_tc(alora_ctx *ctx, const CUtensorMap &tmX, const CUtensorMap &tmA, const AdapterDev *adapters,
                       int K, int max_row_tiles, cudaStream_t s);  // shrink_tcgen05.cu
 
-// Picks the column-tile width: 256 when the q/k/v block boundaries allow it, else 128.
-static int pick_bn(int N, int Nq, int Nkv, bool lora) {
+// Picks the column-tile width: 256 when the q/k/v block boundaries allow it, else 128; 64 for batches of at most
+// 128 rows, where the kernel streams the weights once and more, narrower tiles put more SMs to work.
+static int pick_bn(int N, int Nq, int Nkv, bool lora, int T) {
+    if (T <= kBM && N >= 64 * 48 && Nq % 64 == 0 && Nkv % 64 == 0) return 64;
     if (lora) {
         if (Nq % 256 == 0 && Nkv % 256 == 0) return 256;
         if (Nq % 128 == 0 && Nkv % 128 == 0) return 128;
@@ -422,15 +427,15 @@ int launch_project_tc(alora_ctx *ctx, int layer, const void *hidden, int T, void
     if (T == 0) return 0;
     const Dims &d = ctx->d;
     const bool have_adapters = ctx->layer_has_adapter[layer];
-    const int BN = pick_bn(d.N, d.Nq, d.Nkv, true);
+    const int BN = pick_bn(d.N, d.Nq, d.Nkv, true, T);
     if (BN == 0 || d.H % 8 != 0) return -1;
     CUtensorMap tmX, tmTt;
     if (!make_tensor_map_bf16(&tmX, hidden, T, d.H, d.H, kBM)) return -1;
     if (!make_tensor_map_bf16(&tmTt, ctx->d_t, ctx->cfg.max_tokens, 3 * kTensorRP, 3 * kTensorRP, kBM)) return -1;
     const TcLayerMaps &lm = ctx->tc_maps[layer];
     const AdapterDev *ads = ctx->d_adapters + (size_t)layer * ctx->cfg.max_adapters;
-    const int max_row_tiles = ctx->max_tiles < (T / kBM + 2 * ctx->cfg.max_requests + 2)
-                                  ? ctx->max_tiles : (T / kBM + 2 * ctx->cfg.max_requests + 2);
+    // every row tile holds at least one row; a request contributes at most two partial tiles
+    const int max_row_tiles = std::min(std::min(ctx->max_tiles, T / kBM + 2 * ctx->cfg.max_requests + 2), T);
     int n = 0;
     // Batches whose row tiles would hold only a few rows each may be switched to the row-wise route by the
     // metadata step (a device-side decision): the delta rows are prepared here, and both kernels read the flag.
@@ -440,7 +445,8 @@ int launch_project_tc(alora_ctx *ctx, int layer, const void *hidden, int T, void
         n += launch_lora_delta_rows(ctx, layer, hidden, T, s);
     }
     const bool fuse_shrink = have_adapters && BN == 256;
-    if (have_adapters && !fuse_shrink) {
+    // (a batch that fits one row tile always takes the row-wise route when it has adapter rows: no shrink launch)
+    if (have_adapters && !fuse_shrink && !(may_rowwise && T <= kBM)) {
         ProfScope prof(ctx, KK_SHRINK, s);
         if (!launch_shrink_tc(ctx, tmX, lm.a_all, ads, d.H, max_row_tiles, s)) return -1;
         ++n;
@@ -461,7 +467,9 @@ int launch_project_tc(alora_ctx *ctx, int layer, const void *hidden, int T, void
         const int items = max_row_tiles * ((d.N + BN - 1) / BN + (fuse_shrink ? 1 : 0));
         const bool ok = BN == 256
                             ? launch_gemm_bn<256>(ctx, tmX, lm.wqkv[1], tmTt, lm.b_all_bn[1], lm.a_all, g, items, s)
-                            : launch_gemm_bn<128>(ctx, tmX, lm.wqkv[0], tmTt, lm.b_all_bn[0], lm.a_all, g, items, s);
+                            : BN == 128
+                                  ? launch_gemm_bn<128>(ctx, tmX, lm.wqkv[0], tmTt, lm.b_all_bn[0], lm.a_all, g, items, s)
+                                  : launch_gemm_bn<64>(ctx, tmX, lm.wqkv[2], tmTt, lm.b_all_bn[2], lm.a_all, g, items, s);
         if (!ok) return -1;
         ++n;
     }
@@ -474,7 +482,7 @@ int launch_linear_tc(alora_ctx *ctx, const void *x, const void *W, int T, int K,
     if (T == 0) return 0;
     if (K % 8 != 0 || N % 8 != 0) return -1;
     ProfScope prof(ctx, KK_LINEAR, s);
-    const int BN = pick_bn(N, 0, 0, false);
+    const int BN = pick_bn(N, N, 0, false, T);
     CUtensorMap tmX, tmW;
     if (!make_tensor_map_bf16(&tmX, x, T, K, K, kBM)) return -1;
     if (!make_tensor_map_bf16(&tmW, W, N, K, K, BN)) return -1;
@@ -484,7 +492,8 @@ int launch_linear_tc(alora_ctx *ctx, const void *x, const void *W, int T, int K,
     g.total_adapter_rows = 0; g.status = ctx->d_status;
     const int items = ((T + kBM - 1) / kBM) * ((N + BN - 1) / BN);
     const bool ok = BN == 256 ? launch_gemm_bn<256>(ctx, tmX, tmW, tmX, tmW, tmW, g, items, s)
-                              : launch_gemm_bn<128>(ctx, tmX, tmW, tmX, tmW, tmW, g, items, s);
+                    : BN == 128 ? launch_gemm_bn<128>(ctx, tmX, tmW, tmX, tmW, tmW, g, items, s)
+                                : launch_gemm_bn<64>(ctx, tmX, tmW, tmX, tmW, tmW, g, items, s);
     return ok ? 1 : -1;
 }
 
@@ -497,11 +506,13 @@ bool build_layer_maps(alora_ctx *ctx, int layer) {
     if (lw.wqkv) {
         ok &= make_tensor_map_bf16(&lm.wqkv[0], lw.wqkv, d.N, d.H, d.H, 128);
         ok &= make_tensor_map_bf16(&lm.wqkv[1], lw.wqkv, d.N, d.H, d.H, 256);
+        ok &= make_tensor_map_bf16(&lm.wqkv[2], lw.wqkv, d.N, d.H, d.H, 64);
     }
     const size_t na = (size_t)std::max(1, ctx->cfg.max_adapters);
     ok &= make_tensor_map_bf16(&lm.a_all, ctx->tc_a_all[layer], na * 3 * kTensorRP, d.H, d.H, 3 * kTensorRP);
     ok &= make_tensor_map_bf16(&lm.b_all_bn[0], ctx->tc_b_all[layer], na * d.N, kTensorRP, kTensorRP, 128);
     ok &= make_tensor_map_bf16(&lm.b_all_bn[1], ctx->tc_b_all[layer], na * d.N, kTensorRP, kTensorRP, 256);
+    ok &= make_tensor_map_bf16(&lm.b_all_bn[2], ctx->tc_b_all[layer], na * d.N, kTensorRP, kTensorRP, 64);
     return ok;
 }
 

@@ -5,7 +5,8 @@
 namespace alora {
 
 constexpr int kProjTileRows = 128;
-constexpr int kMetaSmemInts = 8192;   // 32 KB: batches of up to 585 requests
+constexpr int kMetaSmemInts = 7168;   // 28 KB of builder scratch: batches of up to 511 requests
+constexpr int kMetaStageR = 1024;     // per-request inputs of up to this many requests are staged in shared memory
 
 // Request owning flat token t: largest r with query_start_loc[r] <= t (binary search; empty
 // requests are skipped because their start equals their successor's).
@@ -95,23 +96,29 @@ __device__ __forceinline__ void metadata_tiles(const int32_t *__restrict__ a_req
     __syncthreads();
     if (threadIdx.x == 0) {
         int ns = 0, nt = 0;
+        int cur_start = 0, cur_len = 0, cur_ad = -1;   // the run being grown, kept in registers
+        bool have = false;
+#pragma unroll 4
         for (int r = 0; r < R; ++r) {
             const int n_new = rq_new[r];
             if (n_new <= 0) continue;
             const int n_off = rq_off[r];
-            int start[2] = {rq_start[r], rq_start[r] + n_off};
-            int len[2] = {n_off, n_new - n_off};
-            int ad[2] = {-1, rq_k[r]};
+            const int start[2] = {rq_start[r], rq_start[r] + n_off};
+            const int len[2] = {n_off, n_new - n_off};
+            const int ad[2] = {-1, rq_k[r]};
+#pragma unroll
             for (int i = 0; i < 2; ++i) {
                 if (len[i] <= 0) continue;
-                if (ns > 0 && seg_adapter[ns - 1] == ad[i] && seg_start[ns - 1] + seg_len[ns - 1] == start[i]) {
-                    seg_len[ns - 1] += len[i];
+                if (have && cur_ad == ad[i] && cur_start + cur_len == start[i]) {
+                    cur_len += len[i];
                 } else {
-                    seg_start[ns] = start[i]; seg_len[ns] = len[i]; seg_adapter[ns] = ad[i];
-                    ++ns;
+                    if (have) { seg_start[ns] = cur_start; seg_len[ns] = cur_len; seg_adapter[ns] = cur_ad; ++ns; }
+                    cur_start = start[i]; cur_len = len[i]; cur_ad = ad[i];
+                    have = true;
                 }
             }
         }
+        if (have) { seg_start[ns] = cur_start; seg_len[ns] = cur_len; seg_adapter[ns] = cur_ad; ++ns; }
         int n_ad = 0;
         for (int s = 0; s < ns; ++s) {
             seg_tile0[s] = nt;
@@ -126,9 +133,11 @@ __device__ __forceinline__ void metadata_tiles(const int32_t *__restrict__ a_req
         counts[0] = nt;
         counts[2] = n_ad;
         // Row tiles that hold only a few rows each (decode steps, short suffixes of many requests with different
-        // adapters) waste the tensor cores: when the tiles cover more than twice the batch's rows, the projection
-        // takes the row-wise route (dense row tiles + a per-row delta) instead.
-        counts[5] = (n_ad > 0 && T <= rowwise_cap && (long long)nt * kProjTileRows > 2ll * T + 2 * kProjTileRows) ? 1 : 0;
+        // adapters) waste the tensor cores: when the tiles cover more than twice the batch's rows, and always when
+        // the whole batch fits one row tile, the projection takes the row-wise route (dense row tiles + a per-row
+        // delta) instead.
+        const bool wasteful = (long long)nt * kProjTileRows > 2ll * T + 2 * kProjTileRows;
+        counts[5] = (n_ad > 0 && T <= rowwise_cap && (T <= kProjTileRows || wasteful)) ? 1 : 0;
     }
     __syncthreads();
     for (int i = threadIdx.x; i < n_tiles; i += blockDim.x) {
@@ -222,20 +231,28 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
     __shared__ unsigned long long tot_units;
     __shared__ int chunk_units, total_items;
     int32_t *req_cnt = req_scratch, *req_off = req_scratch + R, *req_row = req_scratch + 2 * R;
-    if (threadIdx.x == 0) tot_units = 0ull;
-    __syncthreads();
-    // 64-key units of all blocks, weighted by the blocks' row tiles (an item of mt tiles needs mt * 16 partial rows)
+    // 64-key units of all blocks, weighted by the blocks' row tiles (an item of mt tiles needs mt * 16 partial rows):
+    // per request in parallel, summed by one thread (a shared 64-bit atomic under contention is far slower)
     for (int r = threadIdx.x; r < R; r += blockDim.x) {
         const int n_new = qsl[r + 1] - qsl[r];
-        if (n_new <= 0 || n_new > small_max) continue;
-        int mt, tpb, nblk;
-        small_block_shape(n_new, G, mt, tpb, nblk);
-        unsigned long long units = 0;
-        for (int blk = 0; blk < nblk; ++blk) {
-            const int kv_end = seq_lens[r] - n_new + min(n_new, (blk + 1) * tpb);
-            units += (unsigned long long)((kv_end + 63) / 64);
+        int weighted = 0;
+        if (n_new > 0 && n_new <= small_max) {
+            int mt, tpb, nblk;
+            small_block_shape(n_new, G, mt, tpb, nblk);
+            int units = 0;
+            for (int blk = 0; blk < nblk; ++blk) {
+                const int kv_end = seq_lens[r] - n_new + min(n_new, (blk + 1) * tpb);
+                units += (kv_end + 63) / 64;
+            }
+            weighted = units * Hkv * mt;
         }
-        atomicAdd(&tot_units, units * (unsigned long long)(Hkv * mt));
+        req_cnt[r] = weighted;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        unsigned long long sum = 0ull;
+        for (int r = 0; r < R; ++r) sum += (unsigned long long)req_cnt[r];
+        tot_units = sum;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -284,29 +301,38 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
     }
     __syncthreads();
     if (total_items == 0) return;
-    for (int r = threadIdx.x; r < R; r += blockDim.x) {
+    // one item per thread and step: request by binary search over the item offsets, then block / KV head / range
+    for (int i = threadIdx.x; i < total_items; i += blockDim.x) {
+        int lo = 0, hi = R;   // largest r with req_off[r] <= i among requests that own items
+        while (hi - lo > 1) {
+            const int mid = (lo + hi) >> 1;
+            if (req_off[mid] <= i) lo = mid; else hi = mid;
+        }
+        const int r = lo;
         const int n_new = qsl[r + 1] - qsl[r];
-        if (n_new <= 0 || n_new > small_max) continue;
         int mt, tpb, nblk;
         small_block_shape(n_new, G, mt, tpb, nblk);
-        int idx = req_off[r], row0 = req_row[r];
+        int local = i - req_off[r], row0 = req_row[r];
         for (int blk = 0; blk < nblk; ++blk) {
             const int q_count = min(tpb, n_new - blk * tpb);
             const int pos0 = seq_lens[r] - n_new + blk * tpb;
             const int kv_end = pos0 + q_count;   // last token's position + 1
             const int units = (kv_end + 63) / 64;
             const int n_splits = (units + chunk - 1) / chunk;
+            if (local >= n_splits * Hkv && blk + 1 < nblk) {
+                local -= n_splits * Hkv;
+                row0 += n_splits * Hkv * 16 * mt;
+                continue;
+            }
             const int per = (units + n_splits - 1) / n_splits;   // equal ranges rather than full ones and a stub
-            for (int kvh = 0; kvh < Hkv; ++kvh)
-                for (int sp = 0; sp < n_splits; ++sp) {
-                    AttnSplitWork w;
-                    w.req = r; w.q_start = qsl[r] + blk * tpb; w.q_count = q_count; w.kv_head = kvh;
-                    w.kv_start = sp * per * 64; w.kv_end = min(kv_end, (sp + 1) * per * 64);
-                    w.pos0 = pos0; w.mt = mt; w.split = sp; w.n_splits = n_splits; w.part_row0 = row0; w.pad_ = 0;
-                    group_done[idx] = 0;
-                    items[idx++] = w;
-                    row0 += 16 * mt;
-                }
+            const int kvh = local / n_splits, sp = local % n_splits;
+            AttnSplitWork w;
+            w.req = r; w.q_start = qsl[r] + blk * tpb; w.q_count = q_count; w.kv_head = kvh;
+            w.kv_start = sp * per * 64; w.kv_end = min(kv_end, (sp + 1) * per * 64);
+            w.pos0 = pos0; w.mt = mt; w.split = sp; w.n_splits = n_splits; w.part_row0 = row0 + local * 16 * mt; w.pad_ = 0;
+            group_done[i] = 0;
+            items[i] = w;
+            break;
         }
     }
 }
@@ -314,9 +340,8 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
 // The whole metadata step as one launch: every block handles 256 tokens; block 0 then builds the two
 // work lists (their serial parts are O(R)).
 __global__ void __launch_bounds__(256)
-metadata_kernel(const int32_t *__restrict__ positions, const int32_t *__restrict__ a_req,
-                const int32_t *__restrict__ adapter_ids, const int32_t *__restrict__ qsl,
-                const int32_t *__restrict__ seq_lens, const int32_t *__restrict__ block_tables, int max_blocks,
+metadata_kernel(const int32_t *__restrict__ positions, const int32_t *a_req, const int32_t *adapter_ids,
+                const int32_t *qsl, const int32_t *seq_lens, const int32_t *__restrict__ block_tables, int max_blocks,
                 int num_pages, int page_size, int max_adapters, int T, int R, int mode,
                 int32_t *__restrict__ token_req, int32_t *__restrict__ row_adapter, int32_t *__restrict__ slot_map,
                 int max_tiles, ProjTile *__restrict__ tiles, int32_t *__restrict__ counts, int32_t *seg_scratch,
@@ -325,6 +350,22 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *__restrict
                 int G, int n_sm, int small_max, int max_split_items, int max_split_rows,
                 AttnSplitWork *__restrict__ split_items,
                 int32_t *req_scratch, int32_t *__restrict__ group_done, int rowwise_cap, int32_t *status) {
+    // The per-request inputs are read many times (binary searches, list builders): one parallel pass stages them
+    // in shared memory, so that the later steps do not each pay a round trip to global memory.
+    __shared__ int32_t s_req[4 * kMetaStageR + 1];
+    if (R <= kMetaStageR) {
+        int32_t *s_qsl = s_req, *s_len = s_req + R + 1, *s_ids = s_len + R, *s_areq = s_ids + R;
+        for (int i = threadIdx.x; i <= R; i += blockDim.x) s_qsl[i] = qsl[i];
+        for (int i = threadIdx.x; i < R; i += blockDim.x) {
+            s_len[i] = seq_lens[i];
+            if (adapter_ids) s_ids[i] = adapter_ids[i];
+            if (a_req) s_areq[i] = a_req[i];
+        }
+        __syncthreads();
+        qsl = s_qsl; seq_lens = s_len;
+        if (adapter_ids) adapter_ids = s_ids;
+        if (a_req) a_req = s_areq;
+    }
     metadata_tokens(positions, a_req, adapter_ids, qsl, seq_lens, block_tables, max_blocks, num_pages, page_size,
                     max_adapters, T, R, mode, token_req, row_adapter, slot_map, status);
     if (blockIdx.x != 0) return;

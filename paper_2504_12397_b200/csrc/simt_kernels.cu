@@ -88,12 +88,13 @@ __global__ void shrink_simt_kernel(const T *__restrict__ x, const int32_t *__res
 // Row-wise low-rank delta for batches of few rows per adapter (bf16):
 //     delta[row][n] = s * sum_i B[n][i] (A x_row)[blk(n)][i]          (Eq. 5, the term behind the gate)
 // for every row with an applied adapter, in fp32.  One block per (row, q/k/v block): the row of x is staged in
-// shared memory, each warp forms up to 8 of the block's `rank` inner products with A at once (16-byte loads,
-// eight independent loads in flight per lane), then each thread forms outputs of the block's columns from its
-// B rows.  Adapter storage is the rank-padded tensor-core layout A[3][64][H], B[N][64].  The kernel does
+// shared memory, each of 32 warps forms one or two of the block's `rank` inner products with A (16-byte loads,
+// several in flight per lane), then each thread forms outputs of the block's columns from its B rows.  Adapter storage is the rank-padded tensor-core layout A[3][64][H], B[N][64].  The kernel does
 // nothing unless the metadata step chose the row-wise route for this batch (*rowwise_flag).
 // ---------------------------------------------------------------------------------------------
-__global__ void __launch_bounds__(256)
+constexpr int kDeltaThreads = 1024;  // 32 warps: one or two inner products per warp, many loads in flight per SM
+
+__global__ void __launch_bounds__(kDeltaThreads)
 lora_delta_rows_kernel(const __nv_bfloat16 *__restrict__ x, const int32_t *__restrict__ row_adapter,
                        const AdapterDev *__restrict__ adapters, const int32_t *__restrict__ rowwise_flag, int H,
                        int Nq, int Nkv, int N, float *__restrict__ delta) {
@@ -110,37 +111,36 @@ lora_delta_rows_kernel(const __nv_bfloat16 *__restrict__ x, const int32_t *__res
     for (int i = threadIdx.x; i < hv; i += blockDim.x) x_s4[i] = xg[i];
     __syncthreads();
     {
-        // outputs warp, warp + 8, ..., below rank (rank <= 64: at most 8 per warp)
+        // inner products warp and warp + 32 (rank <= 64)
         const uint4 *A4 = reinterpret_cast<const uint4 *>(ad.A) + (size_t)blk * kRankPadMax * hv;
-        float acc[8];
-#pragma unroll
-        for (int j = 0; j < 8; ++j) acc[j] = 0.f;
-        for (int v = lane; v < hv; v += 32) {
-            const uint4 xv = x_s4[v];
-            const __nv_bfloat162 *x2 = reinterpret_cast<const __nv_bfloat162 *>(&xv);
-            float xf[8];
-#pragma unroll
-            for (int e = 0; e < 4; ++e) { const float2 f = __bfloat1622float2(x2[e]); xf[2 * e] = f.x; xf[2 * e + 1] = f.y; }
-            uint4 av[8];
-#pragma unroll
-            for (int j = 0; j < 8; ++j)
-                av[j] = (warp + 8 * j < ad.rank) ? A4[(size_t)(warp + 8 * j) * hv + v] : make_uint4(0, 0, 0, 0);
-#pragma unroll
-            for (int j = 0; j < 8; ++j) {
-                const __nv_bfloat162 *a2 = reinterpret_cast<const __nv_bfloat162 *>(&av[j]);
+        const bool on0 = warp < ad.rank, on1 = warp + 32 < ad.rank;
+        const uint4 *a0 = A4 + (size_t)warp * hv, *a1 = A4 + (size_t)(warp + 32) * hv;
+        float acc0 = 0.f, acc1 = 0.f;
+        if (on0) {
+#pragma unroll 2
+            for (int v = lane; v < hv; v += 32) {
+                const uint4 xv = x_s4[v];
+                const uint4 av0 = a0[v];
+                const uint4 av1 = on1 ? a1[v] : make_uint4(0, 0, 0, 0);
+                const __nv_bfloat162 *x2 = reinterpret_cast<const __nv_bfloat162 *>(&xv);
+                const __nv_bfloat162 *p0 = reinterpret_cast<const __nv_bfloat162 *>(&av0);
+                const __nv_bfloat162 *p1 = reinterpret_cast<const __nv_bfloat162 *>(&av1);
 #pragma unroll
                 for (int e = 0; e < 4; ++e) {
-                    const float2 af = __bfloat1622float2(a2[e]);
-                    acc[j] = fmaf(af.x, xf[2 * e], acc[j]);
-                    acc[j] = fmaf(af.y, xf[2 * e + 1], acc[j]);
+                    const float2 xf = __bfloat1622float2(x2[e]);
+                    const float2 f0 = __bfloat1622float2(p0[e]), f1 = __bfloat1622float2(p1[e]);
+                    acc0 = fmaf(f0.x, xf.x, acc0); acc0 = fmaf(f0.y, xf.y, acc0);
+                    acc1 = fmaf(f1.x, xf.x, acc1); acc1 = fmaf(f1.y, xf.y, acc1);
                 }
             }
         }
-#pragma unroll
-        for (int j = 0; j < 8; ++j) {
-            float a = acc[j];
-            for (int off = 16; off; off >>= 1) a += __shfl_xor_sync(0xffffffffu, a, off);
-            if (lane == 0 && warp + 8 * j < kRankPadMax) t_s[warp + 8 * j] = (warp + 8 * j < ad.rank) ? a * ad.scale : 0.f;
+        for (int off = 16; off; off >>= 1) {
+            acc0 += __shfl_xor_sync(0xffffffffu, acc0, off);
+            acc1 += __shfl_xor_sync(0xffffffffu, acc1, off);
+        }
+        if (lane == 0) {
+            t_s[warp] = on0 ? acc0 * ad.scale : 0.f;          // zero beyond the rank
+            t_s[warp + 32] = on1 ? acc1 * ad.scale : 0.f;
         }
     }
     __syncthreads();
@@ -151,14 +151,21 @@ lora_delta_rows_kernel(const __nv_bfloat16 *__restrict__ x, const int32_t *__res
     for (int n = n_begin + threadIdx.x; n < n_end; n += blockDim.x) {
         const uint4 *brow = B4 + (size_t)n * (kRankPadMax / 8);
         float acc = 0.f;
-        for (int v = 0; v < rv; ++v) {
-            const uint4 bv = brow[v];
-            const __nv_bfloat162 *b2 = reinterpret_cast<const __nv_bfloat162 *>(&bv);
 #pragma unroll
-            for (int e = 0; e < 4; ++e) {
-                const float2 bf = __bfloat1622float2(b2[e]);
-                acc = fmaf(bf.x, t_s[v * 8 + 2 * e], acc);       // t_s is zero beyond the rank
-                acc = fmaf(bf.y, t_s[v * 8 + 2 * e + 1], acc);
+        for (int half = 0; half < 2; ++half) {   // four 16-byte vectors (32 rank columns) at a time, loads first
+            if (half * 4 >= rv) break;
+            uint4 b[4];
+#pragma unroll
+            for (int v = 0; v < 4; ++v) b[v] = half * 4 + v < rv ? brow[half * 4 + v] : make_uint4(0, 0, 0, 0);
+#pragma unroll
+            for (int v = 0; v < 4; ++v) {
+                const __nv_bfloat162 *p = reinterpret_cast<const __nv_bfloat162 *>(&b[v]);
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    const float2 f = __bfloat1622float2(p[e]);
+                    acc = fmaf(f.x, t_s[(half * 4 + v) * 8 + 2 * e], acc);
+                    acc = fmaf(f.y, t_s[(half * 4 + v) * 8 + 2 * e + 1], acc);
+                }
             }
         }
         delta[(size_t)row * N + n] = acc;
@@ -168,7 +175,7 @@ lora_delta_rows_kernel(const __nv_bfloat16 *__restrict__ x, const int32_t *__res
 int launch_lora_delta_rows(alora_ctx *ctx, int layer, const void *hidden, int T, cudaStream_t s) {
     const Dims &d = ctx->d;
     const AdapterDev *ads = ctx->d_adapters + (size_t)layer * ctx->cfg.max_adapters;
-    lora_delta_rows_kernel<<<dim3(T, 3), 256, (size_t)d.H * 2, s>>>((const __nv_bfloat16 *)hidden, ctx->d_row_adapter, ads,
+    lora_delta_rows_kernel<<<dim3(T, 3), kDeltaThreads, (size_t)d.H * 2, s>>>((const __nv_bfloat16 *)hidden, ctx->d_row_adapter, ads,
                                                                    ctx->d_counts + 5, d.H, d.Nq, d.Nkv, d.N,
                                                                    ctx->d_row_delta);
     return 1;
