@@ -28,6 +28,7 @@ ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
 sys.path.insert(0, os.path.join(ROOT, "tests"))
 
+from paper_2504_12397_b200 import sharding  # noqa: E402
 from paper_2504_12397_b200 import workloads as wl  # noqa: E402
 
 METRIC = "aLoRA suffix-prefill tokens/s on reused base KV"
@@ -260,8 +261,8 @@ def decode_leg(ab, hp, ctx, shape, stream, flush, peaks, steps=256, seed=5, ctx_
         nxt += int(blocks[r])
     g = torch.Generator(device="cuda"); g.manual_seed(seed)
     pool = torch.empty((num_pages, 2, shape.n_kv_heads, ps, shape.head_dim), device="cuda", dtype=torch.bfloat16)
-    for i in range(0, num_pages, 65536):  # filled in slices: no fp32 copy of the whole pool
-        n = min(65536, num_pages - i)
+    for i in range(0, num_pages, 8192):  # filled in slices: no fp32 copy of the whole pool
+        n = min(8192, num_pages - i)
         pool[i:i + n] = torch.randn((n,) + tuple(pool.shape[1:]), generator=g, device="cuda",
                                     dtype=torch.float32).to(torch.bfloat16)
     hidden = torch.randn((R, shape.hidden), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
@@ -352,17 +353,14 @@ def main():
         torch.cuda.synchronize()
 
     def max_over_ranks(x):
-        if world > 1:
-            t = torch.tensor([x], device="cuda")
-            dist.all_reduce(t, op=dist.ReduceOp.MAX)
-            return float(t.item())
-        return x
+        return sharding.max_over_ranks(x, device="cuda")
 
     shape = wl.SHAPE_8B
     extra = not args.no_extra and world == 1
     legs = set(x for x in args.legs.split(",") if x) if extra else set()
     recomp = not args.no_recompute
-    main_case = PrefillCase(hp, shape, args.requests, args.prefix, args.suffix, SEED, with_recompute=recomp)
+    main_case = PrefillCase(hp, shape, args.requests, args.prefix, args.suffix, sharding.rank_seed(SEED, rank),
+                            with_recompute=recomp)   # weak scaling: every rank draws its own batch of the same shape
     case_8k = PrefillCase(hp, shape, 8, 8192, 256, SEED + 1, with_recompute=True) if (recomp and "recompute8k" in legs) else None
     T, R = main_case.T, main_case.R
     max_tokens = max([T] + ([main_case.full_T] if recomp else []) + ([case_8k.full_T] if case_8k else []))
@@ -399,7 +397,7 @@ def main():
     barrier()
     launches = ab.alora_launch_count(ctx) - launches0
     step_ms = max_over_ranks(step_ms)
-    value = world * T / (step_ms / 1e3)
+    value = sharding.aggregate_throughput(T, step_ms / 1e3, world)
 
     # ---- end to end through the C ABI with host buffers: H2D of the step's inputs, D2H of the result ----
     d = main_case.d

@@ -1,0 +1,121 @@
+"""GPU parity at the full sizes of the named configurations, in the launch configuration bench.py times:
+the whole batch runs on the GPU, and the outputs of a few sampled requests (every row of them) are compared
+with the CPU oracle, which computes those requests one by one from the same inputs.  The cached prefix is a
+seeded N(0,1) fill of the page pool made on the device (it stands in for the base model's cache; the rows the
+oracle needs are copied back from the very pool the kernels read)."""
+import numpy as np
+import pytest
+
+from paper_2504_12397_b200 import binding as ab
+from paper_2504_12397_b200 import workloads as wl
+
+import helpers as hp
+
+pytestmark = pytest.mark.gpu
+
+
+def _device_pool(shape, num_pages, seed):
+    import torch
+    g = torch.Generator(device="cuda"); g.manual_seed(seed)
+    pool = torch.empty((num_pages, 2, shape.n_kv_heads, shape.page_size, shape.head_dim), device="cuda",
+                       dtype=torch.bfloat16)
+    for i in range(0, num_pages, 8192):
+        n = min(8192, num_pages - i)
+        pool[i:i + n] = torch.randn((n,) + tuple(pool.shape[1:]), generator=g, device="cuda",
+                                    dtype=torch.float32).to(torch.bfloat16)
+    return pool
+
+
+def _request_kv(pool, b, r, length, shape):
+    """Contiguous (K, V) [length, Nkv] float32 of request r, copied from the device pool through its block table."""
+    import torch
+    nblk = (length + shape.page_size - 1) // shape.page_size
+    pages = torch.from_numpy(b.block_tables[r, :nblk].astype(np.int64)).cuda()
+    blk = pool[pages].to(torch.float32).cpu().numpy()          # [nblk, 2, Hkv, page, hd]
+    kv = blk.transpose(1, 0, 3, 2, 4).reshape(2, nblk * shape.page_size, shape.Nkv)
+    return kv[0, :length], kv[1, :length]
+
+
+def _sub_batch(b, r):
+    q0, q1 = int(b.query_start_loc[r]), int(b.query_start_loc[r + 1])
+    return q0, q1, wl.Batch(positions=b.positions[q0:q1], query_start_loc=np.array([0, q1 - q0], np.int32),
+                            seq_lens=b.seq_lens[r:r + 1], prefix_lens=b.prefix_lens[r:r + 1],
+                            activation_offsets=b.activation_offsets[r:r + 1], adapter_ids=b.adapter_ids[r:r + 1],
+                            block_tables=b.block_tables[r:r + 1], num_pages=b.num_pages, hidden=b.hidden[q0:q1])
+
+
+def _check_requests(oracle, shape, w, b, pool_before, pool_after, out_h, sample, qkv_h=None):
+    for r in sample:
+        P, L = int(b.prefix_lens[r]), int(b.seq_lens[r])
+        K0, V0 = _request_kv(pool_before, b, r, P, shape)
+        q0, q1, sub = _sub_batch(b, r)
+        want = hp.oracle_block(oracle, shape, w.wqkv, w.adapters, sub, [K0 if P else None], [V0 if P else None])
+        assert hp.rel_err(out_h[q0:q1], want["out"]) <= 2e-2, f"attention output of request {r}"
+        if qkv_h is not None:
+            assert hp.rel_err(qkv_h[q0:q1], want["qkv"]) <= 2e-2, f"projection rows of request {r}"
+        K1, V1 = _request_kv(pool_after, b, r, L, shape)
+        assert hp.rel_err(K1[P:], want["K"][0][P:]) <= 2e-2 and hp.rel_err(V1[P:], want["V"][0][P:]) <= 2e-2
+        # the cached prefix of the request is untouched, bit for bit
+        assert np.array_equal(K1[:P].view(np.uint32), K0.view(np.uint32))
+        assert np.array_equal(V1[:P].view(np.uint32), V0.view(np.uint32))
+
+
+def _run_layer(w, seed, decode=False, with_qkv=False):
+    import torch
+    shape, b = w.shape, w.batch
+    g = hp.GpuLayers(shape, [dict(wqkv=w.wqkv)], [w.adapters], b.T, b.R)
+    try:
+        pool = _device_pool(shape, b.num_pages, seed)
+        before = pool.clone()
+        d = hp.DevBatch(b, "bf16")
+        out = g.empty(b.T, shape.Nq)
+        if decode:
+            ab.alora_decode_step(g.ctx, 0, d.hidden, d.positions, d.a_req, d.ids, d.seq_lens, pool, d.bt, d.max_blocks,
+                                 b.num_pages, b.R, out)
+        else:
+            ab.alora_prefill_layer(g.ctx, 0, d.hidden, d.positions, d.a_req, d.ids, d.qsl, d.seq_lens, pool, d.bt,
+                                   d.max_blocks, b.num_pages, b.T, b.R, out)
+        qkv_h = None
+        if with_qkv:
+            qkv = g.empty(b.T, shape.N)
+            ab.alora_project_qkv(g.ctx, 0, ab.MODE_ALORA, d.hidden, d.positions, d.a_req, d.ids, d.qsl, d.seq_lens,
+                                 b.T, b.R, qkv)
+            qkv_h = hp.to_host(qkv)
+        assert g.status() == 0
+        return before, pool, hp.to_host(out), qkv_h
+    finally:
+        g.close()
+
+
+def test_config2_bench_workload_sampled_requests(oracle64):
+    """8 requests x (4096 cached + 256 suffix tokens), rank 32: requests 0 and 7 in full."""
+    w = wl.config2(seed=2)
+    before, after, out_h, qkv_h = _run_layer(w, seed=1002, with_qkv=True)
+    _check_requests(oracle64, w.shape, w, w.batch, before, after, out_h, [0, 7], qkv_h)
+
+
+def test_config3_ragged_multi_adapter_sampled_requests(oracle64):
+    """32 requests over adapters of ranks 8/16/32/64, prefixes 512..16384, suffixes 16..512, shuffled pages:
+    the two requests with the least oracle work and the one with the shortest suffix, in full."""
+    w = wl.config3(seed=3)
+    b = w.batch
+    S = (b.seq_lens - b.prefix_lens).astype(np.int64)
+    work = S * b.seq_lens.astype(np.int64)
+    sample = sorted(set(list(np.argsort(work)[:2]) + [int(np.argmin(S))]))
+    before, after, out_h, _ = _run_layer(w, seed=1003)
+    _check_requests(oracle64, w.shape, w, b, before, after, out_h, sample)
+
+
+def test_config5_decode_step_sampled_requests(oracle64):
+    """64 requests (base model and 4 rank-32 adapters), contexts 1024..32768, one new token each: the shortest,
+    the longest and two more requests, and the projection rows of all 64."""
+    w = wl.config5(seed=5)
+    b = w.batch
+    order = np.argsort(b.seq_lens)
+    sample = sorted({int(order[0]), int(order[-1]), int(order[len(order) // 2]), 3})
+    before, after, out_h, qkv_h = _run_layer(w, seed=1005, decode=True, with_qkv=True)
+    _check_requests(oracle64, w.shape, w, b, before, after, out_h, sample, qkv_h)
+    want, gate = oracle64.project_qkv(b.hidden, w.wqkv, w.shape.Nq, w.shape.Nkv, b.positions, b.query_start_loc,
+                                      b.activation_offsets, b.adapter_ids, hp.oracle_adapters(w.adapters))
+    assert hp.rel_err(qkv_h, want) <= 2e-2
+    assert gate.sum() > 0 and (gate == 0).sum() > 0
