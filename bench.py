@@ -35,6 +35,10 @@ METRIC = "aLoRA suffix-prefill tokens/s on reused base KV"
 UNIT = "tokens/s"
 WORKLOAD = "config2: 8B-shape layer bf16, 8 requests x (4096 cached + 256 suffix), rank-32 adapter, 16-token pages"
 SEED = 2
+NOMINAL_BF16_TFLOPS, NOMINAL_HBM_GBS = 2250.0, 8000.0   # the data-sheet figures the target statement quotes
+# dram__bytes_read.sum + dram__bytes_write.sum per launch of the default workload's kernels, from the ncu captures
+# summarised under profiles/ (valid only for the default requests / prefix / suffix and the kernels as profiled)
+NCU_TRAFFIC_BYTES = {"attention": 159.762176e6 + 6.4768e6, "project_qkv": 100.507648e6 + 12.848128e6}
 
 
 def measured_peaks():
@@ -436,7 +440,11 @@ def main():
     achieved = dom_flops / (dom_ms / 1e3) / 1e12 if dom_ms > 0 else 0.0
     peak = peaks["bf16_tflops"]
     roofline = {"bound": "tensor", "kernel": dominant, "achieved": achieved, "peak": peak, "unit": "TFLOP/s",
-                "frac": achieved / peak, "traffic": None, "peak_source": peaks["source"] + " (burst bf16 GEMM)",
+                "frac": achieved / peak, "frac_of_nominal": achieved / NOMINAL_BF16_TFLOPS,
+                "traffic": (NCU_TRAFFIC_BYTES.get(dominant) if (args.requests, args.prefix, args.suffix) == (8, 4096, 256) else None),
+                "traffic_unit": "bytes per launch (ncu dram read + write)",
+                "algorithmic_bytes": attn_bytes if dominant == "attention" else 2.0 * (T * shape.hidden + shape.N * shape.hidden + T * shape.N),
+                "peak_source": peaks["source"] + " (burst bf16 GEMM)",
                 "ms_per_launch": dom_ms,
                 "per_kernel_ms": {k: round(v, 4) for k, v in kern.items()},
                 "projection": {"tflops": proj_flops / (proj_ms / 1e3) / 1e12 if proj_ms else None,
