@@ -148,7 +148,8 @@ def run_reference(args):
     w = wl.config2(seed=SEED)
     rng = np.random.default_rng(SEED + 1000)
     pool_np = wl.random_kv_pool(w.shape, w.batch.num_pages, rng)
-    n_tok = 32
+    # bounded sample: about 2000 suffix tokens over the whole run, at most 32 per step
+    n_tok = max(2, min(32, 2000 // max(args.steps, 1)))
     for _ in range(args.warmup):
         oracle_sample_rate(w, pool_np, 2)
     times = []
@@ -317,6 +318,92 @@ def short_suffix_leg(ab, hp, ctx, shape, stream, flush, peaks, requests, prefix,
             "attention_hbm_gbs": gbs, "attention_frac_of_hbm_peak": gbs / peaks["hbm_gbs"] if gbs else None}
 
 
+def stack_leg(ab, hp, shape, stream, local, seed=4, requests=4, prefix=32768, suffix=1024, n_layers=32):
+    """Config 4: the full decoder stack at the 8B shape (RMSNorm, attention block, o_proj, SwiGLU MLP; random
+    bf16 weights), 4 requests with 32768 cached positions and 1024 aLoRA suffix tokens each, against the
+    full-LoRA recompute of prefix + suffix through the same stack."""
+    import torch
+    g = torch.Generator(device="cuda"); g.manual_seed(seed)
+
+    def rnd(*dims, std=0.02):
+        return (torch.randn(dims, generator=g, device="cuda", dtype=torch.float32) * std).to(torch.bfloat16)
+
+    R, P, S_ = requests, prefix, suffix
+    T, full_T = R * S_, R * (P + S_)
+    ps = shape.page_size
+    blocks = (P + S_ + ps - 1) // ps
+    num_pages = R * blocks + 3
+    bt = np.arange(R * blocks, dtype=np.int32).reshape(R, blocks)
+    cfg = ab.make_config(hidden=shape.hidden, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
+                         head_dim=shape.head_dim, page_size=ps, n_layers=n_layers, intermediate=shape.intermediate,
+                         max_adapters=1, max_rank=32, dtype=ab.DTYPE_BF16, device=local, max_tokens=full_T, max_requests=R)
+    ctx = ab.alora_create(cfg)
+    keep = []
+    H, I, Nq, Nkv = shape.hidden, shape.intermediate, shape.Nq, shape.Nkv
+    for l in range(n_layers):
+        wts = [rnd(shape.N, H), rnd(H, Nq), rnd(2 * I, H), rnd(H, I),
+               (1.0 + 0.1 * torch.randn(H, generator=g, device="cuda")).to(torch.bfloat16),
+               (1.0 + 0.1 * torch.randn(H, generator=g, device="cuda")).to(torch.bfloat16)]
+        ad = [rnd(32, H), rnd(Nq, 32), rnd(32, H), rnd(Nkv, 32), rnd(32, H), rnd(Nkv, 32)]
+        keep.append((wts, ad))
+        ab.alora_set_layer_weights(ctx, l, *wts)
+        ab.alora_register_adapter(ctx, 0, l, 32, 1.0, *ad)
+    pools = []
+    for l in range(n_layers):   # the base model's cache of every layer: N(0,1) stand-in
+        pool = torch.empty((num_pages, 2, shape.n_kv_heads, ps, shape.head_dim), device="cuda", dtype=torch.bfloat16)
+        for i in range(0, num_pages, 8192):
+            n = min(8192, num_pages - i)
+            pool[i:i + n] = torch.randn((n,) + tuple(pool.shape[1:]), generator=g, device="cuda",
+                                        dtype=torch.float32).to(torch.bfloat16)
+        pools.append(pool)
+    ids = hp.idev(np.zeros(R, np.int32)); d_bt = hp.idev(bt)
+    seq = hp.idev(np.full(R, P + S_, np.int32))
+    # aLoRA side: only the suffix tokens are new
+    pos_a = hp.idev(np.concatenate([np.arange(P, P + S_, dtype=np.int32)] * R))
+    qsl_a = hp.idev(np.arange(R + 1, dtype=np.int32) * S_)
+    areq = hp.idev(np.full(R, P, np.int32))
+    hid_a = rnd(T, H, std=1.0); out_a = torch.empty_like(hid_a)
+    # recompute side: every token is new, the adapter applies everywhere
+    pos_f = hp.idev(np.concatenate([np.arange(P + S_, dtype=np.int32)] * R))
+    qsl_f = hp.idev(np.arange(R + 1, dtype=np.int32) * (P + S_))
+    hid_f = rnd(full_T, H, std=1.0); out_f = torch.empty_like(hid_f)
+    fpools = [torch.zeros_like(pools[0]) for _ in range(2)]   # two private pools, alternated: results are not reused
+
+    def alora():
+        ab.alora_forward_stack(ctx, ab.MODE_ALORA, hid_a, pos_a, areq, ids, qsl_a, seq, pools, d_bt, blocks, num_pages,
+                               T, R, out_a, stream)
+
+    def recompute():
+        ab.alora_forward_stack(ctx, ab.MODE_FULL_LORA, hid_f, pos_f, None, ids, qsl_f, seq,
+                               [fpools[l & 1] for l in range(n_layers)], d_bt, blocks, num_pages, full_T, R, out_f, stream)
+
+    def once(fn, n):
+        fn(); torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(n):
+            fn()
+        e1.record(stream); torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / n
+
+    a_ms = once(alora, 3)
+    kern = profiled(ab, ctx, alora, 1, None)
+    r_ms = once(recompute, 1)
+    status = ab.alora_get_status(ctx)
+    finite = bool(torch.isfinite(out_a.float()).all().item())
+    ab.alora_destroy(ctx)
+    lin = 2.0 * (H * shape.N + Nq * H + 3 * H * I)                    # linear FLOP per token and layer
+    att = lambda s_, p_: 4.0 * shape.head_dim * shape.n_q_heads * (s_ * p_ + s_ * (s_ + 1) / 2)   # noqa: E731
+    flop_a = n_layers * (T * lin + R * att(S_, P))
+    flop_r = n_layers * (full_T * lin + R * att(P + S_, 0))
+    return {"workload": f"config4: {n_layers}-layer 8B-shape stack, {R} requests x ({P} cached + {S_} suffix), rank 32",
+            "alora_ms": a_ms, "alora_suffix_tokens_per_s": T / (a_ms / 1e3), "alora_tflops": flop_a / (a_ms / 1e3) / 1e12,
+            "full_lora_recompute_ms": r_ms, "recompute_tflops": flop_r / (r_ms / 1e3) / 1e12,
+            "speedup_alora_vs_full_lora": r_ms / a_ms, "flop_ratio": flop_r / flop_a,
+            "prefix_plus_suffix_over_suffix": (P + S_) / S_, "per_kernel_ms_alora": {k: round(v, 3) for k, v in kern.items()},
+            "device_status": status, "output_finite": finite}
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -326,8 +413,8 @@ def main():
     ap.add_argument("--no-recompute", action="store_true", help="skip the full-LoRA recompute comparisons")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the decode and short-suffix legs")
-    ap.add_argument("--legs", default="decode,short,recompute8k",
-                    help="extra legs to run after the main workload (comma list of decode, short, recompute8k)")
+    ap.add_argument("--legs", default="decode,short,recompute8k,stack",
+                    help="extra legs to run after the main workload (comma list of decode, short, recompute8k, stack)")
     ap.add_argument("--decode-steps", type=int, default=256)
     ap.add_argument("--decode-ctx-max", type=int, default=32768)
     ap.add_argument("--requests", type=int, default=8)
@@ -479,13 +566,19 @@ def main():
     if "short" in legs:
         short = [short_suffix_leg(ab, hp, ctx, shape, stream, flush, peaks, r_, 4096, s_)
                  for r_, s_ in ((8, 4), (8, 16), (64, 4), (64, 16))]
-    clocks = sampler.stop()
     status = ab.alora_get_status(ctx)
     ab.alora_destroy(ctx)
+    want_cpu = rank == 0 and world == 1 and not args.no_cpu_baseline
+    pool_np = main_case.pool.to(torch.float32).cpu().numpy() if want_cpu else None
+    stack = None
+    if "stack" in legs:
+        del main_case.pool
+        torch.cuda.empty_cache()
+        stack = stack_leg(ab, hp, shape, stream, local)
+    clocks = sampler.stop()
 
     cpu = None
-    if rank == 0 and world == 1 and not args.no_cpu_baseline:
-        pool_np = main_case.pool.to(torch.float32).cpu().numpy()
+    if want_cpu:
         S_ = (main_case.b.seq_lens - main_case.b.prefix_lens)
         rate, threads, dt, done = oracle_sample_rate(w, pool_np, int(S_.max()), requests=range(R), budget_s=20.0)
         cpu = {"value": rate, "unit": UNIT, "cores": threads, "kind": "oracle",
@@ -504,7 +597,7 @@ def main():
                                       "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
             "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
             "full_lora_recompute": recompute, "full_lora_recompute_8k_prefix": recompute_8k,
-            "decode": decode, "short_suffix": short, "device_status": status,
+            "decode": decode, "short_suffix": short, "stack": stack, "device_status": status,
         }))
     if world > 1:
         dist.destroy_process_group()
