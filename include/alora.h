@@ -195,7 +195,8 @@ alora_status alora_prefill_layer(alora_ctx *ctx, int layer, const void *d_hidden
 /*
  * One decode step (Prop. 1, second sentence; Eq. 3): exactly one new token per request (T == R,
  * query_start_loc[r] == r), mixed base / adapter requests.  Same results as alora_prefill_layer on
- * the same arguments, computed by kernels specialised for one query row per request.
+ * the same arguments (requests with at most 16 new tokens take the same few-row attention kernel in
+ * every entry point; this one additionally knows that no request is longer).
  */
 alora_status alora_decode_step(alora_ctx *ctx, int layer, const void *d_hidden,
                                const int32_t *d_positions, const int32_t *d_activation_offsets,
@@ -245,15 +246,6 @@ const char *alora_last_cuda_error(const alora_ctx *ctx);
 int64_t alora_launch_count(const alora_ctx *ctx);
 
 /*
- * Optional per-kernel timing (a measurement aid; the paper has no counterpart).  While enabled,
- * every kernel family launched by this context is bracketed by CUDA events on the launching stream.
- * alora_profile_enable(ctx, 1) clears what was accumulated and starts, (ctx, 0) stops.
- * alora_profile_read synchronises the device and adds up, per family, the elapsed milliseconds and
- * the number of bracketed launch groups; both arrays have ALORA_PROFILE_KINDS entries.
- * Families: 0 batch metadata, 1 rank-r shrink (t = A x), 2 q/k/v projection, 3 KV append,
- * 4 attention, 5 split-KV merge, 6 other dense projections (o_proj, MLP), 7 norm / activation glue.
- */
-/*
  * Gated q/k/v projection (same result as alora_project_qkv in mode ALORA with one adapter) for
  * callers that cannot allocate device memory.  (The paper has no counterpart: this is an
  * integration aid.)  Typical callers: a plug-in running inside a serving engine that already owns
@@ -287,6 +279,16 @@ alora_status alora_project_qkv_static(int dtype, int hidden, int n_q, int n_kv, 
                                       const void *d_Bq, const void *d_Ak, const void *d_Bk, const void *d_Av,
                                       const void *d_Bv, int T, int R, void *d_qkv, void *stream);
 
+/*
+ * Optional per-kernel timing (a measurement aid; the paper has no counterpart).  While enabled,
+ * every kernel family launched by this context is bracketed by CUDA events on the launching stream.
+ * alora_profile_enable(ctx, 1) clears what was accumulated and starts, (ctx, 0) stops.
+ * alora_profile_read synchronises the device and adds up, per family, the elapsed milliseconds and
+ * the number of bracketed launch groups; both arrays have ALORA_PROFILE_KINDS entries.
+ * Families: 0 batch metadata, 1 rank-r shrink (t = A x) when it is a launch of its own, or the per-row
+ * low-rank delta of small batches, 2 q/k/v projection, 3 KV append, 4 attention, 5 unused (key ranges are
+ * merged inside the attention kernel), 6 other dense projections (o_proj, MLP), 7 norm / activation glue.
+ */
 #define ALORA_PROFILE_KINDS 8
 alora_status alora_profile_enable(alora_ctx *ctx, int on);
 alora_status alora_profile_read(alora_ctx *ctx, double *ms_by_kind, int64_t *groups_by_kind);
