@@ -25,9 +25,10 @@
 
 namespace alora {
 
-constexpr int kAttnThreads = 320;
-constexpr int kKeysPerTile = 128;
-constexpr int kKvStages = 2;
+constexpr int kAttnThreads = 352;   // 8 softmax warps, TMA producer, two MMA issuers
+constexpr int kKeysPerTile = 128;   // keys per K/V stage in shared memory
+constexpr int kHalfKeys = 64;       // keys per score / probability tile in tensor memory
+constexpr int kKvStages = 3;
 
 struct AttnArgs {
     const AttnWork *items;
@@ -35,15 +36,58 @@ struct AttnArgs {
     const int32_t *block_tables;
     int max_blocks, num_pages;
     int Hkv, G, page_size;     // G * tokens_per_group == 128
+    int box_rows;              // cache rows per TMA box: 8 (pages of 8), 16 (pages of 16 / 32) or 64 (larger pages)
     int N, Nq;                 // fused row width, query part width
     float scale_log2;          // softmax scale * log2(e)
+    const __nv_bfloat16 *qkv;  // [T][N], query part first
     __nv_bfloat16 *out;        // [T][Nq]
     int32_t *status;
+    // runs: the concatenated key tiles of all items, cut into equal runs, one per block
+    const int32_t *run_counts;  // [0] all key tiles, [1] tiles per run
+    const int32_t *cta_start;   // [blocks] item that holds the first tile of the block's run
+    int32_t *done;              // [2 * items] parts finished per (item, row group)
+    float *part_o;              // [2 * blocks][hd][256] unnormalised output of a part, column-major over the 256 rows
+    float *part_ml;             // [2 * blocks][2][256] exponent reference and row sum of a part
 };
+
+// Walks the pieces of a block's run: one piece = tiles [t0, t1) of one item.  An item cut by run boundaries is
+// worked on by n_parts consecutive blocks (this block holds part `part`, the first of them is block c_first);
+// their partial results are merged by whichever part finishes last.
+struct RunPiece {
+    AttnWork w;
+    int item, t0, t1, n_parts, part, c_first;
+};
+struct RunIter {
+    int gt, gt_end, it, len;
+    __device__ explicit RunIter(const AttnArgs &a) {
+        const int total = a.run_counts[0];
+        len = a.run_counts[1];
+        gt = min(total, (int)blockIdx.x * len);
+        gt_end = min(total, gt + len);
+        it = gt < gt_end ? a.cta_start[blockIdx.x] : 0;
+    }
+    __device__ bool next(const AttnArgs &a, RunPiece &p) {
+        if (gt >= gt_end) return false;
+        p.w = a.items[it];
+        const int n_tiles = (p.w.kv_end + kKeysPerTile - 1) / kKeysPerTile;
+        p.item = it;
+        p.t0 = gt - p.w.split;
+        p.t1 = min(n_tiles, gt_end - p.w.split);
+        p.c_first = p.w.split / len;
+        p.n_parts = (p.w.split + n_tiles - 1) / len - p.c_first + 1;
+        p.part = (int)blockIdx.x - p.c_first;
+        gt = p.w.split + p.t1;
+        ++it;
+        return true;
+    }
+};
+// partial-result slot of part `part` of an item whose first part is held by block c_first: a block holds at
+// most one part > 0 (the piece its run starts with) and at most one part 0 of a cut item (the piece it ends with)
+__device__ __forceinline__ int part_slot(int c_first, int part) { return 2 * (c_first + part) + (part == 0 ? 1 : 0); }
 
 template <int HD>
 struct AttnSmem {
-    static constexpr int kQBytes = 128 * HD * 2;             // one query tile (two 64-wide halves when HD = 128)
+    static constexpr int kQBytes = 128 * (HD - 64) * 2;      // one query tile without its first 64 columns (those live in tensor memory)
     static constexpr int kKvBytes = kKeysPerTile * HD * 2;   // one K or V tile
     static constexpr int kQOff = 0;
     static constexpr int kKOff = 2 * kQBytes;
@@ -53,10 +97,15 @@ struct AttnSmem {
 };
 
 // V tile as the B operand of P V: N = head dim (contiguous in memory: "MN-major"), K = keys.
-// Rows (keys) are 128 bytes apart, 8-key groups 1024 bytes apart (stride byte offset); the two
+// Rows (keys) are 128 bytes apart, 8-key groups `sbo_bytes` apart (stride byte offset); the two
 // 64-wide halves of the head dim are `half_bytes` apart (leading byte offset); 128-byte swizzle.
-__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t smem_addr, uint32_t half_bytes) {
-    return (uint64_t)((smem_addr >> 4) & 0x3FFF) | ((uint64_t)((half_bytes >> 4) & 0x3FFF) << 16) | (64ull << 32) |
+__device__ __forceinline__ uint64_t smem_desc_mn_sw128(uint32_t smem_addr, uint32_t half_bytes, uint32_t sbo_bytes) {
+    return (uint64_t)((smem_addr >> 4) & 0x3FFF) | ((uint64_t)((half_bytes >> 4) & 0x3FFF) << 16) |
+           ((uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32) | (1ull << 46) | (2ull << 61);
+}
+// K-major tile (rows 128 bytes apart inside an 8-row group) whose 8-row groups are `sbo_bytes` apart.
+__device__ __forceinline__ uint64_t smem_desc_k_sw128_sbo(uint32_t smem_addr, uint32_t sbo_bytes) {
+    return (uint64_t)((smem_addr >> 4) & 0x3FFF) | (1ull << 16) | ((uint64_t)((sbo_bytes >> 4) & 0x3FFF) << 32) |
            (1ull << 46) | (2ull << 61);
 }
 
@@ -103,6 +152,67 @@ __device__ __forceinline__ void tma_load_3d(uint32_t smem_dst, const CUtensorMap
         : "memory");
 }
 
+// Two non-negative fp32 values -> packed bf16 pair, rounded to nearest (ties up), with integer instructions only:
+// the float-to-bf16 conversion instruction shares the special-function unit with the exponentials, which is
+// the busiest unit of the softmax.
+__device__ __forceinline__ uint32_t pack_bf16_int(float lo, float hi) {
+    return __byte_perm(__float_as_uint(lo) + 0x8000u, __float_as_uint(hi) + 0x8000u, 0x7632);
+}
+__device__ __forceinline__ bool elect_one() {
+    uint32_t pred;
+    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
+    return pred != 0;
+}
+__device__ __forceinline__ uint32_t pack_cvt(float lo, float hi) {
+    uint32_t r; asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo)); return r;
+}
+__device__ __forceinline__ float max3(float a, float b, float c) {
+    float r; asm("max.f32 %0, %1, %2, %3;" : "=f"(r) : "f"(a), "f"(b), "f"(c)); return r;
+}
+__device__ __forceinline__ void fma2(float &d0, float &d1, float a0, float a1, float b, float c) {
+    uint64_t d, A, B, C;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(A) : "f"(a0), "f"(a1));
+    asm("mov.b64 %0, {%1, %1};" : "=l"(B) : "f"(b));
+    asm("mov.b64 %0, {%1, %1};" : "=l"(C) : "f"(c));
+    asm("fma.rn.f32x2 %0, %1, %2, %3;" : "=l"(d) : "l"(A), "l"(B), "l"(C));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(d0), "=f"(d1) : "l"(d));
+}
+__device__ __forceinline__ void add2(float &d0, float &d1, float a0, float a1) {
+    uint64_t d, A, D;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(A) : "f"(a0), "f"(a1));
+    asm("mov.b64 %0, {%1, %2};" : "=l"(D) : "f"(d0), "f"(d1));
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(D), "l"(A));
+    asm("mov.b64 {%0, %1}, %2;" : "=f"(d0), "=f"(d1) : "l"(d));
+}
+// 2^x for x <= 0 on the FMA pipe: x = n + f with n the nearest integer, a cubic for 2^f on [-0.5, 0.5] (relative
+// error 7.5e-5, below the bf16 rounding of the probabilities), n added to the exponent field
+__device__ __forceinline__ float exp2_poly(float x) {
+    x = fmaxf(x, -125.f);
+    const float magic = 12582912.f;
+    const float xr = x + magic;
+    const float f = x - (xr - magic);
+    float p = fmaf(f, 0.05517113f, 0.24261114f);
+    p = fmaf(p, f, 0.69326111f);
+    p = fmaf(p, f, 0.99992807f);
+    return __uint_as_float(__float_as_uint(p) + (__float_as_uint(xr) << 23));
+}
+// 4 x 4 transpose of 16-byte units across the 4 lanes of a quad (l = lane & 3): on entry u[0..3] are the units of
+// this lane's own row; on return u[j] is unit l of the row held by quad lane j.  Every lane of the warp takes part.
+__device__ __forceinline__ void quad_transpose(uint4 (&u)[4], int l) {
+#pragma unroll
+    for (int s = 2; s >= 1; s >>= 1) {
+        const bool up = (l & s) != 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            if (i & s) continue;
+            const uint4 send = up ? u[i] : u[i ^ s];
+            uint4 recv;
+            recv.x = __shfl_xor_sync(0xffffffffu, send.x, s); recv.y = __shfl_xor_sync(0xffffffffu, send.y, s);
+            recv.z = __shfl_xor_sync(0xffffffffu, send.z, s); recv.w = __shfl_xor_sync(0xffffffffu, send.w, s);
+            if (up) u[i] = recv; else u[i ^ s] = recv;
+        }
+    }
+}
 __device__ __forceinline__ float fast_exp2(float x) {
     float y;
     asm("ex2.approx.ftz.f32 %0, %1;" : "=f"(y) : "f"(x));
@@ -123,25 +233,32 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     // barrier map (8 bytes each)
     const uint32_t q_full = bar0, q_free = bar0 + 8;
     auto k_full = [&](int s) { return bar0 + 16 + 8u * s; };
-    auto k_free = [&](int s) { return bar0 + 32 + 8u * s; };
-    auto v_full = [&](int s) { return bar0 + 48 + 8u * s; };
-    auto v_free = [&](int s) { return bar0 + 64 + 8u * s; };
-    auto s_full = [&](int w) { return bar0 + 80 + 8u * w; };
-    auto p_ready = [&](int w) { return bar0 + 96 + 8u * w; };
-    auto pv_done = [&](int w) { return bar0 + 112 + 8u * w; };
-    const uint32_t drain_bar = bar0 + 128;
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_al + S::kBarOff + 136);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_al + S::kBarOff + 144);
+    auto k_free = [&](int s) { return bar0 + 16 + 8u * (kKvStages + s); };
+    auto v_full = [&](int s) { return bar0 + 16 + 8u * (2 * kKvStages + s); };
+    auto v_free = [&](int s) { return bar0 + 16 + 8u * (3 * kKvStages + s); };
+    const uint32_t bar1 = bar0 + 16 + 8u * 4 * kKvStages;
+    auto s_full = [&](int w) { return bar1 + 8u * w; };
+    auto p_ready = [&](int w) { return bar1 + 16 + 8u * w; };
+    auto pv_done = [&](int w) { return bar1 + 32 + 8u * w; };
+    auto s_free = [&](int w) { return bar1 + 48 + 8u * w; };
+    auto drain_bar = [&](int w) { return bar1 + 64 + 8u * w; };
+    auto q_ready = [&](int w) { return bar1 + 80 + 8u * w; };
+    auto merge_bar = [&](int w) { return bar1 + 96 + 8u * w; };
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_al + S::kBarOff + 16 + 8 * 4 * kKvStages + 112);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_al + S::kBarOff + 16 + 8 * 4 * kKvStages + 120);
+    volatile int *merge_flag = reinterpret_cast<volatile int *>(smem_al + S::kBarOff + 16 + 8 * 4 * kKvStages + 128);   // [2]
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
-        tc::mbar_init(q_full, 1); tc::mbar_init(q_free, 1);
+        tc::mbar_init(q_full, 1); tc::mbar_init(q_free, 2);   // *_free: one commit per group's MMA issuer
         for (int s = 0; s < kKvStages; ++s) {
-            tc::mbar_init(k_full(s), 1); tc::mbar_init(k_free(s), 1);
-            tc::mbar_init(v_full(s), 1); tc::mbar_init(v_free(s), 1);
+            tc::mbar_init(k_full(s), 1); tc::mbar_init(k_free(s), 2);
+            tc::mbar_init(v_full(s), 1); tc::mbar_init(v_free(s), 2);
         }
-        for (int w = 0; w < 2; ++w) { tc::mbar_init(s_full(w), 1); tc::mbar_init(p_ready(w), 4); tc::mbar_init(pv_done(w), 1); }
-        tc::mbar_init(drain_bar, 1);
+        for (int w = 0; w < 2; ++w) { tc::mbar_init(s_full(w), 1); tc::mbar_init(p_ready(w), 4); tc::mbar_init(pv_done(w), 1);
+                                      tc::mbar_init(s_free(w), 4); tc::mbar_init(q_ready(w), 4);
+                                      tc::mbar_init(merge_bar(w), 128); }
+        tc::mbar_init(drain_bar(0), 1); tc::mbar_init(drain_bar(1), 1);
         *abort_flag = 0;
         tc::fence_barrier_init();
         tc::fence_proxy_async();
@@ -151,43 +268,62 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
-    // tensor-memory columns: S_w / P_w at w*128, O_w at 256 + w*128
-    const int n_items = *a.n_items;
+    // tensor-memory columns of group g (base g*256): S_g 0..63, P_g 64..95, the first 64 head-dim columns of Q_g as
+    // bf16 pairs 96..127, O_g 128..255
     const int tok_per_group = 128 / a.G;
-    const int pages_per_tile = kKeysPerTile / a.page_size;
-    const uint32_t page_bytes = (uint32_t)a.page_size * 128u;  // one page's rows inside a 64-wide half
+    // K/V stage layout.  One TMA box ("unit") brings box_rows cache rows of one page, both 64-wide halves of the
+    // head dim: [half][box_rows][128 bytes], 128-byte swizzle inside each half block.  A stage holds the 128 / box_rows
+    // units of a key tile one after the other.  The tensor cores want the 8-row groups of an operand at ONE stride, so
+    // the 64 keys of a half tile are chosen as 8 groups at a fixed stride:
+    //   box_rows 16: group hh of every unit (keys u*16 + hh*8 + 0..7: a permutation of the tile's keys, applied
+    //                alike to the scores, the mask and the V rows), stride = unit size;
+    //   box_rows  8: units 8*hh .. 8*hh+7 (natural key order), stride = unit size;
+    //   box_rows 64: unit hh, its 8 groups (natural key order), stride = 1024 bytes.
+    const uint32_t hstride = (uint32_t)a.box_rows * 128u;            // between the two halves of the head dim in a unit
+    const uint32_t unit_bytes = hstride * kHalves;
+    const int units_per_tile = kKeysPerTile / a.box_rows;
+    const bool perm = a.box_rows == 16;
+    const uint32_t sbo = a.box_rows == 64 ? 1024u : unit_bytes;
+    const uint32_t half_off = a.box_rows == 16 ? 1024u : (a.box_rows == 8 ? 8u * unit_bytes : unit_bytes);
 
     if (warp == 8) {
         // ------------------------------ TMA producer (whole warp) ------------------------------
         uint32_t n_item = 0, kt = 0;
         bool ok = true;
-        for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++n_item) {
-            const AttnWork w = a.items[it];
+        RunIter run(a);
+        RunPiece pc;
+        for (; ok && run.next(a, pc); ++n_item) {
+            const AttnWork &w = pc.w;
             if (lane == 0) {
                 ok = tc::mbar_wait(q_free, (n_item & 1) ^ 1, abort_flag);
                 if (ok) {
-                    tc::mbar_arrive_expect_tx(q_full, 2 * S::kQBytes);
-                    for (int g = 0; g < 2; ++g)
-                        for (int h = 0; h < kHalves; ++h)
-                            tma_load_3d(smem_base + S::kQOff + g * S::kQBytes + h * kHalfQ, &tmQ, q_full, h * 64,
-                                        w.kv_head * a.G, w.q_start + g * tok_per_group);
+                    if (kHalves > 1) {
+                        tc::mbar_arrive_expect_tx(q_full, 2 * S::kQBytes);
+                        for (int g = 0; g < 2; ++g)
+                            for (int h = 1; h < kHalves; ++h)
+                                tma_load_3d(smem_base + S::kQOff + g * S::kQBytes + (h - 1) * kHalfQ, &tmQ, q_full, h * 64,
+                                            w.kv_head * a.G, w.q_start + g * tok_per_group);
+                    } else {
+                        tc::mbar_arrive(q_full);   // nothing of Q goes through shared memory at this head dim
+                    }
                 }
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
-            const int n_tiles = (w.kv_end + kKeysPerTile - 1) / kKeysPerTile;
-            for (int j = 0; j < n_tiles && ok; ++j, ++kt) {
+            for (int j = pc.t0; j < pc.t1 && ok; ++j, ++kt) {
                 const int st = kt % kKvStages;
                 const uint32_t par = ((kt / kKvStages) & 1) ^ 1;
                 const int kbase = j * kKeysPerTile;
-                const int n_pages = min(pages_per_tile, (w.kv_end - kbase + a.page_size - 1) / a.page_size);
-                // every lane looks up one page of the tile
-                int page = -1;
-                if (lane < n_pages) {
-                    page = a.block_tables[(size_t)w.req * a.max_blocks + kbase / a.page_size + lane];
-                    if (page < 0 || page >= a.num_pages) { report(a.status, ALORA_ERR_PAGE_RANGE); page = -1; }
+                const int n_units = min(units_per_tile, (w.kv_end - kbase + a.box_rows - 1) / a.box_rows);
+                // every lane looks up the page of one unit of the tile
+                int row = -1;
+                if (lane < n_units) {
+                    const int key = kbase + lane * a.box_rows;
+                    const int page = a.block_tables[(size_t)w.req * a.max_blocks + key / a.page_size];
+                    if (page < 0 || page >= a.num_pages) report(a.status, ALORA_ERR_PAGE_RANGE);
+                    else row = (page * 2 * a.Hkv + w.kv_head) * a.page_size + key % a.page_size;   // K plane
                 }
-                const unsigned valid = __ballot_sync(0xffffffffu, page >= 0);
-                const uint32_t bytes = (uint32_t)__popc(valid) * page_bytes * kHalves;
+                const unsigned valid = __ballot_sync(0xffffffffu, row >= 0);
+                const uint32_t bytes = (uint32_t)__popc(valid) * unit_bytes;
                 for (int plane = 0; plane < 2 && ok; ++plane) {
                     const uint32_t fullb = plane == 0 ? k_full(st) : v_full(st);
                     const uint32_t freeb = plane == 0 ? k_free(st) : v_free(st);
@@ -196,75 +332,94 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         if (ok) tc::mbar_arrive_expect_tx(fullb, bytes);
                     }
                     ok = __shfl_sync(0xffffffffu, ok, 0);
-                    if (ok && page >= 0) {
-                        const uint32_t dst = smem_base + (plane == 0 ? S::kKOff : S::kVOff) + st * S::kKvBytes +
-                                             lane * page_bytes;
-                        const int row = ((page * 2 + plane) * a.Hkv + w.kv_head) * a.page_size;
-                        for (int h = 0; h < kHalves; ++h)
-                            tc::tma_load_2d(dst + h * kHalfQ, &tmKV, fullb, h * 64, row);
-                    }
+                    if (ok && row >= 0)   // one box: both halves of the head dim
+                        tma_load_3d(smem_base + (plane == 0 ? S::kKOff : S::kVOff) + st * S::kKvBytes + lane * unit_bytes,
+                                    &tmKV, fullb, 0, row + plane * a.Hkv * a.page_size, 0);
                 }
             }
         }
         (void)ok;
-    } else if (warp == 9) {
-        if (lane == 0) {
-            // ------------------------------ MMA issuer ------------------------------
-            constexpr uint32_t idesc_s = tc::idesc_bf16_f32(128, kKeysPerTile);
-            constexpr uint32_t idesc_pv = idesc_bf16_f32_bmn(128, HD);
-            uint32_t n_item = 0, kt = 0, np[2] = {0, 0};
-            bool ok = true;
-            auto issue_s = [&](int w, int st) {
-                const uint32_t qa = smem_base + S::kQOff + w * S::kQBytes;
-                const uint32_t ka = smem_base + S::kKOff + st * S::kKvBytes;
-                for (int h = 0; h < kHalves; ++h) {
-                    const uint64_t da = tc::smem_desc_k_sw128(qa + h * kHalfQ), db = tc::smem_desc_k_sw128(ka + h * kHalfQ);
-                    for (int k = 0; k < 4; ++k)
-                        tc::mma_bf16(tmem_base + w * 128, da + 2 * k, db + 2 * k, idesc_s, (h | k) != 0 ? 1u : 0u);
+    } else if (warp == 9 || warp == 10) {
+        // ------------------------------ MMA issuers: warp 9 for group 0, warp 10 for group 1 ------------------------------
+        // Keys are processed in half tiles of 64.  S_g of the next half is issued as soon as group g has copied the
+        // current scores into registers (s_free), so it runs underneath that group's softmax; P_g V of the current
+        // half follows when the group has written P_g (p_ready).  Each group has its own issuing warp, so neither
+        // group's chain ever waits behind a barrier of the other.  The whole warp walks the schedule (uniform
+        // control flow keeps the descriptors in uniform registers); one elected lane issues the tensor-core
+        // instructions and their commits.
+        const int g = warp - 9;
+        const bool leader = elect_one();
+        constexpr uint32_t idesc_s = tc::idesc_bf16_f32(128, kHalfKeys);
+        constexpr uint32_t idesc_pv = idesc_bf16_f32_bmn(128, HD);
+        uint32_t n_item = 0, kt = 0, nh = 0;   // nh: half tiles handled so far (phase counter of the group's barriers)
+        bool ok = true;
+        const uint32_t qa = smem_base + S::kQOff + g * S::kQBytes;
+        const uint32_t s_tmem = tmem_base + g * 256, p_tmem = s_tmem + 64, q_tmem = s_tmem + 96, o_tmem = s_tmem + 128;
+        // S_g = Q_g K^T for the 64 keys of half `hh` of the K tile in stage st
+        auto issue_s = [&](int st, int hh) {
+            const uint32_t ka = smem_base + S::kKOff + st * S::kKvBytes + hh * half_off;
+            if (leader) {
+                // head-dim columns 0..63: A = Q_g from tensor memory; the rest: A = Q_g from shared memory
+                const uint64_t db0 = smem_desc_k_sw128_sbo(ka, sbo);
+#pragma unroll
+                for (int k = 0; k < 4; ++k) mma_bf16_ts(s_tmem, q_tmem + 8 * k, db0 + 2 * k, idesc_s, k != 0 ? 1u : 0u);
+#pragma unroll
+                for (int h = 1; h < kHalves; ++h) {
+                    const uint64_t da = tc::smem_desc_k_sw128(qa + (h - 1) * kHalfQ), db = smem_desc_k_sw128_sbo(ka + h * hstride, sbo);
+#pragma unroll
+                    for (int k = 0; k < 4; ++k) tc::mma_bf16(s_tmem, da + 2 * k, db + 2 * k, idesc_s, 1u);
                 }
-                tc::mma_commit(s_full(w));
-            };
-            for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x, ++n_item) {
-                const AttnWork w = a.items[it];
-                const int n_tiles = (w.kv_end + kKeysPerTile - 1) / kKeysPerTile;
-                if (!tc::mbar_wait(q_full, n_item & 1, abort_flag)) { ok = false; break; }
-                if (!tc::mbar_wait(k_full(kt % kKvStages), (kt / kKvStages) & 1, abort_flag)) { ok = false; break; }
-                tc::tc_fence_after();
-                issue_s(0, kt % kKvStages);
-                issue_s(1, kt % kKvStages);
-                tc::mma_commit(k_free(kt % kKvStages));
-                if (n_tiles == 1) tc::mma_commit(q_free);
-                for (int j = 0; j < n_tiles && ok; ++j, ++kt) {
-                    const int st = kt % kKvStages;
-                    const bool more = j + 1 < n_tiles;
-                    for (int g = 0; g < 2; ++g) {
-                        if (!tc::mbar_wait(p_ready(g), np[g] & 1, abort_flag)) { ok = false; break; }
-                        ++np[g];
-                        if (g == 0 && !tc::mbar_wait(v_full(st), (kt / kKvStages) & 1, abort_flag)) { ok = false; break; }
-                        tc::tc_fence_after();
-                        const uint32_t va = smem_base + S::kVOff + st * S::kKvBytes;
-                        for (int k = 0; k < kKeysPerTile / 16; ++k)  // 16 keys per step: 8 packed columns of P
-                            mma_bf16_ts(tmem_base + 256 + g * 128, tmem_base + g * 128 + 8 * k,
-                                        smem_desc_mn_sw128(va + k * 2048, kHalfQ), idesc_pv, (j | k) != 0 ? 1u : 0u);
-                        tc::mma_commit(pv_done(g));
-                        if (g == 1) tc::mma_commit(v_free(st));
-                        if (more) {
-                            const int st1 = (kt + 1) % kKvStages;
-                            if (g == 0 && !tc::mbar_wait(k_full(st1), ((kt + 1) / kKvStages) & 1, abort_flag)) { ok = false; break; }
-                            tc::tc_fence_after();
-                            issue_s(g, st1);
-                            if (g == 1) {
-                                tc::mma_commit(k_free(st1));
-                                if (j + 2 == n_tiles) tc::mma_commit(q_free);  // last S products of the item issued
-                            }
-                        }
-                    }
-                }
+                tc::mma_commit(s_full(g));
             }
-            // tensor-core work still in flight must finish before tensor memory is released
-            tc::mma_commit(drain_bar);
+        };
+        auto wait_all = [&](uint32_t bar, uint32_t parity) {
+            return __all_sync(0xffffffffu, tc::mbar_wait(bar, parity, abort_flag));
+        };
+        RunIter run(a);
+        RunPiece pc;
+        for (; ok && run.next(a, pc); ++n_item) {
+            const int n_half = 2 * (pc.t1 - pc.t0);   // both halves of every tile of the piece
+            if (!wait_all(q_full, n_item & 1)) { ok = false; break; }
+            if (!wait_all(q_ready(g), n_item & 1)) { ok = false; break; }
+            if (!wait_all(k_full(kt % kKvStages), (kt / kKvStages) & 1)) { ok = false; break; }
+            tc::tc_fence_after();
+            issue_s(kt % kKvStages, 0);
+            for (int i = 0; i < n_half && ok; ++i) {
+                const int st = kt % kKvStages;          // stage of half i
+                const int hh = i & 1;
+                // ---- scores of half i + 1
+                if (i + 1 < n_half) {
+                    const int st1 = hh ? (kt + 1) % kKvStages : st;
+                    if (hh && !wait_all(k_full(st1), ((kt + 1) / kKvStages) & 1)) { ok = false; break; }
+                    if (!wait_all(s_free(g), nh & 1)) { ok = false; break; }
+                    tc::tc_fence_after();
+                    issue_s(st1, hh ^ 1);
+                    // this group is done with the K tile once its second half has been issued (and with Q at the end)
+                    if (leader && hh == 0) tc::mma_commit(k_free(st1));
+                    if (leader && i + 2 == n_half) tc::mma_commit(q_free);
+                }
+                // ---- P V of half i
+                if (hh == 0 && !wait_all(v_full(st), (kt / kKvStages) & 1)) { ok = false; break; }
+                if (!wait_all(p_ready(g), nh & 1)) { ok = false; break; }
+                ++nh;
+                tc::tc_fence_after();
+                if (leader) {
+                    const uint32_t va = smem_base + S::kVOff + st * S::kKvBytes + hh * half_off;
+#pragma unroll
+                    for (int k = 0; k < kHalfKeys / 16; ++k)  // 16 keys per step (two 8-key groups): 8 packed columns of P
+                        mma_bf16_ts(o_tmem, p_tmem + 8 * k, smem_desc_mn_sw128(va + 2 * k * sbo, hstride, sbo), idesc_pv,
+                                    (i | k) != 0 ? 1u : 0u);
+                    tc::mma_commit(pv_done(g));
+                    if (hh == 1) tc::mma_commit(v_free(st));
+                }
+                if (hh == 1) ++kt;
+            }
+        }
+        // tensor-core work still in flight must finish before tensor memory is released
+        if (leader) {
+            tc::mma_commit(drain_bar(g));
             const long long t0 = clock64();
-            while (!tc::mbar_try_wait(drain_bar, 0) && clock64() - t0 < tc::kWaitCycleLimit) {}
+            while (!tc::mbar_try_wait(drain_bar(g), 0) && clock64() - t0 < tc::kWaitCycleLimit) {}
         }
     } else {
         // ------------------------------ softmax groups (warps 0..7) ------------------------------
@@ -272,127 +427,259 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const int q = warp & 3;                  // tensor-memory lane quarter
         const int row = q * 32 + lane;           // score row of this thread inside the group's tile
         const uint32_t lane_off = (uint32_t)(q * 32) << 16;
-        const uint32_t s_addr = tmem_base + g * 128 + lane_off;
-        const uint32_t o_addr = tmem_base + 256 + g * 128 + lane_off;
-        uint32_t n_s = 0, kt = 0;
+        const uint32_t s_addr = tmem_base + g * 256 + lane_off;          // scores of the current half tile (64 columns)
+        const uint32_t p_addr = s_addr + 64;                              // probabilities, bf16 pairs (32 columns)
+        const uint32_t q_addr = s_addr + 96;                              // first 64 head-dim columns of this Q row
+        const uint32_t o_addr = s_addr + 128;
+        uint32_t n_s = 0, kt = 0;   // n_s: half tiles of this group so far (phase counter of its barriers)
+        uint32_t n_mb = 0;          // phases of the group's merge barrier used so far
         bool ok = true;
-        for (int it = blockIdx.x; it < n_items && ok; it += gridDim.x) {
-            const AttnWork w = a.items[it];
-            const int n_tiles = (w.kv_end + kKeysPerTile - 1) / kKeysPerTile;
-            const int tok_local = g * tok_per_group + row / a.G;
-            const bool row_valid = tok_local < w.q_count;
+        RunIter run(a);
+        RunPiece pc, pc_next;
+        const int tok_local = g * tok_per_group + row / a.G;
+        // the first 64 head-dim columns of this thread's row of Q of a piece: global memory -> registers
+        uint32_t qv[32];
+        auto load_q = [&](const AttnWork &w) {
+            const bool valid = tok_local < w.q_count;
+            const uint4 *src = reinterpret_cast<const uint4 *>(
+                a.qkv + (size_t)(w.q_start + (valid ? tok_local : 0)) * a.N + (size_t)(w.kv_head * a.G + row % a.G) * HD);
+#pragma unroll
+            for (int x = 0; x < 8; ++x) {
+                const uint4 u = valid ? __ldg(src + x) : make_uint4(0, 0, 0, 0);
+                qv[4 * x] = u.x; qv[4 * x + 1] = u.y; qv[4 * x + 2] = u.z; qv[4 * x + 3] = u.w;
+            }
+        };
+        bool have = run.next(a, pc);
+        if (have) load_q(pc.w);
+        while (ok && have) {
+            const AttnWork &w = pc.w;
+            const int n_half = 2 * (pc.t1 - pc.t0);
+            {
+                // registers -> tensor memory, where they are the A operand of the first half of Q K^T (all earlier
+                // Q K^T of this group have completed: the group has consumed their scores)
+                tmem_st_32x32(q_addr, qv);
+                tmem_st_wait();
+                tc::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(q_ready(g));
+            }
             // position of this row's token; rows past the end of the block behave like its last token
             const int pos = w.kv_end - w.q_count + min(tok_local, w.q_count - 1);
             // exponent reference (a running maximum that is only moved when it has drifted by more than
             // 2^8, so the accumulator in tensor memory rarely needs rescaling) and row sum
             float m_ref = -INFINITY, l_run = 0.f;
-            for (int j = 0; j < n_tiles && ok; ++j, ++kt) {
-                const int kbase = j * kKeysPerTile;
+            for (int i = 0; i < n_half && ok; ++i, ++n_s) {
+                const int tbase = (pc.t0 + (i >> 1)) * kKeysPerTile;   // first key of the tile; column e of half hh is key
+                const int hh = i & 1;                        // tbase + (perm ? (e/8)*16 + hh*8 + e%8 : hh*64 + e)
                 if (!tc::mbar_wait(s_full(g), n_s & 1, abort_flag)) { ok = false; break; }
-                ++n_s;
                 tc::tc_fence_after();
-                uint32_t sv[kKeysPerTile];
+                uint32_t sv[kHalfKeys];
 #pragma unroll
-                for (int c = 0; c < kKeysPerTile; c += 32)
+                for (int c = 0; c < kHalfKeys; c += 32)
                     tc::tmem_ld_32x32(s_addr + c, reinterpret_cast<uint32_t(&)[32]>(sv[c]));
                 tc::tmem_ld_wait();
+                // the scores are in registers: the next half tile's Q K^T may overwrite them, underneath this softmax
+                tc::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(s_free(g));
                 float m_tile = -INFINITY;
-                if (kbase + kKeysPerTile - 1 > pos) {  // tile crosses this row's causal limit: mask
+                const bool masked = tbase + kKeysPerTile - 1 > pos;   // tile crosses this row's causal limit
+                if (masked) {
+                    const int k0 = tbase + (perm ? hh * 8 : hh * kHalfKeys);
 #pragma unroll
-                    for (int e = 0; e < kKeysPerTile; ++e) {
-                        if (kbase + e > pos) sv[e] = 0xff800000u;  // -inf
+                    for (int e = 0; e < kHalfKeys; ++e) {
+                        const int key = k0 + (perm ? (e >> 3) * 16 + (e & 7) : e);
+                        if (key > pos) sv[e] = 0xff800000u;  // -inf
                         m_tile = fmaxf(m_tile, __uint_as_float(sv[e]));
                     }
                 } else {
+                    float m0 = -INFINITY, m1 = -INFINITY;
 #pragma unroll
-                    for (int e = 0; e < kKeysPerTile; ++e) m_tile = fmaxf(m_tile, __uint_as_float(sv[e]));
+                    for (int e = 0; e < kHalfKeys; e += 4) {
+                        m0 = max3(m0, __uint_as_float(sv[e]), __uint_as_float(sv[e + 1]));
+                        m1 = max3(m1, __uint_as_float(sv[e + 2]), __uint_as_float(sv[e + 3]));
+                    }
+                    m_tile = fmaxf(m0, m1);
                 }
-                const bool bump = (m_tile - m_ref) * a.scale_log2 > 8.f;  // always true on an item's first tile
+                const bool bump = (m_tile - m_ref) * a.scale_log2 > 8.f;  // always true on an item's first half tile
                 float alpha = 1.f;
                 if (bump) {
                     alpha = fast_exp2((m_ref - m_tile) * a.scale_log2);
                     m_ref = m_tile;
                     l_run *= alpha;
                 }
-                if (j > 0 && __any_sync(0xffffffffu, bump)) {
-                    // O_w holds the earlier tiles' products relative to the old reference: once the last P V
-                    // has completed, scale the rows of this warp whose reference moved
-                    if (!tc::mbar_wait(pv_done(g), n_s & 1, abort_flag)) { ok = false; break; }
-                    tc::tc_fence_after();
-#pragma unroll 1
-                    for (int c = 0; c < HD; c += 32) {
-                        uint32_t v[32];
-                        tc::tmem_ld_32x32(o_addr + c, v);
-                        tc::tmem_ld_wait();
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha);
-                        tmem_st_32x32(o_addr + c, v);
-                    }
-                }
-                // probabilities (bf16) over the score columns, row sum in fp32
-                const float mb = m_ref * a.scale_log2;
+                // probabilities (bf16 pairs) and their row sum in fp32
+                // (a piece that starts at an item's last tile can hold rows that see none of its keys so far)
+                const float mb = m_ref == -INFINITY ? 0.f : m_ref * a.scale_log2;
                 float l0 = 0.f, l1 = 0.f;
+                uint32_t pk[kHalfKeys / 2];
+                if (masked) {
 #pragma unroll
-                for (int c = 0; c < kKeysPerTile; c += 32) {
-                    uint32_t pk[16];
-#pragma unroll
-                    for (int e = 0; e < 32; e += 2) {
-                        const float p0 = fast_exp2(fmaf(__uint_as_float(sv[c + e]), a.scale_log2, -mb));
-                        const float p1 = fast_exp2(fmaf(__uint_as_float(sv[c + e + 1]), a.scale_log2, -mb));
+                    for (int e = 0; e < kHalfKeys; e += 2) {
+                        const float p0 = fast_exp2(fmaf(__uint_as_float(sv[e]), a.scale_log2, -mb));
+                        const float p1 = fast_exp2(fmaf(__uint_as_float(sv[e + 1]), a.scale_log2, -mb));
                         l0 += p0;
                         l1 += p1;
-                        pk[e >> 1] = tc::pack_bf16(p0, p1);
+                        pk[e >> 1] = pack_cvt(p0, p1);
                     }
-                    tmem_st_32x16(s_addr + (c >> 1), pk);
+                } else {
+#pragma unroll
+                    for (int e = 0; e < kHalfKeys; e += 2) {
+                        float x0, x1, p0, p1;
+                        fma2(x0, x1, __uint_as_float(sv[e]), __uint_as_float(sv[e + 1]), a.scale_log2, -mb);
+                        if ((e & 7) == 6) { p0 = exp2_poly(x0); p1 = exp2_poly(x1); }   // a quarter of them on the FMA pipe
+                        else { p0 = fast_exp2(x0); p1 = fast_exp2(x1); }
+                        add2(l0, l1, p0, p1);
+                        pk[e >> 1] = pack_cvt(p0, p1);
+                    }
                 }
                 l_run += l0 + l1;
-                // V rows of keys at or beyond the item's causal limit are cleared before P V uses them
-                if (kbase + kKeysPerTile > w.kv_end) {
+                // P_g and O_g are still in use by the previous half tile's P V until it has completed
+                if (i > 0) {
+                    if (!tc::mbar_wait(pv_done(g), (n_s - 1) & 1, abort_flag)) { ok = false; break; }
+                    tc::tc_fence_after();
+                    if (__any_sync(0xffffffffu, bump)) {
+                        // O_g holds the earlier products relative to the old reference: scale the rows that moved
+#pragma unroll 1
+                        for (int c = 0; c < HD; c += 32) {
+                            uint32_t v[32];
+                            tc::tmem_ld_32x32(o_addr + c, v);
+                            tc::tmem_ld_wait();
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) v[e] = __float_as_uint(__uint_as_float(v[e]) * alpha);
+                            tmem_st_32x32(o_addr + c, v);
+                        }
+                    }
+                }
+                tmem_st_32x16(p_addr, reinterpret_cast<uint32_t(&)[16]>(pk[0]));
+                tmem_st_32x16(p_addr + 16, reinterpret_cast<uint32_t(&)[16]>(pk[16]));
+                // V rows of keys at or beyond the item's causal limit are cleared before the tile's first P V uses them
+                // (thread `row` of each group clears key tbase + row)
+                if (hh == 0) kt += (i > 0);   // tile index of this half
+                if (hh == 0 && tbase + kKeysPerTile > w.kv_end) {
                     const int st = kt % kKvStages;
                     if (!tc::mbar_wait(v_full(st), (kt / kKvStages) & 1, abort_flag)) { ok = false; break; }
-                    if (kbase + row >= w.kv_end) {
-                        uint8_t *vrow = smem_al + S::kVOff + st * S::kKvBytes + row * 128;
+                    if (tbase + row >= w.kv_end) {
+                        uint8_t *vrow = smem_al + S::kVOff + st * S::kKvBytes + (row / a.box_rows) * unit_bytes +
+                                        (row % a.box_rows) * 128;
                         for (int h = 0; h < kHalves; ++h)
 #pragma unroll
                             for (int x = 0; x < 8; ++x)
-                                reinterpret_cast<uint4 *>(vrow + h * kHalfQ)[x] = make_uint4(0, 0, 0, 0);
+                                reinterpret_cast<uint4 *>(vrow + h * hstride)[x] = make_uint4(0, 0, 0, 0);
                     }
                     tc::fence_proxy_async();
                 }
                 tmem_st_wait();
                 tc::tc_fence_before();
                 __syncwarp();
-                if (lane == 0) tc::mbar_arrive(p_ready(g));  // P_w (and O_w, if it was rescaled) ready for P V
+                if (lane == 0) tc::mbar_arrive(p_ready(g));  // P_g (and O_g, if it was rescaled) ready for P V
             }
+            ++kt;  // the piece's last tile
             if (!ok) break;
-            // the item's last P V, normalisation, store
+            // the next piece's rows of Q are fetched underneath this piece's last P V and its output
+            const bool have_next = run.next(a, pc_next);
+            if (have_next) load_q(pc_next.w);
+            // the piece's last P V; then normalisation and store, or (item cut by a run boundary) the partial result
             if (!tc::mbar_wait(pv_done(g), (n_s - 1) & 1, abort_flag)) { ok = false; break; }
             tc::tc_fence_after();
-            float o[HD];
-            {
-                const float inv = 1.f / l_run;
+            // Output rows: 4 adjacent lanes hold 4 adjacent rows.  Their 16-byte units are transposed inside the quad
+            // so that one store instruction writes 64 contiguous bytes of one row per quad (4x fewer memory lines
+            // per instruction than lane = row).
+            const int ql = lane & 3;
+            __nv_bfloat16 *dst_quad[4];
 #pragma unroll
+            for (int j = 0; j < 4; ++j) {
+                const int r = (row & ~3) + j;
+                const int tl = g * tok_per_group + r / a.G;
+                dst_quad[j] = tl < w.q_count
+                                  ? a.out + (size_t)(w.q_start + tl) * a.Nq + (size_t)(w.kv_head * a.G + r % a.G) * HD + ql * 8
+                                  : nullptr;
+            }
+            auto store_chunk = [&](int c, const float (&o)[32]) {   // 32 output columns from column c on
+                uint4 u[4];
+#pragma unroll
+                for (int x = 0; x < 4; ++x) {
+                    u[x].x = tc::pack_bf16(o[8 * x], o[8 * x + 1]); u[x].y = tc::pack_bf16(o[8 * x + 2], o[8 * x + 3]);
+                    u[x].z = tc::pack_bf16(o[8 * x + 4], o[8 * x + 5]); u[x].w = tc::pack_bf16(o[8 * x + 6], o[8 * x + 7]);
+                }
+                quad_transpose(u, ql);
+#pragma unroll
+                for (int j = 0; j < 4; ++j)
+                    if (dst_quad[j]) *reinterpret_cast<uint4 *>(dst_quad[j] + c) = u[j];
+            };
+            if (pc.n_parts == 1) {
+                const float inv = 1.f / l_run;
+#pragma unroll 1
+                for (int c = 0; c < HD; c += 32) {
+                    uint32_t v[32];
+                    tc::tmem_ld_32x32(o_addr + c, v);
+                    tc::tmem_ld_wait();
+                    float o[32];
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) o[e] = __uint_as_float(v[e]) * inv;
+                    store_chunk(c, o);
+                }
+                tc::tc_fence_before();
+            } else {
+                // this part's unnormalised rows, exponent references and sums go to its slot
+                const int grow = g * 128 + row;
+                float *po = a.part_o + (size_t)part_slot(pc.c_first, pc.part) * HD * 256 + grow;
+                float *pml = a.part_ml + (size_t)part_slot(pc.c_first, pc.part) * 512 + grow;
+#pragma unroll 1
                 for (int c = 0; c < HD; c += 32) {
                     uint32_t v[32];
                     tc::tmem_ld_32x32(o_addr + c, v);
                     tc::tmem_ld_wait();
 #pragma unroll
-                    for (int e = 0; e < 32; ++e) o[c + e] = __uint_as_float(v[e]) * inv;
+                    for (int e = 0; e < 32; ++e) __stcg(po + (size_t)(c + e) * 256, __uint_as_float(v[e]));
                 }
-            }
-            tc::tc_fence_before();
-            if (row_valid) {
-                const int token = w.q_start + tok_local;
-                const int head = w.kv_head * a.G + row % a.G;
-                uint4 *dst = reinterpret_cast<uint4 *>(a.out + (size_t)token * a.Nq + (size_t)head * HD);
+                tc::tc_fence_before();
+                __stcg(pml, m_ref);
+                __stcg(pml + 256, l_run);
+                __threadfence();
+                // all 128 rows of the group are in place -> one thread counts the part in -> all learn whether
+                // theirs was the last part of the item
+                tc::mbar_arrive(merge_bar(g));
+                if (!tc::mbar_wait(merge_bar(g), n_mb & 1, abort_flag)) { ok = false; break; }
+                ++n_mb;
+                if (row == 0) merge_flag[g] = atomicAdd(a.done + 2 * pc.item + g, 1);
+                tc::mbar_arrive(merge_bar(g));
+                if (!tc::mbar_wait(merge_bar(g), n_mb & 1, abort_flag)) { ok = false; break; }
+                ++n_mb;
+                if (merge_flag[g] == pc.n_parts - 1) {
+                    // last part in: merge all parts in their fixed order (the result does not depend on which part
+                    // finished last)
+                    __threadfence();
+                    float m_all = -INFINITY;
+                    for (int p = 0; p < pc.n_parts; ++p)
+                        m_all = fmaxf(m_all, __ldcg(a.part_ml + (size_t)part_slot(pc.c_first, p) * 512 + grow));
+                    float l_all = 0.f;
+                    for (int p = 0; p < pc.n_parts; ++p) {
+                        const float *ml = a.part_ml + (size_t)part_slot(pc.c_first, p) * 512 + grow;
+                        const float m_p = __ldcg(ml);
+                        if (m_p != -INFINITY) l_all += __ldcg(ml + 256) * fast_exp2((m_p - m_all) * a.scale_log2);
+                    }
+                    const float inv = 1.f / l_all;
+#pragma unroll 1
+                    for (int c = 0; c < HD; c += 32) {
+                        float o[32];
 #pragma unroll
-                for (int x = 0; x < HD / 8; ++x) {
-                    uint4 u;
-                    u.x = tc::pack_bf16(o[8 * x], o[8 * x + 1]); u.y = tc::pack_bf16(o[8 * x + 2], o[8 * x + 3]);
-                    u.z = tc::pack_bf16(o[8 * x + 4], o[8 * x + 5]); u.w = tc::pack_bf16(o[8 * x + 6], o[8 * x + 7]);
-                    dst[x] = u;
+                        for (int e = 0; e < 32; ++e) o[e] = 0.f;
+                        for (int p = 0; p < pc.n_parts; ++p) {
+                            const int slot = part_slot(pc.c_first, p);
+                            const float m_p = __ldcg(a.part_ml + (size_t)slot * 512 + grow);
+                            if (m_p == -INFINITY) continue;
+                            const float wgt = fast_exp2((m_p - m_all) * a.scale_log2) * inv;
+                            const float *src = a.part_o + ((size_t)slot * HD + c) * 256 + grow;
+#pragma unroll
+                            for (int e = 0; e < 32; ++e) o[e] = fmaf(__ldcg(src + (size_t)e * 256), wgt, o[e]);
+                        }
+                        store_chunk(c, o);
+                    }
                 }
             }
+            pc = pc_next;
+            have = have_next;
         }
     }
 
@@ -442,21 +729,26 @@ int launch_attend_tc(alora_ctx *ctx, const void *qkv, const BatchArgs &b, const 
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return -1;
     }
+    const int box_rows = d.page == 8 ? 8 : (d.page <= 32 ? 16 : 64);
     {
-        cuuint64_t dims[2] = {(cuuint64_t)d.hd, (cuuint64_t)b.num_pages * 2 * d.Hkv * d.page};
-        cuuint64_t strides[1] = {(cuuint64_t)d.hd * 2};
-        cuuint32_t box[2] = {64, (cuuint32_t)d.page};
-        cuuint32_t es[2] = {1, 1};
-        if (enc(&tmKV, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 2, const_cast<void *>(pool), dims, strides, box, es,
+        // the pool as (64 columns, cache rows, 64-wide halves of the head dim): one box = box_rows rows, both halves
+        const cuuint64_t halves = (cuuint64_t)d.hd / 64;
+        cuuint64_t dims[3] = {64, (cuuint64_t)b.num_pages * 2 * d.Hkv * d.page, halves};
+        cuuint64_t strides[2] = {(cuuint64_t)d.hd * 2, 128};
+        cuuint32_t box[3] = {64, (cuuint32_t)box_rows, (cuuint32_t)halves};
+        cuuint32_t es[3] = {1, 1, 1};
+        if (enc(&tmKV, CU_TENSOR_MAP_DATA_TYPE_BFLOAT16, 3, const_cast<void *>(pool), dims, strides, box, es,
                 CU_TENSOR_MAP_INTERLEAVE_NONE, CU_TENSOR_MAP_SWIZZLE_128B, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
                 CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) != CUDA_SUCCESS)
             return -1;
     }
     AttnArgs a{};
     a.items = ctx->d_attn_items; a.n_items = ctx->d_counts + 1; a.block_tables = b.block_tables;
-    a.max_blocks = b.max_blocks; a.num_pages = b.num_pages; a.Hkv = d.Hkv; a.G = d.G; a.page_size = d.page;
-    a.N = d.N; a.Nq = d.Nq; a.scale_log2 = d.softmax_scale * 1.4426950408889634f;
+    a.max_blocks = b.max_blocks; a.num_pages = b.num_pages; a.Hkv = d.Hkv; a.G = d.G; a.page_size = d.page; a.box_rows = box_rows;
+    a.N = d.N; a.Nq = d.Nq; a.qkv = (const __nv_bfloat16 *)qkv; a.scale_log2 = d.softmax_scale * 1.4426950408889634f;
     a.out = (__nv_bfloat16 *)out; a.status = ctx->d_status;
+    a.run_counts = ctx->d_counts + 6; a.cta_start = ctx->d_attn_cta_start; a.done = ctx->d_attn_done;
+    a.part_o = ctx->d_attn_part_o; a.part_ml = ctx->d_attn_part_ml;
     const int max_items = (b.T / ctx->attn_q_block + b.R) * d.Hkv;
     const int grid = std::max(1, std::min(ctx->sm_count, max_items));
     ProfScope prof(ctx, KK_ATTENTION, s);
