@@ -42,48 +42,19 @@ struct AttnArgs {
     const __nv_bfloat16 *qkv;  // [T][N], query part first
     __nv_bfloat16 *out;        // [T][Nq]
     int32_t *status;
-    // runs: the concatenated key tiles of all items, cut into equal runs, one per block
-    const int32_t *run_counts;  // [0] all key tiles, [1] tiles per run
-    const int32_t *cta_start;   // [blocks] item that holds the first tile of the block's run
-    int32_t *done;              // [2 * items] parts finished per (item, row group)
-    float *part_o;              // [2 * blocks][hd][256] unnormalised output of a part, column-major over the 256 rows
-    float *part_ml;             // [2 * blocks][2][256] exponent reference and row sum of a part
 };
 
-// Walks the pieces of a block's run: one piece = tiles [t0, t1) of one item.  An item cut by run boundaries is
-// worked on by n_parts consecutive blocks (this block holds part `part`, the first of them is block c_first);
-// their partial results are merged by whichever part finishes last.
-struct RunPiece {
-    AttnWork w;
-    int item, t0, t1, n_parts, part, c_first;
-};
-struct RunIter {
-    int gt, gt_end, it, len;
-    __device__ explicit RunIter(const AttnArgs &a) {
-        const int total = a.run_counts[0];
-        len = a.run_counts[1];
-        gt = min(total, (int)blockIdx.x * len);
-        gt_end = min(total, gt + len);
-        it = gt < gt_end ? a.cta_start[blockIdx.x] : 0;
-    }
-    __device__ bool next(const AttnArgs &a, RunPiece &p) {
-        if (gt >= gt_end) return false;
-        p.w = a.items[it];
-        const int n_tiles = (p.w.kv_end + kKeysPerTile - 1) / kKeysPerTile;
-        p.item = it;
-        p.t0 = gt - p.w.split;
-        p.t1 = min(n_tiles, gt_end - p.w.split);
-        p.c_first = p.w.split / len;
-        p.n_parts = (p.w.split + n_tiles - 1) / len - p.c_first + 1;
-        p.part = (int)blockIdx.x - p.c_first;
-        gt = p.w.split + p.t1;
-        ++it;
+// The items a block works through: blockIdx, blockIdx + blocks, ...
+struct ItemIter {
+    int it;
+    __device__ ItemIter() : it((int)blockIdx.x) {}
+    __device__ bool next(const AttnArgs &a, int n_items, AttnWork &w) {
+        if (it >= n_items) return false;
+        w = a.items[it];
+        it += (int)gridDim.x;
         return true;
     }
 };
-// partial-result slot of part `part` of an item whose first part is held by block c_first: a block holds at
-// most one part > 0 (the piece its run starts with) and at most one part 0 of a cut item (the piece it ends with)
-__device__ __forceinline__ int part_slot(int c_first, int part) { return 2 * (c_first + part) + (part == 0 ? 1 : 0); }
 
 template <int HD>
 struct AttnSmem {
@@ -243,10 +214,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     auto s_free = [&](int w) { return bar1 + 48 + 8u * w; };
     auto drain_bar = [&](int w) { return bar1 + 64 + 8u * w; };
     auto q_ready = [&](int w) { return bar1 + 80 + 8u * w; };
-    auto merge_bar = [&](int w) { return bar1 + 96 + 8u * w; };
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_al + S::kBarOff + 16 + 8 * 4 * kKvStages + 112);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_al + S::kBarOff + 16 + 8 * 4 * kKvStages + 120);
-    volatile int *merge_flag = reinterpret_cast<volatile int *>(smem_al + S::kBarOff + 16 + 8 * 4 * kKvStages + 128);   // [2]
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_al + S::kBarOff + 16 + 8 * 4 * kKvStages + 96);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_al + S::kBarOff + 16 + 8 * 4 * kKvStages + 104);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
@@ -256,8 +225,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             tc::mbar_init(v_full(s), 1); tc::mbar_init(v_free(s), 2);
         }
         for (int w = 0; w < 2; ++w) { tc::mbar_init(s_full(w), 1); tc::mbar_init(p_ready(w), 4); tc::mbar_init(pv_done(w), 1);
-                                      tc::mbar_init(s_free(w), 4); tc::mbar_init(q_ready(w), 4);
-                                      tc::mbar_init(merge_bar(w), 128); }
+                                      tc::mbar_init(s_free(w), 4); tc::mbar_init(q_ready(w), 4); }
         tc::mbar_init(drain_bar(0), 1); tc::mbar_init(drain_bar(1), 1);
         *abort_flag = 0;
         tc::fence_barrier_init();
@@ -270,6 +238,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const uint32_t tmem_base = *tmem_slot;
     // tensor-memory columns of group g (base g*256): S_g 0..63, P_g 64..95, the first 64 head-dim columns of Q_g as
     // bf16 pairs 96..127, O_g 128..255
+    const int n_items = *a.n_items;
     const int tok_per_group = 128 / a.G;
     // K/V stage layout.  One TMA box ("unit") brings box_rows cache rows of one page, both 64-wide halves of the
     // head dim: [half][box_rows][128 bytes], 128-byte swizzle inside each half block.  A stage holds the 128 / box_rows
@@ -290,10 +259,9 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         // ------------------------------ TMA producer (whole warp) ------------------------------
         uint32_t n_item = 0, kt = 0;
         bool ok = true;
-        RunIter run(a);
-        RunPiece pc;
-        for (; ok && run.next(a, pc); ++n_item) {
-            const AttnWork &w = pc.w;
+        ItemIter items;
+        AttnWork w;
+        for (; ok && items.next(a, n_items, w); ++n_item) {
             if (lane == 0) {
                 ok = tc::mbar_wait(q_free, (n_item & 1) ^ 1, abort_flag);
                 if (ok) {
@@ -309,7 +277,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 }
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
-            for (int j = pc.t0; j < pc.t1 && ok; ++j, ++kt) {
+            const int n_tiles = (w.kv_end + kKeysPerTile - 1) / kKeysPerTile;
+            for (int j = 0; j < n_tiles && ok; ++j, ++kt) {
                 const int st = kt % kKvStages;
                 const uint32_t par = ((kt / kKvStages) & 1) ^ 1;
                 const int kbase = j * kKeysPerTile;
@@ -375,10 +344,10 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         auto wait_all = [&](uint32_t bar, uint32_t parity) {
             return __all_sync(0xffffffffu, tc::mbar_wait(bar, parity, abort_flag));
         };
-        RunIter run(a);
-        RunPiece pc;
-        for (; ok && run.next(a, pc); ++n_item) {
-            const int n_half = 2 * (pc.t1 - pc.t0);   // both halves of every tile of the piece
+        ItemIter items;
+        AttnWork w;
+        for (; ok && items.next(a, n_items, w); ++n_item) {
+            const int n_half = 2 * ((w.kv_end + kKeysPerTile - 1) / kKeysPerTile);   // both halves of every tile
             if (!wait_all(q_full, n_item & 1)) { ok = false; break; }
             if (!wait_all(q_ready(g), n_item & 1)) { ok = false; break; }
             if (!wait_all(k_full(kt % kKvStages), (kt / kKvStages) & 1)) { ok = false; break; }
@@ -432,10 +401,9 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const uint32_t q_addr = s_addr + 96;                              // first 64 head-dim columns of this Q row
         const uint32_t o_addr = s_addr + 128;
         uint32_t n_s = 0, kt = 0;   // n_s: half tiles of this group so far (phase counter of its barriers)
-        uint32_t n_mb = 0;          // phases of the group's merge barrier used so far
         bool ok = true;
-        RunIter run(a);
-        RunPiece pc, pc_next;
+        ItemIter items;
+        AttnWork w, w_next;
         const int tok_local = g * tok_per_group + row / a.G;
         // the first 64 head-dim columns of this thread's row of Q of a piece: global memory -> registers
         uint32_t qv[32];
@@ -449,27 +417,26 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 qv[4 * x] = u.x; qv[4 * x + 1] = u.y; qv[4 * x + 2] = u.z; qv[4 * x + 3] = u.w;
             }
         };
-        bool have = run.next(a, pc);
-        if (have) load_q(pc.w);
+        // registers -> tensor memory, where they are the A operand of the first half of Q K^T (all earlier Q K^T of
+        // this group have completed by then: the group has consumed their scores)
+        auto publish_q = [&]() {
+            tmem_st_32x32(q_addr, qv);
+            tmem_st_wait();
+            tc::tc_fence_before();
+            __syncwarp();
+            if (lane == 0) tc::mbar_arrive(q_ready(g));
+        };
+        bool have = items.next(a, n_items, w);
+        if (have) { load_q(w); publish_q(); }
         while (ok && have) {
-            const AttnWork &w = pc.w;
-            const int n_half = 2 * (pc.t1 - pc.t0);
-            {
-                // registers -> tensor memory, where they are the A operand of the first half of Q K^T (all earlier
-                // Q K^T of this group have completed: the group has consumed their scores)
-                tmem_st_32x32(q_addr, qv);
-                tmem_st_wait();
-                tc::tc_fence_before();
-                __syncwarp();
-                if (lane == 0) tc::mbar_arrive(q_ready(g));
-            }
+            const int n_half = 2 * ((w.kv_end + kKeysPerTile - 1) / kKeysPerTile);
             // position of this row's token; rows past the end of the block behave like its last token
             const int pos = w.kv_end - w.q_count + min(tok_local, w.q_count - 1);
             // exponent reference (a running maximum that is only moved when it has drifted by more than
             // 2^8, so the accumulator in tensor memory rarely needs rescaling) and row sum
             float m_ref = -INFINITY, l_run = 0.f;
             for (int i = 0; i < n_half && ok; ++i, ++n_s) {
-                const int tbase = (pc.t0 + (i >> 1)) * kKeysPerTile;   // first key of the tile; column e of half hh is key
+                const int tbase = (i >> 1) * kKeysPerTile;   // first key of the tile; column e of half hh is key
                 const int hh = i & 1;                        // tbase + (perm ? (e/8)*16 + hh*8 + e%8 : hh*64 + e)
                 if (!tc::mbar_wait(s_full(g), n_s & 1, abort_flag)) { ok = false; break; }
                 tc::tc_fence_after();
@@ -509,8 +476,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     l_run *= alpha;
                 }
                 // probabilities (bf16 pairs) and their row sum in fp32
-                // (a piece that starts at an item's last tile can hold rows that see none of its keys so far)
-                const float mb = m_ref == -INFINITY ? 0.f : m_ref * a.scale_log2;
+                const float mb = m_ref * a.scale_log2;
                 float l0 = 0.f, l1 = 0.f;
                 uint32_t pk[kHalfKeys / 2];
                 if (masked) {
@@ -574,12 +540,13 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(p_ready(g));  // P_g (and O_g, if it was rescaled) ready for P V
             }
-            ++kt;  // the piece's last tile
+            ++kt;  // the item's last tile
             if (!ok) break;
-            // the next piece's rows of Q are fetched underneath this piece's last P V and its output
-            const bool have_next = run.next(a, pc_next);
-            if (have_next) load_q(pc_next.w);
-            // the piece's last P V; then normalisation and store, or (item cut by a run boundary) the partial result
+            // the next item's rows of Q go to tensor memory underneath this item's last P V, so that its first
+            // Q K^T runs underneath this item's output
+            const bool have_next = items.next(a, n_items, w_next);
+            if (have_next) { load_q(w_next); publish_q(); }
+            // the item's last P V, normalisation, store
             if (!tc::mbar_wait(pv_done(g), (n_s - 1) & 1, abort_flag)) { ok = false; break; }
             tc::tc_fence_after();
             // Output rows: 4 adjacent lanes hold 4 adjacent rows.  Their 16-byte units are transposed inside the quad
@@ -607,7 +574,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 for (int j = 0; j < 4; ++j)
                     if (dst_quad[j]) *reinterpret_cast<uint4 *>(dst_quad[j] + c) = u[j];
             };
-            if (pc.n_parts == 1) {
+            {
                 const float inv = 1.f / l_run;
 #pragma unroll 1
                 for (int c = 0; c < HD; c += 32) {
@@ -620,65 +587,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     store_chunk(c, o);
                 }
                 tc::tc_fence_before();
-            } else {
-                // this part's unnormalised rows, exponent references and sums go to its slot
-                const int grow = g * 128 + row;
-                float *po = a.part_o + (size_t)part_slot(pc.c_first, pc.part) * HD * 256 + grow;
-                float *pml = a.part_ml + (size_t)part_slot(pc.c_first, pc.part) * 512 + grow;
-#pragma unroll 1
-                for (int c = 0; c < HD; c += 32) {
-                    uint32_t v[32];
-                    tc::tmem_ld_32x32(o_addr + c, v);
-                    tc::tmem_ld_wait();
-#pragma unroll
-                    for (int e = 0; e < 32; ++e) __stcg(po + (size_t)(c + e) * 256, __uint_as_float(v[e]));
-                }
-                tc::tc_fence_before();
-                __stcg(pml, m_ref);
-                __stcg(pml + 256, l_run);
-                __threadfence();
-                // all 128 rows of the group are in place -> one thread counts the part in -> all learn whether
-                // theirs was the last part of the item
-                tc::mbar_arrive(merge_bar(g));
-                if (!tc::mbar_wait(merge_bar(g), n_mb & 1, abort_flag)) { ok = false; break; }
-                ++n_mb;
-                if (row == 0) merge_flag[g] = atomicAdd(a.done + 2 * pc.item + g, 1);
-                tc::mbar_arrive(merge_bar(g));
-                if (!tc::mbar_wait(merge_bar(g), n_mb & 1, abort_flag)) { ok = false; break; }
-                ++n_mb;
-                if (merge_flag[g] == pc.n_parts - 1) {
-                    // last part in: merge all parts in their fixed order (the result does not depend on which part
-                    // finished last)
-                    __threadfence();
-                    float m_all = -INFINITY;
-                    for (int p = 0; p < pc.n_parts; ++p)
-                        m_all = fmaxf(m_all, __ldcg(a.part_ml + (size_t)part_slot(pc.c_first, p) * 512 + grow));
-                    float l_all = 0.f;
-                    for (int p = 0; p < pc.n_parts; ++p) {
-                        const float *ml = a.part_ml + (size_t)part_slot(pc.c_first, p) * 512 + grow;
-                        const float m_p = __ldcg(ml);
-                        if (m_p != -INFINITY) l_all += __ldcg(ml + 256) * fast_exp2((m_p - m_all) * a.scale_log2);
-                    }
-                    const float inv = 1.f / l_all;
-#pragma unroll 1
-                    for (int c = 0; c < HD; c += 32) {
-                        float o[32];
-#pragma unroll
-                        for (int e = 0; e < 32; ++e) o[e] = 0.f;
-                        for (int p = 0; p < pc.n_parts; ++p) {
-                            const int slot = part_slot(pc.c_first, p);
-                            const float m_p = __ldcg(a.part_ml + (size_t)slot * 512 + grow);
-                            if (m_p == -INFINITY) continue;
-                            const float wgt = fast_exp2((m_p - m_all) * a.scale_log2) * inv;
-                            const float *src = a.part_o + ((size_t)slot * HD + c) * 256 + grow;
-#pragma unroll
-                            for (int e = 0; e < 32; ++e) o[e] = fmaf(__ldcg(src + (size_t)e * 256), wgt, o[e]);
-                        }
-                        store_chunk(c, o);
-                    }
-                }
             }
-            pc = pc_next;
+            w = w_next;
             have = have_next;
         }
     }
@@ -747,8 +657,6 @@ int launch_attend_tc(alora_ctx *ctx, const void *qkv, const BatchArgs &b, const 
     a.max_blocks = b.max_blocks; a.num_pages = b.num_pages; a.Hkv = d.Hkv; a.G = d.G; a.page_size = d.page; a.box_rows = box_rows;
     a.N = d.N; a.Nq = d.Nq; a.qkv = (const __nv_bfloat16 *)qkv; a.scale_log2 = d.softmax_scale * 1.4426950408889634f;
     a.out = (__nv_bfloat16 *)out; a.status = ctx->d_status;
-    a.run_counts = ctx->d_counts + 6; a.cta_start = ctx->d_attn_cta_start; a.done = ctx->d_attn_done;
-    a.part_o = ctx->d_attn_part_o; a.part_ml = ctx->d_attn_part_ml;
     const int max_items = (b.T / ctx->attn_q_block + b.R) * d.Hkv;
     const int grid = std::max(1, std::min(ctx->sm_count, max_items));
     ProfScope prof(ctx, KK_ATTENTION, s);

@@ -166,8 +166,7 @@ __device__ __forceinline__ void metadata_tiles(const int32_t *__restrict__ a_req
 __device__ __forceinline__ void metadata_attn_items(const int32_t *__restrict__ qsl, const int32_t *__restrict__ seq_lens,
                                            int R, int Hkv, int q_block, int small_max, int max_items,
                                            AttnWork *__restrict__ items, int32_t *__restrict__ counts,
-                                           int32_t *blk_off /* [R+1] */, int n_blocks, int32_t *__restrict__ cta_start,
-                                           int32_t *__restrict__ done, int32_t *status) {
+                                           int32_t *blk_off /* [R+1] */, int32_t *status) {
     __shared__ int total;
     for (int r = threadIdx.x; r < R; r += blockDim.x) {
         const int n_new = qsl[r + 1] - qsl[r];
@@ -209,43 +208,6 @@ __device__ __forceinline__ void metadata_attn_items(const int32_t *__restrict__ 
         w.split = 0;
         w.n_splits = 1;
         items[i] = w;
-        done[2 * i] = 0;
-        done[2 * i + 1] = 0;
-    }
-    // The attention kernel cuts the concatenation of all items' 128-key tiles into runs of equal length, one per
-    // block.  items[i].split = tiles before item i; counts[6] = all tiles, counts[7] = run length;
-    // cta_start[c] = the item that holds the first tile of block c's run.
-    __shared__ int warp_sum[32];
-    __shared__ int run_len;
-    __syncthreads();   // this block's writes to items[] are visible to all of its threads
-    const int chunk = (total + (int)blockDim.x - 1) / (int)blockDim.x;
-    const int lo = min(total, (int)threadIdx.x * chunk), hi = min(total, lo + chunk);
-    int sum = 0;
-    for (int i = lo; i < hi; ++i) sum += (items[i].kv_end + kAttnKeysPerTile - 1) / kAttnKeysPerTile;
-    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    int incl = sum;
-    for (int o = 1; o < 32; o <<= 1) {
-        const int v = __shfl_up_sync(0xffffffffu, incl, o);
-        if (lane >= o) incl += v;
-    }
-    if (lane == 31) warp_sum[wid] = incl;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        int acc = 0;
-        for (int w = 0; w < (int)(blockDim.x + 31) / 32; ++w) { const int v = warp_sum[w]; warp_sum[w] = acc; acc += v; }
-        const int len = max((acc + n_blocks - 1) / n_blocks, kAttnMinRunTiles);
-        counts[6] = acc;
-        counts[7] = len;
-        run_len = len;
-    }
-    __syncthreads();
-    int acc = warp_sum[wid] + incl - sum;
-    const int len = run_len;
-    for (int i = lo; i < hi; ++i) {
-        const int n = (items[i].kv_end + kAttnKeysPerTile - 1) / kAttnKeysPerTile;
-        items[i].split = acc;
-        for (int c = (acc + len - 1) / len; c * len < acc + n && c < n_blocks; ++c) cta_start[c] = i;
-        acc += n;
     }
 }
 
@@ -387,8 +349,7 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *a_req, con
                 int Hkv, int q_block, int max_items, AttnWork *__restrict__ items, int32_t *blk_off,
                 int G, int n_sm, int small_max, int max_split_items, int max_split_rows,
                 AttnSplitWork *__restrict__ split_items,
-                int32_t *req_scratch, int32_t *__restrict__ group_done, int rowwise_cap,
-                int32_t *__restrict__ attn_cta_start, int32_t *__restrict__ attn_done, int32_t *status) {
+                int32_t *req_scratch, int32_t *__restrict__ group_done, int rowwise_cap, int32_t *status) {
     // The per-request inputs are read many times (binary searches, list builders): one parallel pass stages them
     // in shared memory, so that the later steps do not each pay a round trip to global memory.
     __shared__ int32_t s_req[4 * kMetaStageR + 1];
@@ -417,8 +378,7 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *a_req, con
                    T, rowwise_cap, shrink_tiles, t_ready, status);
     __syncthreads();  // the next builder reuses the scratch
     if (items != nullptr && block_tables != nullptr)
-        metadata_attn_items(qsl, seq_lens, R, Hkv, q_block, small_max, max_items, items, counts, blk_off,
-                            max(1, min(n_sm, (T / q_block + R) * Hkv)), attn_cta_start, attn_done, status);
+        metadata_attn_items(qsl, seq_lens, R, Hkv, q_block, small_max, max_items, items, counts, blk_off, status);
     __syncthreads();
     if (split_items != nullptr && block_tables != nullptr)
         metadata_split_items(qsl, seq_lens, R, Hkv, G, n_sm, small_max, max_split_items, max_split_rows, split_items, counts,
@@ -440,7 +400,7 @@ int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s) {
         ctx->d.Hkv, ctx->attn_q_block, ctx->max_attn_items, ctx->d_attn_items, ctx->d_attn_off, ctx->d.G,
         ctx->sm_count, ctx->small_max_tokens, ctx->max_split_items, ctx->max_split_rows, ctx->d_split_items,
         ctx->d_req_scratch, ctx->d_group_done, ctx->d_row_delta ? kRowwiseMaxTokens : 0,
-        ctx->d_attn_cta_start, ctx->d_attn_done, ctx->d_status);
+        ctx->d_status);
     return 1;
 }
 
