@@ -17,14 +17,22 @@ int launch_project_simt(alora_ctx *, int, const void *, int, void *, cudaStream_
 int launch_linear_simt(alora_ctx *, const void *, const void *, int, int, int, void *, const void *, cudaStream_t);
 int launch_attend_simt(alora_ctx *, const void *, const BatchArgs &, const void *, void *, cudaStream_t);
 
-int launch_project_tc(alora_ctx *, int, const void *, int, void *, cudaStream_t);
+int launch_project_tc(alora_ctx *, int, const void *, int, void *, cudaStream_t, void *, int);
 int launch_linear_tc(alora_ctx *, const void *, const void *, int, int, int, void *, const void *, cudaStream_t);
 bool build_layer_maps(alora_ctx *ctx, int layer);
 int launch_attend_tc(alora_ctx *, const void *, const BatchArgs &, const void *, void *, cudaStream_t);
 
 // bf16 runs on the tensor cores; the fp32 data type (tiny exact-precision configurations) on CUDA cores.
-int launch_project(alora_ctx *ctx, int layer, const void *hidden, int T, void *qkv, cudaStream_t s) {
-    if (ctx->cfg.dtype == ALORA_DTYPE_BF16) return launch_project_tc(ctx, layer, hidden, T, qkv, s);
+// With a page pool given, the bf16 projection also writes the k / v columns of every row to the row's cache slot
+// (the KV append fused into its epilogue) and sets *kv_appended.
+int launch_project(alora_ctx *ctx, int layer, const void *hidden, int T, void *qkv, cudaStream_t s, void *kv_pool,
+                   int num_pages, bool *kv_appended) {
+    if (kv_appended) *kv_appended = false;
+    if (ctx->cfg.dtype == ALORA_DTYPE_BF16) {
+        const int n = launch_project_tc(ctx, layer, hidden, T, qkv, s, kv_pool, num_pages);
+        if (kv_appended && n >= 0 && kv_pool != nullptr) *kv_appended = true;
+        return n;
+    }
     return launch_project_simt(ctx, layer, hidden, T, qkv, s);
 }
 int launch_linear(alora_ctx *ctx, const void *x, const void *W, int T, int K, int N, void *y,
@@ -62,8 +70,14 @@ static alora_status run_layer(alora_ctx *ctx, int layer, const void *hidden, con
     if (!ctx->layers[layer].wqkv) return ALORA_ERR_NO_WEIGHTS;
     int n = 0, k;
     if ((k = launch_metadata(ctx, b, s)) < 0) return ALORA_ERR_UNSUPPORTED; n += k;
-    if ((k = launch_project(ctx, layer, hidden, b.T, ctx->d_qkv, s)) < 0) return ALORA_ERR_UNSUPPORTED; n += k;
-    if ((k = launch_kv_append(ctx, ctx->d_qkv, b.T, b.num_pages, pool, s)) < 0) return ALORA_ERR_UNSUPPORTED; n += k;
+    bool kv_appended = false;
+    if ((k = launch_project(ctx, layer, hidden, b.T, ctx->d_qkv, s, pool, b.num_pages, &kv_appended)) < 0)
+        return ALORA_ERR_UNSUPPORTED;
+    n += k;
+    if (!kv_appended) {
+        if ((k = launch_kv_append(ctx, ctx->d_qkv, b.T, b.num_pages, pool, s)) < 0) return ALORA_ERR_UNSUPPORTED;
+        n += k;
+    }
     if ((k = launch_attend(ctx, ctx->d_qkv, b, pool, attn_out, s)) < 0) return ALORA_ERR_UNSUPPORTED; n += k;
     return finish(ctx, n);
 }
@@ -367,7 +381,7 @@ alora_status alora_project_qkv(alora_ctx *ctx, int layer, int mode, const void *
     const int32_t *d_block_tables = nullptr; const int max_blocks = 0, num_pages = 0;
     ALORA_BATCH(mode);
     int n = launch_metadata(ctx, b, s), k;
-    if ((k = launch_project(ctx, layer, d_hidden, T, d_qkv, s)) < 0) return ALORA_ERR_UNSUPPORTED;
+    if ((k = launch_project(ctx, layer, d_hidden, T, d_qkv, s, nullptr, 0, nullptr)) < 0) return ALORA_ERR_UNSUPPORTED;
     return finish(ctx, n + k);
 }
 

@@ -182,7 +182,8 @@ int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s);
 int launch_repack_adapter(alora_ctx *ctx, int rank, const void *Aq, const void *Bq, const void *Ak,
                           const void *Bk, const void *Av, const void *Bv, void *A_dst, void *B_dst,
                           cudaStream_t s);
-int launch_project(alora_ctx *ctx, int layer, const void *hidden, int T, void *qkv, cudaStream_t s);
+int launch_project(alora_ctx *ctx, int layer, const void *hidden, int T, void *qkv, cudaStream_t s, void *kv_pool,
+                   int num_pages, bool *kv_appended);
 int launch_kv_append(alora_ctx *ctx, const void *qkv, int T, int num_pages, void *pool, cudaStream_t s);
 int launch_attend(alora_ctx *ctx, const void *qkv, const BatchArgs &b, const void *pool, void *out,
                   cudaStream_t s);

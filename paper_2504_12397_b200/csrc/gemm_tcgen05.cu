@@ -59,6 +59,11 @@ struct GemmArgs {
     const int32_t *rowwise_flag;
     const float *row_delta;
     const int32_t *row_adapter;
+    // KV append fused into the epilogue (nullptr: off): columns Nq .. N of row t also go to the paged cache,
+    // pool[page][plane][head][row in page][:] with page * page_size + row = slot_map[t] (-1: token rejected, skipped)
+    __nv_bfloat16 *kv_pool;
+    const int32_t *slot_map;
+    int kv_hd_shift, kv_heads, kv_page_size, kv_num_pages;
     int32_t *status;
 };
 
@@ -303,6 +308,16 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             // row-wise delta: only rows with an applied adapter add anything (a gated-off row never sees "+ 0")
             const float *drow = (dense && row_ok && a.row_adapter[t.row_start + r] >= 0)
                                     ? a.row_delta + (size_t)(t.row_start + r) * a.N + n0 : nullptr;
+            // fused KV append: where this row's k / v columns go in the page pool
+            int kv_page = -1, kv_row = 0;
+            if (a.kv_pool != nullptr && row_ok && n0 + BN > a.Nq) {
+                const int slot = a.slot_map[t.row_start + r];
+                if (slot >= 0) {
+                    kv_page = slot / a.kv_page_size;
+                    kv_row = slot % a.kv_page_size;
+                    if (kv_page >= a.kv_num_pages) { report(a.status, ALORA_ERR_PAGE_RANGE); kv_page = -1; }
+                }
+            }
 #pragma unroll 1
             for (int c = 0; c < BN; c += 32) {
                 uint32_t v[32];
@@ -335,6 +350,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         o.x = tc::pack_bf16(f[0], f[1]); o.y = tc::pack_bf16(f[2], f[3]);
                         o.z = tc::pack_bf16(f[4], f[5]); o.w = tc::pack_bf16(f[6], f[7]);
                         *reinterpret_cast<uint4 *>(orow + c + 8 * j) = o;
+                        const int kc = n0 + c + 8 * j - a.Nq;   // column inside [k | v]
+                        if (kv_page >= 0 && kc >= 0) {
+                            const int plane = kc >= a.Nkv ? 1 : 0, c2 = kc - plane * a.Nkv;
+                            const int head = c2 >> a.kv_hd_shift, dd = c2 & ((1 << a.kv_hd_shift) - 1);
+                            __nv_bfloat16 *dst = a.kv_pool +
+                                ((((size_t)kv_page * 2 + plane) * a.kv_heads + head) * a.kv_page_size + kv_row << a.kv_hd_shift) + dd;
+                            *reinterpret_cast<uint4 *>(dst) = o;
+                        }
                     }
                 }
             }
@@ -423,7 +446,8 @@ static int pick_bn(int N, int Nq, int Nkv, bool lora, int T) {
 
 // q/k/v projection of one layer on the tensor cores: shrink (t = s A x on adapter tiles), then the
 // base GEMM with the expand step fused.  Returns kernels launched, or -1 when the shape is unsupported.
-int launch_project_tc(alora_ctx *ctx, int layer, const void *hidden, int T, void *qkv, cudaStream_t s) {
+int launch_project_tc(alora_ctx *ctx, int layer, const void *hidden, int T, void *qkv, cudaStream_t s, void *kv_pool,
+                      int num_pages) {
     if (T == 0) return 0;
     const Dims &d = ctx->d;
     const bool have_adapters = ctx->layer_has_adapter[layer];
@@ -459,6 +483,12 @@ int launch_project_tc(alora_ctx *ctx, int layer, const void *hidden, int T, void
         g.Nq = d.Nq; g.Nkv = d.Nkv; g.total_adapter_rows = d.N; g.status = ctx->d_status;
         if (may_rowwise) {
             g.rowwise_flag = ctx->d_counts + 5; g.row_delta = ctx->d_row_delta; g.row_adapter = ctx->d_row_adapter;
+        }
+        if (kv_pool != nullptr) {
+            int shift = 0;
+            while ((1 << shift) < d.hd) ++shift;
+            g.kv_pool = (__nv_bfloat16 *)kv_pool; g.slot_map = ctx->d_slot; g.kv_hd_shift = shift; g.kv_heads = d.Hkv;
+            g.kv_page_size = d.page; g.kv_num_pages = num_pages;
         }
         if (fuse_shrink) {
             g.shrink_tiles = ctx->d_shrink_tiles; g.n_shrink_tiles = ctx->d_counts + 2;
