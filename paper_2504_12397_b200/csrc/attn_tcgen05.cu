@@ -129,11 +129,6 @@ __device__ __forceinline__ void tma_load_3d(uint32_t smem_dst, const CUtensorMap
 __device__ __forceinline__ uint32_t pack_bf16_int(float lo, float hi) {
     return __byte_perm(__float_as_uint(lo) + 0x8000u, __float_as_uint(hi) + 0x8000u, 0x7632);
 }
-__device__ __forceinline__ bool elect_one() {
-    uint32_t pred;
-    asm volatile("{\n\t.reg .pred p;\n\telect.sync _|p, 0xffffffff;\n\tselp.u32 %0, 1, 0, p;\n\t}" : "=r"(pred));
-    return pred != 0;
-}
 __device__ __forceinline__ uint32_t pack_cvt(float lo, float hi) {
     uint32_t r; asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo)); return r;
 }
@@ -317,7 +312,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         // control flow keeps the descriptors in uniform registers); one elected lane issues the tensor-core
         // instructions and their commits.
         const int g = warp - 9;
-        const bool leader = elect_one();
+        const bool leader = tc::elect_one();
         constexpr uint32_t idesc_s = tc::idesc_bf16_f32(128, kHalfKeys);
         constexpr uint32_t idesc_pv = idesc_bf16_f32_bmn(128, HD);
         uint32_t n_item = 0, kt = 0, nh = 0;   // nh: half tiles handled so far (phase counter of the group's barriers)

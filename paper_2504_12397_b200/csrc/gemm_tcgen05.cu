@@ -219,8 +219,15 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             }
         }
     } else if (warp == 1) {
-        if (lane == 0) {
+        {
             // ------------------------------ MMA issuer ------------------------------
+            // The whole warp walks the schedule (uniform control flow keeps descriptors and loop state in uniform
+            // registers, which is what lets the issue rate reach the tensor pipe's); one elected lane issues the
+            // tensor-core instructions and their commits.
+            const bool leader = tc::elect_one();
+            auto wait_all = [&](uint32_t bar, uint32_t parity) {
+                return __all_sync(0xffffffffu, tc::mbar_wait(bar, parity, abort_flag));
+            };
             constexpr uint32_t idesc_main = tc::idesc_bf16_f32(kBM, BN);
             constexpr uint32_t idesc_shrink = tc::idesc_bf16_f32(kBM, BN >= kShrinkCols ? kShrinkCols : BN);
             uint32_t kc = 0, it = 0;
@@ -232,25 +239,31 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                 const int extra_steps = extra ? a.adapters[t.adapter].rpad / 16 : 0;
                 const uint32_t idesc = g.shrink ? idesc_shrink : idesc_main;
                 const uint32_t acc = it & 1;
-                if (!tc::mbar_wait(acce_bar(acc), ((it >> 1) & 1) ^ 1, abort_flag)) { ok = false; break; }
+                if (!wait_all(acce_bar(acc), ((it >> 1) & 1) ^ 1)) { ok = false; break; }
                 tc::tc_fence_after();
                 const uint32_t d_tmem = tmem_base + acc * BN;
                 for (int kb = 0; kb < kb_main + extra; ++kb, ++kc) {
                     const int s = kc % kStages;
-                    if (!tc::mbar_wait(full_bar(s), (kc / kStages) & 1, abort_flag)) { ok = false; break; }
+                    if (!wait_all(full_bar(s), (kc / kStages) & 1)) { ok = false; break; }
                     tc::tc_fence_after();
                     const uint32_t sa = smem_base + s * S::kStageBytes, sb = sa + S::kABytes;
                     const uint64_t da = tc::smem_desc_k_sw128(sa), db = tc::smem_desc_k_sw128(sb);
-                    const int steps = kb < kb_main ? kBK / 16 : extra_steps;
-                    for (int k = 0; k < steps; ++k)
-                        tc::mma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
-                    tc::mma_commit(empty_bar(s));  // slot reusable once these MMAs have read it
+                    if (leader) {
+                        if (kb < kb_main) {
+#pragma unroll
+                            for (int k = 0; k < kBK / 16; ++k)
+                                tc::mma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, (kb | k) != 0 ? 1u : 0u);
+                        } else {
+                            for (int k = 0; k < extra_steps; ++k) tc::mma_bf16(d_tmem, da + 2 * k, db + 2 * k, idesc, 1u);
+                        }
+                        tc::mma_commit(empty_bar(s));  // slot reusable once these MMAs have read it
+                    }
                 }
                 if (!ok) break;
-                tc::mma_commit(accf_bar(acc));      // accumulator complete
+                if (leader) tc::mma_commit(accf_bar(acc));      // accumulator complete
                 ++it;
             }
-            if (!ok) {
+            if (!ok && leader) {
                 tc::mma_commit(drain_bar);          // wait (bounded) for tensor-core work still in flight
                 const long long t0 = clock64();
                 while (!tc::mbar_try_wait(drain_bar, 0) && clock64() - t0 < tc::kWaitCycleLimit) {}
