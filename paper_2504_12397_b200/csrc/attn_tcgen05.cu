@@ -1,20 +1,26 @@
 // Paged causal GQA attention of suffix queries on the 5th-generation tensor cores (Eq. 1 / Eq. 3).
 //
 // One persistent block per SM works through (request, KV head, query block) items.  A query block
-// is 2 x 128 score rows: rows are (token, query head of the KV group) pairs, so the G query heads
-// that share a KV head share every K/V tile brought on chip.  Roles:
-//   warp 8   TMA producer: the two 128 x hd query tiles of the item (3-D boxes d x head x token out
-//            of the fused q/k/v rows) and, per 128-key tile, the K and V rows of up to 128/page
-//            pages fetched through the block table (one 2-D box per page and 64-wide half of hd),
-//            two-deep rings for K and for V;
-//   warp 9   MMA issuer: S_w = Q_w K^T (fp32, tensor memory) for w = 0, 1, then PV_w = P_w V with P_w
-//            read from tensor memory (it overwrites S_w in bf16) and V consumed in place (MN-major);
-//   warps 0-3, 4-7   softmax groups w = 0, 1, one thread per score row: running maximum and sum
-//            (online softmax; a thread owns its whole row, so the row reductions need no
-//            cross-lane traffic), P_w written back to tensor memory; the output O_w accumulates in
-//            tensor memory across tiles and is rescaled only when a row's maximum has moved by more
-//            than 2^8 since the exponent reference was last set; final normalisation and store.
-// While one group does its exponentials the tensor pipe works for the other group.
+// is 2 x 128 score rows ("groups"): rows are (token, query head of the KV group) pairs, so the G
+// query heads that share a KV head share every K/V tile brought on chip.  Keys come in tiles of 128
+// and are consumed as two half tiles of 64.  Roles:
+//   warp 8      TMA producer: the head-dim columns 64.. of the two 128-row query tiles (3-D boxes
+//               d x head x token out of the fused q/k/v rows) and, per key tile, the K and V rows
+//               fetched through the block table (one 3-D box per 8 / 16 / 64 cache rows, both 64-wide
+//               halves of the head dim), three-deep rings for K and for V;
+//   warps 9, 10 MMA issuers of group 0 and 1 (the whole warp walks the schedule, an elected lane
+//               issues): S_g = Q_g K^T of a half tile (fp32, tensor memory; head-dim columns 0..63 of
+//               Q_g are the A operand from tensor memory, the rest from shared memory), issued as soon
+//               as the group has taken the previous scores into registers, and P_g V with P_g read
+//               from tensor memory and V consumed in place (MN-major);
+//   warps 0-3, 4-7   softmax groups g = 0, 1, one thread per score row: they put their Q row's first
+//               64 columns into tensor memory, keep a running exponent reference and sum (online
+//               softmax; a thread owns its whole row, so the row reductions need no cross-lane
+//               traffic), write P_g (bf16 pairs) to tensor memory; the output O_g accumulates in
+//               tensor memory across tiles and is rescaled only when a row's maximum has moved by
+//               more than 2^8 since the reference was last set; final normalisation and store.
+// While one group does its exponentials the tensor pipe works for the other group and on the group's
+// own next scores.
 //
 // Masking: key j is visible to a row at position p iff j <= p; masked probabilities are set to
 // zero explicitly, and V rows of keys at or beyond the item's causal limit are cleared in shared
@@ -123,12 +129,6 @@ __device__ __forceinline__ void tma_load_3d(uint32_t smem_dst, const CUtensorMap
         : "memory");
 }
 
-// Two non-negative fp32 values -> packed bf16 pair, rounded to nearest (ties up), with integer instructions only:
-// the float-to-bf16 conversion instruction shares the special-function unit with the exponentials, which is
-// the busiest unit of the softmax.
-__device__ __forceinline__ uint32_t pack_bf16_int(float lo, float hi) {
-    return __byte_perm(__float_as_uint(lo) + 0x8000u, __float_as_uint(hi) + 0x8000u, 0x7632);
-}
 __device__ __forceinline__ uint32_t pack_cvt(float lo, float hi) {
     uint32_t r; asm("cvt.rn.bf16x2.f32 %0, %1, %2;" : "=r"(r) : "f"(hi), "f"(lo)); return r;
 }
