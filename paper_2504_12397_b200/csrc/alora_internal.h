@@ -152,6 +152,20 @@ alora_status cuda_fail(alora_ctx *ctx, cudaError_t e, const char *what);
     } while (0)
 
 // Brackets the launches of one kernel family with CUDA events while profiling is on.
+// Kernel launch with the programmatic-stream-serialization attribute (`dependent`: the kernel calls
+// tc::grid_dep_wait() before it touches anything its predecessor in the stream wrote or still reads).
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_kernel(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                 bool dependent, Args &&...args) {
+    cudaLaunchConfig_t cfg{};
+    cfg.gridDim = grid; cfg.blockDim = block; cfg.dynamicSmemBytes = smem; cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = dependent ? 1 : 0;
+    cfg.attrs = attr; cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, std::forward<Args>(args)...);
+}
+
 struct ProfScope {
     alora_ctx *ctx;
     cudaStream_t s;

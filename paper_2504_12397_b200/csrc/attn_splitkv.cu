@@ -181,6 +181,8 @@ attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmKV, const SplitArgs a)
         tc::fence_proxy_async();
     }
     __syncthreads();
+    tc::grid_dep_launch();
+    tc::grid_dep_wait();   // work list, q/k/v rows and the cache rows of the new tokens come from earlier kernels
     const int n_items = *a.n_items;
 
     if (warp == kSkConsumerWarps) {
@@ -547,8 +549,9 @@ int launch_attend_splitkv(alora_ctx *ctx, const void *qkv, const BatchArgs &b, c
     const int grid = std::max(1, std::min(ctx->sm_count, ctx->max_split_items));
     {
         ProfScope prof(ctx, KK_ATTENTION, s);
-        if (hi) attn_splitkv_kernel<128><<<grid, kSkThreads, SkSmem<128>::kTotal, s>>>(tmKV, a);
-        else attn_splitkv_kernel<64><<<grid, kSkThreads, SkSmem<64>::kTotal, s>>>(tmKV, a);
+        const cudaError_t e = hi ? launch_kernel(attn_splitkv_kernel<128>, dim3(grid), dim3(kSkThreads), SkSmem<128>::kTotal, s, true, tmKV, a)
+                                 : launch_kernel(attn_splitkv_kernel<64>, dim3(grid), dim3(kSkThreads), SkSmem<64>::kTotal, s, true, tmKV, a);
+        if (e != cudaSuccess) return -1;
     }
     return 1;
 }

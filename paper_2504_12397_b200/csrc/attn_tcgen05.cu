@@ -231,6 +231,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    tc::grid_dep_launch();
+    tc::grid_dep_wait();   // work list, q/k/v rows and the cache rows of the new tokens come from earlier kernels
     // tensor-memory columns of group g (base g*256): S_g 0..63, P_g 64..95, the first 64 head-dim columns of Q_g as
     // bf16 pairs 96..127, O_g 128..255
     const int n_items = *a.n_items;
@@ -665,8 +667,9 @@ int launch_attend_tc(alora_ctx *ctx, const void *qkv, const BatchArgs &b, const 
         if (e != cudaSuccess) return -1;
         attr_set[hi][dev] = true;
     }
-    if (hi) attn_tcgen05_kernel<128><<<grid, kAttnThreads, AttnSmem<128>::kTotal, s>>>(tmQ, tmKV, a);
-    else attn_tcgen05_kernel<64><<<grid, kAttnThreads, AttnSmem<64>::kTotal, s>>>(tmQ, tmKV, a);
+    const cudaError_t le = hi ? launch_kernel(attn_tcgen05_kernel<128>, dim3(grid), dim3(kAttnThreads), AttnSmem<128>::kTotal, s, true, tmQ, tmKV, a)
+                              : launch_kernel(attn_tcgen05_kernel<64>, dim3(grid), dim3(kAttnThreads), AttnSmem<64>::kTotal, s, true, tmQ, tmKV, a);
+    if (le != cudaSuccess) return -1;
     return 1 + n_small;
 }
 

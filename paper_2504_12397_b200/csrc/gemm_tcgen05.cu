@@ -159,6 +159,8 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     __syncthreads();
     tc::tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
+    tc::grid_dep_launch();
+    tc::grid_dep_wait();   // the metadata step's lists, the activations: all written by earlier kernels of the stream
 
     const bool dense = a.rowwise_flag != nullptr && *a.rowwise_flag != 0;
     const int n_m = (a.tiles && !dense) ? *a.n_row_tiles : (a.M + kBM - 1) / kBM;
@@ -437,7 +439,9 @@ static bool launch_gemm_bn(alora_ctx *ctx, const CUtensorMap &tmA, const CUtenso
         attr_set[dev] = true;
     }
     const int grid = std::max(1, std::min(ctx->sm_count, max_items));
-    gemm_tcgen05_kernel<BN><<<grid, kGemmThreads, GemmSmem<BN>::kTotal, s>>>(tmA, tmB, tmT, tmL, tmS, args);
+    if (launch_kernel(gemm_tcgen05_kernel<BN>, dim3(grid), dim3(kGemmThreads), GemmSmem<BN>::kTotal, s, true, tmA, tmB, tmT, tmL,
+                      tmS, args) != cudaSuccess)
+        return false;
     return true;
 }
 

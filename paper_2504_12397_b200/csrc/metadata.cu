@@ -1,6 +1,7 @@
 // Batch metadata: per-token request / applied-adapter / KV-slot arrays and the projection's
 // row-tile list.  Integer work only; every output is compared exactly against the CPU oracle.
 #include "alora_internal.h"
+#include "tc_common.cuh"
 
 namespace alora {
 
@@ -353,6 +354,7 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *a_req, con
     // The per-request inputs are read many times (binary searches, list builders): one parallel pass stages them
     // in shared memory, so that the later steps do not each pay a round trip to global memory.
     __shared__ int32_t s_req[4 * kMetaStageR + 1];
+    tc::grid_dep_launch();   // the next kernel's blocks may start their set-up; they wait for this kernel's results
     if (R <= kMetaStageR) {
         int32_t *s_qsl = s_req, *s_len = s_req + R + 1, *s_ids = s_len + R, *s_areq = s_ids + R;
         for (int i = threadIdx.x; i <= R; i += blockDim.x) s_qsl[i] = qsl[i];

@@ -2,6 +2,7 @@
 // configurations), and the element-wise / copy steps shared by both data types (adapter repack,
 // KV append, RMSNorm, SwiGLU).
 #include "alora_internal.h"
+#include "tc_common.cuh"
 
 namespace alora {
 
@@ -100,6 +101,8 @@ lora_delta_rows_kernel(const __nv_bfloat16 *__restrict__ x, const int32_t *__res
                        int Nq, int Nkv, int N, float *__restrict__ delta) {
     extern __shared__ uint4 x_s4[];  // H bf16
     __shared__ float t_s[kRankPadMax];
+    tc::grid_dep_launch();
+    tc::grid_dep_wait();   // the flag and the row -> adapter map come from the metadata kernel
     if (*rowwise_flag == 0) return;
     const int row = blockIdx.x, blk = blockIdx.y;
     const int k = row_adapter[row];
@@ -175,7 +178,7 @@ lora_delta_rows_kernel(const __nv_bfloat16 *__restrict__ x, const int32_t *__res
 int launch_lora_delta_rows(alora_ctx *ctx, int layer, const void *hidden, int T, cudaStream_t s) {
     const Dims &d = ctx->d;
     const AdapterDev *ads = ctx->d_adapters + (size_t)layer * ctx->cfg.max_adapters;
-    lora_delta_rows_kernel<<<dim3(T, 3), kDeltaThreads, (size_t)d.H * 2, s>>>((const __nv_bfloat16 *)hidden, ctx->d_row_adapter, ads,
+    launch_kernel(lora_delta_rows_kernel, dim3(T, 3), dim3(kDeltaThreads), (size_t)d.H * 2, s, true, (const __nv_bfloat16 *)hidden, (const int32_t *)ctx->d_row_adapter, ads,
                                                                    ctx->d_counts + 5, d.H, d.Nq, d.Nkv, d.N,
                                                                    ctx->d_row_delta);
     return 1;

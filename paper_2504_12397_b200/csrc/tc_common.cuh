@@ -32,6 +32,14 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// Programmatic dependent launch.  A kernel launched with the programmatic-stream-serialization attribute may start
+// while its predecessor in the stream is still running: grid_dep_wait() returns once the predecessor has completed
+// and its writes are visible (it returns at once in a kernel launched the ordinary way), so everything before it
+// may only touch this block's own shared and tensor memory.  Every block executes it before it exits.
+// grid_dep_launch() lets the successor's blocks start as soon as all blocks of this kernel have called it.
+__device__ __forceinline__ void grid_dep_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void grid_dep_launch() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
 // One lane of a converged warp (the same one every time); all 32 lanes must call it.
 __device__ __forceinline__ bool elect_one() {
     uint32_t pred;
