@@ -446,9 +446,28 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 tc::tc_fence_before();
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(s_free(g));
-                float m_tile = -INFINITY;
                 const bool masked = tbase + kKeysPerTile - 1 > pos;   // tile crosses this row's causal limit
+                bool bump = false;     // the exponent reference moved: O_g and the row sum are rescaled by alpha
+                float alpha = 1.f;
+                float l0 = 0.f, l1 = 0.f;
+                uint32_t pk[kHalfKeys / 2];   // probabilities (bf16 pairs); their row sum in fp32
+                auto row_max = [&]() {
+                    float m0 = -INFINITY, m1 = -INFINITY;
+#pragma unroll
+                    for (int e = 0; e < kHalfKeys; e += 4) {
+                        m0 = max3(m0, __uint_as_float(sv[e]), __uint_as_float(sv[e + 1]));
+                        m1 = max3(m1, __uint_as_float(sv[e + 2]), __uint_as_float(sv[e + 3]));
+                    }
+                    return fmaxf(m0, m1);
+                };
+                auto move_reference = [&](float m_tile) {
+                    alpha = fast_exp2((m_ref - m_tile) * a.scale_log2);
+                    m_ref = m_tile;
+                    l_run *= alpha;
+                    bump = true;
+                };
                 if (masked) {
+                    float m_tile = -INFINITY;
                     const int k0 = tbase + (perm ? hh * 8 : hh * kHalfKeys);
 #pragma unroll
                     for (int e = 0; e < kHalfKeys; ++e) {
@@ -456,27 +475,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         if (key > pos) sv[e] = 0xff800000u;  // -inf
                         m_tile = fmaxf(m_tile, __uint_as_float(sv[e]));
                     }
-                } else {
-                    float m0 = -INFINITY, m1 = -INFINITY;
-#pragma unroll
-                    for (int e = 0; e < kHalfKeys; e += 4) {
-                        m0 = max3(m0, __uint_as_float(sv[e]), __uint_as_float(sv[e + 1]));
-                        m1 = max3(m1, __uint_as_float(sv[e + 2]), __uint_as_float(sv[e + 3]));
-                    }
-                    m_tile = fmaxf(m0, m1);
-                }
-                const bool bump = (m_tile - m_ref) * a.scale_log2 > 8.f;  // always true on an item's first half tile
-                float alpha = 1.f;
-                if (bump) {
-                    alpha = fast_exp2((m_ref - m_tile) * a.scale_log2);
-                    m_ref = m_tile;
-                    l_run *= alpha;
-                }
-                // probabilities (bf16 pairs) and their row sum in fp32
-                const float mb = m_ref * a.scale_log2;
-                float l0 = 0.f, l1 = 0.f;
-                uint32_t pk[kHalfKeys / 2];
-                if (masked) {
+                    if ((m_tile - m_ref) * a.scale_log2 > 8.f) move_reference(m_tile);
+                    const float mb = m_ref * a.scale_log2;
 #pragma unroll
                     for (int e = 0; e < kHalfKeys; e += 2) {
                         const float p0 = fast_exp2(fmaf(__uint_as_float(sv[e]), a.scale_log2, -mb));
@@ -486,14 +486,28 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         pk[e >> 1] = pack_cvt(p0, p1);
                     }
                 } else {
+                    // No pass over the scores for their maximum: the exponentials are taken against the current
+                    // reference, and only if their sum says that one of them may have left the safe range
+                    // (> 2^14; also catches inf / NaN) is the true maximum taken and the half tile redone.  The
+                    // first half tile of an item has no reference yet and takes its maximum first.
+                    auto exponentials = [&]() {
+                        const float mb = m_ref * a.scale_log2;
+                        l0 = 0.f; l1 = 0.f;
 #pragma unroll
-                    for (int e = 0; e < kHalfKeys; e += 2) {
-                        float x0, x1, p0, p1;
-                        fma2(x0, x1, __uint_as_float(sv[e]), __uint_as_float(sv[e + 1]), a.scale_log2, -mb);
-                        if ((e & 7) == 6) { p0 = exp2_poly(x0); p1 = exp2_poly(x1); }   // a quarter of them on the FMA pipe
-                        else { p0 = fast_exp2(x0); p1 = fast_exp2(x1); }
-                        add2(l0, l1, p0, p1);
-                        pk[e >> 1] = pack_cvt(p0, p1);
+                        for (int e = 0; e < kHalfKeys; e += 2) {
+                            float x0, x1, p0, p1;
+                            fma2(x0, x1, __uint_as_float(sv[e]), __uint_as_float(sv[e + 1]), a.scale_log2, -mb);
+                            if ((e & 7) == 6) { p0 = exp2_poly(x0); p1 = exp2_poly(x1); }   // a quarter of them on the FMA pipe
+                            else { p0 = fast_exp2(x0); p1 = fast_exp2(x1); }
+                            add2(l0, l1, p0, p1);
+                            pk[e >> 1] = pack_cvt(p0, p1);
+                        }
+                    };
+                    if (m_ref == -INFINITY) move_reference(row_max());
+                    exponentials();
+                    if (!(l0 + l1 <= 16384.f)) {
+                        move_reference(row_max());
+                        exponentials();
                     }
                 }
                 l_run += l0 + l1;
