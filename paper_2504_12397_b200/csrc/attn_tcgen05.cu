@@ -496,7 +496,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #pragma unroll
                         for (int e = 0; e < kHalfKeys; e += 2) {
                             float x0, x1, p0, p1;
-                            fma2(x0, x1, __uint_as_float(sv[e]), __uint_as_float(sv[e + 1]), a.scale_log2, -mb);
+                            x0 = fmaf(__uint_as_float(sv[e]), a.scale_log2, -mb);
+                            x1 = fmaf(__uint_as_float(sv[e + 1]), a.scale_log2, -mb);
                             if ((e & 7) == 6) { p0 = exp2_poly(x0); p1 = exp2_poly(x1); }   // a quarter of them on the FMA pipe
                             else { p0 = fast_exp2(x0); p1 = fast_exp2(x1); }
                             add2(l0, l1, p0, p1);
