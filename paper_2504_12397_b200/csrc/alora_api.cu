@@ -175,6 +175,9 @@ alora_status alora_create(const alora_config *cfg, alora_ctx **out) {
         ctx->max_attn_items = (int)((Tm / ctx->attn_q_block + (size_t)c.max_requests) * d.Hkv);
         alloc((void **)&ctx->d_attn_items, (size_t)ctx->max_attn_items * sizeof(AttnWork));
         alloc((void **)&ctx->d_attn_off, ((size_t)c.max_requests + 1) * 4);
+        alloc((void **)&ctx->d_attn_cta_start, (size_t)ctx->sm_count * 4);
+        alloc((void **)&ctx->d_attn_part_o, (size_t)2 * ctx->sm_count * d.hd * 256 * 4);
+        alloc((void **)&ctx->d_attn_part_ml, (size_t)2 * ctx->sm_count * 2 * 256 * 4);
         if (16 % d.G == 0 && (d.hd == 64 || d.hd == 128)) {
             // few-row attention: at most kSplitItemsPerSm * n_sm key ranges plus one per (request, KV head, row
             // block); a range of mt row tiles owns 16 * mt rows of the partial-result arrays
@@ -239,7 +242,8 @@ alora_status alora_destroy(alora_ctx *ctx) {
     void *ptrs[] = {ctx->d_adapters, ctx->d_token_req, ctx->d_row_adapter, ctx->d_slot, ctx->d_tiles, ctx->d_counts,
                     ctx->d_seg_scratch, ctx->d_shrink_tiles, ctx->d_t_ready, ctx->d_t, ctx->d_qkv, ctx->d_status, ctx->d_act[0], ctx->d_act[1],
                     ctx->d_act[2], ctx->d_act[3], ctx->d_iota, ctx->d_attn_items, ctx->d_attn_off, ctx->d_split_items,
-                    ctx->d_req_scratch, ctx->d_part_o, ctx->d_part_ml, ctx->d_group_done, ctx->d_row_delta};
+                    ctx->d_req_scratch, ctx->d_part_o, ctx->d_part_ml, ctx->d_group_done, ctx->d_row_delta,
+                    ctx->d_attn_cta_start, ctx->d_attn_part_o, ctx->d_attn_part_ml};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (ctx->h_status) cudaFreeHost(ctx->h_status);
     for (ProfEvent &e : ctx->prof_events) { if (e.begin) cudaEventDestroy(e.begin); if (e.end) cudaEventDestroy(e.end); }

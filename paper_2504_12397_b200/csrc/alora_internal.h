@@ -53,9 +53,12 @@ struct AttnWork {
     int32_t kv_head;
     int32_t kv_start;
     int32_t kv_end;
-    int32_t split;     // index of this key range among the splits of the same queries
+    int32_t split;     // 128-key tiles of all earlier items of the work list
     int32_t n_splits;
 };
+constexpr int kAttnKeysPerTile = 128;   // keys per K/V tile of the tensor-core attention kernel
+constexpr int kAttnMinRunTiles = 8;     // shortest run of key tiles given to one block
+constexpr int kAttnCutMinTiles = 128;   // items are cut into runs only when a block has at least this many tiles to do
 
 // One unit of few-row (decode / short suffix) attention work: score rows of `q_count` tokens starting at
 // flat token q_start (rows are (token, query head of the group) pairs, `mt` tiles of 16 rows), one KV
@@ -110,7 +113,9 @@ struct alora_ctx {
     alora::ProjTile *d_tiles = nullptr;
     int32_t *d_counts = nullptr;  // [0] projection row tiles, [1] attention work items, [2] row tiles with an adapter,
                                   // [3] few-row attention items, [4] next unclaimed few-row item,
-                                  // [5] 1 = the projection takes the row-wise route for this batch
+                                  // [5] 1 = the projection takes the row-wise route for this batch,
+                                  // [6] key tiles of the attention items that are cut into runs, [7] tiles per run,
+                                  // [8] attention items taken whole (the first ones), [9] key tiles of those
     int32_t *d_seg_scratch = nullptr;  // [14*max_requests+5] per-request values and merged row runs of the current batch
     int32_t *d_shrink_tiles = nullptr; // [max_tiles] indices of the row tiles with an adapter
     int32_t *d_t_ready = nullptr;      // [max_tiles] per row tile: epilogue warps that have published t
@@ -119,6 +124,10 @@ struct alora_ctx {
     alora::AttnWork *d_attn_items = nullptr;  // tensor-core attention work list (bf16)
     int32_t *d_attn_off = nullptr;            // [max_requests+1] block offsets per request
     int32_t max_attn_items = 0, attn_q_block = 0;
+    // long batches: the tensor-core attention kernel takes some items whole and cuts the key tiles of the rest into runs
+    int32_t *d_attn_cta_start = nullptr;      // [n_sm] first item of each block's run
+    float *d_attn_part_o = nullptr;           // [2 * n_sm][hd][256] unnormalised outputs of the parts of cut items
+    float *d_attn_part_ml = nullptr;          // [2 * n_sm][2][256] their exponent references and row sums
     // few-row attention (requests with at most small_max_tokens new tokens): split-KV work list and partials
     alora::AttnSplitWork *d_split_items = nullptr;
     int32_t *d_req_scratch = nullptr;   // [3][max_requests] items per request, item offset, partial-row offset

@@ -26,6 +26,7 @@
 // zero explicitly, and V rows of keys at or beyond the item's causal limit are cleared in shared
 // memory before use, so stale cache bytes (whatever their bit pattern) cannot reach an output.
 // All waits are bounded; on expiry ALORA_ERR_TIMEOUT is recorded and the block leaves normally.
+#include <type_traits>
 #include "alora_internal.h"
 #include "tc_common.cuh"
 
@@ -48,19 +49,78 @@ struct AttnArgs {
     const __nv_bfloat16 *qkv;  // [T][N], query part first
     __nv_bfloat16 *out;        // [T][Nq]
     int32_t *status;
+    // work split: items below n_whole are taken whole; the key tiles of the others are concatenated and cut into runs
+    const int32_t *run_counts;  // [0] key tiles in the concatenation, [1] tiles per run, [2] n_whole, [3] tiles of the whole items
+    const int32_t *cta_start;   // [blocks] item that holds the first tile of the block's run
+    float *part_o;              // [2 * blocks][hd][256] unnormalised output of a part, column-major over the 256 rows
+    float *part_ml;             // [2 * blocks][2][256] exponent reference and row sum of a part
 };
 
-// The items a block works through: blockIdx, blockIdx + blocks, ...
-struct ItemIter {
-    int it;
-    __device__ ItemIter() : it((int)blockIdx.x) {}
-    __device__ bool next(const AttnArgs &a, int n_items, AttnWork &w) {
-        if (it >= n_items) return false;
-        w = a.items[it];
-        it += (int)gridDim.x;
+// A block's work: whole items blockIdx, blockIdx + blocks, ... below n_whole, then the pieces of its run (tiles
+// [blockIdx * len, +len) of the concatenated key tiles of the items from n_whole on).  One piece = tiles [t0, t1)
+// of one item.  An item cut by run boundaries is worked on by n_parts consecutive blocks (this block holds part
+// `part`, the first of them is block c_first); each writes its partial result to a slot and a merge kernel adds
+// the parts up afterwards.
+struct RunPiece {
+    AttnWork w;
+    int item, t0, t1, n_parts, part, c_first;
+};
+struct RunIter {
+    int gt, gt_end, it, len, off, n_whole, whole;
+    __device__ explicit RunIter(const AttnArgs &a) {
+        const int total = a.run_counts[0];
+        len = a.run_counts[1];
+        n_whole = a.run_counts[2];
+        off = a.run_counts[3];
+        whole = (int)blockIdx.x;
+        gt = min(total, (int)blockIdx.x * len);
+        gt_end = min(total, gt + len);
+        it = gt < gt_end ? a.cta_start[blockIdx.x] : 0;
+    }
+    __device__ bool next(const AttnArgs &a, RunPiece &p) {
+        if (whole < n_whole) {
+            p.item = whole;
+            whole += (int)gridDim.x;
+            p.w = a.items[p.item];
+            p.t0 = 0;
+            p.t1 = (p.w.kv_end + kKeysPerTile - 1) / kKeysPerTile;
+            p.c_first = 0; p.n_parts = 1; p.part = 0;
+            return true;
+        }
+        if (gt >= gt_end) return false;
+        p.item = it;
+        p.w = a.items[it];
+        const int n_tiles = (p.w.kv_end + kKeysPerTile - 1) / kKeysPerTile;
+        const int first = p.w.split - off;    // the item's first tile in the concatenation
+        p.t0 = gt - first;
+        p.t1 = min(n_tiles, gt_end - first);
+        p.c_first = first / len;
+        p.n_parts = (first + n_tiles - 1) / len - p.c_first + 1;
+        p.part = (int)blockIdx.x - p.c_first;
+        gt = first + p.t1;
+        ++it;
         return true;
     }
 };
+// The same interface for batches whose items are all taken whole (what the host can tell in advance for short
+// batches): items blockIdx, blockIdx + blocks, ...
+struct WholeIter {
+    int whole, n_items;
+    __device__ explicit WholeIter(const AttnArgs &a) : whole((int)blockIdx.x), n_items(*a.n_items) {}
+    __device__ bool next(const AttnArgs &a, RunPiece &p) {
+        if (whole >= n_items) return false;
+        p.item = whole;
+        whole += (int)gridDim.x;
+        p.w = a.items[p.item];
+        p.t0 = 0;
+        p.t1 = (p.w.kv_end + kKeysPerTile - 1) / kKeysPerTile;
+        p.c_first = 0; p.n_parts = 1; p.part = 0;
+        return true;
+    }
+};
+// partial-result slot of part `part` of an item whose first part is held by block c_first: a block holds at
+// most one part > 0 (the piece its run starts with) and at most one part 0 of a cut item (the piece it ends with)
+__host__ __device__ __forceinline__ int part_slot(int c_first, int part) { return 2 * (c_first + part) + (part == 0 ? 1 : 0); }
 
 template <int HD>
 struct AttnSmem {
@@ -185,11 +245,12 @@ __device__ __forceinline__ float fast_exp2(float x) {
     return y;
 }
 
-template <int HD>
+template <int HD, bool kRuns>   // kRuns: items may be cut into runs (RunIter); else all items are whole (WholeIter)
 __global__ void __launch_bounds__(kAttnThreads, 1)
 attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_constant__ CUtensorMap tmKV,
                     const AttnArgs a) {
     using S = AttnSmem<HD>;
+    using Iter = typename std::conditional<kRuns, RunIter, WholeIter>::type;
     constexpr int kHalves = HD / 64;             // 64-wide column halves of the head dim
     constexpr int kHalfQ = 128 * 128;            // bytes of one 128-row x 64-col bf16 block
     extern __shared__ uint8_t smem_raw[];
@@ -235,7 +296,6 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     tc::grid_dep_wait();   // work list, q/k/v rows and the cache rows of the new tokens come from earlier kernels
     // tensor-memory columns of group g (base g*256): S_g 0..63, P_g 64..95, the first 64 head-dim columns of Q_g as
     // bf16 pairs 96..127, O_g 128..255
-    const int n_items = *a.n_items;
     const int tok_per_group = 128 / a.G;
     // K/V stage layout.  One TMA box ("unit") brings box_rows cache rows of one page, both 64-wide halves of the
     // head dim: [half][box_rows][128 bytes], 128-byte swizzle inside each half block.  A stage holds the 128 / box_rows
@@ -256,9 +316,10 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         // ------------------------------ TMA producer (whole warp) ------------------------------
         uint32_t n_item = 0, kt = 0;
         bool ok = true;
-        ItemIter items;
-        AttnWork w;
-        for (; ok && items.next(a, n_items, w); ++n_item) {
+        Iter run(a);
+        RunPiece pc;
+        for (; ok && run.next(a, pc); ++n_item) {
+            const AttnWork &w = pc.w;
             if (lane == 0) {
                 ok = tc::mbar_wait(q_free, (n_item & 1) ^ 1, abort_flag);
                 if (ok) {
@@ -274,8 +335,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 }
             }
             ok = __shfl_sync(0xffffffffu, ok, 0);
-            const int n_tiles = (w.kv_end + kKeysPerTile - 1) / kKeysPerTile;
-            for (int j = 0; j < n_tiles && ok; ++j, ++kt) {
+            for (int j = pc.t0; j < pc.t1 && ok; ++j, ++kt) {
                 const int st = kt % kKvStages;
                 const uint32_t par = ((kt / kKvStages) & 1) ^ 1;
                 const int kbase = j * kKeysPerTile;
@@ -341,10 +401,10 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         auto wait_all = [&](uint32_t bar, uint32_t parity) {
             return __all_sync(0xffffffffu, tc::mbar_wait(bar, parity, abort_flag));
         };
-        ItemIter items;
-        AttnWork w;
-        for (; ok && items.next(a, n_items, w); ++n_item) {
-            const int n_half = 2 * ((w.kv_end + kKeysPerTile - 1) / kKeysPerTile);   // both halves of every tile
+        Iter run(a);
+        RunPiece pc;
+        for (; ok && run.next(a, pc); ++n_item) {
+            const int n_half = 2 * (pc.t1 - pc.t0);   // both halves of every tile of the piece
             if (!wait_all(q_full, n_item & 1)) { ok = false; break; }
             if (!wait_all(q_ready(g), n_item & 1)) { ok = false; break; }
             if (!wait_all(k_full(kt % kKvStages), (kt / kKvStages) & 1)) { ok = false; break; }
@@ -399,8 +459,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const uint32_t o_addr = s_addr + 128;
         uint32_t n_s = 0, kt = 0;   // n_s: half tiles of this group so far (phase counter of its barriers)
         bool ok = true;
-        ItemIter items;
-        AttnWork w, w_next;
+        Iter run(a);
+        RunPiece pc, pc_next;
         const int tok_local = g * tok_per_group + row / a.G;
         // the first 64 head-dim columns of this thread's row of Q of a piece: global memory -> registers
         uint32_t qv[32];
@@ -423,17 +483,18 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             __syncwarp();
             if (lane == 0) tc::mbar_arrive(q_ready(g));
         };
-        bool have = items.next(a, n_items, w);
-        if (have) { load_q(w); publish_q(); }
+        bool have = run.next(a, pc);
+        if (have) { load_q(pc.w); publish_q(); }
         while (ok && have) {
-            const int n_half = 2 * ((w.kv_end + kKeysPerTile - 1) / kKeysPerTile);
+            const AttnWork &w = pc.w;
+            const int n_half = 2 * (pc.t1 - pc.t0);
             // position of this row's token; rows past the end of the block behave like its last token
             const int pos = w.kv_end - w.q_count + min(tok_local, w.q_count - 1);
             // exponent reference (a running maximum that is only moved when it has drifted by more than
             // 2^8, so the accumulator in tensor memory rarely needs rescaling) and row sum
             float m_ref = -INFINITY, l_run = 0.f;
             for (int i = 0; i < n_half && ok; ++i, ++n_s) {
-                const int tbase = (i >> 1) * kKeysPerTile;   // first key of the tile; column e of half hh is key
+                const int tbase = (pc.t0 + (i >> 1)) * kKeysPerTile;   // first key of the tile; column e of half hh is key
                 const int hh = i & 1;                        // tbase + (perm ? (e/8)*16 + hh*8 + e%8 : hh*64 + e)
                 if (!tc::mbar_wait(s_full(g), n_s & 1, abort_flag)) { ok = false; break; }
                 tc::tc_fence_after();
@@ -476,7 +537,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         m_tile = fmaxf(m_tile, __uint_as_float(sv[e]));
                     }
                     if ((m_tile - m_ref) * a.scale_log2 > 8.f) move_reference(m_tile);
-                    const float mb = m_ref * a.scale_log2;
+                    // (a piece that starts at an item's last tile can hold rows that see none of its keys so far)
+                    const float mb = m_ref == -INFINITY ? 0.f : m_ref * a.scale_log2;
 #pragma unroll
                     for (int e = 0; e < kHalfKeys; e += 2) {
                         const float p0 = fast_exp2(fmaf(__uint_as_float(sv[e]), a.scale_log2, -mb));
@@ -556,8 +618,8 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             if (!ok) break;
             // the next item's rows of Q go to tensor memory underneath this item's last P V, so that its first
             // Q K^T runs underneath this item's output
-            const bool have_next = items.next(a, n_items, w_next);
-            if (have_next) { load_q(w_next); publish_q(); }
+            const bool have_next = run.next(a, pc_next);
+            if (have_next) { load_q(pc_next.w); publish_q(); }
             // the item's last P V, normalisation, store
             if (!tc::mbar_wait(pv_done(g), (n_s - 1) & 1, abort_flag)) { ok = false; break; }
             tc::tc_fence_after();
@@ -586,7 +648,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 for (int j = 0; j < 4; ++j)
                     if (dst_quad[j]) *reinterpret_cast<uint4 *>(dst_quad[j] + c) = u[j];
             };
-            {
+            if (!kRuns || pc.n_parts == 1) {
                 const float inv = 1.f / l_run;
 #pragma unroll 1
                 for (int c = 0; c < HD; c += 32) {
@@ -599,8 +661,24 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                     store_chunk(c, o);
                 }
                 tc::tc_fence_before();
+            } else {
+                // part of a cut item: unnormalised rows, exponent references and sums go to the part's slot
+                const int grow = g * 128 + row;
+                float *po = a.part_o + (size_t)part_slot(pc.c_first, pc.part) * HD * 256 + grow;
+                float *pml = a.part_ml + (size_t)part_slot(pc.c_first, pc.part) * 512 + grow;
+#pragma unroll 1
+                for (int c = 0; c < HD; c += 32) {
+                    uint32_t v[32];
+                    tc::tmem_ld_32x32(o_addr + c, v);
+                    tc::tmem_ld_wait();
+#pragma unroll
+                    for (int e = 0; e < 32; ++e) po[(size_t)(c + e) * 256] = __uint_as_float(v[e]);
+                }
+                tc::tc_fence_before();
+                pml[0] = m_ref;
+                pml[256] = l_run;
             }
-            w = w_next;
+            pc = pc_next;
             have = have_next;
         }
     }
@@ -614,6 +692,53 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     }
 }
 
+
+// Merge of the parts of the cut items.  Blocks 2 * (c - 1) + g, c = 1 .. runs - 1: if run boundary c falls
+// strictly inside an item and is the first boundary inside it, the block merges the rows of group g of that
+// item: O = sum_p 2^((m_p - m) scale) O_p / sum_p 2^((m_p - m) scale) l_p, m = max_p m_p, parts in order.
+// Thread = (row, quarter of the head dim).
+template <int HD>
+__global__ void __launch_bounds__(512) attn_merge_kernel(const AttnArgs a) {
+    tc::grid_dep_launch();
+    tc::grid_dep_wait();
+    const int total = a.run_counts[0], len = a.run_counts[1], off = a.run_counts[3];
+    const int c = (int)blockIdx.x / 2 + 1, g = (int)blockIdx.x & 1;
+    if ((long long)c * len >= total) return;
+    const int item = a.cta_start[c];
+    const AttnWork w = a.items[item];
+    const int first = w.split - off, n_tiles = (w.kv_end + kKeysPerTile - 1) / kKeysPerTile;
+    const int c_first = first / len;
+    const int n_parts = (first + n_tiles - 1) / len - c_first + 1;
+    if (first == c * len || c != c_first + 1) return;   // boundary not inside the item / not its first boundary
+    const int row = threadIdx.x & 127, quarter = threadIdx.x >> 7, grow = g * 128 + row;
+    constexpr int kCols = HD / 4;
+    const int col0 = quarter * kCols;
+    const int tl = g * (128 / a.G) + row / a.G;
+    float m_all = -INFINITY;
+    for (int p = 0; p < n_parts; ++p) m_all = fmaxf(m_all, a.part_ml[(size_t)part_slot(c_first, p) * 512 + grow]);
+    float l_all = 0.f, acc[kCols];
+#pragma unroll
+    for (int e = 0; e < kCols; ++e) acc[e] = 0.f;
+    for (int p = 0; p < n_parts; ++p) {
+        const int slot = part_slot(c_first, p);
+        const float m_p = a.part_ml[(size_t)slot * 512 + grow];
+        const float wgt = m_p == -INFINITY ? 0.f : exp2f((m_p - m_all) * a.scale_log2);
+        l_all = fmaf(a.part_ml[(size_t)slot * 512 + 256 + grow], wgt, l_all);
+        const float *src = a.part_o + ((size_t)slot * HD + col0) * 256 + grow;
+#pragma unroll
+        for (int e = 0; e < kCols; ++e) acc[e] = fmaf(src[(size_t)e * 256], wgt, acc[e]);
+    }
+    if (tl >= w.q_count) return;
+    const float inv = 1.f / l_all;
+    __nv_bfloat16 *dst = a.out + (size_t)(w.q_start + tl) * a.Nq + (size_t)(w.kv_head * a.G + row % a.G) * HD + col0;
+#pragma unroll
+    for (int x = 0; x < kCols / 8; ++x) {
+        uint4 u;
+        u.x = tc::pack_bf16(acc[8 * x] * inv, acc[8 * x + 1] * inv); u.y = tc::pack_bf16(acc[8 * x + 2] * inv, acc[8 * x + 3] * inv);
+        u.z = tc::pack_bf16(acc[8 * x + 4] * inv, acc[8 * x + 5] * inv); u.w = tc::pack_bf16(acc[8 * x + 6] * inv, acc[8 * x + 7] * inv);
+        reinterpret_cast<uint4 *>(dst)[x] = u;
+    }
+}
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
                                   const cuuint64_t *, const cuuint32_t *, const cuuint32_t *, CUtensorMapInterleave,
@@ -669,23 +794,38 @@ int launch_attend_tc(alora_ctx *ctx, const void *qkv, const BatchArgs &b, const 
     a.max_blocks = b.max_blocks; a.num_pages = b.num_pages; a.Hkv = d.Hkv; a.G = d.G; a.page_size = d.page; a.box_rows = box_rows;
     a.N = d.N; a.Nq = d.Nq; a.qkv = (const __nv_bfloat16 *)qkv; a.scale_log2 = d.softmax_scale * 1.4426950408889634f;
     a.out = (__nv_bfloat16 *)out; a.status = ctx->d_status;
+    a.run_counts = ctx->d_counts + 6; a.cta_start = ctx->d_attn_cta_start;
+    a.part_o = ctx->d_attn_part_o; a.part_ml = ctx->d_attn_part_ml;
     const int max_items = (b.T / ctx->attn_q_block + b.R) * d.Hkv;
     const int grid = std::max(1, std::min(ctx->sm_count, max_items));
     ProfScope prof(ctx, KK_ATTENTION, s);
     static bool attr_set[2][64] = {};
     const int dev = ctx->cfg.device, hi = d.hd == 128;
+    // Items are cut into runs (and need the merge kernel) only when the batch has at least kAttnCutMinTiles key tiles
+    // per block; an upper bound from what the host knows decides whether that can be the case.
+    const long long max_tiles = (long long)max_items * (((long long)b.max_blocks * d.page + kKeysPerTile - 1) / kKeysPerTile);
+    const bool runs = grid > 1 && max_tiles >= (long long)kAttnCutMinTiles * grid;
     if (dev >= 0 && dev < 64 && !attr_set[hi][dev]) {
-        cudaError_t e = hi ? cudaFuncSetAttribute(attn_tcgen05_kernel<128>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                  AttnSmem<128>::kTotal)
-                           : cudaFuncSetAttribute(attn_tcgen05_kernel<64>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                                  AttnSmem<64>::kTotal);
+        cudaError_t e = hi ? cudaFuncSetAttribute(attn_tcgen05_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<128>::kTotal)
+                           : cudaFuncSetAttribute(attn_tcgen05_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<64>::kTotal);
+        if (e == cudaSuccess)
+            e = hi ? cudaFuncSetAttribute(attn_tcgen05_kernel<128, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<128>::kTotal)
+                   : cudaFuncSetAttribute(attn_tcgen05_kernel<64, true>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<64>::kTotal);
         if (e != cudaSuccess) return -1;
         attr_set[hi][dev] = true;
     }
-    const cudaError_t le = hi ? launch_kernel(attn_tcgen05_kernel<128>, dim3(grid), dim3(kAttnThreads), AttnSmem<128>::kTotal, s, true, tmQ, tmKV, a)
-                              : launch_kernel(attn_tcgen05_kernel<64>, dim3(grid), dim3(kAttnThreads), AttnSmem<64>::kTotal, s, true, tmQ, tmKV, a);
+    const dim3 g3(grid), b3(kAttnThreads);
+    cudaError_t le;
+    if (runs) le = hi ? launch_kernel(attn_tcgen05_kernel<128, true>, g3, b3, AttnSmem<128>::kTotal, s, true, tmQ, tmKV, a)
+                      : launch_kernel(attn_tcgen05_kernel<64, true>, g3, b3, AttnSmem<64>::kTotal, s, true, tmQ, tmKV, a);
+    else le = hi ? launch_kernel(attn_tcgen05_kernel<128, false>, g3, b3, AttnSmem<128>::kTotal, s, true, tmQ, tmKV, a)
+                 : launch_kernel(attn_tcgen05_kernel<64, false>, g3, b3, AttnSmem<64>::kTotal, s, true, tmQ, tmKV, a);
     if (le != cudaSuccess) return -1;
-    return 1 + n_small;
+    if (!runs) return 1 + n_small;
+    const cudaError_t me = hi ? launch_kernel(attn_merge_kernel<128>, dim3(2 * (grid - 1)), dim3(512), 0, s, true, a)
+                              : launch_kernel(attn_merge_kernel<64>, dim3(2 * (grid - 1)), dim3(512), 0, s, true, a);
+    if (me != cudaSuccess) return -1;
+    return 2 + n_small;
 }
 
 }  // namespace alora

@@ -1,5 +1,6 @@
 // Batch metadata: per-token request / applied-adapter / KV-slot arrays and the projection's
 // row-tile list.  Integer work only; every output is compared exactly against the CPU oracle.
+#include <climits>
 #include "alora_internal.h"
 #include "tc_common.cuh"
 
@@ -167,7 +168,8 @@ __device__ __forceinline__ void metadata_tiles(const int32_t *__restrict__ a_req
 __device__ __forceinline__ void metadata_attn_items(const int32_t *__restrict__ qsl, const int32_t *__restrict__ seq_lens,
                                            int R, int Hkv, int q_block, int small_max, int max_items,
                                            AttnWork *__restrict__ items, int32_t *__restrict__ counts,
-                                           int32_t *blk_off /* [R+1] */, int32_t *status) {
+                                           int32_t *blk_off /* [R+1] */, int n_blocks, int32_t *__restrict__ cta_start,
+                                           int32_t *status) {
     __shared__ int total;
     for (int r = threadIdx.x; r < R; r += blockDim.x) {
         const int n_new = qsl[r + 1] - qsl[r];
@@ -188,6 +190,7 @@ __device__ __forceinline__ void metadata_attn_items(const int32_t *__restrict__ 
         counts[1] = n;
     }
     __syncthreads();
+    int sum = 0, tmin = INT_MAX, tmax = 0;   // key tiles of this thread's items
     for (int i = threadIdx.x; i < total; i += blockDim.x) {
         int lo = 0, hi = R;      // blk_off[lo] * Hkv <= i < blk_off[hi] * Hkv
         while (hi - lo > 1) {
@@ -209,6 +212,79 @@ __device__ __forceinline__ void metadata_attn_items(const int32_t *__restrict__ 
         w.split = 0;
         w.n_splits = 1;
         items[i] = w;
+        const int n = (w.kv_end + kAttnKeysPerTile - 1) / kAttnKeysPerTile;
+        sum += n; tmin = min(tmin, n); tmax = max(tmax, n);
+    }
+    // Work split of the attention kernel over its n_blocks blocks.  Short batches (fewer than kAttnCutMinTiles key
+    // tiles per block): every item is taken whole, round-robin.  Long ones: when the items are of (nearly) equal
+    // length the first n_whole = n_blocks * floor(items / n_blocks) items are taken whole, round-robin; the key
+    // tiles of the remaining items (of all items when their lengths differ) are concatenated and cut into runs of
+    // equal length, one per block, so an item can be cut into parts that different blocks work on (a merge kernel
+    // adds the parts up).
+    //   items[i].split = tiles before item i;  counts[6] = tiles in the concatenation, counts[7] = run length,
+    //   counts[8] = n_whole, counts[9] = tiles before item n_whole;
+    //   cta_start[c] = the item that holds the first tile of block c's run.
+    __shared__ int warp_sum[32], warp_min[32], warp_max[32];
+    __shared__ int run_len, run_off, run_first;
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    for (int o = 1; o < 32; o <<= 1) {
+        sum += __shfl_xor_sync(0xffffffffu, sum, o);
+        tmin = min(tmin, __shfl_xor_sync(0xffffffffu, tmin, o));
+        tmax = max(tmax, __shfl_xor_sync(0xffffffffu, tmax, o));
+    }
+    if (lane == 0) { warp_sum[wid] = sum; warp_min[wid] = tmin; warp_max[wid] = tmax; }
+    __syncthreads();   // (also: this block's writes to items[] are visible to all of its threads)
+    if (threadIdx.x == 0) {
+        int acc = 0, mn = INT_MAX, mx = 0;
+        for (int w = 0; w < (int)(blockDim.x + 31) / 32; ++w) {
+            acc += warp_sum[w];
+            mn = min(mn, warp_min[w]); mx = max(mx, warp_max[w]);
+        }
+        const bool cut = acc >= kAttnCutMinTiles * n_blocks;
+        const bool uniform = total >= n_blocks && mx - mn <= max(1, mx / 16);
+        run_first = !cut ? -1 : (uniform ? n_blocks * (total / n_blocks) : 0);
+        run_len = acc;   // all tiles, for now
+        if (!cut) { counts[6] = 0; counts[7] = kAttnMinRunTiles; counts[8] = total; counts[9] = acc; }
+    }
+    __syncthreads();
+    if (run_first < 0) return;   // short batch: every item whole, nothing more to prepare
+    // tiles before each item: contiguous chunks of items per thread, scanned over the block
+    const int chunk = (total + (int)blockDim.x - 1) / (int)blockDim.x;
+    const int lo = min(total, (int)threadIdx.x * chunk), hi = min(total, lo + chunk);
+    sum = 0;
+    for (int i = lo; i < hi; ++i) sum += (items[i].kv_end + kAttnKeysPerTile - 1) / kAttnKeysPerTile;
+    int incl = sum;
+    for (int o = 1; o < 32; o <<= 1) {
+        const int v = __shfl_up_sync(0xffffffffu, incl, o);
+        if (lane >= o) incl += v;
+    }
+    __syncthreads();   // warp_sum is reused
+    if (lane == 31) warp_sum[wid] = incl;
+    __syncthreads();
+    int acc = incl - sum;
+    for (int w = 0; w < wid; ++w) acc += warp_sum[w];
+    for (int i = lo; i < hi; ++i) {
+        items[i].split = acc;
+        acc += (items[i].kv_end + kAttnKeysPerTile - 1) / kAttnKeysPerTile;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        const int all = run_len, first = run_first;
+        const int off = first < total ? items[first].split : all;
+        const int len = max((all - off + n_blocks - 1) / n_blocks, kAttnMinRunTiles);
+        counts[6] = all - off;
+        counts[7] = len;
+        counts[8] = first;
+        counts[9] = off;
+        run_len = len;
+        run_off = off;
+    }
+    __syncthreads();
+    const int len = run_len, off = run_off;
+    for (int i = max(lo, run_first); i < hi; ++i) {
+        const int rel = items[i].split - off;
+        const int n = (items[i].kv_end + kAttnKeysPerTile - 1) / kAttnKeysPerTile;
+        for (int c = (rel + len - 1) / len; c * len < rel + n && c < n_blocks; ++c) cta_start[c] = i;
     }
 }
 
@@ -350,7 +426,8 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *a_req, con
                 int Hkv, int q_block, int max_items, AttnWork *__restrict__ items, int32_t *blk_off,
                 int G, int n_sm, int small_max, int max_split_items, int max_split_rows,
                 AttnSplitWork *__restrict__ split_items,
-                int32_t *req_scratch, int32_t *__restrict__ group_done, int rowwise_cap, int32_t *status) {
+                int32_t *req_scratch, int32_t *__restrict__ group_done, int rowwise_cap,
+                int32_t *__restrict__ attn_cta_start, int32_t *status) {
     // The per-request inputs are read many times (binary searches, list builders): one parallel pass stages them
     // in shared memory, so that the later steps do not each pay a round trip to global memory.
     __shared__ int32_t s_req[4 * kMetaStageR + 1];
@@ -380,7 +457,8 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *a_req, con
                    T, rowwise_cap, shrink_tiles, t_ready, status);
     __syncthreads();  // the next builder reuses the scratch
     if (items != nullptr && block_tables != nullptr)
-        metadata_attn_items(qsl, seq_lens, R, Hkv, q_block, small_max, max_items, items, counts, blk_off, status);
+        metadata_attn_items(qsl, seq_lens, R, Hkv, q_block, small_max, max_items, items, counts, blk_off,
+                            max(1, min(n_sm, (T / q_block + R) * Hkv)), attn_cta_start, status);
     __syncthreads();
     if (split_items != nullptr && block_tables != nullptr)
         metadata_split_items(qsl, seq_lens, R, Hkv, G, n_sm, small_max, max_split_items, max_split_rows, split_items, counts,
@@ -402,7 +480,7 @@ int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s) {
         ctx->d.Hkv, ctx->attn_q_block, ctx->max_attn_items, ctx->d_attn_items, ctx->d_attn_off, ctx->d.G,
         ctx->sm_count, ctx->small_max_tokens, ctx->max_split_items, ctx->max_split_rows, ctx->d_split_items,
         ctx->d_req_scratch, ctx->d_group_done, ctx->d_row_delta ? kRowwiseMaxTokens : 0,
-        ctx->d_status);
+        ctx->d_attn_cta_start, ctx->d_status);
     return 1;
 }
 
