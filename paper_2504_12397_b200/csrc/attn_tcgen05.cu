@@ -802,9 +802,10 @@ int launch_attend_tc(alora_ctx *ctx, const void *qkv, const BatchArgs &b, const 
     static bool attr_set[2][64] = {};
     const int dev = ctx->cfg.device, hi = d.hd == 128;
     // Items are cut into runs (and need the merge kernel) only when the batch has at least kAttnCutMinTiles key tiles
-    // per block; an upper bound from what the host knows decides whether that can be the case.
+    // per block and kAttnCutMinWaves items per block; upper bounds from what the host knows decide whether that
+    // can be the case.
     const long long max_tiles = (long long)max_items * (((long long)b.max_blocks * d.page + kKeysPerTile - 1) / kKeysPerTile);
-    const bool runs = grid > 1 && max_tiles >= (long long)kAttnCutMinTiles * grid;
+    const bool runs = grid > 1 && max_tiles >= (long long)kAttnCutMinTiles * grid && max_items >= kAttnCutMinWaves * grid;
     if (dev >= 0 && dev < 64 && !attr_set[hi][dev]) {
         cudaError_t e = hi ? cudaFuncSetAttribute(attn_tcgen05_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<128>::kTotal)
                            : cudaFuncSetAttribute(attn_tcgen05_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<64>::kTotal);

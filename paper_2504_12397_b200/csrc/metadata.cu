@@ -215,12 +215,12 @@ __device__ __forceinline__ void metadata_attn_items(const int32_t *__restrict__ 
         const int n = (w.kv_end + kAttnKeysPerTile - 1) / kAttnKeysPerTile;
         sum += n; tmin = min(tmin, n); tmax = max(tmax, n);
     }
-    // Work split of the attention kernel over its n_blocks blocks.  Short batches (fewer than kAttnCutMinTiles key
-    // tiles per block): every item is taken whole, round-robin.  Long ones: when the items are of (nearly) equal
-    // length the first n_whole = n_blocks * floor(items / n_blocks) items are taken whole, round-robin; the key
-    // tiles of the remaining items (of all items when their lengths differ) are concatenated and cut into runs of
-    // equal length, one per block, so an item can be cut into parts that different blocks work on (a merge kernel
-    // adds the parts up).
+    // Work split of the attention kernel over its n_blocks blocks.  Normally every item is taken whole, round-robin.
+    // Long batches (at least kAttnCutMinTiles key tiles per block) of items of nearly equal length that make at
+    // least kAttnCutMinWaves full rounds: the first n_whole = n_blocks * floor(items / n_blocks) items are taken
+    // whole, round-robin; the key tiles of the remaining items are concatenated and cut into runs of equal length,
+    // one per block, so an item can be cut into parts that different blocks work on (a merge kernel adds the
+    // parts up).
     //   items[i].split = tiles before item i;  counts[6] = tiles in the concatenation, counts[7] = run length,
     //   counts[8] = n_whole, counts[9] = tiles before item n_whole;
     //   cta_start[c] = the item that holds the first tile of block c's run.
@@ -240,9 +240,12 @@ __device__ __forceinline__ void metadata_attn_items(const int32_t *__restrict__ 
             acc += warp_sum[w];
             mn = min(mn, warp_min[w]); mx = max(mx, warp_max[w]);
         }
-        const bool cut = acc >= kAttnCutMinTiles * n_blocks;
-        const bool uniform = total >= n_blocks && mx - mn <= max(1, mx / 16);
-        run_first = !cut ? -1 : (uniform ? n_blocks * (total / n_blocks) : 0);
+        // cutting pays when most of the work is still done on whole items (whose sibling query blocks share their
+        // K/V tiles in L2): items of nearly equal length, at least kAttnCutMinWaves full rounds of whole items
+        const bool uniform = mx - mn <= max(1, mx / 16);
+        const bool cut = acc >= kAttnCutMinTiles * n_blocks && uniform && total >= kAttnCutMinWaves * n_blocks &&
+                         total % n_blocks != 0;
+        run_first = !cut ? -1 : n_blocks * (total / n_blocks);
         run_len = acc;   // all tiles, for now
         if (!cut) { counts[6] = 0; counts[7] = kAttnMinRunTiles; counts[8] = total; counts[9] = acc; }
     }

@@ -107,14 +107,14 @@ def test_config3_ragged_multi_adapter_sampled_requests(oracle64):
 
 
 def test_long_uniform_batch_whole_items_and_cut_items(oracle64):
-    """19 requests x (15900 cached + 512 suffix tokens) on a small layer shape: 152 attention work items of about
-    127 key tiles each, enough work per block for the kernel to balance it: 148 items are taken whole and the last
-    4 are cut into runs of key tiles that many blocks work on, merged afterwards.  Request 18 holds the cut items,
-    request 0 only whole ones."""
+    """28 requests x (15400 cached + 1024 suffix tokens) on a small layer shape: 448 attention work items of about
+    125 key tiles each, three full rounds over the 148 blocks plus 4 items.  The kernel takes 444 items whole and
+    cuts the last 4 into runs of key tiles that many blocks work on, merged afterwards.  Request 27 holds the cut
+    items, request 0 only whole ones."""
     shape = wl.LayerShape(hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=64, page_size=16, dtype="bf16")
-    w = wl.config2(seed=11, requests=19, prefix=15900, suffix=512, shape=shape, rank=8)
+    w = wl.config2(seed=11, requests=28, prefix=15400, suffix=1024, shape=shape, rank=8)
     before, after, out_h, _ = _run_layer(w, seed=1011)
-    _check_requests(oracle64, w.shape, w, w.batch, before, after, out_h, [0, 18])
+    _check_requests(oracle64, w.shape, w, w.batch, before, after, out_h, [0, 27])
 
 
 def test_config5_decode_step_sampled_requests(oracle64):
