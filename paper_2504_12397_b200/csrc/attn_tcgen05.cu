@@ -17,8 +17,9 @@
 //               64 columns into tensor memory, keep a running exponent reference and sum (online
 //               softmax; a thread owns its whole row, so the row reductions need no cross-lane
 //               traffic), write P_g (bf16 pairs) to tensor memory; the output O_g accumulates in
-//               tensor memory across tiles and is rescaled only when a row's maximum has moved by
-//               more than 2^8 since the reference was last set; final normalisation and store.
+//               tensor memory across tiles and is rescaled only when the reference moves: when a half
+//               tile's probabilities sum to more than 2^14 (2^8 for a single one on masked tiles);
+//               final normalisation and store.
 // While one group does its exponentials the tensor pipe works for the other group and on the group's
 // own next scores.
 //
@@ -750,16 +751,31 @@ EncodeTiledFn tensor_map_encoder();  // gemm_tcgen05.cu
 int launch_attend_splitkv(alora_ctx *ctx, const void *qkv, const BatchArgs &b, const void *pool, void *out,
                           cudaStream_t s);  // attn_splitkv.cu
 
+static int launch_attend_long(alora_ctx *ctx, const void *qkv, const BatchArgs &b, const void *pool, void *out,
+                              cudaStream_t s);
+
 int launch_attend_tc(alora_ctx *ctx, const void *qkv, const BatchArgs &b, const void *pool, void *out,
                      cudaStream_t s) {
     if (b.T == 0) return 0;
-    // requests with few new tokens (decode, short suffixes) are on the few-row work list
-    int n_small = 0;
-    if (ctx->max_split_items > 0) {
-        n_small = launch_attend_splitkv(ctx, qkv, b, pool, out, s);
-        if (n_small < 0) return -1;
-        if (b.all_small) return n_small;
+    // Requests with few new tokens (decode, short suffixes) are on the few-row work list, the others on the
+    // tensor-core kernel's; the two kernels write disjoint output rows.  The few-row kernel goes second: when its
+    // list is empty (a prefill batch) its blocks come and go in the shadow of the first kernel's tail.
+    int n = 0;
+    if (!(b.all_small && ctx->max_split_items > 0)) {
+        n = launch_attend_long(ctx, qkv, b, pool, out, s);
+        if (n < 0) return -1;
     }
+    if (ctx->max_split_items > 0) {
+        const int n_small = launch_attend_splitkv(ctx, qkv, b, pool, out, s);
+        if (n_small < 0) return -1;
+        n += n_small;
+    }
+    return n;
+}
+
+static int launch_attend_long(alora_ctx *ctx, const void *qkv, const BatchArgs &b, const void *pool, void *out,
+                              cudaStream_t s) {
+    const int n_small = 0;
     const Dims &d = ctx->d;
     const bool page_ok = d.page >= 8 && d.page <= 128 && (d.page & (d.page - 1)) == 0;
     if ((d.hd != 64 && d.hd != 128) || 128 % d.G != 0 || !page_ok) return -1;
