@@ -117,6 +117,26 @@ def test_long_uniform_batch_whole_items_and_cut_items(oracle64):
     _check_requests(oracle64, w.shape, w, w.batch, before, after, out_h, [0, 27])
 
 
+def test_five_adapters_on_one_shared_prefix_cache(oracle64):
+    """Five requests (four different adapters and the base model) whose block tables point at the SAME physical
+    pages for their 512 cached positions: every request reads the one base-model prefix cache, writes only its own
+    suffix pages, and the shared pages stay bit-identical."""
+    shape = wl.LayerShape(hidden=256, n_q_heads=8, n_kv_heads=2, head_dim=128, page_size=16, dtype="bf16")
+    rng = np.random.default_rng(77)
+    P, S, ids = 512, [40, 24, 17, 33, 64], [0, 1, 2, -1, 3]
+    wqkv = wl.make_wqkv(shape, rng)
+    ads = [wl.make_adapter(shape, r, rng, scale=4.0) for r in (8, 16, 32, 8)]
+    b = wl.make_batch(shape, [P] * 5, S, ids, rng, shuffle_pages=True)
+    b.block_tables[1:, :P // shape.page_size] = b.block_tables[0, :P // shape.page_size]
+    w = wl.Workload("shared_prefix", shape, wqkv, ads, b, 77)
+    before, after, out_h, qkv_h = _run_layer(w, seed=1077, with_qkv=True)
+    _check_requests(oracle64, shape, w, b, before, after, out_h, range(5), qkv_h)
+    shared = b.block_tables[0, :P // shape.page_size].astype(np.int64)
+    import torch
+    idx = torch.from_numpy(shared).cuda()
+    assert torch.equal(before[idx], after[idx])
+
+
 def test_config5_decode_step_sampled_requests(oracle64):
     """64 requests (base model and 4 rank-32 adapters), contexts 1024..32768, one new token each: the shortest,
     the longest and two more requests, and the projection rows of all 64."""
