@@ -511,8 +511,66 @@ def main():
     for _ in range(3):
         e2e_step()
     barrier()
-    e2e_ms = max_over_ranks(timed(e2e_step, args.steps, stream, flush))
-    h2d = h_hidden.numel() * 2 + sum(t.numel() * 4 for t in h_ints)
+    e2e_serial_ms = max_over_ranks(timed(e2e_step, args.steps, stream, flush))
+
+    # The same steps as a pipeline, the way a server would run them: inputs and outputs double-buffered, the H2D
+    # copy of step i+1 and the D2H copy of step i-1 on streams of their own beside step i's kernels.  Every step
+    # still copies its own inputs in and its own result out inside the timed region.
+    s_in, s_out = torch.cuda.Stream(), torch.cuda.Stream()
+    # the six small integer arrays travel as one pinned buffer (each padded to 16 bytes) and one copy
+    offs, tot = [], 0
+    for t in h_ints:
+        offs.append(tot)
+        tot += (t.numel() + 3) // 4 * 4
+    h_pack = torch.zeros(tot, dtype=torch.int32).pin_memory()
+    for o, t in zip(offs, h_ints):
+        h_pack[o:o + t.numel()] = t.reshape(-1)
+    bufs = []
+    for _ in range(2):
+        d_pack = torch.empty(tot, dtype=torch.int32, device=d.hidden.device)
+        views = [d_pack[o:o + t.numel()].view(t.shape) for o, t in zip(offs, h_ints)]
+        bufs.append(dict(hidden=torch.empty_like(d.hidden), pack=d_pack, ints=views,
+                         out=torch.empty_like(main_case.out),
+                         h_out=torch.empty((T, shape.Nq), dtype=torch.bfloat16).pin_memory(),
+                         in_ev=torch.cuda.Event(), comp_ev=torch.cuda.Event(), out_ev=torch.cuda.Event(), used=False))
+
+    def e2e_pipeline(n):
+        for i in range(n):
+            bf = bufs[i % 2]
+            if bf["used"]:
+                s_in.wait_event(bf["comp_ev"])            # the step that last read these inputs is done
+            with torch.cuda.stream(s_in):
+                bf["hidden"].copy_(h_hidden, non_blocking=True)
+                bf["pack"].copy_(h_pack, non_blocking=True)
+                bf["in_ev"].record(s_in)
+            stream.wait_event(bf["in_ev"])
+            if bf["used"]:
+                stream.wait_event(bf["out_ev"])           # the result last written here has been read back
+            if flush is not None:
+                flush.zero_()
+            ab.alora_prefill_layer(ctx, 0, bf["hidden"], bf["ints"][0], bf["ints"][1], bf["ints"][2], bf["ints"][3],
+                                   bf["ints"][4], main_case.pool, bf["ints"][5], d.max_blocks, main_case.b.num_pages,
+                                   T, R, bf["out"], stream)
+            bf["comp_ev"].record(stream)
+            s_out.wait_event(bf["comp_ev"])
+            with torch.cuda.stream(s_out):
+                bf["h_out"].copy_(bf["out"], non_blocking=True)
+                bf["out_ev"].record(s_out)
+            bf["used"] = True
+
+    e2e_pipeline(4)
+    torch.cuda.synchronize()
+    barrier()
+    p0 = torch.cuda.Event(enable_timing=True); p1 = torch.cuda.Event(enable_timing=True)
+    p0.record(stream)
+    s_in.wait_event(p0); s_out.wait_event(p0)
+    e2e_pipeline(args.steps)
+    stream.wait_stream(s_out); stream.wait_stream(s_in)
+    p1.record(stream)
+    torch.cuda.synchronize()
+    e2e_ms = max_over_ranks(p0.elapsed_time(p1) / args.steps)
+    assert torch.equal(bufs[0]["h_out"], h_out) and torch.equal(bufs[1]["h_out"], h_out)
+    h2d = h_hidden.numel() * 2 + h_pack.numel() * 4
     d2h = h_out.numel() * 2
 
     # ---- roofline of the dominant kernel: per-kernel event times from a separate profiled pass -----
@@ -594,7 +652,8 @@ def main():
                        "tokens_per_step_per_gpu": T, "l2": "flushed between steps (256 MB memset outside the timed events)",
                        "timing": "mean of per-step CUDA-event durations on the launching stream, max over ranks"},
             "clocks": clocks, "e2e": {"value": world * T / (e2e_ms / 1e3), "unit": UNIT, "h2d_bytes_per_step": h2d,
-                                      "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms},
+                                      "d2h_bytes_per_step": d2h, "ms_per_step": e2e_ms, "serial_ms_per_step": e2e_serial_ms,
+                                      "how": "K steps as a 3-stream pipeline (H2D, kernels, D2H; double-buffered), total time / K; serial = one step at a time"},
             "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
             "full_lora_recompute": recompute, "full_lora_recompute_8k_prefix": recompute_8k,
             "decode": decode, "short_suffix": short, "stack": stack, "device_status": status,
