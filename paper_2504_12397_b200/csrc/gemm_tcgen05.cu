@@ -523,12 +523,19 @@ int launch_project_tc(alora_ctx *ctx, int layer, const void *hidden, int T, void
     return n;
 }
 
+int launch_linear256_tc(alora_ctx *ctx, const void *x, const void *W, int T, int K, int N, void *y,
+                        const void *residual, cudaStream_t s);  // gemm256_tcgen05.cu
+
 // Plain dense projection y = x W^T (+ residual) for o_proj and the MLP matrices.
 int launch_linear_tc(alora_ctx *ctx, const void *x, const void *W, int T, int K, int N, void *y,
                      const void *residual, cudaStream_t s) {
     if (T == 0) return 0;
     if (K % 8 != 0 || N % 8 != 0) return -1;
     ProfScope prof(ctx, KK_LINEAR, s);
+    {
+        const int r = launch_linear256_tc(ctx, x, W, T, K, N, y, residual, s);   // many rows: 256 x 256 tiles
+        if (r != 0) return r;
+    }
     const int BN = pick_bn(N, N, 0, false, T);
     CUtensorMap tmX, tmW;
     if (!make_tensor_map_bf16(&tmX, x, T, K, K, kBM)) return -1;

@@ -394,6 +394,32 @@ def test_two_layer_stack(oracle64):
         g.close()
 
 
+def test_stack_layer_with_many_rows_takes_the_256_row_gemm(oracle64):
+    """One decoder layer on 2048 tokens with a wide MLP: gate/up (2048 x 9472 outputs = 296 tiles of 256 x 256) runs
+    on the 256-row GEMM kernel, o_proj and down (one column tile) on the 128-row kernel."""
+    shape = wl.LayerShape(hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=64, page_size=16, dtype="bf16",
+                          intermediate=4736)
+    rng = np.random.default_rng(41)
+    layers = [wl.make_stack_weights(shape, rng)]
+    ads = [[wl.make_adapter(shape, 8, rng)]]
+    b = wl.make_batch(shape, [0] * 8, [256] * 8, [0, -1] * 4, rng, activation_offsets=[100] * 8, shuffle_pages=True)
+    g = hp.GpuLayers(shape, layers, ads, 2048, 8)
+    try:
+        d = hp.DevBatch(b, shape.dtype)
+        pools = [g.new_pool(b.num_pages)]
+        hout = g.empty(b.T, shape.hidden)
+        ab.alora_forward_stack(g.ctx, ab.MODE_ALORA, d.hidden, d.positions, d.a_req, d.ids, d.qsl, d.seq_lens, pools,
+                               d.bt, d.max_blocks, b.num_pages, d.T, d.R, hout)
+        assert g.status() == 0
+        x, _ = oracle64.decoder_layer(b.hidden.astype(np.float64), layers[0], shape.Nq, shape.Nkv, shape.n_q_heads,
+                                      shape.n_kv_heads, shape.head_dim, 1e-5, b.positions, b.query_start_loc,
+                                      b.activation_offsets, b.adapter_ids, hp.oracle_adapters(ads[0]),
+                                      [None] * b.R, [None] * b.R)
+        assert hp.rel_err(hp.to_host(hout), x) <= 2e-2
+    finally:
+        g.close()
+
+
 def test_empty_and_degenerate_batches():
     w, ads, b = _mid_workload()
     g = hp.GpuLayers(MID, [dict(wqkv=w)], [ads], 256, 8)
