@@ -86,6 +86,11 @@ struct TcLayerMaps {
     CUtensorMap wqkv[3];      // W_qkv [N][H], boxes of 128 / 256 / 64 rows
     CUtensorMap a_all;        // all adapters' A rows [max_adapters*192][H], box 192 rows
     CUtensorMap b_all_bn[3];  // all adapters' B rows [max_adapters*N][64], boxes of 128 / 256 / 64 rows
+    // for the 256 x 192 tiles of gemm_pair_tcgen05.cu: W in boxes of 192 rows; per q / k / v block the B rows of all
+    // adapters as (rank column, row inside the block, adapter), boxes of 192 rows
+    CUtensorMap wqkv192;
+    CUtensorMap b_blk[3];
+    bool pair_ok = false;
 };
 
 struct Dims {

@@ -463,11 +463,19 @@ static int pick_bn(int N, int Nq, int Nkv, bool lora, int T) {
 
 // q/k/v projection of one layer on the tensor cores: shrink (t = s A x on adapter tiles), then the
 // base GEMM with the expand step fused.  Returns kernels launched, or -1 when the shape is unsupported.
+int launch_project_pair_tc(alora_ctx *ctx, int layer, const void *hidden, int T, void *qkv, cudaStream_t s,
+                           void *kv_pool, int num_pages);  // gemm_pair_tcgen05.cu
+
 int launch_project_tc(alora_ctx *ctx, int layer, const void *hidden, int T, void *qkv, cudaStream_t s, void *kv_pool,
                       int num_pages) {
     if (T == 0) return 0;
     const Dims &d = ctx->d;
     const bool have_adapters = ctx->layer_has_adapter[layer];
+    if (ctx->tc_maps[layer].pair_ok) {   // many rows: two row tiles per block, 192-wide column tiles
+        ProfScope prof(ctx, KK_PROJECT, s);
+        const int r = launch_project_pair_tc(ctx, layer, hidden, T, qkv, s, kv_pool, num_pages);
+        if (r != 0) return r;
+    }
     const int BN = pick_bn(d.N, d.Nq, d.Nkv, true, T);
     if (BN == 0 || d.H % 8 != 0) return -1;
     CUtensorMap tmX, tmTt;
@@ -525,6 +533,7 @@ int launch_project_tc(alora_ctx *ctx, int layer, const void *hidden, int T, void
 
 int launch_linear256_tc(alora_ctx *ctx, const void *x, const void *W, int T, int K, int N, void *y,
                         const void *residual, cudaStream_t s);  // gemm256_tcgen05.cu
+bool build_pair_maps(alora_ctx *ctx, int layer);                 // gemm_pair_tcgen05.cu
 
 // Plain dense projection y = x W^T (+ residual) for o_proj and the MLP matrices.
 int launch_linear_tc(alora_ctx *ctx, const void *x, const void *W, int T, int K, int N, void *y,
@@ -567,6 +576,7 @@ bool build_layer_maps(alora_ctx *ctx, int layer) {
     ok &= make_tensor_map_bf16(&lm.b_all_bn[0], ctx->tc_b_all[layer], na * d.N, kTensorRP, kTensorRP, 128);
     ok &= make_tensor_map_bf16(&lm.b_all_bn[1], ctx->tc_b_all[layer], na * d.N, kTensorRP, kTensorRP, 256);
     ok &= make_tensor_map_bf16(&lm.b_all_bn[2], ctx->tc_b_all[layer], na * d.N, kTensorRP, kTensorRP, 64);
+    lm.pair_ok = lw.wqkv != nullptr && build_pair_maps(ctx, layer);   // optional: the 128-row kernel serves every shape
     return ok;
 }
 
