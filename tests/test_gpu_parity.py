@@ -236,6 +236,19 @@ def test_projection_row_tile_route_with_fused_shrink(oracle64):
     _check_projection(oracle64, MID, w, ads, b, n_off_expected=130 + 130 + 195)
 
 
+def test_projection_of_many_rows_two_row_tiles_per_block(oracle64):
+    """Many rows (and enough tiles to fill the blocks): the projection takes 256 x 192 tiles (two row tiles per block).  With this shape's
+    blocks of 1024 / 256 / 256 columns the 192-wide column tiles straddle the q | k and k | v boundaries, some
+    row tiles are partial, one request runs on the base model and gates open in the middle of requests."""
+    rng = np.random.default_rng(45)
+    w = wl.make_wqkv(MID, rng)
+    ads = _boosted_adapters(MID, rng, ((8, 1.0), (64, 0.5), (32, 2.0)))
+    b = wl.make_batch(MID, [0, 300, 20, 5, 0], [1500, 1390, 530, 760, 428], [1, 0, -1, 2, 0], rng,
+                      activation_offsets=[130, 300, 0, 200, 77])
+    assert b.T == 4608   # 18 row pairs x 8 column tiles = 144 items for 148 blocks: the launcher prefers this tile shape
+    _check_projection(oracle64, MID, w, ads, b, n_off_expected=130 + 530 + 195 + 77)
+
+
 def test_projection_row_wise_route_many_short_requests(oracle64):
     """Many requests of 1..9 new tokens over different adapters and the base model, some gated off: the row
     tiles would hold a few rows each, so the batch takes the row-wise delta route."""
