@@ -1,5 +1,6 @@
 // Batch metadata: per-token request / applied-adapter / KV-slot arrays and the projection's
 // row-tile list.  Integer work only; every output is compared exactly against the CPU oracle.
+#include <algorithm>
 #include <climits>
 #include "alora_internal.h"
 #include "tc_common.cuh"
@@ -450,20 +451,27 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *a_req, con
     }
     metadata_tokens(positions, a_req, adapter_ids, qsl, seq_lens, block_tables, max_blocks, num_pages, page_size,
                     max_adapters, T, R, mode, token_req, row_adapter, slot_map, status);
-    if (blockIdx.x != 0) return;
+    // The three list builders are independent of one another: blocks 0, 1 and 2 take one each (a launch has at least
+    // three blocks; with fewer, block 0 would run them one after the other).
+    const int nb = (int)gridDim.x;
+    const int b_tiles = 0, b_attn = nb > 1 ? 1 : 0, b_split = nb > 2 ? 2 : 0;
+    if ((int)blockIdx.x != b_tiles && (int)blockIdx.x != b_attn && (int)blockIdx.x != b_split) return;
     // the per-request scratch of the list builders (their serial parts walk it) lives in shared memory when the
-    // batch is small enough, else in the context's global scratch
+    // batch is small enough, else in the context's global scratch (one buffer per builder)
     __shared__ int32_t smem_scratch[kMetaSmemInts];
     if (14 * R + 5 <= kMetaSmemInts) seg_scratch = blk_off = req_scratch = smem_scratch;
     __syncthreads();
-    metadata_tiles(a_req, adapter_ids, qsl, seq_lens, R, mode, max_adapters, max_tiles, tiles, counts, seg_scratch,
-                   T, rowwise_cap, shrink_tiles, t_ready, status);
-    __syncthreads();  // the next builder reuses the scratch
-    if (items != nullptr && block_tables != nullptr)
+    if ((int)blockIdx.x == b_tiles) {
+        metadata_tiles(a_req, adapter_ids, qsl, seq_lens, R, mode, max_adapters, max_tiles, tiles, counts, seg_scratch,
+                       T, rowwise_cap, shrink_tiles, t_ready, status);
+        __syncthreads();  // a builder that follows in this block reuses the scratch
+    }
+    if ((int)blockIdx.x == b_attn && items != nullptr && block_tables != nullptr) {
         metadata_attn_items(qsl, seq_lens, R, Hkv, q_block, small_max, max_items, items, counts, blk_off,
                             max(1, min(n_sm, (T / q_block + R) * Hkv)), attn_cta_start, status);
-    __syncthreads();
-    if (split_items != nullptr && block_tables != nullptr)
+        __syncthreads();
+    }
+    if ((int)blockIdx.x == b_split && split_items != nullptr && block_tables != nullptr)
         metadata_split_items(qsl, seq_lens, R, Hkv, G, n_sm, small_max, max_split_items, max_split_rows, split_items, counts,
                              req_scratch, group_done, status);
 }
@@ -475,7 +483,7 @@ int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s) {
     }
     ProfScope prof(ctx, KK_METADATA, s);
     const int threads = 256;
-    metadata_kernel<<<(b.T + threads - 1) / threads, threads, 0, s>>>(
+    metadata_kernel<<<std::max(3, (b.T + threads - 1) / threads), threads, 0, s>>>(
         b.positions, b.activation_offsets, b.adapter_ids, b.query_start_loc, b.seq_lens, b.block_tables,
         b.max_blocks, b.num_pages, ctx->d.page, ctx->cfg.max_adapters, b.T, b.R, b.mode, ctx->d_token_req,
         ctx->d_row_adapter, ctx->d_slot, ctx->max_tiles, ctx->d_tiles, ctx->d_counts, ctx->d_seg_scratch,
