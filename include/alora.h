@@ -30,7 +30,9 @@
  *   - Paged cache of one layer: pool[num_pages][2][Hkv][page_size][hd] (K plane, then V plane).
  *     Position p of request r lives in page block_tables[r][p / page_size], row p % page_size.
  *   - `stream` is a cudaStream_t passed as void* (NULL = default stream).  Work is enqueued and the
- *     call returns; nothing synchronises unless stated.
+ *     call returns; nothing synchronises unless stated.  Most kernels are launched with programmatic
+ *     stream serialization: their set-up may run under the tail of the preceding kernel of the stream,
+ *     but they read and write the call's buffers only after everything enqueued earlier has completed.
  *   - Every call returns an alora_status.  Host-side argument errors are detected before anything
  *     is launched.  Device-side findings (page id out of range, inconsistent positions, a bounded
  *     wait that ran out) are recorded in a status word readable with alora_get_status after the
@@ -286,8 +288,10 @@ alora_status alora_project_qkv_static(int dtype, int hidden, int n_q, int n_kv, 
  * alora_profile_read synchronises the device and adds up, per family, the elapsed milliseconds and
  * the number of bracketed launch groups; both arrays have ALORA_PROFILE_KINDS entries.
  * Families: 0 batch metadata, 1 rank-r shrink (t = A x) when it is a launch of its own, or the per-row
- * low-rank delta of small batches, 2 q/k/v projection, 3 KV append, 4 attention, 5 unused (key ranges are
- * merged inside the attention kernel), 6 other dense projections (o_proj, MLP), 7 norm / activation glue.
+ * low-rank delta of small batches, 2 q/k/v projection (on the bf16 layer paths it also appends the new k / v rows
+ * to the cache), 3 KV append as a launch of its own (alora_kv_append, fp32 layers), 4 attention (both attention
+ * kernels and the merge of cut work items), 5 unused, 6 other dense projections (o_proj, MLP), 7 norm / activation
+ * glue.
  */
 #define ALORA_PROFILE_KINDS 8
 alora_status alora_profile_enable(alora_ctx *ctx, int on);
