@@ -15,7 +15,8 @@
 // adapter) whose out-of-range rows read as zero, so the columns of the other block get no contribution.
 //
 //   warp 0   TMA producer (4 slots of 56 KB)      warp 1   MMA issuer (whole warp walks, elected lane issues)
-//   warps 2-5  epilogue: tcgen05.ld one row per thread, bf16, 16-byte stores, KV append, or t for shrink items
+//   warps 2-5 / 6-9  epilogue of the first / second row tile: tcgen05.ld one row per thread, bf16, 16-byte stores,
+//              KV append, or t for shrink items
 // All waits are bounded; on expiry ALORA_ERR_TIMEOUT is recorded and the block leaves normally.
 #include <algorithm>
 
@@ -25,7 +26,7 @@
 namespace alora {
 
 namespace {
-constexpr int kBNp = 192, kBKp = 64, kStagesP = 4, kThreadsP = 192;
+constexpr int kBNp = 192, kBKp = 64, kStagesP = 4, kThreadsP = 320;   // producer, issuer, 2 x 4 epilogue warps
 constexpr int kTensorRP = 64;                      // the tensor path stores adapters padded to 64 rank columns
 constexpr int kHalfAp = 128 * kBKp * 2;            // one row tile's x (or t) block: 16 KB
 constexpr int kBBytesP = kBNp * kBKp * 2;          // 24 KB
@@ -262,8 +263,9 @@ gemm_pair_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_c
             while (!tc::mbar_try_wait(drain_bar, 0) && clock64() - t0 < tc::kWaitCycleLimit) {}
         }
     } else {
-        // ------------------------------ epilogue (warps 2..5) ------------------------------
-        const int q = warp & 3;  // tensor-memory lane quarter this warp may read
+        // ------------------------------ epilogue (warps 2..5: first row tile, warps 6..9: second) ------------------------------
+        const int q = warp & 3;           // tensor-memory lane quarter this warp may read
+        const int my_h = (warp - 2) >> 2; // the half of tensor memory (row tile of the pair) this warp drains
         uint32_t it = 0;
         bool ok = true;
         for (int item = blockIdx.x; item < total && ok; item += gridDim.x, ++it) {
@@ -271,6 +273,12 @@ gemm_pair_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_c
             if (!tc::mbar_wait(accf_bar, it & 1, abort_flag)) { ok = false; break; }
             tc::tc_fence_after();
             const int r = q * 32 + lane;
+            if (g.shrink && my_h == 1) {   // a shrink item has one row tile only
+                tc::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(acce_bar(1));
+                continue;
+            }
             if (g.shrink) {
                 // t = s A x of this row tile: 192 columns, scaled, rounded to bf16
                 const ProjTile t = g.t[0];
@@ -302,12 +310,11 @@ gemm_pair_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_c
                 if (lane == 0) {
                     atomicAdd(a.t_ready + g.m[0], 1);
                     tc::mbar_arrive(acce_bar(0));
-                    tc::mbar_arrive(acce_bar(1));
                 }
                 continue;
             }
-#pragma unroll 1
-            for (int h = 0; h < 2; ++h) {
+            {
+                const int h = my_h;
                 if (g.m[h] >= 0) {
                     const ProjTile t = g.t[h];
                     const bool row_ok = r < t.row_count;
