@@ -179,10 +179,14 @@ alora_status alora_create(const alora_config *cfg, alora_ctx **out) {
         alloc((void **)&ctx->d_attn_part_o, (size_t)2 * ctx->sm_count * d.hd * 256 * 4);
         alloc((void **)&ctx->d_attn_part_ml, (size_t)2 * ctx->sm_count * 2 * 256 * 4);
         if (16 % d.G == 0 && (d.hd == 64 || d.hd == 128)) {
-            // few-row attention: at most kSplitItemsPerSm * n_sm key ranges plus one per (request, KV head, row
-            // block); a range of mt row tiles owns 16 * mt rows of the partial-result arrays
-            ctx->small_max_tokens = 16;
-            const int blocks_per_req = std::max(1, (16 * d.G + 63) / 64);
+            // few-row attention, for requests whose new tokens make at most 16 score rows per KV head (decode steps,
+            // suffixes of up to 16 / G tokens); longer ones go to the tensor-core kernel, which is the faster of
+            // the two from 32 rows on (measured: 8- and 16-token suffixes of 64 requests on 4096 cached tokens
+            // reach 0.71 / 0.72 of the HBM bandwidth there against 0.57 / 0.37 here).  At most kSplitItemsPerSm * n_sm
+            // key ranges plus one per (request, KV head, row block); a range of mt row tiles owns 16 * mt rows of
+            // the partial-result arrays
+            ctx->small_max_tokens = std::max(1, 16 / d.G);
+            const int blocks_per_req = std::max(1, (ctx->small_max_tokens * d.G + 63) / 64);
             const int groups = c.max_requests * blocks_per_req * d.Hkv;
             ctx->max_split_items = kSplitItemsPerSm * ctx->sm_count + groups;
             ctx->max_split_rows = 16 * (kSplitItemsPerSm * ctx->sm_count + 4 * groups);

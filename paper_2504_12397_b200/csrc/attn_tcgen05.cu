@@ -379,6 +379,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         constexpr uint32_t idesc_s = tc::idesc_bf16_f32(128, kHalfKeys);
         constexpr uint32_t idesc_pv = idesc_bf16_f32_bmn(128, HD);
         uint32_t n_item = 0, kt = 0, nh = 0;   // nh: half tiles handled so far (phase counter of the group's barriers)
+        uint32_t n_act = 0;                     // items in which this group had rows (phase counter of q_ready)
         bool ok = true;
         const uint32_t qa = smem_base + S::kQOff + g * S::kQBytes;
         const uint32_t s_tmem = tmem_base + g * 256, p_tmem = s_tmem + 64, q_tmem = s_tmem + 96, o_tmem = s_tmem + 128;
@@ -407,7 +408,23 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         for (; ok && run.next(a, pc); ++n_item) {
             const int n_half = 2 * (pc.t1 - pc.t0);   // both halves of every tile of the piece
             if (!wait_all(q_full, n_item & 1)) { ok = false; break; }
-            if (!wait_all(q_ready(g), n_item & 1)) { ok = false; break; }
+            if (g == 1 && pc.w.q_count <= tok_per_group) {
+                // A short block of tokens: all its score rows are in group 0.  This group's issuer only hands the
+                // piece's K/V stages and Q back (each after it has been filled, so that it never runs ahead of the
+                // producer by a whole phase), and the group's softmax warps skip the piece.
+                for (int j = pc.t0; j < pc.t1 && ok; ++j, ++kt) {
+                    const int st = kt % kKvStages;
+                    const uint32_t par = (kt / kKvStages) & 1;
+                    if (!wait_all(k_full(st), par)) { ok = false; break; }
+                    if (leader) tc::mbar_arrive(k_free(st));
+                    if (!wait_all(v_full(st), par)) { ok = false; break; }
+                    if (leader) tc::mbar_arrive(v_free(st));
+                }
+                if (ok && leader) tc::mbar_arrive(q_free);
+                continue;
+            }
+            if (!wait_all(q_ready(g), n_act & 1)) { ok = false; break; }
+            ++n_act;
             if (!wait_all(k_full(kt % kKvStages), (kt / kKvStages) & 1)) { ok = false; break; }
             tc::tc_fence_after();
             issue_s(kt % kKvStages, 0);
@@ -484,7 +501,16 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             __syncwarp();
             if (lane == 0) tc::mbar_arrive(q_ready(g));
         };
-        bool have = run.next(a, pc);
+        // the next piece in which this group has rows (a short block of tokens has none in group 1); the key tiles of
+        // the pieces passed over still count for the position in the K/V ring
+        auto next_piece = [&](RunPiece &p) {
+            while (run.next(a, p)) {
+                if (!(g == 1 && p.w.q_count <= tok_per_group)) return true;
+                kt += p.t1 - p.t0;
+            }
+            return false;
+        };
+        bool have = next_piece(pc);
         if (have) { load_q(pc.w); publish_q(); }
         while (ok && have) {
             const AttnWork &w = pc.w;
@@ -619,7 +645,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             if (!ok) break;
             // the next item's rows of Q go to tensor memory underneath this item's last P V, so that its first
             // Q K^T runs underneath this item's output
-            const bool have_next = run.next(a, pc_next);
+            const bool have_next = next_piece(pc_next);
             if (have_next) { load_q(pc_next.w); publish_q(); }
             // the item's last P V, normalisation, store
             if (!tc::mbar_wait(pv_done(g), (n_s - 1) & 1, abort_flag)) { ok = false; break; }
@@ -711,6 +737,7 @@ __global__ void __launch_bounds__(512) attn_merge_kernel(const AttnArgs a) {
     const int c_first = first / len;
     const int n_parts = (first + n_tiles - 1) / len - c_first + 1;
     if (first == c * len || c != c_first + 1) return;   // boundary not inside the item / not its first boundary
+    if (g == 1 && w.q_count <= 128 / a.G) return;       // no rows of the item in this group
     const int row = threadIdx.x & 127, quarter = threadIdx.x >> 7, grow = g * 128 + row;
     constexpr int kCols = HD / 4;
     const int col0 = quarter * kCols;

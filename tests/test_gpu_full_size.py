@@ -137,6 +137,24 @@ def test_five_adapters_on_one_shared_prefix_cache(oracle64):
     assert torch.equal(before[idx], after[idx])
 
 
+def test_short_suffixes_of_many_requests_on_long_prefixes(oracle64):
+    """40 requests with 1 .. 64 new tokens on 700 .. 2300 cached ones (6 .. 19 key tiles), base model and two
+    adapters.  Up to 16 score rows per KV head (here 4 tokens) a request is on the few-row kernel's list; from 5
+    to 32 tokens all its rows fall into the first query group of a tensor-core work item, whose second group then
+    skips the item; from 33 tokens on both groups work.  One request of every kind is checked in full."""
+    shape = wl.LayerShape(hidden=256, n_q_heads=8, n_kv_heads=2, head_dim=128, page_size=16, dtype="bf16")
+    rng = np.random.default_rng(91)
+    S = [1, 4, 5, 8, 16, 31, 32, 33, 47, 64] * 4
+    P = [int(x) for x in rng.integers(700, 2300, size=len(S))]
+    ids = [(-1, 0, 1)[i % 3] for i in range(len(S))]
+    wqkv = wl.make_wqkv(shape, rng)
+    ads = [wl.make_adapter(shape, r, rng, scale=4.0) for r in (8, 32)]
+    b = wl.make_batch(shape, P, S, ids, rng, shuffle_pages=True)
+    w = wl.Workload("short_suffixes", shape, wqkv, ads, b, 91)
+    before, after, out_h, qkv_h = _run_layer(w, seed=1091, with_qkv=True)
+    _check_requests(oracle64, shape, w, b, before, after, out_h, [10, 21, 12, 33, 4, 25, 36, 17, 38, 9], qkv_h)
+
+
 def test_config5_decode_step_sampled_requests(oracle64):
     """64 requests (base model and 4 rank-32 adapters), contexts 1024..32768, one new token each: the shortest,
     the longest and two more requests, and the projection rows of all 64."""
