@@ -4,10 +4,10 @@
 // is 2 x 128 score rows ("groups"): rows are (token, query head of the KV group) pairs, so the G
 // query heads that share a KV head share every K/V tile brought on chip.  Keys come in tiles of 128
 // and are consumed as two half tiles of 64.  Roles:
-//   warp 8      TMA producer: the head-dim columns 64.. of the two 128-row query tiles (3-D boxes
-//               d x head x token out of the fused q/k/v rows) and, per key tile, the K and V rows
-//               fetched through the block table (one 3-D box per 8 / 16 / 64 cache rows, both 64-wide
-//               halves of the head dim), three-deep rings for K and for V;
+//   warps 8, 11 TMA producers.  Warp 8: the head-dim columns 64.. of the two 128-row query tiles (3-D boxes
+//               d x head x token out of the fused q/k/v rows) and, per key tile, the K rows fetched through
+//               the block table (one 3-D box per 8 / 16 / 64 cache rows, both 64-wide halves of the head
+//               dim); warp 11: the V rows likewise.  Three-deep rings for K and for V;
 //   warps 9, 10 MMA issuers of group 0 and 1 (the whole warp walks the schedule, an elected lane
 //               issues): S_g = Q_g K^T of a half tile (fp32, tensor memory; head-dim columns 0..63 of
 //               Q_g are the A operand from tensor memory, the rest from shared memory), issued as soon
@@ -21,7 +21,9 @@
 //               tile's probabilities sum to more than 2^14 (2^8 for a single one on masked tiles);
 //               final normalisation and store.
 // While one group does its exponentials the tensor pipe works for the other group and on the group's
-// own next scores.
+// own next scores.  A block of at most 128 / G tokens (a short suffix) has score rows for one group only:
+// both groups then hold the same rows, group g takes half g of every key tile, and the two partial results
+// are merged out of tensor memory at the end of the item.
 //
 // Masking: key j is visible to a row at position p iff j <= p; masked probabilities are set to
 // zero explicitly, and V rows of keys at or beyond the item's causal limit are cleared in shared
@@ -33,7 +35,7 @@
 
 namespace alora {
 
-constexpr int kAttnThreads = 352;   // 8 softmax warps, TMA producer, two MMA issuers
+constexpr int kAttnThreads = 384;   // 8 softmax warps, TMA producer for Q and K, two MMA issuers, TMA producer for V
 constexpr int kKeysPerTile = 128;   // keys per K/V stage in shared memory
 constexpr int kHalfKeys = 64;       // keys per score / probability tile in tensor memory
 constexpr int kKvStages = 3;
@@ -180,6 +182,12 @@ __device__ __forceinline__ void tmem_st_32x32(uint32_t taddr, const uint32_t (&r
           "r"(r[24]), "r"(r[25]), "r"(r[26]), "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
         : "memory");
 }
+__device__ __forceinline__ void tmem_st_32x2(uint32_t taddr, uint32_t r0, uint32_t r1) {
+    asm volatile("tcgen05.st.sync.aligned.32x32b.x2.b32 [%0], {%1, %2};" ::"r"(taddr), "r"(r0), "r"(r1) : "memory");
+}
+__device__ __forceinline__ void tmem_ld_32x2(uint32_t taddr, uint32_t &r0, uint32_t &r1) {
+    asm volatile("tcgen05.ld.sync.aligned.32x32b.x2.b32 {%0, %1}, [%2];" : "=r"(r0), "=r"(r1) : "r"(taddr) : "memory");
+}
 __device__ __forceinline__ void tmem_st_wait() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
 
 __device__ __forceinline__ void tma_load_3d(uint32_t smem_dst, const CUtensorMap *map, uint32_t bar, int c0, int c1,
@@ -271,8 +279,10 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     auto s_free = [&](int w) { return bar1 + 48 + 8u * w; };
     auto drain_bar = [&](int w) { return bar1 + 64 + 8u * w; };
     auto q_ready = [&](int w) { return bar1 + 80 + 8u * w; };
-    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_al + S::kBarOff + 16 + 8 * 4 * kKvStages + 96);
-    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_al + S::kBarOff + 16 + 8 * 4 * kKvStages + 104);
+    // shared items (see below): both groups have their part of the result in tensor memory / have read the other's
+    const uint32_t merge_bar = bar1 + 96, merge_done = bar1 + 104;
+    volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(smem_al + S::kBarOff + 16 + 8 * 4 * kKvStages + 112);
+    volatile int *abort_flag = reinterpret_cast<volatile int *>(smem_al + S::kBarOff + 16 + 8 * 4 * kKvStages + 120);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
@@ -284,6 +294,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         for (int w = 0; w < 2; ++w) { tc::mbar_init(s_full(w), 1); tc::mbar_init(p_ready(w), 4); tc::mbar_init(pv_done(w), 1);
                                       tc::mbar_init(s_free(w), 4); tc::mbar_init(q_ready(w), 4); }
         tc::mbar_init(drain_bar(0), 1); tc::mbar_init(drain_bar(1), 1);
+        tc::mbar_init(merge_bar, 8); tc::mbar_init(merge_done, 8);
         *abort_flag = 0;
         tc::fence_barrier_init();
         tc::fence_proxy_async();
@@ -297,6 +308,10 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     tc::grid_dep_wait();   // work list, q/k/v rows and the cache rows of the new tokens come from earlier kernels
     // tensor-memory columns of group g (base g*256): S_g 0..63, P_g 64..95, the first 64 head-dim columns of Q_g as
     // bf16 pairs 96..127, O_g 128..255
+    // A work item with more than 128 / G tokens gives each group its own 128 score rows, and each group takes both
+    // 64-key halves of every key tile.  A SHARED item (at most 128 / G tokens: a short suffix) has score rows for
+    // one group only; both groups then hold the same rows, group g takes half g of every key tile, and the two
+    // partial results (both in tensor memory) are merged when the item's last P V has completed.
     const int tok_per_group = 128 / a.G;
     // K/V stage layout.  One TMA box ("unit") brings box_rows cache rows of one page, both 64-wide halves of the
     // head dim: [half][box_rows][128 bytes], 128-byte swizzle inside each half block.  A stage holds the 128 / box_rows
@@ -313,56 +328,66 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
     const uint32_t sbo = a.box_rows == 64 ? 1024u : unit_bytes;
     const uint32_t half_off = a.box_rows == 16 ? 1024u : (a.box_rows == 8 ? 8u * unit_bytes : unit_bytes);
 
-    if (warp == 8) {
-        // ------------------------------ TMA producer (whole warp) ------------------------------
+    if (warp == 8 || warp == 11) {
+        // ------------------------------ TMA producers (whole warps): warp 8 for Q and K, warp 11 for V ------------------------------
+        // One box per unit of a tile, each issued by the lane that looked its page up.  A warp's copies of one tile
+        // are issued one after the other (about 70 cycles each), and a page lookup is a dependent load from global
+        // memory (about 1000 cycles): so K and V have a warp each, and the lookup of tile j + 1 is in flight
+        // underneath the copies of tile j.
+        const int plane = warp == 8 ? 0 : 1;
         uint32_t n_item = 0, kt = 0;
         bool ok = true;
         Iter run(a);
         RunPiece pc;
         for (; ok && run.next(a, pc); ++n_item) {
             const AttnWork &w = pc.w;
-            if (lane == 0) {
-                ok = tc::mbar_wait(q_free, (n_item & 1) ^ 1, abort_flag);
-                if (ok) {
-                    if (kHalves > 1) {
-                        tc::mbar_arrive_expect_tx(q_full, 2 * S::kQBytes);
-                        for (int g = 0; g < 2; ++g)
-                            for (int h = 1; h < kHalves; ++h)
-                                tma_load_3d(smem_base + S::kQOff + g * S::kQBytes + (h - 1) * kHalfQ, &tmQ, q_full, h * 64,
-                                            w.kv_head * a.G, w.q_start + g * tok_per_group);
-                    } else {
-                        tc::mbar_arrive(q_full);   // nothing of Q goes through shared memory at this head dim
+            if (plane == 0) {
+                if (lane == 0) {
+                    ok = tc::mbar_wait(q_free, (n_item & 1) ^ 1, abort_flag);
+                    if (ok) {
+                        if (kHalves > 1) {
+                            tc::mbar_arrive_expect_tx(q_full, 2 * S::kQBytes);
+                            for (int g = 0; g < 2; ++g)
+                                for (int h = 1; h < kHalves; ++h)
+                                    tma_load_3d(smem_base + S::kQOff + g * S::kQBytes + (h - 1) * kHalfQ, &tmQ, q_full, h * 64,
+                                                w.kv_head * a.G, w.q_start + (w.q_count <= tok_per_group ? 0 : g * tok_per_group));
+                        } else {
+                            tc::mbar_arrive(q_full);   // nothing of Q goes through shared memory at this head dim
+                        }
                     }
                 }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
             }
-            ok = __shfl_sync(0xffffffffu, ok, 0);
-            for (int j = pc.t0; j < pc.t1 && ok; ++j, ++kt) {
-                const int st = kt % kKvStages;
-                const uint32_t par = ((kt / kKvStages) & 1) ^ 1;
+            // page of this lane's unit of tile j (-2: the tile has no such unit); only loaded here, looked at later
+            auto page_of = [&](int j) {
                 const int kbase = j * kKeysPerTile;
                 const int n_units = min(units_per_tile, (w.kv_end - kbase + a.box_rows - 1) / a.box_rows);
-                // every lane looks up the page of one unit of the tile
+                return lane < n_units ? a.block_tables[(size_t)w.req * a.max_blocks + (kbase + lane * a.box_rows) / a.page_size] : -2;
+            };
+            int page = page_of(pc.t0);
+            for (int j = pc.t0; j < pc.t1 && ok; ++j, ++kt) {
+                const int page_next = j + 1 < pc.t1 ? page_of(j + 1) : -2;
+                const int st = kt % kKvStages;
+                const uint32_t par = ((kt / kKvStages) & 1) ^ 1;
                 int row = -1;
-                if (lane < n_units) {
-                    const int key = kbase + lane * a.box_rows;
-                    const int page = a.block_tables[(size_t)w.req * a.max_blocks + key / a.page_size];
+                if (page != -2) {
+                    const int key = j * kKeysPerTile + lane * a.box_rows;
                     if (page < 0 || page >= a.num_pages) report(a.status, ALORA_ERR_PAGE_RANGE);
-                    else row = (page * 2 * a.Hkv + w.kv_head) * a.page_size + key % a.page_size;   // K plane
+                    else row = ((page * 2 + plane) * a.Hkv + w.kv_head) * a.page_size + key % a.page_size;
                 }
                 const unsigned valid = __ballot_sync(0xffffffffu, row >= 0);
                 const uint32_t bytes = (uint32_t)__popc(valid) * unit_bytes;
-                for (int plane = 0; plane < 2 && ok; ++plane) {
-                    const uint32_t fullb = plane == 0 ? k_full(st) : v_full(st);
-                    const uint32_t freeb = plane == 0 ? k_free(st) : v_free(st);
-                    if (lane == 0) {
-                        ok = tc::mbar_wait(freeb, par, abort_flag);
-                        if (ok) tc::mbar_arrive_expect_tx(fullb, bytes);
-                    }
-                    ok = __shfl_sync(0xffffffffu, ok, 0);
-                    if (ok && row >= 0)   // one box: both halves of the head dim
-                        tma_load_3d(smem_base + (plane == 0 ? S::kKOff : S::kVOff) + st * S::kKvBytes + lane * unit_bytes,
-                                    &tmKV, fullb, 0, row + plane * a.Hkv * a.page_size, 0);
+                const uint32_t fullb = plane == 0 ? k_full(st) : v_full(st);
+                const uint32_t freeb = plane == 0 ? k_free(st) : v_free(st);
+                if (lane == 0) {
+                    ok = tc::mbar_wait(freeb, par, abort_flag);
+                    if (ok) tc::mbar_arrive_expect_tx(fullb, bytes);
                 }
+                ok = __shfl_sync(0xffffffffu, ok, 0);
+                if (ok && row >= 0)   // one box: both halves of the head dim
+                    tma_load_3d(smem_base + (plane == 0 ? S::kKOff : S::kVOff) + st * S::kKvBytes + lane * unit_bytes,
+                                &tmKV, fullb, 0, row, 0);
+                page = page_next;
             }
         }
         (void)ok;
@@ -379,7 +404,6 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         constexpr uint32_t idesc_s = tc::idesc_bf16_f32(128, kHalfKeys);
         constexpr uint32_t idesc_pv = idesc_bf16_f32_bmn(128, HD);
         uint32_t n_item = 0, kt = 0, nh = 0;   // nh: half tiles handled so far (phase counter of the group's barriers)
-        uint32_t n_act = 0;                     // items in which this group had rows (phase counter of q_ready)
         bool ok = true;
         const uint32_t qa = smem_base + S::kQOff + g * S::kQBytes;
         const uint32_t s_tmem = tmem_base + g * 256, p_tmem = s_tmem + 64, q_tmem = s_tmem + 96, o_tmem = s_tmem + 128;
@@ -406,44 +430,33 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         Iter run(a);
         RunPiece pc;
         for (; ok && run.next(a, pc); ++n_item) {
-            const int n_half = 2 * (pc.t1 - pc.t0);   // both halves of every tile of the piece
+            const bool shared = pc.w.q_count <= tok_per_group;
+            const int n_steps = (pc.t1 - pc.t0) << (shared ? 0 : 1);   // half tiles of this group in the piece
             if (!wait_all(q_full, n_item & 1)) { ok = false; break; }
-            if (g == 1 && pc.w.q_count <= tok_per_group) {
-                // A short block of tokens: all its score rows are in group 0.  This group's issuer only hands the
-                // piece's K/V stages and Q back (each after it has been filled, so that it never runs ahead of the
-                // producer by a whole phase), and the group's softmax warps skip the piece.
-                for (int j = pc.t0; j < pc.t1 && ok; ++j, ++kt) {
-                    const int st = kt % kKvStages;
-                    const uint32_t par = (kt / kKvStages) & 1;
-                    if (!wait_all(k_full(st), par)) { ok = false; break; }
-                    if (leader) tc::mbar_arrive(k_free(st));
-                    if (!wait_all(v_full(st), par)) { ok = false; break; }
-                    if (leader) tc::mbar_arrive(v_free(st));
-                }
-                if (ok && leader) tc::mbar_arrive(q_free);
-                continue;
-            }
-            if (!wait_all(q_ready(g), n_act & 1)) { ok = false; break; }
-            ++n_act;
+            if (!wait_all(q_ready(g), n_item & 1)) { ok = false; break; }
             if (!wait_all(k_full(kt % kKvStages), (kt / kKvStages) & 1)) { ok = false; break; }
             tc::tc_fence_after();
-            issue_s(kt % kKvStages, 0);
-            for (int i = 0; i < n_half && ok; ++i) {
-                const int st = kt % kKvStages;          // stage of half i
-                const int hh = i & 1;
-                // ---- scores of half i + 1
-                if (i + 1 < n_half) {
-                    const int st1 = hh ? (kt + 1) % kKvStages : st;
-                    if (hh && !wait_all(k_full(st1), ((kt + 1) / kKvStages) & 1)) { ok = false; break; }
+            issue_s(kt % kKvStages, shared ? g : 0);
+            // this group is done with a K tile once its last half of it has been issued, and with Q at the end
+            if (leader && shared) tc::mma_commit(k_free(kt % kKvStages));
+            if (leader && n_steps == 1) tc::mma_commit(q_free);
+            for (int i = 0; i < n_steps && ok; ++i) {
+                const int st = kt % kKvStages;          // stage of step i
+                const int hh = shared ? g : (i & 1);    // its half of the tile
+                const bool tile_end = shared || hh == 1;
+                // ---- scores of step i + 1
+                if (i + 1 < n_steps) {
+                    const int st1 = tile_end ? (kt + 1) % kKvStages : st;
+                    if (tile_end && !wait_all(k_full(st1), ((kt + 1) / kKvStages) & 1)) { ok = false; break; }
                     if (!wait_all(s_free(g), nh & 1)) { ok = false; break; }
                     tc::tc_fence_after();
-                    issue_s(st1, hh ^ 1);
-                    // this group is done with the K tile once its second half has been issued (and with Q at the end)
-                    if (leader && hh == 0) tc::mma_commit(k_free(st1));
-                    if (leader && i + 2 == n_half) tc::mma_commit(q_free);
+                    const int hh1 = shared ? g : (hh ^ 1);
+                    issue_s(st1, hh1);
+                    if (leader && (shared || hh1 == 1)) tc::mma_commit(k_free(st1));
+                    if (leader && i + 2 == n_steps) tc::mma_commit(q_free);
                 }
-                // ---- P V of half i
-                if (hh == 0 && !wait_all(v_full(st), (kt / kKvStages) & 1)) { ok = false; break; }
+                // ---- P V of step i
+                if ((shared || hh == 0) && !wait_all(v_full(st), (kt / kKvStages) & 1)) { ok = false; break; }
                 if (!wait_all(p_ready(g), nh & 1)) { ok = false; break; }
                 ++nh;
                 tc::tc_fence_after();
@@ -454,9 +467,9 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         mma_bf16_ts(o_tmem, p_tmem + 8 * k, smem_desc_mn_sw128(va + 2 * k * sbo, hstride, sbo), idesc_pv,
                                     (i | k) != 0 ? 1u : 0u);
                     tc::mma_commit(pv_done(g));
-                    if (hh == 1) tc::mma_commit(v_free(st));
+                    if (tile_end) tc::mma_commit(v_free(st));
                 }
-                if (hh == 1) ++kt;
+                if (tile_end) ++kt;
             }
         }
         // tensor-core work still in flight must finish before tensor memory is released
@@ -465,8 +478,10 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             const long long t0 = clock64();
             while (!tc::mbar_try_wait(drain_bar(g), 0) && clock64() - t0 < tc::kWaitCycleLimit) {}
         }
-    } else {
+    } else if (warp < 8) {
         // ------------------------------ softmax groups (warps 0..7) ------------------------------
+        // (warps q and 4 + q own the same quarter of the tensor-memory lanes, so a thread can read the other
+        // group's accumulator rows of its own row index: that is how the two parts of a shared item are merged)
         const int g = warp >> 2;                 // group 0 / 1
         const int q = warp & 3;                  // tensor-memory lane quarter
         const int row = q * 32 + lane;           // score row of this thread inside the group's tile
@@ -475,14 +490,20 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const uint32_t p_addr = s_addr + 64;                              // probabilities, bf16 pairs (32 columns)
         const uint32_t q_addr = s_addr + 96;                              // first 64 head-dim columns of this Q row
         const uint32_t o_addr = s_addr + 128;
+        const uint32_t o_other = tmem_base + (g ^ 1) * 256 + lane_off + 128;   // the other group's O, same rows
+        const uint32_t ml_addr = s_addr + 64, ml_other = tmem_base + (g ^ 1) * 256 + lane_off + 64;
         uint32_t n_s = 0, kt = 0;   // n_s: half tiles of this group so far (phase counter of its barriers)
+        uint32_t n_merge = 0;       // shared items so far (phase counter of the merge barriers)
+        bool merge_pending = false; // the other group may still be reading this group's part of a shared item
         bool ok = true;
         Iter run(a);
         RunPiece pc, pc_next;
-        const int tok_local = g * tok_per_group + row / a.G;
+        // first token of this group's rows inside an item (a shared item: both groups hold the same rows)
+        auto tok_base = [&](const AttnWork &w) { return w.q_count <= tok_per_group ? 0 : g * tok_per_group; };
         // the first 64 head-dim columns of this thread's row of Q of a piece: global memory -> registers
         uint32_t qv[32];
         auto load_q = [&](const AttnWork &w) {
+            const int tok_local = tok_base(w) + row / a.G;
             const bool valid = tok_local < w.q_count;
             const uint4 *src = reinterpret_cast<const uint4 *>(
                 a.qkv + (size_t)(w.q_start + (valid ? tok_local : 0)) * a.N + (size_t)(w.kv_head * a.G + row % a.G) * HD);
@@ -501,28 +522,22 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             __syncwarp();
             if (lane == 0) tc::mbar_arrive(q_ready(g));
         };
-        // the next piece in which this group has rows (a short block of tokens has none in group 1); the key tiles of
-        // the pieces passed over still count for the position in the K/V ring
-        auto next_piece = [&](RunPiece &p) {
-            while (run.next(a, p)) {
-                if (!(g == 1 && p.w.q_count <= tok_per_group)) return true;
-                kt += p.t1 - p.t0;
-            }
-            return false;
-        };
-        bool have = next_piece(pc);
+        bool have = run.next(a, pc);
         if (have) { load_q(pc.w); publish_q(); }
         while (ok && have) {
             const AttnWork &w = pc.w;
-            const int n_half = 2 * (pc.t1 - pc.t0);
+            const bool shared = w.q_count <= tok_per_group;
+            const int n_half = (pc.t1 - pc.t0) << (shared ? 0 : 1);   // half tiles of this group in the piece
+            const int tok_local = tok_base(w) + row / a.G;
             // position of this row's token; rows past the end of the block behave like its last token
             const int pos = w.kv_end - w.q_count + min(tok_local, w.q_count - 1);
             // exponent reference (a running maximum that is only moved when it has drifted by more than
             // 2^8, so the accumulator in tensor memory rarely needs rescaling) and row sum
             float m_ref = -INFINITY, l_run = 0.f;
             for (int i = 0; i < n_half && ok; ++i, ++n_s) {
-                const int tbase = (pc.t0 + (i >> 1)) * kKeysPerTile;   // first key of the tile; column e of half hh is key
-                const int hh = i & 1;                        // tbase + (perm ? (e/8)*16 + hh*8 + e%8 : hh*64 + e)
+                const int tbase = (pc.t0 + (shared ? i : i >> 1)) * kKeysPerTile;   // first key of the tile; column e of half hh
+                const int hh = shared ? g : (i & 1);         // is key tbase + (perm ? (e/8)*16 + hh*8 + e%8 : hh*64 + e)
+                const bool tile_begin = shared || hh == 0;   // this group's first half of the tile
                 if (!tc::mbar_wait(s_full(g), n_s & 1, abort_flag)) { ok = false; break; }
                 tc::tc_fence_after();
                 uint32_t sv[kHalfKeys];
@@ -618,12 +633,19 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                         }
                     }
                 }
+                if (merge_pending) {
+                    // the previous (shared) item: its exponent reference and row sum sit in two columns of P_g, and
+                    // its O_g is overwritten by this item's first P V; the other group must have read both
+                    if (!tc::mbar_wait(merge_done, (n_merge - 1) & 1, abort_flag)) { ok = false; break; }
+                    tc::tc_fence_after();
+                    merge_pending = false;
+                }
                 tmem_st_32x16(p_addr, reinterpret_cast<uint32_t(&)[16]>(pk[0]));
                 tmem_st_32x16(p_addr + 16, reinterpret_cast<uint32_t(&)[16]>(pk[16]));
                 // V rows of keys at or beyond the item's causal limit are cleared before the tile's first P V uses them
                 // (thread `row` of each group clears key tbase + row)
-                if (hh == 0) kt += (i > 0);   // tile index of this half
-                if (hh == 0 && tbase + kKeysPerTile > w.kv_end) {
+                if (tile_begin) kt += (i > 0);   // tile index of this half
+                if (tile_begin && tbase + kKeysPerTile > w.kv_end) {
                     const int st = kt % kKvStages;
                     if (!tc::mbar_wait(v_full(st), (kt / kKvStages) & 1, abort_flag)) { ok = false; break; }
                     if (tbase + row >= w.kv_end) {
@@ -645,7 +667,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             if (!ok) break;
             // the next item's rows of Q go to tensor memory underneath this item's last P V, so that its first
             // Q K^T runs underneath this item's output
-            const bool have_next = next_piece(pc_next);
+            const bool have_next = run.next(a, pc_next);
             if (have_next) { load_q(pc_next.w); publish_q(); }
             // the item's last P V, normalisation, store
             if (!tc::mbar_wait(pv_done(g), (n_s - 1) & 1, abort_flag)) { ok = false; break; }
@@ -658,7 +680,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 #pragma unroll
             for (int j = 0; j < 4; ++j) {
                 const int r = (row & ~3) + j;
-                const int tl = g * tok_per_group + r / a.G;
+                const int tl = tok_base(w) + r / a.G;
                 dst_quad[j] = tl < w.q_count
                                   ? a.out + (size_t)(w.q_start + tl) * a.Nq + (size_t)(w.kv_head * a.G + r % a.G) * HD + ql * 8
                                   : nullptr;
@@ -675,7 +697,60 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 for (int j = 0; j < 4; ++j)
                     if (dst_quad[j]) *reinterpret_cast<uint4 *>(dst_quad[j] + c) = u[j];
             };
-            if (!kRuns || pc.n_parts == 1) {
+            if (shared) {
+                // Both groups hold a partial result for the same rows (over different halves of the key tiles).  Each
+                // thread puts its exponent reference and row sum next to its O_g in tensor memory, then both groups
+                // read both parts; group g normalises and stores half g of the head-dim columns.
+                tmem_st_32x2(ml_addr, __float_as_uint(m_ref), __float_as_uint(l_run));
+                tmem_st_wait();
+                tc::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(merge_bar);
+                if (!tc::mbar_wait(merge_bar, n_merge & 1, abort_flag)) { ok = false; break; }
+                ++n_merge;
+                tc::tc_fence_after();
+                uint32_t mo, lo;
+                tmem_ld_32x2(ml_other, mo, lo);
+                tc::tmem_ld_wait();
+                const float m_oth = __uint_as_float(mo), l_oth = __uint_as_float(lo);
+                const float m_all = fmaxf(m_ref, m_oth);   // (finite: the row's own position is in one of the halves)
+                const float w_own = m_ref == -INFINITY ? 0.f : fast_exp2((m_ref - m_all) * a.scale_log2);
+                const float w_oth = m_oth == -INFINITY ? 0.f : fast_exp2((m_oth - m_all) * a.scale_log2);
+                const float l_all = fmaf(l_run, w_own, l_oth * w_oth);
+                const bool whole = !kRuns || pc.n_parts == 1;
+                const float inv = whole ? 1.f / l_all : 1.f;
+                // part of a cut item: the merged, unnormalised rows go to the part's slot as rows of group 0
+                float *po = a.part_o, *pml = a.part_ml;
+                if (kRuns && !whole) {
+                    po += (size_t)part_slot(pc.c_first, pc.part) * HD * 256 + row;
+                    pml += (size_t)part_slot(pc.c_first, pc.part) * 512 + row;
+                }
+#pragma unroll 1
+                for (int c = g * (HD / 2); c < (g + 1) * (HD / 2); c += 32) {
+                    uint32_t v[32], u[32];
+                    tc::tmem_ld_32x32(o_addr + c, v);
+                    tc::tmem_ld_32x32(o_other + c, u);
+                    tc::tmem_ld_wait();
+                    float o[32];
+#pragma unroll
+                    for (int e = 0; e < 32; ++e)
+                        o[e] = fmaf(__uint_as_float(v[e]), w_own, __uint_as_float(u[e]) * w_oth) * inv;
+                    if (whole) {
+                        store_chunk(c, o);
+                    } else {
+#pragma unroll
+                        for (int e = 0; e < 32; ++e) po[(size_t)(c + e) * 256] = o[e];
+                    }
+                }
+                if (kRuns && !whole && g == 0) {
+                    pml[0] = m_all;
+                    pml[256] = l_all;
+                }
+                tc::tc_fence_before();
+                __syncwarp();
+                if (lane == 0) tc::mbar_arrive(merge_done);
+                merge_pending = true;
+            } else if (!kRuns || pc.n_parts == 1) {
                 const float inv = 1.f / l_run;
 #pragma unroll 1
                 for (int c = 0; c < HD; c += 32) {
