@@ -330,10 +330,10 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 
     if (warp == 8 || warp == 11) {
         // ------------------------------ TMA producers (whole warps): warp 8 for Q and K, warp 11 for V ------------------------------
-        // One box per unit of a tile, each issued by the lane that looked its page up.  A warp's copies of one tile
-        // are issued one after the other (about 70 cycles each), and a page lookup is a dependent load from global
-        // memory (about 1000 cycles): so K and V have a warp each, and the lookup of tile j + 1 is in flight
-        // underneath the copies of tile j.
+        // One box per unit of a tile, each issued by the lane that holds its page.  A warp's copies of one tile are
+        // issued one after the other (about 70 cycles each), and a block-table entry is a dependent load from global
+        // memory (1000 cycles and more): so K and V have a warp each, and the table is read 32 entries at a time,
+        // one window ahead.
         const int plane = warp == 8 ? 0 : 1;
         uint32_t n_item = 0, kt = 0;
         bool ok = true;
@@ -358,20 +358,27 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
             }
-            // page of this lane's unit of tile j (-2: the tile has no such unit); only loaded here, looked at later
-            auto page_of = [&](int j) {
-                const int kbase = j * kKeysPerTile;
-                const int n_units = min(units_per_tile, (w.kv_end - kbase + a.box_rows - 1) / a.box_rows);
-                return lane < n_units ? a.block_tables[(size_t)w.req * a.max_blocks + (kbase + lane * a.box_rows) / a.page_size] : -2;
-            };
-            int page = page_of(pc.t0);
+            // Window of the request's block-table row: lane l holds entry win0 + l (win0 a multiple of 32; 32 entries
+            // cover a whole number of key tiles), the following window is in flight while this one is used.
+            const int32_t *bt_row = a.block_tables + (size_t)w.req * a.max_blocks;
+            auto load_window = [&](int w0) { return w0 + lane < a.max_blocks ? bt_row[w0 + lane] : -1; };
+            int win0 = (pc.t0 * kKeysPerTile / a.page_size) & ~31;
+            int win = load_window(win0), win_next = load_window(win0 + 32);
             for (int j = pc.t0; j < pc.t1 && ok; ++j, ++kt) {
-                const int page_next = j + 1 < pc.t1 ? page_of(j + 1) : -2;
+                const int kbase = j * kKeysPerTile;
+                if (kbase / a.page_size >= win0 + 32) {
+                    win0 += 32;
+                    win = win_next;
+                    win_next = load_window(win0 + 32);
+                }
                 const int st = kt % kKvStages;
                 const uint32_t par = ((kt / kKvStages) & 1) ^ 1;
+                // this lane's unit of the tile, if the tile has that many
+                const int n_units = min(units_per_tile, (w.kv_end - kbase + a.box_rows - 1) / a.box_rows);
+                const int page = __shfl_sync(0xffffffffu, win, ((kbase + lane * a.box_rows) / a.page_size - win0) & 31);
                 int row = -1;
-                if (page != -2) {
-                    const int key = j * kKeysPerTile + lane * a.box_rows;
+                if (lane < n_units) {
+                    const int key = kbase + lane * a.box_rows;
                     if (page < 0 || page >= a.num_pages) report(a.status, ALORA_ERR_PAGE_RANGE);
                     else row = ((page * 2 + plane) * a.Hkv + w.kv_head) * a.page_size + key % a.page_size;
                 }
@@ -387,7 +394,6 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 if (ok && row >= 0)   // one box: both halves of the head dim
                     tma_load_3d(smem_base + (plane == 0 ? S::kKOff : S::kVOff) + st * S::kKvBytes + lane * unit_bytes,
                                 &tmKV, fullb, 0, row, 0);
-                page = page_next;
             }
         }
         (void)ok;
@@ -494,7 +500,6 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         const uint32_t ml_addr = s_addr + 64, ml_other = tmem_base + (g ^ 1) * 256 + lane_off + 64;
         uint32_t n_s = 0, kt = 0;   // n_s: half tiles of this group so far (phase counter of its barriers)
         uint32_t n_merge = 0;       // shared items so far (phase counter of the merge barriers)
-        bool merge_pending = false; // the other group may still be reading this group's part of a shared item
         bool ok = true;
         Iter run(a);
         RunPiece pc, pc_next;
@@ -527,7 +532,9 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
         while (ok && have) {
             const AttnWork &w = pc.w;
             const bool shared = w.q_count <= tok_per_group;
-            const int n_half = (pc.t1 - pc.t0) << (shared ? 0 : 1);   // half tiles of this group in the piece
+            // step i of the group works on half (i & step_sh) | half0 of tile t0 + (i >> step_sh)
+            const int step_sh = shared ? 0 : 1, half0 = shared ? g : 0;
+            const int n_half = (pc.t1 - pc.t0) << step_sh;   // half tiles of this group in the piece
             const int tok_local = tok_base(w) + row / a.G;
             // position of this row's token; rows past the end of the block behave like its last token
             const int pos = w.kv_end - w.q_count + min(tok_local, w.q_count - 1);
@@ -535,9 +542,9 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             // 2^8, so the accumulator in tensor memory rarely needs rescaling) and row sum
             float m_ref = -INFINITY, l_run = 0.f;
             for (int i = 0; i < n_half && ok; ++i, ++n_s) {
-                const int tbase = (pc.t0 + (shared ? i : i >> 1)) * kKeysPerTile;   // first key of the tile; column e of half hh
-                const int hh = shared ? g : (i & 1);         // is key tbase + (perm ? (e/8)*16 + hh*8 + e%8 : hh*64 + e)
-                const bool tile_begin = shared || hh == 0;   // this group's first half of the tile
+                const int tbase = (pc.t0 + (i >> step_sh)) * kKeysPerTile;   // first key of the tile; column e of half hh
+                const int hh = (i & step_sh) | half0;        // is key tbase + (perm ? (e/8)*16 + hh*8 + e%8 : hh*64 + e)
+                const bool tile_begin = hh == half0;         // this group's first half of the tile
                 if (!tc::mbar_wait(s_full(g), n_s & 1, abort_flag)) { ok = false; break; }
                 tc::tc_fence_after();
                 uint32_t sv[kHalfKeys];
@@ -632,13 +639,6 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                             tmem_st_32x32(o_addr + c, v);
                         }
                     }
-                }
-                if (merge_pending) {
-                    // the previous (shared) item: its exponent reference and row sum sit in two columns of P_g, and
-                    // its O_g is overwritten by this item's first P V; the other group must have read both
-                    if (!tc::mbar_wait(merge_done, (n_merge - 1) & 1, abort_flag)) { ok = false; break; }
-                    tc::tc_fence_after();
-                    merge_pending = false;
                 }
                 tmem_st_32x16(p_addr, reinterpret_cast<uint32_t(&)[16]>(pk[0]));
                 tmem_st_32x16(p_addr + 16, reinterpret_cast<uint32_t(&)[16]>(pk[16]));
@@ -749,7 +749,10 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 tc::tc_fence_before();
                 __syncwarp();
                 if (lane == 0) tc::mbar_arrive(merge_done);
-                merge_pending = true;
+                // the reference and sum sit in two columns of P_g and O_g is overwritten by the next item's first
+                // P V: the other group must have read both before this group goes on
+                if (!tc::mbar_wait(merge_done, (n_merge - 1) & 1, abort_flag)) { ok = false; break; }
+                tc::tc_fence_after();
             } else if (!kRuns || pc.n_parts == 1) {
                 const float inv = 1.f / l_run;
 #pragma unroll 1
