@@ -343,7 +343,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
             const AttnWork &w = pc.w;
             if (plane == 0) {
                 if (lane == 0) {
-                    ok = tc::mbar_wait(q_free, (n_item & 1) ^ 1, abort_flag);
+                    ok = tc::mbar_wait_relaxed(q_free, (n_item & 1) ^ 1, abort_flag);
                     if (ok) {
                         if (kHalves > 1) {
                             tc::mbar_arrive_expect_tx(q_full, 2 * S::kQBytes);
@@ -387,7 +387,7 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
                 const uint32_t fullb = plane == 0 ? k_full(st) : v_full(st);
                 const uint32_t freeb = plane == 0 ? k_free(st) : v_free(st);
                 if (lane == 0) {
-                    ok = tc::mbar_wait(freeb, par, abort_flag);
+                    ok = tc::mbar_wait_relaxed(freeb, par, abort_flag);
                     if (ok) tc::mbar_arrive_expect_tx(fullb, bytes);
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);

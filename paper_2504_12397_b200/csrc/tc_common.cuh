@@ -74,6 +74,22 @@ __device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatil
     }
 }
 
+// The same bounded wait for a warp whose reaction time does not matter (a producer several ring slots ahead of
+// its consumers): it sleeps between polls, leaving the issue slots of its scheduler to the warps that compute.
+__device__ __forceinline__ bool mbar_wait_relaxed(uint32_t bar, uint32_t parity, volatile int *abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (true) {
+        __nanosleep(200);
+        if (mbar_try_wait(bar, parity)) return true;
+        if (*abort_flag) return false;
+        if (clock64() - t0 > kWaitCycleLimit) {
+            *abort_flag = 1;
+            return false;
+        }
+    }
+}
+
 // 2-D TMA tile load global -> shared, completion counted on an mbarrier.  c0 is the innermost
 // coordinate (elements); c0 * element size must be a multiple of 16 bytes.
 __device__ __forceinline__ void tma_load_2d(uint32_t smem_dst, const CUtensorMap *map, uint32_t bar, int c0, int c1) {
