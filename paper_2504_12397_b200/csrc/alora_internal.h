@@ -60,6 +60,7 @@ constexpr int kAttnKeysPerTile = 128;   // keys per K/V tile of the tensor-core 
 constexpr int kAttnMinRunTiles = 8;     // shortest run of key tiles given to one block
 constexpr int kAttnCutMinTiles = 128;   // items are cut into runs only when a block has at least this many tiles to do
 constexpr int kAttnCutMinWaves = 3;     // ... and the items make at least this many full rounds over the blocks
+constexpr int kAttnSpreadMinGain = 24; // fewer items than blocks: spread them only if the longest item is this many tiles longer than a block's run
 
 // One unit of few-row (decode / short suffix) attention work: score rows of `q_count` tokens starting at
 // flat token q_start (rows are (token, query head of the group) pairs, `mt` tiles of 16 rows), one KV

@@ -798,10 +798,10 @@ attn_tcgen05_kernel(const __grid_constant__ CUtensorMap tmQ, const __grid_consta
 }
 
 
-// Merge of the parts of the cut items.  Blocks 2 * (c - 1) + g, c = 1 .. runs - 1: if run boundary c falls
-// strictly inside an item and is the first boundary inside it, the block merges the rows of group g of that
-// item: O = sum_p 2^((m_p - m) scale) O_p / sum_p 2^((m_p - m) scale) l_p, m = max_p m_p, parts in order.
-// Thread = (row, quarter of the head dim).
+// Merge of the parts of the cut items.  Blocks (2 * (c - 1) + g, j), c = 1 .. runs - 1, j = 0 .. 3: if run boundary c
+// falls strictly inside an item and is the first boundary inside it, the four blocks j merge the rows of group g of
+// that item: O = sum_p 2^((m_p - m) scale) O_p / sum_p 2^((m_p - m) scale) l_p, m = max_p m_p, parts in order.
+// Thread = (row, sixteenth of the head dim): block j holds quarter j of the columns.
 template <int HD>
 __global__ void __launch_bounds__(512) attn_merge_kernel(const AttnArgs a) {
     tc::grid_dep_launch();
@@ -816,34 +816,36 @@ __global__ void __launch_bounds__(512) attn_merge_kernel(const AttnArgs a) {
     const int n_parts = (first + n_tiles - 1) / len - c_first + 1;
     if (first == c * len || c != c_first + 1) return;   // boundary not inside the item / not its first boundary
     if (g == 1 && w.q_count <= 128 / a.G) return;       // no rows of the item in this group
-    const int row = threadIdx.x & 127, quarter = threadIdx.x >> 7, grow = g * 128 + row;
-    constexpr int kCols = HD / 4;
-    const int col0 = quarter * kCols;
+    const int row = threadIdx.x & 127, grow = g * 128 + row;
+    constexpr int kCols = HD / 16;
+    const int col0 = ((int)blockIdx.y * 4 + (int)(threadIdx.x >> 7)) * kCols;
     const int tl = g * (128 / a.G) + row / a.G;
+    if (tl >= w.q_count) return;
+    const float *__restrict__ ml = a.part_ml + grow;
+    const float *__restrict__ po = a.part_o + (size_t)col0 * 256 + grow;
     float m_all = -INFINITY;
-    for (int p = 0; p < n_parts; ++p) m_all = fmaxf(m_all, a.part_ml[(size_t)part_slot(c_first, p) * 512 + grow]);
+#pragma unroll 4
+    for (int p = 0; p < n_parts; ++p) m_all = fmaxf(m_all, ml[(size_t)part_slot(c_first, p) * 512]);
     float l_all = 0.f, acc[kCols];
 #pragma unroll
     for (int e = 0; e < kCols; ++e) acc[e] = 0.f;
+#pragma unroll 4
     for (int p = 0; p < n_parts; ++p) {
         const int slot = part_slot(c_first, p);
-        const float m_p = a.part_ml[(size_t)slot * 512 + grow];
+        const float m_p = ml[(size_t)slot * 512];
         const float wgt = m_p == -INFINITY ? 0.f : exp2f((m_p - m_all) * a.scale_log2);
-        l_all = fmaf(a.part_ml[(size_t)slot * 512 + 256 + grow], wgt, l_all);
-        const float *src = a.part_o + ((size_t)slot * HD + col0) * 256 + grow;
+        l_all = fmaf(ml[(size_t)slot * 512 + 256], wgt, l_all);
+        const float *src = po + (size_t)slot * HD * 256;
 #pragma unroll
         for (int e = 0; e < kCols; ++e) acc[e] = fmaf(src[(size_t)e * 256], wgt, acc[e]);
     }
-    if (tl >= w.q_count) return;
     const float inv = 1.f / l_all;
     __nv_bfloat16 *dst = a.out + (size_t)(w.q_start + tl) * a.Nq + (size_t)(w.kv_head * a.G + row % a.G) * HD + col0;
+    uint32_t u[kCols / 2];
 #pragma unroll
-    for (int x = 0; x < kCols / 8; ++x) {
-        uint4 u;
-        u.x = tc::pack_bf16(acc[8 * x] * inv, acc[8 * x + 1] * inv); u.y = tc::pack_bf16(acc[8 * x + 2] * inv, acc[8 * x + 3] * inv);
-        u.z = tc::pack_bf16(acc[8 * x + 4] * inv, acc[8 * x + 5] * inv); u.w = tc::pack_bf16(acc[8 * x + 6] * inv, acc[8 * x + 7] * inv);
-        reinterpret_cast<uint4 *>(dst)[x] = u;
-    }
+    for (int x = 0; x < kCols / 2; ++x) u[x] = tc::pack_bf16(acc[2 * x] * inv, acc[2 * x + 1] * inv);
+    if constexpr (kCols == 8) *reinterpret_cast<uint4 *>(dst) = make_uint4(u[0], u[1], u[2], u[3]);
+    else *reinterpret_cast<uint2 *>(dst) = make_uint2(u[0], u[1]);
 }
 
 typedef CUresult (*EncodeTiledFn)(CUtensorMap *, CUtensorMapDataType, cuuint32_t, void *, const cuuint64_t *,
@@ -918,15 +920,21 @@ static int launch_attend_long(alora_ctx *ctx, const void *qkv, const BatchArgs &
     a.run_counts = ctx->d_counts + 6; a.cta_start = ctx->d_attn_cta_start;
     a.part_o = ctx->d_attn_part_o; a.part_ml = ctx->d_attn_part_ml;
     const int max_items = (b.T / ctx->attn_q_block + b.R) * d.Hkv;
-    const int grid = std::max(1, std::min(ctx->sm_count, max_items));
     ProfScope prof(ctx, KK_ATTENTION, s);
     static bool attr_set[2][64] = {};
     const int dev = ctx->cfg.device, hi = d.hd == 128;
     // Items are cut into runs (and need the merge kernel) only when the batch has at least kAttnCutMinTiles key tiles
     // per block and kAttnCutMinWaves items per block; upper bounds from what the host knows decide whether that
     // can be the case.
+    // A batch that cannot have more items than there are SMs is cut too if its items can be long enough to give
+    // every block a run of kAttnMinRunTiles key tiles (a few requests with long contexts); the work-list builder, which
+    // knows the lengths, has the last word in both cases.
+    const int n_sm = ctx->sm_count;
     const long long max_tiles = (long long)max_items * (((long long)b.max_blocks * d.page + kKeysPerTile - 1) / kKeysPerTile);
-    const bool runs = grid > 1 && max_tiles >= (long long)kAttnCutMinTiles * grid && max_items >= kAttnCutMinWaves * grid;
+    const bool long_batch = max_tiles >= (long long)kAttnCutMinTiles * n_sm && max_items >= kAttnCutMinWaves * n_sm;
+    const bool few_items = max_items < n_sm && max_tiles >= (long long)kAttnMinRunTiles * n_sm;
+    const bool runs = n_sm > 1 && (long_batch || few_items);
+    const int grid = runs ? n_sm : std::max(1, std::min(n_sm, max_items));
     if (dev >= 0 && dev < 64 && !attr_set[hi][dev]) {
         cudaError_t e = hi ? cudaFuncSetAttribute(attn_tcgen05_kernel<128, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<128>::kTotal)
                            : cudaFuncSetAttribute(attn_tcgen05_kernel<64, false>, cudaFuncAttributeMaxDynamicSharedMemorySize, AttnSmem<64>::kTotal);
@@ -944,8 +952,8 @@ static int launch_attend_long(alora_ctx *ctx, const void *qkv, const BatchArgs &
                  : launch_kernel(attn_tcgen05_kernel<64, false>, g3, b3, AttnSmem<64>::kTotal, s, true, tmQ, tmKV, a);
     if (le != cudaSuccess) return -1;
     if (!runs) return 1 + n_small;
-    const cudaError_t me = hi ? launch_kernel(attn_merge_kernel<128>, dim3(2 * (grid - 1)), dim3(512), 0, s, true, a)
-                              : launch_kernel(attn_merge_kernel<64>, dim3(2 * (grid - 1)), dim3(512), 0, s, true, a);
+    const cudaError_t me = hi ? launch_kernel(attn_merge_kernel<128>, dim3(2 * (grid - 1), 4), dim3(512), 0, s, true, a)
+                              : launch_kernel(attn_merge_kernel<64>, dim3(2 * (grid - 1), 4), dim3(512), 0, s, true, a);
     if (me != cudaSuccess) return -1;
     return 2 + n_small;
 }

@@ -216,7 +216,8 @@ __device__ __forceinline__ void metadata_attn_items(const int32_t *__restrict__ 
         const int n = (w.kv_end + kAttnKeysPerTile - 1) / kAttnKeysPerTile;
         sum += n; tmin = min(tmin, n); tmax = max(tmax, n);
     }
-    // Work split of the attention kernel over its n_blocks blocks.  Normally every item is taken whole, round-robin.
+    // Work split of the attention kernel over its n_blocks blocks (the launch uses that many whenever a cut is
+    // possible).  Normally every item is taken whole, round-robin.
     // Long batches (at least kAttnCutMinTiles key tiles per block) of items of nearly equal length that make at
     // least kAttnCutMinWaves full rounds: the first n_whole = n_blocks * floor(items / n_blocks) items are taken
     // whole, round-robin; the key tiles of the remaining items are concatenated and cut into runs of equal length,
@@ -244,8 +245,14 @@ __device__ __forceinline__ void metadata_attn_items(const int32_t *__restrict__ 
         // cutting pays when most of the work is still done on whole items (whose sibling query blocks share their
         // K/V tiles in L2): items of nearly equal length, at least kAttnCutMinWaves full rounds of whole items
         const bool uniform = mx - mn <= max(1, mx / 16);
-        const bool cut = acc >= kAttnCutMinTiles * n_blocks && uniform && total >= kAttnCutMinWaves * n_blocks &&
-                         total % n_blocks != 0;
+        const bool long_batch = acc >= kAttnCutMinTiles * n_blocks && uniform && total >= kAttnCutMinWaves * n_blocks &&
+                                total % n_blocks != 0;
+        // ... and a batch with fewer items than blocks (a few requests with long contexts) is spread over all blocks
+        // when that still leaves every block a run of at least kAttnMinRunTiles key tiles and shortens the longest
+        // block's work by more than the merge costs (about the time of kAttnSpreadMinGain key tiles, measured)
+        const bool few_items = total > 0 && total < n_blocks && acc >= kAttnMinRunTiles * n_blocks &&
+                               mx >= acc / n_blocks + kAttnSpreadMinGain;
+        const bool cut = long_batch || few_items;
         run_first = !cut ? -1 : n_blocks * (total / n_blocks);
         run_len = acc;   // all tiles, for now
         if (!cut) { counts[6] = 0; counts[7] = kAttnMinRunTiles; counts[8] = total; counts[9] = acc; }
@@ -468,7 +475,7 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *a_req, con
     }
     if ((int)blockIdx.x == b_attn && items != nullptr && block_tables != nullptr) {
         metadata_attn_items(qsl, seq_lens, R, Hkv, q_block, small_max, max_items, items, counts, blk_off,
-                            max(1, min(n_sm, (T / q_block + R) * Hkv)), attn_cta_start, status);
+                            n_sm, attn_cta_start, status);
         __syncthreads();
     }
     if ((int)blockIdx.x == b_split && split_items != nullptr && block_tables != nullptr)

@@ -155,6 +155,22 @@ def test_short_suffixes_of_many_requests_on_long_prefixes(oracle64):
     _check_requests(oracle64, shape, w, b, before, after, out_h, [10, 21, 12, 33, 4, 25, 36, 17, 38, 9], qkv_h)
 
 
+def test_few_requests_with_long_contexts_are_spread_over_all_blocks(oracle64):
+    """Three requests with 37 000 .. 52 000 cached tokens and 16, 40 and 100 new ones on a small layer shape: 8
+    attention work items of 290 .. 407 key tiles for 148 blocks.  The work-list builder cuts them into runs of
+    about 19 tiles, one per block; the parts of an item (for the 16-token request: rows shared by the kernel's two
+    query groups) are merged afterwards.  All three requests in full."""
+    shape = wl.LayerShape(hidden=256, n_q_heads=8, n_kv_heads=2, head_dim=128, page_size=16, dtype="bf16")
+    rng = np.random.default_rng(93)
+    P, S, ids = [52000, 37000, 41000], [16, 40, 100], [0, -1, 1]
+    wqkv = wl.make_wqkv(shape, rng)
+    ads = [wl.make_adapter(shape, r, rng, scale=4.0) for r in (8, 32)]
+    b = wl.make_batch(shape, P, S, ids, rng, shuffle_pages=True)
+    w = wl.Workload("few_long", shape, wqkv, ads, b, 93)
+    before, after, out_h, _ = _run_layer(w, seed=1093)
+    _check_requests(oracle64, shape, w, b, before, after, out_h, [0, 1, 2])
+
+
 def test_config5_decode_step_sampled_requests(oracle64):
     """64 requests (base model and 4 rank-32 adapters), contexts 1024..32768, one new token each: the shortest,
     the longest and two more requests, and the projection rows of all 64."""
