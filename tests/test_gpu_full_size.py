@@ -155,6 +155,24 @@ def test_short_suffixes_of_many_requests_on_long_prefixes(oracle64):
     _check_requests(oracle64, shape, w, b, before, after, out_h, [10, 21, 12, 33, 4, 25, 36, 17, 38, 9], qkv_h)
 
 
+def test_many_requests_with_two_to_four_new_tokens_take_the_tensor_core_kernel(oracle64):
+    """200 requests with 1 .. 4 new tokens (G = 4: at most 16 score rows per KV head) on 300 .. 1500 cached ones.
+    160 of them have 2 .. 4 tokens: 320 KV streams for 148 SMs, so the work-list builder sends those to the
+    tensor-core kernel (as items shared by its two query groups) and only the one-token requests to the few-row
+    kernel.  One request of every length, and the projection rows of all."""
+    shape = wl.LayerShape(hidden=256, n_q_heads=8, n_kv_heads=2, head_dim=128, page_size=16, dtype="bf16")
+    rng = np.random.default_rng(95)
+    S = [2, 3, 4, 1, 4] * 40
+    P = [int(x) for x in rng.integers(300, 1500, size=len(S))]
+    ids = [(-1, 0, 1)[i % 3] for i in range(len(S))]
+    wqkv = wl.make_wqkv(shape, rng)
+    ads = [wl.make_adapter(shape, r, rng, scale=4.0) for r in (8, 32)]
+    b = wl.make_batch(shape, P, S, ids, rng, shuffle_pages=True)
+    w = wl.Workload("many_short", shape, wqkv, ads, b, 95)
+    before, after, out_h, qkv_h = _run_layer(w, seed=1095, with_qkv=True)
+    _check_requests(oracle64, shape, w, b, before, after, out_h, [0, 51, 102, 153, 199], qkv_h)
+
+
 def test_few_requests_with_long_contexts_are_spread_over_all_blocks(oracle64):
     """Three requests with 37 000 .. 52 000 cached tokens and 16, 40 and 100 new ones on a small layer shape: 8
     attention work items of 290 .. 407 key tiles for 148 blocks.  The work-list builder cuts them into runs of
