@@ -197,8 +197,8 @@ alora_status alora_prefill_layer(alora_ctx *ctx, int layer, const void *d_hidden
 /*
  * One decode step (Prop. 1, second sentence; Eq. 3): exactly one new token per request (T == R,
  * query_start_loc[r] == r), mixed base / adapter requests.  Same results as alora_prefill_layer on
- * the same arguments (requests whose new tokens make at most 16 score rows per KV head take the same
- * few-row attention kernel in every entry point; this one additionally knows that no request is longer).
+ * the same arguments (a one-token request takes the same few-row attention kernel in every entry
+ * point; this one additionally knows that no request is longer, and launches nothing else).
  */
 alora_status alora_decode_step(alora_ctx *ctx, int layer, const void *d_hidden,
                                const int32_t *d_positions, const int32_t *d_activation_offsets,

@@ -275,6 +275,40 @@ def test_projection_with_128_wide_kv_blocks(oracle64):
     _check_projection(oracle64, shape, w, ads, b, n_off_expected=100)
 
 
+def test_short_suffixes_on_an_empty_or_tiny_cache(oracle64):
+    """Requests with 5 .. 40 new tokens and 0 .. 70 cached ones: attention work items of one or two key tiles whose
+    rows all fall into one query group of the tensor-core kernel (both groups then share the item, one 64-key half
+    of the tile each), including items where one half holds no visible key at all, and the NaN-proofing of V rows
+    beyond the causal limit (the pool starts as all-ones bit patterns)."""
+    import torch
+    rng = np.random.default_rng(47)
+    w = wl.make_wqkv(MID, rng)
+    ads = _boosted_adapters(MID, rng, ((8, 1.0), (32, 1.0)))
+    P = [0, 0, 3, 0, 70, 0, 12]
+    S = [5, 9, 20, 40, 6, 32, 33]
+    ids = [0, 1, -1, 0, 1, 0, 1]
+    b = wl.make_batch(MID, P, S, ids, rng, shuffle_pages=True, with_prefix_hidden=True)
+    g = hp.GpuLayers(MID, [dict(wqkv=w)], [ads], 256, 8)
+    try:
+        pool = g.new_pool(b.num_pages)
+        pool.view(torch.int16).fill_(-1)   # bf16 NaN everywhere a kernel does not write
+        _run_base_prefill(g, MID, b, pool)
+        d = hp.DevBatch(b, MID.dtype)
+        out = g.empty(b.T, MID.Nq)
+        ab.alora_prefill_layer(g.ctx, 0, d.hidden, d.positions, d.a_req, d.ids, d.qsl, d.seq_lens, pool, d.bt,
+                               d.max_blocks, b.num_pages, d.T, d.R, out)
+        assert g.status() == 0
+        Ks, Vs = hp.oracle_base_prefix(oracle64, MID, w, b)
+        want = hp.oracle_block(oracle64, MID, w, ads, b, Ks, Vs)
+        out_h = hp.to_host(out)
+        assert np.isfinite(out_h).all()
+        for r in range(b.R):
+            q0, q1 = int(b.query_start_loc[r]), int(b.query_start_loc[r + 1])
+            assert hp.rel_err(out_h[q0:q1], want["out"][q0:q1]) <= 2e-2, f"request {r}"
+    finally:
+        g.close()
+
+
 def test_full_lora_recompute_matches_eq4(oracle64):
     w, ads, b = _mid_workload(seed=13)
     fb = hp.full_sequence_batch(MID, b)
