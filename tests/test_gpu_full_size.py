@@ -189,6 +189,46 @@ def test_few_requests_with_long_contexts_are_spread_over_all_blocks(oracle64):
     _check_requests(oracle64, shape, w, b, before, after, out_h, [0, 1, 2])
 
 
+_SWEEP_SHAPES = (dict(hidden=256, n_q_heads=8, n_kv_heads=2, head_dim=128, page_size=16),
+                 dict(hidden=256, n_q_heads=4, n_kv_heads=2, head_dim=64, page_size=32),
+                 dict(hidden=256, n_q_heads=8, n_kv_heads=1, head_dim=128, page_size=64))
+
+
+@pytest.mark.parametrize("seed", range(10))
+def test_randomised_batches_over_all_attention_routes(oracle64, seed):
+    """Seeded random batches on three layer shapes (group sizes 4, 2, 8; head dims 128, 64; pages of 16, 32, 64):
+    many requests with 1 .. 5 new tokens, one to three requests with 20 000 .. 60 000 cached tokens, ragged mixes,
+    short suffixes of a medium number of requests, and tiny caches.  Between them they take every route of the
+    attention (few-row kernel, whole / shared / cut work items of the tensor-core kernel, merge of the parts).  The
+    requests with the least, the median and the most work plus three random ones are checked in full (those the
+    oracle finishes in seconds)."""
+    rng = np.random.default_rng(1000 + seed)
+    shape = wl.LayerShape(dtype="bf16", **_SWEEP_SHAPES[seed % 3])
+    kind = seed % 5
+    if kind == 0:
+        R = int(rng.integers(100, 330)); S = rng.integers(1, 6, size=R); P = rng.integers(0, 900, size=R)
+    elif kind == 1:
+        R = int(rng.integers(1, 4)); S = rng.integers(5, 200, size=R); P = rng.integers(20000, 60000, size=R)
+    elif kind == 2:
+        R = int(rng.integers(2, 30)); S = rng.integers(1, 300, size=R); P = rng.integers(0, 3000, size=R)
+    elif kind == 3:
+        R = int(rng.integers(8, 80)); S = rng.integers(1, 40, size=R); P = rng.integers(100, 5000, size=R)
+    else:
+        R = int(rng.integers(1, 12)); S = rng.integers(1, 70, size=R); P = rng.integers(0, 80, size=R)
+    ids = [int(x) for x in rng.integers(-1, 2, size=R)]
+    wqkv = wl.make_wqkv(shape, rng)
+    ads = [wl.make_adapter(shape, r, rng, scale=4.0) for r in (8, 32)]
+    b = wl.make_batch(shape, [int(x) for x in P], [int(x) for x in S], ids, rng, shuffle_pages=True)
+    w = wl.Workload("sweep", shape, wqkv, ads, b, seed)
+    before, after, out_h, _ = _run_layer(w, seed=5000 + seed)
+    assert np.isfinite(out_h).all()
+    work = b.seq_lens.astype(np.int64) * S
+    order = np.argsort(work)
+    sample = sorted({int(order[0]), int(order[len(order) // 2]), int(order[-1])} | {int(x) for x in rng.integers(0, R, size=3)})
+    sample = [r for r in sample if work[r] < 6e6] or [int(order[0])]
+    _check_requests(oracle64, shape, w, b, before, after, out_h, sample)
+
+
 def test_config5_decode_step_sampled_requests(oracle64):
     """64 requests (base model and 4 rank-32 adapters), contexts 1024..32768, one new token each: the shortest,
     the longest and two more requests, and the projection rows of all 64."""
