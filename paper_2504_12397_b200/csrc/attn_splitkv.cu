@@ -213,20 +213,33 @@ attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmKV, const SplitArgs a)
             if (!ok || it < 0) break;
             const AttnSplitWork w = a.items[it];
             const int n_st = (w.kv_end - w.kv_start + kSkStageKeys - 1) / kSkStageKeys;
+            // Window of the request's block-table row: lane l holds entry win0 + l (win0 a multiple of 32; 32 entries
+            // cover a whole number of 64-key stages, and key ranges start at multiples of 64).  A table entry is a
+            // dependent load from global memory that would otherwise sit in front of every stage's copies; the
+            // following window is in flight while this one is used.
+            const int32_t *bt_row = a.block_tables + (size_t)w.req * a.max_blocks;
+            auto load_window = [&](int w0) { return w0 + lane < a.max_blocks ? bt_row[w0 + lane] : -1; };
+            int win0 = (w.kv_start / a.page_size) & ~31;
+            int win = load_window(win0), win_next = load_window(win0 + 32);
             for (int j = 0; j < n_st && ok; ++j, ++kt) {
                 const int st = kt % kSkStages;
                 const int kbase = w.kv_start + j * kSkStageKeys;
+                if (kbase / a.page_size >= win0 + 32) {
+                    win0 += 32;
+                    win = win_next;
+                    win_next = load_window(win0 + 32);
+                }
                 const int units = min(units_per_stage, (w.kv_end - kbase + a.box_rows - 1) / a.box_rows);
+                const int page = __shfl_sync(0xffffffffu, win, ((kbase + lane * a.box_rows) / a.page_size - win0) & 31);
                 int row = -1;
                 if (lane < units) {
                     const int key = kbase + lane * a.box_rows;
-                    const int page = a.block_tables[(size_t)w.req * a.max_blocks + key / a.page_size];
                     if (page < 0 || page >= a.num_pages) report(a.status, ALORA_ERR_PAGE_RANGE);
                     else row = (page * 2 * a.Hkv + w.kv_head) * a.page_size + key % a.page_size;
                 }
                 const unsigned valid = __ballot_sync(0xffffffffu, row >= 0);
                 if (lane == 0) {
-                    ok = tc::mbar_wait(empty_bar(st), ((kt / kSkStages) & 1) ^ 1, abort_flag);
+                    ok = tc::mbar_wait_relaxed(empty_bar(st), ((kt / kSkStages) & 1) ^ 1, abort_flag);
                     if (ok) tc::mbar_arrive_expect_tx(full_bar(st), (uint32_t)__popc(valid) * unit_bytes);
                 }
                 ok = __shfl_sync(0xffffffffu, ok, 0);
