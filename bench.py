@@ -318,6 +318,133 @@ def short_suffix_leg(ab, hp, ctx, shape, stream, flush, peaks, requests, prefix,
             "attention_hbm_gbs": gbs, "attention_frac_of_hbm_peak": gbs / peaks["hbm_gbs"] if gbs else None}
 
 
+def evaluator_leg(ab, hp, shape, stream, local, n_eval, seed=9, convs=8, prompt=4096, gen=256, inv=16, eval_steps=16):
+    """The paper's evaluator workload on one layer: `convs` conversations get a base-model prefill of `prompt` tokens
+    and `gen` base decode steps; then `n_eval` adapters each read the conversation and answer: `inv` invocation
+    tokens prefilled, `eval_steps` tokens decoded.  aLoRA: the evaluators' block tables point at the conversation's
+    own pages (the base model's cache, reused as it is) and only the invocation is prefilled, adapted from its
+    first token on.  LoRA: every evaluator prefills prompt + generation + invocation again with its adapter on all
+    tokens, into pages of its own.  Both pipelines are timed as a whole with CUDA events."""
+    import torch
+    rng = np.random.default_rng(seed)
+    ps = shape.page_size
+    ctx_len = prompt + gen
+    assert ctx_len % ps == 0, "the evaluators' own tokens start on a fresh page"
+    R2 = convs * n_eval
+    conv_blocks, own_blocks = ctx_len // ps, (inv + eval_steps + ps - 1) // ps
+    full_blocks = conv_blocks + own_blocks
+    num_pages = convs * conv_blocks + R2 * own_blocks + R2 * full_blocks + 3
+    order = rng.permutation(num_pages).astype(np.int32)
+    nxt = 0
+
+    def take(n):
+        nonlocal nxt
+        out = order[nxt:nxt + n]
+        nxt += n
+        return out
+    bt_conv = np.zeros((convs, full_blocks), np.int32)
+    for c in range(convs):
+        bt_conv[c, :conv_blocks] = take(conv_blocks)
+    bt_alora = np.zeros((R2, full_blocks), np.int32)
+    bt_lora = np.zeros((R2, full_blocks), np.int32)
+    for c in range(convs):
+        for n in range(n_eval):
+            r = c * n_eval + n
+            bt_alora[r, :conv_blocks] = bt_conv[c, :conv_blocks]
+            bt_alora[r, conv_blocks:] = take(own_blocks)
+            bt_lora[r] = take(full_blocks)
+    ids_eval = np.tile(np.arange(n_eval, dtype=np.int32), convs)
+    T_re = R2 * (ctx_len + inv)
+    cfg = ab.make_config(hidden=shape.hidden, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
+                         head_dim=shape.head_dim, page_size=ps, max_adapters=max(n_eval, 1), max_rank=32,
+                         dtype=ab.DTYPE_BF16, device=local, max_tokens=max(T_re, convs * prompt), max_requests=max(R2, convs))
+    ctx = ab.alora_create(cfg)
+    keep = []
+    g = torch.Generator(device="cuda"); g.manual_seed(seed)
+
+    def rnd(*dims, std=1.0):
+        return (torch.randn(dims, generator=g, device="cuda", dtype=torch.float32) * std).to(torch.bfloat16)
+    wq = rnd(shape.N, shape.hidden, std=0.02)
+    ab.alora_set_layer_weights(ctx, 0, wq)
+    for i in range(n_eval):
+        mats = []
+        for blk in (shape.Nq, shape.Nkv, shape.Nkv):
+            mats += [rnd(32, shape.hidden, std=0.02), rnd(blk, 32, std=0.02)]
+        keep.append(mats)
+        ab.alora_register_adapter(ctx, i, 0, 32, 1.0, *mats)
+    pool = torch.zeros((num_pages, 2, shape.n_kv_heads, ps, shape.head_dim), device="cuda", dtype=torch.bfloat16)
+    hid = rnd(max(T_re, convs * prompt), shape.hidden)
+    out = torch.empty((max(T_re, convs * prompt), shape.Nq), dtype=torch.bfloat16, device="cuda")
+    i32 = lambda a: hp.idev(np.ascontiguousarray(a, dtype=np.int32))  # noqa: E731
+    # phase 1: base prefill of the prompts
+    p1 = dict(pos=i32(np.tile(np.arange(prompt), convs)), qsl=i32(np.arange(convs + 1) * prompt),
+              lens=i32(np.full(convs, prompt)), ids=i32(np.full(convs, -1)), bt=i32(bt_conv))
+    # phase 2: base decode steps
+    p2_pos = i32(prompt + np.arange(gen)[:, None] + np.zeros((1, convs), np.int64))
+    p2_len = (p2_pos + 1).contiguous()
+    areq_conv = i32(np.zeros(convs))
+    # phase 3 (aLoRA): invocation prefill on the reused cache, adapted from its first token on
+    p3 = dict(pos=i32(np.tile(ctx_len + np.arange(inv), R2)), qsl=i32(np.arange(R2 + 1) * inv),
+              lens=i32(np.full(R2, ctx_len + inv)), ids=i32(ids_eval), areq=i32(np.full(R2, ctx_len)), bt=i32(bt_alora))
+    # phase 3' (LoRA): the whole sequence again with the adapter on every token
+    L3 = ctx_len + inv
+    p3l = dict(pos=i32(np.tile(np.arange(L3), R2)), qsl=i32(np.arange(R2 + 1) * L3), lens=i32(np.full(R2, L3)),
+               ids=i32(ids_eval), bt=i32(bt_lora))
+    # phase 4: the evaluators' decode steps (aLoRA: gate opens at the invocation; LoRA: open everywhere)
+    p4_pos = i32(L3 + np.arange(eval_steps)[:, None] + np.zeros((1, R2), np.int64))
+    p4_len = (p4_pos + 1).contiguous()
+    areq_open = i32(np.zeros(R2))
+
+    def base_phases():
+        ab.alora_full_lora_prefill_layer(ctx, 0, hid, p1["pos"], p1["ids"], p1["qsl"], p1["lens"], pool, p1["bt"],
+                                         full_blocks, num_pages, convs * prompt, convs, out, stream)
+        for i in range(gen):
+            ab.alora_decode_step(ctx, 0, hid, p2_pos[i], areq_conv, p1["ids"], p2_len[i], pool, p1["bt"], full_blocks,
+                                 num_pages, convs, out, stream)
+
+    def alora_eval():
+        ab.alora_prefill_layer(ctx, 0, hid, p3["pos"], p3["areq"], p3["ids"], p3["qsl"], p3["lens"], pool, p3["bt"],
+                               full_blocks, num_pages, R2 * inv, R2, out, stream)
+        for i in range(eval_steps):
+            ab.alora_decode_step(ctx, 0, hid, p4_pos[i], p3["areq"], p3["ids"], p4_len[i], pool, p3["bt"], full_blocks,
+                                 num_pages, R2, out, stream)
+
+    def lora_eval():
+        ab.alora_full_lora_prefill_layer(ctx, 0, hid, p3l["pos"], p3l["ids"], p3l["qsl"], p3l["lens"], pool, p3l["bt"],
+                                         full_blocks, num_pages, T_re, R2, out, stream)
+        for i in range(eval_steps):
+            ab.alora_decode_step(ctx, 0, hid, p4_pos[i], areq_open, p3l["ids"], p4_len[i], pool, p3l["bt"], full_blocks,
+                                 num_pages, R2, out, stream)
+
+    def once(fn, reps):
+        fn()
+        torch.cuda.synchronize()
+        e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        e0.record(stream)
+        for _ in range(reps):
+            fn()
+        e1.record(stream)
+        torch.cuda.synchronize()
+        return e0.elapsed_time(e1) / reps
+    base_ms = once(base_phases, 2)
+    alora_ms = once(alora_eval, 5)
+    lora_ms = once(lora_eval, 2)
+    status = ab.alora_get_status(ctx)
+    finite = bool(torch.isfinite(out[:R2].float()).all())
+    ab.alora_destroy(ctx)
+    page_bytes = 2 * shape.n_kv_heads * ps * shape.head_dim * 2
+    return {"workload": f"one 8B-shape layer: {convs} conversations x ({prompt} prompt tokens, {gen} base decode steps), then "
+                        f"{n_eval} evaluator adapter(s) x ({inv} invocation tokens + {eval_steps} decode steps)",
+            "base_prefill_and_generation_ms": base_ms,
+            "evaluators_alora_ms": alora_ms, "evaluators_lora_ms": lora_ms,
+            "evaluator_stage_speedup": lora_ms / alora_ms,
+            "pipeline_alora_ms": base_ms + alora_ms, "pipeline_lora_ms": base_ms + lora_ms,
+            "pipeline_speedup": (base_ms + lora_ms) / (base_ms + alora_ms),
+            "evaluator_cache_bytes_alora": R2 * own_blocks * page_bytes,
+            "evaluator_cache_bytes_lora": R2 * full_blocks * page_bytes,
+            "device_status": status, "output_finite": finite}
+
+
 def stack_leg(ab, hp, shape, stream, local, seed=4, requests=4, prefix=32768, suffix=1024, n_layers=32):
     """Config 4: the full decoder stack at the 8B shape (RMSNorm, attention block, o_proj, SwiGLU MLP; random
     bf16 weights), 4 requests with 32768 cached positions and 1024 aLoRA suffix tokens each, against the
@@ -413,8 +540,8 @@ def main():
     ap.add_argument("--no-recompute", action="store_true", help="skip the full-LoRA recompute comparisons")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the decode and short-suffix legs")
-    ap.add_argument("--legs", default="decode,short,recompute8k,stack",
-                    help="extra legs to run after the main workload (comma list of decode, short, recompute8k, stack)")
+    ap.add_argument("--legs", default="decode,short,recompute8k,evaluators,stack",
+                    help="extra legs to run after the main workload (comma list of decode, short, recompute8k, evaluators, stack)")
     ap.add_argument("--decode-steps", type=int, default=256)
     ap.add_argument("--decode-ctx-max", type=int, default=32768)
     ap.add_argument("--requests", type=int, default=8)
@@ -633,10 +760,14 @@ def main():
     ab.alora_destroy(ctx)
     want_cpu = rank == 0 and world == 1 and not args.no_cpu_baseline
     pool_np = main_case.pool.to(torch.float32).cpu().numpy() if want_cpu else None
-    stack = None
-    if "stack" in legs:
+    stack = evaluators = None
+    if "evaluators" in legs or "stack" in legs:
         del main_case.pool
         torch.cuda.empty_cache()
+    if "evaluators" in legs:
+        evaluators = [evaluator_leg(ab, hp, shape, stream, local, n) for n in (1, 5)]
+        torch.cuda.empty_cache()
+    if "stack" in legs:
         stack = stack_leg(ab, hp, shape, stream, local)
     clocks_rest = sampler_rest.stop()
 
@@ -661,7 +792,7 @@ def main():
                                       "how": "K steps as a 3-stream pipeline (H2D, kernels, D2H; double-buffered), total time / K; serial = one step at a time"},
             "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
             "full_lora_recompute": recompute, "full_lora_recompute_8k_prefix": recompute_8k,
-            "decode": decode, "short_suffix": short, "stack": stack, "device_status": status,
+            "decode": decode, "short_suffix": short, "evaluator_pipeline": evaluators, "stack": stack, "device_status": status,
         }))
     if world > 1:
         dist.destroy_process_group()
