@@ -40,6 +40,10 @@ constexpr int kGemmThreads = 192;
 constexpr int kTensorRP = 64; // the tensor path stores adapters padded to 64 rank columns
 
 struct GemmArgs {
+    // Bytes one copy of the activation tile brings (0: the full 128-row tile).  A batch of at most 64 rows uses a
+    // 64-row box: the other half of the tile in shared memory is never filled, the accumulator rows it feeds are
+    // never read, and the shared-memory fill of a stage, which bounds this shape, drops by a third.
+    int a_tile_bytes;
     const ProjTile *tiles;        // nullptr: dense row tiles 0..ceil(M/128)-1, no adapters
     const int32_t *n_row_tiles;   // device count of `tiles` entries (when tiles != nullptr)
     int M, N, K;
@@ -173,6 +177,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         if (lane == 0) {
             // ------------------------------ TMA producer ------------------------------
             tc::tma_prefetch_desc(&tmA); tc::tma_prefetch_desc(&tmB);
+            const uint32_t a_bytes = a.a_tile_bytes ? (uint32_t)a.a_tile_bytes : (uint32_t)S::kABytes;
             uint32_t kc = 0;        // ring slots filled so far
             bool ok = true;
             for (int item = blockIdx.x; item < total && ok; item += gridDim.x) {
@@ -185,11 +190,11 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     if (!tc::mbar_wait(empty_bar(s), ((kc / kStages) & 1) ^ 1, abort_flag)) { ok = false; break; }
                     const uint32_t sa = smem_base + s * S::kStageBytes, sb = sa + S::kABytes;
                     if (g.shrink) {
-                        tc::mbar_arrive_expect_tx(full_bar(s), S::kABytes + kShrinkCols * kBK * 2);
+                        tc::mbar_arrive_expect_tx(full_bar(s), a_bytes + kShrinkCols * kBK * 2);
                         tc::tma_load_2d(sa, &tmA, full_bar(s), kb * kBK, t.row_start);
                         tc::tma_load_2d(sb, &tmS, full_bar(s), kb * kBK, t.adapter * kShrinkCols);
                     } else if (kb < kb_main) {
-                        tc::mbar_arrive_expect_tx(full_bar(s), S::kStageBytes);
+                        tc::mbar_arrive_expect_tx(full_bar(s), a_bytes + S::kBBytes);
                         tc::tma_load_2d(sa, &tmA, full_bar(s), kb * kBK, t.row_start);
                         tc::tma_load_2d(sb, &tmB, full_bar(s), kb * kBK, n0);
                     } else {
@@ -478,8 +483,10 @@ int launch_project_tc(alora_ctx *ctx, int layer, const void *hidden, int T, void
     }
     const int BN = pick_bn(d.N, d.Nq, d.Nkv, true, T);
     if (BN == 0 || d.H % 8 != 0) return -1;
-    CUtensorMap tmX, tmTt;
+    CUtensorMap tmX, tmTt, tmX64;
     if (!make_tensor_map_bf16(&tmX, hidden, T, d.H, d.H, kBM)) return -1;
+    const bool half_box = T <= kBM / 2;   // see GemmArgs::a_tile_bytes
+    if (half_box && !make_tensor_map_bf16(&tmX64, hidden, T, d.H, d.H, kBM / 2)) return -1;
     if (!make_tensor_map_bf16(&tmTt, ctx->d_t, ctx->cfg.max_tokens, 3 * kTensorRP, 3 * kTensorRP, kBM)) return -1;
     const TcLayerMaps &lm = ctx->tc_maps[layer];
     const AdapterDev *ads = ctx->d_adapters + (size_t)layer * ctx->cfg.max_adapters;
@@ -503,6 +510,8 @@ int launch_project_tc(alora_ctx *ctx, int layer, const void *hidden, int T, void
     {
         ProfScope prof(ctx, KK_PROJECT, s);
         GemmArgs g{};
+        g.a_tile_bytes = half_box ? (kBM / 2) * kBK * 2 : 0;
+        const CUtensorMap &tmXg = half_box ? tmX64 : tmX;
         g.tiles = ctx->d_tiles; g.n_row_tiles = ctx->d_counts; g.M = T; g.N = d.N; g.K = d.H;
         g.out = (__nv_bfloat16 *)qkv; g.ldo = d.N; g.residual = nullptr; g.adapters = ads;
         g.Nq = d.Nq; g.Nkv = d.Nkv; g.total_adapter_rows = d.N; g.status = ctx->d_status;
@@ -521,10 +530,10 @@ int launch_project_tc(alora_ctx *ctx, int layer, const void *hidden, int T, void
         }
         const int items = max_row_tiles * ((d.N + BN - 1) / BN + (fuse_shrink ? 1 : 0));
         const bool ok = BN == 256
-                            ? launch_gemm_bn<256>(ctx, tmX, lm.wqkv[1], tmTt, lm.b_all_bn[1], lm.a_all, g, items, s)
+                            ? launch_gemm_bn<256>(ctx, tmXg, lm.wqkv[1], tmTt, lm.b_all_bn[1], lm.a_all, g, items, s)
                             : BN == 128
-                                  ? launch_gemm_bn<128>(ctx, tmX, lm.wqkv[0], tmTt, lm.b_all_bn[0], lm.a_all, g, items, s)
-                                  : launch_gemm_bn<64>(ctx, tmX, lm.wqkv[2], tmTt, lm.b_all_bn[2], lm.a_all, g, items, s);
+                                  ? launch_gemm_bn<128>(ctx, tmXg, lm.wqkv[0], tmTt, lm.b_all_bn[0], lm.a_all, g, items, s)
+                                  : launch_gemm_bn<64>(ctx, tmXg, lm.wqkv[2], tmTt, lm.b_all_bn[2], lm.a_all, g, items, s);
         if (!ok) return -1;
         ++n;
     }
@@ -547,9 +556,11 @@ int launch_linear_tc(alora_ctx *ctx, const void *x, const void *W, int T, int K,
     }
     const int BN = pick_bn(N, N, 0, false, T);
     CUtensorMap tmX, tmW;
-    if (!make_tensor_map_bf16(&tmX, x, T, K, K, kBM)) return -1;
+    const bool half_box = T <= kBM / 2;   // see GemmArgs::a_tile_bytes
+    if (!make_tensor_map_bf16(&tmX, x, T, K, K, half_box ? kBM / 2 : kBM)) return -1;
     if (!make_tensor_map_bf16(&tmW, W, N, K, K, BN)) return -1;
     GemmArgs g{};
+    g.a_tile_bytes = half_box ? (kBM / 2) * kBK * 2 : 0;
     g.tiles = nullptr; g.n_row_tiles = nullptr; g.M = T; g.N = N; g.K = K; g.out = (__nv_bfloat16 *)y; g.ldo = N;
     g.residual = (const __nv_bfloat16 *)residual; g.adapters = nullptr; g.Nq = N; g.Nkv = 0;
     g.total_adapter_rows = 0; g.status = ctx->d_status;
