@@ -367,13 +367,14 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
     }
     __syncthreads();
     if (threadIdx.x == 0) {
-        // Range length: a range costs a fixed few microseconds beyond its streaming time (query fetch, combining
-        // the warps, publishing the partial result), and the last ranges of a launch leave SMs idle for up to one
-        // range.  With t = streaming time of all units on one SM (0.74 us per 64-key unit at an SM's share of
-        // the HBM bandwidth) the sum of both losses is smallest near sqrt(t / 3 us) ranges per SM, capped by the
-        // capacity of the work list.
+        // Range length: a range costs a fixed time beyond its streaming time (item claim, first table window and
+        // first copies, query fetch, combining the warps, publishing the partial result, a share of the merge), and
+        // the last ranges of a launch leave SMs idle for up to one range.  With t = streaming time of all units on
+        // one SM (0.74 us per 64-key unit at an SM's share of the HBM bandwidth) the sum of both losses is smallest
+        // near sqrt(t / c) ranges per SM, capped by the capacity of the work list; c = 12 us is what batches of 2
+        // to 64 requests with 4096 to 32768 cached tokens run fastest with (3 us: 5 .. 16 % slower on the small ones).
         const float t_us = (float)tot_units * 0.74f / (float)max(n_sm, 1);
-        const float per_sm = fminf(fmaxf(sqrtf(t_us / 3.f), 1.f), (float)kSplitItemsPerSm);
+        const float per_sm = fminf(fmaxf(sqrtf(t_us / 12.f), 1.f), (float)kSplitItemsPerSm);
         const unsigned long long target = (unsigned long long)ceilf(per_sm * (float)max(n_sm, 1));
         chunk_units = (int)max(4ull, (tot_units + target - 1) / target);
     }
