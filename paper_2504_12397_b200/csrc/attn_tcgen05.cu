@@ -932,7 +932,10 @@ static int launch_attend_long(alora_ctx *ctx, const void *qkv, const BatchArgs &
     const int n_sm = ctx->sm_count;
     const long long max_tiles = (long long)max_items * (((long long)b.max_blocks * d.page + kKeysPerTile - 1) / kKeysPerTile);
     const bool long_batch = max_tiles >= (long long)kAttnCutMinTiles * n_sm && max_items >= kAttnCutMinWaves * n_sm;
-    const bool few_items = max_items < n_sm && max_tiles >= (long long)kAttnMinRunTiles * n_sm;
+    // (not for a batch that looks like few-row work only, a handful of new tokens per request: an unused merge
+    // launch would only lengthen its step; should a long request hide in such a batch it is taken whole)
+    const bool few_items = max_items < n_sm && max_tiles >= (long long)kAttnMinRunTiles * n_sm &&
+                           (long long)b.T > (long long)b.R * ctx->small_max_tokens;
     const bool runs = n_sm > 1 && (long_batch || few_items);
     const int grid = runs ? n_sm : std::max(1, std::min(n_sm, max_items));
     if (dev >= 0 && dev < 64 && !attr_set[hi][dev]) {
