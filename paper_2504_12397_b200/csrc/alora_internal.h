@@ -57,6 +57,7 @@ struct AttnWork {
     int32_t n_splits;
 };
 constexpr int kAttnKeysPerTile = 128;   // keys per K/V tile of the tensor-core attention kernel
+constexpr int kRowwiseAlwaysRows = 24;  // batches of at most this many rows always take the projection's row-wise route
 constexpr int kAttnMinRunTiles = 8;     // shortest run of key tiles given to one block
 constexpr int kAttnCutMinTiles = 128;   // items are cut into runs only when a block has at least this many tiles to do
 constexpr int kAttnCutMinWaves = 3;     // ... and the items make at least this many full rounds over the blocks

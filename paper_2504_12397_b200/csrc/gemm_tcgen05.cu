@@ -501,8 +501,9 @@ int launch_project_tc(alora_ctx *ctx, int layer, const void *hidden, int T, void
         n += launch_lora_delta_rows(ctx, layer, hidden, T, s);
     }
     const bool fuse_shrink = have_adapters && BN == 256;
-    // (a batch that fits one row tile always takes the row-wise route when it has adapter rows: no shrink launch)
-    if (have_adapters && !fuse_shrink && !(may_rowwise && T <= kBM)) {
+    // (a batch of at most kRowwiseAlwaysRows rows always takes the row-wise route when it has adapter rows: no shrink
+    // launch; otherwise the shrink kernel looks at the flag itself)
+    if (have_adapters && !fuse_shrink && !(may_rowwise && T <= kRowwiseAlwaysRows)) {
         ProfScope prof(ctx, KK_SHRINK, s);
         if (!launch_shrink_tc(ctx, tmX, lm.a_all, ads, d.H, max_row_tiles, s)) return -1;
         ++n;

@@ -137,10 +137,11 @@ __device__ __forceinline__ void metadata_tiles(const int32_t *__restrict__ a_req
         counts[2] = n_ad;
         // Row tiles that hold only a few rows each (decode steps, short suffixes of many requests with different
         // adapters) waste the tensor cores: when the tiles cover more than twice the batch's rows, and always when
-        // the whole batch fits one row tile, the projection takes the row-wise route (dense row tiles + a per-row
-        // delta) instead.
+        // the batch has at most kRowwiseAlwaysRows rows, the projection takes the row-wise route (dense row tiles + a
+        // per-row delta) instead.  (The per-row delta costs about 0.4 us per row, the tensor-core shrink of a few
+        // tiles about 8 us whatever their rows.)
         const bool wasteful = (long long)nt * kProjTileRows > 2ll * T + 2 * kProjTileRows;
-        counts[5] = (n_ad > 0 && T <= rowwise_cap && (T <= kProjTileRows || wasteful)) ? 1 : 0;
+        counts[5] = (n_ad > 0 && T <= rowwise_cap && (T <= kRowwiseAlwaysRows || wasteful)) ? 1 : 0;
     }
     __syncthreads();
     for (int i = threadIdx.x; i < n_tiles; i += blockDim.x) {
