@@ -17,7 +17,8 @@ def rel_err(got: np.ndarray, want: np.ndarray) -> float:
 
 
 def tol(shape: wl.LayerShape) -> float:
-    # bf16: the method's stated bound; fp32: derived from H-length fp32 dot products
+    # bf16: the method's stated bound; fp32: H-length fp32 dot products err by about sqrt(H) * 2^-24 ~ 1e-6
+    # relative, taken with a tenfold margin
     return 2e-2 if shape.dtype == "bf16" else 1e-5
 
 
