@@ -23,7 +23,9 @@
  * identity, B = 0 => base, a_req = 0 => merged-weight LoRA (Eq. 4) against a library matmul,
  * attention against a library softmax-attention routine and closed forms (single key, uniform
  * scores, two-key logistic weight, constant V), decode == prefill row, page-permutation
- * invariance, brute-force slot indices, and Prop. 2's closed-form pair and row counts.
+ * invariance, brute-force slot indices, the cache layout read back by plain array indexing, and
+ * Prop. 2's closed-form pair and row counts.  tests/test_oracle_mutants.py plants one-line
+ * mistakes in a copy of this file and checks that the pins notice.
  * No function in this file is "parity unpinned".
  */
 #include <math.h>

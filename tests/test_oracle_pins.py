@@ -422,3 +422,108 @@ def test_prop1_holds_through_a_two_layer_stack(oracle64):
         np.testing.assert_array_equal(Ka[:a_req], Kb[:a_req])
         np.testing.assert_array_equal(Va[:a_req], Vb[:a_req])
         assert np.abs(xa[a_req:] - xb[a_req:]).max() > 1e-6
+
+
+# ---- decoder layer against an independent restatement; pool layout by plain indexing ----------------
+
+STACK_SHAPE = wl.LayerShape(hidden=32, n_q_heads=4, n_kv_heads=2, head_dim=8, page_size=4, dtype="fp32",
+                            intermediate=48)
+
+
+def _torch_decoder_layer(h, lw, ad, shape, eps, positions, qsl, a_req, ids, prefix_K, prefix_V):
+    """Pre-norm residual decoder layer written with library ops only (fp64): rms_norm, matmul,
+    scaled_dot_product_attention under an explicit visibility mask, silu.  One request at a time."""
+    F = torch.nn.functional
+    t64 = lambda a: torch.from_numpy(np.asarray(a, np.float64))
+    H, Nq, Nkv, Hq, Hkv, hd, I = (shape.hidden, shape.Nq, shape.Nkv, shape.n_q_heads, shape.n_kv_heads,
+                                  shape.head_dim, shape.intermediate)
+    out = torch.empty((len(positions), H), dtype=torch.float64)
+    for r in range(len(qsl) - 1):
+        lo, hi = int(qsl[r]), int(qsl[r + 1])
+        x, pos = t64(h[lo:hi]), torch.as_tensor(np.asarray(positions[lo:hi], np.int64))
+        xn = F.rms_norm(x, (H,), t64(lw["norm_attn"]), eps)
+        qkv = xn @ t64(lw["wqkv"]).T
+        if ids[r] >= 0:
+            a = ad[ids[r]]
+            delta = torch.cat([(xn @ t64(a.Aq).T) @ t64(a.Bq).T, (xn @ t64(a.Ak).T) @ t64(a.Bk).T,
+                               (xn @ t64(a.Av).T) @ t64(a.Bv).T], dim=1) * a.scale
+            qkv = torch.where((pos >= int(a_req[r]))[:, None], qkv + delta, qkv)
+        K = torch.cat([t64(prefix_K[r]), qkv[:, Nq:Nq + Nkv]]) if prefix_K[r] is not None else qkv[:, Nq:Nq + Nkv]
+        V = torch.cat([t64(prefix_V[r]), qkv[:, Nq + Nkv:]]) if prefix_V[r] is not None else qkv[:, Nq + Nkv:]
+        L = K.shape[0]
+        q = qkv[:, :Nq].reshape(hi - lo, Hq, hd).transpose(0, 1)
+        Kh = K.reshape(L, Hkv, hd).transpose(0, 1).repeat_interleave(Hq // Hkv, dim=0)
+        Vh = V.reshape(L, Hkv, hd).transpose(0, 1).repeat_interleave(Hq // Hkv, dim=0)
+        visible = torch.arange(L)[None, :] <= pos[:, None]
+        o = F.scaled_dot_product_attention(q, Kh, Vh, attn_mask=visible)
+        h1 = x + o.transpose(0, 1).reshape(hi - lo, Nq) @ t64(lw["wo"]).T
+        xm = F.rms_norm(h1, (H,), t64(lw["norm_mlp"]), eps)
+        gu = xm @ t64(lw["wgate_up"]).T
+        out[lo:hi] = h1 + (F.silu(gu[:, :I]) * gu[:, I:]) @ t64(lw["wdown"]).T
+    return out.numpy()
+
+
+def test_decoder_layer_against_library_restatement(oracle64):
+    """The layer composition (norm, gated q/k/v, attention over cached ++ new rows, o_proj and its
+    residual, norm, SwiGLU MLP and its residual) against the same layer written with torch ops:
+    two requests, one with an adapter whose gate opens in the middle of its new tokens, both on
+    cached prefixes.  Weights are scaled up so that either residual branch, either norm gain and
+    the delta each move the result by far more than the tolerance."""
+    shape, eps = STACK_SHAPE, 1e-5
+    rng = np.random.default_rng(11)
+    lw = wl.make_stack_weights(shape, rng)
+    for k in ("wqkv", "wo", "wgate_up", "wdown"):
+        lw[k] = lw[k] * 10
+    ad = [wl.make_adapter(shape, 4, rng)]
+    for n in ("Aq", "Bq", "Ak", "Bk", "Av", "Bv"):
+        setattr(ad[0], n, getattr(ad[0], n) * 20)
+    prefix, new, ids, a_req = (6, 9), (7, 5), (0, -1), (9, 0)
+    T = sum(new)
+    h = rng.standard_normal((T, shape.hidden))
+    qsl = np.asarray([0, new[0], T], np.int32)
+    pos = np.concatenate([np.arange(p, p + n) for p, n in zip(prefix, new)]).astype(np.int32)
+    pK = [rng.standard_normal((p, shape.Nkv)) for p in prefix]
+    pV = [rng.standard_normal((p, shape.Nkv)) for p in prefix]
+    got, blk = oracle64.decoder_layer(h, lw, shape.Nq, shape.Nkv, shape.n_q_heads, shape.n_kv_heads,
+                                      shape.head_dim, eps, pos, qsl, a_req, ids, [_ad(ad[0])], pK, pV)
+    want = _torch_decoder_layer(h, lw, ad, shape, eps, pos, qsl, a_req, ids, pK, pV)
+    np.testing.assert_allclose(got, want, rtol=1e-10, atol=1e-11)
+    assert blk["gate"].tolist() == [0, 0, 0, 1, 1, 1, 1] + [0] * 5
+    # each part of the composition carries weight here: leaving it out is far outside the tolerance
+    assert np.abs(got - h).max() > 0.1
+
+
+def test_pool_layout_by_plain_indexing(oracle64):
+    """The cache layout pool[page][plane][kv head][row][hd] (plane 0 = K, 1 = V), read back with
+    numpy indexing after an append: row p of a request sits in page block_table[p // page] at row
+    p % page, K in plane 0, V in plane 1, head g in pool[..., g, row, :].  Heads, planes, rows and
+    head-dim extents all differ, so a layout with any two of them exchanged cannot pass."""
+    Hkv, ps, hd = 3, 4, 5
+    rng = np.random.default_rng(12)
+    bt = np.asarray([[5, 2, 7], [1, 6, 0]], np.int32)
+    prefix, new = (3, 0), (6, 5)
+    qsl = np.asarray([0, 6, 11], np.int32)
+    pos = np.concatenate([np.arange(p, p + n) for p, n in zip(prefix, new)]).astype(np.int32)
+    T = 11
+    k = rng.standard_normal((T, Hkv * hd)).astype(np.float32)
+    v = rng.standard_normal((T, Hkv * hd)).astype(np.float32)
+    pool = np.full((9, 2, Hkv, ps, hd), -7.0, np.float32)
+    slots = oracle64.slot_mapping(pos, qsl, bt, ps)
+    oracle64.paged_append(pool, k, v, slots, Hkv, ps, hd)
+    untouched = np.ones(pool.shape, bool)
+    for r in range(2):
+        for t in range(qsl[r], qsl[r + 1]):
+            page, row = bt[r, pos[t] // ps], pos[t] % ps
+            assert slots[t] == page * ps + row
+            for g in range(Hkv):
+                np.testing.assert_array_equal(pool[page, 0, g, row, :], k[t, g * hd:(g + 1) * hd])
+                np.testing.assert_array_equal(pool[page, 1, g, row, :], v[t, g * hd:(g + 1) * hd])
+            untouched[page, :, :, row, :] = False
+    assert (pool[untouched] == -7).all()
+    # the gather reads the same layout: fill a pool by indexing, gather it, compare
+    pool2 = rng.standard_normal(pool.shape).astype(np.float32)
+    K, V = oracle64.paged_gather(pool2, bt[0], 9, Hkv, ps, hd)
+    for p in range(9):
+        for g in range(Hkv):
+            np.testing.assert_array_equal(K[p, g * hd:(g + 1) * hd], pool2[bt[0, p // ps], 0, g, p % ps, :])
+            np.testing.assert_array_equal(V[p, g * hd:(g + 1) * hd], pool2[bt[0, p // ps], 1, g, p % ps, :])
