@@ -8,6 +8,9 @@ Metric: suffix tokens per second.  Prints ONE JSON line (rank 0).
 
     python bench.py [--gpus N] [--steps K] [--warmup W] [--impl reference] [--no-recompute]
 
+With --gpus N > 1 and no launcher around it, the script starts N ranks of itself (torch.distributed.run on
+127.0.0.1); under torchrun it reads RANK / LOCAL_RANK / WORLD_SIZE as usual.
+
 --impl reference times the CPU oracle (oracle/) on the host cores on a bounded sample of the same
 workload.  With N > 1 (torchrun) every rank runs the same per-GPU batch on its own GPU (requests are
 independent: weak scaling, no data-path collective).
@@ -26,7 +29,6 @@ import numpy as np
 
 ROOT = os.path.dirname(os.path.abspath(__file__))
 sys.path.insert(0, ROOT)
-sys.path.insert(0, os.path.join(ROOT, "tests"))
 
 from paper_2504_12397_b200 import sharding  # noqa: E402
 from paper_2504_12397_b200 import workloads as wl  # noqa: E402
@@ -118,10 +120,10 @@ def oracle_sample_rate(w: wl.Workload, pool_np: np.ndarray, n_tokens: int, reque
     """Times the CPU oracle on the first n_tokens suffix tokens of each listed request (projection of those
     rows + their attention over the request's cache), stopping once budget_s has been spent.
     Returns (tokens/s, threads, seconds, tokens done)."""
-    from oracle import Oracle
-    import helpers as hp
+    from oracle import Adapter, Oracle
     orc = Oracle("f64")
     shape, b = w.shape, w.batch
+    ads = [Adapter(a.rank, a.scale, a.Aq, a.Bq, a.Ak, a.Bk, a.Av, a.Bv) for a in w.adapters]
     total_s, done = 0.0, 0
     for r in requests:
         P = int(b.prefix_lens[r])
@@ -133,7 +135,8 @@ def oracle_sample_rate(w: wl.Workload, pool_np: np.ndarray, n_tokens: int, reque
                        activation_offsets=b.activation_offsets[r:r + 1], adapter_ids=b.adapter_ids[r:r + 1],
                        block_tables=b.block_tables[r:r + 1], num_pages=b.num_pages, hidden=b.hidden[q0:q0 + n])
         t0 = time.perf_counter()
-        hp.oracle_block(orc, shape, w.wqkv, w.adapters, sub, [K0], [V0])
+        orc.attention_block(sub.hidden, w.wqkv, shape.Nq, shape.Nkv, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
+                            sub.positions, sub.query_start_loc, sub.activation_offsets, sub.adapter_ids, ads, [K0], [V0])
         total_s += time.perf_counter() - t0
         done += n
         if total_s > budget_s:
@@ -167,6 +170,49 @@ def run_reference(args):
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": threads, "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
+
+
+def launch_ranks(n: int) -> int:
+    """`python bench.py --gpus N` without a launcher: start N ranks of this script on this node (one per GPU) under
+    torch.distributed.run, with the same arguments, and pass their exit status on."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), os.path.abspath(__file__)] + sys.argv[1:]
+    rc = subprocess.call(cmd)
+    if rc != 0:
+        sys.exit(rc)
+    return rc
+
+
+def dry_run(args, world: int, rank: int) -> None:
+    """The multi-rank plumbing without a GPU: every rank joins the process group, takes its share of a request
+    partition and its batch seed, the ranks agree on a (made-up) per-rank time by barrier + max over ranks, and rank
+    0 prints the JSON line with the number of ranks that really took part.  Nothing is measured."""
+    import torch
+    import torch.distributed as dist
+    if world > 1:
+        dist.init_process_group(args.backend)
+    try:
+        lo, hi = sharding.partition_requests(args.requests * world, world)[rank]
+        fake_ms = 1.0 + rank
+        if world > 1:
+            dist.barrier()
+        ms = sharding.max_over_ranks(fake_ms)
+        took_part = torch.ones(1, dtype=torch.int64)
+        if world > 1:
+            dist.all_reduce(took_part)
+        if rank == 0:
+            print(json.dumps({"metric": METRIC, "value": None, "unit": UNIT, "n_gpus": int(took_part.item()),
+                              "steps": args.steps, "warmup": args.warmup, "ms_per_step": ms, "scaling": "weak",
+                              "dry_run": True, "backend": args.backend if world > 1 else None,
+                              "config": {"workload": WORKLOAD, "requests_per_gpu": hi - lo,
+                                         "rank_seeds": [sharding.rank_seed(SEED, r) for r in range(world)]}}))
+    finally:
+        if world > 1:
+            dist.destroy_process_group()
 
 
 def _events(n):
@@ -547,22 +593,31 @@ def main():
     ap.add_argument("--requests", type=int, default=8)
     ap.add_argument("--prefix", type=int, default=4096)
     ap.add_argument("--suffix", type=int, default=256)
+    ap.add_argument("--backend", default="nccl", help="process-group backend of a multi-rank run (gloo with --dry-run)")
+    ap.add_argument("--dry-run", action="store_true",
+                    help="exercise the multi-rank launch, barrier and max-over-ranks without touching a GPU")
     args = ap.parse_args()
     if args.impl == "reference":
         return run_reference(args)
 
-    import torch
-    import helpers as hp
-    from paper_2504_12397_b200 import binding as ab
-    from paper_2504_12397_b200.build import build_library
-    build_library()
-
+    if "WORLD_SIZE" not in os.environ and args.gpus > 1:
+        return launch_ranks(args.gpus)
     world = int(os.environ.get("WORLD_SIZE", "1"))
     rank = int(os.environ.get("RANK", "0"))
     local = int(os.environ.get("LOCAL_RANK", "0"))
+    if args.dry_run:
+        return dry_run(args, world, rank)
+
+    import torch
+    from paper_2504_12397_b200 import binding as ab
+    from paper_2504_12397_b200 import device as hp
+    from paper_2504_12397_b200.build import build_library
+    build_library()
+
     torch.cuda.set_device(local)
     if world > 1:
         import torch.distributed as dist
+        os.environ.setdefault("NCCL_DEBUG", "INFO")   # the communicator lines (transport, NVLS) go to stderr
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
 
     def barrier():

@@ -52,10 +52,12 @@ typedef struct alora_ctx alora_ctx;
 
 typedef enum alora_status {
     ALORA_OK = 0,
-    ALORA_ERR_INVALID_ARG = 1,   /* null pointer, negative size, misaligned pointer            */
+    ALORA_ERR_INVALID_ARG = 1,   /* null pointer, negative size, misaligned pointer, T > 0 with R == 0 */
     ALORA_ERR_UNSUPPORTED = 2,   /* shape or dtype the kernels are not built for               */
     ALORA_ERR_CAPACITY = 3,      /* T, R, rank or adapter id beyond what alora_create was told */
-    ALORA_ERR_NO_WEIGHTS = 4,    /* layer weights or a referenced adapter were never set       */
+    ALORA_ERR_NO_WEIGHTS = 4,    /* layer weights never set (return value); or, as a device finding,
+                                    a row whose gate is open names an adapter that was never
+                                    registered on the layer: that row gets the base projection  */
     ALORA_ERR_CUDA = 5,          /* a CUDA runtime/driver call failed (see alora_last_cuda_error) */
     ALORA_ERR_BAD_BATCH = 6,     /* batch metadata inconsistent (host validation or device check) */
     ALORA_ERR_PAGE_RANGE = 7,    /* a block-table entry is outside [0, num_pages)              */
@@ -224,6 +226,9 @@ alora_status alora_full_lora_prefill_layer(alora_ctx *ctx, int layer, const void
  * * up) of norm(h)), adapters on q/k/v only, MLP and o_proj with base weights.  d_paged_kv_layers
  * is a HOST array of n_layers device pointers (one pool per layer, same block tables).
  * d_hidden_in[T][H] -> d_hidden_out[T][H] (may alias).  `mode` selects Eq. 5 / Eq. 4 / Eq. 2.
+ * A step whose shape the kernels do not serve (for the tensor-core path: hidden, Nq or intermediate not a
+ * multiple of 8) or whose launch fails ends the call there with ALORA_ERR_UNSUPPORTED / ALORA_ERR_CUDA; the
+ * steps before it have been enqueued and d_hidden_out then holds an unfinished residual stream.
  */
 alora_status alora_forward_stack(alora_ctx *ctx, int mode, const void *d_hidden_in,
                                  const int32_t *d_positions, const int32_t *d_activation_offsets,
@@ -280,6 +285,16 @@ alora_status alora_project_qkv_static(int dtype, int hidden, int n_q, int n_kv, 
                                       const int32_t *d_adapter_on, int rank, float scale, const void *d_Aq,
                                       const void *d_Bq, const void *d_Ak, const void *d_Bk, const void *d_Av,
                                       const void *d_Bv, int T, int R, void *d_qkv, void *stream);
+
+/*
+ * Self-test of the bounded waits (the paper has no counterpart).  Every wait inside the tensor-core kernels
+ * (on a shared-memory barrier, on another block's ready counter) gives up after a cycle limit, records
+ * ALORA_ERR_TIMEOUT in the status word and lets the kernel return through its normal exit.  This call runs that
+ * give-up path on purpose and harmlessly: one block of one warp waits on a barrier that nobody arrives at, with
+ * the given limit (1 .. 200 000 000 clock cycles, i.e. at most about 0.1 s), then returns.  Afterwards
+ * alora_get_status reads ALORA_ERR_TIMEOUT (and clears it); the context remains usable.  Asynchronous on `stream`.
+ */
+alora_status alora_selftest_wait_timeout(alora_ctx *ctx, int64_t limit_cycles, void *stream);
 
 /*
  * Optional per-kernel timing (a measurement aid; the paper has no counterpart).  While enabled,

@@ -240,6 +240,13 @@ def alora_get_status(ctx, stream=None) -> int:
     return int(out.value)
 
 
+def alora_selftest_wait_timeout(ctx, limit_cycles: int, stream=None) -> None:
+    f = load_library().alora_selftest_wait_timeout
+    f.argtypes = [C.c_void_p, C.c_int64, _VP]
+    f.restype = C.c_int
+    _check(ctx, f(ctx, int(limit_cycles), _stream(stream)), "alora_selftest_wait_timeout")
+
+
 def alora_launch_count(ctx) -> int:
     return int(load_library().alora_launch_count(ctx))
 

@@ -51,6 +51,7 @@ static bool aligned16(const void *p) { return (reinterpret_cast<uintptr_t>(p) & 
 static alora_status check_batch_args(alora_ctx *ctx, int T, int R) {
     if (!ctx) return ALORA_ERR_INVALID_ARG;
     if (T < 0 || R < 0) return ALORA_ERR_INVALID_ARG;
+    if (T > 0 && R == 0) return ALORA_ERR_INVALID_ARG;   // tokens that belong to no request
     if (T > ctx->cfg.max_tokens || R > ctx->cfg.max_requests) return ALORA_ERR_CAPACITY;
     return ALORA_OK;
 }
@@ -64,10 +65,12 @@ static alora_status finish(alora_ctx *ctx, int launched) {
 }
 
 // Steps 1-3 of one layer, in the order of Prop. 2's proof.
-static alora_status run_layer(alora_ctx *ctx, int layer, const void *hidden, const BatchArgs &b, void *pool,
+static alora_status run_layer(alora_ctx *ctx, int layer, const void *hidden, const BatchArgs &b_in, void *pool,
                               void *attn_out, cudaStream_t s) {
     if (layer < 0 || layer >= ctx->cfg.n_layers) return ALORA_ERR_INVALID_ARG;
     if (!ctx->layers[layer].wqkv) return ALORA_ERR_NO_WEIGHTS;
+    BatchArgs b = b_in;
+    b.layer = layer;
     int n = 0, k;
     if ((k = launch_metadata(ctx, b, s)) < 0) return ALORA_ERR_UNSUPPORTED; n += k;
     bool kv_appended = false;
@@ -168,6 +171,7 @@ alora_status alora_create(const alora_config *cfg, alora_ctx **out) {
     alloc(&ctx->d_t, Tm * 3 * d.RP * 4);
     alloc(&ctx->d_qkv, Tm * d.N * es);
     alloc((void **)&ctx->d_status, 4);
+    alloc((void **)&ctx->d_iota, ((size_t)c.max_requests + 1) * 4);   // 0, 1, ..: query_start_loc of a decode batch
     ctx->layer_has_adapter.assign(c.n_layers, 0);
     if (c.dtype == ALORA_DTYPE_BF16 && 128 % d.G == 0) {
         // tensor-core attention: one work item per (request, KV head, block of 2 * 128/G tokens)
@@ -230,6 +234,11 @@ alora_status alora_create(const alora_config *cfg, alora_ctx **out) {
         e = cudaMemset(ctx->d_status, 0, 4);
         if (e == cudaSuccess) e = cudaMemset(ctx->d_adapters, 0, n_ad * sizeof(AdapterDev));
         if (e == cudaSuccess) e = cudaMemset(ctx->d_counts, 0, 64);
+        if (e == cudaSuccess) {
+            std::vector<int32_t> iota((size_t)c.max_requests + 1);
+            for (size_t i = 0; i < iota.size(); ++i) iota[i] = (int32_t)i;
+            e = cudaMemcpy(ctx->d_iota, iota.data(), iota.size() * 4, cudaMemcpyHostToDevice);
+        }
         if (e != cudaSuccess) st = cuda_fail(ctx, e, "cudaMemset");
     }
     if (st != ALORA_OK) { alora_destroy(ctx); return st; }
@@ -388,6 +397,7 @@ alora_status alora_project_qkv(alora_ctx *ctx, int layer, int mode, const void *
     ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
     const int32_t *d_block_tables = nullptr; const int max_blocks = 0, num_pages = 0;
     ALORA_BATCH(mode);
+    b.layer = layer;
     int n = launch_metadata(ctx, b, s), k;
     if ((k = launch_project(ctx, layer, d_hidden, T, d_qkv, s, nullptr, 0, nullptr)) < 0) return ALORA_ERR_UNSUPPORTED;
     return finish(ctx, n + k);
@@ -406,9 +416,9 @@ alora_status alora_kv_append(alora_ctx *ctx, const void *d_qkv, const int32_t *d
     ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
     const int32_t *d_activation_offsets = nullptr, *d_adapter_ids = nullptr;
     ALORA_BATCH(ALORA_MODE_BASE);
-    int n = launch_metadata(ctx, b, s);
-    n += launch_kv_append(ctx, d_qkv, T, num_pages, d_paged_kv, s);
-    return finish(ctx, n);
+    int n = launch_metadata(ctx, b, s), k;
+    if ((k = launch_kv_append(ctx, d_qkv, T, num_pages, d_paged_kv, s)) < 0) return ALORA_ERR_UNSUPPORTED;
+    return finish(ctx, n + k);
 }
 
 alora_status alora_attend(alora_ctx *ctx, const void *d_qkv, const int32_t *d_positions,
@@ -477,14 +487,7 @@ alora_status alora_decode_step(alora_ctx *ctx, int layer, const void *d_hidden, 
     if (!ctx) return ALORA_ERR_INVALID_ARG;
     if (R < 0) return ALORA_ERR_INVALID_ARG;
     if (R > ctx->cfg.max_requests || R > ctx->cfg.max_tokens) return ALORA_ERR_CAPACITY;
-    // query_start_loc of a decode batch is 0, 1, ..., R: kept in the context, built on first use
-    ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
-    if (!ctx->d_iota) {
-        std::vector<int32_t> iota((size_t)ctx->cfg.max_requests + 1);
-        for (size_t i = 0; i < iota.size(); ++i) iota[i] = (int32_t)i;
-        ALORA_CUDA(ctx, cudaMalloc((void **)&ctx->d_iota, iota.size() * 4));
-        ALORA_CUDA(ctx, cudaMemcpy(ctx->d_iota, iota.data(), iota.size() * 4, cudaMemcpyHostToDevice));
-    }
+    // query_start_loc of a decode batch is 0, 1, ..., R: kept in the context since alora_create
     return layer_entry(ctx, layer, ALORA_MODE_ALORA, d_hidden, d_positions, d_activation_offsets, d_adapter_ids,
                        ctx->d_iota, d_seq_lens, d_paged_kv, d_block_tables, max_blocks, num_pages, R, R, d_attn_out,
                        stream, /*one_token_per_request=*/true);
@@ -515,23 +518,35 @@ alora_status alora_forward_stack(alora_ctx *ctx, int mode, const void *d_hidden_
     if (d_hidden_out != d_hidden_in && T > 0)
         ALORA_CUDA(ctx, cudaMemcpyAsync(d_hidden_out, d_hidden_in, (size_t)T * d.H * ctx->esize, cudaMemcpyDeviceToDevice, s));
     char *h = (char *)d_hidden_out;  // residual stream, updated in place
-    int n = 0;
+    int n = 0, k;
+    // a launcher that returns < 0 has launched nothing (unsupported shape, failed tensor map or launch): the call
+    // stops there with the residual stream as the completed steps left it
+#define ALORA_STEP(call)                                                          \
+    do {                                                                          \
+        if ((k = (call)) < 0) {                                                   \
+            ctx->launches += n;                                                   \
+            cudaError_t e__ = cudaGetLastError();                                 \
+            return e__ != cudaSuccess ? cuda_fail(ctx, e__, #call) : ALORA_ERR_UNSUPPORTED; \
+        }                                                                         \
+        n += k;                                                                   \
+    } while (0)
     for (int l = 0; l < ctx->cfg.n_layers; ++l) {
         const LayerWeights &lw = ctx->layers[l];
-        n += launch_rmsnorm(ctx, h, lw.norm_attn, T, ctx->d_act[0], s);
+        ALORA_STEP(launch_rmsnorm(ctx, h, lw.norm_attn, T, ctx->d_act[0], s));
         st = run_layer(ctx, l, ctx->d_act[0], b, h_paged_kv_layers[l], ctx->d_act[1], s);
         if (st != ALORA_OK) return st;
-        n += launch_linear(ctx, ctx->d_act[1], lw.wo, T, d.Nq, d.H, h, h, s);           // h += o_proj(attn)
-        n += launch_rmsnorm(ctx, h, lw.norm_mlp, T, ctx->d_act[0], s);
+        ALORA_STEP(launch_linear(ctx, ctx->d_act[1], lw.wo, T, d.Nq, d.H, h, h, s));           // h += o_proj(attn)
+        ALORA_STEP(launch_rmsnorm(ctx, h, lw.norm_mlp, T, ctx->d_act[0], s));
         for (int t0 = 0; t0 < T; t0 += kMlpChunk) {                                        // MLP, token chunks
             const int tc = std::min(kMlpChunk, T - t0);
             const char *xm = (const char *)ctx->d_act[0] + (size_t)t0 * d.H * ctx->esize;
             char *hc = h + (size_t)t0 * d.H * ctx->esize;
-            n += launch_linear(ctx, xm, lw.wgate_up, tc, d.H, 2 * d.I, ctx->d_act[2], nullptr, s);
-            n += launch_swiglu(ctx, ctx->d_act[2], tc, ctx->d_act[3], s);
-            n += launch_linear(ctx, ctx->d_act[3], lw.wdown, tc, d.I, d.H, hc, hc, s);  // h += down(...)
+            ALORA_STEP(launch_linear(ctx, xm, lw.wgate_up, tc, d.H, 2 * d.I, ctx->d_act[2], nullptr, s));
+            ALORA_STEP(launch_swiglu(ctx, ctx->d_act[2], tc, ctx->d_act[3], s));
+            ALORA_STEP(launch_linear(ctx, ctx->d_act[3], lw.wdown, tc, d.I, d.H, hc, hc, s));  // h += down(...)
         }
     }
+#undef ALORA_STEP
     return finish(ctx, n);
 }
 

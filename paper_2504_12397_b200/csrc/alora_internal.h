@@ -207,6 +207,7 @@ struct BatchArgs {
     const int32_t *positions, *activation_offsets, *adapter_ids, *query_start_loc, *seq_lens, *block_tables;
     int max_blocks, num_pages, T, R, mode;
     int all_small;  // host-side knowledge that no request has more than small_max_tokens new tokens (decode)
+    int layer = -1; // layer whose adapter table the gate is checked against (-1: no check)
 };
 
 int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s);

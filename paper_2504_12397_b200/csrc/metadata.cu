@@ -25,8 +25,8 @@ __device__ __forceinline__ int find_request(const int32_t *qsl, int R, int t) {
 // Per token: request index, adapter applied to the row (the gate of Eq. 5: position >= activation
 // offset; always open in full-LoRA mode, always closed in base mode), and the token slot
 // page * page_size + position % page_size.  Findings (inconsistent positions, page id out of
-// range, adapter id out of range) go to the status word; the row then gets adapter -1 / slot -1 so
-// that later kernels skip it.
+// range, adapter id out of range, an open gate on an adapter that was never registered on the layer) go
+// to the status word; the row then gets adapter -1 / slot -1 so that later kernels skip it.
 __device__ __forceinline__ void metadata_tokens(const int32_t *__restrict__ positions,
                                       const int32_t *__restrict__ a_req,
                                       const int32_t *__restrict__ adapter_ids,
@@ -34,7 +34,8 @@ __device__ __forceinline__ void metadata_tokens(const int32_t *__restrict__ posi
                                       const int32_t *__restrict__ block_tables, int max_blocks,
                                       int num_pages, int page_size, int max_adapters, int T, int R, int mode,
                                       int32_t *__restrict__ token_req, int32_t *__restrict__ row_adapter,
-                                      int32_t *__restrict__ slot_map, int32_t *status) {
+                                      int32_t *__restrict__ slot_map, const AdapterDev *__restrict__ adapters,
+                                      int32_t *status) {
     int t = blockIdx.x * blockDim.x + threadIdx.x;
     if (t >= T) return;
     int r = find_request(qsl, R, t);
@@ -48,6 +49,8 @@ __device__ __forceinline__ void metadata_tokens(const int32_t *__restrict__ posi
         k = adapter_ids[r];
         if (k >= max_adapters || k < -1) { report(status, ALORA_ERR_BAD_BATCH); k = -1; }
         if (k >= 0 && mode == ALORA_MODE_ALORA && p < a_req[r]) k = -1;
+        // a row whose gate is open needs its adapter's weights on this layer
+        if (k >= 0 && adapters != nullptr && adapters[k].rank == 0) { report(status, ALORA_ERR_NO_WEIGHTS); k = -1; }
     }
     if (token_req) token_req[t] = r;
     if (row_adapter) row_adapter[t] = ok ? k : -1;
@@ -463,7 +466,7 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *a_req, con
                 int G, int n_sm, int small_max, int max_split_items, int max_split_rows,
                 AttnSplitWork *__restrict__ split_items,
                 int32_t *req_scratch, int32_t *__restrict__ group_done, int rowwise_cap,
-                int32_t *__restrict__ attn_cta_start, int32_t *status) {
+                int32_t *__restrict__ attn_cta_start, const AdapterDev *__restrict__ adapters, int32_t *status) {
     // The per-request inputs are read many times (binary searches, list builders): one parallel pass stages them
     // in shared memory, so that the later steps do not each pay a round trip to global memory.
     __shared__ int32_t s_req[4 * kMetaStageR + 1];
@@ -482,7 +485,7 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *a_req, con
         if (a_req) a_req = s_areq;
     }
     metadata_tokens(positions, a_req, adapter_ids, qsl, seq_lens, block_tables, max_blocks, num_pages, page_size,
-                    max_adapters, T, R, mode, token_req, row_adapter, slot_map, status);
+                    max_adapters, T, R, mode, token_req, row_adapter, slot_map, adapters, status);
     // The three list builders are independent of one another: blocks 0, 1 and 2 take one each (a launch has at least
     // three blocks; with fewer, block 0 would run them one after the other).
     const int nb = (int)gridDim.x;
@@ -523,7 +526,8 @@ int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s) {
         ctx->d.Hkv, ctx->attn_q_block, ctx->max_attn_items, ctx->d_attn_items, ctx->d_attn_off, ctx->d.G,
         ctx->sm_count, ctx->small_max_tokens, ctx->max_split_items, ctx->max_split_rows, ctx->d_split_items,
         ctx->d_req_scratch, ctx->d_group_done, ctx->d_row_delta ? kRowwiseMaxTokens : 0,
-        ctx->d_attn_cta_start, ctx->d_status);
+        ctx->d_attn_cta_start,
+        b.layer >= 0 ? ctx->d_adapters + (size_t)b.layer * ctx->cfg.max_adapters : nullptr, ctx->d_status);
     return 1;
 }
 

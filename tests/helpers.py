@@ -4,100 +4,81 @@ from __future__ import annotations
 
 import numpy as np
 
-from paper_2504_12397_b200 import binding as ab
+from paper_2504_12397_b200 import binding as ab  # noqa: F401
 from paper_2504_12397_b200 import workloads as wl
+from paper_2504_12397_b200.device import DevBatch, GpuLayers, idev, to_dev, to_host  # noqa: F401
 
 
 def rel_err(got: np.ndarray, want: np.ndarray) -> float:
     """Tensor-max-normalised error: max|got - want| / max|want|."""
     want = np.asarray(want, np.float64)
     got = np.asarray(got, np.float64)
-    denom = np.abs(want).max()
-    return float(np.abs(got - want).max() / (denom if denom > 0 else 1.0))
+    denom = np.abs(want).max() if want.size else 0.0
+    return float(np.abs(got - want).max() / (denom if denom > 0 else 1.0)) if want.size else 0.0
+
+
+def rel_err_elementwise(got: np.ndarray, want: np.ndarray) -> float:
+    """Second measure: max over elements of |got - want| / (|want| + 1e-2 * rms(want)).  Every element is
+    judged against its own magnitude, with a floor of one percent of the tensor's rms so that elements
+    near zero do not divide by nothing."""
+    want = np.asarray(want, np.float64)
+    got = np.asarray(got, np.float64)
+    if not want.size:
+        return 0.0
+    rms = float(np.sqrt(np.mean(want * want)))
+    return float((np.abs(got - want) / (np.abs(want) + 1e-2 * (rms if rms > 0 else 1.0))).max())
+
+
+def rel_err_blocks(got: np.ndarray, want: np.ndarray, block: int) -> float:
+    """Third measure: the tensor-max-normalised error taken separately for every (row, block of `block`
+    columns) -- one head of one token -- so that a head or a token of small magnitude cannot hide behind a
+    large one elsewhere in the tensor.  Blocks whose expected values are all below 1e-3 of the tensor's
+    maximum are normalised by that floor instead."""
+    want = np.asarray(want, np.float64)
+    got = np.asarray(got, np.float64)
+    if not want.size:
+        return 0.0
+    T, N = want.shape
+    assert N % block == 0
+    w = np.abs(want).reshape(T, N // block, block).max(axis=2)
+    d = np.abs(got - want).reshape(T, N // block, block).max(axis=2)
+    floor = 1e-3 * np.abs(want).max()
+    return float((d / np.maximum(w, floor if floor > 0 else 1.0)).max())
+
+
+# Bounds of the three measures for bf16 results against the fp64 oracle.  The first is the method's stated
+# bound.  The other two judge single elements or single heads: an element's error is that of a bf16 rounding
+# of the output (2^-9 relative) plus the accumulated operand roundings, which do not shrink with the element, so
+# elements far below the tensor's rms see a larger relative error; the elementwise floor (1e-2 rms) and the bound
+# below leave room for exactly that and nothing more: a wrong head, row or block is off by O(1).
+TOL_ELEMENTWISE_BF16 = 0.5
+TOL_BLOCKS_BF16 = 6e-2
+
+
+WORST = {}   # largest value of each measure seen in this session, per data type (printed by conftest at the end)
+
+
+def assert_close(got, want, shape_or_tol, what: str = "", block: int = 0):
+    """All parity assertions go through here: the stated tensor-wide bound, plus the elementwise and (when a
+    block width is given) per-(row, head) measures.  Returns the three figures for reporting."""
+    tol_ = shape_or_tol if isinstance(shape_or_tol, float) else tol(shape_or_tol)
+    bf16 = tol_ > 1e-3
+    e1 = rel_err(got, want)
+    e2 = rel_err_elementwise(got, want)
+    e3 = rel_err_blocks(got, want, block) if block else 0.0
+    rec = WORST.setdefault("bf16" if bf16 else "fp32", [0.0, 0.0, 0.0])
+    rec[0], rec[1], rec[2] = max(rec[0], e1), max(rec[1], e2), max(rec[2], e3)
+    assert e1 <= tol_, f"{what}: max|d|/max|want| = {e1:.3e} > {tol_:g}"
+    assert e2 <= (TOL_ELEMENTWISE_BF16 if bf16 else 1e-3), f"{what}: elementwise measure {e2:.3e}"
+    if block:
+        assert e3 <= (TOL_BLOCKS_BF16 if bf16 else 1e-4), f"{what}: per-(row, head) measure {e3:.3e}"
+    return e1, e2, e3
 
 
 def tol(shape: wl.LayerShape) -> float:
     # bf16: the method's stated bound; fp32: H-length fp32 dot products err by about sqrt(H) * 2^-24 ~ 1e-6
     # relative, taken with a tenfold margin
     return 2e-2 if shape.dtype == "bf16" else 1e-5
-
-
-def to_dev(a: np.ndarray, dtype: str):
-    import torch
-    t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.float32)).cuda()
-    return t.to(torch.bfloat16).contiguous() if dtype == "bf16" else t.contiguous()
-
-
-def to_host(t) -> np.ndarray:
-    import torch
-    return t.detach().to(torch.float32).cpu().numpy()
-
-
-def idev(a):
-    import torch
-    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).cuda()
-
-
-class GpuLayers:
-    """A context plus device copies of weights/adapters for `n_layers` layers of one shape."""
-
-    def __init__(self, shape: wl.LayerShape, layer_weights, adapters_per_layer, max_tokens, max_requests,
-                 n_adapters=None):
-        import torch
-        self.shape = shape
-        self.n_layers = len(layer_weights)
-        n_ad = n_adapters if n_adapters is not None else max([len(a) for a in adapters_per_layer] + [1])
-        max_rank = max([a.rank for per in adapters_per_layer for a in per] + [8])
-        self.cfg = ab.make_config(
-            hidden=shape.hidden, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads, head_dim=shape.head_dim,
-            page_size=shape.page_size, n_layers=self.n_layers, intermediate=shape.intermediate if "wo" in layer_weights[0] else 0,
-            max_adapters=n_ad, max_rank=max_rank, dtype=ab.DTYPE_BF16 if shape.dtype == "bf16" else ab.DTYPE_FP32,
-            max_tokens=max_tokens, max_requests=max_requests)
-        self.ctx = ab.alora_create(self.cfg)
-        self.keep = []
-        for l, lw in enumerate(layer_weights):
-            dev = {k: to_dev(v, shape.dtype) for k, v in lw.items()}
-            self.keep.append(dev)
-            ab.alora_set_layer_weights(self.ctx, l, dev["wqkv"], dev.get("wo"), dev.get("wgate_up"), dev.get("wdown"),
-                                       dev.get("norm_attn"), dev.get("norm_mlp"))
-            for i, a in enumerate(adapters_per_layer[l]):
-                mats = [to_dev(getattr(a, n), shape.dtype) for n in ("Aq", "Bq", "Ak", "Bk", "Av", "Bv")]
-                ab.alora_register_adapter(self.ctx, i, l, a.rank, a.scale, *mats)
-        torch.cuda.synchronize()
-        self.torch_dtype = torch.bfloat16 if shape.dtype == "bf16" else torch.float32
-
-    def close(self):
-        if self.ctx:
-            ab.alora_destroy(self.ctx)
-            self.ctx = None
-
-    def new_pool(self, num_pages, fill=None):
-        import torch
-        s = self.shape
-        if fill is None:
-            return torch.zeros((num_pages, 2, s.n_kv_heads, s.page_size, s.head_dim), dtype=self.torch_dtype, device="cuda")
-        return to_dev(fill, s.dtype)
-
-    def empty(self, *shape):
-        import torch
-        return torch.empty(shape, dtype=self.torch_dtype, device="cuda")
-
-    def status(self) -> int:
-        return ab.alora_get_status(self.ctx)
-
-
-class DevBatch:
-    def __init__(self, b: wl.Batch, dtype: str):
-        self.b = b
-        self.positions = idev(b.positions)
-        self.qsl = idev(b.query_start_loc)
-        self.seq_lens = idev(b.seq_lens)
-        self.a_req = idev(b.activation_offsets)
-        self.ids = idev(b.adapter_ids)
-        self.bt = idev(b.block_tables)
-        self.max_blocks = b.block_tables.shape[1]
-        self.hidden = to_dev(b.hidden, dtype) if b.hidden is not None else None
-        self.T, self.R = b.T, b.R
 
 
 def full_sequence_batch(shape: wl.LayerShape, b: wl.Batch) -> wl.Batch:

@@ -50,11 +50,13 @@ def _check_requests(oracle, shape, w, b, pool_before, pool_after, out_h, sample,
         K0, V0 = _request_kv(pool_before, b, r, P, shape)
         q0, q1, sub = _sub_batch(b, r)
         want = hp.oracle_block(oracle, shape, w.wqkv, w.adapters, sub, [K0 if P else None], [V0 if P else None])
-        assert hp.rel_err(out_h[q0:q1], want["out"]) <= 2e-2, f"attention output of request {r}"
+        hd = shape.head_dim
+        hp.assert_close(out_h[q0:q1], want["out"], 2e-2, f"attention output of request {r}", block=hd)
         if qkv_h is not None:
-            assert hp.rel_err(qkv_h[q0:q1], want["qkv"]) <= 2e-2, f"projection rows of request {r}"
+            hp.assert_close(qkv_h[q0:q1], want["qkv"], 2e-2, f"projection rows of request {r}", block=hd)
         K1, V1 = _request_kv(pool_after, b, r, L, shape)
-        assert hp.rel_err(K1[P:], want["K"][0][P:]) <= 2e-2 and hp.rel_err(V1[P:], want["V"][0][P:]) <= 2e-2
+        hp.assert_close(K1[P:], want["K"][0][P:], 2e-2, f"appended K rows of request {r}", block=hd)
+        hp.assert_close(V1[P:], want["V"][0][P:], 2e-2, f"appended V rows of request {r}", block=hd)
         # the cached prefix of the request is untouched, bit for bit
         assert np.array_equal(K1[:P].view(np.uint32), K0.view(np.uint32))
         assert np.array_equal(V1[:P].view(np.uint32), V0.view(np.uint32))
@@ -88,22 +90,32 @@ def _run_layer(w, seed, decode=False, with_qkv=False):
 
 
 def test_config2_bench_workload_sampled_requests(oracle64):
-    """8 requests x (4096 cached + 256 suffix tokens), rank 32: requests 0 and 7 in full."""
+    """8 requests x (4096 cached + 256 suffix tokens), rank 32: the whole workload, every row of every request."""
     w = wl.config2(seed=2)
     before, after, out_h, qkv_h = _run_layer(w, seed=1002, with_qkv=True)
-    _check_requests(oracle64, w.shape, w, w.batch, before, after, out_h, [0, 7], qkv_h)
+    _check_requests(oracle64, w.shape, w, w.batch, before, after, out_h, range(w.batch.R), qkv_h)
 
 
 def test_config3_ragged_multi_adapter_sampled_requests(oracle64):
     """32 requests over adapters of ranks 8/16/32/64, prefixes 512..16384, suffixes 16..512, shuffled pages:
-    the two requests with the least oracle work and the one with the shortest suffix, in full."""
+    in full, the request with the most work (longest suffix x context), the request with the most work on the
+    rank-64 adapter and on the rank-8 adapter, the two with the least work and the one with the shortest suffix;
+    and the projection rows of the whole batch."""
     w = wl.config3(seed=3)
     b = w.batch
     S = (b.seq_lens - b.prefix_lens).astype(np.int64)
     work = S * b.seq_lens.astype(np.int64)
-    sample = sorted(set(list(np.argsort(work)[:2]) + [int(np.argmin(S))]))
-    before, after, out_h, _ = _run_layer(w, seed=1003)
-    _check_requests(oracle64, w.shape, w, b, before, after, out_h, sample)
+    by_work = np.argsort(work)
+    sample = {int(by_work[-1]), int(by_work[0]), int(by_work[1]), int(np.argmin(S))}
+    for ad in (0, 3):   # ranks 8 and 64
+        on = np.nonzero(b.adapter_ids == ad)[0]
+        assert len(on) > 0
+        sample.add(int(on[np.argmax(work[on])]))
+    before, after, out_h, qkv_h = _run_layer(w, seed=1003, with_qkv=True)
+    _check_requests(oracle64, w.shape, w, b, before, after, out_h, sorted(sample), qkv_h)
+    want, gate = oracle64.project_qkv(b.hidden, w.wqkv, w.shape.Nq, w.shape.Nkv, b.positions, b.query_start_loc,
+                                      b.activation_offsets, b.adapter_ids, hp.oracle_adapters(w.adapters))
+    hp.assert_close(qkv_h, want, 2e-2, "projection rows of the whole batch", block=w.shape.head_dim)
 
 
 def test_long_uniform_batch_whole_items_and_cut_items(oracle64):
@@ -240,5 +252,69 @@ def test_config5_decode_step_sampled_requests(oracle64):
     _check_requests(oracle64, w.shape, w, b, before, after, out_h, sample, qkv_h)
     want, gate = oracle64.project_qkv(b.hidden, w.wqkv, w.shape.Nq, w.shape.Nkv, b.positions, b.query_start_loc,
                                       b.activation_offsets, b.adapter_ids, hp.oracle_adapters(w.adapters))
-    assert hp.rel_err(qkv_h, want) <= 2e-2
+    hp.assert_close(qkv_h, want, 2e-2, "")
     assert gate.sum() > 0 and (gate == 0).sum() > 0
+
+
+def test_config4_size_layer_one_request_and_cache_reuse_identity(oracle64):
+    """One 8B-shape layer at the size of the 32-layer stack workload: 4 requests x (32768 cached + 1024 suffix
+    tokens).  The base model's cache is made on the GPU by a base prefill of the prefix hidden states (131072
+    tokens).  (i) The suffix prefill on that cache takes the long-batch attention route (whole items, then items
+    cut into runs and merged) at head dim 128 and group size 4; every row of the last request, which holds the cut
+    items, and of the first request is compared with the oracle, which is given the layer's own input and that
+    request's cache rows read back from the pool.  (ii) The cache-reuse identity between two GPU runs at this
+    size: a masked prefill of all 33792 tokens per request from scratch (gate closed before position 32768) must
+    leave bit-identical K/V for the prefix positions and suffix outputs within the tolerance."""
+    import torch
+    shape = wl.SHAPE_8B
+    R, P, S = 4, 32768, 1024
+    rng = np.random.default_rng(4)
+    wqkv = wl.make_wqkv(shape, rng)
+    ads = [wl.make_adapter(shape, 32, rng)]
+    b = wl.make_batch(shape, [P] * R, [S] * R, [0] * R, rng, shuffle_pages=True)
+    w = wl.Workload("config4_layer", shape, wqkv, ads, b, 4)
+    full_T = R * (P + S)
+    g = hp.GpuLayers(shape, [dict(wqkv=wqkv)], [ads], full_T, R)
+    try:
+        gen = torch.Generator(device="cuda"); gen.manual_seed(44)
+        # prefix hidden states drawn on the device (bf16-rounded N(0,1)); the suffix rows come from the workload
+        hid_full = torch.randn((full_T, shape.hidden), generator=gen, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        d = hp.DevBatch(b, "bf16")
+        for r in range(R):
+            hid_full[r * (P + S) + P:(r + 1) * (P + S)] = d.hidden[r * S:(r + 1) * S]
+        pre_rows = torch.cat([torch.arange(r * (P + S), r * (P + S) + P, device="cuda") for r in range(R)])
+        hid_pre = hid_full[pre_rows].contiguous()
+        i32 = lambda a: hp.idev(np.ascontiguousarray(a, np.int32))   # noqa: E731
+        pos_pre, qsl_pre = i32(np.tile(np.arange(P), R)), i32(np.arange(R + 1) * P)
+        pos_full, qsl_full = i32(np.tile(np.arange(P + S), R)), i32(np.arange(R + 1) * (P + S))
+        base_ids, len_pre = i32(np.full(R, -1)), i32(np.full(R, P))
+        # run A: base prefill of the prefixes, then the aLoRA suffix prefill on that cache
+        pool_a = g.new_pool(b.num_pages)
+        scratch = g.empty(R * P, shape.Nq)
+        ab.alora_full_lora_prefill_layer(g.ctx, 0, hid_pre, pos_pre, base_ids, qsl_pre, len_pre, pool_a, d.bt,
+                                         d.max_blocks, b.num_pages, R * P, R, scratch)
+        del scratch
+        before = pool_a.clone()
+        out_a = g.empty(b.T, shape.Nq)
+        ab.alora_prefill_layer(g.ctx, 0, d.hidden, d.positions, d.a_req, d.ids, d.qsl, d.seq_lens, pool_a, d.bt,
+                               d.max_blocks, b.num_pages, b.T, R, out_a)
+        assert g.status() == 0
+        out_a_h = hp.to_host(out_a)
+        _check_requests(oracle64, shape, w, b, before, pool_a, out_a_h, [0, R - 1])
+        # run B: every token new, gate closed before the activation offset
+        pool_b = g.new_pool(b.num_pages)
+        out_b = g.empty(full_T, shape.Nq)
+        ab.alora_prefill_layer(g.ctx, 0, hid_full, pos_full, d.a_req, d.ids, qsl_full, d.seq_lens, pool_b, d.bt,
+                               d.max_blocks, b.num_pages, full_T, R, out_b)
+        assert g.status() == 0
+        for r in range(R):
+            Ka, Va = _request_kv(pool_a, b, r, P + S, shape)
+            Kb, Vb = _request_kv(pool_b, b, r, P + S, shape)
+            assert np.array_equal(Ka[:P].view(np.uint32), Kb[:P].view(np.uint32)), f"prefix K of request {r}"
+            assert np.array_equal(Va[:P].view(np.uint32), Vb[:P].view(np.uint32)), f"prefix V of request {r}"
+            hp.assert_close(Kb[P:], Ka[P:], 2e-2, f"suffix K of request {r}", block=shape.head_dim)
+            hp.assert_close(Vb[P:], Va[P:], 2e-2, f"suffix V of request {r}", block=shape.head_dim)
+            tail = hp.to_host(out_b[r * (P + S) + P:(r + 1) * (P + S)])
+            hp.assert_close(tail, out_a_h[r * S:(r + 1) * S], 2e-2, f"suffix outputs of request {r}", block=shape.head_dim)
+    finally:
+        g.close()

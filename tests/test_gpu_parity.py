@@ -100,12 +100,12 @@ def test_config1_tiny_fp32_layer(oracle64):
         Ks, Vs = hp.oracle_base_prefix(oracle64, shape, w.wqkv, b)
         want = hp.oracle_block(oracle64, shape, w.wqkv, w.adapters, b, Ks, Vs)
         assert want["gate"].all()
-        assert hp.rel_err(hp.to_host(qkv), want["qkv"]) <= 1e-5
-        assert hp.rel_err(hp.to_host(out), want["out"]) <= 1e-5
+        hp.assert_close(hp.to_host(qkv), want["qkv"], 1e-5, "")
+        hp.assert_close(hp.to_host(out), want["out"], 1e-5, "")
         got = _gather_pool(oracle64, shape, hp.to_host(pool), b)
         for r in range(b.R):
-            assert hp.rel_err(got[r][0], want["K"][r]) <= 1e-5
-            assert hp.rel_err(got[r][1], want["V"][r]) <= 1e-5
+            hp.assert_close(got[r][0], want["K"][r], 1e-5, "")
+            hp.assert_close(got[r][1], want["V"][r], 1e-5, "")
         # the delta matters in this configuration: the base model's answer is outside the tolerance
         b0 = wl.Batch(**{**b.__dict__, "adapter_ids": np.array([-1], np.int32)})
         base = hp.oracle_block(oracle64, shape, w.wqkv, w.adapters, b0, Ks, Vs)
@@ -136,8 +136,8 @@ def test_ragged_multi_adapter_layer_bf16(oracle64):
         Ks, Vs = hp.oracle_base_prefix(oracle64, MID, w, b)
         want = hp.oracle_block(oracle64, MID, w, ads, b, Ks, Vs)
         qkv_h, base_h, out_h = hp.to_host(qkv), hp.to_host(base), hp.to_host(out)
-        assert hp.rel_err(qkv_h, want["qkv"]) <= 2e-2
-        assert hp.rel_err(out_h, want["out"]) <= 2e-2
+        hp.assert_close(qkv_h, want["qkv"], 2e-2, "")
+        hp.assert_close(out_h, want["out"], 2e-2, "")
         # rows whose gate is closed: bit-identical to the GPU base-only projection (Prop. 1)
         off = want["gate"] == 0
         assert off.sum() > 100 and (~off).sum() > 100
@@ -154,8 +154,8 @@ def test_ragged_multi_adapter_layer_bf16(oracle64):
         # prefix rows in the cache are the base model's (made by the base prefill) within tolerance
         got = _gather_pool(oracle64, MID, pool_after, b)
         for r in range(b.R):
-            assert hp.rel_err(got[r][0], want["K"][r]) <= 2e-2
-            assert hp.rel_err(got[r][1], want["V"][r]) <= 2e-2
+            hp.assert_close(got[r][0], want["K"][r], 2e-2, "")
+            hp.assert_close(got[r][1], want["V"][r], 2e-2, "")
     finally:
         g.close()
 
@@ -187,7 +187,7 @@ def test_sub_steps_compose_to_the_layer_call(oracle64):
         want, _ = oracle64.attention(qkv_h[:, :MID.Nq], np.concatenate([k for k, _ in kv]),
                                      np.concatenate([v for _, v in kv]), kvl, b.positions, b.query_start_loc,
                                      MID.n_q_heads, MID.n_kv_heads, MID.head_dim)
-        assert hp.rel_err(hp.to_host(out2), want) <= 2e-2
+        hp.assert_close(hp.to_host(out2), want, 2e-2, "")
     finally:
         g.close()
 
@@ -211,7 +211,7 @@ def _check_projection(oracle64, shape, w, ads, b, n_off_expected=None):
         want, gate = oracle64.project_qkv(b.hidden, w, shape.Nq, shape.Nkv, b.positions, b.query_start_loc,
                                           b.activation_offsets, b.adapter_ids, hp.oracle_adapters(ads))
         qkv_h, base_h = hp.to_host(qkv), hp.to_host(base)
-        assert hp.rel_err(qkv_h, want) <= 2e-2
+        hp.assert_close(qkv_h, want, 2e-2, "")
         off = gate == 0
         if n_off_expected is not None:
             assert off.sum() == n_off_expected
@@ -304,7 +304,7 @@ def test_short_suffixes_on_an_empty_or_tiny_cache(oracle64):
         assert np.isfinite(out_h).all()
         for r in range(b.R):
             q0, q1 = int(b.query_start_loc[r]), int(b.query_start_loc[r + 1])
-            assert hp.rel_err(out_h[q0:q1], want["out"][q0:q1]) <= 2e-2, f"request {r}"
+            hp.assert_close(out_h[q0:q1], want["out"][q0:q1], 2e-2, f"request {r}")
     finally:
         g.close()
 
@@ -321,11 +321,11 @@ def test_full_lora_recompute_matches_eq4(oracle64):
                                          d.max_blocks, b.num_pages, d.T, d.R, out)
         assert g.status() == 0
         want = hp.oracle_block(oracle64, MID, w, ads, fb, [None] * fb.R, [None] * fb.R, force_all=True)
-        assert hp.rel_err(hp.to_host(out), want["out"]) <= 2e-2
+        hp.assert_close(hp.to_host(out), want["out"], 2e-2, "")
         got = _gather_pool(oracle64, MID, hp.to_host(pool), fb)
         for r in range(fb.R):
-            assert hp.rel_err(got[r][0], want["K"][r]) <= 2e-2
-            assert hp.rel_err(got[r][1], want["V"][r]) <= 2e-2
+            hp.assert_close(got[r][0], want["K"][r], 2e-2, "")
+            hp.assert_close(got[r][1], want["V"][r], 2e-2, "")
     finally:
         g.close()
 
@@ -357,10 +357,11 @@ def test_cache_reuse_identity_on_gpu(oracle64):
             # prefix rows: exact (both are base-only arithmetic on the same inputs)
             assert np.array_equal(ka[r][0][:P].view(np.uint32), kb[r][0][:P].view(np.uint32))
             assert np.array_equal(ka[r][1][:P].view(np.uint32), kb[r][1][:P].view(np.uint32))
-            assert hp.rel_err(ka[r][0], kb[r][0]) <= 2e-2 and hp.rel_err(ka[r][1], kb[r][1]) <= 2e-2
+            hp.assert_close(ka[r][0], kb[r][0], 2e-2, "K")
+            hp.assert_close(ka[r][1], kb[r][1], 2e-2, "V")
             lo, hi = b.query_start_loc[r], b.query_start_loc[r + 1]
             tail = slice(fb.query_start_loc[r] + P, fb.query_start_loc[r + 1])
-            assert hp.rel_err(ob[tail], oa[lo:hi]) <= 2e-2
+            hp.assert_close(ob[tail], oa[lo:hi], 2e-2, "")
     finally:
         g.close()
 
@@ -400,9 +401,9 @@ def test_decode_steps_match_prefill_rows(oracle64):
         assert g.status() == 0
         Ks, Vs = hp.oracle_base_prefix(oracle64, MID, w, b)
         want = hp.oracle_block(oracle64, MID, w, ads, b, Ks, Vs)
-        assert hp.rel_err(out_h, want["out"]) <= 2e-2
-        assert hp.rel_err(dec, want["out"]) <= 2e-2
-        assert hp.rel_err(hp.to_host(pool_dec), hp.to_host(pool)) <= 2e-2
+        hp.assert_close(out_h, want["out"], 2e-2, "")
+        hp.assert_close(dec, want["out"], 2e-2, "")
+        hp.assert_close(hp.to_host(pool_dec), hp.to_host(pool), 2e-2, "")
     finally:
         g.close()
 
@@ -435,8 +436,8 @@ def test_two_layer_stack(oracle64):
                                             [None] * b.R, [None] * b.R)
             got = _gather_pool(oracle64, shape, hp.to_host(pools[l]), b)
             for r in range(b.R):
-                assert hp.rel_err(got[r][0], blk["K"][r]) <= 2e-2
-        assert hp.rel_err(hp.to_host(hout), x) <= 2e-2
+                hp.assert_close(got[r][0], blk["K"][r], 2e-2, "")
+        hp.assert_close(hp.to_host(hout), x, 2e-2, "")
     finally:
         g.close()
 
@@ -462,7 +463,7 @@ def test_stack_layer_with_many_rows_takes_the_256_row_gemm(oracle64):
                                       shape.n_kv_heads, shape.head_dim, 1e-5, b.positions, b.query_start_loc,
                                       b.activation_offsets, b.adapter_ids, hp.oracle_adapters(ads[0]),
                                       [None] * b.R, [None] * b.R)
-        assert hp.rel_err(hp.to_host(hout), x) <= 2e-2
+        hp.assert_close(hp.to_host(hout), x, 2e-2, "")
     finally:
         g.close()
 

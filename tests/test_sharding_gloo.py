@@ -69,3 +69,23 @@ def test_two_gloo_ranks_agree_on_partition_and_timing():
     assert t0 == t1 == 2.0                      # max over ranks, identical on both
     assert s0 != s1                             # every rank draws its own batch
     assert v0 == v1 == 2 * 2048 / 2e-3
+
+
+def test_bench_starts_its_own_ranks_and_agrees_on_the_timing():
+    """`python bench.py --gpus 2` with no launcher around it starts two ranks itself; with --dry-run on the gloo
+    backend the ranks do everything but the GPU work: process group, request partition, barrier, max over ranks.
+    The line rank 0 prints counts the ranks that really took part and carries the slower rank's time."""
+    import json
+    import subprocess
+    import sys
+    root = os.path.dirname(os.path.dirname(os.path.abspath(__file__)))
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_ADDR", "MASTER_PORT")}
+    out = subprocess.run([sys.executable, os.path.join(root, "bench.py"), "--gpus", "2", "--backend", "gloo", "--dry-run"],
+                         capture_output=True, text=True, timeout=300, env=env)
+    assert out.returncode == 0, out.stderr[-2000:]
+    lines = [l for l in out.stdout.splitlines() if l.startswith("{")]
+    assert len(lines) == 1, out.stdout
+    rec = json.loads(lines[0])
+    assert rec["n_gpus"] == 2 and rec["dry_run"] is True and rec["backend"] == "gloo"
+    assert rec["ms_per_step"] == 2.0                       # rank 1 reports 2.0 ms, rank 0 1.0 ms: the max
+    assert rec["config"]["requests_per_gpu"] == 8 and len(set(rec["config"]["rank_seeds"])) == 2
