@@ -20,6 +20,7 @@ int launch_attend_simt(alora_ctx *, const void *, const BatchArgs &, const void 
 int launch_project_tc(alora_ctx *, int, const void *, int, void *, cudaStream_t, void *, int);
 int launch_linear_tc(alora_ctx *, const void *, const void *, int, int, int, void *, const void *, cudaStream_t);
 bool build_layer_maps(alora_ctx *ctx, int layer);
+bool project_is_few_row(const alora_ctx *ctx, int layer, int T);   // gemm_tcgen05.cu
 int launch_attend_tc(alora_ctx *, const void *, const BatchArgs &, const void *, void *, cudaStream_t);
 
 // bf16 runs on the tensor cores; the fp32 data type (tiny exact-precision configurations) on CUDA cores.
@@ -71,12 +72,22 @@ static alora_status run_layer(alora_ctx *ctx, int layer, const void *hidden, con
     if (!ctx->layers[layer].wqkv) return ALORA_ERR_NO_WEIGHTS;
     BatchArgs b = b_in;
     b.layer = layer;
+    b.few_row = project_is_few_row(ctx, layer, b.T) ? 1 : 0;
     int n = 0, k;
-    if ((k = launch_metadata(ctx, b, s)) < 0) return ALORA_ERR_UNSUPPORTED; n += k;
+    // The per-token arrays and the projection's lists first; the attention work lists are built beside the
+    // projection (the few-row projection launches them between its two kernels, the other routes right after).
+    if ((k = launch_metadata(ctx, b, s, kMetaProjection)) < 0) return ALORA_ERR_UNSUPPORTED; n += k;
     bool kv_appended = false;
-    if ((k = launch_project(ctx, layer, hidden, b.T, ctx->d_qkv, s, pool, b.num_pages, &kv_appended)) < 0)
-        return ALORA_ERR_UNSUPPORTED;
+    ctx->pending_attn_meta = &b;
+    k = launch_project(ctx, layer, hidden, b.T, ctx->d_qkv, s, pool, b.num_pages, &kv_appended);
+    const bool attn_meta_pending = ctx->pending_attn_meta != nullptr;
+    ctx->pending_attn_meta = nullptr;
+    if (k < 0) return ALORA_ERR_UNSUPPORTED;
     n += k;
+    if (attn_meta_pending) {
+        if ((k = launch_metadata(ctx, b, s, kMetaAttention)) < 0) return ALORA_ERR_UNSUPPORTED;
+        n += k;
+    }
     if (!kv_appended) {
         if ((k = launch_kv_append(ctx, ctx->d_qkv, b.T, b.num_pages, pool, s)) < 0) return ALORA_ERR_UNSUPPORTED;
         n += k;
@@ -202,6 +213,18 @@ alora_status alora_create(const alora_config *cfg, alora_ctx **out) {
         }
     }
     if (c.dtype == ALORA_DTYPE_BF16) {
+        {
+            // few-row projection: one 128 x 256 fp32 partial per work item (at most one item per SM, or one per column
+            // tile of the widest matrix), and the partial shrink results of the q/k/v projection's K slices
+            const int widest = std::max(std::max(d.N, d.H), 2 * d.I);
+            ctx->skinny_max_items = std::max(ctx->sm_count, (widest + 255) / 256);
+            ctx->skinny_p_cap = std::min(std::max(c.max_adapters, 0), 128);
+            const int n_tiles = (d.N + 255) / 256, kb = (d.H + 63) / 64;
+            const int ksplit = std::max(1, std::min(kb, ctx->sm_count / std::max(n_tiles, 1)));
+            alloc((void **)&ctx->d_skinny_part, (size_t)ctx->skinny_max_items * 128 * 256 * 4);
+            alloc((void **)&ctx->d_skinny_t, (size_t)ksplit * 128 * std::max(ctx->skinny_p_cap, 1) * 192 * 4);
+            alloc(&ctx->d_skinny_meta, sizeof(FewRowMeta));
+        }
         alloc((void **)&ctx->d_row_delta, std::min<size_t>(Tm, kRowwiseMaxTokens) * d.N * 4);
         const size_t na = (size_t)std::max(1, c.max_adapters);
         ctx->tc_a_all.assign(c.n_layers, nullptr);
@@ -256,6 +279,7 @@ alora_status alora_destroy(alora_ctx *ctx) {
                     ctx->d_seg_scratch, ctx->d_shrink_tiles, ctx->d_t_ready, ctx->d_t, ctx->d_qkv, ctx->d_status, ctx->d_act[0], ctx->d_act[1],
                     ctx->d_act[2], ctx->d_act[3], ctx->d_iota, ctx->d_attn_items, ctx->d_attn_off, ctx->d_split_items,
                     ctx->d_req_scratch, ctx->d_part_o, ctx->d_part_ml, ctx->d_group_done, ctx->d_row_delta,
+                    ctx->d_skinny_part, ctx->d_skinny_t, ctx->d_skinny_meta,
                     ctx->d_attn_cta_start, ctx->d_attn_part_o, ctx->d_attn_part_ml};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (ctx->h_status) cudaFreeHost(ctx->h_status);
@@ -372,7 +396,8 @@ alora_status alora_batch_metadata(alora_ctx *ctx, int mode, const int32_t *d_pos
     cudaStream_t s = (cudaStream_t)stream;
     ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
     ALORA_BATCH(mode);
-    int n = launch_metadata(ctx, b, s);
+    int n = launch_metadata(ctx, b, s, kMetaProjection);
+    if (n < 0) return ALORA_ERR_UNSUPPORTED;
     if (T > 0) {
         if (d_token_request) ALORA_CUDA(ctx, cudaMemcpyAsync(d_token_request, ctx->d_token_req, (size_t)T * 4, cudaMemcpyDeviceToDevice, s));
         if (d_row_adapter) ALORA_CUDA(ctx, cudaMemcpyAsync(d_row_adapter, ctx->d_row_adapter, (size_t)T * 4, cudaMemcpyDeviceToDevice, s));
@@ -398,7 +423,9 @@ alora_status alora_project_qkv(alora_ctx *ctx, int layer, int mode, const void *
     const int32_t *d_block_tables = nullptr; const int max_blocks = 0, num_pages = 0;
     ALORA_BATCH(mode);
     b.layer = layer;
-    int n = launch_metadata(ctx, b, s), k;
+    b.few_row = project_is_few_row(ctx, layer, T) ? 1 : 0;
+    int n = launch_metadata(ctx, b, s, kMetaProjection), k;
+    if (n < 0) return ALORA_ERR_UNSUPPORTED;
     if ((k = launch_project(ctx, layer, d_hidden, T, d_qkv, s, nullptr, 0, nullptr)) < 0) return ALORA_ERR_UNSUPPORTED;
     return finish(ctx, n + k);
 }
@@ -416,7 +443,8 @@ alora_status alora_kv_append(alora_ctx *ctx, const void *d_qkv, const int32_t *d
     ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
     const int32_t *d_activation_offsets = nullptr, *d_adapter_ids = nullptr;
     ALORA_BATCH(ALORA_MODE_BASE);
-    int n = launch_metadata(ctx, b, s), k;
+    int n = launch_metadata(ctx, b, s, kMetaProjection), k;
+    if (n < 0) return ALORA_ERR_UNSUPPORTED;
     if ((k = launch_kv_append(ctx, d_qkv, T, num_pages, d_paged_kv, s)) < 0) return ALORA_ERR_UNSUPPORTED;
     return finish(ctx, n + k);
 }
@@ -436,6 +464,7 @@ alora_status alora_attend(alora_ctx *ctx, const void *d_qkv, const int32_t *d_po
     const int32_t *d_activation_offsets = nullptr, *d_adapter_ids = nullptr;
     ALORA_BATCH(ALORA_MODE_BASE);
     int n = launch_metadata(ctx, b, s), k;
+    if (n < 0) return ALORA_ERR_UNSUPPORTED;
     if ((k = launch_attend(ctx, d_qkv, b, d_paged_kv, d_attn_out, s)) < 0) return ALORA_ERR_UNSUPPORTED;
     return finish(ctx, n + k);
 }

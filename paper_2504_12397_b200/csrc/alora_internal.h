@@ -74,6 +74,19 @@ struct AttnSplitWork {
 };
 constexpr int kSplitItemsPerSm = 16;   // target number of (row tile, key range) pairs per SM
 
+// Few-row projection (batches of at most kFewRowMax rows): what its two kernels need to know about the batch's
+// adapters, written by the batch-metadata step: the adapters that occur among the rows' applied adapters
+// (ascending ids), per slot the padded rank and the scale, and per row the slot of its adapter.
+constexpr int kFewRowMax = 128;
+struct FewRowMeta {
+    int32_t n_present;
+    int32_t pad_[3];
+    int32_t slot_of_row[kFewRowMax];  // -1: the row adds no delta
+    int32_t id[kFewRowMax];           // adapter id of each slot
+    int32_t rpad[kFewRowMax];         // its rank rounded up to 16
+    float scale[kFewRowMax];
+};
+
 // Kernel families, for the optional per-kernel timing (alora_profile_*).
 enum KernelKind { KK_METADATA = 0, KK_SHRINK, KK_PROJECT, KK_KV_APPEND, KK_ATTENTION, KK_ATTN_MERGE, KK_LINEAR,
                   KK_GLUE, KK_COUNT };
@@ -87,6 +100,7 @@ struct ProfEvent {
 struct TcLayerMaps {
     CUtensorMap wqkv[3];      // W_qkv [N][H], boxes of 128 / 256 / 64 rows
     CUtensorMap a_all;        // all adapters' A rows [max_adapters*192][H], box 192 rows
+    CUtensorMap a_all16;      // the same rows in boxes of 16 (shrink chunks of the few-row projection)
     CUtensorMap b_all_bn[3];  // all adapters' B rows [max_adapters*N][64], boxes of 128 / 256 / 64 rows
     // for the 256 x 192 tiles of gemm_pair_tcgen05.cu: W in boxes of 192 rows; per q / k / v block the B rows of all
     // adapters as (rank column, row inside the block, adapter), boxes of 192 rows
@@ -101,6 +115,8 @@ struct Dims {
 };
 
 }  // namespace alora
+
+namespace alora { struct BatchArgs; }
 
 struct alora_ctx {
     alora_config cfg;
@@ -144,6 +160,12 @@ struct alora_ctx {
     int32_t max_split_items = 0, max_split_rows = 0, small_max_tokens = 0;
     void *d_t = nullptr;          // [max_tokens][3][RP] rank-r intermediate
     float *d_row_delta = nullptr; // [min(max_tokens, kRowwiseMaxTokens)][N] fp32 delta rows (bf16 row-wise route)
+    // few-row projection (batches of <= 128 rows): K-slice partial products and partial shrink results
+    float *d_skinny_part = nullptr;   // [skinny_max_items][128][256] fp32
+    float *d_skinny_t = nullptr;      // [slices of the q/k/v projection][128][skinny_p_cap][192] fp32
+    void *d_skinny_meta = nullptr;    // FewRowMeta of the current batch
+    const alora::BatchArgs *pending_attn_meta = nullptr;   // run_layer: attention lists still to be built for this batch
+    int skinny_max_items = 0, skinny_p_cap = 0;
     void *d_qkv = nullptr;        // [max_tokens][N]
     void *d_act[4] = {nullptr, nullptr, nullptr, nullptr};  // stack activations
     int32_t *d_status = nullptr;
@@ -208,9 +230,15 @@ struct BatchArgs {
     int max_blocks, num_pages, T, R, mode;
     int all_small;  // host-side knowledge that no request has more than small_max_tokens new tokens (decode)
     int layer = -1; // layer whose adapter table the gate is checked against (-1: no check)
+    int few_row = 0; // the projection of this batch takes the few-row route: build FewRowMeta instead of row tiles
 };
 
-int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s);
+// phases: bit 0 = per-token arrays and the projection's lists, bit 1 = the attention work lists.  A launch of
+// the attention lists alone is a programmatic dependent launch: it may run beside the projection kernel that
+// precedes it in the stream.  `timed`: bracket it with profiling events of the metadata family.
+constexpr int kMetaProjection = 1, kMetaAttention = 2;
+int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s, int phases = kMetaProjection | kMetaAttention,
+                    bool timed = true);
 int launch_repack_adapter(alora_ctx *ctx, int rank, const void *Aq, const void *Bq, const void *Ak,
                           const void *Bk, const void *Av, const void *Bv, void *A_dst, void *B_dst,
                           cudaStream_t s);

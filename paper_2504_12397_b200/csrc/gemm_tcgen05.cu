@@ -471,11 +471,32 @@ static int pick_bn(int N, int Nq, int Nkv, bool lora, int T) {
 int launch_project_pair_tc(alora_ctx *ctx, int layer, const void *hidden, int T, void *qkv, cudaStream_t s,
                            void *kv_pool, int num_pages);  // gemm_pair_tcgen05.cu
 
+bool skinny_route(const alora_ctx *ctx, int T, int N, int K, bool lora, int Nq, int Nkv);   // gemm_skinny_tcgen05.cu
+int launch_skinny_tc(alora_ctx *ctx, const void *x, const CUtensorMap &tmW, const CUtensorMap *tmA16,
+                     const AdapterDev *adapters, const void *b_all, int T, int K, int N, int Nq, int Nkv, void *out,
+                     const void *residual, void *kv_pool, int num_pages, cudaStream_t s);
+
+// Whether the q/k/v projection of a batch of T rows on this layer takes the few-row route (the batch-metadata step
+// then prepares that route's adapter facts instead of row tiles).
+bool project_is_few_row(const alora_ctx *ctx, int layer, int T) {
+    if (ctx->cfg.dtype != ALORA_DTYPE_BF16 || layer < 0 || layer >= ctx->cfg.n_layers) return false;
+    const Dims &d = ctx->d;
+    return skinny_route(ctx, T, d.N, d.H, ctx->layer_has_adapter[layer] != 0, d.Nq, d.Nkv);
+}
+
 int launch_project_tc(alora_ctx *ctx, int layer, const void *hidden, int T, void *qkv, cudaStream_t s, void *kv_pool,
                       int num_pages) {
     if (T == 0) return 0;
     const Dims &d = ctx->d;
     const bool have_adapters = ctx->layer_has_adapter[layer];
+    if (skinny_route(ctx, T, d.N, d.H, have_adapters, d.Nq, d.Nkv)) {   // at most 128 rows: weight-streaming route
+        ProfScope prof(ctx, KK_PROJECT, s);
+        const TcLayerMaps &lm = ctx->tc_maps[layer];
+        const AdapterDev *ads = ctx->d_adapters + (size_t)layer * ctx->cfg.max_adapters;
+        return launch_skinny_tc(ctx, hidden, lm.wqkv[1], have_adapters ? &lm.a_all16 : nullptr,
+                                have_adapters ? ads : nullptr, ctx->tc_b_all[layer], T, d.H, d.N, d.Nq, d.Nkv, qkv, nullptr,
+                                kv_pool, num_pages, s);
+    }
     if (ctx->tc_maps[layer].pair_ok) {   // many rows: two row tiles per block, 192-wide column tiles
         ProfScope prof(ctx, KK_PROJECT, s);
         const int r = launch_project_pair_tc(ctx, layer, hidden, T, qkv, s, kv_pool, num_pages);
@@ -551,6 +572,11 @@ int launch_linear_tc(alora_ctx *ctx, const void *x, const void *W, int T, int K,
     if (T == 0) return 0;
     if (K % 8 != 0 || N % 8 != 0) return -1;
     ProfScope prof(ctx, KK_LINEAR, s);
+    if (skinny_route(ctx, T, N, K, false, N, 0)) {
+        CUtensorMap tmW256;
+        if (!make_tensor_map_bf16(&tmW256, W, N, K, K, 256)) return -1;
+        return launch_skinny_tc(ctx, x, tmW256, nullptr, nullptr, nullptr, T, K, N, N, 0, y, residual, nullptr, 0, s);
+    }
     {
         const int r = launch_linear256_tc(ctx, x, W, T, K, N, y, residual, s);   // many rows: 256 x 256 tiles
         if (r != 0) return r;
@@ -585,6 +611,7 @@ bool build_layer_maps(alora_ctx *ctx, int layer) {
     }
     const size_t na = (size_t)std::max(1, ctx->cfg.max_adapters);
     ok &= make_tensor_map_bf16(&lm.a_all, ctx->tc_a_all[layer], na * 3 * kTensorRP, d.H, d.H, 3 * kTensorRP);
+    ok &= make_tensor_map_bf16(&lm.a_all16, ctx->tc_a_all[layer], na * 3 * kTensorRP, d.H, d.H, 16);
     ok &= make_tensor_map_bf16(&lm.b_all_bn[0], ctx->tc_b_all[layer], na * d.N, kTensorRP, kTensorRP, 128);
     ok &= make_tensor_map_bf16(&lm.b_all_bn[1], ctx->tc_b_all[layer], na * d.N, kTensorRP, kTensorRP, 256);
     ok &= make_tensor_map_bf16(&lm.b_all_bn[2], ctx->tc_b_all[layer], na * d.N, kTensorRP, kTensorRP, 64);

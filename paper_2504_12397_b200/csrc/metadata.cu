@@ -453,8 +453,56 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
     }
 }
 
-// The whole metadata step as one launch: every block handles 256 tokens; block 0 then builds the two
-// work lists (their serial parts are O(R)).
+// FewRowMeta of a batch of at most kFewRowMax rows (all of them in block 0): the adapters that occur in
+// row_adapter[0 .. T), ascending, each one's padded rank and scale, and every row's slot.  Called by all
+// threads of block 0 after they have written row_adapter.
+__device__ __forceinline__ void metadata_few_row(const int32_t *row_adapter, const AdapterDev *__restrict__ adapters,
+                                                 int T, int max_adapters, FewRowMeta *__restrict__ meta) {
+    __shared__ uint32_t bits[32];
+    __shared__ int16_t ids[kFewRowMax];
+    __shared__ int n_present;
+    if (threadIdx.x < 32) bits[threadIdx.x] = 0u;
+    __syncthreads();   // (also orders this block's row_adapter writes before the reads below)
+    int k_mine = -1;
+    if ((int)threadIdx.x < T && (int)threadIdx.x < kFewRowMax) {
+        k_mine = row_adapter[threadIdx.x];
+        if (k_mine >= 0 && k_mine < max_adapters && k_mine < 1024) atomicOr(&bits[k_mine >> 5], 1u << (k_mine & 31));
+        else k_mine = -1;
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int n = 0;
+        for (int w = 0; w < 32; ++w) {
+            uint32_t b = bits[w];
+            while (b && n < kFewRowMax) {
+                const int i = __ffs(b) - 1;
+                b &= b - 1;
+                ids[n++] = (int16_t)(w * 32 + i);
+            }
+        }
+        n_present = n;
+        meta->n_present = n;
+    }
+    __syncthreads();
+    const int n = n_present;
+    if ((int)threadIdx.x < n) {
+        const AdapterDev ad = adapters[ids[threadIdx.x]];
+        meta->id[threadIdx.x] = ids[threadIdx.x]; meta->rpad[threadIdx.x] = ad.rpad; meta->scale[threadIdx.x] = ad.scale;
+    }
+    if ((int)threadIdx.x < kFewRowMax) {
+        int slot = -1;
+        if (k_mine >= 0)
+            for (int p = 0; p < n; ++p) if (ids[p] == k_mine) slot = p;
+        meta->slot_of_row[threadIdx.x] = slot;
+    }
+}
+
+// The metadata step.  Phase bit 0: every block handles 256 tokens (request, applied adapter, slot); block 0 then
+// builds the projection's row-tile list, or the few-row route's adapter facts.  Phase bit 1: the two attention
+// work lists, one block each (their serial parts are O(R)).  Both phases in one launch: blocks 0, 1, 2 take one
+// builder each.  The attention phase alone is launched as a programmatic dependent of the projection kernel, beside
+// which it runs (it reads nothing that kernel writes); its blocks wait for that kernel before they exit, so that
+// whatever follows in the stream still sees the projection complete.
 __global__ void __launch_bounds__(256)
 metadata_kernel(const int32_t *__restrict__ positions, const int32_t *a_req, const int32_t *adapter_ids,
                 const int32_t *qsl, const int32_t *seq_lens, const int32_t *__restrict__ block_tables, int max_blocks,
@@ -466,7 +514,8 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *a_req, con
                 int G, int n_sm, int small_max, int max_split_items, int max_split_rows,
                 AttnSplitWork *__restrict__ split_items,
                 int32_t *req_scratch, int32_t *__restrict__ group_done, int rowwise_cap,
-                int32_t *__restrict__ attn_cta_start, const AdapterDev *__restrict__ adapters, int32_t *status) {
+                int32_t *__restrict__ attn_cta_start, const AdapterDev *__restrict__ adapters, int phases,
+                FewRowMeta *__restrict__ few_row_meta, int32_t *status) {
     // The per-request inputs are read many times (binary searches, list builders): one parallel pass stages them
     // in shared memory, so that the later steps do not each pay a round trip to global memory.
     __shared__ int32_t s_req[4 * kMetaStageR + 1];
@@ -484,21 +533,31 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *a_req, con
         if (adapter_ids) adapter_ids = s_ids;
         if (a_req) a_req = s_areq;
     }
-    metadata_tokens(positions, a_req, adapter_ids, qsl, seq_lens, block_tables, max_blocks, num_pages, page_size,
-                    max_adapters, T, R, mode, token_req, row_adapter, slot_map, adapters, status);
-    // The three list builders are independent of one another: blocks 0, 1 and 2 take one each (a launch has at least
-    // three blocks; with fewer, block 0 would run them one after the other).
+    if (phases & kMetaProjection)
+        metadata_tokens(positions, a_req, adapter_ids, qsl, seq_lens, block_tables, max_blocks, num_pages, page_size,
+                        max_adapters, T, R, mode, token_req, row_adapter, slot_map, adapters, status);
+    // The three list builders are independent of one another: blocks 0, 1 and 2 take one each (a launch of both
+    // phases has at least three blocks, one of the attention phase alone two).
     const int nb = (int)gridDim.x;
-    const int b_tiles = 0, b_attn = nb > 1 ? 1 : 0, b_split = nb > 2 ? 2 : 0;
-    if ((int)blockIdx.x != b_tiles && (int)blockIdx.x != b_attn && (int)blockIdx.x != b_split) return;
+    const bool proj = (phases & kMetaProjection) != 0, attn = (phases & kMetaAttention) != 0;
+    const int b_tiles = proj ? 0 : -1;
+    const int b_attn = !attn ? -1 : (proj ? (nb > 1 ? 1 : 0) : 0);
+    const int b_split = !attn ? -1 : (proj ? (nb > 2 ? 2 : 0) : (nb > 1 ? 1 : 0));
+    if ((int)blockIdx.x != b_tiles && (int)blockIdx.x != b_attn && (int)blockIdx.x != b_split) {
+        if (!proj) tc::grid_dep_wait();
+        return;
+    }
     // the per-request scratch of the list builders (their serial parts walk it) lives in shared memory when the
     // batch is small enough, else in the context's global scratch (one buffer per builder)
     __shared__ int32_t smem_scratch[kMetaSmemInts];
     if (14 * R + 5 <= kMetaSmemInts) seg_scratch = blk_off = req_scratch = smem_scratch;
     __syncthreads();
     if ((int)blockIdx.x == b_tiles) {
-        metadata_tiles(a_req, adapter_ids, qsl, seq_lens, R, mode, max_adapters, max_tiles, tiles, counts, seg_scratch,
-                       T, rowwise_cap, shrink_tiles, t_ready, status);
+        if (few_row_meta != nullptr && adapters != nullptr && row_adapter != nullptr)
+            metadata_few_row(row_adapter, adapters, T, max_adapters, few_row_meta);   // the few-row route has no row tiles
+        else
+            metadata_tiles(a_req, adapter_ids, qsl, seq_lens, R, mode, max_adapters, max_tiles, tiles, counts, seg_scratch,
+                           T, rowwise_cap, shrink_tiles, t_ready, status);
         __syncthreads();  // a builder that follows in this block reuses the scratch
     }
     if ((int)blockIdx.x == b_attn && items != nullptr && block_tables != nullptr) {
@@ -509,16 +568,24 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *a_req, con
     if ((int)blockIdx.x == b_split && split_items != nullptr && block_tables != nullptr)
         metadata_split_items(qsl, seq_lens, R, Hkv, G, n_sm, small_max, max_split_items, max_split_rows, split_items, counts,
                              req_scratch, group_done, status);
+    if (!proj) tc::grid_dep_wait();
 }
 
-int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s) {
+int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s, int phases, bool timed) {
     if (b.T == 0) {
-        cudaMemsetAsync(ctx->d_counts, 0, 6 * sizeof(int32_t), s);
+        if (phases & kMetaProjection) cudaMemsetAsync(ctx->d_counts, 0, 6 * sizeof(int32_t), s);
         return 0;
     }
+    const bool saved = ctx->profiling;
+    if (!timed) ctx->profiling = false;
     ProfScope prof(ctx, KK_METADATA, s);
+    ctx->profiling = saved;
     const int threads = 256;
-    metadata_kernel<<<std::max(3, (b.T + threads - 1) / threads), threads, 0, s>>>(
+    const bool attn_only = phases == kMetaAttention;
+    const int grid = attn_only ? 2 : std::max((phases & kMetaAttention) ? 3 : 1, (b.T + threads - 1) / threads);
+    const AdapterDev *ads = b.layer >= 0 ? ctx->d_adapters + (size_t)b.layer * ctx->cfg.max_adapters : nullptr;
+    FewRowMeta *few = (b.few_row && ads != nullptr) ? (FewRowMeta *)ctx->d_skinny_meta : nullptr;
+    const cudaError_t e = launch_kernel(metadata_kernel, dim3(grid), dim3(threads), 0, s, attn_only,
         b.positions, b.activation_offsets, b.adapter_ids, b.query_start_loc, b.seq_lens, b.block_tables,
         b.max_blocks, b.num_pages, ctx->d.page, ctx->cfg.max_adapters, b.T, b.R, b.mode, ctx->d_token_req,
         ctx->d_row_adapter, ctx->d_slot, ctx->max_tiles, ctx->d_tiles, ctx->d_counts, ctx->d_seg_scratch,
@@ -526,9 +593,8 @@ int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s) {
         ctx->d.Hkv, ctx->attn_q_block, ctx->max_attn_items, ctx->d_attn_items, ctx->d_attn_off, ctx->d.G,
         ctx->sm_count, ctx->small_max_tokens, ctx->max_split_items, ctx->max_split_rows, ctx->d_split_items,
         ctx->d_req_scratch, ctx->d_group_done, ctx->d_row_delta ? kRowwiseMaxTokens : 0,
-        ctx->d_attn_cta_start,
-        b.layer >= 0 ? ctx->d_adapters + (size_t)b.layer * ctx->cfg.max_adapters : nullptr, ctx->d_status);
-    return 1;
+        ctx->d_attn_cta_start, ads, phases, few, ctx->d_status);
+    return e == cudaSuccess ? 1 : -1;
 }
 
 }  // namespace alora

@@ -32,6 +32,10 @@ __device__ __forceinline__ void mbar_arrive(uint32_t bar) {
 __device__ __forceinline__ void mbar_arrive_expect_tx(uint32_t bar, uint32_t bytes) {
     asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
 }
+// Adds to the bytes a barrier phase expects without arriving on it (a later arrive.expect_tx completes the count).
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.expect_tx.relaxed.cta.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
 // Programmatic dependent launch.  A kernel launched with the programmatic-stream-serialization attribute may start
 // while its predecessor in the stream is still running: grid_dep_wait() returns once the predecessor has completed
 // and its writes are visible (it returns at once in a kernel launched the ordinary way), so everything before it

@@ -46,12 +46,17 @@ def rel_err_blocks(got: np.ndarray, want: np.ndarray, block: int) -> float:
     return float((d / np.maximum(w, floor if floor > 0 else 1.0)).max())
 
 
-# Bounds of the three measures for bf16 results against the fp64 oracle.  The first is the method's stated
-# bound.  The other two judge single elements or single heads: an element's error is that of a bf16 rounding
-# of the output (2^-9 relative) plus the accumulated operand roundings, which do not shrink with the element, so
-# elements far below the tensor's rms see a larger relative error; the elementwise floor (1e-2 rms) and the bound
-# below leave room for exactly that and nothing more: a wrong head, row or block is off by O(1).
-TOL_ELEMENTWISE_BF16 = 0.5
+# Bounds of the three measures for bf16 results against the fp64 oracle.
+# (1) Tensor-wide: the method's stated bound, 2e-2.
+# (2) Elementwise, |d| / (|want| + 1e-2 rms): decided by the elements near zero, whose error does not shrink with
+#     them.  Each bf16 rounding on the way (q/k/v rows, softmax probabilities, outputs; through a decoder layer
+#     about ten of them) leaves noise of about 2^-9 / sqrt(3) of the tensor's rms, so a 5-sigma element of ten
+#     stages is off by ~0.02 .. 0.04 rms and reads 2 .. 4 here (measured: up to 3.1 through a two-layer stack, 0.5
+#     .. 1.7 for single kernels).  The stated bound (1) itself admits 2e-2 * max|want| ~ 0.1 rms, i.e. ~10 here.  The
+#     bound sits between the two.  A wrong element (missing delta, wrong head or row) is off by O(rms): ~100.
+# (3) Per (row, head): the same absolute error against a head's own maximum, which is 2 .. 3 sigma where the
+#     tensor's is ~5 sigma: three times the stated bound.  Measured: up to 1.7e-2.
+TOL_ELEMENTWISE_BF16 = 8.0
 TOL_BLOCKS_BF16 = 6e-2
 
 

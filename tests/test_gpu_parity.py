@@ -264,6 +264,81 @@ def test_projection_row_wise_route_many_short_requests(oracle64):
     _check_projection(oracle64, MID, w, ads, b)
 
 
+@pytest.mark.parametrize("T", [1, 24, 33, 64, 65, 128])
+def test_projection_few_row_route_mixed_adapters(oracle64, T):
+    """Batches of at most 128 rows (decode steps): the weight-streaming route, K split over the SMs, the shrink of
+    every present adapter riding along, slice partials added in fixed order.  One token per request, requests mixing
+    the base model and four adapters of different ranks in no particular order, every third adapter request with
+    its gate still closed.  Checked: oracle, closed-gate rows bit-identical to the base-only call, determinism."""
+    rng = np.random.default_rng(100 + T)
+    w = wl.make_wqkv(MID, rng)
+    ads = _boosted_adapters(MID, rng, ((8, 1.0), (64, 0.5), (32, 2.0), (16, 1.0)))
+    R = T
+    ids = [int(x) for x in rng.integers(-1, 4, R)]
+    if R >= 24:
+        ids[:5] = [3, -1, 0, 2, 1]
+    else:
+        ids[0] = 2
+    P = [int(x) for x in rng.integers(0, 300, R)]
+    a_req = [P[i] + (1 if (ids[i] >= 0 and i % 3 == 1) else 0) for i in range(R)]   # gate closed on this step
+    if R == 1:
+        b2 = wl.make_batch(MID, P + [7], [1, 1], ids + [1], rng, activation_offsets=a_req + [8])   # one open, one closed row
+        return _check_projection(oracle64, MID, w, ads, b2)
+    b = wl.make_batch(MID, P, [1] * R, ids, rng, activation_offsets=a_req)
+    _check_projection(oracle64, MID, w, ads, b)
+
+
+def test_projection_few_row_route_short_suffixes_one_adapter(oracle64):
+    """8 requests x 16 new tokens (128 rows), one adapter, gates opening inside the chunk."""
+    rng = np.random.default_rng(49)
+    w = wl.make_wqkv(MID, rng)
+    ads = _boosted_adapters(MID, rng, ((32, 1.0),))
+    P = [100 + 13 * i for i in range(8)]
+    a_req = [P[i] + (5 if i % 2 else 0) for i in range(8)]
+    b = wl.make_batch(MID, P, [16] * 8, [0] * 8, rng, activation_offsets=a_req)
+    _check_projection(oracle64, MID, w, ads, b, n_off_expected=20)
+
+
+def test_decode_sized_stack_takes_the_few_row_projections(oracle64):
+    """Two decoder layers on a batch of 40 rows (requests of 1 .. 6 new tokens on cached prefixes made by a base
+    prefill through the same stack): q/k/v, o_proj, gate/up and down all run on the few-row route, the last three
+    with the residual added in its second kernel."""
+    shape = wl.LayerShape(hidden=512, n_q_heads=4, n_kv_heads=2, head_dim=128, page_size=16, dtype="bf16",
+                          intermediate=1024)
+    rng = np.random.default_rng(33)
+    layers = [wl.make_stack_weights(shape, rng) for _ in range(2)]
+    ads = [[wl.make_adapter(shape, 16, rng), wl.make_adapter(shape, 8, rng)] for _ in range(2)]
+    for per in ads:
+        for a in per:
+            for n in ("Bq", "Bk", "Bv"):
+                setattr(a, n, wl.bf16_round(getattr(a, n) * 8))
+    S = [1, 6, 2, 5, 3, 4, 1, 6, 2, 5, 3, 2]
+    assert sum(S) == 40
+    ids = [0, 1, -1, 0, 1, -1, 1, 0, -1, 1, 0, 1]
+    b = wl.make_batch(shape, [0] * len(S), S, ids, rng, activation_offsets=[2 if i % 4 == 1 else 0 for i in range(len(S))],
+                      shuffle_pages=True)
+    g = hp.GpuLayers(shape, layers, ads, 128, 16)
+    try:
+        d = hp.DevBatch(b, shape.dtype)
+        pools = [g.new_pool(b.num_pages) for _ in range(2)]
+        hout = g.empty(b.T, shape.hidden)
+        ab.alora_forward_stack(g.ctx, ab.MODE_ALORA, d.hidden, d.positions, d.a_req, d.ids, d.qsl, d.seq_lens, pools,
+                               d.bt, d.max_blocks, b.num_pages, d.T, d.R, hout)
+        assert g.status() == 0
+        x = b.hidden.astype(np.float64)
+        for l in range(2):
+            x, blk = oracle64.decoder_layer(x, layers[l], shape.Nq, shape.Nkv, shape.n_q_heads, shape.n_kv_heads,
+                                            shape.head_dim, 1e-5, b.positions, b.query_start_loc,
+                                            b.activation_offsets, b.adapter_ids, hp.oracle_adapters(ads[l]),
+                                            [None] * b.R, [None] * b.R)
+            got = _gather_pool(oracle64, shape, hp.to_host(pools[l]), b)
+            for r in range(b.R):
+                hp.assert_close(got[r][0], blk["K"][r], 2e-2, f"layer {l} K rows of request {r}")
+        hp.assert_close(hp.to_host(hout), x, 2e-2, "stack output")
+    finally:
+        g.close()
+
+
 def test_projection_with_128_wide_kv_blocks(oracle64):
     """One KV head of 128 columns: the q/k/v block boundaries force 128-wide column tiles, and the rank-r
     shrink then runs as the separate cluster split-K kernel."""
