@@ -571,6 +571,36 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *a_req, con
     if (!proj) tc::grid_dep_wait();
 }
 
+// The projection phase for a batch on the few-row route (at most kFewRowMax tokens, one block): per-token arrays
+// and the adapter facts, nothing else.  A kernel of its own because every step of a decode loop waits for it: it
+// runs once per call on one SM, so what it costs is mostly the fetch of its instructions, and this one is short.
+__global__ void __launch_bounds__(kFewRowMax)
+metadata_few_row_kernel(const int32_t *__restrict__ positions, const int32_t *a_req, const int32_t *adapter_ids,
+                        const int32_t *qsl, const int32_t *seq_lens, const int32_t *__restrict__ block_tables,
+                        int max_blocks, int num_pages, int page_size, int max_adapters, int T, int R, int mode,
+                        int32_t *__restrict__ token_req, int32_t *__restrict__ row_adapter,
+                        int32_t *__restrict__ slot_map, const AdapterDev *__restrict__ adapters,
+                        FewRowMeta *__restrict__ few_row_meta, int32_t *status) {
+    __shared__ int32_t s_req[4 * kFewRowMax + 1];
+    tc::grid_dep_launch();
+    if (R <= kFewRowMax) {   // the per-request inputs are read several times (binary search): stage them
+        int32_t *s_qsl = s_req, *s_len = s_req + R + 1, *s_ids = s_len + R, *s_areq = s_ids + R;
+        for (int i = threadIdx.x; i <= R; i += blockDim.x) s_qsl[i] = qsl[i];
+        for (int i = threadIdx.x; i < R; i += blockDim.x) {
+            s_len[i] = seq_lens[i];
+            if (adapter_ids) s_ids[i] = adapter_ids[i];
+            if (a_req) s_areq[i] = a_req[i];
+        }
+        __syncthreads();
+        qsl = s_qsl; seq_lens = s_len;
+        if (adapter_ids) adapter_ids = s_ids;
+        if (a_req) a_req = s_areq;
+    }
+    metadata_tokens(positions, a_req, adapter_ids, qsl, seq_lens, block_tables, max_blocks, num_pages, page_size,
+                    max_adapters, T, R, mode, token_req, row_adapter, slot_map, adapters, status);
+    if (few_row_meta != nullptr) metadata_few_row(row_adapter, adapters, T, max_adapters, few_row_meta);
+}
+
 int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s, int phases, bool timed) {
     if (b.T == 0) {
         if (phases & kMetaProjection) cudaMemsetAsync(ctx->d_counts, 0, 6 * sizeof(int32_t), s);
@@ -585,6 +615,13 @@ int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s, int phas
     const int grid = attn_only ? 2 : std::max((phases & kMetaAttention) ? 3 : 1, (b.T + threads - 1) / threads);
     const AdapterDev *ads = b.layer >= 0 ? ctx->d_adapters + (size_t)b.layer * ctx->cfg.max_adapters : nullptr;
     FewRowMeta *few = (b.few_row && ads != nullptr) ? (FewRowMeta *)ctx->d_skinny_meta : nullptr;
+    if (phases == kMetaProjection && b.few_row && b.T <= kFewRowMax) {
+        metadata_few_row_kernel<<<1, kFewRowMax, 0, s>>>(
+            b.positions, b.activation_offsets, b.adapter_ids, b.query_start_loc, b.seq_lens, b.block_tables, b.max_blocks,
+            b.num_pages, ctx->d.page, ctx->cfg.max_adapters, b.T, b.R, b.mode, ctx->d_token_req, ctx->d_row_adapter,
+            ctx->d_slot, ads, few, ctx->d_status);
+        return 1;
+    }
     const cudaError_t e = launch_kernel(metadata_kernel, dim3(grid), dim3(threads), 0, s, attn_only,
         b.positions, b.activation_offsets, b.adapter_ids, b.query_start_loc, b.seq_lens, b.block_tables,
         b.max_blocks, b.num_pages, ctx->d.page, ctx->cfg.max_adapters, b.T, b.R, b.mode, ctx->d_token_req,
