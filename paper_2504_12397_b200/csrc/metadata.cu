@@ -343,7 +343,7 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
                                                      int32_t *req_scratch /* [3][R] */,
                                                      int32_t *__restrict__ group_done, int32_t *status) {
     __shared__ unsigned long long tot_units;
-    __shared__ int chunk_units, total_items;
+    __shared__ int chunk_units, total_items, few_ranges;
     small_max = few_row_limit(qsl, R, Hkv, n_sm, small_max);
     int32_t *req_cnt = req_scratch, *req_off = req_scratch + R, *req_row = req_scratch + 2 * R;
     // 64-key units of all blocks, weighted by the blocks' row tiles (an item of mt tiles needs mt * 16 partial rows):
@@ -381,8 +381,51 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
         const float per_sm = fminf(fmaxf(sqrtf(t_us / 12.f), 1.f), (float)kSplitItemsPerSm);
         const unsigned long long target = (unsigned long long)ceilf(per_sm * (float)max(n_sm, 1));
         chunk_units = (int)max(4ull, (tot_units + target - 1) / target);
+        few_ranges = per_sm < 2.5f ? 1 : 0;
     }
     __syncthreads();
+    // With only one or two ranges per SM the rule above ignores how the ranges fall into rounds over the SMs: 192
+    // equal ranges on 148 SMs take as long as 296.  Such batches (a few requests) instead take the shortest range
+    // length whose ranges fit into exactly one round, or into two, whichever the same cost model says is faster:
+    // rounds x (12 us + range length x 0.74 us).  The range count for a given length is a sum over the requests.
+    if (few_ranges) {
+        constexpr int kMaxChunkUnits = 1 << 14;   // 64-key units: a million keys
+        __shared__ int cnt_acc;
+        int best_chunk[2];
+        for (int w = 1; w <= 2; ++w) {
+            const int cap = w * n_sm;
+            int lo = 4, hi = kMaxChunkUnits;   // smallest chunk in [lo, hi] whose range count fits into cap (hi: one range per stream)
+            while (lo < hi) {
+                const int mid = (lo + hi) >> 1;
+                if (threadIdx.x == 0) cnt_acc = 0;
+                __syncthreads();
+                int mine = 0;
+                for (int r = threadIdx.x; r < R; r += blockDim.x) {
+                    const int n_new = qsl[r + 1] - qsl[r];
+                    if (n_new > 0 && n_new <= small_max) {
+                        int mt, tpb, nblk;
+                        small_block_shape(n_new, G, mt, tpb, nblk);
+                        for (int blk = 0; blk < nblk; ++blk) {
+                            const int kv_end = seq_lens[r] - n_new + min(n_new, (blk + 1) * tpb);
+                            mine += ((((kv_end + 63) / 64) + mid - 1) / mid) * Hkv;
+                        }
+                    }
+                }
+                if (mine) atomicAdd(&cnt_acc, mine);
+                __syncthreads();
+                const int cnt = cnt_acc;
+                __syncthreads();
+                if (cnt <= cap) hi = mid; else lo = mid + 1;
+            }
+            best_chunk[w - 1] = lo;
+        }
+        if (threadIdx.x == 0) {
+            const float c1 = 12.f + 0.74f * (float)best_chunk[0], c2 = 2.f * (12.f + 0.74f * (float)best_chunk[1]);
+            if (best_chunk[0] < kMaxChunkUnits && c1 <= c2) chunk_units = best_chunk[0];
+            else if (best_chunk[1] < kMaxChunkUnits) chunk_units = best_chunk[1];
+        }
+        __syncthreads();
+    }
     const int chunk = chunk_units;
     for (int r = threadIdx.x; r < R; r += blockDim.x) {
         const int n_new = qsl[r + 1] - qsl[r];
