@@ -58,7 +58,7 @@ class ClockSampler:
     REASONS = {"hw_slowdown": 0x8, "sw_power_cap": 0x4, "sw_thermal_slowdown": 0x20, "hw_thermal_slowdown": 0x40,
                "hw_power_brake_slowdown": 0x80}
 
-    def __init__(self, gpu_index: int, period_s: float = 0.005):
+    def __init__(self, gpu_index: int, period_s: float = 0.002):
         self.gpu, self.period = gpu_index, period_s
         self.sm, self.reasons, self.power = [], set(), []
         self.stop_flag = threading.Event()
@@ -215,6 +215,44 @@ def dry_run(args, world: int, rank: int) -> None:
             dist.destroy_process_group()
 
 
+def fractions(peaks, roofline, sustained, config3, decode, short, recompute_8k, stack_8k, stack, evaluators):
+    """Compact summary of the roofline fractions and speed-ups of all legs (None where a leg did not run)."""
+    r3 = lambda x: None if x is None else round(float(x), 3)   # noqa: E731
+    out = {"peaks": {"bf16_tflops": peaks["bf16_tflops"], "bf16_tflops_sustained": peaks["bf16_tflops_sustained"],
+                     "hbm_gbs": peaks["hbm_gbs"], "source": peaks["source"]},
+           "config2_projection_tensor": r3(roofline["projection"]["frac_of_tensor_peak"]),
+           "config2_attention_tensor": r3(roofline["attention"]["frac_of_tensor_peak"])}
+    if sustained:
+        out["config2_step_of_sustained_tensor"] = r3(sustained["frac_of_sustained_bf16_peak"])
+    if config3:
+        out["config3_projection_tensor"] = r3(config3["projection_frac_of_tensor_peak"])
+        out["config3_attention_tensor"] = r3(config3["attention_frac_of_tensor_peak"])
+        out["config3_tokens_per_s"] = r3(config3["suffix_tokens_per_s"])
+    if decode:
+        out["config5_decode_attention_hbm"] = r3(decode["attention_frac_of_hbm_peak"])
+        out["config5_decode_ms_per_step"] = r3(decode["ms_per_step"])
+        out["config5_decode_projection_ms"] = r3(decode["per_kernel_ms"].get("project_qkv", 0.0) + decode["per_kernel_ms"].get("shrink", 0.0))
+    if short:
+        for s_ in short:
+            key = f"short_{s_['requests']}x{s_['suffix']}"
+            out[key + "_attention_hbm"] = r3(s_["attention_frac_of_hbm_peak"])
+            out[key + "_ms_per_step"] = r3(s_["ms_per_step"])
+            out[key + "_projection_ms"] = r3(s_["per_kernel_ms"].get("project_qkv", 0.0) + s_["per_kernel_ms"].get("shrink", 0.0))
+    if recompute_8k:
+        out["speedup_8k_prefix_qkv_attention"] = r3(recompute_8k["speedup_alora_vs_full_lora"])
+    if stack_8k:
+        out["speedup_8k_prefix_whole_layers"] = r3(stack_8k["speedup_alora_vs_full_lora"])
+        out["flop_ratio_8k_prefix_whole_layers"] = r3(stack_8k["flop_ratio"])
+        out["token_ratio_8k_prefix"] = r3(stack_8k["prefix_plus_suffix_over_suffix"])
+    if stack:
+        out["speedup_config4_stack"] = r3(stack["speedup_alora_vs_full_lora"])
+        out["flop_ratio_config4_stack"] = r3(stack["flop_ratio"])
+    if evaluators:
+        out["evaluator_stage_speedup"] = [r3(e["evaluator_stage_speedup"]) for e in evaluators]
+        out["evaluator_pipeline_speedup"] = [r3(e["pipeline_speedup"]) for e in evaluators]
+    return out
+
+
 def _events(n):
     import torch
     return [(torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)) for _ in range(n)]
@@ -364,6 +402,95 @@ def short_suffix_leg(ab, hp, ctx, shape, stream, flush, peaks, requests, prefix,
             "attention_hbm_gbs": gbs, "attention_frac_of_hbm_peak": gbs / peaks["hbm_gbs"] if gbs else None}
 
 
+def config3_leg(ab, hp, stream, local, flush, peaks, seed=3):
+    """Config 3: ragged multi-adapter batch at the 8B layer shape: 32 requests over adapters of ranks 8/16/32/64,
+    prefixes U[512, 16384], suffixes U[16, 512], activation at the prefix end, shuffled 16-token pages."""
+    import torch
+    w = wl.config3(seed=seed)
+    shape, b = w.shape, w.batch
+    cfg = ab.make_config(hidden=shape.hidden, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads,
+                         head_dim=shape.head_dim, page_size=shape.page_size, max_adapters=len(w.adapters), max_rank=64,
+                         dtype=ab.DTYPE_BF16, device=local, max_tokens=b.T, max_requests=b.R)
+    ctx = ab.alora_create(cfg)
+    try:
+        wq = hp.to_dev(w.wqkv, "bf16")
+        ab.alora_set_layer_weights(ctx, 0, wq)
+        keep = []
+        for i, a in enumerate(w.adapters):
+            mats = [hp.to_dev(getattr(a, n), "bf16") for n in ("Aq", "Bq", "Ak", "Bk", "Av", "Bv")]
+            keep.append(mats)
+            ab.alora_register_adapter(ctx, i, 0, a.rank, a.scale, *mats)
+        d = hp.DevBatch(b, "bf16")
+        g = torch.Generator(device="cuda"); g.manual_seed(seed + 1000)
+        pool = torch.empty((b.num_pages, 2, shape.n_kv_heads, shape.page_size, shape.head_dim), device="cuda", dtype=torch.bfloat16)
+        for i in range(0, b.num_pages, 8192):
+            n = min(8192, b.num_pages - i)
+            pool[i:i + n] = torch.randn((n,) + tuple(pool.shape[1:]), generator=g, device="cuda", dtype=torch.float32).to(torch.bfloat16)
+        out = torch.empty((b.T, shape.Nq), dtype=torch.bfloat16, device="cuda")
+
+        def step():
+            ab.alora_prefill_layer(ctx, 0, d.hidden, d.positions, d.a_req, d.ids, d.qsl, d.seq_lens, pool, d.bt,
+                                   d.max_blocks, b.num_pages, b.T, b.R, out, stream)
+        for _ in range(5):
+            step()
+        ms = timed(step, 30, stream, flush)
+        kern = profiled(ab, ctx, step, 30, flush)
+        status = ab.alora_get_status(ctx)
+    finally:
+        ab.alora_destroy(ctx)
+    H, N, hd, Hq = shape.hidden, shape.N, shape.head_dim, shape.n_q_heads
+    P_, S_ = b.prefix_lens.astype(np.int64), (b.seq_lens - b.prefix_lens).astype(np.int64)
+    ranks = np.array([w.adapters[k].rank for k in b.adapter_ids], np.int64)
+    proj = float((2.0 * S_ * H * (N + 3 * ranks) + 2.0 * S_ * ranks * N).sum())
+    attn = 4.0 * hd * Hq * float((S_ * P_ + S_ * (S_ + 1) // 2).sum())
+    kv_bytes = float(b.seq_lens.sum()) * shape.n_kv_heads * hd * 2 * 2 + 2.0 * b.T * shape.Nq * 2
+    proj_ms = kern.get("project_qkv", 0.0) + kern.get("shrink", 0.0)
+    attn_ms = kern.get("attention", 0.0) + kern.get("attn_merge", 0.0)
+    peak = peaks["bf16_tflops"]
+    return {"workload": f"config3: {b.R} requests over adapters of ranks 8/16/32/64, prefixes U[512,16384] (sum "
+                        f"{int(P_.sum())}), suffixes U[16,512] (sum {b.T}), shuffled 16-token pages; KV read "
+                        f"{kv_bytes / 1e9:.2f} GB per step exceeds L2",
+            "ms_per_step": ms, "suffix_tokens_per_s": b.T / (ms / 1e3),
+            "per_kernel_ms": {k: round(v, 4) for k, v in kern.items()},
+            "projection_tflops": proj / (proj_ms / 1e3) / 1e12 if proj_ms else None,
+            "projection_frac_of_tensor_peak": proj / (proj_ms / 1e3) / 1e12 / peak if proj_ms else None,
+            "attention_tflops": attn / (attn_ms / 1e3) / 1e12 if attn_ms else None,
+            "attention_frac_of_tensor_peak": attn / (attn_ms / 1e3) / 1e12 / peak if attn_ms else None,
+            "attention_hbm_gbs": kv_bytes / (attn_ms / 1e3) / 1e9 if attn_ms else None,
+            "attention_frac_of_hbm_peak": kv_bytes / (attn_ms / 1e3) / 1e9 / peaks["hbm_gbs"] if attn_ms else None,
+            "step_tflops": (proj + attn) / (ms / 1e3) / 1e12, "device_status": status}
+
+
+def sustained_leg(step, stream, flush, local, min_seconds, step_flops, peaks):
+    """The headline step repeated until at least `min_seconds` of step time have been timed (per-step CUDA events,
+    L2 flushed between steps), with the SM clock sampled every millisecond: the layer call under the power cap."""
+    import torch
+    sampler = ClockSampler(local, period_s=0.001)
+    sampler.start()
+    total_ms, times = 0.0, []
+    while total_ms < min_seconds * 1e3 and len(times) < 200000:
+        n = 200
+        ev = _events(n)
+        for e0, e1 in ev:
+            flush.zero_()
+            e0.record(stream)
+            step()
+            e1.record(stream)
+        torch.cuda.synchronize()
+        batch = [e0.elapsed_time(e1) for e0, e1 in ev]
+        times += batch
+        total_ms += sum(batch)
+    clocks = sampler.stop()
+    ms = float(np.mean(times))
+    tail = float(np.mean(times[len(times) // 2:]))   # the second half: clocks have settled
+    mhz = clocks.get("sm_mhz")
+    return {"steps": len(times), "timed_seconds": total_ms / 1e3, "ms_per_step": ms, "ms_per_step_second_half": tail,
+            "sm_mhz_median": mhz, "ms_x_sm_mhz": ms * mhz if mhz else None, "clocks": clocks,
+            "step_tflops": step_flops / (tail / 1e3) / 1e12,
+            "frac_of_sustained_bf16_peak": step_flops / (tail / 1e3) / 1e12 / peaks["bf16_tflops_sustained"],
+            "peak": peaks["bf16_tflops_sustained"], "peak_source": peaks["source"] + " (sustained bf16 GEMM)"}
+
+
 def evaluator_leg(ab, hp, shape, stream, local, n_eval, seed=9, convs=8, prompt=4096, gen=256, inv=16, eval_steps=16):
     """The paper's evaluator workload on one layer: `convs` conversations get a base-model prefill of `prompt` tokens
     and `gen` base decode steps; then `n_eval` adapters each read the conversation and answer: `inv` invocation
@@ -491,10 +618,12 @@ def evaluator_leg(ab, hp, shape, stream, local, n_eval, seed=9, convs=8, prompt=
             "device_status": status, "output_finite": finite}
 
 
-def stack_leg(ab, hp, shape, stream, local, seed=4, requests=4, prefix=32768, suffix=1024, n_layers=32):
-    """Config 4: the full decoder stack at the 8B shape (RMSNorm, attention block, o_proj, SwiGLU MLP; random
-    bf16 weights), 4 requests with 32768 cached positions and 1024 aLoRA suffix tokens each, against the
-    full-LoRA recompute of prefix + suffix through the same stack."""
+def stack_leg(ab, hp, shape, stream, local, seed=4, requests=4, prefix=32768, suffix=1024, n_layers=32, name="config4"):
+    """The decoder stack at the 8B shape (RMSNorm, attention block, o_proj, SwiGLU MLP; random bf16 weights):
+    `requests` requests with `prefix` cached positions and `suffix` aLoRA suffix tokens each, against the
+    full-LoRA recompute of prefix + suffix through the same stack.  Config 4 is 32 layers, 4 x (32768 + 1024);
+    the 8K-prefix comparison runs 4 layers of 8 x (8192 + 256) (every layer costs the same, so the ratio is that
+    of the whole stack)."""
     import torch
     g = torch.Generator(device="cuda"); g.manual_seed(seed)
 
@@ -569,7 +698,7 @@ def stack_leg(ab, hp, shape, stream, local, seed=4, requests=4, prefix=32768, su
     att = lambda s_, p_: 4.0 * shape.head_dim * shape.n_q_heads * (s_ * p_ + s_ * (s_ + 1) / 2)   # noqa: E731
     flop_a = n_layers * (T * lin + R * att(S_, P))
     flop_r = n_layers * (full_T * lin + R * att(P + S_, 0))
-    return {"workload": f"config4: {n_layers}-layer 8B-shape stack, {R} requests x ({P} cached + {S_} suffix), rank 32",
+    return {"workload": f"{name}: {n_layers}-layer 8B-shape stack, {R} requests x ({P} cached + {S_} suffix), rank 32",
             "alora_ms": a_ms, "alora_suffix_tokens_per_s": T / (a_ms / 1e3), "alora_tflops": flop_a / (a_ms / 1e3) / 1e12,
             "full_lora_recompute_ms": r_ms, "recompute_tflops": flop_r / (r_ms / 1e3) / 1e12,
             "speedup_alora_vs_full_lora": r_ms / a_ms, "flop_ratio": flop_r / flop_a,
@@ -586,8 +715,11 @@ def main():
     ap.add_argument("--no-recompute", action="store_true", help="skip the full-LoRA recompute comparisons")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the decode and short-suffix legs")
-    ap.add_argument("--legs", default="decode,short,recompute8k,evaluators,stack",
-                    help="extra legs to run after the main workload (comma list of decode, short, recompute8k, evaluators, stack)")
+    ap.add_argument("--legs", default="sustained,config3,decode,short,recompute8k,stack8k,evaluators,stack",
+                    help="extra legs to run after the main workload (comma list of sustained, config3, decode, short, "
+                         "recompute8k, stack8k, evaluators, stack)")
+    ap.add_argument("--min-seconds", type=float, default=1.0,
+                    help="length of the sustained pass: the headline step repeated until this much time has been timed")
     ap.add_argument("--decode-steps", type=int, default=256)
     ap.add_argument("--decode-ctx-max", type=int, default=32768)
     ap.add_argument("--requests", type=int, default=8)
@@ -804,7 +936,9 @@ def main():
             s8()
         recompute_8k = recompute_of(case_8k, timed(s8, 50, stream, flush))
 
-    decode = short = None
+    decode = short = sustained = None
+    if "sustained" in legs:
+        sustained = sustained_leg(step, stream, flush, local, args.min_seconds, proj_flops + attn_flops, peaks)
     if "decode" in legs:
         decode = decode_leg(ab, hp, ctx, shape, stream, flush, peaks, steps=args.decode_steps,
                             ctx_max=args.decode_ctx_max)
@@ -815,9 +949,16 @@ def main():
     ab.alora_destroy(ctx)
     want_cpu = rank == 0 and world == 1 and not args.no_cpu_baseline
     pool_np = main_case.pool.to(torch.float32).cpu().numpy() if want_cpu else None
-    stack = evaluators = None
-    if "evaluators" in legs or "stack" in legs:
+    stack = evaluators = config3 = stack_8k = None
+    if legs & {"evaluators", "stack", "stack8k", "config3"}:
         del main_case.pool
+        torch.cuda.empty_cache()
+    if "config3" in legs:
+        config3 = config3_leg(ab, hp, stream, local, flush, peaks)
+        torch.cuda.empty_cache()
+    if "stack8k" in legs:
+        stack_8k = stack_leg(ab, hp, shape, stream, local, seed=8, requests=8, prefix=8192, suffix=256, n_layers=4,
+                             name="8K-prefix comparison through whole layers")
         torch.cuda.empty_cache()
     if "evaluators" in legs:
         evaluators = [evaluator_leg(ab, hp, shape, stream, local, n) for n in (1, 5)]
@@ -847,7 +988,10 @@ def main():
                                       "how": "K steps as a 3-stream pipeline (H2D, kernels, D2H; double-buffered), total time / K; serial = one step at a time"},
             "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
             "full_lora_recompute": recompute, "full_lora_recompute_8k_prefix": recompute_8k,
-            "decode": decode, "short_suffix": short, "evaluator_pipeline": evaluators, "stack": stack, "device_status": status,
+            "sustained": sustained, "config3": config3, "decode": decode, "short_suffix": short,
+            "evaluator_pipeline": evaluators, "stack_8k_prefix": stack_8k, "stack": stack, "device_status": status,
+            # the figures of merit in one place, last, so that a truncated copy of this line still carries them
+            "fractions": fractions(peaks, roofline, sustained, config3, decode, short, recompute_8k, stack_8k, stack, evaluators),
         }))
     if world > 1:
         dist.destroy_process_group()
