@@ -212,13 +212,25 @@ class Oracle:
         assert rc == 0
         return y
 
+    # ---- optional rotary position embedding ------------------------------------------------------
+    def rope(self, x, positions, n_heads: int, hd: int, theta: float) -> np.ndarray:
+        """Rotate-half rotary embedding of rows [T, n_heads*hd] at the given positions; returns a new array."""
+        x = _f64(x).copy()
+        positions = _i32(positions)
+        T = x.shape[0]
+        assert x.shape[1] == n_heads * hd and len(positions) == T
+        rc = self.lib.oracle_rope(_p(x, C.c_double), _p(positions, C.c_int32), T, n_heads, hd, C.c_double(float(theta)))
+        assert rc == 0, "oracle_rope: bad arguments"
+        return x
+
     # ---- compositions (no arithmetic of their own) ---------------------------------------------
     def attention_block(self, x, W, Nq, Nkv, Hq, Hkv, hd, positions, query_start_loc,
                         activation_offsets, adapter_ids, adapters, prefix_K, prefix_V,
-                        force_all=False, softmax_scale=None):
+                        force_all=False, softmax_scale=None, rope_theta=0.0):
         """One layer's attention block for new tokens on top of per-request cached K/V.
 
-        prefix_K[r], prefix_V[r]: [P_r, Nkv] arrays (P_r may be 0) holding positions 0..P_r-1;
+        prefix_K[r], prefix_V[r]: [P_r, Nkv] arrays (P_r may be 0) holding positions 0..P_r-1 (with
+        rope_theta set: keys as cached, i.e. already rotated);
         the new tokens of request r must be positions P_r, P_r+1, ...  Steps, in the order of
         Prop. 2's proof: (1) new q/k/v rows with the gate of Eq. 5, (2) append the new k/v rows
         behind the cached ones, (3) causal softmax attention of the new queries over all rows.
@@ -229,6 +241,11 @@ class Oracle:
         positions = _i32(positions)
         qkv, gate = self.project_qkv(x, W, Nq, Nkv, positions, qsl, activation_offsets, adapter_ids,
                                      adapters, force_all)
+        if rope_theta:
+            # optional: rotate the new query and key rows by their positions before the keys are cached
+            # (the cached prefix keys must then be post-rotation too)
+            qkv[:, :Nq] = self.rope(qkv[:, :Nq], positions, Hq, hd, rope_theta)
+            qkv[:, Nq:Nq + Nkv] = self.rope(qkv[:, Nq:Nq + Nkv], positions, Hkv, hd, rope_theta)
         Ks, Vs, kvl = [], [], [0]
         for r in range(R):
             lo, hi = qsl[r], qsl[r + 1]
@@ -247,12 +264,13 @@ class Oracle:
         return dict(qkv=qkv, gate=gate, K=Ks, V=Vs, out=out, pairs=pairs)
 
     def decoder_layer(self, h, lw: dict, Nq, Nkv, Hq, Hkv, hd, eps, positions, query_start_loc,
-                      activation_offsets, adapter_ids, adapters, prefix_K, prefix_V, force_all=False):
+                      activation_offsets, adapter_ids, adapters, prefix_K, prefix_V, force_all=False,
+                      rope_theta=0.0):
         """Pre-norm residual decoder layer: h + o_proj(attn(norm(h))), then + down(swiglu(gate_up(norm)))."""
         xn = self.rmsnorm(h, lw["norm_attn"], eps)
         blk = self.attention_block(xn, lw["wqkv"], Nq, Nkv, Hq, Hkv, hd, positions, query_start_loc,
                                    activation_offsets, adapter_ids, adapters, prefix_K, prefix_V,
-                                   force_all)
+                                   force_all, rope_theta=rope_theta)
         h1 = _f64(h) + self.linear(blk["out"], lw["wo"])
         xm = self.rmsnorm(h1, lw["norm_mlp"], eps)
         h2 = h1 + self.linear(self.swiglu(self.linear(xm, lw["wgate_up"])), lw["wdown"])

@@ -24,7 +24,9 @@
  * attention against a library softmax-attention routine and closed forms (single key, uniform
  * scores, two-key logistic weight, constant V), decode == prefill row, page-permutation
  * invariance, brute-force slot indices, the cache layout read back by plain array indexing, and
- * Prop. 2's closed-form pair and row counts.  tests/test_oracle_mutants.py plants one-line
+ * Prop. 2's closed-form pair and row counts; the optional rotary embedding by a complex-multiplication
+ * restatement, a hand example, norm preservation and the relative-position property.
+ * tests/test_oracle_mutants.py plants one-line
  * mistakes in a copy of this file and checks that the pins notice.
  * No function in this file is "parity unpinned".
  */
@@ -269,6 +271,35 @@ int oracle_paged_gather(const uint8_t *pool, int elem_size, const int32_t *block
                    pool + pool_row_offset(slot, 1, g, Hkv, page_size, hd) * elem_size, rowb);
         }
     }
+    return ORACLE_OK;
+}
+
+/*
+ * Rotary position embedding, "rotate-half" pairing, applied in place to rows of n_heads heads of hd columns.
+ * The paper's equations carry no positional encoding (positions enter only through the gate and the causal
+ * mask); the model families it evaluates are rotary models, so the rotation is an OPTION of the layer, off unless
+ * a base theta is given.  Reading taken: within a head, column i (0 <= i < hd/2) is paired with column i + hd/2;
+ * the pair at position p is turned by the angle p * theta^(-2i/hd):
+ *     x'[i]        = x[i] cos(a) - x[i + hd/2] sin(a)
+ *     x'[i + hd/2] = x[i + hd/2] cos(a) + x[i] sin(a)
+ * It is applied to the query and key rows after the projection (delta included) and before the keys are
+ * cached, so cached keys are post-rotation and a query-key score depends on the two positions only through
+ * their difference.
+ */
+int oracle_rope(double *x, const int32_t *positions, int T, int n_heads, int hd, double theta) {
+    if (!x || !positions || T < 0 || n_heads <= 0 || hd <= 0 || hd % 2 != 0 || !(theta > 0)) return ORACLE_ERR_ARG;
+    const int half = hd / 2;
+    for (int t = 0; t < T; ++t)
+        for (int h = 0; h < n_heads; ++h) {
+            double *v = x + ((size_t)t * n_heads + h) * hd;
+            for (int i = 0; i < half; ++i) {
+                const double a = (double)positions[t] * pow(theta, -2.0 * (double)i / (double)hd);
+                const real c = (real)cos(a), s = (real)sin(a);
+                const real lo = (real)v[i], hi = (real)v[i + half];
+                v[i] = (double)(lo * c - hi * s);
+                v[i + half] = (double)(hi * c + lo * s);
+            }
+        }
     return ORACLE_OK;
 }
 

@@ -72,6 +72,17 @@ C_MUTANTS = [
     ("return ((((size_t)page * 2 + (size_t)plane) * Hkv + (size_t)head) * page_size + (size_t)row) * hd;",
      "return ((((size_t)page * 2 + (size_t)plane) * page_size + (size_t)row) * Hkv + (size_t)head) * hd;",
      ["test_pool_layout_by_plain_indexing"]),
+    # rotary embedding: neighbouring columns paired instead of the two halves of the head
+    ("const real lo = (real)v[i], hi = (real)v[i + half];\n                v[i] = (double)(lo * c - hi * s);\n                v[i + half] = (double)(hi * c + lo * s);",
+     "const real lo = (real)v[2 * i], hi = (real)v[2 * i + 1];\n                v[2 * i] = (double)(lo * c - hi * s);\n                v[2 * i + 1] = (double)(hi * c + lo * s);",
+     ["test_rope_against_complex_multiplication_and_hand_example"]),
+    # ... the rotation turned the other way
+    ("v[i] = (double)(lo * c - hi * s);", "v[i] = (double)(lo * c + hi * s);",
+     ["test_rope_against_complex_multiplication_and_hand_example", "test_rope_scores_depend_on_the_position_difference_only"]),
+    # ... the frequency exponent without its factor two
+    ("const double a = (double)positions[t] * pow(theta, -2.0 * (double)i / (double)hd);",
+     "const double a = (double)positions[t] * pow(theta, -1.0 * (double)i / (double)hd);",
+     ["test_rope_against_complex_multiplication_and_hand_example"]),
     ("const real u = (real)gate_up[(size_t)t * 2 * I + I + i];",
      "const real u = (real)gate_up[(size_t)t * 2 * I + i]; (void)I;",
      ["test_rmsnorm_swiglu_linear_against_library", "test_decoder_layer_against_library_restatement"]),

@@ -527,3 +527,87 @@ def test_pool_layout_by_plain_indexing(oracle64):
         for g in range(Hkv):
             np.testing.assert_array_equal(K[p, g * hd:(g + 1) * hd], pool2[bt[0, p // ps], 0, g, p % ps, :])
             np.testing.assert_array_equal(V[p, g * hd:(g + 1) * hd], pool2[bt[0, p // ps], 1, g, p % ps, :])
+
+
+# ---- optional rotary position embedding -----------------------------------------------------------------
+
+def _rope_complex(x, positions, n_heads, hd, theta):
+    """Independent restatement: the pair (x[i], x[i + hd/2]) as the complex number x[i] + j x[i + hd/2], multiplied
+    by exp(j p theta^(-2i/hd))."""
+    T = x.shape[0]
+    v = np.asarray(x, np.float64).reshape(T, n_heads, 2, hd // 2)
+    z = v[:, :, 0, :] + 1j * v[:, :, 1, :]
+    freq = theta ** (-2.0 * np.arange(hd // 2) / hd)
+    z = z * np.exp(1j * np.asarray(positions, np.float64)[:, None, None] * freq[None, None, :])
+    return np.stack([z.real, z.imag], axis=2).reshape(T, n_heads * hd)
+
+
+def test_rope_against_complex_multiplication_and_hand_example(oracle64):
+    rng = np.random.default_rng(21)
+    x = rng.standard_normal((9, 3 * 16))
+    pos = np.array([0, 1, 2, 3, 17, 100, 1000, 4095, 32767], np.int32)
+    got = oracle64.rope(x, pos, 3, 16, 10000.0)
+    np.testing.assert_allclose(got, _rope_complex(x, pos, 3, 16, 10000.0), rtol=1e-12, atol=1e-12)
+    # position 0 is the identity; every head keeps its norm
+    np.testing.assert_array_equal(got[0], x[0])
+    np.testing.assert_allclose(np.linalg.norm(got.reshape(9, 3, 16), axis=2), np.linalg.norm(x.reshape(9, 3, 16), axis=2),
+                               rtol=1e-12)
+    assert np.abs(got[1:] - x[1:]).max() > 0.1
+    # hand-worked values (tests/golden/rope_hand_example.txt)
+    vals = {}
+    for line in open(os.path.join(os.path.dirname(__file__), "golden", "rope_hand_example.txt")):
+        line = line.split("#")[0].strip()
+        if "=" in line:
+            k, v = line.split("=")
+            vals[k.strip()] = [float(t) for t in v.split()]
+    y = oracle64.rope(np.array([vals["x"]]), [int(vals["p"][0])], 1, int(vals["hd"][0]), vals["theta"][0])
+    np.testing.assert_allclose(y[0], vals["y"], rtol=1e-13)
+
+
+def test_rope_scores_depend_on_the_position_difference_only(oracle64):
+    """<R_m q, R_n k> = <R_(m+s) q, R_(n+s) k> for any shift s: what makes cached post-rotation keys reusable."""
+    rng = np.random.default_rng(22)
+    q, k = rng.standard_normal((1, 32)), rng.standard_normal((1, 32))
+    base = None
+    for s in (0, 5, 900):
+        qm = oracle64.rope(q, [7 + s], 1, 32, 500.0)
+        kn = oracle64.rope(k, [3 + s], 1, 32, 500.0)
+        dot = float(qm[0] @ kn[0])
+        base = dot if base is None else base
+        assert abs(dot - base) < 1e-10
+    # ... and it does depend on the difference
+    assert abs(float(oracle64.rope(q, [8], 1, 32, 500.0)[0] @ oracle64.rope(k, [3], 1, 32, 500.0)[0]) - base) > 1e-3
+
+
+def test_rope_in_the_attention_block_is_rotation_then_plain_attention(oracle64):
+    """With rope_theta set the block equals: project, rotate q and k rows by hand (complex restatement), then the
+    plain block's attention on cached rotated keys.  Rows before the activation offset still equal the base
+    model's (Prop. 1 does not care about the rotation: it is the same function of the row on both sides)."""
+    W, ads, b = _setup(a_req=(9, 12))
+    A = [_ad(a) for a in ads]
+    kw = dict(Nq=SMALL.Nq, Nkv=SMALL.Nkv, Hq=4, Hkv=2, hd=8)
+    theta = 100.0
+    rng = np.random.default_rng(5)
+    Ks = [rng.standard_normal((int(p), SMALL.Nkv)) for p in b.prefix_lens]
+    Vs = [rng.standard_normal((int(p), SMALL.Nkv)) for p in b.prefix_lens]
+    got = oracle64.attention_block(b.hidden, W, positions=b.positions, query_start_loc=b.query_start_loc,
+                                   activation_offsets=b.activation_offsets, adapter_ids=b.adapter_ids, adapters=A,
+                                   prefix_K=Ks, prefix_V=Vs, rope_theta=theta, **kw)
+    qkv, _ = oracle64.project_qkv(b.hidden, W, SMALL.Nq, SMALL.Nkv, b.positions, b.query_start_loc,
+                                  b.activation_offsets, b.adapter_ids, A)
+    q = _rope_complex(qkv[:, :SMALL.Nq], b.positions, 4, 8, theta)
+    k = _rope_complex(qkv[:, SMALL.Nq:SMALL.Nq + SMALL.Nkv], b.positions, 2, 8, theta)
+    np.testing.assert_allclose(got["qkv"][:, :SMALL.Nq], q, rtol=1e-11, atol=1e-12)
+    np.testing.assert_allclose(got["qkv"][:, SMALL.Nq:SMALL.Nq + SMALL.Nkv], k, rtol=1e-11, atol=1e-12)
+    np.testing.assert_array_equal(got["qkv"][:, SMALL.Nq + SMALL.Nkv:], qkv[:, SMALL.Nq + SMALL.Nkv:])   # v is not rotated
+    Kc = np.concatenate([np.concatenate([Ks[r], k[b.query_start_loc[r]:b.query_start_loc[r + 1]]]) for r in range(b.R)])
+    Vc = np.concatenate([np.concatenate([Vs[r], qkv[b.query_start_loc[r]:b.query_start_loc[r + 1], SMALL.Nq + SMALL.Nkv:]])
+                         for r in range(b.R)])
+    kvl = np.concatenate([[0], np.cumsum(b.seq_lens)])
+    want, _ = oracle64.attention(q, Kc, Vc, kvl, b.positions, b.query_start_loc, 4, 2, 8)
+    np.testing.assert_allclose(got["out"], want, rtol=1e-11, atol=1e-12)
+    base = oracle64.attention_block(b.hidden, W, positions=b.positions, query_start_loc=b.query_start_loc,
+                                    activation_offsets=b.activation_offsets, adapter_ids=[-1, -1], adapters=A,
+                                    prefix_K=Ks, prefix_V=Vs, rope_theta=theta, **kw)
+    off = got["gate"] == 0
+    assert off.sum() == 2 and np.array_equal(got["qkv"][off], base["qkv"][off])
