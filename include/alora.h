@@ -89,9 +89,21 @@ typedef struct alora_config {
     int32_t max_tokens;    /* largest T of any call; sizes the context's workspaces               */
     int32_t max_requests;  /* largest R of any call                                               */
     float rms_eps;         /* RMSNorm epsilon (stack entry)                                       */
-    float rope_theta;      /* must be 0: the method's equations carry no positional rotation      */
+    float rope_theta;      /* 0 (default): no positional rotation, as in the method's equations;
+                              > 0: rotary embedding with this base, see below                      */
     float softmax_scale;   /* 0 => 1/sqrt(head_dim) (Eq. 1)                                       */
 } alora_config;
+
+/*
+ * Rotary position embedding (an option; the paper's equations carry no positional encoding, the model families it
+ * evaluates are rotary models).  With cfg->rope_theta > 0 the new query and key rows are rotated by their
+ * positions after the projection (delta included) and before the keys are cached: within a head, column i pairs
+ * with column i + head_dim/2 and the pair at position p turns by p * rope_theta^(-2i/head_dim).  Cached keys are
+ * therefore post-rotation, in every mode alike; rows whose gate is closed still equal the base model's rows bit
+ * for bit.  alora_project_qkv then hands out the rotated q and k rows (what alora_kv_append would cache and
+ * alora_attend would read).  On the layer paths the rotation and the KV append are one kernel.
+ * alora_project_qkv_static does not rotate.
+ */
 
 /*
  * Create a context on cfg->device.  Allocates the context-owned workspaces (per-token metadata,

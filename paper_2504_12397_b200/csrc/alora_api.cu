@@ -1,6 +1,7 @@
 // C ABI of the library: context management, argument checks, and the order in which the kernels
 // of one layer are enqueued.  No arithmetic of the method lives here.
 #include <algorithm>
+#include <cmath>
 #include <cstring>
 #include <new>
 
@@ -78,8 +79,9 @@ static alora_status run_layer(alora_ctx *ctx, int layer, const void *hidden, con
     // projection (the few-row projection launches them between its two kernels, the other routes right after).
     if ((k = launch_metadata(ctx, b, s, kMetaProjection)) < 0) return ALORA_ERR_UNSUPPORTED; n += k;
     bool kv_appended = false;
+    const bool rope = ctx->d_rope_inv_freq != nullptr;   // the rotation comes between projection and append
     ctx->pending_attn_meta = &b;
-    k = launch_project(ctx, layer, hidden, b.T, ctx->d_qkv, s, pool, b.num_pages, &kv_appended);
+    k = launch_project(ctx, layer, hidden, b.T, ctx->d_qkv, s, rope ? nullptr : pool, b.num_pages, &kv_appended);
     const bool attn_meta_pending = ctx->pending_attn_meta != nullptr;
     ctx->pending_attn_meta = nullptr;
     if (k < 0) return ALORA_ERR_UNSUPPORTED;
@@ -88,7 +90,10 @@ static alora_status run_layer(alora_ctx *ctx, int layer, const void *hidden, con
         if ((k = launch_metadata(ctx, b, s, kMetaAttention)) < 0) return ALORA_ERR_UNSUPPORTED;
         n += k;
     }
-    if (!kv_appended) {
+    if (rope) {   // rotate the new q and k rows by their positions and append the rotated keys and the values
+        if ((k = launch_rope(ctx, ctx->d_qkv, b.positions, b.T, pool, b.num_pages, s)) < 0) return ALORA_ERR_UNSUPPORTED;
+        n += k;
+    } else if (!kv_appended) {
         if ((k = launch_kv_append(ctx, ctx->d_qkv, b.T, b.num_pages, pool, s)) < 0) return ALORA_ERR_UNSUPPORTED;
         n += k;
     }
@@ -130,7 +135,7 @@ alora_status alora_create(const alora_config *cfg, alora_ctx **out) {
         return ALORA_ERR_INVALID_ARG;
     if (c.n_q_heads % c.n_kv_heads != 0) return ALORA_ERR_INVALID_ARG;
     if (c.dtype != ALORA_DTYPE_BF16 && c.dtype != ALORA_DTYPE_FP32) return ALORA_ERR_UNSUPPORTED;
-    if (c.rope_theta != 0.f) return ALORA_ERR_UNSUPPORTED;
+    if (c.rope_theta < 0.f || (c.rope_theta != 0.f && c.head_dim % 2 != 0)) return ALORA_ERR_INVALID_ARG;
     if (c.max_rank > kRankPadMax) return ALORA_ERR_UNSUPPORTED;
     if (c.head_dim != 32 && c.head_dim != 64 && c.head_dim != 128) return ALORA_ERR_UNSUPPORTED;
     if (c.n_q_heads / c.n_kv_heads > 8) return ALORA_ERR_UNSUPPORTED;
@@ -182,6 +187,7 @@ alora_status alora_create(const alora_config *cfg, alora_ctx **out) {
     alloc(&ctx->d_t, Tm * 3 * d.RP * 4);
     alloc(&ctx->d_qkv, Tm * d.N * es);
     alloc((void **)&ctx->d_status, 4);
+    if (c.rope_theta != 0.f) alloc((void **)&ctx->d_rope_inv_freq, (size_t)(c.head_dim / 2) * sizeof(double));
     alloc((void **)&ctx->d_iota, ((size_t)c.max_requests + 1) * 4);   // 0, 1, ..: query_start_loc of a decode batch
     ctx->layer_has_adapter.assign(c.n_layers, 0);
     if (c.dtype == ALORA_DTYPE_BF16 && 128 % d.G == 0) {
@@ -257,6 +263,11 @@ alora_status alora_create(const alora_config *cfg, alora_ctx **out) {
         e = cudaMemset(ctx->d_status, 0, 4);
         if (e == cudaSuccess) e = cudaMemset(ctx->d_adapters, 0, n_ad * sizeof(AdapterDev));
         if (e == cudaSuccess) e = cudaMemset(ctx->d_counts, 0, 64);
+        if (e == cudaSuccess && ctx->d_rope_inv_freq) {
+            std::vector<double> f((size_t)c.head_dim / 2);
+            for (size_t i = 0; i < f.size(); ++i) f[i] = pow((double)c.rope_theta, -2.0 * (double)i / (double)c.head_dim);
+            e = cudaMemcpy(ctx->d_rope_inv_freq, f.data(), f.size() * sizeof(double), cudaMemcpyHostToDevice);
+        }
         if (e == cudaSuccess) {
             std::vector<int32_t> iota((size_t)c.max_requests + 1);
             for (size_t i = 0; i < iota.size(); ++i) iota[i] = (int32_t)i;
@@ -279,7 +290,7 @@ alora_status alora_destroy(alora_ctx *ctx) {
                     ctx->d_seg_scratch, ctx->d_shrink_tiles, ctx->d_t_ready, ctx->d_t, ctx->d_qkv, ctx->d_status, ctx->d_act[0], ctx->d_act[1],
                     ctx->d_act[2], ctx->d_act[3], ctx->d_iota, ctx->d_attn_items, ctx->d_attn_off, ctx->d_split_items,
                     ctx->d_req_scratch, ctx->d_part_o, ctx->d_part_ml, ctx->d_group_done, ctx->d_row_delta,
-                    ctx->d_skinny_part, ctx->d_skinny_t, ctx->d_skinny_meta,
+                    ctx->d_skinny_part, ctx->d_skinny_t, ctx->d_skinny_meta, ctx->d_rope_inv_freq,
                     ctx->d_attn_cta_start, ctx->d_attn_part_o, ctx->d_attn_part_ml};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (ctx->h_status) cudaFreeHost(ctx->h_status);
@@ -427,6 +438,11 @@ alora_status alora_project_qkv(alora_ctx *ctx, int layer, int mode, const void *
     int n = launch_metadata(ctx, b, s, kMetaProjection), k;
     if (n < 0) return ALORA_ERR_UNSUPPORTED;
     if ((k = launch_project(ctx, layer, d_hidden, T, d_qkv, s, nullptr, 0, nullptr)) < 0) return ALORA_ERR_UNSUPPORTED;
+    if (ctx->d_rope_inv_freq != nullptr) {   // the rows handed out are the rotated ones, as they would be cached
+        int k2 = launch_rope(ctx, d_qkv, d_positions, T, nullptr, 0, s);
+        if (k2 < 0) return ALORA_ERR_UNSUPPORTED;
+        k += k2;
+    }
     return finish(ctx, n + k);
 }
 

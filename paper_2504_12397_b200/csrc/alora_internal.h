@@ -168,6 +168,7 @@ struct alora_ctx {
     int skinny_max_items = 0, skinny_p_cap = 0;
     void *d_qkv = nullptr;        // [max_tokens][N]
     void *d_act[4] = {nullptr, nullptr, nullptr, nullptr};  // stack activations
+    double *d_rope_inv_freq = nullptr;   // [hd / 2] theta^(-2i/hd), only with a rotary base configured
     int32_t *d_status = nullptr;
     int32_t *h_status = nullptr;  // pinned
 
@@ -245,6 +246,7 @@ int launch_repack_adapter(alora_ctx *ctx, int rank, const void *Aq, const void *
 int launch_project(alora_ctx *ctx, int layer, const void *hidden, int T, void *qkv, cudaStream_t s, void *kv_pool,
                    int num_pages, bool *kv_appended);
 int launch_kv_append(alora_ctx *ctx, const void *qkv, int T, int num_pages, void *pool, cudaStream_t s);
+int launch_rope(alora_ctx *ctx, void *qkv, const int32_t *positions, int T, void *pool, int num_pages, cudaStream_t s);
 int launch_attend(alora_ctx *ctx, const void *qkv, const BatchArgs &b, const void *pool, void *out,
                   cudaStream_t s);
 int launch_linear(alora_ctx *ctx, const void *x, const void *W, int T, int K, int N, void *y,

@@ -285,6 +285,121 @@ int launch_kv_append(alora_ctx *ctx, const void *qkv, int T, int num_pages, void
 }
 
 // ---------------------------------------------------------------------------------------------
+// Optional rotary position embedding fused with the KV append (both data types).  The paper's equations carry no
+// positional rotation; with a base theta configured, the new query and key rows are rotated by their positions
+// ("rotate-half": column i of a head pairs with column i + hd/2, angle p * theta^(-2i/hd)) after the projection and
+// before the keys are cached, so the cache holds post-rotation keys.  One thread per (token, head, 16-byte vector
+// of pair indices): it rotates the pairs in place in the fused q/k/v row and, for key heads, also writes the rotated
+// vectors to the token's cache slot; a second index range copies the value rows to the cache.  The angle is formed
+// and reduced to [-pi, pi] in double precision (positions reach tens of thousands of radians), the sine and
+// cosine of the remainder in single.  Without a pool only the in-place rotation happens.
+// ---------------------------------------------------------------------------------------------
+template <typename T> struct Vec16;
+template <> struct Vec16<float> { static constexpr int kElems = 4; };
+template <> struct Vec16<__nv_bfloat16> { static constexpr int kElems = 8; };
+
+__device__ __forceinline__ void unpack16(const uint4 &u, float (&f)[4]) {
+    f[0] = __uint_as_float(u.x); f[1] = __uint_as_float(u.y); f[2] = __uint_as_float(u.z); f[3] = __uint_as_float(u.w);
+}
+__device__ __forceinline__ void unpack16(const uint4 &u, float (&f)[8]) {
+    const uint32_t w[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+    for (int e = 0; e < 4; ++e) {
+        const __nv_bfloat162 b2 = *reinterpret_cast<const __nv_bfloat162 *>(&w[e]);
+        f[2 * e] = __low2float(b2); f[2 * e + 1] = __high2float(b2);
+    }
+}
+__device__ __forceinline__ uint4 pack16(const float (&f)[4]) {
+    return make_uint4(__float_as_uint(f[0]), __float_as_uint(f[1]), __float_as_uint(f[2]), __float_as_uint(f[3]));
+}
+__device__ __forceinline__ uint4 pack16(const float (&f)[8]) {
+    uint4 u;
+    __nv_bfloat162 v;
+    v = __floats2bfloat162_rn(f[0], f[1]); u.x = *reinterpret_cast<uint32_t *>(&v);
+    v = __floats2bfloat162_rn(f[2], f[3]); u.y = *reinterpret_cast<uint32_t *>(&v);
+    v = __floats2bfloat162_rn(f[4], f[5]); u.z = *reinterpret_cast<uint32_t *>(&v);
+    v = __floats2bfloat162_rn(f[6], f[7]); u.w = *reinterpret_cast<uint32_t *>(&v);
+    return u;
+}
+
+template <typename T>
+__global__ void rope_append_kernel(uint4 *__restrict__ qkv, const int32_t *__restrict__ positions,
+                                   const int32_t *__restrict__ slot_map, const double *__restrict__ inv_freq, int Tn,
+                                   int N_vec, int n_rot_heads, int n_q_heads, int hd_vec, int Hkv, int page_size,
+                                   int num_pages, uint4 *__restrict__ pool, int32_t *status) {
+    constexpr int kE = Vec16<T>::kElems;
+    const int half_vec = hd_vec / 2;                       // vectors per half head
+    const int rot_units = n_rot_heads * half_vec;          // per token: (head, vector of pair indices)
+    const int copy_units = pool != nullptr ? Hkv * hd_vec : 0;   // per token: vectors of the value row
+    const int per_tok = rot_units + copy_units;
+    const size_t total = (size_t)Tn * per_tok;
+    for (size_t idx = blockIdx.x * (size_t)blockDim.x + threadIdx.x; idx < total; idx += (size_t)gridDim.x * blockDim.x) {
+        const int t = (int)(idx / per_tok), u = (int)(idx % per_tok);
+        int page = -1, prow = 0;
+        if (pool != nullptr) {
+            const int slot = slot_map[t];
+            if (slot >= 0) {
+                page = slot / page_size; prow = slot % page_size;
+                if (page >= num_pages) { report(status, ALORA_ERR_PAGE_RANGE); page = -1; }
+            }
+        }
+        uint4 *row = qkv + (size_t)t * N_vec;
+        if (u < rot_units) {
+            const int h = u / half_vec, iv = u % half_vec;   // heads 0 .. n_q_heads-1 are queries, the rest keys
+            uint4 *lo_p = row + (size_t)h * hd_vec + iv, *hi_p = lo_p + half_vec;
+            float lo[kE], hi[kE];
+            unpack16(*lo_p, lo); unpack16(*hi_p, hi);
+            const double p = (double)positions[t];
+#pragma unroll
+            for (int e = 0; e < kE; ++e) {
+                const double a = p * inv_freq[iv * kE + e];
+                const float r = (float)(a - 6.283185307179586476925 * rint(a * 0.15915494309189533577));
+                float sn, cs;
+                sincosf(r, &sn, &cs);
+                const float x0 = lo[e], x1 = hi[e];
+                lo[e] = x0 * cs - x1 * sn;
+                hi[e] = x1 * cs + x0 * sn;
+            }
+            const uint4 lo_u = pack16(lo), hi_u = pack16(hi);
+            *lo_p = lo_u; *hi_p = hi_u;
+            if (h >= n_q_heads && page >= 0) {   // a key head: the rotated vectors also go to the cache slot
+                const int kh = h - n_q_heads;
+                uint4 *dst = pool + ((((size_t)page * 2 + 0) * Hkv + kh) * page_size + prow) * hd_vec + iv;
+                dst[0] = lo_u; dst[half_vec] = hi_u;
+            }
+        } else if (page >= 0) {
+            const int c = u - rot_units, kh = c / hd_vec, dv = c % hd_vec;
+            pool[((((size_t)page * 2 + 1) * Hkv + kh) * page_size + prow) * hd_vec + dv] =
+                row[(size_t)(n_rot_heads + kh) * hd_vec + dv];
+        }
+    }
+}
+
+// Rotates the query and key parts of qkv[T][N] in place; with a pool also appends the (rotated) keys and the values.
+int launch_rope(alora_ctx *ctx, void *qkv, const int32_t *positions, int T, void *pool, int num_pages, cudaStream_t s) {
+    if (T == 0) return 0;
+    const Dims &d = ctx->d;
+    if (ctx->d_rope_inv_freq == nullptr) return -1;
+    const int vec = 16 / (int)ctx->esize;
+    if (d.hd % (2 * vec) != 0) return -1;
+    ProfScope prof(ctx, KK_KV_APPEND, s);
+    const int hd_vec = d.hd / vec;
+    const size_t per_tok = (size_t)(d.Hq + d.Hkv) * (hd_vec / 2) + (pool ? (size_t)d.Hkv * hd_vec : 0);
+    const size_t total = (size_t)T * per_tok;
+    int blocks = (int)std::min<size_t>((total + 255) / 256, (size_t)ctx->sm_count * 16);
+    if (ctx->cfg.dtype == ALORA_DTYPE_FP32)
+        rope_append_kernel<float><<<blocks, 256, 0, s>>>((uint4 *)qkv, positions, ctx->d_slot, ctx->d_rope_inv_freq, T,
+                                                         d.N / vec, d.Hq + d.Hkv, d.Hq, hd_vec, d.Hkv, d.page, num_pages,
+                                                         (uint4 *)pool, ctx->d_status);
+    else
+        rope_append_kernel<__nv_bfloat16><<<blocks, 256, 0, s>>>((uint4 *)qkv, positions, ctx->d_slot,
+                                                                 ctx->d_rope_inv_freq, T, d.N / vec, d.Hq + d.Hkv, d.Hq,
+                                                                 hd_vec, d.Hkv, d.page, num_pages, (uint4 *)pool,
+                                                                 ctx->d_status);
+    return 1;
+}
+
+// ---------------------------------------------------------------------------------------------
 // CUDA-core attention (Eq. 1 / Eq. 3): one warp per (token, query head); the block holds the G query
 // heads that share a KV head.  Keys are taken 32 at a time: lane j scores key j0 + j against the
 // query kept in shared memory, the warp combines the 32 scores with shuffles (running maximum and

@@ -119,8 +119,9 @@ def oracle_adapters(ads):
     return [Adapter(a.rank, a.scale, a.Aq, a.Bq, a.Ak, a.Bk, a.Av, a.Bv) for a in ads]
 
 
-def oracle_base_prefix(orc, shape, wqkv, b: wl.Batch):
-    """Base-model K/V of every request's prefix, from the prefix hidden states (Eq. 2)."""
+def oracle_base_prefix(orc, shape, wqkv, b: wl.Batch, rope_theta: float = 0.0):
+    """Base-model K/V of every request's prefix, from the prefix hidden states (Eq. 2); with a rotary base, keys as
+    they would be cached (rotated by their positions)."""
     Ks, Vs = [], []
     for r in range(b.R):
         P = int(b.prefix_lens[r])
@@ -128,11 +129,14 @@ def oracle_base_prefix(orc, shape, wqkv, b: wl.Batch):
             Ks.append(None); Vs.append(None)
             continue
         qkv, _ = orc.project_qkv(b.prefix_hidden[r], wqkv, shape.Nq, shape.Nkv, np.arange(P), [0, P], [0], [-1], [])
-        Ks.append(qkv[:, shape.Nq:shape.Nq + shape.Nkv]); Vs.append(qkv[:, shape.Nq + shape.Nkv:])
+        k = qkv[:, shape.Nq:shape.Nq + shape.Nkv]
+        if rope_theta:
+            k = orc.rope(k, np.arange(P), shape.n_kv_heads, shape.head_dim, rope_theta)
+        Ks.append(k); Vs.append(qkv[:, shape.Nq + shape.Nkv:])
     return Ks, Vs
 
 
-def oracle_block(orc, shape, wqkv, ads, b: wl.Batch, Ks, Vs, force_all=False):
+def oracle_block(orc, shape, wqkv, ads, b: wl.Batch, Ks, Vs, force_all=False, rope_theta: float = 0.0):
     return orc.attention_block(b.hidden, wqkv, shape.Nq, shape.Nkv, shape.n_q_heads, shape.n_kv_heads, shape.head_dim,
                                b.positions, b.query_start_loc, b.activation_offsets, b.adapter_ids,
-                               oracle_adapters(ads), Ks, Vs, force_all=force_all)
+                               oracle_adapters(ads), Ks, Vs, force_all=force_all, rope_theta=rope_theta)
