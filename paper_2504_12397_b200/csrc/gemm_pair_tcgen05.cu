@@ -32,7 +32,8 @@ constexpr int kHalfAp = 128 * kBKp * 2;            // one row tile's x (or t) bl
 constexpr int kBBytesP = kBNp * kBKp * 2;          // 24 KB
 constexpr int kStageBytesP = 2 * kHalfAp + kBBytesP;
 constexpr int kBarOffP = kStagesP * kStageBytesP;
-constexpr int kSmemTotalP = kBarOffP + 256 + 1024;
+constexpr int kItemRingOffP = kBarOffP + 256;
+constexpr int kSmemTotalP = kItemRingOffP + 128 + 1024;
 constexpr int kShrinkColsP = 3 * kTensorRP;        // 192 columns of t = one column tile
 
 struct PairArgs {
@@ -50,6 +51,7 @@ struct PairArgs {
     __nv_bfloat16 *kv_pool;
     const int32_t *slot_map;
     int kv_hd_shift, kv_heads, kv_page_size, kv_num_pages;
+    int32_t *item_counters;         // [2] next unclaimed work item of the launch, blocks that have finished
     int32_t *status;
 };
 
@@ -119,8 +121,10 @@ gemm_pair_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_c
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(bars + 2 * kStagesP + 4);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 2 * kStagesP + 5);
 
+    tc::ItemRing ring{smem_base + kItemRingOffP, reinterpret_cast<volatile int *>(smem_al + kItemRingOffP + 16 * tc::kItemSlots)};
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     if (threadIdx.x == 0) {
+        ring.init(9);   // the issuing warp and the eight epilogue warps
         for (int s = 0; s < kStagesP; ++s) { tc::mbar_init(full_bar(s), 1); tc::mbar_init(empty_bar(s), 1); }
         tc::mbar_init(accf_bar, 1);
         tc::mbar_init(acce_bar(0), 4); tc::mbar_init(acce_bar(1), 4);
@@ -149,7 +153,34 @@ gemm_pair_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_c
             tc::tma_prefetch_desc(&tmX); tc::tma_prefetch_desc(&tmW);
             uint32_t kc = 0;        // ring slots filled so far
             bool ok = true;
-            for (int item = blockIdx.x; item < total && ok; item += gridDim.x) {
+            // Order of this block's items.  Shrink items (the head of the list) are claimed from a global counter by
+            // the blocks (see below which), one at a time, until none is left; only then does the block walk its
+            // projection items, which are dealt out by block index as if the shrink items sat at list positions
+            // 0 .. n_shrink-1 (what the first blocks to start normally take).  A projection item that waits for its row
+            // tile's t therefore waits for a shrink item that a RUNNING block has claimed, however few blocks are
+            // resident; and in the usual case every block keeps the items (and the L2 neighbours) it always had.
+            bool shrink_phase = n_shrink > 0;
+            int stat = (int)blockIdx.x;
+            if (shrink_phase && (int)blockIdx.x >= n_shrink) {
+                // The blocks with the lowest indices have a free place in their list and normally take the shrink items
+                // within a microsecond.  The others look on for a short while (about 30 us) and join the claiming
+                // only if the shrink items are still not all taken by then (blocks that have not been scheduled).
+                const long long t0 = clock64();
+                while (ld_acquire_p(a.item_counters) < n_shrink && clock64() - t0 < 60000) {}
+                if (ld_acquire_p(a.item_counters) >= n_shrink) shrink_phase = false;
+            }
+            while (ok) {
+                int item = -1;
+                if (shrink_phase) {
+                    item = atomicAdd(a.item_counters, 1);
+                    if (item >= n_shrink) { shrink_phase = false; item = -1; }
+                }
+                if (!shrink_phase && item < 0) {
+                    while (stat < n_shrink) stat += (int)gridDim.x;
+                    if (stat < total) { item = stat; stat += (int)gridDim.x; }
+                }
+                if (!ring.put(item, abort_flag)) { ok = false; break; }
+                if (item < 0) break;
                 const PairItem g = decode_pair(a, item, n_shrink, n_m, n_n);
                 const bool two = g.m[1] >= 0;
                 for (int kb = 0; kb < kb_main && ok; ++kb, ++kc) {
@@ -166,8 +197,8 @@ gemm_pair_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_c
                 // expand: per row tile with an adapter, one K block per q/k/v block the column tile touches
                 for (int h = 0; h < 2 && ok; ++h) {
                     if (g.m[h] < 0 || g.t[h].adapter < 0) continue;
-                    // t of this row tile is written by another block's shrink item: wait until its four
-                    // epilogue warps have published, then order the TMA read after their writes
+                    // t of this row tile is written by a shrink item (earlier in the list, so claimed by a running
+                    // block): wait until its four epilogue warps have published, then order the TMA read after it
                     const long long t0 = clock64();
                     while (ld_acquire_p(a.t_ready + g.m[h]) < 4) {
                         if (*abort_flag || clock64() - t0 > tc::kWaitCycleLimit) { *abort_flag = 1; ok = false; break; }
@@ -206,7 +237,9 @@ gemm_pair_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_c
         constexpr uint32_t idesc = tc::idesc_bf16_f32(128, kBNp);
         uint32_t kc = 0, it = 0;
         bool ok = true;
-        for (int item = blockIdx.x; item < total && ok; item += gridDim.x, ++it) {
+        for (;; ++it) {
+            const int item = ring.take(abort_flag);
+            if (item < 0) { ok = item == -1; break; }
             const PairItem g = decode_pair(a, item, n_shrink, n_m, n_n);
             const bool two = g.m[1] >= 0;
             for (int kb = 0; kb < kb_main && ok; ++kb, ++kc) {
@@ -268,7 +301,9 @@ gemm_pair_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_c
         const int my_h = (warp - 2) >> 2; // the half of tensor memory (row tile of the pair) this warp drains
         uint32_t it = 0;
         bool ok = true;
-        for (int item = blockIdx.x; item < total && ok; item += gridDim.x, ++it) {
+        for (;; ++it) {
+            const int item = ring.take(abort_flag);
+            if (item < 0) break;
             const PairItem g = decode_pair(a, item, n_shrink, n_m, n_n);
             if (!tc::mbar_wait(accf_bar, it & 1, abort_flag)) { ok = false; break; }
             tc::tc_fence_after();
@@ -366,6 +401,7 @@ gemm_pair_tcgen05_kernel(const __grid_constant__ CUtensorMap tmX, const __grid_c
     tc::tc_fence_before();
     __syncthreads();
     if (threadIdx.x == 0 && *abort_flag) report(a.status, ALORA_ERR_TIMEOUT);
+    if (threadIdx.x == 0) tc::item_counter_release(a.item_counters);
     if (warp == 1) {
         tc::tc_fence_after();
         tc::tmem_dealloc(tmem_base, 512);
@@ -436,6 +472,7 @@ int launch_project_pair_tc(alora_ctx *ctx, int layer, const void *hidden, int T,
     g.adapters = ctx->d_adapters + (size_t)layer * ctx->cfg.max_adapters;
     g.shrink_tiles = ctx->d_shrink_tiles; g.n_shrink_tiles = ctx->d_counts + 2;
     g.t_ready = ctx->d_t_ready; g.t_out = (__nv_bfloat16 *)ctx->d_t;
+    g.item_counters = ctx->d_counts + 10;
     if (kv_pool != nullptr) {
         int shift = 0;
         while ((1 << shift) < d.hd) ++shift;

@@ -68,6 +68,7 @@ struct GemmArgs {
     __nv_bfloat16 *kv_pool;
     const int32_t *slot_map;
     int kv_hd_shift, kv_heads, kv_page_size, kv_num_pages;
+    int32_t *item_counters;         // [2] next unclaimed work item of the launch, blocks that have finished
     int32_t *status;
 };
 
@@ -80,7 +81,8 @@ struct GemmSmem {
     static constexpr int kBBytes = BN * kBK * 2;
     static constexpr int kStageBytes = kABytes + kBBytes;
     static constexpr int kBarOffset = kStages * kStageBytes;
-    static constexpr int kTotal = kBarOffset + 256 + 1024;  // barriers + slack for 1024-byte alignment
+    static constexpr int kItemRingOffset = kBarOffset + 256;
+    static constexpr int kTotal = kItemRingOffset + 128 + 1024;  // barriers, item ring, slack for 1024-byte alignment
 };
 
 __device__ __forceinline__ ProjTile load_tile(const GemmArgs &a, int m, bool dense) {
@@ -146,11 +148,14 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     const uint32_t drain_bar = bar0 + 8u * (2 * kStages + 4);
     volatile uint32_t *tmem_slot = reinterpret_cast<volatile uint32_t *>(bars + 2 * kStages + 5);
     volatile int *abort_flag = reinterpret_cast<volatile int *>(bars + 2 * kStages + 6);
+    tc::ItemRing ring{smem_base + S::kItemRingOffset,
+                      reinterpret_cast<volatile int *>(smem_al + S::kItemRingOffset + 16 * tc::kItemSlots)};
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     constexpr uint32_t kTmemCols = (2 * BN <= 256) ? 256 : 512;
 
     if (threadIdx.x == 0) {
+        ring.init(5);   // the issuing warp and the four epilogue warps
         for (int s = 0; s < kStages; ++s) { tc::mbar_init(full_bar(s), 1); tc::mbar_init(empty_bar(s), 1); }
         for (int i = 0; i < 2; ++i) { tc::mbar_init(accf_bar(i), 1); tc::mbar_init(acce_bar(i), 4); }
         tc::mbar_init(drain_bar, 1);
@@ -180,7 +185,34 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             const uint32_t a_bytes = a.a_tile_bytes ? (uint32_t)a.a_tile_bytes : (uint32_t)S::kABytes;
             uint32_t kc = 0;        // ring slots filled so far
             bool ok = true;
-            for (int item = blockIdx.x; item < total && ok; item += gridDim.x) {
+            // Order of this block's items.  Shrink items (the head of the list) are claimed from a global counter by
+            // the blocks (see below which), one at a time, until none is left; only then does the block walk its
+            // projection items, which are dealt out by block index as if the shrink items sat at list positions
+            // 0 .. n_shrink-1 (what the first blocks to start normally take).  A projection item that waits for its row
+            // tile's t therefore waits for a shrink item that a RUNNING block has claimed, however few blocks are
+            // resident; and in the usual case every block keeps the items (and the L2 neighbours) it always had.
+            bool shrink_phase = n_shrink > 0;
+            int stat = (int)blockIdx.x;
+            if (shrink_phase && (int)blockIdx.x >= n_shrink) {
+                // The blocks with the lowest indices have a free place in their list and normally take the shrink items
+                // within a microsecond.  The others look on for a short while (about 30 us) and join the claiming
+                // only if the shrink items are still not all taken by then (blocks that have not been scheduled).
+                const long long t0 = clock64();
+                while (ld_acquire(a.item_counters) < n_shrink && clock64() - t0 < 60000) {}
+                if (ld_acquire(a.item_counters) >= n_shrink) shrink_phase = false;
+            }
+            while (ok) {
+                int item = -1;
+                if (shrink_phase) {
+                    item = atomicAdd(a.item_counters, 1);
+                    if (item >= n_shrink) { shrink_phase = false; item = -1; }
+                }
+                if (!shrink_phase && item < 0) {
+                    while (stat < n_shrink) stat += (int)gridDim.x;
+                    if (stat < total) { item = stat; stat += (int)gridDim.x; }
+                }
+                if (!ring.put(item, abort_flag)) { ok = false; break; }
+                if (item < 0) break;
                 const GemmItem g = decode_item(a, item, n_shrink, n_n, BN, dense);
                 const ProjTile t = g.t;
                 const int n0 = g.n0;
@@ -199,8 +231,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                         tc::tma_load_2d(sb, &tmB, full_bar(s), kb * kBK, n0);
                     } else {
                         if (n_shrink > 0) {
-                            // t of this row tile is written by another block's shrink item: wait until its four
-                            // epilogue warps have published, then order the TMA read after their writes
+                            // t of this row tile is written by a shrink item, which comes earlier in the list and has
+                            // therefore been claimed by a running block: wait until its four epilogue warps have
+                            // published, then order the TMA read after their writes
                             const long long t0 = clock64();
                             while (ld_acquire(a.t_ready + g.m) < 4) {
                                 if (*abort_flag || clock64() - t0 > tc::kWaitCycleLimit) { *abort_flag = 1; ok = false; break; }
@@ -239,7 +272,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             constexpr uint32_t idesc_shrink = tc::idesc_bf16_f32(kBM, BN >= kShrinkCols ? kShrinkCols : BN);
             uint32_t kc = 0, it = 0;
             bool ok = true;
-            for (int item = blockIdx.x; item < total && ok; item += gridDim.x) {
+            while (ok) {
+                const int item = ring.take(abort_flag);
+                if (item < 0) { ok = item == -1; break; }
                 const GemmItem g = decode_item(a, item, n_shrink, n_n, BN, dense);
                 const ProjTile t = g.t;
                 const int extra = (!g.shrink && t.adapter >= 0) ? 1 : 0;
@@ -281,7 +316,9 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
         const int q = warp & 3;  // tensor-memory lane quarter this warp may read
         uint32_t it = 0;
         bool ok = true;
-        for (int item = blockIdx.x; item < total && ok; item += gridDim.x) {
+        while (ok) {
+            const int item = ring.take(abort_flag);
+            if (item < 0) break;
             const GemmItem g = decode_item(a, item, n_shrink, n_n, BN, dense);
             const ProjTile t = g.t;
             const int n0 = g.n0;
@@ -391,6 +428,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
     tc::tc_fence_before();
     __syncthreads();
     if (threadIdx.x == 0 && *abort_flag) report(a.status, ALORA_ERR_TIMEOUT);
+    if (threadIdx.x == 0) tc::item_counter_release(a.item_counters);
     if (warp == 1) {
         tc::tc_fence_after();
         tc::tmem_dealloc(tmem_base, kTmemCols);
@@ -537,6 +575,7 @@ int launch_project_tc(alora_ctx *ctx, int layer, const void *hidden, int T, void
         g.tiles = ctx->d_tiles; g.n_row_tiles = ctx->d_counts; g.M = T; g.N = d.N; g.K = d.H;
         g.out = (__nv_bfloat16 *)qkv; g.ldo = d.N; g.residual = nullptr; g.adapters = ads;
         g.Nq = d.Nq; g.Nkv = d.Nkv; g.total_adapter_rows = d.N; g.status = ctx->d_status;
+        g.item_counters = ctx->d_counts + 10;
         if (may_rowwise) {
             g.rowwise_flag = ctx->d_counts + 5; g.row_delta = ctx->d_row_delta; g.row_adapter = ctx->d_row_adapter;
         }
@@ -590,7 +629,7 @@ int launch_linear_tc(alora_ctx *ctx, const void *x, const void *W, int T, int K,
     g.a_tile_bytes = half_box ? (kBM / 2) * kBK * 2 : 0;
     g.tiles = nullptr; g.n_row_tiles = nullptr; g.M = T; g.N = N; g.K = K; g.out = (__nv_bfloat16 *)y; g.ldo = N;
     g.residual = (const __nv_bfloat16 *)residual; g.adapters = nullptr; g.Nq = N; g.Nkv = 0;
-    g.total_adapter_rows = 0; g.status = ctx->d_status;
+    g.total_adapter_rows = 0; g.status = ctx->d_status; g.item_counters = ctx->d_counts + 10;
     const int items = ((T + kBM - 1) / kBM) * ((N + BN - 1) / BN);
     const bool ok = BN == 256 ? launch_gemm_bn<256>(ctx, tmX, tmW, tmX, tmW, tmW, g, items, s)
                     : BN == 128 ? launch_gemm_bn<128>(ctx, tmX, tmW, tmX, tmW, tmW, g, items, s)

@@ -162,6 +162,54 @@ __device__ __forceinline__ void tmem_ld_32x32(uint32_t taddr, uint32_t (&r)[32])
 }
 __device__ __forceinline__ void tmem_ld_wait() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
 
+// A block's work items travel from the one thread that decides their order (its producer) to the block's other
+// roles through a small ring in shared memory.  The producer may take items from a global counter: an item that
+// waits for the result of another item (a projection item for its row tile's shrink item) is only started once
+// every item it can wait for has been claimed, and a claimed item is on a block that is running, so no block ever
+// depends on one that has not been scheduled yet, however few blocks are resident.
+// Layout at `base` (shared memory): full[kItemSlots], empty[kItemSlots] barriers, then kItemSlots ints.
+constexpr int kItemSlots = 4;
+constexpr int kItemRingBytes = 16 * kItemSlots + 4 * kItemSlots;
+struct ItemRing {
+    uint32_t bar0;          // shared-memory address of full[0]
+    volatile int *slots;
+    uint32_t n = 0;         // items passed through this role so far
+    __device__ __forceinline__ uint32_t full(int s) const { return bar0 + 8u * s; }
+    __device__ __forceinline__ uint32_t empty(int s) const { return bar0 + 8u * (kItemSlots + s); }
+    __device__ __forceinline__ void init(int n_consumers) const {   // one thread, before the block-wide sync
+        for (int s = 0; s < kItemSlots; ++s) { mbar_init(full(s), 1); mbar_init(empty(s), n_consumers); }
+    }
+    // producer (one thread): publish `item` (-1: the list is exhausted); false when a wait expired
+    __device__ __forceinline__ bool put(int item, volatile int *abort_flag) {
+        const int s = n % kItemSlots;
+        if (!mbar_wait(empty(s), ((n / kItemSlots) & 1) ^ 1, abort_flag)) return false;
+        slots[s] = item;
+        mbar_arrive(full(s));
+        ++n;
+        return true;
+    }
+    // consumer (a whole warp): the next item, -1 at the end of the list, -2 when a wait expired
+    __device__ __forceinline__ int take(volatile int *abort_flag) {
+        const int s = n % kItemSlots;
+        const bool got = __all_sync(0xffffffffu, mbar_wait(full(s), (n / kItemSlots) & 1, abort_flag));
+        const int item = got ? slots[s] : -2;
+        __syncwarp();
+        if (got && (threadIdx.x & 31) == 0) mbar_arrive(empty(s));
+        ++n;
+        return item;
+    }
+};
+// At the end of a kernel that hands items out through a global counter: the last block to get here clears
+// the counter for the next launch.  counters[0] = next item, counters[1] = blocks that have finished.
+__device__ __forceinline__ void item_counter_release(int32_t *counters) {
+    __threadfence();
+    if (atomicAdd(counters + 1, 1) == (int)gridDim.x - 1) {
+        counters[0] = 0;
+        counters[1] = 0;
+        __threadfence();
+    }
+}
+
 __device__ __forceinline__ uint32_t pack_bf16(float lo, float hi) {
     __nv_bfloat162 v = __floats2bfloat162_rn(lo, hi);
     return *reinterpret_cast<uint32_t *>(&v);
