@@ -299,6 +299,32 @@ alora_status alora_project_qkv_static(int dtype, int hidden, int n_q, int n_kv, 
                                       const void *d_Bv, int T, int R, void *d_qkv, void *stream);
 
 /*
+ * Several adapters on one reused base-model cache (paper, section "Activated LoRA": N adapters invoked on the same
+ * conversation share its cache; Prop. 2, the N-adapter clause).  Requests whose block tables begin with the same
+ * physical pages read them through the same memory; no page is copied.  The attention of decode-sized requests
+ * (at most 16 / G new tokens each) additionally GROUPS neighbouring requests of a batch that have at least 256
+ * leading keys in common (whole pages before every member's first new position, up to 64 stacked score rows): the
+ * shared keys are then read once for all members, each member's own keys beyond them separately, and the parts are
+ * merged by their running maximum and sum.  The results are those of the ungrouped computation up to rounding.
+ *
+ * alora_prefix_groups reports the grouping of the last layer / attend call of this context: per request the index
+ * of its group's first request (its own index when ungrouped) and the number of keys the group shares (0 when
+ * ungrouped).  Device arrays of R int32 each; asynchronous on `stream`.  ALORA_ERR_UNSUPPORTED on an fp32 context.
+ *
+ * alora_cow_tail_pages is the copy-on-write step a caller needs when the reused length is not a multiple of the
+ * page size: the page that holds the last reused positions would also receive a request's first new rows.  For
+ * every request r with d_fresh_pages[r] >= 0 (a page id the caller took from its free list; -1: nothing to do) the
+ * rows of the reused positions on that page are copied to the fresh page (both planes, all KV heads) and
+ * d_block_tables[r] is redirected to it, in place.  Run it before the layer call; alora_validate_batch rejects a
+ * batch in which two requests would still write the same page.  Findings (fresh page out of range, request
+ * without new tokens) go to the status word.
+ */
+alora_status alora_prefix_groups(alora_ctx *ctx, int R, int32_t *d_group_first, int32_t *d_shared_keys, void *stream);
+alora_status alora_cow_tail_pages(alora_ctx *ctx, const int32_t *d_query_start_loc, const int32_t *d_seq_lens,
+                                  int32_t *d_block_tables, int max_blocks, int num_pages, int R,
+                                  const int32_t *d_fresh_pages, void *d_paged_kv, void *stream);
+
+/*
  * Self-test of the bounded waits (the paper has no counterpart).  Every wait inside the tensor-core kernels
  * (on a shared-memory barrier, on another block's ready counter) gives up after a cycle limit, records
  * ALORA_ERR_TIMEOUT in the status word and lets the kernel return through its normal exit.  This call runs that

@@ -240,6 +240,22 @@ def alora_get_status(ctx, stream=None) -> int:
     return int(out.value)
 
 
+def alora_prefix_groups(ctx, R, group_first, shared_keys, stream=None) -> None:
+    f = load_library().alora_prefix_groups
+    f.argtypes = [C.c_void_p, _I, _VP, _VP, _VP]
+    f.restype = C.c_int
+    _check(ctx, f(ctx, R, _ptr(group_first), _ptr(shared_keys), _stream(stream)), "alora_prefix_groups")
+
+
+def alora_cow_tail_pages(ctx, query_start_loc, seq_lens, block_tables, max_blocks, num_pages, R, fresh_pages, paged_kv,
+                         stream=None) -> None:
+    f = load_library().alora_cow_tail_pages
+    f.argtypes = [C.c_void_p, _VP, _VP, _VP, _I, _I, _I, _VP, _VP, _VP]
+    f.restype = C.c_int
+    _check(ctx, f(ctx, _ptr(query_start_loc), _ptr(seq_lens), _ptr(block_tables), max_blocks, num_pages, R,
+                  _ptr(fresh_pages), _ptr(paged_kv), _stream(stream)), "alora_cow_tail_pages")
+
+
 def alora_selftest_wait_timeout(ctx, limit_cycles: int, stream=None) -> None:
     f = load_library().alora_selftest_wait_timeout
     f.argtypes = [C.c_void_p, C.c_int64, _VP]

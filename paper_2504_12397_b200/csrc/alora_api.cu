@@ -208,11 +208,13 @@ alora_status alora_create(const alora_config *cfg, alora_ctx **out) {
             // the partial-result arrays
             ctx->small_max_tokens = std::max(1, 16 / d.G);
             const int blocks_per_req = std::max(1, (ctx->small_max_tokens * d.G + 63) / 64);
-            const int groups = c.max_requests * blocks_per_req * d.Hkv;
+            // (twice: in a prefix group every member adds a stream of its own keys to the shared one)
+            const int groups = 2 * c.max_requests * blocks_per_req * d.Hkv;
             ctx->max_split_items = kSplitItemsPerSm * ctx->sm_count + groups;
             ctx->max_split_rows = 16 * (kSplitItemsPerSm * ctx->sm_count + 4 * groups);
             alloc((void **)&ctx->d_split_items, (size_t)ctx->max_split_items * sizeof(AttnSplitWork));
-            alloc((void **)&ctx->d_req_scratch, (size_t)3 * c.max_requests * 4);
+            alloc((void **)&ctx->d_req_scratch, (size_t)5 * c.max_requests * 4);
+            alloc((void **)&ctx->d_prefix_groups, (size_t)2 * c.max_requests * 4);
             alloc((void **)&ctx->d_part_o, (size_t)ctx->max_split_rows * d.hd * 4);
             alloc((void **)&ctx->d_part_ml, (size_t)ctx->max_split_rows * 2 * 4);
             alloc((void **)&ctx->d_group_done, (size_t)ctx->max_split_items * 4);
@@ -290,7 +292,7 @@ alora_status alora_destroy(alora_ctx *ctx) {
                     ctx->d_seg_scratch, ctx->d_shrink_tiles, ctx->d_t_ready, ctx->d_t, ctx->d_qkv, ctx->d_status, ctx->d_act[0], ctx->d_act[1],
                     ctx->d_act[2], ctx->d_act[3], ctx->d_iota, ctx->d_attn_items, ctx->d_attn_off, ctx->d_split_items,
                     ctx->d_req_scratch, ctx->d_part_o, ctx->d_part_ml, ctx->d_group_done, ctx->d_row_delta,
-                    ctx->d_skinny_part, ctx->d_skinny_t, ctx->d_skinny_meta, ctx->d_rope_inv_freq,
+                    ctx->d_skinny_part, ctx->d_skinny_t, ctx->d_skinny_meta, ctx->d_rope_inv_freq, ctx->d_prefix_groups,
                     ctx->d_attn_cta_start, ctx->d_attn_part_o, ctx->d_attn_part_ml};
     for (void *p : ptrs) if (p) cudaFree(p);
     if (ctx->h_status) cudaFreeHost(ctx->h_status);
@@ -593,6 +595,32 @@ alora_status alora_forward_stack(alora_ctx *ctx, int mode, const void *d_hidden_
     }
 #undef ALORA_STEP
     return finish(ctx, n);
+}
+
+alora_status alora_prefix_groups(alora_ctx *ctx, int R, int32_t *d_group_first, int32_t *d_shared_keys, void *stream) {
+    if (!ctx || R < 0 || !d_group_first || !d_shared_keys) return ALORA_ERR_INVALID_ARG;
+    if (R > ctx->cfg.max_requests) return ALORA_ERR_CAPACITY;
+    if (!ctx->d_prefix_groups) return ALORA_ERR_UNSUPPORTED;
+    cudaStream_t s = (cudaStream_t)stream;
+    ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    if (R > 0) {
+        ALORA_CUDA(ctx, cudaMemcpyAsync(d_group_first, ctx->d_prefix_groups, (size_t)R * 4, cudaMemcpyDeviceToDevice, s));
+        ALORA_CUDA(ctx, cudaMemcpyAsync(d_shared_keys, ctx->d_prefix_groups + R, (size_t)R * 4, cudaMemcpyDeviceToDevice, s));
+    }
+    return ALORA_OK;
+}
+
+alora_status alora_cow_tail_pages(alora_ctx *ctx, const int32_t *d_query_start_loc, const int32_t *d_seq_lens,
+                                  int32_t *d_block_tables, int max_blocks, int num_pages, int R,
+                                  const int32_t *d_fresh_pages, void *d_paged_kv, void *stream) {
+    if (!ctx || R < 0 || !d_query_start_loc || !d_seq_lens || !d_block_tables || !d_fresh_pages || !d_paged_kv)
+        return ALORA_ERR_INVALID_ARG;
+    if (R > ctx->cfg.max_requests) return ALORA_ERR_CAPACITY;
+    if (max_blocks <= 0 || num_pages <= 0 || !aligned16(d_paged_kv)) return ALORA_ERR_INVALID_ARG;
+    cudaStream_t s = (cudaStream_t)stream;
+    ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    return finish(ctx, launch_cow_tail_pages(ctx, d_query_start_loc, d_seq_lens, d_block_tables, max_blocks, num_pages, R,
+                                             d_fresh_pages, d_paged_kv, s));
 }
 
 alora_status alora_profile_enable(alora_ctx *ctx, int on) {

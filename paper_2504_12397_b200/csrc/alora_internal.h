@@ -70,7 +70,10 @@ constexpr int kAttnSpreadMinGain = 24; // fewer items than blocks: spread them o
 struct AttnSplitWork {
     int32_t req, q_start, q_count, kv_head;
     int32_t kv_start, kv_end, pos0, mt;      // pos0 = position of the first token of the block
-    int32_t split, n_splits, part_row0, pad_;  // part_row0 = first row of this item in the partial-result arrays
+    int32_t split, n_splits, part_row0;        // part_row0 = first row of this item in the partial-result arrays
+    int32_t pad_;   // 0: every token of the block sees keys up to its own position; else tok_lo | tok_n << 16: only tokens
+                    // [tok_lo, tok_lo + tok_n) of the block see this item's keys (token tok_lo at position pos0), the
+                    // other rows see none of them (a member's own keys in a prefix group)
 };
 constexpr int kSplitItemsPerSm = 16;   // target number of (row tile, key range) pairs per SM
 
@@ -154,7 +157,9 @@ struct alora_ctx {
     float *d_attn_part_ml = nullptr;          // [2 * n_sm][2][256] their exponent references and row sums
     // few-row attention (requests with at most small_max_tokens new tokens): split-KV work list and partials
     alora::AttnSplitWork *d_split_items = nullptr;
-    int32_t *d_req_scratch = nullptr;   // [3][max_requests] items per request, item offset, partial-row offset
+    int32_t *d_req_scratch = nullptr;   // [5][max_requests] items per request, item offset, partial-row offset, prefix groups
+    int32_t *d_prefix_groups = nullptr; // [2][max_requests] per request of the last batch: first request of its prefix
+                                        // group, keys the group shares (0: ungrouped)
     float *d_part_o = nullptr, *d_part_ml = nullptr;
     int32_t *d_group_done = nullptr;    // [max_split_items] finished key ranges per group (first item's index)
     int32_t max_split_items = 0, max_split_rows = 0, small_max_tokens = 0;
@@ -246,6 +251,8 @@ int launch_repack_adapter(alora_ctx *ctx, int rank, const void *Aq, const void *
 int launch_project(alora_ctx *ctx, int layer, const void *hidden, int T, void *qkv, cudaStream_t s, void *kv_pool,
                    int num_pages, bool *kv_appended);
 int launch_kv_append(alora_ctx *ctx, const void *qkv, int T, int num_pages, void *pool, cudaStream_t s);
+int launch_cow_tail_pages(alora_ctx *ctx, const int32_t *qsl, const int32_t *seq_lens, int32_t *block_tables, int max_blocks,
+                          int num_pages, int R, const int32_t *fresh_pages, void *pool, cudaStream_t s);
 int launch_rope(alora_ctx *ctx, void *qkv, const int32_t *positions, int T, void *pool, int num_pages, cudaStream_t s);
 int launch_attend(alora_ctx *ctx, const void *qkv, const BatchArgs &b, const void *pool, void *out,
                   cudaStream_t s);

@@ -302,8 +302,12 @@ attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmKV, const SplitArgs a)
             // causal limits of this thread's two rows (clamped to the item's key range)
             const int tok_lo = min((my_mt * 16 + qr) / a.G, w.q_count - 1);
             const int tok_hi = min((my_mt * 16 + qr + 8) / a.G, w.q_count - 1);
-            const int lim_lo = min(w.pos0 + tok_lo, w.kv_end - 1);
-            const int lim_hi = min(w.pos0 + tok_hi, w.kv_end - 1);
+            // (a member's own keys in a prefix group: only the member's tokens see them, the other rows nothing)
+            const int win_lo = w.pad_ & 0xffff, win_n = w.pad_ >> 16;
+            const bool in_lo = win_n == 0 || (tok_lo >= win_lo && tok_lo < win_lo + win_n);
+            const bool in_hi = win_n == 0 || (tok_hi >= win_lo && tok_hi < win_lo + win_n);
+            const int lim_lo = in_lo ? min(w.pos0 + tok_lo - win_lo, w.kv_end - 1) : -1;
+            const int lim_hi = in_hi ? min(w.pos0 + tok_hi - win_lo, w.kv_end - 1) : -1;
 
             float o[kNTiles][4];
 #pragma unroll

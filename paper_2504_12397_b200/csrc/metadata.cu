@@ -337,31 +337,144 @@ __device__ __forceinline__ void small_block_shape(int n_new, int G, int &mt, int
     nblk = (n_new + tok_per_blk - 1) / tok_per_blk;
 }
 
+// Requests that read one shared prefix cache (several adapters invoked on the same conversation: their block tables
+// start with the same physical pages).  Neighbouring requests of the few-row route are put into one PREFIX GROUP when
+// they have leading pages in common, so that the attention reads those pages once for all of them:
+//   common(r)  = the number of leading block-table entries that requests r-1 and r have in common, counted only over
+//                pages that lie wholly before both requests' first new position;
+//   a group starts at an eligible request f (1 .. small_max new tokens) and is extended by f+1, f+2, ... while the
+//   next request is eligible, common(next) * page_size >= kMinSharedKeys, and the stacked score rows (new tokens of
+//   all members x G) still fit into 64;  a group needs at least two members;
+//   its shared length is the smallest common() of its pairs, in keys, rounded down to a multiple of 64.
+// Output per request: grp_first (index of the group's first request; r itself when ungrouped) and grp_shared (the
+// shared keys, 0 when ungrouped).  Called by all threads of a block.
+constexpr int kMinSharedKeys = 256;
+__device__ __forceinline__ void metadata_prefix_groups(const int32_t *__restrict__ qsl, const int32_t *__restrict__ seq_lens,
+                                                       const int32_t *__restrict__ block_tables, int max_blocks, int R,
+                                                       int page_size, int G, int small_max,
+                                                       int32_t *__restrict__ grp_first, int32_t *__restrict__ grp_shared) {
+    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, n_warps = (int)blockDim.x >> 5;
+    // common(r), one warp per pair: 32 table entries at a time, the first mismatch found by a vote
+    for (int r = wid; r < R; r += n_warps) {
+        int common = 0;
+        if (r > 0) {
+            const int na = qsl[r] - qsl[r - 1], nb = qsl[r + 1] - qsl[r];
+            const int lim = min(min((seq_lens[r - 1] - na) / page_size, (seq_lens[r] - nb) / page_size), max_blocks);
+            const int32_t *ta = block_tables + (size_t)(r - 1) * max_blocks, *tb = block_tables + (size_t)r * max_blocks;
+            bool open = na > 0 && nb > 0 && na <= small_max && nb <= small_max;
+            for (int b0 = 0; b0 < lim && open; b0 += 32) {
+                const int b = b0 + lane;
+                const bool same = b < lim && ta[b] == tb[b];
+                const unsigned diff = __ballot_sync(0xffffffffu, !same);
+                if (diff == 0u) { common = b0 + 32; } else { common = b0 + (__ffs(diff) - 1); open = false; }
+            }
+            common = min(common, max(lim, 0));
+        }
+        if (lane == 0) grp_shared[r] = common * page_size;    // for now: keys in common with the left neighbour
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int f = 0;
+        while (f < R) {
+            const int nf = qsl[f + 1] - qsl[f];
+            int e = f + 1;
+            int shared = 0;
+            if (nf > 0 && nf <= small_max) {
+                int rows = nf * G, mn = 0x7fffffff;
+                while (e < R) {
+                    const int ne = qsl[e + 1] - qsl[e];
+                    const int c = grp_shared[e];
+                    if (!(ne > 0 && ne <= small_max) || c < kMinSharedKeys || rows + ne * G > 64) break;
+                    rows += ne * G;
+                    mn = min(mn, c);
+                    ++e;
+                }
+                if (e - f >= 2) shared = mn & ~63;
+            }
+            if (shared <= 0) { e = f + 1; shared = 0; }
+            for (int m = f; m < e; ++m) { grp_first[m] = f; }
+            // grp_shared[f + 1 .. e) still hold the pair values that the loop above read; overwrite after use
+            for (int m = f; m < e; ++m) grp_shared[m] = shared;
+            f = e;
+        }
+    }
+    __syncthreads();
+}
+
+// Work list of the few-row attention kernel.  A STREAM is one block of score rows with the keys it reads: for an
+// ungrouped request its blocks of up to 16 * mt rows over keys 0 .. causal limit; for a prefix group the stacked rows
+// of all members, over the shared prefix (read once, nothing masked) followed by every member's own keys beyond it
+// (masked so that only that member's rows see them).  A stream's keys are cut into ranges of at most `chunk` 64-key
+// units; the ranges of one (stream, KV head) are consecutive items and are merged by whichever block finishes last.
+// A group is owned by its first request: that request accounts for all of the group's items.
+struct GroupShape {
+    int n_members, n_tok, shared, mt;
+};
+__device__ __forceinline__ GroupShape group_shape(const int32_t *qsl, const int32_t *grp_first, const int32_t *grp_shared,
+                                                  int R, int f, int G) {
+    GroupShape g;
+    g.shared = grp_shared[f];
+    int e = f + 1;
+    while (e < R && grp_first[e] == f) ++e;
+    g.n_members = e - f;
+    g.n_tok = qsl[e] - qsl[f];
+    const int rows = g.n_tok * G;
+    g.mt = rows <= 16 ? 1 : (rows <= 32 ? 2 : 4);
+    return g;
+}
+// ranges of request r's share of the list for a given range length; also the 64-key units (weighted by row tiles)
+__device__ __forceinline__ void request_ranges(const int32_t *qsl, const int32_t *seq_lens, const int32_t *grp_first,
+                                               const int32_t *grp_shared, int R, int r, int G, int small_max, int chunk,
+                                               int &n_ranges, int &weighted_units, int &mt_out) {
+    n_ranges = 0; weighted_units = 0; mt_out = 1;
+    const int n_new = qsl[r + 1] - qsl[r];
+    if (n_new <= 0 || n_new > small_max) return;
+    if (grp_first[r] != r) return;                       // a member of a group: accounted for by the group's owner
+    if (grp_shared[r] > 0) {
+        const GroupShape g = group_shape(qsl, grp_first, grp_shared, R, r, G);
+        int units = g.shared / 64;
+        n_ranges = (units + chunk - 1) / chunk;
+        for (int m = r; m < r + g.n_members; ++m) {
+            const int tu = (seq_lens[m] - g.shared + 63) / 64;
+            units += tu;
+            n_ranges += (tu + chunk - 1) / chunk;
+        }
+        weighted_units = units * g.mt;
+        mt_out = g.mt;
+        return;
+    }
+    int mt, tpb, nblk;
+    small_block_shape(n_new, G, mt, tpb, nblk);
+    for (int blk = 0; blk < nblk; ++blk) {
+        const int kv_end = seq_lens[r] - n_new + min(n_new, (blk + 1) * tpb);
+        const int u = (kv_end + 63) / 64;
+        weighted_units += u * mt;
+        n_ranges += (u + chunk - 1) / chunk;
+    }
+    mt_out = mt;
+}
+
 __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__ qsl, const int32_t *__restrict__ seq_lens,
+                                                     const int32_t *__restrict__ block_tables, int max_blocks, int page_size,
                                                      int R, int Hkv, int G, int n_sm, int small_max, int max_items, int max_rows,
                                                      AttnSplitWork *__restrict__ items, int32_t *__restrict__ counts,
-                                                     int32_t *req_scratch /* [3][R] */,
-                                                     int32_t *__restrict__ group_done, int32_t *status) {
+                                                     int32_t *req_scratch /* [5][R] */,
+                                                     int32_t *__restrict__ group_done, int32_t *__restrict__ groups_out,
+                                                     int32_t *status) {
     __shared__ unsigned long long tot_units;
     __shared__ int chunk_units, total_items, few_ranges;
     small_max = few_row_limit(qsl, R, Hkv, n_sm, small_max);
     int32_t *req_cnt = req_scratch, *req_off = req_scratch + R, *req_row = req_scratch + 2 * R;
-    // 64-key units of all blocks, weighted by the blocks' row tiles (an item of mt tiles needs mt * 16 partial rows):
+    int32_t *grp_first = req_scratch + 3 * R, *grp_shared = req_scratch + 4 * R;
+    metadata_prefix_groups(qsl, seq_lens, block_tables, max_blocks, R, page_size, G, small_max, grp_first, grp_shared);
+    if (groups_out != nullptr)
+        for (int r = threadIdx.x; r < R; r += blockDim.x) { groups_out[r] = grp_first[r]; groups_out[R + r] = grp_shared[r]; }
+    // 64-key units of all streams, weighted by their row tiles (an item of mt tiles needs mt * 16 partial rows):
     // per request in parallel, summed by one thread (a shared 64-bit atomic under contention is far slower)
     for (int r = threadIdx.x; r < R; r += blockDim.x) {
-        const int n_new = qsl[r + 1] - qsl[r];
-        int weighted = 0;
-        if (n_new > 0 && n_new <= small_max) {
-            int mt, tpb, nblk;
-            small_block_shape(n_new, G, mt, tpb, nblk);
-            int units = 0;
-            for (int blk = 0; blk < nblk; ++blk) {
-                const int kv_end = seq_lens[r] - n_new + min(n_new, (blk + 1) * tpb);
-                units += (kv_end + 63) / 64;
-            }
-            weighted = units * Hkv * mt;
-        }
-        req_cnt[r] = weighted;
+        int n, wu, mt;
+        request_ranges(qsl, seq_lens, grp_first, grp_shared, R, r, G, small_max, 1 << 20, n, wu, mt);
+        req_cnt[r] = wu * Hkv;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -401,15 +514,9 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
                 __syncthreads();
                 int mine = 0;
                 for (int r = threadIdx.x; r < R; r += blockDim.x) {
-                    const int n_new = qsl[r + 1] - qsl[r];
-                    if (n_new > 0 && n_new <= small_max) {
-                        int mt, tpb, nblk;
-                        small_block_shape(n_new, G, mt, tpb, nblk);
-                        for (int blk = 0; blk < nblk; ++blk) {
-                            const int kv_end = seq_lens[r] - n_new + min(n_new, (blk + 1) * tpb);
-                            mine += ((((kv_end + 63) / 64) + mid - 1) / mid) * Hkv;
-                        }
-                    }
+                    int n, wu, mt;
+                    request_ranges(qsl, seq_lens, grp_first, grp_shared, R, r, G, small_max, mid, n, wu, mt);
+                    mine += n * Hkv;
                 }
                 if (mine) atomicAdd(&cnt_acc, mine);
                 __syncthreads();
@@ -428,19 +535,10 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
     }
     const int chunk = chunk_units;
     for (int r = threadIdx.x; r < R; r += blockDim.x) {
-        const int n_new = qsl[r + 1] - qsl[r];
-        int cnt = 0, mt = 1;
-        if (n_new > 0 && n_new <= small_max) {
-            int tpb, nblk;
-            small_block_shape(n_new, G, mt, tpb, nblk);
-            for (int blk = 0; blk < nblk; ++blk) {
-                const int kv_end = seq_lens[r] - n_new + min(n_new, (blk + 1) * tpb);
-                cnt += (((kv_end + 63) / 64) + chunk - 1) / chunk;
-            }
-            cnt *= Hkv;
-        }
-        req_cnt[r] = cnt;
-        req_row[r] = cnt * 16 * mt;
+        int n, wu, mt;
+        request_ranges(qsl, seq_lens, grp_first, grp_shared, R, r, G, small_max, chunk, n, wu, mt);
+        req_cnt[r] = n * Hkv;
+        req_row[r] = n * Hkv * 16 * mt;
     }
     __syncthreads();
     if (threadIdx.x == 0) {
@@ -460,7 +558,7 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
     }
     __syncthreads();
     if (total_items == 0) return;
-    // one item per thread and step: request by binary search over the item offsets, then block / KV head / range
+    // one item per thread and step: owner request by binary search over the item offsets, then stream / KV head / range
     for (int i = threadIdx.x; i < total_items; i += blockDim.x) {
         int lo = 0, hi = R;   // largest r with req_off[r] <= i among requests that own items
         while (hi - lo > 1) {
@@ -468,10 +566,42 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
             if (req_off[mid] <= i) lo = mid; else hi = mid;
         }
         const int r = lo;
+        int local = i - req_off[r], row0 = req_row[r];
+        AttnSplitWork w;
+        if (grp_shared[r] > 0) {
+            // ---- a prefix group: per KV head [ranges of the shared prefix | ranges of member 0's own keys | member 1's | ..]
+            const GroupShape g = group_shape(qsl, grp_first, grp_shared, R, r, G);
+            const int pu = g.shared / 64, np = (pu + chunk - 1) / chunk;
+            int n_splits = np;
+            for (int m = r; m < r + g.n_members; ++m) n_splits += (((seq_lens[m] - g.shared + 63) / 64) + chunk - 1) / chunk;
+            const int kvh = local / n_splits, sp = local % n_splits;
+            w.q_start = qsl[r]; w.q_count = g.n_tok; w.kv_head = kvh; w.mt = g.mt; w.split = sp; w.n_splits = n_splits;
+            w.part_row0 = row0 + local * 16 * g.mt;
+            if (sp < np) {
+                const int per = (pu + np - 1) / np;
+                w.req = r; w.kv_start = sp * per * 64; w.kv_end = min(g.shared, (sp + 1) * per * 64);
+                w.pos0 = g.shared;    // every row sees every key of the shared prefix
+                w.pad_ = 0;
+            } else {
+                int sp2 = sp - np, m = r;
+                for (; m < r + g.n_members; ++m) {
+                    const int nt = (((seq_lens[m] - g.shared + 63) / 64) + chunk - 1) / chunk;
+                    if (sp2 < nt) break;
+                    sp2 -= nt;
+                }
+                const int tu = (seq_lens[m] - g.shared + 63) / 64, nt = (tu + chunk - 1) / chunk, per = (tu + nt - 1) / nt;
+                const int n_new = qsl[m + 1] - qsl[m];
+                w.req = m; w.kv_start = g.shared + sp2 * per * 64; w.kv_end = min(seq_lens[m], g.shared + (sp2 + 1) * per * 64);
+                w.pos0 = seq_lens[m] - n_new;                                     // position of the member's first new token
+                w.pad_ = (qsl[m] - qsl[r]) | (n_new << 16);                      // only the member's own tokens see these keys
+            }
+            group_done[i] = 0;
+            items[i] = w;
+            continue;
+        }
         const int n_new = qsl[r + 1] - qsl[r];
         int mt, tpb, nblk;
         small_block_shape(n_new, G, mt, tpb, nblk);
-        int local = i - req_off[r], row0 = req_row[r];
         for (int blk = 0; blk < nblk; ++blk) {
             const int q_count = min(tpb, n_new - blk * tpb);
             const int pos0 = seq_lens[r] - n_new + blk * tpb;
@@ -485,7 +615,6 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
             }
             const int per = (units + n_splits - 1) / n_splits;   // equal ranges rather than full ones and a stub
             const int kvh = local / n_splits, sp = local % n_splits;
-            AttnSplitWork w;
             w.req = r; w.q_start = qsl[r] + blk * tpb; w.q_count = q_count; w.kv_head = kvh;
             w.kv_start = sp * per * 64; w.kv_end = min(kv_end, (sp + 1) * per * 64);
             w.pos0 = pos0; w.mt = mt; w.split = sp; w.n_splits = n_splits; w.part_row0 = row0 + local * 16 * mt; w.pad_ = 0;
@@ -558,7 +687,7 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *a_req, con
                 AttnSplitWork *__restrict__ split_items,
                 int32_t *req_scratch, int32_t *__restrict__ group_done, int rowwise_cap,
                 int32_t *__restrict__ attn_cta_start, const AdapterDev *__restrict__ adapters, int phases,
-                FewRowMeta *__restrict__ few_row_meta, int32_t *status) {
+                FewRowMeta *__restrict__ few_row_meta, int32_t *__restrict__ prefix_groups, int32_t *status) {
     // The per-request inputs are read many times (binary searches, list builders): one parallel pass stages them
     // in shared memory, so that the later steps do not each pay a round trip to global memory.
     __shared__ int32_t s_req[4 * kMetaStageR + 1];
@@ -609,8 +738,8 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *a_req, con
         __syncthreads();
     }
     if ((int)blockIdx.x == b_split && split_items != nullptr && block_tables != nullptr)
-        metadata_split_items(qsl, seq_lens, R, Hkv, G, n_sm, small_max, max_split_items, max_split_rows, split_items, counts,
-                             req_scratch, group_done, status);
+        metadata_split_items(qsl, seq_lens, block_tables, max_blocks, page_size, R, Hkv, G, n_sm, small_max, max_split_items,
+                             max_split_rows, split_items, counts, req_scratch, group_done, prefix_groups, status);
     if (!proj) tc::grid_dep_wait();
 }
 
@@ -673,7 +802,7 @@ int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s, int phas
         ctx->d.Hkv, ctx->attn_q_block, ctx->max_attn_items, ctx->d_attn_items, ctx->d_attn_off, ctx->d.G,
         ctx->sm_count, ctx->small_max_tokens, ctx->max_split_items, ctx->max_split_rows, ctx->d_split_items,
         ctx->d_req_scratch, ctx->d_group_done, ctx->d_row_delta ? kRowwiseMaxTokens : 0,
-        ctx->d_attn_cta_start, ads, phases, few, ctx->d_status);
+        ctx->d_attn_cta_start, ads, phases, few, ctx->d_prefix_groups, ctx->d_status);
     return e == cudaSuccess ? 1 : -1;
 }
 

@@ -375,6 +375,46 @@ __global__ void rope_append_kernel(uint4 *__restrict__ qkv, const int32_t *__res
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Copy-on-write of a shared partial tail page.  Requests that reuse one base-model cache point at the same physical
+// pages; when the reused length is not a multiple of the page size, the page that holds the last cached positions
+// would also receive the request's first new rows.  Before the layer call, every such request gets a page of its
+// own: rows 0 .. (first new position % page_size) - 1 of the shared page are copied to the fresh page (both planes,
+// all KV heads) and the request's block-table entry is redirected.  One block per request.
+// ---------------------------------------------------------------------------------------------
+__global__ void cow_tail_pages_kernel(const int32_t *__restrict__ qsl, const int32_t *__restrict__ seq_lens,
+                                      int32_t *__restrict__ block_tables, int max_blocks, int num_pages, int page_size,
+                                      int Hkv, int hd_vec, const int32_t *__restrict__ fresh_pages,
+                                      uint4 *__restrict__ pool, int32_t *status) {
+    const int r = blockIdx.x;
+    const int fresh = fresh_pages[r];
+    if (fresh < 0) return;
+    const int n_new = qsl[r + 1] - qsl[r];
+    const int p_first = seq_lens[r] - n_new;
+    const int blk = p_first / page_size, rows = p_first % page_size;
+    if (n_new <= 0 || p_first < 0 || blk >= max_blocks) { if (threadIdx.x == 0) report(status, ALORA_ERR_BAD_BATCH); return; }
+    const int old = block_tables[(size_t)r * max_blocks + blk];
+    if (fresh >= num_pages || old < 0 || old >= num_pages) { if (threadIdx.x == 0) report(status, ALORA_ERR_PAGE_RANGE); return; }
+    const int per_head = rows * hd_vec, total = 2 * Hkv * per_head;
+    for (int i = threadIdx.x; i < total; i += blockDim.x) {
+        const int ph = i / per_head, v = i % per_head;    // (plane, head), vector inside the head's first `rows` rows
+        const size_t off = (size_t)ph * page_size * hd_vec + v;
+        pool[(size_t)fresh * 2 * Hkv * page_size * hd_vec + off] = pool[(size_t)old * 2 * Hkv * page_size * hd_vec + off];
+    }
+    __syncthreads();
+    if (threadIdx.x == 0) block_tables[(size_t)r * max_blocks + blk] = fresh;
+}
+
+int launch_cow_tail_pages(alora_ctx *ctx, const int32_t *qsl, const int32_t *seq_lens, int32_t *block_tables, int max_blocks,
+                          int num_pages, int R, const int32_t *fresh_pages, void *pool, cudaStream_t s) {
+    if (R == 0) return 0;
+    const Dims &d = ctx->d;
+    const int vec = 16 / (int)ctx->esize;
+    cow_tail_pages_kernel<<<R, 256, 0, s>>>(qsl, seq_lens, block_tables, max_blocks, num_pages, d.page, d.Hkv, d.hd / vec,
+                                            fresh_pages, (uint4 *)pool, ctx->d_status);
+    return 1;
+}
+
 // Rotates the query and key parts of qkv[T][N] in place; with a pool also appends the (rotated) keys and the values.
 int launch_rope(alora_ctx *ctx, void *qkv, const int32_t *positions, int T, void *pool, int num_pages, cudaStream_t s) {
     if (T == 0) return 0;
