@@ -71,10 +71,13 @@ struct AttnSplitWork {
     int32_t req, q_start, q_count, kv_head;
     int32_t kv_start, kv_end, pos0, mt;      // pos0 = position of the first token of the block
     int32_t split, n_splits, part_row0;        // part_row0 = first row of this item in the partial-result arrays
-    int32_t pad_;   // 0: every token of the block sees keys up to its own position; else tok_lo | tok_n << 16: only tokens
-                    // [tok_lo, tok_lo + tok_n) of the block see this item's keys (token tok_lo at position pos0), the
-                    // other rows see none of them (a member's own keys in a prefix group)
+    int32_t pad_;   // 0: every token of the block sees keys up to its own position.  kSplitOwnKeys | n_members: the item
+                    // covers the OWN keys of a prefix group's members (requests req .. req + n_members - 1), i.e. their
+                    // keys from position pos0 (the shared length) on, as one sequence of 64-key stages, member after
+                    // member; kv_start / kv_end count those stages (x 64); a stage's keys are seen by its member's
+                    // tokens only, up to each token's own position
 };
+constexpr int32_t kSplitOwnKeys = 0x40000000;
 constexpr int kSplitItemsPerSm = 16;   // target number of (row tile, key range) pairs per SM
 
 // Few-row projection (batches of at most kFewRowMax rows): what its two kernels need to know about the batch's

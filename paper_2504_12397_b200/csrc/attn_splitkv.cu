@@ -38,6 +38,7 @@ struct SplitArgs {
     const AttnSplitWork *items;
     const int32_t *n_items;
     const int32_t *block_tables;
+    const int32_t *qsl, *seq_lens;   // per request: first new token (flat), sequence length (prefix groups' own keys)
     int max_blocks, num_pages;
     int Hkv, G, page_size, box_rows;
     int N, Nq;
@@ -104,6 +105,18 @@ __device__ __forceinline__ bool consumer_barrier_or(bool pred) {
         "selp.u32 %0, 1, 0, p;\n\t}"
         : "=r"(r) : "r"((uint32_t)pred) : "memory");
     return r != 0;
+}
+
+// Stage `v` of the own keys of a prefix group's members (requests f .. f + n - 1, own keys from position `shared` on,
+// member after member in 64-key stages): which member, and the stage's first key position.
+__device__ __forceinline__ void own_key_stage(const int32_t *seq_lens, int f, int n, int shared, int v, int &member, int &kbase) {
+    int acc = 0;
+    member = f + n - 1; kbase = shared;
+    for (int m = f; m < f + n; ++m) {
+        const int nst = (seq_lens[m] - shared + kSkStageKeys - 1) / kSkStageKeys;
+        if (v < acc + nst) { member = m; kbase = shared + (v - acc) * kSkStageKeys; return; }
+        acc += nst;
+    }
 }
 
 // Merge of the key ranges of one block of rows: out = sum_s O_s 2^(m_s - M) / sum_s l_s 2^(m_s - M).
@@ -217,6 +230,34 @@ attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmKV, const SplitArgs a)
             // cover a whole number of 64-key stages, and key ranges start at multiples of 64).  A table entry is a
             // dependent load from global memory that would otherwise sit in front of every stage's copies; the
             // following window is in flight while this one is used.
+            if (w.pad_ & kSplitOwnKeys) {
+                // the own keys of a prefix group's members: every stage has its own request (table row) and positions
+                const int n_mem = w.pad_ & 0xffff;
+                for (int j = 0; j < n_st && ok; ++j, ++kt) {
+                    const int st = kt % kSkStages;
+                    int member, kbase;
+                    own_key_stage(a.seq_lens, w.req, n_mem, w.pos0, w.kv_start / kSkStageKeys + j, member, kbase);
+                    const int kend = a.seq_lens[member];
+                    const int units = min(units_per_stage, (kend - kbase + a.box_rows - 1) / a.box_rows);
+                    int row = -1;
+                    if (lane < units) {
+                        const int key = kbase + lane * a.box_rows;
+                        const int blk = key / a.page_size;
+                        const int page = blk < a.max_blocks ? a.block_tables[(size_t)member * a.max_blocks + blk] : -1;
+                        if (page < 0 || page >= a.num_pages) report(a.status, ALORA_ERR_PAGE_RANGE);
+                        else row = (page * 2 * a.Hkv + w.kv_head) * a.page_size + key % a.page_size;
+                    }
+                    const unsigned valid = __ballot_sync(0xffffffffu, row >= 0);
+                    if (lane == 0) {
+                        ok = tc::mbar_wait_relaxed(empty_bar(st), ((kt / kSkStages) & 1) ^ 1, abort_flag);
+                        if (ok) tc::mbar_arrive_expect_tx(full_bar(st), (uint32_t)__popc(valid) * unit_bytes);
+                    }
+                    ok = __shfl_sync(0xffffffffu, ok, 0);
+                    if (ok && row >= 0)
+                        tma_load_4d(smem_base + st * S::kStageBytes + lane * unit_bytes, &tmKV, full_bar(st), 0, row, 0, 0);
+                }
+                continue;
+            }
             const int32_t *bt_row = a.block_tables + (size_t)w.req * a.max_blocks;
             auto load_window = [&](int w0) { return w0 + lane < a.max_blocks ? bt_row[w0 + lane] : -1; };
             int win0 = (w.kv_start / a.page_size) & ~31;
@@ -302,12 +343,10 @@ attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmKV, const SplitArgs a)
             // causal limits of this thread's two rows (clamped to the item's key range)
             const int tok_lo = min((my_mt * 16 + qr) / a.G, w.q_count - 1);
             const int tok_hi = min((my_mt * 16 + qr + 8) / a.G, w.q_count - 1);
-            // (a member's own keys in a prefix group: only the member's tokens see them, the other rows nothing)
-            const int win_lo = w.pad_ & 0xffff, win_n = w.pad_ >> 16;
-            const bool in_lo = win_n == 0 || (tok_lo >= win_lo && tok_lo < win_lo + win_n);
-            const bool in_hi = win_n == 0 || (tok_hi >= win_lo && tok_hi < win_lo + win_n);
-            const int lim_lo = in_lo ? min(w.pos0 + tok_lo - win_lo, w.kv_end - 1) : -1;
-            const int lim_hi = in_hi ? min(w.pos0 + tok_hi - win_lo, w.kv_end - 1) : -1;
+            const bool own_keys = (w.pad_ & kSplitOwnKeys) != 0;   // a prefix group's own keys: limits change per stage
+            int lim_lo = min(w.pos0 + tok_lo, w.kv_end - 1);
+            int lim_hi = min(w.pos0 + tok_hi, w.kv_end - 1);
+            int kv_end_st = w.kv_end;
 
             float o[kNTiles][4];
 #pragma unroll
@@ -318,20 +357,30 @@ attn_splitkv_kernel(const __grid_constant__ CUtensorMap tmKV, const SplitArgs a)
                 const int st = kt % kSkStages;
                 if (!__all_sync(0xffffffffu, tc::mbar_wait(full_bar(st), (kt / kSkStages) & 1, abort_flag))) { ok = false; break; }
                 const uint32_t k_u32 = smem_base + st * S::kStageBytes;
-                const int kbase = w.kv_start + j * kSkStageKeys;
+                int kbase = w.kv_start + j * kSkStageKeys;
+                if (own_keys) {
+                    // this stage holds keys of one member: its tokens see them up to their own positions, the other
+                    // rows of the stacked block see none of them
+                    int member;
+                    own_key_stage(a.seq_lens, w.req, w.pad_ & 0xffff, w.pos0, w.kv_start / kSkStageKeys + j, member, kbase);
+                    kv_end_st = a.seq_lens[member];
+                    const int t0 = a.qsl[member] - w.q_start, nn = a.qsl[member + 1] - a.qsl[member], p0 = kv_end_st - nn;
+                    lim_lo = (tok_lo >= t0 && tok_lo < t0 + nn) ? p0 + tok_lo - t0 : -1;
+                    lim_hi = (tok_hi >= t0 && tok_hi < t0 + nn) ? p0 + tok_hi - t0 : -1;
+                }
 #pragma unroll 1
                 for (int sb = 0; sb < 4; ++sb) {
                     // 16-key sub-blocks are dealt round-robin over the key shares, across stages
                     if (((j * 4 + sb) & (n_kg - 1)) != kg) continue;
                     const int k0 = kbase + sb * 16;
-                    if (k0 >= w.kv_end) break;
-                    if (k0 + 16 > w.kv_end) {
+                    if (k0 >= kv_end_st) break;
+                    if (k0 + 16 > kv_end_st) {
                         // rows of keys beyond the range may hold anything: clear their V rows
                         uint8_t *v_gen = smem_al + st * S::kStageBytes + plane_bytes;
                         for (int i = lane; i < 16 * 8 * kHalves; i += 32) {
                             const int r = i / (8 * kHalves), c = i % (8 * kHalves);
                             const int key_l = sb * 16 + r;
-                            if (k0 + r >= w.kv_end)
+                            if (k0 + r >= kv_end_st)
                                 *reinterpret_cast<uint4 *>(v_gen + (key_l >> box_shift) * unit_bytes + (c / 8) * half_bytes +
                                                            (key_l & (a.box_rows - 1)) * 128 + (c % 8) * 16) = make_uint4(0, 0, 0, 0);
                         }
@@ -548,6 +597,7 @@ int launch_attend_splitkv(alora_ctx *ctx, const void *qkv, const BatchArgs &b, c
     }
     SplitArgs a{};
     a.items = ctx->d_split_items; a.n_items = ctx->d_counts + 3; a.block_tables = b.block_tables;
+    a.qsl = b.query_start_loc; a.seq_lens = b.seq_lens;
     a.max_blocks = b.max_blocks; a.num_pages = b.num_pages; a.Hkv = d.Hkv; a.G = d.G; a.page_size = d.page;
     a.box_rows = box_rows; a.N = d.N; a.Nq = d.Nq; a.scale_log2 = d.softmax_scale * 1.4426950408889634f;
     a.qkv = (const __nv_bfloat16 *)qkv; a.out = (__nv_bfloat16 *)out; a.part_o = ctx->d_part_o;

@@ -353,25 +353,31 @@ __device__ __forceinline__ void metadata_prefix_groups(const int32_t *__restrict
                                                        const int32_t *__restrict__ block_tables, int max_blocks, int R,
                                                        int page_size, int G, int small_max,
                                                        int32_t *__restrict__ grp_first, int32_t *__restrict__ grp_shared) {
-    const int lane = threadIdx.x & 31, wid = threadIdx.x >> 5, n_warps = (int)blockDim.x >> 5;
-    // common(r), one warp per pair: 32 table entries at a time, the first mismatch found by a vote
-    for (int r = wid; r < R; r += n_warps) {
-        int common = 0;
+    // common(r) for all pairs.  First the pairs that can share at all (both on this route, same first page): most
+    // pairs of unrelated requests end here.  Then, pair after pair, all threads compare the table entries below the
+    // pair's limit at once and keep the smallest mismatching index; no thread waits for another pair's loads.
+    for (int r = threadIdx.x; r < R; r += blockDim.x) {
+        int lim = 0;
         if (r > 0) {
             const int na = qsl[r] - qsl[r - 1], nb = qsl[r + 1] - qsl[r];
-            const int lim = min(min((seq_lens[r - 1] - na) / page_size, (seq_lens[r] - nb) / page_size), max_blocks);
-            const int32_t *ta = block_tables + (size_t)(r - 1) * max_blocks, *tb = block_tables + (size_t)r * max_blocks;
-            bool open = na > 0 && nb > 0 && na <= small_max && nb <= small_max;
-            for (int b0 = 0; b0 < lim && open; b0 += 32) {
-                const int b = b0 + lane;
-                const bool same = b < lim && ta[b] == tb[b];
-                const unsigned diff = __ballot_sync(0xffffffffu, !same);
-                if (diff == 0u) { common = b0 + 32; } else { common = b0 + (__ffs(diff) - 1); open = false; }
+            if (na > 0 && nb > 0 && na <= small_max && nb <= small_max) {
+                lim = min(min((seq_lens[r - 1] - na) / page_size, (seq_lens[r] - nb) / page_size), max_blocks);
+                if (lim > 0 && block_tables[(size_t)(r - 1) * max_blocks] != block_tables[(size_t)r * max_blocks]) lim = 0;
             }
-            common = min(common, max(lim, 0));
         }
-        if (lane == 0) grp_shared[r] = common * page_size;    // for now: keys in common with the left neighbour
+        grp_first[r] = max(lim, 0);    // for now: the pair's limit (0: nothing in common)
+        grp_shared[r] = max(lim, 0);   // for now: the first mismatching entry found so far (none yet)
     }
+    __syncthreads();
+    for (int r = 1; r < R; ++r) {
+        const int lim = grp_first[r];
+        if (lim <= 1) continue;
+        const int32_t *ta = block_tables + (size_t)(r - 1) * max_blocks, *tb = block_tables + (size_t)r * max_blocks;
+        for (int b = 1 + (int)threadIdx.x; b < lim; b += blockDim.x)
+            if (ta[b] != tb[b]) atomicMin(&grp_shared[r], b);
+    }
+    __syncthreads();
+    for (int r = threadIdx.x; r < R; r += blockDim.x) grp_shared[r] *= page_size;   // keys in common with the left neighbour
     __syncthreads();
     if (threadIdx.x == 0) {
         int f = 0;
@@ -432,14 +438,11 @@ __device__ __forceinline__ void request_ranges(const int32_t *qsl, const int32_t
     if (grp_first[r] != r) return;                       // a member of a group: accounted for by the group's owner
     if (grp_shared[r] > 0) {
         const GroupShape g = group_shape(qsl, grp_first, grp_shared, R, r, G);
-        int units = g.shared / 64;
-        n_ranges = (units + chunk - 1) / chunk;
-        for (int m = r; m < r + g.n_members; ++m) {
-            const int tu = (seq_lens[m] - g.shared + 63) / 64;
-            units += tu;
-            n_ranges += (tu + chunk - 1) / chunk;
-        }
-        weighted_units = units * g.mt;
+        const int pu = g.shared / 64;
+        int tu = 0;   // the members' own keys beyond the shared ones, member after member, in 64-key stages
+        for (int m = r; m < r + g.n_members; ++m) tu += (seq_lens[m] - g.shared + 63) / 64;
+        n_ranges = (pu + chunk - 1) / chunk + (tu + chunk - 1) / chunk;
+        weighted_units = (pu + tu) * g.mt;
         mt_out = g.mt;
         return;
     }
@@ -569,11 +572,14 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
         int local = i - req_off[r], row0 = req_row[r];
         AttnSplitWork w;
         if (grp_shared[r] > 0) {
-            // ---- a prefix group: per KV head [ranges of the shared prefix | ranges of member 0's own keys | member 1's | ..]
+            // ---- a prefix group: per KV head [ranges of the shared prefix | ranges of the members' own keys]; the own
+            // keys of all members form one sequence of 64-key stages (member after member) that is cut like any other
             const GroupShape g = group_shape(qsl, grp_first, grp_shared, R, r, G);
             const int pu = g.shared / 64, np = (pu + chunk - 1) / chunk;
-            int n_splits = np;
-            for (int m = r; m < r + g.n_members; ++m) n_splits += (((seq_lens[m] - g.shared + 63) / 64) + chunk - 1) / chunk;
+            int tu = 0;
+            for (int m = r; m < r + g.n_members; ++m) tu += (seq_lens[m] - g.shared + 63) / 64;
+            const int nt = (tu + chunk - 1) / chunk;
+            const int n_splits = np + nt;
             const int kvh = local / n_splits, sp = local % n_splits;
             w.q_start = qsl[r]; w.q_count = g.n_tok; w.kv_head = kvh; w.mt = g.mt; w.split = sp; w.n_splits = n_splits;
             w.part_row0 = row0 + local * 16 * g.mt;
@@ -583,17 +589,12 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
                 w.pos0 = g.shared;    // every row sees every key of the shared prefix
                 w.pad_ = 0;
             } else {
-                int sp2 = sp - np, m = r;
-                for (; m < r + g.n_members; ++m) {
-                    const int nt = (((seq_lens[m] - g.shared + 63) / 64) + chunk - 1) / chunk;
-                    if (sp2 < nt) break;
-                    sp2 -= nt;
-                }
-                const int tu = (seq_lens[m] - g.shared + 63) / 64, nt = (tu + chunk - 1) / chunk, per = (tu + nt - 1) / nt;
-                const int n_new = qsl[m + 1] - qsl[m];
-                w.req = m; w.kv_start = g.shared + sp2 * per * 64; w.kv_end = min(seq_lens[m], g.shared + (sp2 + 1) * per * 64);
-                w.pos0 = seq_lens[m] - n_new;                                     // position of the member's first new token
-                w.pad_ = (qsl[m] - qsl[r]) | (n_new << 16);                      // only the member's own tokens see these keys
+                // stages [kv_start / 64, kv_end / 64) of the members' own keys (not key positions: the kernel walks the
+                // members to find each stage's request, key positions and rows)
+                const int sp2 = sp - np, per = (tu + nt - 1) / nt;
+                w.req = r; w.kv_start = sp2 * per * 64; w.kv_end = min(tu, (sp2 + 1) * per) * 64;
+                w.pos0 = g.shared;
+                w.pad_ = kSplitOwnKeys | g.n_members;
             }
             group_done[i] = 0;
             items[i] = w;
