@@ -215,7 +215,8 @@ def dry_run(args, world: int, rank: int) -> None:
             dist.destroy_process_group()
 
 
-def fractions(peaks, roofline, sustained, config3, decode, short, recompute_8k, stack_8k, stack, evaluators):
+def fractions(peaks, roofline, sustained, config3, decode, short, recompute_8k, stack_8k, stack, evaluators,
+              evaluators_stack=None):
     """Compact summary of the roofline fractions and speed-ups of all legs (None where a leg did not run)."""
     r3 = lambda x: None if x is None else round(float(x), 3)   # noqa: E731
     out = {"peaks": {"bf16_tflops": peaks["bf16_tflops"], "bf16_tflops_sustained": peaks["bf16_tflops_sustained"],
@@ -250,6 +251,9 @@ def fractions(peaks, roofline, sustained, config3, decode, short, recompute_8k, 
     if evaluators:
         out["evaluator_stage_speedup"] = [r3(e["evaluator_stage_speedup"]) for e in evaluators]
         out["evaluator_pipeline_speedup"] = [r3(e["pipeline_speedup"]) for e in evaluators]
+    if evaluators_stack:
+        out["evaluator_stage_speedup_32_layers"] = [r3(e["evaluator_stage_speedup"]) for e in evaluators_stack]
+        out["evaluator_pipeline_speedup_32_layers"] = [r3(e["pipeline_speedup"]) for e in evaluators_stack]
     return out
 
 
@@ -618,6 +622,131 @@ def evaluator_leg(ab, hp, shape, stream, local, n_eval, seed=9, convs=8, prompt=
             "device_status": status, "output_finite": finite}
 
 
+def evaluator_stack_leg(ab, hp, shape, stream, local, n_eval, n_layers=32, seed=9, convs=8, prompt=4096, gen=256, inv=16,
+                        eval_steps=16):
+    """The evaluator workload of evaluator_leg through the whole decoder stack (n_layers layers: RMSNorm, attention
+    block with adapters on q/k/v, o_proj, SwiGLU MLP; random bf16 weights): base prefill of the prompts, `gen` base
+    decode steps, then `n_eval` adapters per conversation x (`inv` invocation tokens + `eval_steps` decode steps).
+    aLoRA evaluators reuse the conversation's pages in every layer; LoRA evaluators prefill everything again."""
+    import torch
+    rng = np.random.default_rng(seed)
+    ps = shape.page_size
+    ctx_len = prompt + gen
+    assert ctx_len % ps == 0
+    R2 = convs * n_eval
+    conv_blocks, own_blocks = ctx_len // ps, (inv + eval_steps + ps - 1) // ps
+    full_blocks = conv_blocks + own_blocks
+    num_pages = convs * conv_blocks + R2 * own_blocks + R2 * full_blocks + 3
+    order = rng.permutation(num_pages).astype(np.int32)
+    nxt = 0
+
+    def take(n):
+        nonlocal nxt
+        out = order[nxt:nxt + n]
+        nxt += n
+        return out
+    bt_conv = np.zeros((convs, full_blocks), np.int32)
+    for c in range(convs):
+        bt_conv[c, :conv_blocks] = take(conv_blocks)
+    bt_alora = np.zeros((R2, full_blocks), np.int32)
+    bt_lora = np.zeros((R2, full_blocks), np.int32)
+    for c in range(convs):
+        for n in range(n_eval):
+            r = c * n_eval + n
+            bt_alora[r, :conv_blocks] = bt_conv[c, :conv_blocks]
+            bt_alora[r, conv_blocks:] = take(own_blocks)
+            bt_lora[r] = take(full_blocks)
+    ids_eval = np.tile(np.arange(n_eval, dtype=np.int32), convs)
+    T_re = R2 * (ctx_len + inv)
+    T_max = max(T_re, convs * prompt)
+    H, I, Nq, Nkv = shape.hidden, shape.intermediate, shape.Nq, shape.Nkv
+    cfg = ab.make_config(hidden=H, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads, head_dim=shape.head_dim,
+                         page_size=ps, n_layers=n_layers, intermediate=I, max_adapters=max(n_eval, 1), max_rank=32,
+                         dtype=ab.DTYPE_BF16, device=local, max_tokens=T_max, max_requests=max(R2, convs))
+    ctx = ab.alora_create(cfg)
+    try:
+        keep = []
+        g = torch.Generator(device="cuda"); g.manual_seed(seed)
+
+        def rnd(*dims, std=0.02):
+            return (torch.randn(dims, generator=g, device="cuda", dtype=torch.float32) * std).to(torch.bfloat16)
+        for l in range(n_layers):
+            wts = [rnd(shape.N, H), rnd(H, Nq), rnd(2 * I, H), rnd(H, I),
+                   (1.0 + 0.1 * torch.randn(H, generator=g, device="cuda")).to(torch.bfloat16),
+                   (1.0 + 0.1 * torch.randn(H, generator=g, device="cuda")).to(torch.bfloat16)]
+            keep.append(wts)
+            ab.alora_set_layer_weights(ctx, l, *wts)
+            for i in range(n_eval):
+                ad = [rnd(32, H), rnd(Nq, 32), rnd(32, H), rnd(Nkv, 32), rnd(32, H), rnd(Nkv, 32)]
+                keep.append(ad)
+                ab.alora_register_adapter(ctx, i, l, 32, 1.0, *ad)
+        pools = [torch.zeros((num_pages, 2, shape.n_kv_heads, ps, shape.head_dim), device="cuda", dtype=torch.bfloat16)
+                 for _ in range(n_layers)]
+        hid = rnd(T_max, H, std=1.0)
+        out = torch.empty((T_max, H), dtype=torch.bfloat16, device="cuda")
+        i32 = lambda a: hp.idev(np.ascontiguousarray(a, dtype=np.int32))  # noqa: E731
+        p1 = dict(pos=i32(np.tile(np.arange(prompt), convs)), qsl=i32(np.arange(convs + 1) * prompt),
+                  lens=i32(np.full(convs, prompt)), ids=i32(np.full(convs, -1)), bt=i32(bt_conv))
+        p2_pos = i32(prompt + np.arange(gen)[:, None] + np.zeros((1, convs), np.int64))
+        p2_len = (p2_pos + 1).contiguous()
+        areq_conv = i32(np.zeros(convs))
+        p3 = dict(pos=i32(np.tile(ctx_len + np.arange(inv), R2)), qsl=i32(np.arange(R2 + 1) * inv),
+                  lens=i32(np.full(R2, ctx_len + inv)), ids=i32(ids_eval), areq=i32(np.full(R2, ctx_len)), bt=i32(bt_alora))
+        L3 = ctx_len + inv
+        p3l = dict(pos=i32(np.tile(np.arange(L3), R2)), qsl=i32(np.arange(R2 + 1) * L3), lens=i32(np.full(R2, L3)),
+                   ids=i32(ids_eval), bt=i32(bt_lora))
+        p4_pos = i32(L3 + np.arange(eval_steps)[:, None] + np.zeros((1, R2), np.int64))
+        p4_len = (p4_pos + 1).contiguous()
+        areq_open = i32(np.zeros(R2))
+
+        def base_phases():
+            ab.alora_forward_stack(ctx, ab.MODE_BASE, hid, p1["pos"], None, p1["ids"], p1["qsl"], p1["lens"], pools, p1["bt"],
+                                   full_blocks, num_pages, convs * prompt, convs, out, stream)
+            for i in range(gen):
+                ab.alora_decode_stack(ctx, hid, p2_pos[i], areq_conv, p1["ids"], p2_len[i], pools, p1["bt"], full_blocks,
+                                      num_pages, convs, out, stream)
+
+        def alora_eval():
+            ab.alora_forward_stack(ctx, ab.MODE_ALORA, hid, p3["pos"], p3["areq"], p3["ids"], p3["qsl"], p3["lens"], pools,
+                                   p3["bt"], full_blocks, num_pages, R2 * inv, R2, out, stream)
+            for i in range(eval_steps):
+                ab.alora_decode_stack(ctx, hid, p4_pos[i], p3["areq"], p3["ids"], p4_len[i], pools, p3["bt"], full_blocks,
+                                      num_pages, R2, out, stream)
+
+        def lora_eval():
+            ab.alora_forward_stack(ctx, ab.MODE_FULL_LORA, hid, p3l["pos"], None, p3l["ids"], p3l["qsl"], p3l["lens"], pools,
+                                   p3l["bt"], full_blocks, num_pages, T_re, R2, out, stream)
+            for i in range(eval_steps):
+                ab.alora_decode_stack(ctx, hid, p4_pos[i], areq_open, p3l["ids"], p4_len[i], pools, p3l["bt"], full_blocks,
+                                      num_pages, R2, out, stream)
+
+        def once(fn, warm):
+            if warm:
+                fn()
+            torch.cuda.synchronize()
+            e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            e0.record(stream)
+            fn()
+            e1.record(stream)
+            torch.cuda.synchronize()
+            return e0.elapsed_time(e1)
+        base_ms = once(base_phases, True)
+        alora_ms = once(alora_eval, True)
+        lora_ms = once(lora_eval, False)
+        status = ab.alora_get_status(ctx)
+        finite = bool(torch.isfinite(out[:R2].float()).all())
+    finally:
+        ab.alora_destroy(ctx)
+    return {"workload": f"{n_layers}-layer 8B-shape stack: {convs} conversations x ({prompt} prompt tokens, {gen} base decode "
+                        f"steps), then {n_eval} evaluator adapter(s) x ({inv} invocation tokens + {eval_steps} decode steps)",
+            "base_prefill_and_generation_ms": base_ms, "base_decode_ms_per_step_upper_bound": base_ms / gen,
+            "evaluators_alora_ms": alora_ms, "evaluators_lora_ms": lora_ms,
+            "evaluator_stage_speedup": lora_ms / alora_ms,
+            "pipeline_alora_ms": base_ms + alora_ms, "pipeline_lora_ms": base_ms + lora_ms,
+            "pipeline_speedup": (base_ms + lora_ms) / (base_ms + alora_ms),
+            "device_status": status, "output_finite": finite}
+
+
 def stack_leg(ab, hp, shape, stream, local, seed=4, requests=4, prefix=32768, suffix=1024, n_layers=32, name="config4"):
     """The decoder stack at the 8B shape (RMSNorm, attention block, o_proj, SwiGLU MLP; random bf16 weights):
     `requests` requests with `prefix` cached positions and `suffix` aLoRA suffix tokens each, against the
@@ -715,9 +844,9 @@ def main():
     ap.add_argument("--no-recompute", action="store_true", help="skip the full-LoRA recompute comparisons")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the decode and short-suffix legs")
-    ap.add_argument("--legs", default="sustained,config3,decode,short,recompute8k,stack8k,evaluators,stack",
+    ap.add_argument("--legs", default="sustained,config3,decode,short,recompute8k,stack8k,evaluators,evaluators_stack,stack",
                     help="extra legs to run after the main workload (comma list of sustained, config3, decode, short, "
-                         "recompute8k, stack8k, evaluators, stack)")
+                         "recompute8k, stack8k, evaluators, evaluators_stack, stack)")
     ap.add_argument("--min-seconds", type=float, default=1.0,
                     help="length of the sustained pass: the headline step repeated until this much time has been timed")
     ap.add_argument("--decode-steps", type=int, default=256)
@@ -949,8 +1078,8 @@ def main():
     ab.alora_destroy(ctx)
     want_cpu = rank == 0 and world == 1 and not args.no_cpu_baseline
     pool_np = main_case.pool.to(torch.float32).cpu().numpy() if want_cpu else None
-    stack = evaluators = config3 = stack_8k = None
-    if legs & {"evaluators", "stack", "stack8k", "config3"}:
+    stack = evaluators = config3 = stack_8k = evaluators_stack = None
+    if legs & {"evaluators", "evaluators_stack", "stack", "stack8k", "config3"}:
         del main_case.pool
         torch.cuda.empty_cache()
     if "config3" in legs:
@@ -963,6 +1092,11 @@ def main():
     if "evaluators" in legs:
         evaluators = [evaluator_leg(ab, hp, shape, stream, local, n) for n in (1, 5)]
         torch.cuda.empty_cache()
+    if "evaluators_stack" in legs:
+        evaluators_stack = []
+        for n in (1, 5):
+            evaluators_stack.append(evaluator_stack_leg(ab, hp, shape, stream, local, n))
+            torch.cuda.empty_cache()
     if "stack" in legs:
         stack = stack_leg(ab, hp, shape, stream, local)
     clocks_rest = sampler_rest.stop()
@@ -989,9 +1123,11 @@ def main():
             "gpu_launches": int(launches), "roofline": roofline, "cpu_baseline": cpu,
             "full_lora_recompute": recompute, "full_lora_recompute_8k_prefix": recompute_8k,
             "sustained": sustained, "config3": config3, "decode": decode, "short_suffix": short,
-            "evaluator_pipeline": evaluators, "stack_8k_prefix": stack_8k, "stack": stack, "device_status": status,
+            "evaluator_pipeline": evaluators, "evaluator_pipeline_32_layers": evaluators_stack,
+            "stack_8k_prefix": stack_8k, "stack": stack, "device_status": status,
             # the figures of merit in one place, last, so that a truncated copy of this line still carries them
-            "fractions": fractions(peaks, roofline, sustained, config3, decode, short, recompute_8k, stack_8k, stack, evaluators),
+            "fractions": fractions(peaks, roofline, sustained, config3, decode, short, recompute_8k, stack_8k, stack, evaluators,
+                                   evaluators_stack),
         }))
     if world > 1:
         dist.destroy_process_group()

@@ -299,6 +299,18 @@ alora_status alora_project_qkv_static(int dtype, int hidden, int n_q, int n_kv, 
                                       const void *d_Bv, int T, int R, void *d_qkv, void *stream);
 
 /*
+ * One decode step through all n_layers decoder layers: alora_forward_stack for a batch of R requests with one new
+ * token each (position d_positions[r] = d_seq_lens[r] - 1; Prop. 1, second sentence).  Rows before a request's
+ * activation offset, and requests with adapter id -1, run on the base weights.  d_hidden_in / d_hidden_out are
+ * [R][H]; the other arguments are those of alora_forward_stack and alora_decode_step.
+ */
+alora_status alora_decode_stack(alora_ctx *ctx, const void *d_hidden_in, const int32_t *d_positions,
+                                const int32_t *d_activation_offsets, const int32_t *d_adapter_ids,
+                                const int32_t *d_seq_lens, void *const *h_paged_kv_layers,
+                                const int32_t *d_block_tables, int max_blocks, int num_pages, int R,
+                                void *d_hidden_out, void *stream);
+
+/*
  * Several adapters on one reused base-model cache (paper, section "Activated LoRA": N adapters invoked on the same
  * conversation share its cache; Prop. 2, the N-adapter clause).  Requests whose block tables begin with the same
  * physical pages read them through the same memory; no page is copied.  The attention of decode-sized requests

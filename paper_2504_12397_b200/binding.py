@@ -234,6 +234,16 @@ def alora_forward_stack(ctx, mode, hidden_in, positions, activation_offsets, ada
     _check(ctx, rc, "alora_forward_stack")
 
 
+def alora_decode_stack(ctx, hidden_in, positions, activation_offsets, adapter_ids, seq_lens, paged_kv_layers: Sequence,
+                       block_tables, max_blocks, num_pages, R, hidden_out, stream=None):
+    arr = (_VP * len(paged_kv_layers))(*[_ptr(p) for p in paged_kv_layers])
+    f = load_library().alora_decode_stack
+    f.argtypes = [C.c_void_p] + [_VP] * 5 + [C.POINTER(_VP), _VP, _I, _I, _I, _VP, _VP]
+    f.restype = C.c_int
+    _check(ctx, f(ctx, _ptr(hidden_in), _ptr(positions), _ptr(activation_offsets), _ptr(adapter_ids), _ptr(seq_lens), arr,
+                  _ptr(block_tables), max_blocks, num_pages, R, _ptr(hidden_out), _stream(stream)), "alora_decode_stack")
+
+
 def alora_get_status(ctx, stream=None) -> int:
     out = C.c_int32(0)
     _check(ctx, load_library().alora_get_status(ctx, _stream(stream), C.byref(out)), "alora_get_status")

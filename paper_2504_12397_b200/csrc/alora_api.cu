@@ -623,6 +623,19 @@ alora_status alora_cow_tail_pages(alora_ctx *ctx, const int32_t *d_query_start_l
                                              d_fresh_pages, d_paged_kv, s));
 }
 
+alora_status alora_decode_stack(alora_ctx *ctx, const void *d_hidden_in, const int32_t *d_positions,
+                                const int32_t *d_activation_offsets, const int32_t *d_adapter_ids,
+                                const int32_t *d_seq_lens, void *const *h_paged_kv_layers, const int32_t *d_block_tables,
+                                int max_blocks, int num_pages, int R, void *d_hidden_out, void *stream) {
+    if (!ctx) return ALORA_ERR_INVALID_ARG;
+    if (R < 0) return ALORA_ERR_INVALID_ARG;
+    if (R > ctx->cfg.max_requests || R > ctx->cfg.max_tokens) return ALORA_ERR_CAPACITY;
+    // one new token per request: query_start_loc is 0, 1, ..., R (kept in the context)
+    return alora_forward_stack(ctx, ALORA_MODE_ALORA, d_hidden_in, d_positions, d_activation_offsets, d_adapter_ids,
+                               ctx->d_iota, d_seq_lens, h_paged_kv_layers, d_block_tables, max_blocks, num_pages, R, R,
+                               d_hidden_out, stream);
+}
+
 alora_status alora_profile_enable(alora_ctx *ctx, int on) {
     if (!ctx) return ALORA_ERR_INVALID_ARG;
     ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));

@@ -604,3 +604,61 @@ def test_device_side_findings_are_reported_not_trapped():
         assert g.status() == 0
     finally:
         g.close()
+
+
+def test_decode_steps_through_the_stack_match_the_prefill_rows(oracle64):
+    """Two decoder layers: a prefill of all but the last three tokens of every request, then three decode steps
+    through alora_decode_stack; the rows the steps produce equal the rows of the oracle's stack over the whole
+    sequences (Prop. 1, second sentence), for requests on two adapters and on the base model, with gates that open
+    before, inside and after the prefilled part."""
+    shape = wl.LayerShape(hidden=512, n_q_heads=4, n_kv_heads=2, head_dim=128, page_size=16, dtype="bf16",
+                          intermediate=1024)
+    rng = np.random.default_rng(37)
+    layers = [wl.make_stack_weights(shape, rng) for _ in range(2)]
+    ads = [[wl.make_adapter(shape, 16, rng), wl.make_adapter(shape, 8, rng)] for _ in range(2)]
+    for per in ads:
+        for a in per:
+            for n in ("Bq", "Bk", "Bv"):
+                setattr(a, n, wl.bf16_round(getattr(a, n) * 8))
+    L = [40, 23, 64, 9, 31]
+    ids = [0, 1, -1, 0, 1]
+    a_req = [10, 22, 0, 0, 100]
+    n_dec = 3
+    full = wl.make_batch(shape, [0] * len(L), L, ids, rng, activation_offsets=a_req, shuffle_pages=True)
+    R = full.R
+    g = hp.GpuLayers(shape, layers, ads, 256, 8)
+    try:
+        pools = [g.new_pool(full.num_pages) for _ in range(2)]
+        # prefill part: tokens 0 .. L-4 of every request
+        keep = np.concatenate([np.arange(full.query_start_loc[r], full.query_start_loc[r + 1] - n_dec) for r in range(R)])
+        pre = wl.Batch(positions=full.positions[keep],
+                       query_start_loc=np.concatenate([[0], np.cumsum(np.array(L) - n_dec)]).astype(np.int32),
+                       seq_lens=(np.array(L) - n_dec).astype(np.int32), prefix_lens=np.zeros(R, np.int32),
+                       activation_offsets=full.activation_offsets, adapter_ids=full.adapter_ids,
+                       block_tables=full.block_tables, num_pages=full.num_pages, hidden=full.hidden[keep])
+        d = hp.DevBatch(pre, shape.dtype)
+        hout = g.empty(pre.T, shape.hidden)
+        ab.alora_forward_stack(g.ctx, ab.MODE_ALORA, d.hidden, d.positions, d.a_req, d.ids, d.qsl, d.seq_lens, pools,
+                               d.bt, d.max_blocks, full.num_pages, d.T, d.R, hout)
+        got = np.zeros((R, n_dec, shape.hidden), np.float32)
+        for i in range(n_dec):
+            rows = full.query_start_loc[1:] - n_dec + i
+            pos = full.positions[rows]
+            hid = hp.to_dev(full.hidden[rows], "bf16")
+            o = g.empty(R, shape.hidden)
+            ab.alora_decode_stack(g.ctx, hid, hp.idev(pos), d.a_req, d.ids, hp.idev(pos + 1), pools, d.bt, d.max_blocks,
+                                  full.num_pages, R, o)
+            got[:, i] = hp.to_host(o)
+        assert g.status() == 0
+        x = full.hidden.astype(np.float64)
+        for l in range(2):
+            x, _ = oracle64.decoder_layer(x, layers[l], shape.Nq, shape.Nkv, shape.n_q_heads, shape.n_kv_heads,
+                                          shape.head_dim, 1e-5, full.positions, full.query_start_loc,
+                                          full.activation_offsets, full.adapter_ids, hp.oracle_adapters(ads[l]),
+                                          [None] * R, [None] * R)
+        for i in range(n_dec):
+            rows = full.query_start_loc[1:] - n_dec + i
+            hp.assert_close(got[:, i], x[rows], 2e-2, f"decode step {i} through the stack")
+        hp.assert_close(hp.to_host(hout), x[keep], 2e-2, "prefilled rows")
+    finally:
+        g.close()
