@@ -369,7 +369,7 @@ def decode_leg(ab, hp, ctx, shape, stream, flush, peaks, steps=256, seed=5, ctx_
         for i in range(n):
             ab.alora_decode_step(ctx, 0, hidden, pos_all[i], d_areq, d_ids, len_all[i], pool, d_bt, bt.shape[1],
                                  num_pages, R, out, stream)
-    run(8)
+    run(min(8, steps))
     torch.cuda.synchronize()
     assert ab.alora_get_status(ctx) == 0, "device-side finding in the decode leg"
     e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
@@ -851,6 +851,8 @@ def main():
                     help="length of the sustained pass: the headline step repeated until this much time has been timed")
     ap.add_argument("--decode-steps", type=int, default=256)
     ap.add_argument("--decode-ctx-max", type=int, default=32768)
+    ap.add_argument("--short-cases", default="8x4,8x16,64x4,64x16",
+                    help="the short-suffix leg's cases as requests x suffix tokens (on 4096 cached tokens each)")
     ap.add_argument("--requests", type=int, default=8)
     ap.add_argument("--prefix", type=int, default=4096)
     ap.add_argument("--suffix", type=int, default=256)
@@ -1073,7 +1075,7 @@ def main():
                             ctx_max=args.decode_ctx_max)
     if "short" in legs:
         short = [short_suffix_leg(ab, hp, ctx, shape, stream, flush, peaks, r_, 4096, s_)
-                 for r_, s_ in ((8, 4), (8, 16), (64, 4), (64, 16))]
+                 for r_, s_ in [tuple(int(v) for v in c.split("x")) for c in args.short_cases.split(",") if c]]
     status = ab.alora_get_status(ctx)
     ab.alora_destroy(ctx)
     want_cpu = rank == 0 and world == 1 and not args.no_cpu_baseline

@@ -497,7 +497,7 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
         const float per_sm = fminf(fmaxf(sqrtf(t_us / 12.f), 1.f), (float)kSplitItemsPerSm);
         const unsigned long long target = (unsigned long long)ceilf(per_sm * (float)max(n_sm, 1));
         chunk_units = (int)max(4ull, (tot_units + target - 1) / target);
-        few_ranges = per_sm < 2.5f ? 1 : 0;
+        few_ranges = (tot_units > 0 && per_sm < 2.5f) ? 1 : 0;
     }
     __syncthreads();
     // With only one or two ranges per SM the rule above ignores how the ranges fall into rounds over the SMs: 192
