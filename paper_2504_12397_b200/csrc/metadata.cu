@@ -377,8 +377,19 @@ __device__ __forceinline__ void metadata_prefix_groups(const int32_t *__restrict
             if (ta[b] != tb[b]) atomicMin(&grp_shared[r], b);
     }
     __syncthreads();
-    for (int r = threadIdx.x; r < R; r += blockDim.x) grp_shared[r] *= page_size;   // keys in common with the left neighbour
-    __syncthreads();
+    // keys in common with the left neighbour; most batches have no pair that shares enough: then nobody is grouped and
+    // the serial pass below (one thread walking the requests) is not needed
+    bool any = false;
+    for (int r = threadIdx.x; r < R; r += blockDim.x) {
+        const int keys = grp_shared[r] * page_size;
+        grp_shared[r] = keys;
+        any |= keys >= kMinSharedKeys;
+    }
+    if (!__syncthreads_or(any)) {
+        for (int r = threadIdx.x; r < R; r += blockDim.x) { grp_first[r] = r; grp_shared[r] = 0; }
+        __syncthreads();
+        return;
+    }
     if (threadIdx.x == 0) {
         int f = 0;
         while (f < R) {
@@ -463,14 +474,16 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
                                                      AttnSplitWork *__restrict__ items, int32_t *__restrict__ counts,
                                                      int32_t *req_scratch /* [5][R] */,
                                                      int32_t *__restrict__ group_done, int32_t *__restrict__ groups_out,
-                                                     int32_t *status) {
+                                                     int part, int n_parts, int32_t *status) {
+    // (several blocks may build the list together: each repeats the cheap per-request passes and fills the items
+    // part, part + n_parts, ..; block `part` 0 alone writes the counts and reports findings)
     __shared__ unsigned long long tot_units;
     __shared__ int chunk_units, total_items, few_ranges;
     small_max = few_row_limit(qsl, R, Hkv, n_sm, small_max);
     int32_t *req_cnt = req_scratch, *req_off = req_scratch + R, *req_row = req_scratch + 2 * R;
     int32_t *grp_first = req_scratch + 3 * R, *grp_shared = req_scratch + 4 * R;
     metadata_prefix_groups(qsl, seq_lens, block_tables, max_blocks, R, page_size, G, small_max, grp_first, grp_shared);
-    if (groups_out != nullptr)
+    if (groups_out != nullptr && part == 0)
         for (int r = threadIdx.x; r < R; r += blockDim.x) { groups_out[r] = grp_first[r]; groups_out[R + r] = grp_shared[r]; }
     // 64-key units of all streams, weighted by their row tiles (an item of mt tiles needs mt * 16 partial rows):
     // per request in parallel, summed by one thread (a shared 64-bit atomic under contention is far slower)
@@ -505,34 +518,31 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
     // length whose ranges fit into exactly one round, or into two, whichever the same cost model says is faster:
     // rounds x (12 us + range length x 0.74 us).  The range count for a given length is a sum over the requests.
     if (few_ranges) {
-        constexpr int kMaxChunkUnits = 1 << 14;   // 64-key units: a million keys
-        __shared__ int cnt_acc;
-        int best_chunk[2];
-        for (int w = 1; w <= 2; ++w) {
-            const int cap = w * n_sm;
-            int lo = 4, hi = kMaxChunkUnits;   // smallest chunk in [lo, hi] whose range count fits into cap (hi: one range per stream)
-            while (lo < hi) {
-                const int mid = (lo + hi) >> 1;
-                if (threadIdx.x == 0) cnt_acc = 0;
-                __syncthreads();
-                int mine = 0;
-                for (int r = threadIdx.x; r < R; r += blockDim.x) {
-                    int n, wu, mt;
-                    request_ranges(qsl, seq_lens, grp_first, grp_shared, R, r, G, small_max, mid, n, wu, mt);
-                    mine += n * Hkv;
-                }
-                if (mine) atomicAdd(&cnt_acc, mine);
-                __syncthreads();
-                const int cnt = cnt_acc;
-                __syncthreads();
-                if (cnt <= cap) hi = mid; else lo = mid + 1;
+        // every thread tries one candidate length (a grid over 4 .. the longest stream) and counts the ranges of the
+        // whole batch for it; the shortest candidates that fit one round and two rounds are kept
+        __shared__ int max_units, best1, best2;
+        if (threadIdx.x == 0) { max_units = 4; best1 = 0x7fffffff; best2 = 0x7fffffff; }
+        __syncthreads();
+        int mu = 0;
+        for (int r = threadIdx.x; r < R; r += blockDim.x) mu = max(mu, (seq_lens[r] + 63) / 64);
+        if (mu > 4) atomicMax(&max_units, mu);
+        __syncthreads();
+        const int step = (max_units - 4 + (int)blockDim.x - 1) / (int)blockDim.x + 0, cand = 4 + (int)threadIdx.x * max(step, 1);
+        if (cand <= max_units + max(step, 1)) {
+            int cnt = 0;
+            for (int r = 0; r < R; ++r) {
+                int n, wu, mt;
+                request_ranges(qsl, seq_lens, grp_first, grp_shared, R, r, G, small_max, cand, n, wu, mt);
+                cnt += n * Hkv;
             }
-            best_chunk[w - 1] = lo;
+            if (cnt <= n_sm) atomicMin(&best1, cand);
+            if (cnt <= 2 * n_sm) atomicMin(&best2, cand);
         }
+        __syncthreads();
         if (threadIdx.x == 0) {
-            const float c1 = 12.f + 0.74f * (float)best_chunk[0], c2 = 2.f * (12.f + 0.74f * (float)best_chunk[1]);
-            if (best_chunk[0] < kMaxChunkUnits && c1 <= c2) chunk_units = best_chunk[0];
-            else if (best_chunk[1] < kMaxChunkUnits) chunk_units = best_chunk[1];
+            const float c1 = 12.f + 0.74f * (float)best1, c2 = 2.f * (12.f + 0.74f * (float)best2);
+            if (best1 != 0x7fffffff && c1 <= c2) chunk_units = best1;
+            else if (best2 != 0x7fffffff) chunk_units = best2;
         }
         __syncthreads();
     }
@@ -552,17 +562,19 @@ __device__ __forceinline__ void metadata_split_items(const int32_t *__restrict__
             acc += c; rows += n;
         }
         if (acc > max_items || rows > max_rows) {
-            report(status, ALORA_ERR_CAPACITY);
+            if (part == 0) report(status, ALORA_ERR_CAPACITY);
             acc = 0;
         }
         total_items = acc;
-        counts[3] = acc;
-        counts[4] = 0;   // work counter of the few-row kernel
+        if (part == 0) {
+            counts[3] = acc;
+            counts[4] = 0;   // work counter of the few-row kernel
+        }
     }
     __syncthreads();
     if (total_items == 0) return;
     // one item per thread and step: owner request by binary search over the item offsets, then stream / KV head / range
-    for (int i = threadIdx.x; i < total_items; i += blockDim.x) {
+    for (int i = part * (int)blockDim.x + (int)threadIdx.x; i < total_items; i += n_parts * (int)blockDim.x) {
         int lo = 0, hi = R;   // largest r with req_off[r] <= i among requests that own items
         while (hi - lo > 1) {
             const int mid = (lo + hi) >> 1;
@@ -716,7 +728,10 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *a_req, con
     const int b_tiles = proj ? 0 : -1;
     const int b_attn = !attn ? -1 : (proj ? (nb > 1 ? 1 : 0) : 0);
     const int b_split = !attn ? -1 : (proj ? (nb > 2 ? 2 : 0) : (nb > 1 ? 1 : 0));
-    if ((int)blockIdx.x != b_tiles && (int)blockIdx.x != b_attn && (int)blockIdx.x != b_split) {
+    // the attention phase alone: block 0 builds the tensor-core kernel's list, all the others share the few-row list
+    const int split_parts = (!proj && attn && nb > 1) ? nb - 1 : 1;
+    const bool split_helper = !proj && attn && (int)blockIdx.x > b_split;
+    if ((int)blockIdx.x != b_tiles && (int)blockIdx.x != b_attn && (int)blockIdx.x != b_split && !split_helper) {
         if (!proj) tc::grid_dep_wait();
         return;
     }
@@ -738,9 +753,10 @@ metadata_kernel(const int32_t *__restrict__ positions, const int32_t *a_req, con
                             n_sm, attn_cta_start, status);
         __syncthreads();
     }
-    if ((int)blockIdx.x == b_split && split_items != nullptr && block_tables != nullptr)
+    if (((int)blockIdx.x == b_split || split_helper) && split_items != nullptr && block_tables != nullptr)
         metadata_split_items(qsl, seq_lens, block_tables, max_blocks, page_size, R, Hkv, G, n_sm, small_max, max_split_items,
-                             max_split_rows, split_items, counts, req_scratch, group_done, prefix_groups, status);
+                             max_split_rows, split_items, counts, req_scratch, group_done, prefix_groups,
+                             split_helper ? (int)blockIdx.x - b_split : 0, split_parts, status);
     if (!proj) tc::grid_dep_wait();
 }
 
@@ -785,7 +801,10 @@ int launch_metadata(alora_ctx *ctx, const BatchArgs &b, cudaStream_t s, int phas
     ctx->profiling = saved;
     const int threads = 256;
     const bool attn_only = phases == kMetaAttention;
-    const int grid = attn_only ? 2 : std::max((phases & kMetaAttention) ? 3 : 1, (b.T + threads - 1) / threads);
+    // (attention phase alone: one block for the tensor-core list, kSplitBuilders for the few-row list; they need the
+    // shared-memory scratch, i.e. batches of at most 511 requests, else one block builds it in the global scratch)
+    constexpr int kSplitBuilders = 8;
+    const int grid = attn_only ? (14 * b.R + 5 <= kMetaSmemInts ? 1 + kSplitBuilders : 2) : std::max((phases & kMetaAttention) ? 3 : 1, (b.T + threads - 1) / threads);
     const AdapterDev *ads = b.layer >= 0 ? ctx->d_adapters + (size_t)b.layer * ctx->cfg.max_adapters : nullptr;
     FewRowMeta *few = (b.few_row && ads != nullptr) ? (FewRowMeta *)ctx->d_skinny_meta : nullptr;
     if (phases == kMetaProjection && b.few_row && b.T <= kFewRowMax) {
