@@ -235,7 +235,7 @@ def fractions(peaks, roofline, sustained, config3, decode, short, recompute_8k, 
         out["config5_decode_projection_ms"] = r3(decode["per_kernel_ms"].get("project_qkv", 0.0) + decode["per_kernel_ms"].get("shrink", 0.0))
     if short:
         for s_ in short:
-            key = f"short_{s_['requests']}x{s_['suffix']}"
+            key = f"short_{s_['requests']}x{s_['suffix']}" + ("" if s_["prefix"] == 4096 else f"_at{s_['prefix']}")
             out[key + "_attention_hbm"] = r3(s_["attention_frac_of_hbm_peak"])
             out[key + "_ms_per_step"] = r3(s_["ms_per_step"])
             out[key + "_projection_ms"] = r3(s_["per_kernel_ms"].get("project_qkv", 0.0) + s_["per_kernel_ms"].get("shrink", 0.0))
@@ -389,6 +389,13 @@ def decode_leg(ab, hp, ctx, shape, stream, flush, peaks, steps=256, seed=5, ctx_
             "attention_hbm_gbs": gbs, "attention_frac_of_hbm_peak": gbs / peaks["hbm_gbs"] if gbs else None,
             "step_hbm_gbs": (kv_bytes + 2.0 * shape.N * shape.hidden) / (ms / 1e3) / 1e9,
             "peak_source": peaks["source"]}
+
+
+def parse_short_case(text):
+    """'8x4' -> (8 requests, 4 new tokens, 4096 cached); '64x16@16384' names the cached length too."""
+    shape, _, prefix = text.partition("@")
+    r, s = (int(v) for v in shape.split("x"))
+    return r, s, int(prefix) if prefix else 4096
 
 
 def short_suffix_leg(ab, hp, ctx, shape, stream, flush, peaks, requests, prefix, suffix, seed=7):
@@ -852,7 +859,8 @@ def main():
     ap.add_argument("--decode-steps", type=int, default=256)
     ap.add_argument("--decode-ctx-max", type=int, default=32768)
     ap.add_argument("--short-cases", default="8x4,8x16,64x4,64x16",
-                    help="the short-suffix leg's cases as requests x suffix tokens (on 4096 cached tokens each)")
+                    help="the short-suffix leg's cases as requests x suffix tokens, on 4096 cached tokens each unless "
+                         "'@cached' follows (64x4@16384)")
     ap.add_argument("--requests", type=int, default=8)
     ap.add_argument("--prefix", type=int, default=4096)
     ap.add_argument("--suffix", type=int, default=256)
@@ -1074,8 +1082,8 @@ def main():
         decode = decode_leg(ab, hp, ctx, shape, stream, flush, peaks, steps=args.decode_steps,
                             ctx_max=args.decode_ctx_max)
     if "short" in legs:
-        short = [short_suffix_leg(ab, hp, ctx, shape, stream, flush, peaks, r_, 4096, s_)
-                 for r_, s_ in [tuple(int(v) for v in c.split("x")) for c in args.short_cases.split(",") if c]]
+        short = [short_suffix_leg(ab, hp, ctx, shape, stream, flush, peaks, r_, p_, s_)
+                 for r_, s_, p_ in [parse_short_case(c) for c in args.short_cases.split(",") if c]]
     status = ab.alora_get_status(ctx)
     ab.alora_destroy(ctx)
     want_cpu = rank == 0 and world == 1 and not args.no_cpu_baseline
