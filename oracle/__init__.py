@@ -54,6 +54,20 @@ class Adapter:
     Bv: np.ndarray  # [Nkv, r]
 
 
+@dataclass
+class MlpAdapter:
+    """The same adapter's low-rank pairs on the MLP block's gate, up and down projections (the paper's remark that
+    MLP blocks are adapted by the equations corresponding to Eq. 5)."""
+    rank: int
+    scale: float
+    Ag: np.ndarray  # [r, H]
+    Bg: np.ndarray  # [I, r]
+    Au: np.ndarray  # [r, H]
+    Bu: np.ndarray  # [I, r]
+    Ad: np.ndarray  # [r, I]
+    Bd: np.ndarray  # [H, r]
+
+
 def _f32(a):
     return np.ascontiguousarray(a, dtype=np.float32)
 
@@ -129,6 +143,36 @@ class Oracle:
             int(bool(force_all)), _p(qkv, C.c_double), _p(gate, C.c_uint8))
         assert rc == 0, "oracle_project_qkv: bad arguments"
         return qkv, gate
+
+    # ---- the equation corresponding to Eq. 5 for one MLP weight matrix ------------------------------
+    def gated_linear(self, x, W, positions, query_start_loc, activation_offsets, adapter_ids, ranks, scales,
+                     As, Bs, force_all: bool = False) -> np.ndarray:
+        """y_t = W x_t, plus scale * B (A x_t) on the rows of adapter requests at or after the activation offset.
+        As[k] is [rank_k, K], Bs[k] is [N, rank_k], indexed by adapter id."""
+        x, W = _f64(x), _f32(W)
+        T, K = x.shape
+        N = W.shape[0]
+        assert W.shape[1] == K
+        positions, qsl = _i32(positions), _i32(query_start_loc)
+        R = len(qsl) - 1
+        a_req, ids = _i32(activation_offsets), _i32(adapter_ids)
+        n = len(As)
+        assert len(Bs) == n and len(ranks) == n and len(scales) == n
+        rk, sc = _i32(list(ranks) or [0]), _f32(list(scales) or [0])
+        keep_a = [_f32(a) for a in As]
+        keep_b = [_f32(b) for b in Bs]
+        pa = (C.POINTER(C.c_float) * max(n, 1))()
+        pb = (C.POINTER(C.c_float) * max(n, 1))()
+        for i in range(n):
+            assert keep_a[i].shape == (rk[i], K) and keep_b[i].shape == (N, rk[i])
+            pa[i], pb[i] = _p(keep_a[i], C.c_float), _p(keep_b[i], C.c_float)
+        y = np.empty((T, N), np.float64)
+        rc = self.lib.oracle_gated_linear(_p(x, C.c_double), _p(W, C.c_float), T, K, N, _p(positions, C.c_int32),
+                                          _p(qsl, C.c_int32), R, _p(a_req, C.c_int32), _p(ids, C.c_int32), n,
+                                          _p(rk, C.c_int32), _p(sc, C.c_float), pa, pb, int(bool(force_all)),
+                                          _p(y, C.c_double))
+        assert rc == 0, "oracle_gated_linear: bad arguments"
+        return y
 
     # ---- Eq. 1 / Eq. 3 ----------------------------------------------------------------------------
     def attention(self, q, K, V, kv_start_loc, positions, query_start_loc, Hq: int, Hkv: int,
@@ -265,13 +309,27 @@ class Oracle:
 
     def decoder_layer(self, h, lw: dict, Nq, Nkv, Hq, Hkv, hd, eps, positions, query_start_loc,
                       activation_offsets, adapter_ids, adapters, prefix_K, prefix_V, force_all=False,
-                      rope_theta=0.0):
-        """Pre-norm residual decoder layer: h + o_proj(attn(norm(h))), then + down(swiglu(gate_up(norm)))."""
+                      rope_theta=0.0, mlp_adapters: Optional[Sequence[MlpAdapter]] = None):
+        """Pre-norm residual decoder layer: h + o_proj(attn(norm(h))), then + down(swiglu(gate_up(norm))).
+        With `mlp_adapters` (indexed by adapter id like `adapters`) the gate, up and down projections are adapted
+        under the same per-token gate as q/k/v."""
         xn = self.rmsnorm(h, lw["norm_attn"], eps)
         blk = self.attention_block(xn, lw["wqkv"], Nq, Nkv, Hq, Hkv, hd, positions, query_start_loc,
                                    activation_offsets, adapter_ids, adapters, prefix_K, prefix_V,
                                    force_all, rope_theta=rope_theta)
         h1 = _f64(h) + self.linear(blk["out"], lw["wo"])
         xm = self.rmsnorm(h1, lw["norm_mlp"], eps)
-        h2 = h1 + self.linear(self.swiglu(self.linear(xm, lw["wgate_up"])), lw["wdown"])
+        if not mlp_adapters:
+            h2 = h1 + self.linear(self.swiglu(self.linear(xm, lw["wgate_up"])), lw["wdown"])
+            return h2, blk
+        inter = lw["wgate_up"].shape[0] // 2
+        ranks = [m.rank for m in mlp_adapters]
+        scales = [m.scale for m in mlp_adapters]
+        gated = lambda x, W, a, b: self.gated_linear(  # noqa: E731
+            x, W, positions, query_start_loc, activation_offsets, adapter_ids, ranks, scales,
+            [getattr(m, a) for m in mlp_adapters], [getattr(m, b) for m in mlp_adapters], force_all)
+        gate = gated(xm, lw["wgate_up"][:inter], "Ag", "Bg")
+        up = gated(xm, lw["wgate_up"][inter:], "Au", "Bu")
+        act = self.swiglu(np.concatenate([gate, up], axis=1))
+        h2 = h1 + gated(act, lw["wdown"], "Ad", "Bd")
         return h2, blk

@@ -25,7 +25,10 @@
  * scores, two-key logistic weight, constant V), decode == prefill row, page-permutation
  * invariance, brute-force slot indices, the cache layout read back by plain array indexing, and
  * Prop. 2's closed-form pair and row counts; the optional rotary embedding by a complex-multiplication
- * restatement, a hand example, norm preservation and the relative-position property.
+ * restatement, a hand example, norm preservation and the relative-position property; the gated
+ * MLP adaptation by B = 0 => base, a_req = 0 => merged weights against a library matmul, bit-equal
+ * pre-activation rows, a library restatement of the adapted layer, and the cache-reuse identity
+ * through two adapted layers (which fails when the MLP gate is left open).
  * tests/test_oracle_mutants.py plants one-line
  * mistakes in a copy of this file and checks that the pins notice.
  * No function in this file is "parity unpinned".
@@ -142,6 +145,61 @@ int oracle_project_qkv(const double *x, const float *W, int T, int H, int Nq, in
                 for (int i = 0; i < rk; ++i) d += (real)Bs[b][(size_t)n * rk + i] * u[i];
                 yt[first[b] + n] = (double)((real)yt[first[b] + n] + s * d);
             }
+        }
+        free(u);
+    }
+    return bad ? ORACLE_ERR_ARG : ORACLE_OK;
+}
+
+/*
+ * Gated low-rank adaptation of ONE weight matrix of an MLP block (gate, up or down projection).
+ * The paper states that MLP blocks can be adapted by the equations that correspond to Eq. 5 for
+ * Q, K and V (Sec. 2, remark on MLP blocks; Sec. 3, the sentence after Eq. 5): a token before the
+ * activation offset is multiplied by the base weight alone, a token at or after it by W + s B A.
+ *
+ *   y_t = W x_t                        if the request has no adapter, or p_t < a_req
+ *   y_t = W x_t + s * B (A x_t)        if adapter k and p_t >= a_req
+ *
+ * x[T][K], W[N][K]; per adapter id: rank, scale, A[r][K], B[N][r].  As in the q/k/v projection a
+ * gated-off row executes no adapter arithmetic.  force_all != 0 opens every adapter row's gate (Eq. 4).
+ */
+int oracle_gated_linear(const double *x, const float *W, int T, int K, int N,
+                        const int32_t *positions, const int32_t *query_start_loc, int R,
+                        const int32_t *activation_offsets, const int32_t *adapter_ids,
+                        int n_adapters, const int32_t *ranks, const float *scales,
+                        const float *const *A, const float *const *B, int force_all, double *y) {
+    if (!x || !W || !y || !positions || !query_start_loc || T < 0 || R < 0 || K <= 0 || N <= 0) return ORACLE_ERR_ARG;
+    int bad = 0;
+#pragma omp parallel for schedule(static)
+    for (int t = 0; t < T; ++t) {
+        const int r = request_of_token(query_start_loc, R, t);
+        if (r < 0) { bad = 1; continue; }
+        const double *xt = x + (size_t)t * K;
+        double *yt = y + (size_t)t * N;
+        const int k = adapter_ids ? adapter_ids[r] : -1;
+        int gate = 0;
+        if (k >= 0) {
+            if (k >= n_adapters) { bad = 1; continue; }
+            gate = force_all || positions[t] >= activation_offsets[r];   /* the MLP gate */
+        }
+        for (int n = 0; n < N; ++n) {
+            real acc = 0;
+            for (int h = 0; h < K; ++h) acc += (real)W[(size_t)n * K + h] * (real)xt[h];
+            yt[n] = (double)acc;
+        }
+        if (!gate) continue;
+        const int rk = ranks[k];
+        const real s = (real)scales[k];
+        real *u = (real *)malloc(sizeof(real) * (size_t)(rk > 0 ? rk : 1));
+        for (int i = 0; i < rk; ++i) {
+            real acc = 0;
+            for (int h = 0; h < K; ++h) acc += (real)A[k][(size_t)i * K + h] * (real)xt[h];
+            u[i] = acc;
+        }
+        for (int n = 0; n < N; ++n) {
+            real d = 0;
+            for (int i = 0; i < rk; ++i) d += (real)B[k][(size_t)n * rk + i] * u[i];   /* MLP expand */
+            yt[n] = (double)((real)yt[n] + s * d);   /* MLP delta add */
         }
         free(u);
     }

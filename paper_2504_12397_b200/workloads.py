@@ -82,6 +82,19 @@ class AdapterWeights:
 
 
 @dataclass
+class MlpAdapterWeights:
+    """The low-rank pairs of one adapter on the MLP block: gate, up ([r, H] / [I, r]) and down ([r, I] / [H, r])."""
+    rank: int
+    scale: float
+    Ag: np.ndarray
+    Bg: np.ndarray
+    Au: np.ndarray
+    Bu: np.ndarray
+    Ad: np.ndarray
+    Bd: np.ndarray
+
+
+@dataclass
 class Batch:
     """A ragged batch of new tokens on top of per-request cached prefixes."""
     positions: np.ndarray            # [T] int32, position of each new token in its sequence
@@ -123,6 +136,21 @@ def make_adapter(shape: LayerShape, rank: int, rng: np.random.Generator, scale: 
         return _round(np.zeros_like(m) if zero_b else m, shape.dtype)
 
     return AdapterWeights(rank, scale, A(), B(shape.Nq), A(), B(shape.Nkv), A(), B(shape.Nkv))
+
+
+def make_mlp_adapter(shape: LayerShape, rank: int, rng: np.random.Generator, scale: float = 1.0,
+                     zero_b: bool = False) -> MlpAdapterWeights:
+    """Random-weight MLP adapter with the distribution of the q/k/v ones (N(0, 0.02^2), rounded to the layer dtype)."""
+    H, I = shape.hidden, shape.intermediate
+
+    def A(k):
+        return _round(rng.normal(0.0, 0.02, (rank, k)), shape.dtype)
+
+    def B(n):
+        m = rng.normal(0.0, 0.02, (n, rank))
+        return _round(np.zeros_like(m) if zero_b else m, shape.dtype)
+
+    return MlpAdapterWeights(rank, scale, A(H), B(I), A(H), B(I), A(I), B(H))
 
 
 def make_stack_weights(shape: LayerShape, rng: np.random.Generator) -> dict:

@@ -119,6 +119,11 @@ def oracle_adapters(ads):
     return [Adapter(a.rank, a.scale, a.Aq, a.Bq, a.Ak, a.Bk, a.Av, a.Bv) for a in ads]
 
 
+def oracle_mlp_adapters(ads):
+    from oracle import MlpAdapter
+    return [MlpAdapter(a.rank, a.scale, a.Ag, a.Bg, a.Au, a.Bu, a.Ad, a.Bd) for a in ads]
+
+
 def oracle_base_prefix(orc, shape, wqkv, b: wl.Batch, rope_theta: float = 0.0):
     """Base-model K/V of every request's prefix, from the prefix hidden states (Eq. 2); with a rotary base, keys as
     they would be cached (rotated by their positions)."""

@@ -86,6 +86,16 @@ C_MUTANTS = [
     ("const real u = (real)gate_up[(size_t)t * 2 * I + I + i];",
      "const real u = (real)gate_up[(size_t)t * 2 * I + i]; (void)I;",
      ["test_rmsnorm_swiglu_linear_against_library", "test_decoder_layer_against_library_restatement"]),
+    # the gated MLP matrix: gate one position late, scale dropped, B read transposed
+    ("gate = force_all || positions[t] >= activation_offsets[r];   /* the MLP gate */",
+     "gate = force_all || positions[t] > activation_offsets[r];",
+     ["test_mlp_gated_linear_special_cases", "test_decoder_layer_with_mlp_adapters_against_library_restatement"]),
+    ("yt[n] = (double)((real)yt[n] + s * d);   /* MLP delta add */",
+     "yt[n] = (double)((real)yt[n] + d); (void)s;",
+     ["test_mlp_gated_linear_special_cases", "test_decoder_layer_with_mlp_adapters_against_library_restatement"]),
+    ("d += (real)B[k][(size_t)n * rk + i] * u[i];   /* MLP expand */",
+     "d += (real)B[k][(size_t)i * N + n] * u[i];",
+     ["test_mlp_gated_linear_special_cases"]),
 ]
 
 
@@ -122,12 +132,27 @@ PY_MUTANTS = [
     ('xm = self.rmsnorm(h1, lw["norm_mlp"], eps)', 'xm = h1'),
     # attention residual dropped
     ('h1 = _f64(h) + self.linear(blk["out"], lw["wo"])', 'h1 = self.linear(blk["out"], lw["wo"])'),
+    # adapted MLP: the up projection given the gate projection's pair, the down pair applied to the normed input's
+    # width-compatible sibling (the gate pair's B is [I, r], so the down projection's pair must be its own), the MLP
+    # gate left open, the adapted down projection fed the un-activated gate output
+    ('up = gated(xm, lw["wgate_up"][inter:], "Au", "Bu")', 'up = gated(xm, lw["wgate_up"][inter:], "Ag", "Bg")',
+     "test_decoder_layer_with_mlp_adapters_against_library_restatement"),
+    ('gate = gated(xm, lw["wgate_up"][:inter], "Ag", "Bg")', 'gate = gated(xm, lw["wgate_up"][:inter], "Au", "Bu")',
+     "test_decoder_layer_with_mlp_adapters_against_library_restatement"),
+    ("[getattr(m, a) for m in mlp_adapters], [getattr(m, b) for m in mlp_adapters], force_all)",
+     "[getattr(m, a) for m in mlp_adapters], [getattr(m, b) for m in mlp_adapters], True)",
+     "test_cache_reuse_identity_through_two_layers_with_mlp_adapters"),
+    ('h2 = h1 + gated(act, lw["wdown"], "Ad", "Bd")', 'h2 = h1 + self.linear(act, lw["wdown"])',
+     "test_decoder_layer_with_mlp_adapters_against_library_restatement"),
+    ('act = self.swiglu(np.concatenate([gate, up], axis=1))', 'act = self.swiglu(np.concatenate([up, gate], axis=1))',
+     "test_decoder_layer_with_mlp_adapters_against_library_restatement"),
 ]
 
 
 @pytest.mark.parametrize("idx", range(len(PY_MUTANTS)))
 def test_planted_mistake_in_the_layer_composition_fails_its_pin(oracle64, idx):
-    old, new = PY_MUTANTS[idx]
+    old, new, *pin = PY_MUTANTS[idx]
+    pin_fn = getattr(pins, pin[0] if pin else "test_decoder_layer_against_library_restatement")
     src = textwrap.dedent(inspect.getsource(Oracle.decoder_layer))
     assert src.count(old) == 1, old
     ns = dict(vars(oracle_pkg))
@@ -140,6 +165,6 @@ def test_planted_mistake_in_the_layer_composition_fails_its_pin(oracle64, idx):
             self.precision, self.lib = base.precision, base.lib
 
     with pytest.raises(AssertionError):
-        pins.test_decoder_layer_against_library_restatement(Mutant(oracle64))
+        pin_fn(Mutant(oracle64))
     # and the unpatched composition passes the same call
-    pins.test_decoder_layer_against_library_restatement(oracle64)
+    pin_fn(oracle64)

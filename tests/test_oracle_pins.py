@@ -13,7 +13,7 @@ import numpy as np
 import pytest
 import torch
 
-from oracle import Adapter
+from oracle import Adapter, MlpAdapter
 from paper_2504_12397_b200 import workloads as wl
 
 SMALL = wl.LayerShape(hidden=32, n_q_heads=4, n_kv_heads=2, head_dim=8, page_size=4, dtype="fp32")
@@ -491,6 +491,176 @@ def test_decoder_layer_against_library_restatement(oracle64):
     assert blk["gate"].tolist() == [0, 0, 0, 1, 1, 1, 1] + [0] * 5
     # each part of the composition carries weight here: leaving it out is far outside the tolerance
     assert np.abs(got - h).max() > 0.1
+
+
+# ---- gated adapters on the MLP block (the equations corresponding to Eq. 5) ---------------------------
+
+def _mlp_ad(a: wl.MlpAdapterWeights) -> MlpAdapter:
+    return MlpAdapter(a.rank, a.scale, a.Ag, a.Bg, a.Au, a.Bu, a.Ad, a.Bd)
+
+
+def _mlp_linear_case(seed=21):
+    rng = np.random.default_rng(seed)
+    K, N = 24, 40
+    W = (rng.standard_normal((N, K)) * 0.3).astype(np.float32)
+    ranks, scales = [3, 5], [1.0, 0.5]
+    As = [(rng.standard_normal((r, K)) * 0.4).astype(np.float32) for r in ranks]
+    Bs = [(rng.standard_normal((N, r)) * 0.4).astype(np.float32) for r in ranks]
+    prefix, new, ids = (4, 9, 2), (6, 5, 3), (1, -1, 0)
+    qsl = np.concatenate([[0], np.cumsum(new)]).astype(np.int32)
+    pos = np.concatenate([np.arange(p, p + n) for p, n in zip(prefix, new)]).astype(np.int32)
+    x = rng.standard_normal((sum(new), K))
+    return x, W, pos, qsl, ids, ranks, scales, As, Bs, prefix, new
+
+
+def test_mlp_gated_linear_special_cases(oracle64):
+    """One adapted MLP matrix: rows before the activation offset are bit-equal to the plain product, B = 0 gives the
+    plain product everywhere, an offset of 0 gives the merged matrix W + s B A (library matmul), and a mid-chunk
+    offset gives the row-wise mix of the two; adapters 0 and 1 have different ranks and scales."""
+    x, W, pos, qsl, ids, ranks, scales, As, Bs, prefix, new = _mlp_linear_case()
+    base = oracle64.linear(x, W)
+    a_req = [prefix[0] + 2, 0, prefix[2] + 1]            # opens inside request 0 and request 2
+    y = oracle64.gated_linear(x, W, pos, qsl, a_req, ids, ranks, scales, As, Bs)
+    W64 = W.astype(np.float64)
+    for r in range(3):
+        lo, hi = qsl[r], qsl[r + 1]
+        if ids[r] < 0:
+            np.testing.assert_array_equal(y[lo:hi], base[lo:hi])
+            continue
+        k = ids[r]
+        merged = W64 + scales[k] * Bs[k].astype(np.float64) @ As[k].astype(np.float64)
+        open_ = pos[lo:hi] >= a_req[r]
+        assert open_.any() and not open_.all()
+        np.testing.assert_array_equal(y[lo:hi][~open_], base[lo:hi][~open_])
+        np.testing.assert_allclose(y[lo:hi][open_], x[lo:hi][open_] @ merged.T, rtol=1e-11, atol=1e-12)
+        assert np.abs(y[lo:hi][open_] - base[lo:hi][open_]).max() > 1e-2
+    zero = oracle64.gated_linear(x, W, pos, qsl, [0, 0, 0], ids, ranks, scales, As, [b * 0 for b in Bs])
+    np.testing.assert_array_equal(zero, base)
+    late = oracle64.gated_linear(x, W, pos, qsl, [10 ** 6] * 3, ids, ranks, scales, As, Bs)
+    np.testing.assert_array_equal(late, base)
+    forced = oracle64.gated_linear(x, W, pos, qsl, [10 ** 6] * 3, ids, ranks, scales, As, Bs, force_all=True)
+    lo, hi = qsl[0], qsl[1]
+    np.testing.assert_allclose(forced[lo:hi], x[lo:hi] @ (W64 + scales[1] * Bs[1].astype(np.float64) @ As[1].astype(np.float64)).T,
+                               rtol=1e-11, atol=1e-12)
+
+
+def _torch_adapted_mlp(h1, lw, mlp, shape, eps, pos, a_req, adapter):
+    """norm, adapted gate / up, SwiGLU, adapted down and the residual of ONE request in torch fp64 ops."""
+    F = torch.nn.functional
+    t64 = lambda a: torch.from_numpy(np.asarray(a, np.float64))
+    H, I = shape.hidden, shape.intermediate
+    h1 = t64(h1)
+    xm = F.rms_norm(h1, (H,), t64(lw["norm_mlp"]), eps)
+    open_ = (torch.as_tensor(np.asarray(pos, np.int64)) >= int(a_req))[:, None] if adapter is not None else None
+    wg, wu = t64(lw["wgate_up"][:I]), t64(lw["wgate_up"][I:])
+
+    def lin(x, W, A, B):
+        y = x @ W.T
+        if adapter is None:
+            return y
+        return torch.where(open_, y + adapter.scale * ((x @ t64(A).T) @ t64(B).T), y)
+
+    m = adapter
+    gate = lin(xm, wg, m.Ag if m else None, m.Bg if m else None)
+    up = lin(xm, wu, m.Au if m else None, m.Bu if m else None)
+    act = F.silu(gate) * up
+    return (h1 + lin(act, t64(lw["wdown"]), m.Ad if m else None, m.Bd if m else None)).numpy()
+
+
+def test_decoder_layer_with_mlp_adapters_against_library_restatement(oracle64):
+    """The layer with adapters on q/k/v AND on gate, up and down: the attention half is taken from the oracle's own
+    layer without MLP adapters (pinned above), the MLP half is restated in torch ops.  The gate opens in the middle
+    of request 0's new tokens; request 1 runs the base model.  Every adapted matrix carries weight: zeroing any one
+    of Bg, Bu, Bd moves the result by far more than the tolerance."""
+    shape, eps = STACK_SHAPE, 1e-5
+    rng = np.random.default_rng(12)
+    lw = wl.make_stack_weights(shape, rng)
+    for k in ("wqkv", "wo", "wgate_up", "wdown"):
+        lw[k] = lw[k] * 10
+    ad = [wl.make_adapter(shape, 4, rng)]
+    mlp = [wl.make_mlp_adapter(shape, 4, rng, scale=0.5)]
+    for n in ("Ag", "Bg", "Au", "Bu", "Ad", "Bd"):
+        setattr(mlp[0], n, getattr(mlp[0], n) * 20)
+    prefix, new, ids, a_req = (6, 9), (7, 5), (0, -1), (9, 0)
+    T = sum(new)
+    h = rng.standard_normal((T, shape.hidden))
+    qsl = np.asarray([0, new[0], T], np.int32)
+    pos = np.concatenate([np.arange(p, p + n) for p, n in zip(prefix, new)]).astype(np.int32)
+    pK = [rng.standard_normal((p, shape.Nkv)) for p in prefix]
+    pV = [rng.standard_normal((p, shape.Nkv)) for p in prefix]
+    args = (h, lw, shape.Nq, shape.Nkv, shape.n_q_heads, shape.n_kv_heads, shape.head_dim, eps, pos, qsl, a_req, ids,
+            [_ad(ad[0])], pK, pV)
+    got, blk = oracle64.decoder_layer(*args, mlp_adapters=[_mlp_ad(mlp[0])])
+    # h1 = the state after the attention half, from the composition pinned by the test above
+    h1 = h + oracle64.linear(blk["out"], lw["wo"])
+    want = np.concatenate([_torch_adapted_mlp(h1[:7], lw, mlp, shape, eps, pos[:7], a_req[0], mlp[0]),
+                           _torch_adapted_mlp(h1[7:], lw, mlp, shape, eps, pos[7:], a_req[1], None)])
+    np.testing.assert_allclose(got, want, rtol=1e-10, atol=1e-11)
+    plain, _ = oracle64.decoder_layer(*args)
+    np.testing.assert_array_equal(got[:3], plain[:3])       # rows before the offset: the layer without MLP adapters
+    np.testing.assert_array_equal(got[7:], plain[7:])       # the base-model request
+    assert np.abs(got[3:7] - plain[3:7]).max() > 0.1
+    for name in ("Bg", "Bu", "Bd"):
+        z = _mlp_ad(mlp[0])
+        setattr(z, name, getattr(z, name) * 0)
+        other, _ = oracle64.decoder_layer(*args, mlp_adapters=[z])
+        assert np.abs(other[3:7] - got[3:7]).max() > 1e-2, name
+
+
+def test_cache_reuse_identity_through_two_layers_with_mlp_adapters(oracle64):
+    """Prop. 1 with adapted MLP blocks: because the MLP adapters are gated like q/k/v, a whole sequence run from
+    scratch leaves, in BOTH layers, prefix K/V bit-equal to the base model's, and the suffix computed on the base
+    model's caches equals the suffix rows of the from-scratch run.  With the MLP gate left open on the prefix
+    (ordinary LoRA on the MLP) the second layer's prefix K/V differ: the identity needs the gate."""
+    shape, eps = STACK_SHAPE, 1e-5
+    rng = np.random.default_rng(13)
+    layers = [wl.make_stack_weights(shape, rng) for _ in range(2)]
+    for lw in layers:
+        for k in ("wqkv", "wo", "wgate_up", "wdown"):
+            lw[k] = lw[k] * 10
+    ads = [[wl.make_adapter(shape, 4, rng)] for _ in range(2)]
+    mlps = [[wl.make_mlp_adapter(shape, 4, rng)] for _ in range(2)]
+    for per in mlps:
+        for n in ("Ag", "Bg", "Au", "Bu", "Ad", "Bd"):
+            setattr(per[0], n, getattr(per[0], n) * 20)
+    P, S = 9, 5
+    L = P + S
+    h = rng.standard_normal((L, shape.hidden))
+    kw = dict(Nq=shape.Nq, Nkv=shape.Nkv, Hq=shape.n_q_heads, Hkv=shape.n_kv_heads, hd=shape.head_dim, eps=eps)
+
+    def run(x, pos, a_req, ids, caches, mlp_gate_open=False):
+        out = []
+        for l in range(2):
+            m = [_mlp_ad(mlps[l][0])]
+            if mlp_gate_open:   # ordinary LoRA on the MLP only: a separate call with offset 0 for the MLP half
+                x1, blk = oracle64.decoder_layer(x, layers[l], positions=pos, query_start_loc=[0, len(pos)],
+                                                 activation_offsets=[a_req], adapter_ids=ids,
+                                                 adapters=[_ad(ads[l][0])], prefix_K=[caches[l][0]],
+                                                 prefix_V=[caches[l][1]], **kw)
+                h1 = x + oracle64.linear(blk["out"], layers[l]["wo"])
+                x = _torch_adapted_mlp(h1, layers[l], None, shape, eps, pos, 0, mlps[l][0])
+            else:
+                x, blk = oracle64.decoder_layer(x, layers[l], positions=pos, query_start_loc=[0, len(pos)],
+                                                activation_offsets=[a_req], adapter_ids=ids,
+                                                adapters=[_ad(ads[l][0])], prefix_K=[caches[l][0]],
+                                                prefix_V=[caches[l][1]], mlp_adapters=m, **kw)
+            out.append((x, blk["K"][0], blk["V"][0]))
+        return out
+
+    none = [(None, None)] * 2
+    base = run(h[:P], np.arange(P), 0, [-1], none)                       # base model prefills the prefix
+    scratch = run(h, np.arange(L), P, [0], none)                         # aLoRA on the whole sequence
+    reuse = run(h[P:], np.arange(P, L), P, [0], [(K, V) for _, K, V in base])
+    # hidden states entering layer 2 on the reuse path are the suffix rows of layer 1's output
+    for l in range(2):
+        np.testing.assert_array_equal(scratch[l][1][:P], base[l][1])
+        np.testing.assert_array_equal(scratch[l][2][:P], base[l][2])
+        np.testing.assert_allclose(reuse[l][0], scratch[l][0][P:], rtol=1e-11, atol=1e-12)
+        np.testing.assert_allclose(reuse[l][1][P:], scratch[l][1][P:], rtol=1e-11, atol=1e-12)
+    assert np.abs(scratch[1][0][P:] - run(h, np.arange(L), P, [-1], none)[1][0][P:]).max() > 1e-2
+    lora_mlp = run(h, np.arange(L), P, [0], none, mlp_gate_open=True)
+    np.testing.assert_array_equal(lora_mlp[0][1][:P], base[0][1])        # layer 1's keys see no MLP yet
+    assert np.abs(lora_mlp[1][1][:P] - base[1][1]).max() > 1e-3          # layer 2's prefix keys are no longer the base's
 
 
 def test_pool_layout_by_plain_indexing(oracle64):
