@@ -137,6 +137,25 @@ alora_status alora_register_adapter(alora_ctx *ctx, int adapter_id, int layer, i
                                     void *stream);
 
 /*
+ * Extend adapter `adapter_id` of `layer` to the MLP block: gate, up and down projections each get
+ * Delta = scale * B A under the SAME per-token gate as q/k/v (the paper adapts q, k and v and remarks,
+ * in its background section and after Eq. 5, that MLP blocks are adapted by the corresponding
+ * equations).  d_Agate and d_Aup are [rank][H], d_Bgate and d_Bup are [I][rank], d_Adown is [rank][I],
+ * d_Bdown is [H][rank]; I = intermediate size.  Only alora_forward_stack and alora_decode_stack run
+ * the MLP block, so only they use these matrices: rows whose gate is open get the deltas, rows whose
+ * gate is closed (and every row in ALORA_MODE_BASE) keep the bits of the base MLP.  The matrices are
+ * COPIED on the given stream.  The first registration on a layer allocates that layer's slabs
+ * (cudaMalloc; about 2 * max_adapters * 64 * (H + 3 I) bytes), so register before timing anything.
+ * Errors: ALORA_ERR_NO_WEIGHTS when the adapter has no q/k/v part on this layer yet (its gate is the
+ * q/k/v adapter's); ALORA_ERR_UNSUPPORTED for fp32 contexts, contexts without an MLP (intermediate = 0)
+ * and sizes where H or I is not a multiple of 32; ALORA_ERR_CAPACITY for the id or rank.
+ */
+alora_status alora_register_mlp_adapter(alora_ctx *ctx, int adapter_id, int layer, int rank, float scale,
+                                        const void *d_Agate, const void *d_Bgate, const void *d_Aup,
+                                        const void *d_Bup, const void *d_Adown, const void *d_Bdown,
+                                        void *stream);
+
+/*
  * Host-side consistency check of batch metadata (all pointers HOST memory; launches nothing, needs
  * no device).  Verifies: query_start_loc non-decreasing from 0 to T; positions of each request
  * consecutive and ending at seq_lens[r]-1; adapter ids in [-1, max_adapters); activation offsets

@@ -44,6 +44,8 @@ def _signatures(lib):
     lib.alora_destroy.argtypes = [_VP]
     lib.alora_set_layer_weights.argtypes = [_VP, _I] + [_VP] * 6
     lib.alora_register_adapter.argtypes = [_VP, _I, _I, _I, C.c_float] + [_VP] * 6 + [_VP]
+    lib.alora_register_mlp_adapter.argtypes = [_VP, _I, _I, _I, C.c_float] + [_VP] * 6 + [_VP]
+    lib.alora_register_mlp_adapter.restype = C.c_int
     lib.alora_validate_batch.argtypes = [C.POINTER(alora_config)] + [_IP] * 6 + [_I] * 4
     lib.alora_batch_metadata.argtypes = [_VP, _I] + [_IP] * 6 + [_I] * 4 + [_IP] * 3 + [_VP]
     lib.alora_project_qkv.argtypes = [_VP, _I, _I, _VP] + [_IP] * 5 + [_I, _I, _VP, _VP]
@@ -143,6 +145,12 @@ def alora_register_adapter(ctx, adapter_id, layer, rank, scale, Aq, Bq, Ak, Bk, 
     rc = load_library().alora_register_adapter(ctx, adapter_id, layer, rank, scale, _ptr(Aq), _ptr(Bq), _ptr(Ak),
                                                _ptr(Bk), _ptr(Av), _ptr(Bv), _stream(stream))
     _check(ctx, rc, "alora_register_adapter")
+
+
+def alora_register_mlp_adapter(ctx, adapter_id, layer, rank, scale, Ag, Bg, Au, Bu, Ad, Bd, stream=None):
+    rc = load_library().alora_register_mlp_adapter(ctx, adapter_id, layer, rank, scale, _ptr(Ag), _ptr(Bg), _ptr(Au),
+                                                   _ptr(Bu), _ptr(Ad), _ptr(Bd), _stream(stream))
+    _check(ctx, rc, "alora_register_mlp_adapter")
 
 
 def alora_validate_batch(cfg: alora_config, positions, activation_offsets, adapter_ids, query_start_loc,

@@ -20,6 +20,10 @@ int launch_attend_simt(alora_ctx *, const void *, const BatchArgs &, const void 
 
 int launch_project_tc(alora_ctx *, int, const void *, int, void *, cudaStream_t, void *, int);
 int launch_linear_tc(alora_ctx *, const void *, const void *, int, int, int, void *, const void *, cudaStream_t);
+int launch_repack_mlp(const void *, const void *, const void *, const void *, int, int, int, int, int, void *, void *,
+                      cudaStream_t);   // mlp_adapter.cu
+int launch_mlp_expand(alora_ctx *, void *, int, int, const void *, int, const void *, int, int, int, const int32_t *,
+                      const MlpAdapterDev *, int, cudaStream_t);
 bool build_layer_maps(alora_ctx *ctx, int layer);
 bool project_is_few_row(const alora_ctx *ctx, int layer, int T);   // gemm_tcgen05.cu
 int launch_attend_tc(alora_ctx *, const void *, const BatchArgs &, const void *, void *, cudaStream_t);
@@ -288,6 +292,10 @@ alora_status alora_destroy(alora_ctx *ctx) {
     for (void *p : ctx->adapter_storage) if (p) cudaFree(p);
     for (void *p : ctx->tc_a_all) if (p) cudaFree(p);
     for (void *p : ctx->tc_b_all) if (p) cudaFree(p);
+    for (auto *v : {&ctx->mlp_a_gu, &ctx->mlp_b_gu, &ctx->mlp_a_dn, &ctx->mlp_b_dn})
+        for (void *p : *v) if (p) cudaFree(p);
+    if (ctx->d_mlp_adapters) cudaFree(ctx->d_mlp_adapters);
+    if (ctx->d_mlp_t) cudaFree(ctx->d_mlp_t);
     void *ptrs[] = {ctx->d_adapters, ctx->d_token_req, ctx->d_row_adapter, ctx->d_slot, ctx->d_tiles, ctx->d_counts,
                     ctx->d_seg_scratch, ctx->d_shrink_tiles, ctx->d_t_ready, ctx->d_t, ctx->d_qkv, ctx->d_status, ctx->d_act[0], ctx->d_act[1],
                     ctx->d_act[2], ctx->d_act[3], ctx->d_iota, ctx->d_attn_items, ctx->d_attn_off, ctx->d_split_items,
@@ -348,6 +356,70 @@ alora_status alora_register_adapter(alora_ctx *ctx, int adapter_id, int layer, i
     // the table entry is a kernel argument of later launches on this stream: order the update after
     // earlier work by copying on the same stream (source is context-owned host memory).
     ALORA_CUDA(ctx, cudaMemcpyAsync(ctx->d_adapters + idx, &ctx->h_adapters[idx], sizeof(AdapterDev),
+                                    cudaMemcpyHostToDevice, s));
+    return finish(ctx, n);
+}
+
+// Rows of the down projection's A slab: every adapter's RP rows, rounded up to whole 128-row GEMM tiles.
+static size_t mlp_dn_rows(const alora_ctx *ctx) {
+    return ((size_t)std::max(1, ctx->cfg.max_adapters) * ctx->d.RP + 127) / 128 * 128;
+}
+
+alora_status alora_register_mlp_adapter(alora_ctx *ctx, int adapter_id, int layer, int rank, float scale,
+                                        const void *d_Agate, const void *d_Bgate, const void *d_Aup, const void *d_Bup,
+                                        const void *d_Adown, const void *d_Bdown, void *stream) {
+    if (!ctx || !d_Agate || !d_Bgate || !d_Aup || !d_Bup || !d_Adown || !d_Bdown) return ALORA_ERR_INVALID_ARG;
+    if (layer < 0 || layer >= ctx->cfg.n_layers) return ALORA_ERR_INVALID_ARG;
+    if (adapter_id < 0 || adapter_id >= ctx->cfg.max_adapters) return ALORA_ERR_CAPACITY;
+    if (rank < 1 || rank > ctx->cfg.max_rank) return ALORA_ERR_CAPACITY;
+    const Dims &d = ctx->d;
+    if (ctx->cfg.dtype != ALORA_DTYPE_BF16 || d.I <= 0 || d.I % 32 != 0 || d.H % 32 != 0) return ALORA_ERR_UNSUPPORTED;
+    // the per-row gate of a batch is the q/k/v adapter's: the MLP part extends an adapter registered on this layer
+    if (ctx->h_adapters[(size_t)layer * ctx->cfg.max_adapters + adapter_id].rank == 0) return ALORA_ERR_NO_WEIGHTS;
+    cudaStream_t s = (cudaStream_t)stream;
+    ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
+    const size_t na = (size_t)std::max(1, ctx->cfg.max_adapters), es = ctx->esize;
+    const size_t a_gu = (size_t)2 * d.RP * d.H * es, b_gu = (size_t)2 * d.I * d.RP * es;
+    const size_t a_dn = (size_t)d.RP * d.I * es, b_dn = (size_t)d.H * d.RP * es;
+    if (ctx->mlp_a_gu.empty()) {
+        ctx->mlp_a_gu.assign(ctx->cfg.n_layers, nullptr); ctx->mlp_b_gu.assign(ctx->cfg.n_layers, nullptr);
+        ctx->mlp_a_dn.assign(ctx->cfg.n_layers, nullptr); ctx->mlp_b_dn.assign(ctx->cfg.n_layers, nullptr);
+        ctx->mlp_n_adapters.assign(ctx->cfg.n_layers, 0);
+        ctx->h_mlp_adapters.assign((size_t)ctx->cfg.n_layers * na, MlpAdapterDev{0, 0.f});
+    }
+    if (!ctx->d_mlp_adapters) {
+        const size_t bytes = ctx->h_mlp_adapters.size() * sizeof(MlpAdapterDev);
+        ALORA_CUDA(ctx, cudaMalloc((void **)&ctx->d_mlp_adapters, bytes));
+        ALORA_CUDA(ctx, cudaMemsetAsync(ctx->d_mlp_adapters, 0, bytes, s));
+    }
+    if (!ctx->d_mlp_t) {
+        const size_t rows = (size_t)std::min(std::max(ctx->cfg.max_tokens, 1), kMlpChunk);
+        ALORA_CUDA(ctx, cudaMalloc(&ctx->d_mlp_t, rows * na * 2 * d.RP * es));
+    }
+    if (!ctx->mlp_a_gu[layer]) {
+        struct { void **p; size_t bytes; } slabs[] = {{&ctx->mlp_a_gu[layer], na * a_gu}, {&ctx->mlp_b_gu[layer], na * b_gu},
+                                                      {&ctx->mlp_a_dn[layer], mlp_dn_rows(ctx) * d.I * es},
+                                                      {&ctx->mlp_b_dn[layer], na * b_dn}};
+        for (auto &sl : slabs) {
+            ALORA_CUDA(ctx, cudaMalloc(sl.p, sl.bytes));
+            ALORA_CUDA(ctx, cudaMemsetAsync(*sl.p, 0, sl.bytes, s));
+        }
+    }
+    int n = 0, k;
+    k = launch_repack_mlp(d_Agate, d_Aup, d_Bgate, d_Bup, 2, rank, d.RP, d.H, d.I,
+                          (char *)ctx->mlp_a_gu[layer] + (size_t)adapter_id * a_gu,
+                          (char *)ctx->mlp_b_gu[layer] + (size_t)adapter_id * b_gu, s);
+    if (k < 0) return cuda_fail(ctx, cudaGetLastError(), "repack_mlp_kernel");
+    n += k;
+    k = launch_repack_mlp(d_Adown, nullptr, d_Bdown, nullptr, 1, rank, d.RP, d.I, d.H,
+                          (char *)ctx->mlp_a_dn[layer] + (size_t)adapter_id * a_dn,
+                          (char *)ctx->mlp_b_dn[layer] + (size_t)adapter_id * b_dn, s);
+    if (k < 0) return cuda_fail(ctx, cudaGetLastError(), "repack_mlp_kernel");
+    n += k;
+    const size_t idx = (size_t)layer * na + adapter_id;
+    ctx->h_mlp_adapters[idx] = MlpAdapterDev{(rank + 15) / 16 * 16, scale};
+    ctx->mlp_n_adapters[layer] = std::max(ctx->mlp_n_adapters[layer], adapter_id + 1);
+    ALORA_CUDA(ctx, cudaMemcpyAsync(ctx->d_mlp_adapters + idx, &ctx->h_mlp_adapters[idx], sizeof(MlpAdapterDev),
                                     cudaMemcpyHostToDevice, s));
     return finish(ctx, n);
 }
@@ -588,9 +660,26 @@ alora_status alora_forward_stack(alora_ctx *ctx, int mode, const void *d_hidden_
             const int tc = std::min(kMlpChunk, T - t0);
             const char *xm = (const char *)ctx->d_act[0] + (size_t)t0 * d.H * ctx->esize;
             char *hc = h + (size_t)t0 * d.H * ctx->esize;
+            // adapters on the MLP block: shrink against all of the layer's A rows (one more GEMM), then the expand
+            // step adds each open-gate row's delta in place (the row's applied adapter comes from this layer's
+            // batch metadata; base-model batches and closed gates have none)
+            const int n_mlp = (mode != ALORA_MODE_BASE && !ctx->mlp_n_adapters.empty()) ? ctx->mlp_n_adapters[l] : 0;
+            const MlpAdapterDev *mlp_tab = n_mlp ? ctx->d_mlp_adapters + (size_t)l * std::max(1, ctx->cfg.max_adapters) : nullptr;
             ALORA_STEP(launch_linear(ctx, xm, lw.wgate_up, tc, d.H, 2 * d.I, ctx->d_act[2], nullptr, s));
+            if (n_mlp) {
+                const int tw = n_mlp * 2 * d.RP;
+                ALORA_STEP(launch_linear(ctx, xm, ctx->mlp_a_gu[l], tc, d.H, tw, ctx->d_mlp_t, nullptr, s));
+                ALORA_STEP(launch_mlp_expand(ctx, ctx->d_act[2], 2 * d.I, tc, ctx->d_mlp_t, tw, ctx->mlp_b_gu[l], 2 * d.I,
+                                             d.I, 2, ctx->d_row_adapter + t0, mlp_tab, n_mlp, s));
+            }
             ALORA_STEP(launch_swiglu(ctx, ctx->d_act[2], tc, ctx->d_act[3], s));
             ALORA_STEP(launch_linear(ctx, ctx->d_act[3], lw.wdown, tc, d.I, d.H, hc, hc, s));  // h += down(...)
+            if (n_mlp) {
+                const int tw = (n_mlp * d.RP + 127) / 128 * 128;
+                ALORA_STEP(launch_linear(ctx, ctx->d_act[3], ctx->mlp_a_dn[l], tc, d.I, tw, ctx->d_mlp_t, nullptr, s));
+                ALORA_STEP(launch_mlp_expand(ctx, hc, d.H, tc, ctx->d_mlp_t, tw, ctx->mlp_b_dn[l], d.H, d.H, 1,
+                                             ctx->d_row_adapter + t0, mlp_tab, n_mlp, s));
+            }
         }
     }
 #undef ALORA_STEP

@@ -29,6 +29,12 @@ struct AdapterDev {
     int32_t pad_;
 };
 
+// One adapter's part on the MLP block of one layer (gate, up and down projections share rank and scale).
+struct MlpAdapterDev {
+    int32_t rpad;   // rank rounded up to 16; 0 = no MLP part registered
+    float scale;
+};
+
 struct LayerWeights {
     const void *wqkv = nullptr, *wo = nullptr, *wgate_up = nullptr, *wdown = nullptr;
     const void *norm_attn = nullptr, *norm_mlp = nullptr;
@@ -137,6 +143,14 @@ struct alora_ctx {
     std::vector<void *> tc_a_all, tc_b_all;          // [layer] -> [max_adapters][3*64][H], [max_adapters][N][64]
     std::vector<alora::TcLayerMaps> tc_maps;         // [layer]
     std::vector<char> layer_has_adapter;             // [layer] any adapter registered
+    // adapters on the MLP block (bf16), allocated when the first one is registered on a layer: the A rows of all
+    // adapters as one weight matrix per projection pair, the B rows per adapter
+    std::vector<void *> mlp_a_gu, mlp_b_gu;          // [layer] -> [max_adapters][2][RP][H], [max_adapters][2 I][RP]
+    std::vector<void *> mlp_a_dn, mlp_b_dn;          // [layer] -> [max_adapters][RP][I] (rows padded to 128), [max_adapters][H][RP]
+    std::vector<int> mlp_n_adapters;                 // [layer] highest registered MLP adapter id + 1
+    std::vector<alora::MlpAdapterDev> h_mlp_adapters;   // [layer * max_adapters + id], mirrors d_mlp_adapters
+    alora::MlpAdapterDev *d_mlp_adapters = nullptr;
+    void *d_mlp_t = nullptr;                         // [min(max_tokens, kMlpChunk)][max_adapters * 2 * RP] shrink results
 
     // per-call workspaces
     int32_t *d_token_req = nullptr, *d_row_adapter = nullptr, *d_slot = nullptr;

@@ -29,12 +29,14 @@ class GpuLayers:
     """A context plus device copies of weights/adapters for `n_layers` layers of one shape."""
 
     def __init__(self, shape: wl.LayerShape, layer_weights, adapters_per_layer, max_tokens, max_requests,
-                 n_adapters=None, rope_theta: float = 0.0):
+                 n_adapters=None, rope_theta: float = 0.0, mlp_adapters_per_layer=None):
         import torch
         self.shape = shape
         self.n_layers = len(layer_weights)
         n_ad = n_adapters if n_adapters is not None else max([len(a) for a in adapters_per_layer] + [1])
         max_rank = max([a.rank for per in adapters_per_layer for a in per] + [8])
+        if mlp_adapters_per_layer:
+            max_rank = max([max_rank] + [a.rank for per in mlp_adapters_per_layer for a in per if a is not None])
         self.cfg = ab.make_config(
             hidden=shape.hidden, n_q_heads=shape.n_q_heads, n_kv_heads=shape.n_kv_heads, head_dim=shape.head_dim,
             page_size=shape.page_size, n_layers=self.n_layers, intermediate=shape.intermediate if "wo" in layer_weights[0] else 0,
@@ -50,6 +52,12 @@ class GpuLayers:
             for i, a in enumerate(adapters_per_layer[l]):
                 mats = [to_dev(getattr(a, n), shape.dtype) for n in ("Aq", "Bq", "Ak", "Bk", "Av", "Bv")]
                 ab.alora_register_adapter(self.ctx, i, l, a.rank, a.scale, *mats)
+            # MLP parts (optional; None = this adapter has none on this layer), after the q/k/v parts they extend
+            for i, a in enumerate(mlp_adapters_per_layer[l] if mlp_adapters_per_layer else []):
+                if a is None:
+                    continue
+                mats = [to_dev(getattr(a, n), shape.dtype) for n in ("Ag", "Bg", "Au", "Bu", "Ad", "Bd")]
+                ab.alora_register_mlp_adapter(self.ctx, i, l, a.rank, a.scale, *mats)
         torch.cuda.synchronize()
         self.torch_dtype = torch.bfloat16 if shape.dtype == "bf16" else torch.float32
 
