@@ -216,7 +216,7 @@ def dry_run(args, world: int, rank: int) -> None:
 
 
 def fractions(peaks, roofline, sustained, config3, decode, short, recompute_8k, stack_8k, stack, evaluators,
-              evaluators_stack=None):
+              evaluators_stack=None, mlp_adapters=None):
     """Compact summary of the roofline fractions and speed-ups of all legs (None where a leg did not run)."""
     r3 = lambda x: None if x is None else round(float(x), 3)   # noqa: E731
     out = {"peaks": {"bf16_tflops": peaks["bf16_tflops"], "bf16_tflops_sustained": peaks["bf16_tflops_sustained"],
@@ -245,6 +245,10 @@ def fractions(peaks, roofline, sustained, config3, decode, short, recompute_8k, 
         out["speedup_8k_prefix_whole_layers"] = r3(stack_8k["speedup_alora_vs_full_lora"])
         out["flop_ratio_8k_prefix_whole_layers"] = r3(stack_8k["flop_ratio"])
         out["token_ratio_8k_prefix"] = r3(stack_8k["prefix_plus_suffix_over_suffix"])
+    if mlp_adapters and mlp_adapters.get("with_mlp_adapters"):
+        out["mlp_adapters_alora_overhead"] = r3(mlp_adapters["with_mlp_adapters"]["alora_overhead"])
+        out["mlp_adapters_recompute_overhead"] = r3(mlp_adapters["with_mlp_adapters"]["recompute_overhead"])
+        out["speedup_8k_prefix_mlp_adapters"] = r3(mlp_adapters["with_mlp_adapters"]["speedup_alora_vs_full_lora"])
     if stack:
         out["speedup_config4_stack"] = r3(stack["speedup_alora_vs_full_lora"])
         out["flop_ratio_config4_stack"] = r3(stack["flop_ratio"])
@@ -773,12 +777,14 @@ def evaluator_stack_leg(ab, hp, shape, stream, local, n_eval, n_layers=32, seed=
             "device_status": status, "output_finite": finite}
 
 
-def stack_leg(ab, hp, shape, stream, local, seed=4, requests=4, prefix=32768, suffix=1024, n_layers=32, name="config4"):
+def stack_leg(ab, hp, shape, stream, local, seed=4, requests=4, prefix=32768, suffix=1024, n_layers=32, name="config4",
+              with_mlp_adapters=False):
     """The decoder stack at the 8B shape (RMSNorm, attention block, o_proj, SwiGLU MLP; random bf16 weights):
     `requests` requests with `prefix` cached positions and `suffix` aLoRA suffix tokens each, against the
     full-LoRA recompute of prefix + suffix through the same stack.  Config 4 is 32 layers, 4 x (32768 + 1024);
     the 8K-prefix comparison runs 4 layers of 8 x (8192 + 256) (every layer costs the same, so the ratio is that
-    of the whole stack)."""
+    of the whole stack).  `with_mlp_adapters`: both arms are then timed once more with rank-32 adapters on the gate,
+    up and down projections of every layer as well (gated like q/k/v)."""
     import torch
     g = torch.Generator(device="cuda"); g.manual_seed(seed)
 
@@ -846,6 +852,21 @@ def stack_leg(ab, hp, shape, stream, local, seed=4, requests=4, prefix=32768, su
     a_ms = once(alora, 3)
     kern = profiled(ab, ctx, alora, 1, None)
     r_ms = once(recompute, 1)
+    mlp = None
+    if with_mlp_adapters:
+        a_hot_ms = once(alora, 3)        # the plain stack once more, in the clock state the adapted one will see
+        for l in range(n_layers):
+            m = [rnd(32, H), rnd(I, 32), rnd(32, H), rnd(I, 32), rnd(32, I), rnd(H, 32)]
+            keep.append(m)
+            ab.alora_register_mlp_adapter(ctx, 0, l, 32, 1.0, *m)
+        torch.cuda.synchronize()
+        am_ms = once(alora, 3)
+        kern_m = profiled(ab, ctx, alora, 1, None)
+        rm_ms = once(recompute, 1)
+        mlp = {"alora_ms": am_ms, "alora_ms_without": a_hot_ms, "alora_overhead": am_ms / a_hot_ms - 1.0,
+               "full_lora_recompute_ms": rm_ms,
+               "recompute_overhead": rm_ms / r_ms - 1.0, "speedup_alora_vs_full_lora": rm_ms / am_ms,
+               "per_kernel_ms_alora": {k: round(v, 3) for k, v in kern_m.items()}}
     status = ab.alora_get_status(ctx)
     finite = bool(torch.isfinite(out_a.float()).all().item())
     ab.alora_destroy(ctx)
@@ -858,7 +879,7 @@ def stack_leg(ab, hp, shape, stream, local, seed=4, requests=4, prefix=32768, su
             "full_lora_recompute_ms": r_ms, "recompute_tflops": flop_r / (r_ms / 1e3) / 1e12,
             "speedup_alora_vs_full_lora": r_ms / a_ms, "flop_ratio": flop_r / flop_a,
             "prefix_plus_suffix_over_suffix": (P + S_) / S_, "per_kernel_ms_alora": {k: round(v, 3) for k, v in kern.items()},
-            "device_status": status, "output_finite": finite}
+            "with_mlp_adapters": mlp, "device_status": status, "output_finite": finite}
 
 
 def main():
@@ -870,9 +891,9 @@ def main():
     ap.add_argument("--no-recompute", action="store_true", help="skip the full-LoRA recompute comparisons")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the decode and short-suffix legs")
-    ap.add_argument("--legs", default="sustained,config3,decode,short,recompute8k,stack8k,evaluators,evaluators_stack,stack",
+    ap.add_argument("--legs", default="sustained,config3,decode,short,recompute8k,stack8k,mlp,evaluators,evaluators_stack,stack",
                     help="extra legs to run after the main workload (comma list of sustained, config3, decode, short, "
-                         "recompute8k, stack8k, evaluators, evaluators_stack, stack)")
+                         "recompute8k, stack8k, mlp, evaluators, evaluators_stack, stack)")
     ap.add_argument("--min-seconds", type=float, default=1.0,
                     help="length of the sustained pass: the headline step repeated until this much time has been timed")
     ap.add_argument("--decode-steps", type=int, default=256)
@@ -1107,8 +1128,8 @@ def main():
     ab.alora_destroy(ctx)
     want_cpu = rank == 0 and world == 1 and not args.no_cpu_baseline
     pool_np = main_case.pool.to(torch.float32).cpu().numpy() if want_cpu else None
-    stack = evaluators = config3 = stack_8k = evaluators_stack = None
-    if legs & {"evaluators", "evaluators_stack", "stack", "stack8k", "config3"}:
+    stack = evaluators = config3 = stack_8k = evaluators_stack = mlp_adapters = None
+    if legs & {"evaluators", "evaluators_stack", "stack", "stack8k", "config3", "mlp"}:
         del main_case.pool
         torch.cuda.empty_cache()
     if "config3" in legs:
@@ -1117,6 +1138,10 @@ def main():
     if "stack8k" in legs:
         stack_8k = stack_leg(ab, hp, shape, stream, local, seed=8, requests=8, prefix=8192, suffix=256, n_layers=4,
                              name="8K-prefix comparison through whole layers")
+        torch.cuda.empty_cache()
+    if "mlp" in legs:
+        mlp_adapters = stack_leg(ab, hp, shape, stream, local, seed=9, requests=8, prefix=8192, suffix=256, n_layers=2,
+                                 name="adapters on the MLP block as well", with_mlp_adapters=True)
         torch.cuda.empty_cache()
     if "evaluators" in legs:
         evaluators = [evaluator_leg(ab, hp, shape, stream, local, n) for n in (1, 5)]
@@ -1153,10 +1178,10 @@ def main():
             "full_lora_recompute": recompute, "full_lora_recompute_8k_prefix": recompute_8k,
             "sustained": sustained, "config3": config3, "decode": decode, "short_suffix": short,
             "evaluator_pipeline": evaluators, "evaluator_pipeline_32_layers": evaluators_stack,
-            "stack_8k_prefix": stack_8k, "stack": stack, "device_status": status,
+            "stack_8k_prefix": stack_8k, "mlp_adapters": mlp_adapters, "stack": stack, "device_status": status,
             # the figures of merit in one place, last, so that a truncated copy of this line still carries them
             "fractions": fractions(peaks, roofline, sustained, config3, decode, short, recompute_8k, stack_8k, stack, evaluators,
-                                   evaluators_stack),
+                                   evaluators_stack, mlp_adapters),
         }))
     if world > 1:
         dist.destroy_process_group()

@@ -148,7 +148,7 @@ alora_status alora_register_adapter(alora_ctx *ctx, int adapter_id, int layer, i
  * (cudaMalloc; about 2 * max_adapters * 64 * (H + 3 I) bytes), so register before timing anything.
  * Errors: ALORA_ERR_NO_WEIGHTS when the adapter has no q/k/v part on this layer yet (its gate is the
  * q/k/v adapter's); ALORA_ERR_UNSUPPORTED for fp32 contexts, contexts without an MLP (intermediate = 0)
- * and sizes where H or I is not a multiple of 32; ALORA_ERR_CAPACITY for the id or rank.
+ * and sizes where H or I is not a multiple of 256; ALORA_ERR_CAPACITY for the id or rank.
  */
 alora_status alora_register_mlp_adapter(alora_ctx *ctx, int adapter_id, int layer, int rank, float scale,
                                         const void *d_Agate, const void *d_Bgate, const void *d_Aup,

@@ -373,7 +373,7 @@ alora_status alora_register_mlp_adapter(alora_ctx *ctx, int adapter_id, int laye
     if (adapter_id < 0 || adapter_id >= ctx->cfg.max_adapters) return ALORA_ERR_CAPACITY;
     if (rank < 1 || rank > ctx->cfg.max_rank) return ALORA_ERR_CAPACITY;
     const Dims &d = ctx->d;
-    if (ctx->cfg.dtype != ALORA_DTYPE_BF16 || d.I <= 0 || d.I % 32 != 0 || d.H % 32 != 0) return ALORA_ERR_UNSUPPORTED;
+    if (ctx->cfg.dtype != ALORA_DTYPE_BF16 || d.I <= 0 || d.I % 256 != 0 || d.H % 256 != 0) return ALORA_ERR_UNSUPPORTED;
     // the per-row gate of a batch is the q/k/v adapter's: the MLP part extends an adapter registered on this layer
     if (ctx->h_adapters[(size_t)layer * ctx->cfg.max_adapters + adapter_id].rank == 0) return ALORA_ERR_NO_WEIGHTS;
     cudaStream_t s = (cudaStream_t)stream;

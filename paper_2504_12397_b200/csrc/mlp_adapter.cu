@@ -46,7 +46,10 @@ int launch_repack_mlp(const void *a0, const void *a1, const void *b0, const void
     return cudaGetLastError() == cudaSuccess ? 1 : -1;
 }
 
-constexpr int kMxRows = 64, kMxCols = 256, kMxThreads = 256;
+constexpr int kMxRows = 64, kMxCols = 128, kMxThreads = 128;   // block tile of the expand step; one warp per 32 columns
+constexpr int kMxRowsPerWarp = 32 / (kMxThreads / 32);            // rows of a 32-row pass that one warp updates
+constexpr int kMxPieces = kMxCols / 128;                          // 8-byte pieces of a row per lane (32 lanes x 4 columns)
+static_assert(kMxCols == 32 * (kMxThreads / 32) && kMxCols % 128 == 0 && 32 % (kMxThreads / 32) == 0, "tile shape");
 
 struct MlpExpandArgs {
     __nv_bfloat16 *y;                  // [rows][ldy], updated in place on open-gate rows
@@ -63,27 +66,67 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
-// Block = 64 rows x 256 columns of y; warp w owns columns w * 32 .. w * 32 + 31 (four 8-wide tiles) of all 64 rows
-// (four 16-row tiles).  The rows of a request are adjacent, so the applied adapter is constant along runs of rows: the
-// block walks the runs of its 64 rows and, per run with an adapter, accumulates t (rows outside the run masked to
-// zero) times that adapter's B rows.  Every row belongs to one run, so its accumulator holds its own adapter's
-// product alone and the scale is applied per row at the end.
-__global__ void __launch_bounds__(kMxThreads) mlp_expand_add_kernel(const MlpExpandArgs a) {
+__device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void *smem_row) {
+    const uint32_t addr = (uint32_t)__cvta_generic_to_shared(smem_row);
+    asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
+                 : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+
+constexpr int kMxLd = 72;   // shared-memory row length of the t and B tiles in bf16: 64 + 8 (144 bytes: rows stay
+                            // 16-byte aligned and eight consecutive rows fall into different banks for ldmatrix)
+constexpr int kMxSB = kMxCols * kMxLd * 2, kMxST = kMxRows * kMxLd * 2;
+
+// Block = 64 rows x 128 columns of y (all of one block of the projection: gate or up); warp w owns columns
+// w * 32 .. w * 32 + 31 (four 8-wide tiles) of all 64 rows (four 16-row tiles).  The rows of a request are adjacent, so
+// the applied adapter is constant along runs of rows: the block walks the runs of its 64 rows and, per run with an
+// adapter, brings that adapter's 128 B rows and the run's t rows (rows outside the run as zeros) into shared memory
+// with 16-byte loads, takes the fragments by ldmatrix and accumulates.  Every row belongs to one run, so its
+// accumulator holds its own adapter's product alone and the scale is applied per row at the end.
+__global__ void __launch_bounds__(kMxThreads, 4) mlp_expand_add_kernel(const MlpExpandArgs a) {
     tc::grid_dep_launch();
     tc::grid_dep_wait();
     __shared__ int s_ad[kMxRows];
-    const int row0 = (int)blockIdx.x * kMxRows;
+    __shared__ unsigned s_starts[2];                    // bit i of word w: row 32 w + i starts a run
+    __shared__ __align__(16) unsigned char s_raw[kMxSB + kMxST];
+    __nv_bfloat16 *sB = reinterpret_cast<__nv_bfloat16 *>(s_raw);
+    __nv_bfloat16 *sT = reinterpret_cast<__nv_bfloat16 *>(s_raw + kMxSB);
+    // (column blocks are the fast grid dimension: the blocks that run together cover whole rows of y)
+    const int row0 = (int)blockIdx.y * kMxRows, cbase = (int)blockIdx.x * kMxCols;
     const int warp = (int)threadIdx.x >> 5, lane = (int)threadIdx.x & 31, g = lane >> 2, q = lane & 3;
-    const int col0 = (int)blockIdx.y * kMxCols + warp * 32;
+    const int col0 = cbase + warp * 32;
     if (threadIdx.x < kMxRows) {
+        // the row's applied adapter, or -1: gate closed, base model, past the last row, no MLP part registered
+        auto applied = [&](int r) {
+            const int k = r < a.rows ? a.row_adapter[r] : -1;
+            return (k < 0 || k >= a.n_adapters || a.table[k].rpad <= 0) ? -1 : k;
+        };
         const int r = row0 + (int)threadIdx.x;
-        int k = r < a.rows ? a.row_adapter[r] : -1;
-        if (k >= a.n_adapters || (k >= 0 && a.table[k].rpad <= 0)) k = -1;   // no MLP part registered: base rows
+        const int k = applied(r);
         s_ad[threadIdx.x] = k;
+        const bool start = threadIdx.x == 0 || k != applied(r - 1);
+        const unsigned starts = __ballot_sync(0xffffffffu, start);
+        if (lane == 0) s_starts[warp] = starts;
     }
     __syncthreads();
-    if (col0 >= a.ncols) return;
-    const int blk = col0 / a.width;
+    const unsigned long long run_starts = (unsigned long long)s_starts[0] | ((unsigned long long)s_starts[1] << 32);
+    const bool warp_in = col0 < a.ncols;               // (warps past the last column still fill tiles and join barriers)
+    const int blk = cbase / a.width;                   // the width is a multiple of the block's columns
+    // The y values this thread will update are requested now: their trip to DRAM overlaps the tile fills and the
+    // MMAs, and a block keeps its whole tile of reads in flight from its first microsecond on.
+    uint2 yv[2][kMxRowsPerWarp][kMxPieces];
+#pragma unroll
+    for (int pass = 0; pass < 2; ++pass)
+#pragma unroll
+        for (int i = 0; i < kMxRowsPerWarp; ++i) {
+            const int lr = pass * 32 + warp * kMxRowsPerWarp + i;
+            const bool open = s_ad[lr] >= 0;
+            const __nv_bfloat16 *yr = a.y + (size_t)(row0 + lr) * a.ldy + cbase;
+#pragma unroll
+            for (int h = 0; h < kMxPieces; ++h) {
+                const int c = h * 128 + lane * 4;
+                yv[pass][i][h] = (open && cbase + c < a.ncols) ? *reinterpret_cast<const uint2 *>(yr + c) : make_uint2(0u, 0u);
+            }
+        }
     float acc[4][4][4];
 #pragma unroll
     for (int mt = 0; mt < 4; ++mt)
@@ -92,59 +135,96 @@ __global__ void __launch_bounds__(kMxThreads) mlp_expand_add_kernel(const MlpExp
 #pragma unroll
             for (int e = 0; e < 4; ++e) acc[mt][nt][e] = 0.f;
     bool any = false;
-    for (int ra = 0; ra < kMxRows;) {
+    for (int ra = 0; ra < kMxRows;) {                  // (block-uniform: every thread sees the same runs)
         const int k = s_ad[ra];
-        int rb = ra + 1;
-        while (rb < kMxRows && s_ad[rb] == k) ++rb;
+        const unsigned long long later = ra + 1 < kMxRows ? run_starts >> (ra + 1) : 0ull;
+        const int rb = later ? ra + __ffsll((long long)later) : kMxRows;     // the next run's first row
         if (k >= 0) {
-            any = true;
             const int rpad = min(a.table[k].rpad, a.RP);
+            const int cpr = rpad >> 3;                 // 16-byte pieces per row
+            if (any) __syncthreads();                  // the previous run's fragments have been taken
+            any = true;
             const __nv_bfloat16 *tk = a.t + (size_t)(k * a.nblk + blk) * a.RP;
-            const __nv_bfloat16 *bk = a.b + ((size_t)k * a.ncols + col0) * a.RP;
-            for (int ks = 0; ks < rpad; ks += 16) {
-                uint32_t bf[4][2];
+            const __nv_bfloat16 *bk = a.b + ((size_t)k * a.ncols + cbase) * a.RP;
+            for (int i = (int)threadIdx.x; i < kMxRows * cpr; i += kMxThreads) {
+                const int r = i / cpr, c = i - r * cpr;
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (r >= ra && r < rb) v = *reinterpret_cast<const uint4 *>(tk + (size_t)(row0 + r) * a.t_ld + c * 8);
+                *reinterpret_cast<uint4 *>(sT + r * kMxLd + c * 8) = v;
+            }
+            for (int i = (int)threadIdx.x; i < kMxCols * cpr; i += kMxThreads) {
+                const int n = i / cpr, c = i - n * cpr;
+                uint4 v = make_uint4(0u, 0u, 0u, 0u);
+                if (cbase + n < a.ncols) v = *reinterpret_cast<const uint4 *>(bk + (size_t)n * a.RP + c * 8);
+                *reinterpret_cast<uint4 *>(sB + n * kMxLd + c * 8) = v;
+            }
+            __syncthreads();
+            if (warp_in) {
+                for (int ks = 0; ks < rpad; ks += 16) {
+                    // B fragments of two 8-column tiles per ldmatrix: rows = columns of y, 16 ranks wide
+                    uint32_t bf[2][4];
 #pragma unroll
-                for (int nt = 0; nt < 4; ++nt) {
-                    const bool in = col0 + nt * 8 + g < a.ncols;
-                    const __nv_bfloat16 *p = bk + (size_t)(nt * 8 + g) * a.RP + ks + 2 * q;
-                    bf[nt][0] = in ? *reinterpret_cast<const uint32_t *>(p) : 0u;
-                    bf[nt][1] = in ? *reinterpret_cast<const uint32_t *>(p + 8) : 0u;
-                }
+                    for (int np = 0; np < 2; ++np)
+                        ldmatrix_x4(bf[np], sB + (warp * 32 + np * 16 + (lane & 7) + ((lane >> 4) & 1) * 8) * kMxLd + ks +
+                                                ((lane >> 3) & 1) * 8);
 #pragma unroll
-                for (int mt = 0; mt < 4; ++mt) {
-                    if (rb <= mt * 16 || ra >= mt * 16 + 16) continue;   // the run has no row in this tile
-                    const int lo = mt * 16 + g, hi = lo + 8;
-                    const bool in_lo = lo >= ra && lo < rb, in_hi = hi >= ra && hi < rb;
-                    const __nv_bfloat16 *plo = tk + (size_t)(row0 + lo) * a.t_ld + ks + 2 * q;
-                    const __nv_bfloat16 *phi = tk + (size_t)(row0 + hi) * a.t_ld + ks + 2 * q;
-                    uint32_t af[4];
-                    af[0] = in_lo ? *reinterpret_cast<const uint32_t *>(plo) : 0u;
-                    af[1] = in_hi ? *reinterpret_cast<const uint32_t *>(phi) : 0u;
-                    af[2] = in_lo ? *reinterpret_cast<const uint32_t *>(plo + 8) : 0u;
-                    af[3] = in_hi ? *reinterpret_cast<const uint32_t *>(phi + 8) : 0u;
+                    for (int mt = 0; mt < 4; ++mt) {
+                        if (rb <= mt * 16 || ra >= mt * 16 + 16) continue;   // the run has no row in this tile
+                        uint32_t af[4];
+                        ldmatrix_x4(af, sT + (mt * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * kMxLd + ks + (lane >> 4) * 8);
 #pragma unroll
-                    for (int nt = 0; nt < 4; ++nt) mma_bf16_16816(acc[mt][nt], af, bf[nt][0], bf[nt][1]);
+                        for (int nt = 0; nt < 4; ++nt)
+                            mma_bf16_16816(acc[mt][nt], af, bf[nt >> 1][(nt & 1) * 2], bf[nt >> 1][(nt & 1) * 2 + 1]);
+                    }
                 }
             }
         }
         ra = rb;
     }
-    if (!any) return;
+    // The deltas go through shared memory, 32 rows at a time, so that y is read and written in whole 256-byte row
+    // segments (a lane's accumulator elements are 4-byte pieces of eight different rows: updating y straight from
+    // the registers scatters 16-byte accesses over as many DRAM pages and ran 14x slower).  The staging rows reuse
+    // the B tile's memory.
+    static_assert(32 * (kMxCols + 8) * 4 <= kMxSB, "the delta rows fit into the B tile");
+    float (*s_delta)[kMxCols + 8] = reinterpret_cast<float (*)[kMxCols + 8]>(s_raw);   // read as float4, written as float2
+    if (!any) return;                                  // (block-uniform) no open-gate row in this tile
+    __syncthreads();                                   // every warp has taken its last fragments
 #pragma unroll
-    for (int mt = 0; mt < 4; ++mt) {
+    for (int pass = 0; pass < 2; ++pass) {
+        if (pass) __syncthreads();
 #pragma unroll
-        for (int half = 0; half < 2; ++half) {
-            const int lr = mt * 16 + g + half * 8;
-            const int k = s_ad[lr];
-            if (k < 0) continue;
-            const float sc = a.table[k].scale;
-            __nv_bfloat16 *yr = a.y + (size_t)(row0 + lr) * a.ldy + col0 + 2 * q;
+        for (int m2 = 0; m2 < 2; ++m2) {
+            const int mt = pass * 2 + m2;
 #pragma unroll
-            for (int nt = 0; nt < 4; ++nt) {
-                if (col0 + nt * 8 + 2 * q >= a.ncols) continue;
-                __nv_bfloat162 *p = reinterpret_cast<__nv_bfloat162 *>(yr + nt * 8);
-                const float2 v = __bfloat1622float2(*p);
-                *p = __floats2bfloat162_rn(fmaf(sc, acc[mt][nt][half * 2], v.x), fmaf(sc, acc[mt][nt][half * 2 + 1], v.y));
+            for (int half = 0; half < 2; ++half) {
+                const int lr = mt * 16 + g + half * 8;
+                const int k = s_ad[lr];
+                const float sc = k >= 0 ? a.table[k].scale : 0.f;
+#pragma unroll
+                for (int nt = 0; nt < 4; ++nt)
+                    *reinterpret_cast<float2 *>(&s_delta[lr - pass * 32][warp * 32 + nt * 8 + 2 * q]) =
+                        make_float2(sc * acc[mt][nt][half * 2], sc * acc[mt][nt][half * 2 + 1]);
+            }
+        }
+        __syncthreads();
+#pragma unroll
+        for (int i = 0; i < kMxRowsPerWarp; ++i) {
+            const int lr = pass * 32 + warp * kMxRowsPerWarp + i;
+            if (s_ad[lr] < 0) continue;                        // closed gate: the row is neither read nor written
+            __nv_bfloat16 *yr = a.y + (size_t)(row0 + lr) * a.ldy + cbase;
+#pragma unroll
+            for (int h = 0; h < kMxPieces; ++h) {
+                const int c = h * 128 + lane * 4;
+                if (cbase + c >= a.ncols) continue;
+                const float4 dl = *reinterpret_cast<const float4 *>(&s_delta[lr - pass * 32][c]);
+                uint2 *p = reinterpret_cast<uint2 *>(yr + c);
+                const uint2 raw = yv[pass][i][h];
+                const float2 v0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&raw.x));
+                const float2 v1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&raw.y));
+                uint2 out;
+                *reinterpret_cast<__nv_bfloat162 *>(&out.x) = __floats2bfloat162_rn(v0.x + dl.x, v0.y + dl.y);
+                *reinterpret_cast<__nv_bfloat162 *>(&out.y) = __floats2bfloat162_rn(v1.x + dl.z, v1.y + dl.w);
+                *p = out;
             }
         }
     }
@@ -156,14 +236,14 @@ int launch_mlp_expand(alora_ctx *ctx, void *y, int ldy, int rows, const void *t,
                       int width, int nblk, const int32_t *row_adapter, const MlpAdapterDev *table, int n_adapters,
                       cudaStream_t s) {
     if (rows <= 0) return 0;
-    if (ncols % 8 != 0 || width % 32 != 0 || ldy % 2 != 0 || t_ld % 2 != 0) return -1;
+    if (ncols % 8 != 0 || width % kMxCols != 0 || ldy % 4 != 0 || t_ld % 8 != 0 || ((uintptr_t)y & 7) != 0) return -1;
     MlpExpandArgs a{};
     a.y = (__nv_bfloat16 *)y; a.t = (const __nv_bfloat16 *)t; a.b = (const __nv_bfloat16 *)b;
     a.row_adapter = row_adapter; a.table = table;
     a.rows = rows; a.ldy = ldy; a.ncols = ncols; a.width = width; a.nblk = nblk; a.t_ld = t_ld; a.RP = ctx->d.RP;
     a.n_adapters = n_adapters;
     ProfScope prof(ctx, KK_LINEAR, s);
-    const dim3 grid((rows + kMxRows - 1) / kMxRows, (ncols + kMxCols - 1) / kMxCols);
+    const dim3 grid((ncols + kMxCols - 1) / kMxCols, (rows + kMxRows - 1) / kMxRows);
     if (launch_kernel(mlp_expand_add_kernel, grid, dim3(kMxThreads), 0, s, true, a) != cudaSuccess) return -1;
     return 1;
 }
