@@ -216,7 +216,7 @@ def dry_run(args, world: int, rank: int) -> None:
 
 
 def fractions(peaks, roofline, sustained, config3, decode, short, recompute_8k, stack_8k, stack, evaluators,
-              evaluators_stack=None, mlp_adapters=None):
+              evaluators_stack=None, mlp_adapters=None, regime2=None):
     """Compact summary of the roofline fractions and speed-ups of all legs (None where a leg did not run)."""
     r3 = lambda x: None if x is None else round(float(x), 3)   # noqa: E731
     out = {"peaks": {"bf16_tflops": peaks["bf16_tflops"], "bf16_tflops_sustained": peaks["bf16_tflops_sustained"],
@@ -239,6 +239,9 @@ def fractions(peaks, roofline, sustained, config3, decode, short, recompute_8k, 
             out[key + "_attention_hbm"] = r3(s_["attention_frac_of_hbm_peak"])
             out[key + "_ms_per_step"] = r3(s_["ms_per_step"])
             out[key + "_projection_ms"] = r3(s_["per_kernel_ms"].get("project_qkv", 0.0) + s_["per_kernel_ms"].get("shrink", 0.0))
+    if regime2:
+        out["chunk_straddling_ms_per_step"] = r3(regime2["ms_per_step"])
+        out["chunk_straddling_vs_activation_at_chunk_start"] = r3(regime2["ms_per_step"] / regime2["ms_per_step_activation_at_chunk_start"])
     if recompute_8k:
         out["speedup_8k_prefix_qkv_attention"] = r3(recompute_8k["speedup_alora_vs_full_lora"])
     if stack_8k:
@@ -316,9 +319,9 @@ def profiled(ab, ctx, step, n, flush):
 class PrefillCase:
     """Device buffers of one suffix-prefill batch at the 8B layer shape plus its full-LoRA recompute twin."""
 
-    def __init__(self, hp, shape, requests, prefix, suffix, seed, with_recompute):
+    def __init__(self, hp, shape, requests, prefix, suffix, seed, with_recompute, activation_shift=0):
         import torch
-        self.w = wl.config2(seed=seed, requests=requests, prefix=prefix, suffix=suffix)
+        self.w = wl.config2(seed=seed, requests=requests, prefix=prefix, suffix=suffix, activation_shift=activation_shift)
         b = self.b = self.w.batch
         self.T, self.R = b.T, b.R
         self.full_T = int(b.seq_lens.sum())
@@ -421,9 +424,11 @@ def parse_short_case(text):
     return r, s, int(prefix) if prefix else 4096
 
 
-def short_suffix_leg(ab, hp, ctx, shape, stream, flush, peaks, requests, prefix, suffix, seed=7):
-    """The paper-shaped short invocation: `suffix` new tokens per request on a reused cache (HBM-bound attention)."""
-    c = PrefillCase(hp, shape, requests, prefix, suffix, seed, with_recompute=False)
+def short_suffix_leg(ab, hp, ctx, shape, stream, flush, peaks, requests, prefix, suffix, seed=7, activation_shift=0):
+    """The paper-shaped short invocation: `suffix` new tokens per request on a reused cache (HBM-bound attention).
+    With `activation_shift` the adapter activates that many tokens into the new chunk (an uncached context tail
+    prefilled with the base weights in the same call as the invocation)."""
+    c = PrefillCase(hp, shape, requests, prefix, suffix, seed, with_recompute=False, activation_shift=activation_shift)
     for _ in range(5):
         c.step(ab, ctx, stream)
     ms = timed(lambda: c.step(ab, ctx, stream), 50, stream, flush)
@@ -431,7 +436,7 @@ def short_suffix_leg(ab, hp, ctx, shape, stream, flush, peaks, requests, prefix,
     attn_ms = kern.get("attention", 0.0) + kern.get("attn_merge", 0.0)
     _, _, attn_bytes = c.flops_bytes(shape, 32)
     gbs = attn_bytes / (attn_ms / 1e3) / 1e9 if attn_ms else None
-    return {"requests": requests, "prefix": prefix, "suffix": suffix, "ms_per_step": ms,
+    return {"requests": requests, "prefix": prefix, "suffix": suffix, "activation_shift": activation_shift, "ms_per_step": ms,
             "tokens_per_s": c.T / (ms / 1e3), "per_kernel_ms": {k: round(v, 4) for k, v in kern.items()},
             "attention_hbm_gbs": gbs, "attention_frac_of_hbm_peak": gbs / peaks["hbm_gbs"] if gbs else None}
 
@@ -891,9 +896,9 @@ def main():
     ap.add_argument("--no-recompute", action="store_true", help="skip the full-LoRA recompute comparisons")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     ap.add_argument("--no-extra", action="store_true", help="skip the decode and short-suffix legs")
-    ap.add_argument("--legs", default="sustained,config3,decode,short,recompute8k,stack8k,mlp,evaluators,evaluators_stack,stack",
+    ap.add_argument("--legs", default="sustained,config3,decode,short,regime2,recompute8k,stack8k,mlp,evaluators,evaluators_stack,stack",
                     help="extra legs to run after the main workload (comma list of sustained, config3, decode, short, "
-                         "recompute8k, stack8k, mlp, evaluators, evaluators_stack, stack)")
+                         "regime2, recompute8k, stack8k, mlp, evaluators, evaluators_stack, stack)")
     ap.add_argument("--min-seconds", type=float, default=1.0,
                     help="length of the sustained pass: the headline step repeated until this much time has been timed")
     ap.add_argument("--decode-steps", type=int, default=256)
@@ -1124,6 +1129,13 @@ def main():
     if "short" in legs:
         short = [short_suffix_leg(ab, hp, ctx, shape, stream, flush, peaks, r_, p_, s_)
                  for r_, s_, p_ in [parse_short_case(c) for c in args.short_cases.split(",") if c]]
+    regime2 = None
+    if "regime2" in legs:
+        # the headline shape with the activation offset 192 tokens into the 256 new ones: an uncached tail of the
+        # context goes through the base weights, the 64-token invocation through the adapter, in ONE call
+        regime2 = short_suffix_leg(ab, hp, ctx, shape, stream, flush, peaks, args.requests, args.prefix, args.suffix,
+                                   seed=12, activation_shift=(3 * args.suffix) // 4)
+        regime2["ms_per_step_activation_at_chunk_start"] = step_ms
     status = ab.alora_get_status(ctx)
     ab.alora_destroy(ctx)
     want_cpu = rank == 0 and world == 1 and not args.no_cpu_baseline
@@ -1178,10 +1190,10 @@ def main():
             "full_lora_recompute": recompute, "full_lora_recompute_8k_prefix": recompute_8k,
             "sustained": sustained, "config3": config3, "decode": decode, "short_suffix": short,
             "evaluator_pipeline": evaluators, "evaluator_pipeline_32_layers": evaluators_stack,
-            "stack_8k_prefix": stack_8k, "mlp_adapters": mlp_adapters, "stack": stack, "device_status": status,
+            "chunk_straddling_prefill": regime2, "stack_8k_prefix": stack_8k, "mlp_adapters": mlp_adapters, "stack": stack, "device_status": status,
             # the figures of merit in one place, last, so that a truncated copy of this line still carries them
             "fractions": fractions(peaks, roofline, sustained, config3, decode, short, recompute_8k, stack_8k, stack, evaluators,
-                                   evaluators_stack, mlp_adapters),
+                                   evaluators_stack, mlp_adapters, regime2),
         }))
     if world > 1:
         dist.destroy_process_group()

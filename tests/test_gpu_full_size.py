@@ -96,6 +96,34 @@ def test_config2_bench_workload_sampled_requests(oracle64):
     _check_requests(oracle64, w.shape, w, w.batch, before, after, out_h, range(w.batch.R), qkv_h)
 
 
+def test_chunk_straddling_prefill_at_the_bench_shape(oracle64):
+    """The headline shape with the activation offset 192 tokens into the 256 new ones (the paper's second regime: an
+    uncached tail of the context and the invocation in one call).  Requests 0 and 7 against the oracle; and the
+    rows before the offset are BASE-EXACT: their projection rows and their appended K/V have the bits of a call
+    with every gate closed, so the base model can later reuse what this call cached for them."""
+    w = wl.config2(seed=12, activation_shift=192)
+    b, shape = w.batch, w.shape
+    before, after, out_h, qkv_h = _run_layer(w, seed=1012, with_qkv=True)
+    _check_requests(oracle64, shape, w, b, before, after, out_h, [0, b.R - 1], qkv_h)
+    import copy
+    wb = copy.copy(w)
+    wb.batch = copy.copy(b)
+    wb.batch.adapter_ids = np.full(b.R, -1, np.int32)
+    _, after_b, _, qkv_b = _run_layer(wb, seed=1012, with_qkv=True)
+    S = 256
+    closed = np.concatenate([np.arange(r * S, r * S + 192) for r in range(b.R)])
+    opened = np.setdiff1d(np.arange(b.T), closed)
+    assert np.array_equal(qkv_h[closed].view(np.uint32), qkv_b[closed].view(np.uint32))
+    assert hp.rel_err(qkv_h[opened], qkv_b[opened]) > 1e-3
+    for r in (0, 3, b.R - 1):
+        P = int(b.prefix_lens[r])
+        Ka, Va = _request_kv(after, b, r, P + S, shape)
+        Kb, Vb = _request_kv(after_b, b, r, P + S, shape)
+        assert np.array_equal(Ka[:P + 192].view(np.uint32), Kb[:P + 192].view(np.uint32)), f"base-exact K of request {r}"
+        assert np.array_equal(Va[:P + 192].view(np.uint32), Vb[:P + 192].view(np.uint32)), f"base-exact V of request {r}"
+        assert not np.array_equal(Ka[P + 192:], Kb[P + 192:])
+
+
 def test_config3_ragged_multi_adapter_sampled_requests(oracle64):
     """32 requests over adapters of ranks 8/16/32/64, prefixes 512..16384, suffixes 16..512, shuffled pages:
     in full, the request with the most work (longest suffix x context), the request with the most work on the
