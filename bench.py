@@ -319,9 +319,10 @@ def profiled(ab, ctx, step, n, flush):
 class PrefillCase:
     """Device buffers of one suffix-prefill batch at the 8B layer shape plus its full-LoRA recompute twin."""
 
-    def __init__(self, hp, shape, requests, prefix, suffix, seed, with_recompute, activation_shift=0):
+    def __init__(self, hp, shape, requests, prefix, suffix, seed, with_recompute, activation_shift=0, shuffle_pages=False):
         import torch
-        self.w = wl.config2(seed=seed, requests=requests, prefix=prefix, suffix=suffix, activation_shift=activation_shift)
+        self.w = wl.config2(seed=seed, requests=requests, prefix=prefix, suffix=suffix, activation_shift=activation_shift,
+                            shuffle_pages=shuffle_pages)
         b = self.b = self.w.batch
         self.T, self.R = b.T, b.R
         self.full_T = int(b.seq_lens.sum())
@@ -424,11 +425,13 @@ def parse_short_case(text):
     return r, s, int(prefix) if prefix else 4096
 
 
-def short_suffix_leg(ab, hp, ctx, shape, stream, flush, peaks, requests, prefix, suffix, seed=7, activation_shift=0):
+def short_suffix_leg(ab, hp, ctx, shape, stream, flush, peaks, requests, prefix, suffix, seed=7, activation_shift=0,
+                     shuffle_pages=False):
     """The paper-shaped short invocation: `suffix` new tokens per request on a reused cache (HBM-bound attention).
     With `activation_shift` the adapter activates that many tokens into the new chunk (an uncached context tail
     prefilled with the base weights in the same call as the invocation)."""
-    c = PrefillCase(hp, shape, requests, prefix, suffix, seed, with_recompute=False, activation_shift=activation_shift)
+    c = PrefillCase(hp, shape, requests, prefix, suffix, seed, with_recompute=False, activation_shift=activation_shift,
+                    shuffle_pages=shuffle_pages)
     for _ in range(5):
         c.step(ab, ctx, stream)
     ms = timed(lambda: c.step(ab, ctx, stream), 50, stream, flush)
@@ -436,7 +439,8 @@ def short_suffix_leg(ab, hp, ctx, shape, stream, flush, peaks, requests, prefix,
     attn_ms = kern.get("attention", 0.0) + kern.get("attn_merge", 0.0)
     _, _, attn_bytes = c.flops_bytes(shape, 32)
     gbs = attn_bytes / (attn_ms / 1e3) / 1e9 if attn_ms else None
-    return {"requests": requests, "prefix": prefix, "suffix": suffix, "activation_shift": activation_shift, "ms_per_step": ms,
+    return {"requests": requests, "prefix": prefix, "suffix": suffix, "activation_shift": activation_shift,
+            "pages": "shuffled" if shuffle_pages else "contiguous", "ms_per_step": ms,
             "tokens_per_s": c.T / (ms / 1e3), "per_kernel_ms": {k: round(v, 4) for k, v in kern.items()},
             "attention_hbm_gbs": gbs, "attention_frac_of_hbm_peak": gbs / peaks["hbm_gbs"] if gbs else None}
 
@@ -906,6 +910,8 @@ def main():
     ap.add_argument("--short-cases", default="8x4,8x16,64x4,64x16",
                     help="the short-suffix leg's cases as requests x suffix tokens, on 4096 cached tokens each unless "
                          "'@cached' follows (64x4@16384)")
+    ap.add_argument("--short-pages", default="contiguous", choices=["contiguous", "shuffled"],
+                    help="physical page order of the short-suffix leg's caches")
     ap.add_argument("--requests", type=int, default=8)
     ap.add_argument("--prefix", type=int, default=4096)
     ap.add_argument("--suffix", type=int, default=256)
@@ -1127,7 +1133,7 @@ def main():
         decode = decode_leg(ab, hp, ctx, shape, stream, flush, peaks, steps=args.decode_steps,
                             ctx_max=args.decode_ctx_max)
     if "short" in legs:
-        short = [short_suffix_leg(ab, hp, ctx, shape, stream, flush, peaks, r_, p_, s_)
+        short = [short_suffix_leg(ab, hp, ctx, shape, stream, flush, peaks, r_, p_, s_, shuffle_pages=args.short_pages == "shuffled")
                  for r_, s_, p_ in [parse_short_case(c) for c in args.short_cases.split(",") if c]]
     regime2 = None
     if "regime2" in legs:

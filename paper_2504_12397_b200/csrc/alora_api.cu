@@ -634,6 +634,9 @@ alora_status alora_forward_stack(alora_ctx *ctx, int mode, const void *d_hidden_
     ALORA_CUDA(ctx, cudaSetDevice(ctx->cfg.device));
     const Dims &d = ctx->d;
     ALORA_BATCH(mode);
+    // one token per request (the decode entry passes the context's own 0, 1, ..., R as query_start_loc): every request
+    // is on the few-row attention list, the tensor-core attention kernel has nothing to do and is not launched
+    b.all_small = (d_query_start_loc == ctx->d_iota && T == R) ? 1 : 0;
     if (d_hidden_out != d_hidden_in && T > 0)
         ALORA_CUDA(ctx, cudaMemcpyAsync(d_hidden_out, d_hidden_in, (size_t)T * d.H * ctx->esize, cudaMemcpyDeviceToDevice, s));
     char *h = (char *)d_hidden_out;  // residual stream, updated in place

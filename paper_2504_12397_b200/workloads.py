@@ -238,7 +238,8 @@ def config1(seed: int = 0) -> Workload:
 
 
 def config2(seed: int = 2, requests: int = 8, prefix: int = 4096, suffix: int = 256,
-            shape: LayerShape = SHAPE_8B, rank: int = 32, activation_shift: int = 0) -> Workload:
+            shape: LayerShape = SHAPE_8B, rank: int = 32, activation_shift: int = 0,
+            shuffle_pages: bool = False) -> Workload:
     """One 8B-shape bf16 layer: 8 requests x (4096 cached + 256 new at the activation offset).  With
     `activation_shift` > 0 the adapter activates that many tokens INTO the new chunk: the call prefills an
     uncached tail of the context with the base weights and the invocation with the adapter (the paper's second
@@ -247,7 +248,7 @@ def config2(seed: int = 2, requests: int = 8, prefix: int = 4096, suffix: int = 
     w = make_wqkv(shape, rng)
     ad = [make_adapter(shape, rank, rng)]
     b = make_batch(shape, [prefix] * requests, [suffix] * requests, [0] * requests, rng,
-                   activation_offsets=[prefix + activation_shift] * requests)
+                   activation_offsets=[prefix + activation_shift] * requests, shuffle_pages=shuffle_pages)
     return Workload("config2_8b_layer", shape, w, ad, b, seed)
 
 
