@@ -366,6 +366,26 @@ alora_status alora_cow_tail_pages(alora_ctx *ctx, const int32_t *d_query_start_l
 alora_status alora_selftest_wait_timeout(alora_ctx *ctx, int64_t limit_cycles, void *stream);
 
 /*
+ * Several contexts, streams and processes may use one GPU at the same time: they share its SMs, and a launch of
+ * this library never assumes that all of its blocks are running at once.  Where one work item of a launch needs
+ * another's result (a projection item needs its row tile's shrink item), the needed items are handed out through
+ * a counter to blocks that are running, and no block starts on a dependent item before every needed item has been
+ * claimed (csrc/claim_order.h).  Every in-kernel wait is bounded (about a second): if one still runs out, the
+ * kernel returns through its normal exit, ALORA_ERR_TIMEOUT is recorded in the status word, and the outputs of
+ * that call are not valid; the context stays usable.
+ *
+ * alora_selftest_claim_order is a HOST-ONLY model of that item order (no device, no context): a launch of `grid`
+ * blocks with n_shrink shrink items and n_row_tiles x n_col_tiles projection items runs on a GPU that keeps only
+ * `resident_slots` blocks running at a time, blocks entering free slots highest index first
+ * (high_blocks_first != 0) or lowest first.  *completed = 1 when every item completes, 0 when running blocks end
+ * up waiting for items that no running block holds.  static_order != 0 models dealing ALL items by block index
+ * instead (the order the counter replaced), for comparison.  ALORA_ERR_INVALID_ARG for sizes out of range.
+ */
+alora_status alora_selftest_claim_order(int grid, int n_shrink, int n_row_tiles, int n_col_tiles,
+                                        int resident_slots, int high_blocks_first, int static_order,
+                                        int *completed);
+
+/*
  * Optional per-kernel timing (a measurement aid; the paper has no counterpart).  While enabled,
  * every kernel family launched by this context is bracketed by CUDA events on the launching stream.
  * alora_profile_enable(ctx, 1) clears what was accumulated and starts, (ctx, 0) stops.

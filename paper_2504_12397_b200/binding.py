@@ -153,6 +153,20 @@ def alora_register_mlp_adapter(ctx, adapter_id, layer, rank, scale, Ag, Bg, Au, 
     _check(ctx, rc, "alora_register_mlp_adapter")
 
 
+def alora_selftest_claim_order(grid, n_shrink, n_row_tiles, n_col_tiles, resident_slots, high_blocks_first=True,
+                               static_order=False) -> bool:
+    """Host-only model of the projection launch's item order; True when every item completes."""
+    lib = load_library()
+    lib.alora_selftest_claim_order.argtypes = [_I] * 7 + [C.POINTER(C.c_int)]
+    lib.alora_selftest_claim_order.restype = C.c_int
+    done = C.c_int(-1)
+    rc = lib.alora_selftest_claim_order(grid, n_shrink, n_row_tiles, n_col_tiles, resident_slots,
+                                        int(bool(high_blocks_first)), int(bool(static_order)), C.byref(done))
+    if rc != 0:
+        raise AloraError(rc, "alora_selftest_claim_order", "")
+    return done.value == 1
+
+
 def alora_validate_batch(cfg: alora_config, positions, activation_offsets, adapter_ids, query_start_loc,
                          seq_lens, block_tables, num_pages: int) -> int:
     """Host-side check; arguments are numpy int32 arrays (block_tables 2-D).  Returns the status code."""

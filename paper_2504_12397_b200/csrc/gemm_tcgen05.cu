@@ -31,6 +31,7 @@
 // outstanding copies and tensor-core work with bounded waits, frees its tensor memory and returns.
 #include "alora_internal.h"
 #include "tc_common.cuh"
+#include "claim_order.h"
 
 namespace alora {
 
@@ -193,7 +194,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
             // resident; and in the usual case every block keeps the items (and the L2 neighbours) it always had.
             bool shrink_phase = n_shrink > 0;
             int stat = (int)blockIdx.x;
-            if (shrink_phase && (int)blockIdx.x >= n_shrink) {
+            if (shrink_phase && !claims_at_once((int)blockIdx.x, n_shrink)) {
                 // The blocks with the lowest indices have a free place in their list and normally take the shrink items
                 // within a microsecond.  The others look on for a short while (about 30 us) and join the claiming
                 // only if the shrink items are still not all taken by then (blocks that have not been scheduled).
@@ -208,8 +209,7 @@ gemm_tcgen05_kernel(const __grid_constant__ CUtensorMap tmA, const __grid_consta
                     if (item >= n_shrink) { shrink_phase = false; item = -1; }
                 }
                 if (!shrink_phase && item < 0) {
-                    while (stat < n_shrink) stat += (int)gridDim.x;
-                    if (stat < total) { item = stat; stat += (int)gridDim.x; }
+                    item = next_dealt_item(stat, n_shrink, total, (int)gridDim.x);
                 }
                 if (!ring.put(item, abort_flag)) { ok = false; break; }
                 if (item < 0) break;

@@ -112,3 +112,21 @@ def test_missing_library_is_reported(tmp_path, monkeypatch):
     monkeypatch.setattr(ab, "LIB_PATH", str(tmp_path / "nope.so"))
     with pytest.raises(ab.AloraLibraryMissing):
         ab.load_library()
+
+
+def test_projection_item_order_never_waits_for_a_block_that_is_not_running():
+    """Host-side model of the order in which a projection launch's blocks take their items (csrc/claim_order.h, the
+    two decisions the kernels use): with shrink items claimed from a counter every item completes however few blocks
+    are running and whichever blocks start first; dealing all items by block index (the order it replaced) leaves
+    running blocks waiting for shrink items of blocks that never get a slot."""
+    from paper_2504_12397_b200 import binding as ab
+    for grid, n_shrink, rows, cols in ((148, 16, 16, 24), (148, 200, 264, 24), (8, 3, 5, 2), (4, 9, 9, 1), (148, 1, 40, 32)):
+        for slots in (1, 2, 7, grid):
+            for high_first in (True, False):
+                assert ab.alora_selftest_claim_order(grid, n_shrink, rows, cols, slots, high_first), (grid, n_shrink, slots, high_first)
+    # the replaced order: fine when every block runs, stuck when the low blocks cannot start
+    assert ab.alora_selftest_claim_order(148, 16, 16, 24, 148, True, static_order=True)
+    assert not ab.alora_selftest_claim_order(148, 16, 16, 24, 100, True, static_order=True)
+    assert not ab.alora_selftest_claim_order(8, 3, 5, 2, 2, True, static_order=True)
+    # no shrink items at all (a base-only launch): nothing to claim, nothing to wait for
+    assert ab.alora_selftest_claim_order(148, 0, 16, 24, 3, True)
