@@ -139,8 +139,8 @@ alora_status alora_register_adapter(alora_ctx *ctx, int adapter_id, int layer, i
 /*
  * Extend adapter `adapter_id` of `layer` to the MLP block: gate, up and down projections each get
  * Delta = scale * B A under the SAME per-token gate as q/k/v (the paper adapts q, k and v and remarks,
- * in its background section and after Eq. 5, that MLP blocks are adapted by the corresponding
- * equations).  d_Agate and d_Aup are [rank][H], d_Bgate and d_Bup are [I][rank], d_Adown is [rank][I],
+ * in its background section and after Eq. 5, that MLP blocks can be adapted in the same manner).
+ * d_Agate and d_Aup are [rank][H], d_Bgate and d_Bup are [I][rank], d_Adown is [rank][I],
  * d_Bdown is [H][rank]; I = intermediate size.  Only alora_forward_stack and alora_decode_stack run
  * the MLP block, so only they use these matrices: rows whose gate is open get the deltas, rows whose
  * gate is closed (and every row in ALORA_MODE_BASE) keep the bits of the base MLP.  The matrices are

@@ -57,7 +57,7 @@ class Adapter:
 @dataclass
 class MlpAdapter:
     """The same adapter's low-rank pairs on the MLP block's gate, up and down projections (the paper's remark that
-    MLP blocks are adapted by the equations corresponding to Eq. 5)."""
+    MLP blocks can be adapted in the same manner as q, k and v in Eq. 5)."""
     rank: int
     scale: float
     Ag: np.ndarray  # [r, H]
@@ -144,7 +144,7 @@ class Oracle:
         assert rc == 0, "oracle_project_qkv: bad arguments"
         return qkv, gate
 
-    # ---- the equation corresponding to Eq. 5 for one MLP weight matrix ------------------------------
+    # ---- Eq. 5's gate applied to one MLP weight matrix -------------- ------------------------------
     def gated_linear(self, x, W, positions, query_start_loc, activation_offsets, adapter_ids, ranks, scales,
                      As, Bs, force_all: bool = False) -> np.ndarray:
         """y_t = W x_t, plus scale * B (A x_t) on the rows of adapter requests at or after the activation offset.

@@ -153,8 +153,8 @@ int oracle_project_qkv(const double *x, const float *W, int T, int H, int Nq, in
 
 /*
  * Gated low-rank adaptation of ONE weight matrix of an MLP block (gate, up or down projection).
- * The paper states that MLP blocks can be adapted by the equations that correspond to Eq. 5 for
- * Q, K and V (Sec. 2, remark on MLP blocks; Sec. 3, the sentence after Eq. 5): a token before the
+ * The paper remarks that MLP blocks can be adapted in the same manner as Q, K and V in Eq. 5
+ * (Sec. 2, remark on MLP blocks; Sec. 3, the sentence after Eq. 5): a token before the
  * activation offset is multiplied by the base weight alone, a token at or after it by W + s B A.
  *
  *   y_t = W x_t                        if the request has no adapter, or p_t < a_req

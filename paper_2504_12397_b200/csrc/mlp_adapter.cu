@@ -1,5 +1,5 @@
 // Gated low-rank adapters on the MLP block's gate, up and down projections.  The paper adapts q, k and v and remarks
-// that MLP blocks are adapted "by the corresponding equations": a row at or after its request's activation offset sees
+// that MLP blocks can be adapted in the same manner: a row at or after its request's activation offset sees
 // W + s B A, a row before it the base weight alone (the form of Eq. 5).  The dense product y = W x is the stack's
 // ordinary GEMM; the low-rank part runs beside it in two steps:
 //   shrink   t[row][k][blk][i] = sum_h A_k,blk[i][h] x[row][h]    for ALL registered adapters k of the layer at once:

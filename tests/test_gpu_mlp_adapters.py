@@ -1,5 +1,5 @@
 """GPU parity of gated adapters on the MLP block (gate, up and down projections adapted under the same per-token gate
-as q/k/v, the equations corresponding to Eq. 5): the decoder stack through the C ABI against the CPU oracle."""
+as q/k/v, Eq. 5's form per matrix): the decoder stack through the C ABI against the CPU oracle."""
 import numpy as np
 import pytest
 

@@ -493,7 +493,7 @@ def test_decoder_layer_against_library_restatement(oracle64):
     assert np.abs(got - h).max() > 0.1
 
 
-# ---- gated adapters on the MLP block (the equations corresponding to Eq. 5) ---------------------------
+# ---- gated adapters on the MLP block (Eq. 5's form applied to gate, up, down) ---------------------------
 
 def _mlp_ad(a: wl.MlpAdapterWeights) -> MlpAdapter:
     return MlpAdapter(a.rank, a.scale, a.Ag, a.Bg, a.Au, a.Bu, a.Ad, a.Bd)
