@@ -51,11 +51,12 @@ def brute_force_groups(b: wl.Batch, page, G, small_max):
     return first, shared
 
 
-def _conversation_batch(rng, convs, per_conv, new_tokens, base_lens, own_extra):
+def _conversation_batch(rng, convs, per_conv, new_tokens, base_lens, own_extra, shape=None):
     """`convs` conversations; conversation c has base_lens[c] cached keys on pages of its own; per_conv[c] requests
     point their leading block-table entries at those pages (whole pages only), have own_extra[...] further cached
     keys on private pages, and new_tokens[...] new tokens."""
-    page = SHAPE.page_size
+    shape = shape or SHAPE
+    page = shape.page_size
     prefix, new, ids, owners = [], [], [], []
     k = 0
     for c in range(convs):
@@ -65,7 +66,7 @@ def _conversation_batch(rng, convs, per_conv, new_tokens, base_lens, own_extra):
             ids.append((k % 3) - 1)
             owners.append(c)
             k += 1
-    b = wl.make_batch(SHAPE, prefix, new, ids, rng, shuffle_pages=True, spare_pages=convs * 300)
+    b = wl.make_batch(shape, prefix, new, ids, rng, shuffle_pages=True, spare_pages=convs * 300)
     # the conversations' own pages are taken from the spare pages at the end of the shuffled pool
     used = set(int(x) for r in range(b.R) for x in b.block_tables[r, :(b.seq_lens[r] + page - 1) // page])
     free = [p for p in range(b.num_pages) if p not in used]
@@ -78,7 +79,7 @@ def _conversation_batch(rng, convs, per_conv, new_tokens, base_lens, own_extra):
     return b, owners
 
 
-def _run(oracle64, b, check_groups=True):
+def _run(oracle64, b, check_groups=True, SHAPE=SHAPE):
     import torch
     rng = np.random.default_rng(5)
     wqkv = wl.make_wqkv(SHAPE, rng)
@@ -132,6 +133,25 @@ def test_five_evaluators_per_conversation_decode_step(oracle64):
     first, shared = _run(oracle64, b)
     assert all(first[r] == (r // 5) * 5 for r in range(b.R))
     assert all(shared[r] == (base[r // 5] // 16 * 16) // 64 * 64 for r in range(b.R))
+
+
+def test_five_evaluators_per_conversation_at_the_8b_layer_shape(oracle64):
+    """The decode step of the evaluator pipeline at full size: the 8B layer shape (8 KV heads, group size 4), 8
+    conversations of 4100 .. 4400 cached tokens, each read by 5 requests (two adapters and the base model) with 16 .. 48
+    cached tokens of their own and one new token.  Eight prefix groups of five (20 stacked score rows each); every
+    request against the oracle, the grouping against the brute-force rule, the shared pages bit-identical."""
+    rng = np.random.default_rng(24)
+    shape = wl.SHAPE_8B
+    convs = 8
+    base = [int(x) for x in rng.integers(4100, 4401, convs)]
+    n = convs * 5
+    b, owners = _conversation_batch(rng, convs, [5] * convs, [1] * n, base, [int(x) for x in rng.integers(16, 49, n)],
+                                    shape=shape)
+    first, shared = _run(oracle64, b, SHAPE=shape)
+    for c in range(convs):
+        members = [r for r in range(b.R) if owners[r] == c]
+        assert all(first[r] == members[0] for r in members)
+        assert all(shared[r] == base[c] // shape.page_size * shape.page_size // 64 * 64 for r in members)
 
 
 def test_mixed_groups_loners_and_long_requests(oracle64):
