@@ -393,8 +393,9 @@ alora_status alora_selftest_claim_order(int grid, int n_shrink, int n_row_tiles,
  * the number of bracketed launch groups; both arrays have ALORA_PROFILE_KINDS entries.
  * Families: 0 batch metadata, 1 rank-r shrink (t = A x) when it is a launch of its own, or the per-row
  * low-rank delta of small batches, 2 q/k/v projection (on the bf16 layer paths it also appends the new k / v rows
- * to the cache), 3 KV append as a launch of its own (alora_kv_append, fp32 layers), 4 attention (both attention
- * kernels and the merge of cut work items), 5 unused, 6 other dense projections (o_proj, MLP), 7 norm / activation
+ * to the cache), 3 KV append as a launch of its own (alora_kv_append, fp32 layers), 4 attention on the tensor-core
+ * kernel (with the merge of cut work items) and the fp32 kernel, 5 attention on the few-row split-KV kernel (decode
+ * steps, shortest suffixes, prefix groups), 6 other dense projections (o_proj, MLP), 7 norm / activation
  * glue.
  */
 #define ALORA_PROFILE_KINDS 8

@@ -299,7 +299,7 @@ def alora_launch_count(ctx) -> int:
     return int(load_library().alora_launch_count(ctx))
 
 
-PROFILE_KINDS = ("metadata", "shrink", "project_qkv", "kv_append", "attention", "attn_merge", "linear", "glue")
+PROFILE_KINDS = ("metadata", "shrink", "project_qkv", "kv_append", "attention", "attention_few_row", "linear", "glue")
 
 
 def alora_profile_enable(ctx, on: bool) -> None:

@@ -100,7 +100,7 @@ struct FewRowMeta {
 };
 
 // Kernel families, for the optional per-kernel timing (alora_profile_*).
-enum KernelKind { KK_METADATA = 0, KK_SHRINK, KK_PROJECT, KK_KV_APPEND, KK_ATTENTION, KK_ATTN_MERGE, KK_LINEAR,
+enum KernelKind { KK_METADATA = 0, KK_SHRINK, KK_PROJECT, KK_KV_APPEND, KK_ATTENTION, KK_ATTN_FEW_ROW, KK_LINEAR,
                   KK_GLUE, KK_COUNT };
 
 struct ProfEvent {

@@ -615,7 +615,7 @@ int launch_attend_splitkv(alora_ctx *ctx, const void *qkv, const BatchArgs &b, c
     }
     const int grid = std::max(1, std::min(ctx->sm_count, ctx->max_split_items));
     {
-        ProfScope prof(ctx, KK_ATTENTION, s);
+        ProfScope prof(ctx, KK_ATTN_FEW_ROW, s);
         const cudaError_t e = hi ? launch_kernel(attn_splitkv_kernel<128>, dim3(grid), dim3(kSkThreads), SkSmem<128>::kTotal, s, true, tmKV, a)
                                  : launch_kernel(attn_splitkv_kernel<64>, dim3(grid), dim3(kSkThreads), SkSmem<64>::kTotal, s, true, tmKV, a);
         if (e != cudaSuccess) return -1;
