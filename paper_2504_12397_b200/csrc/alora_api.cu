@@ -24,6 +24,8 @@ int launch_repack_mlp(const void *, const void *, const void *, const void *, in
                       cudaStream_t);   // mlp_adapter.cu
 int launch_mlp_expand(alora_ctx *, void *, int, int, const void *, int, const void *, int, int, int, const int32_t *,
                       const MlpAdapterDev *, int, cudaStream_t);
+int launch_mlp_shrink(alora_ctx *, const void *, const void *, int, int, int, void *, float *, size_t, int32_t *, int,
+                      cudaStream_t);
 bool build_layer_maps(alora_ctx *ctx, int layer);
 bool project_is_few_row(const alora_ctx *ctx, int layer, int T);   // gemm_tcgen05.cu
 int launch_attend_tc(alora_ctx *, const void *, const BatchArgs &, const void *, void *, cudaStream_t);
@@ -296,6 +298,8 @@ alora_status alora_destroy(alora_ctx *ctx) {
         for (void *p : *v) if (p) cudaFree(p);
     if (ctx->d_mlp_adapters) cudaFree(ctx->d_mlp_adapters);
     if (ctx->d_mlp_t) cudaFree(ctx->d_mlp_t);
+    if (ctx->d_mlp_part) cudaFree(ctx->d_mlp_part);
+    if (ctx->d_mlp_done) cudaFree(ctx->d_mlp_done);
     void *ptrs[] = {ctx->d_adapters, ctx->d_token_req, ctx->d_row_adapter, ctx->d_slot, ctx->d_tiles, ctx->d_counts,
                     ctx->d_seg_scratch, ctx->d_shrink_tiles, ctx->d_t_ready, ctx->d_t, ctx->d_qkv, ctx->d_status, ctx->d_act[0], ctx->d_act[1],
                     ctx->d_act[2], ctx->d_act[3], ctx->d_iota, ctx->d_attn_items, ctx->d_attn_off, ctx->d_split_items,
@@ -394,7 +398,15 @@ alora_status alora_register_mlp_adapter(alora_ctx *ctx, int adapter_id, int laye
     }
     if (!ctx->d_mlp_t) {
         const size_t rows = (size_t)std::min(std::max(ctx->cfg.max_tokens, 1), kMlpChunk);
+        const size_t rows_pad = (rows + 63) / 64 * 64;
         ALORA_CUDA(ctx, cudaMalloc(&ctx->d_mlp_t, rows * na * 2 * d.RP * es));
+        // K-slice partials of the shrink kernel: room for four slices of the widest result, at most 64 MB (the
+        // kernel takes fewer slices when a batch's partials would not fit)
+        ctx->mlp_part_floats = std::min<size_t>(4 * rows_pad * na * 2 * d.RP, (size_t)16 << 20);
+        ALORA_CUDA(ctx, cudaMalloc((void **)&ctx->d_mlp_part, ctx->mlp_part_floats * 4));
+        ctx->mlp_done_ints = (int)((rows_pad / 64) * ((na * 2 * d.RP + 63) / 64));
+        ALORA_CUDA(ctx, cudaMalloc((void **)&ctx->d_mlp_done, (size_t)ctx->mlp_done_ints * 4));
+        ALORA_CUDA(ctx, cudaMemsetAsync(ctx->d_mlp_done, 0, (size_t)ctx->mlp_done_ints * 4, s));
     }
     if (!ctx->mlp_a_gu[layer]) {
         struct { void **p; size_t bytes; } slabs[] = {{&ctx->mlp_a_gu[layer], na * a_gu}, {&ctx->mlp_b_gu[layer], na * b_gu},
@@ -663,7 +675,7 @@ alora_status alora_forward_stack(alora_ctx *ctx, int mode, const void *d_hidden_
             const int tc = std::min(kMlpChunk, T - t0);
             const char *xm = (const char *)ctx->d_act[0] + (size_t)t0 * d.H * ctx->esize;
             char *hc = h + (size_t)t0 * d.H * ctx->esize;
-            // adapters on the MLP block: shrink against all of the layer's A rows (one more GEMM), then the expand
+            // adapters on the MLP block: shrink against all of the layer's A rows (one launch), then the expand
             // step adds each open-gate row's delta in place (the row's applied adapter comes from this layer's
             // batch metadata; base-model batches and closed gates have none)
             const int n_mlp = (mode != ALORA_MODE_BASE && !ctx->mlp_n_adapters.empty()) ? ctx->mlp_n_adapters[l] : 0;
@@ -671,15 +683,17 @@ alora_status alora_forward_stack(alora_ctx *ctx, int mode, const void *d_hidden_
             ALORA_STEP(launch_linear(ctx, xm, lw.wgate_up, tc, d.H, 2 * d.I, ctx->d_act[2], nullptr, s));
             if (n_mlp) {
                 const int tw = n_mlp * 2 * d.RP;
-                ALORA_STEP(launch_linear(ctx, xm, ctx->mlp_a_gu[l], tc, d.H, tw, ctx->d_mlp_t, nullptr, s));
+                ALORA_STEP(launch_mlp_shrink(ctx, xm, ctx->mlp_a_gu[l], tc, d.H, tw, ctx->d_mlp_t, ctx->d_mlp_part,
+                                             ctx->mlp_part_floats, ctx->d_mlp_done, ctx->mlp_done_ints, s));
                 ALORA_STEP(launch_mlp_expand(ctx, ctx->d_act[2], 2 * d.I, tc, ctx->d_mlp_t, tw, ctx->mlp_b_gu[l], 2 * d.I,
                                              d.I, 2, ctx->d_row_adapter + t0, mlp_tab, n_mlp, s));
             }
             ALORA_STEP(launch_swiglu(ctx, ctx->d_act[2], tc, ctx->d_act[3], s));
             ALORA_STEP(launch_linear(ctx, ctx->d_act[3], lw.wdown, tc, d.I, d.H, hc, hc, s));  // h += down(...)
             if (n_mlp) {
-                const int tw = (n_mlp * d.RP + 127) / 128 * 128;
-                ALORA_STEP(launch_linear(ctx, ctx->d_act[3], ctx->mlp_a_dn[l], tc, d.I, tw, ctx->d_mlp_t, nullptr, s));
+                const int tw = n_mlp * d.RP;
+                ALORA_STEP(launch_mlp_shrink(ctx, ctx->d_act[3], ctx->mlp_a_dn[l], tc, d.I, tw, ctx->d_mlp_t, ctx->d_mlp_part,
+                                             ctx->mlp_part_floats, ctx->d_mlp_done, ctx->mlp_done_ints, s));
                 ALORA_STEP(launch_mlp_expand(ctx, hc, d.H, tc, ctx->d_mlp_t, tw, ctx->mlp_b_dn[l], d.H, d.H, 1,
                                              ctx->d_row_adapter + t0, mlp_tab, n_mlp, s));
             }

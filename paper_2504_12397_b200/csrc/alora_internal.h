@@ -151,6 +151,10 @@ struct alora_ctx {
     std::vector<alora::MlpAdapterDev> h_mlp_adapters;   // [layer * max_adapters + id], mirrors d_mlp_adapters
     alora::MlpAdapterDev *d_mlp_adapters = nullptr;
     void *d_mlp_t = nullptr;                         // [min(max_tokens, kMlpChunk)][max_adapters * 2 * RP] shrink results
+    float *d_mlp_part = nullptr;                     // K-slice partials of the shrink kernel
+    size_t mlp_part_floats = 0;
+    int32_t *d_mlp_done = nullptr;                   // per 64 x 64 tile of the shrink result: slices stored (zero between launches)
+    int mlp_done_ints = 0;
 
     // per-call workspaces
     int32_t *d_token_req = nullptr, *d_row_adapter = nullptr, *d_slot = nullptr;

@@ -3,11 +3,13 @@
 // W + s B A, a row before it the base weight alone (the form of Eq. 5).  The dense product y = W x is the stack's
 // ordinary GEMM; the low-rank part runs beside it in two steps:
 //   shrink   t[row][k][blk][i] = sum_h A_k,blk[i][h] x[row][h]    for ALL registered adapters k of the layer at once:
-//            one dense GEMM against the layer's slab of A rows (a few hundred output columns against the tens of
-//            thousands of the base product), rounded to bf16 like every GEMM output;
+//            one launch against the layer's slab of A rows (a few hundred output columns against the tens of
+//            thousands of the base product), rounded to bf16 like every GEMM output: mlp_shrink_kernel below;
 //   expand   y[row][c] += s_k * sum_i t[row][k][blk(c)][i] B_k[c][i]    only on rows whose gate is open, k = the
 //            row's applied adapter: mlp_expand_add_kernel below (mma.sync, fp32 accumulation, one pass over y).
 // Rows whose gate is closed are neither read nor written by the expand step, so they keep the bits of the base MLP.
+#include <algorithm>
+
 #include "alora_internal.h"
 #include "tc_common.cuh"
 
@@ -70,6 +72,162 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void *smem_r
     const uint32_t addr = (uint32_t)__cvta_generic_to_shared(smem_row);
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
                  : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]) : "r"(addr));
+}
+
+// ---------------------------------------------------------------------------------------------------------------
+// Shrink: t[row][c] = sum_h x[row][h] A[c][h] for the A rows of all the layer's MLP adapters (c = (adapter, block, rank
+// row), a few hundred at most) -- a product with very many rows, a long inner dimension and very few columns, which the
+// tile kernels of the dense projections serve badly (one 128-column tile per 128 rows: 16 of 148 SMs busy on 2048
+// rows).  Here a block takes 64 rows x 64 columns x one slice of K (mma.sync, fp32 accumulation, operands staged in
+// shared memory with the next K chunk's loads in flight under the current chunk's arithmetic); K is cut into as
+// many slices (at most 8) as it takes to give every SM about two blocks.  With more than one slice the blocks store fp32 partial tiles
+// and count themselves per (row tile, column tile); the block that stores a tile's last slice adds the partials in
+// slice order (fixed order: run-to-run identical) and writes bf16.
+// ---------------------------------------------------------------------------------------------------------------
+constexpr int kShRows = 64, kShCols = 64, kShChunk = 64, kShThreads = 128, kShLd = 72, kShMaxSplit = 8;
+
+struct MlpShrinkArgs {
+    const __nv_bfloat16 *x;     // [rows][K]
+    const __nv_bfloat16 *a;     // [n_cols][K]: the layer's slab of A rows
+    __nv_bfloat16 *t;           // [rows][n_cols]
+    float *part;                // [ksplit][row tiles * 64][n_cols] fp32 (ksplit > 1)
+    int32_t *done;              // [row tiles * column tiles] slices stored so far; the finishing block puts 0 back
+    int rows, K, n_cols, ksplit;
+};
+
+__global__ void __launch_bounds__(kShThreads) mlp_shrink_kernel(const MlpShrinkArgs a) {
+    tc::grid_dep_launch();
+    tc::grid_dep_wait();
+    __shared__ __align__(16) __nv_bfloat16 xs[2][kShRows * kShLd];
+    __shared__ __align__(16) __nv_bfloat16 as[2][kShCols * kShLd];
+    __shared__ int last_s;
+    const int warp = (int)threadIdx.x >> 5, lane = (int)threadIdx.x & 31, g = lane >> 2, q = lane & 3;
+    const int col0 = (int)blockIdx.x * kShCols, row0 = (int)blockIdx.y * kShRows, ks = (int)blockIdx.z;
+    const int n_chunks = (a.K + kShChunk - 1) / kShChunk;
+    const int c_base = n_chunks / a.ksplit, c_rem = n_chunks % a.ksplit;
+    const int c0 = ks * c_base + min(ks, c_rem), nc = c_base + (ks < c_rem ? 1 : 0);
+    // a thread's four 16-byte pieces of each operand tile: piece p = threadIdx.x + 128 i -> row p / 8, vector p % 8
+    uint4 xr[4], ar[4];
+    auto fetch = [&](int chunk) {
+        const int k0 = chunk * kShChunk;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int p = (int)threadIdx.x + kShThreads * i, r = p >> 3, v = p & 7;
+            const int k = k0 + v * 8;
+            const bool kin = k < a.K;   // K is a multiple of 8: a vector is inside or outside as a whole
+            const int xrow = min(row0 + r, a.rows - 1);   // rows past the end repeat the last row; their results are dropped
+            xr[i] = kin ? *reinterpret_cast<const uint4 *>(a.x + (size_t)xrow * a.K + k) : make_uint4(0u, 0u, 0u, 0u);
+            const int acol = col0 + r;
+            ar[i] = (kin && acol < a.n_cols) ? *reinterpret_cast<const uint4 *>(a.a + (size_t)acol * a.K + k) : make_uint4(0u, 0u, 0u, 0u);
+        }
+    };
+    auto stash = [&](int buf) {
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int p = (int)threadIdx.x + kShThreads * i, r = p >> 3, v = p & 7;
+            *reinterpret_cast<uint4 *>(&xs[buf][r * kShLd + v * 8]) = xr[i];
+            *reinterpret_cast<uint4 *>(&as[buf][r * kShLd + v * 8]) = ar[i];
+        }
+    };
+    float acc[8][4];
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt)
+#pragma unroll
+        for (int e = 0; e < 4; ++e) acc[nt][e] = 0.f;
+    if (nc > 0) fetch(c0);
+    for (int c = 0; c < nc; ++c) {
+        const int buf = c & 1;
+        stash(buf);
+        __syncthreads();                       // the chunk is in shared memory; the other buffer's readers are done
+        if (c + 1 < nc) fetch(c0 + c + 1);     // the next chunk's loads fly under this chunk's arithmetic
+#pragma unroll
+        for (int kk = 0; kk < kShChunk; kk += 16) {
+            uint32_t af[4];
+            ldmatrix_x4(af, &xs[buf][(warp * 16 + (lane & 7) + ((lane >> 3) & 1) * 8) * kShLd + kk + (lane >> 4) * 8]);
+#pragma unroll
+            for (int np = 0; np < 4; ++np) {
+                uint32_t bf[4];
+                ldmatrix_x4(bf, &as[buf][(np * 16 + (lane & 7) + ((lane >> 4) & 1) * 8) * kShLd + kk + ((lane >> 3) & 1) * 8]);
+                mma_bf16_16816(acc[2 * np], af, bf[0], bf[1]);
+                mma_bf16_16816(acc[2 * np + 1], af, bf[2], bf[3]);
+            }
+        }
+    }
+    // this thread's accumulator elements: rows row0 + warp * 16 + g (+ 8), columns col0 + nt * 8 + 2 q (+ 1)
+    const int r_lo = row0 + warp * 16 + g, r_hi = r_lo + 8;
+    if (a.ksplit == 1) {
+#pragma unroll
+        for (int nt = 0; nt < 8; ++nt) {
+            const int col = col0 + nt * 8 + 2 * q;
+            if (col >= a.n_cols) continue;
+            if (r_lo < a.rows) *reinterpret_cast<__nv_bfloat162 *>(a.t + (size_t)r_lo * a.n_cols + col) = __floats2bfloat162_rn(acc[nt][0], acc[nt][1]);
+            if (r_hi < a.rows) *reinterpret_cast<__nv_bfloat162 *>(a.t + (size_t)r_hi * a.n_cols + col) = __floats2bfloat162_rn(acc[nt][2], acc[nt][3]);
+        }
+        return;
+    }
+    const size_t rows_pad = (size_t)gridDim.y * kShRows;
+    float *mine = a.part + (size_t)ks * rows_pad * a.n_cols;
+#pragma unroll
+    for (int nt = 0; nt < 8; ++nt) {
+        const int col = col0 + nt * 8 + 2 * q;
+        if (col >= a.n_cols) continue;
+        *reinterpret_cast<float2 *>(mine + (size_t)r_lo * a.n_cols + col) = make_float2(acc[nt][0], acc[nt][1]);
+        *reinterpret_cast<float2 *>(mine + (size_t)r_hi * a.n_cols + col) = make_float2(acc[nt][2], acc[nt][3]);
+    }
+    __threadfence();
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        int32_t *cnt = a.done + (size_t)blockIdx.y * gridDim.x + blockIdx.x;
+        const int last = atomicAdd(cnt, 1) == a.ksplit - 1 ? 1 : 0;
+        if (last) *cnt = 0;      // (nobody else counts on this tile any more in this launch)
+        last_s = last;
+    }
+    __syncthreads();
+    if (!last_s) return;
+    __threadfence();
+    // 64 rows x 64 columns = 1024 float4; thread i takes float4 i, i + 128, ...: row = idx / 16, columns 4 (idx % 16) ..
+    for (int idx = (int)threadIdx.x; idx < kShRows * (kShCols / 4); idx += kShThreads) {
+        const int r = row0 + idx / (kShCols / 4), col = col0 + (idx % (kShCols / 4)) * 4;
+        if (r >= a.rows || col >= a.n_cols) continue;     // n_cols is a multiple of 8
+        // all slices' loads in flight together (one round trip to L2 per output vector, not one per slice), then
+        // added in slice order
+        float4 v[kShMaxSplit];
+#pragma unroll
+        for (int s2 = 0; s2 < kShMaxSplit; ++s2)
+            if (s2 < a.ksplit)
+                v[s2] = __ldcg(reinterpret_cast<const float4 *>(a.part + ((size_t)s2 * rows_pad + r) * a.n_cols + col));
+        float4 sum = make_float4(0.f, 0.f, 0.f, 0.f);
+#pragma unroll
+        for (int s2 = 0; s2 < kShMaxSplit; ++s2)
+            if (s2 < a.ksplit) { sum.x += v[s2].x; sum.y += v[s2].y; sum.z += v[s2].z; sum.w += v[s2].w; }
+        uint2 o;
+        *reinterpret_cast<__nv_bfloat162 *>(&o.x) = __floats2bfloat162_rn(sum.x, sum.y);
+        *reinterpret_cast<__nv_bfloat162 *>(&o.y) = __floats2bfloat162_rn(sum.z, sum.w);
+        *reinterpret_cast<uint2 *>(a.t + (size_t)r * a.n_cols + col) = o;
+    }
+}
+
+// t[rows][n_cols] = x[rows][K] A[n_cols][K]^T, bf16.  `part` holds part_floats floats, `done` one counter per 64 x 64
+// tile (zero between launches).  Returns kernels launched, or -1.
+int launch_mlp_shrink(alora_ctx *ctx, const void *x, const void *A, int rows, int K, int n_cols, void *t, float *part,
+                      size_t part_floats, int32_t *done, int done_ints, cudaStream_t s) {
+    if (rows <= 0) return 0;
+    if (K % 8 != 0 || n_cols % 8 != 0 || n_cols <= 0) return -1;
+    const int col_tiles = (n_cols + kShCols - 1) / kShCols, row_tiles = (rows + kShRows - 1) / kShRows;
+    const int n_chunks = (K + kShChunk - 1) / kShChunk;
+    // about two blocks per SM, at least two K chunks per block (more slices were slower: the kernel is bound by its
+    // shared-memory traffic, and every slice adds a partial tile to store and to add up)
+    int ksplit = (2 * ctx->sm_count + col_tiles * row_tiles - 1) / (col_tiles * row_tiles);
+    ksplit = std::max(1, std::min(std::min(ksplit, kShMaxSplit), n_chunks / 2));
+    while (ksplit > 1 && (size_t)ksplit * row_tiles * kShRows * n_cols > part_floats) --ksplit;
+    if (col_tiles * row_tiles > done_ints) ksplit = 1;
+    MlpShrinkArgs a{};
+    a.x = (const __nv_bfloat16 *)x; a.a = (const __nv_bfloat16 *)A; a.t = (__nv_bfloat16 *)t; a.part = part; a.done = done;
+    a.rows = rows; a.K = K; a.n_cols = n_cols; a.ksplit = ksplit;
+    ProfScope prof(ctx, KK_LINEAR, s);
+    if (launch_kernel(mlp_shrink_kernel, dim3(col_tiles, row_tiles, ksplit), dim3(kShThreads), 0, s, true, a) != cudaSuccess)
+        return -1;
+    return 1;
 }
 
 constexpr int kMxLd = 72;   // shared-memory row length of the t and B tiles in bf16: 64 + 8 (144 bytes: rows stay
