@@ -145,7 +145,8 @@ alora_status alora_register_adapter(alora_ctx *ctx, int adapter_id, int layer, i
  * the MLP block, so only they use these matrices: rows whose gate is open get the deltas, rows whose
  * gate is closed (and every row in ALORA_MODE_BASE) keep the bits of the base MLP.  The matrices are
  * COPIED on the given stream.  The first registration on a layer allocates that layer's slabs
- * (cudaMalloc; about 2 * max_adapters * 64 * (H + 3 I) bytes), so register before timing anything.
+ * (cudaMalloc; about 384 * max_adapters * (H + I) bytes per layer, plus once per context the shrink results
+ * and their partial sums), so register before timing anything.
  * Errors: ALORA_ERR_NO_WEIGHTS when the adapter has no q/k/v part on this layer yet (its gate is the
  * q/k/v adapter's); ALORA_ERR_UNSUPPORTED for fp32 contexts, contexts without an MLP (intermediate = 0)
  * and sizes where H or I is not a multiple of 256; ALORA_ERR_CAPACITY for the id or rank.
