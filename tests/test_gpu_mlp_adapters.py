@@ -180,6 +180,50 @@ def test_mlp_adapters_across_token_chunks_of_the_mlp(oracle64):
         g.close()
 
 
+def test_one_layer_at_the_8b_shape(oracle64):
+    """One decoder layer at the 8B layer shape (hidden 4096, intermediate 14336: gate / up rows of 57 KB, a down
+    projection with K = 14336) with adapters on q/k/v and on the MLP: three requests (rank 32 and rank 8 adapters and
+    the base model), 160 new tokens, one gate opening inside its chunk; every row against the oracle, closed rows
+    bit-equal to the base-mode call."""
+    shape = wl.SHAPE_8B
+    rng = np.random.default_rng(47)
+    layers = [wl.make_stack_weights(shape, rng)]
+    ads = [[wl.make_adapter(shape, r, rng) for r in (32, 8)]]
+    mlps = [[wl.make_mlp_adapter(shape, r, rng, scale=s) for r, s in ((32, 1.0), (8, 2.0))]]
+    for a in ads[0]:
+        for n in ("Bq", "Bk", "Bv"):
+            setattr(a, n, wl.bf16_round(getattr(a, n) * 8))
+    for a in mlps[0]:
+        for n in ("Bg", "Bu", "Bd"):
+            setattr(a, n, wl.bf16_round(getattr(a, n) * 8))
+    S, ids, a_req = [70, 50, 40], [0, -1, 1], [33, 0, 0]
+    b = wl.make_batch(shape, [0] * 3, S, ids, rng, activation_offsets=a_req, shuffle_pages=True)
+    g = hp.GpuLayers(shape, layers, ads, 256, 4, mlp_adapters_per_layer=mlps)
+    try:
+        d = hp.DevBatch(b, shape.dtype)
+
+        def run(mode):
+            pools = [g.new_pool(b.num_pages)]
+            hout = g.empty(b.T, shape.hidden)
+            ab.alora_forward_stack(g.ctx, mode, d.hidden, d.positions, d.a_req, d.ids, d.qsl, d.seq_lens, pools, d.bt,
+                                   d.max_blocks, b.num_pages, d.T, d.R, hout)
+            assert g.status() == 0
+            return hp.to_host(hout)
+
+        got, base = run(ab.MODE_ALORA), run(ab.MODE_BASE)
+        x, _ = oracle64.decoder_layer(b.hidden.astype(np.float64), layers[0], shape.Nq, shape.Nkv, shape.n_q_heads,
+                                      shape.n_kv_heads, shape.head_dim, 1e-5, b.positions, b.query_start_loc,
+                                      b.activation_offsets, b.adapter_ids, hp.oracle_adapters(ads[0]), [None] * 3,
+                                      [None] * 3, mlp_adapters=hp.oracle_mlp_adapters(mlps[0]))
+        hp.assert_close(got, x, 2e-2, "8B-shape layer with MLP adapters", block=shape.head_dim)
+        closed = np.concatenate([np.arange(0, 33), np.arange(70, 120)])
+        assert np.array_equal(got[closed].view(np.uint32), base[closed].view(np.uint32))
+        opened = np.concatenate([np.arange(33, 70), np.arange(120, 160)])
+        assert hp.rel_err(got[opened], base[opened]) > 0.02
+    finally:
+        g.close()
+
+
 def test_mlp_adapter_registration_errors():
     rng = np.random.default_rng(46)
     layers, ads, mlps = _weights(rng, 1)
