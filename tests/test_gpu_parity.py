@@ -543,6 +543,35 @@ def test_stack_layer_with_many_rows_takes_the_256_row_gemm(oracle64):
         g.close()
 
 
+def test_stack_layer_at_the_8b_shape_with_1024_rows(oracle64):
+    """One decoder layer at the 8B layer shape on 4 x 256 new tokens: q/k/v on the 128-row tile route with the fused
+    shrink, o_proj, gate / up (28672 columns) and down (K = 14336) on the 256 x 256 dense kernel, the 16-byte norm and
+    SwiGLU kernels at their real row lengths.  Every row against the oracle (about 0.23 TFLOP of oracle work)."""
+    shape = wl.SHAPE_8B
+    rng = np.random.default_rng(48)
+    layers = [wl.make_stack_weights(shape, rng)]
+    ads = [[wl.make_adapter(shape, 32, rng)]]
+    for n in ("Bq", "Bk", "Bv"):
+        setattr(ads[0][0], n, wl.bf16_round(getattr(ads[0][0], n) * 8))
+    b = wl.make_batch(shape, [0] * 4, [256] * 4, [0, -1, 0, 0], rng, activation_offsets=[100, 0, 0, 255],
+                      shuffle_pages=True)
+    g = hp.GpuLayers(shape, layers, ads, 1024, 4)
+    try:
+        d = hp.DevBatch(b, shape.dtype)
+        pools = [g.new_pool(b.num_pages)]
+        hout = g.empty(b.T, shape.hidden)
+        ab.alora_forward_stack(g.ctx, ab.MODE_ALORA, d.hidden, d.positions, d.a_req, d.ids, d.qsl, d.seq_lens, pools,
+                               d.bt, d.max_blocks, b.num_pages, d.T, d.R, hout)
+        assert g.status() == 0
+        x, _ = oracle64.decoder_layer(b.hidden.astype(np.float64), layers[0], shape.Nq, shape.Nkv, shape.n_q_heads,
+                                      shape.n_kv_heads, shape.head_dim, 1e-5, b.positions, b.query_start_loc,
+                                      b.activation_offsets, b.adapter_ids, hp.oracle_adapters(ads[0]),
+                                      [None] * b.R, [None] * b.R)
+        hp.assert_close(hp.to_host(hout), x, 2e-2, "8B-shape layer, 1024 rows", block=shape.head_dim)
+    finally:
+        g.close()
+
+
 def test_empty_and_degenerate_batches():
     w, ads, b = _mid_workload()
     g = hp.GpuLayers(MID, [dict(wqkv=w)], [ads], 256, 8)
