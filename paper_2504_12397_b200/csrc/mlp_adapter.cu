@@ -50,8 +50,10 @@ int launch_repack_mlp(const void *a0, const void *a1, const void *b0, const void
 
 constexpr int kMxRows = 64, kMxCols = 128, kMxThreads = 128;   // block tile of the expand step; one warp per 32 columns
 constexpr int kMxRowsPerWarp = 32 / (kMxThreads / 32);            // rows of a 32-row pass that one warp updates
-constexpr int kMxPieces = kMxCols / 128;                          // 8-byte pieces of a row per lane (32 lanes x 4 columns)
-static_assert(kMxCols == 32 * (kMxThreads / 32) && kMxCols % 128 == 0 && 32 % (kMxThreads / 32) == 0, "tile shape");
+constexpr int kMxLanesPerRow = kMxCols / 8;                       // a lane updates a 16-byte piece (8 columns) of a row
+constexpr int kMxRowsPerInst = 32 / kMxLanesPerRow;               // rows one warp instruction covers
+constexpr int kMxUpdates = kMxRowsPerWarp / kMxRowsPerInst;       // update instructions per warp and pass
+static_assert(kMxCols == 32 * (kMxThreads / 32) && 32 % kMxLanesPerRow == 0 && kMxRowsPerWarp % kMxRowsPerInst == 0, "tile shape");
 
 struct MlpExpandArgs {
     __nv_bfloat16 *y;                  // [rows][ldy], updated in place on open-gate rows
@@ -271,19 +273,18 @@ __global__ void __launch_bounds__(kMxThreads, 4) mlp_expand_add_kernel(const Mlp
     const int blk = cbase / a.width;                   // the width is a multiple of the block's columns
     // The y values this thread will update are requested now: their trip to DRAM overlaps the tile fills and the
     // MMAs, and a block keeps its whole tile of reads in flight from its first microsecond on.
-    uint2 yv[2][kMxRowsPerWarp][kMxPieces];
+    // (a lane owns the 16-byte piece uc of row pass * 32 + warp * kMxRowsPerWarp + i * kMxRowsPerInst + ur)
+    const int ur = lane / kMxLanesPerRow, uc = (lane % kMxLanesPerRow) * 8;
+    const bool col_in = cbase + uc < a.ncols;          // ncols is a multiple of 8: a piece is inside or outside as a whole
+    uint4 yv[2][kMxUpdates];
 #pragma unroll
     for (int pass = 0; pass < 2; ++pass)
 #pragma unroll
-        for (int i = 0; i < kMxRowsPerWarp; ++i) {
-            const int lr = pass * 32 + warp * kMxRowsPerWarp + i;
-            const bool open = s_ad[lr] >= 0;
-            const __nv_bfloat16 *yr = a.y + (size_t)(row0 + lr) * a.ldy + cbase;
-#pragma unroll
-            for (int h = 0; h < kMxPieces; ++h) {
-                const int c = h * 128 + lane * 4;
-                yv[pass][i][h] = (open && cbase + c < a.ncols) ? *reinterpret_cast<const uint2 *>(yr + c) : make_uint2(0u, 0u);
-            }
+        for (int i = 0; i < kMxUpdates; ++i) {
+            const int lr = pass * 32 + warp * kMxRowsPerWarp + i * kMxRowsPerInst + ur;
+            yv[pass][i] = (s_ad[lr] >= 0 && col_in)
+                              ? *reinterpret_cast<const uint4 *>(a.y + (size_t)(row0 + lr) * a.ldy + cbase + uc)
+                              : make_uint4(0u, 0u, 0u, 0u);
         }
     float acc[4][4][4];
 #pragma unroll
@@ -366,24 +367,22 @@ __global__ void __launch_bounds__(kMxThreads, 4) mlp_expand_add_kernel(const Mlp
         }
         __syncthreads();
 #pragma unroll
-        for (int i = 0; i < kMxRowsPerWarp; ++i) {
-            const int lr = pass * 32 + warp * kMxRowsPerWarp + i;
-            if (s_ad[lr] < 0) continue;                        // closed gate: the row is neither read nor written
-            __nv_bfloat16 *yr = a.y + (size_t)(row0 + lr) * a.ldy + cbase;
-#pragma unroll
-            for (int h = 0; h < kMxPieces; ++h) {
-                const int c = h * 128 + lane * 4;
-                if (cbase + c >= a.ncols) continue;
-                const float4 dl = *reinterpret_cast<const float4 *>(&s_delta[lr - pass * 32][c]);
-                uint2 *p = reinterpret_cast<uint2 *>(yr + c);
-                const uint2 raw = yv[pass][i][h];
-                const float2 v0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&raw.x));
-                const float2 v1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&raw.y));
-                uint2 out;
-                *reinterpret_cast<__nv_bfloat162 *>(&out.x) = __floats2bfloat162_rn(v0.x + dl.x, v0.y + dl.y);
-                *reinterpret_cast<__nv_bfloat162 *>(&out.y) = __floats2bfloat162_rn(v1.x + dl.z, v1.y + dl.w);
-                *p = out;
-            }
+        for (int i = 0; i < kMxUpdates; ++i) {
+            const int lr = pass * 32 + warp * kMxRowsPerWarp + i * kMxRowsPerInst + ur;
+            if (s_ad[lr] < 0 || !col_in) continue;             // closed gate: the row is neither read nor written
+            const float4 d0 = *reinterpret_cast<const float4 *>(&s_delta[lr - pass * 32][uc]);
+            const float4 d1 = *reinterpret_cast<const float4 *>(&s_delta[lr - pass * 32][uc + 4]);
+            const uint4 raw = yv[pass][i];
+            const float2 v0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&raw.x));
+            const float2 v1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&raw.y));
+            const float2 v2 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&raw.z));
+            const float2 v3 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&raw.w));
+            uint4 out;
+            *reinterpret_cast<__nv_bfloat162 *>(&out.x) = __floats2bfloat162_rn(v0.x + d0.x, v0.y + d0.y);
+            *reinterpret_cast<__nv_bfloat162 *>(&out.y) = __floats2bfloat162_rn(v1.x + d0.z, v1.y + d0.w);
+            *reinterpret_cast<__nv_bfloat162 *>(&out.z) = __floats2bfloat162_rn(v2.x + d1.x, v2.y + d1.y);
+            *reinterpret_cast<__nv_bfloat162 *>(&out.w) = __floats2bfloat162_rn(v3.x + d1.z, v3.y + d1.w);
+            *reinterpret_cast<uint4 *>(a.y + (size_t)(row0 + lr) * a.ldy + cbase + uc) = out;
         }
     }
 }
@@ -394,7 +393,7 @@ int launch_mlp_expand(alora_ctx *ctx, void *y, int ldy, int rows, const void *t,
                       int width, int nblk, const int32_t *row_adapter, const MlpAdapterDev *table, int n_adapters,
                       cudaStream_t s) {
     if (rows <= 0) return 0;
-    if (ncols % 8 != 0 || width % kMxCols != 0 || ldy % 4 != 0 || t_ld % 8 != 0 || ((uintptr_t)y & 7) != 0) return -1;
+    if (ncols % 8 != 0 || width % kMxCols != 0 || ldy % 8 != 0 || t_ld % 8 != 0 || ((uintptr_t)y & 15) != 0) return -1;
     MlpExpandArgs a{};
     a.y = (__nv_bfloat16 *)y; a.t = (const __nv_bfloat16 *)t; a.b = (const __nv_bfloat16 *)b;
     a.row_adapter = row_adapter; a.table = table;
