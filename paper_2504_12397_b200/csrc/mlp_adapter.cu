@@ -370,8 +370,12 @@ __global__ void __launch_bounds__(kMxThreads, 4) mlp_expand_add_kernel(const Mlp
         for (int i = 0; i < kMxUpdates; ++i) {
             const int lr = pass * 32 + warp * kMxRowsPerWarp + i * kMxRowsPerInst + ur;
             if (s_ad[lr] < 0 || !col_in) continue;             // closed gate: the row is neither read nor written
-            const float4 d0 = *reinterpret_cast<const float4 *>(&s_delta[lr - pass * 32][uc]);
-            const float4 d1 = *reinterpret_cast<const float4 *>(&s_delta[lr - pass * 32][uc + 4]);
+            // (lanes 4 .. 7 of every eight read their second half first: the eight 16-byte reads of a quarter warp then
+            // fall into different banks)
+            const int sw = (lane >> 2) & 1;
+            const float4 da = *reinterpret_cast<const float4 *>(&s_delta[lr - pass * 32][uc + 4 * sw]);
+            const float4 db = *reinterpret_cast<const float4 *>(&s_delta[lr - pass * 32][uc + 4 * (sw ^ 1)]);
+            const float4 d0 = sw ? db : da, d1 = sw ? da : db;
             const uint4 raw = yv[pass][i];
             const float2 v0 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&raw.x));
             const float2 v1 = __bfloat1622float2(*reinterpret_cast<const __nv_bfloat162 *>(&raw.y));
