@@ -70,6 +70,12 @@ __device__ __forceinline__ void mma_bf16_16816(float (&c)[4], const uint32_t (&a
                  : "r"(a[0]), "r"(a[1]), "r"(a[2]), "r"(a[3]), "r"(b0), "r"(b1));
 }
 
+// 16-byte asynchronous copy global -> shared; src_bytes (0 or 16) of the source are read, the rest is zero-filled
+__device__ __forceinline__ void cp_async_16(void *smem_dst, const void *gmem_src, int src_bytes) {
+    const uint32_t dst = (uint32_t)__cvta_generic_to_shared(smem_dst);
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16, %2;" ::"r"(dst), "l"(gmem_src), "r"(src_bytes) : "memory");
+}
+
 __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void *smem_row) {
     const uint32_t addr = (uint32_t)__cvta_generic_to_shared(smem_row);
     asm volatile("ldmatrix.sync.aligned.m8n8.x4.shared.b16 {%0, %1, %2, %3}, [%4];"
@@ -80,8 +86,8 @@ __device__ __forceinline__ void ldmatrix_x4(uint32_t (&r)[4], const void *smem_r
 // Shrink: t[row][c] = sum_h x[row][h] A[c][h] for the A rows of all the layer's MLP adapters (c = (adapter, block, rank
 // row), a few hundred at most) -- a product with very many rows, a long inner dimension and very few columns, which the
 // tile kernels of the dense projections serve badly (one 128-column tile per 128 rows: 16 of 148 SMs busy on 2048
-// rows).  Here a block takes 64 rows x 64 columns x one slice of K (mma.sync, fp32 accumulation, operands staged in
-// shared memory with the next K chunk's loads in flight under the current chunk's arithmetic); K is cut into as
+// rows).  Here a block takes 64 rows x 64 columns x one slice of K (mma.sync, fp32 accumulation, operands brought to
+// shared memory by asynchronous copies, the next K chunk's in flight under the current chunk's arithmetic); K is cut into as
 // many slices (at most 8) as it takes to give every SM about two blocks.  With more than one slice the blocks store fp32 partial tiles
 // and count themselves per (row tile, column tile); the block that stores a tile's last slice adds the partials in
 // slice order (fixed order: run-to-run identical) and writes bf16.
@@ -108,40 +114,42 @@ __global__ void __launch_bounds__(kShThreads) mlp_shrink_kernel(const MlpShrinkA
     const int n_chunks = (a.K + kShChunk - 1) / kShChunk;
     const int c_base = n_chunks / a.ksplit, c_rem = n_chunks % a.ksplit;
     const int c0 = ks * c_base + min(ks, c_rem), nc = c_base + (ks < c_rem ? 1 : 0);
-    // a thread's four 16-byte pieces of each operand tile: piece p = threadIdx.x + 128 i -> row p / 8, vector p % 8
-    uint4 xr[4], ar[4];
-    auto fetch = [&](int chunk) {
+    // a thread's four 16-byte pieces of each operand tile: piece p = threadIdx.x + 128 i -> row p / 8, vector p % 8.
+    // The pieces go from global to shared memory by asynchronous copies (no trip through registers and no store
+    // instruction: the kernel is bound by its shared-memory traffic); a piece outside K or past the last A row is
+    // filled with zeros (zero source bytes), rows past the end repeat the last row and their results are dropped.
+    auto issue = [&](int chunk, int buf) {
         const int k0 = chunk * kShChunk;
 #pragma unroll
         for (int i = 0; i < 4; ++i) {
             const int p = (int)threadIdx.x + kShThreads * i, r = p >> 3, v = p & 7;
             const int k = k0 + v * 8;
             const bool kin = k < a.K;   // K is a multiple of 8: a vector is inside or outside as a whole
-            const int xrow = min(row0 + r, a.rows - 1);   // rows past the end repeat the last row; their results are dropped
-            xr[i] = kin ? *reinterpret_cast<const uint4 *>(a.x + (size_t)xrow * a.K + k) : make_uint4(0u, 0u, 0u, 0u);
+            const int xrow = min(row0 + r, a.rows - 1);
             const int acol = col0 + r;
-            ar[i] = (kin && acol < a.n_cols) ? *reinterpret_cast<const uint4 *>(a.a + (size_t)acol * a.K + k) : make_uint4(0u, 0u, 0u, 0u);
+            const bool ain = kin && acol < a.n_cols;
+            const __nv_bfloat16 *sx = a.x + (size_t)xrow * a.K + (kin ? k : 0);
+            const __nv_bfloat16 *sa = a.a + (ain ? (size_t)acol * a.K + k : 0);
+            cp_async_16(&xs[buf][r * kShLd + v * 8], sx, kin ? 16 : 0);
+            cp_async_16(&as[buf][r * kShLd + v * 8], sa, ain ? 16 : 0);
         }
-    };
-    auto stash = [&](int buf) {
-#pragma unroll
-        for (int i = 0; i < 4; ++i) {
-            const int p = (int)threadIdx.x + kShThreads * i, r = p >> 3, v = p & 7;
-            *reinterpret_cast<uint4 *>(&xs[buf][r * kShLd + v * 8]) = xr[i];
-            *reinterpret_cast<uint4 *>(&as[buf][r * kShLd + v * 8]) = ar[i];
-        }
+        asm volatile("cp.async.commit_group;" ::: "memory");
     };
     float acc[8][4];
 #pragma unroll
     for (int nt = 0; nt < 8; ++nt)
 #pragma unroll
         for (int e = 0; e < 4; ++e) acc[nt][e] = 0.f;
-    if (nc > 0) fetch(c0);
+    if (nc > 0) issue(c0, 0);
     for (int c = 0; c < nc; ++c) {
         const int buf = c & 1;
-        stash(buf);
-        __syncthreads();                       // the chunk is in shared memory; the other buffer's readers are done
-        if (c + 1 < nc) fetch(c0 + c + 1);     // the next chunk's loads fly under this chunk's arithmetic
+        if (c + 1 < nc) {
+            issue(c0 + c + 1, buf ^ 1);        // the next chunk's copies fly under this chunk's arithmetic
+            asm volatile("cp.async.wait_group 1;" ::: "memory");   // all but the copies just issued have landed
+        } else {
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
+        }
+        __syncthreads();                       // every thread's pieces of this chunk are in shared memory
 #pragma unroll
         for (int kk = 0; kk < kShChunk; kk += 16) {
             uint32_t af[4];
@@ -154,6 +162,7 @@ __global__ void __launch_bounds__(kShThreads) mlp_shrink_kernel(const MlpShrinkA
                 mma_bf16_16816(acc[2 * np + 1], af, bf[2], bf[3]);
             }
         }
+        __syncthreads();                       // this buffer may be overwritten by the copies of chunk c + 2
     }
     // this thread's accumulator elements: rows row0 + warp * 16 + g (+ 8), columns col0 + nt * 8 + 2 q (+ 1)
     const int r_lo = row0 + warp * 16 + g, r_hi = r_lo + 8;
