@@ -314,18 +314,19 @@ __global__ void __launch_bounds__(kMxThreads, 4) mlp_expand_add_kernel(const Mlp
             any = true;
             const __nv_bfloat16 *tk = a.t + (size_t)(k * a.nblk + blk) * a.RP;
             const __nv_bfloat16 *bk = a.b + ((size_t)k * a.ncols + cbase) * a.RP;
+            // (asynchronous copies; a piece outside the run or past the last column reads nothing and is zero-filled)
             for (int i = (int)threadIdx.x; i < kMxRows * cpr; i += kMxThreads) {
                 const int r = i / cpr, c = i - r * cpr;
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (r >= ra && r < rb) v = *reinterpret_cast<const uint4 *>(tk + (size_t)(row0 + r) * a.t_ld + c * 8);
-                *reinterpret_cast<uint4 *>(sT + r * kMxLd + c * 8) = v;
+                const bool in = r >= ra && r < rb;
+                cp_async_16(sT + r * kMxLd + c * 8, in ? tk + (size_t)(row0 + r) * a.t_ld + c * 8 : a.t, in ? 16 : 0);
             }
             for (int i = (int)threadIdx.x; i < kMxCols * cpr; i += kMxThreads) {
                 const int n = i / cpr, c = i - n * cpr;
-                uint4 v = make_uint4(0u, 0u, 0u, 0u);
-                if (cbase + n < a.ncols) v = *reinterpret_cast<const uint4 *>(bk + (size_t)n * a.RP + c * 8);
-                *reinterpret_cast<uint4 *>(sB + n * kMxLd + c * 8) = v;
+                const bool in = cbase + n < a.ncols;
+                cp_async_16(sB + n * kMxLd + c * 8, in ? bk + (size_t)n * a.RP + c * 8 : a.b, in ? 16 : 0);
             }
+            asm volatile("cp.async.commit_group;" ::: "memory");
+            asm volatile("cp.async.wait_group 0;" ::: "memory");
             __syncthreads();
             if (warp_in) {
                 for (int ks = 0; ks < rpad; ks += 16) {
