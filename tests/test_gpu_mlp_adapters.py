@@ -224,6 +224,34 @@ def test_one_layer_at_the_8b_shape(oracle64):
         g.close()
 
 
+def test_registering_again_replaces_the_mlp_part(oracle64):
+    """Registering an adapter's MLP part a second time replaces it: with a smaller rank (the padding of the first
+    registration must not leak) and then with B = 0 (the stack then equals the one with q/k/v adapters only)."""
+    rng = np.random.default_rng(49)
+    layers, ads, mlps = _weights(rng, 1, mlp_ranks=(32, 16))
+    b = wl.make_batch(SHAPE, [0, 0], [75, 30], [0, 1], rng, activation_offsets=[20, 0], shuffle_pages=True)
+    g = hp.GpuLayers(SHAPE, layers, ads, 256, 4, mlp_adapters_per_layer=mlps)
+    try:
+        def register(i, m):
+            mats = [hp.to_dev(getattr(m, n), "bf16") for n in ("Ag", "Bg", "Au", "Bu", "Ad", "Bd")]
+            ab.alora_register_mlp_adapter(g.ctx, i, 0, m.rank, m.scale, *mats)
+            return mats
+        small = wl.make_mlp_adapter(SHAPE, 8, rng, scale=2.0)
+        for n in ("Bg", "Bu", "Bd"):
+            setattr(small, n, wl.bf16_round(getattr(small, n) * 8))
+        keep = register(0, small)
+        got, _ = _run_stack(g, b)
+        want, _ = _oracle_stack(oracle64, layers, ads, [[small, mlps[0][1]]], b)
+        hp.assert_close(got, want, 2e-2, "after replacing adapter 0's MLP part by a rank-8 one", block=SHAPE.head_dim)
+        zero = wl.make_mlp_adapter(SHAPE, 16, rng, zero_b=True)
+        keep += register(0, zero) + register(1, zero)
+        got, _ = _run_stack(g, b)
+        want, _ = _oracle_stack(oracle64, layers, ads, mlps, b, with_mlp=False)
+        hp.assert_close(got, want, 2e-2, "after replacing both MLP parts by B = 0", block=SHAPE.head_dim)
+    finally:
+        g.close()
+
+
 def test_mlp_adapter_registration_errors():
     rng = np.random.default_rng(46)
     layers, ads, mlps = _weights(rng, 1)
